@@ -1,0 +1,177 @@
+/* hydra.h -- C ABI of libhydra: one Hydra speculative-decode step on one sm_100a GPU.
+ *
+ * The calls follow the paper's statement of the problem (Hydra: Sequentially-Dependent Draft Heads
+ * for Medusa Decoding): a static candidate tree is populated by the draft heads (Background, "Tree
+ * decoding"; Section "Hydra Heads", second displayed equation; Section "Hydra++"), verified by one
+ * base-model forward in which a token attends only to its ancestors (Background, "Tree decoding"),
+ * a prefix is accepted by the greedy criterion (Background, verification criteria) and the rest is
+ * discarded (Background, "Speculative decoding").
+ *
+ * Conventions
+ *  - Every call returns a hydra_status; nothing throws, aborts or exits.
+ *  - "dev" pointers are device pointers, "host" pointers are host pointers.  All matrices are
+ *    row-major [out][in].  dtype 0: weights, KV cache and GEMM operands are float; dtype 1: they
+ *    are bfloat16, while accumulation, residual stream, norms and softmax stay float.
+ *  - The caller owns the weights, the workspace and every in/out buffer and keeps them alive until
+ *    hydra_destroy.  The library owns only the opaque context; KV caches, tables and scratch are
+ *    carved out of the caller's workspace (hydra_workspace_bytes, 256-byte aligned base).
+ *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and do not synchronise, except
+ *    hydra_create (uploads tables), hydra_poll_status and hydra_destroy.
+ *  - Order: create -> prefill -> (draft -> verify -> accept_compact | step)*.  A call out of order
+ *    returns HYDRA_ERR_STATE.  The host keeps an upper bound of every sequence length (it grows by
+ *    K+1 per step); a step that could exceed max_seq returns HYDRA_ERR_CAPACITY before any launch.
+ *  - Device-side problems (token id / slot out of range, a bounded wait that ran out) set a status
+ *    word that hydra_poll_status returns; kernels skip the offending access and never trap.
+ */
+#ifndef HYDRA_H_
+#define HYDRA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hydra_ctx hydra_ctx;
+
+typedef enum {
+  HYDRA_OK = 0,
+  HYDRA_ERR_INVALID = 1,     /* null pointer, non-positive size, malformed tree */
+  HYDRA_ERR_CAPACITY = 2,    /* workspace too small, or a sequence could outgrow max_seq */
+  HYDRA_ERR_STATE = 3,       /* call out of order */
+  HYDRA_ERR_UNSUPPORTED = 4, /* shape outside what the kernels cover */
+  HYDRA_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (see hydra_last_error) */
+  HYDRA_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out */
+  HYDRA_ERR_BOUNDS = 7       /* a device-side index check failed */
+} hydra_status;
+
+/* Base model: Llama-style decoder (RMSNorm, rotary embedding with half-split pairing, SiLU-gated FFN). */
+typedef struct {
+  int n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+  float rms_eps, rope_theta;
+  int dtype;               /* 0 = float, 1 = bfloat16 */
+  int max_batch, max_seq;  /* capacity of the KV caches */
+} hydra_model_cfg;
+
+/* Draft model: K heads, head i an m-layer residual SiLU MLP over [h ; E[x_t] ; E of the i-1 tokens
+ * speculated before it] (Section "Hydra Heads"); prefix_attn adds the extra decoder layer that is
+ * queried once per step (Section "Hydra++", "Prefix Attention"). */
+typedef struct {
+  int n_heads;       /* K */
+  int n_mlp_layers;  /* m >= 1 */
+  int prefix_attn;   /* 0 | 1 */
+  int has_bias;      /* 0 | 1 */
+} hydra_head_cfg;
+
+/* Static candidate tree (Background, "Tree decoding").  parent is a HOST array of n_rows entries:
+ * parent[0] = -1 (root = the committed token not yet run through the base model), 0 <= parent[i] < i,
+ * rows ordered by (depth, rank path), depth <= K, n_rows <= 64. */
+typedef struct {
+  int n_rows;
+  const int32_t* parent;
+} hydra_tree_cfg;
+
+/* Device weight pointers.  Arrays of pointers (attn_norm[l], ...) are HOST arrays of n_layers (or K)
+ * DEVICE pointers.  wqkv rows are q, k, v in that order; w_gate_up rows are gate then up. */
+typedef struct {
+  const void *embed /*[V][d]*/, *lm_head /*[V][d]*/, *final_norm /*[d]*/;
+  const void *const *attn_norm /*[d]*/, *const *wqkv /*[3d][d]*/, *const *wo /*[d][d]*/;
+  const void *const *ffn_norm /*[d]*/, *const *w_gate_up /*[2f][d]*/, *const *w_down /*[d][f]*/;
+  const void *const *head_w1 /*[K] -> [d][(i+1)d], i = 1..K*/, *const *head_b1 /*[K] -> [d]*/;
+  const void *const *head_wr /*[K] -> [m-1][d][d]*/, *const *head_br /*[K] -> [m-1][d]*/;
+  const void *pfx_attn_norm, *pfx_wqkv, *pfx_wo, *pfx_ffn_norm, *pfx_w_gate_up, *pfx_w_down; /* prefix layer or NULL */
+} hydra_weights;
+
+/* Bytes of device workspace hydra_create needs for these configs (0 if they are invalid). */
+size_t hydra_workspace_bytes(const hydra_model_cfg*, const hydra_head_cfg*, const hydra_tree_cfg*);
+
+/* Validate the configs, build and upload the tree tables (depth, ancestor bitmask, paths, levels),
+ * carve the workspace (256-byte aligned; it is cleared by this call). */
+hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg*, const hydra_head_cfg*, const hydra_tree_cfg*,
+                          const hydra_weights*, void* workspace_dev, size_t workspace_bytes);
+hydra_status hydra_destroy(hydra_ctx*);
+
+/* Base-model forward over the prompts (ordinary causal attention) filling the KV caches; leaves, per
+ * sequence, the committed length, the root token (argmax after the last prompt token) and the last
+ * hidden state.  tokens_dev holds the prompts back to back; seq_offsets_host has batch+1 entries. */
+hydra_status hydra_prefill(hydra_ctx*, int batch, const int32_t* tokens_dev, const int32_t* seq_offsets_host,
+                           void* stream);
+
+/* Populate the candidate tree level by level: children of a node = its head's top tokens in
+ * descending order (ties: lower token id first).  tree_tok_dev [batch][n_rows] out, row 0 = root. */
+hydra_status hydra_draft(hydra_ctx*, int32_t* tree_tok_dev, void* stream);
+
+/* One base forward over all tree rows of all sequences with the ancestor mask; K,V of row i land in
+ * cache slot len+i.  amax_dev [batch][n_rows] out: argmax of each row's logits (ties: lowest id).
+ * logits_dev [batch][n_rows][vocab] float out, or NULL.  tree_tok_dev may be edited by the caller. */
+hydra_status hydra_verify(hydra_ctx*, const int32_t* tree_tok_dev, int32_t* amax_dev, float* logits_dev, void* stream);
+
+/* Greedy acceptance and in-place cache compaction in one kernel.  A candidate is accepted when it
+ * equals amax of its parent and its parent is accepted; the deepest accepted row wins (lowest row
+ * among equals).  n_acc_dev [batch]: accepted candidates (0..K); path_dev [batch][K+1]: accepted rows
+ * root..best, -1 padded; out_tok_dev [batch][K+1]: accepted tokens then the bonus token, -1 padded.
+ * Any of the three outputs may be NULL.  Updates the committed lengths, root tokens and hidden rows. */
+hydra_status hydra_accept_compact(hydra_ctx*, const int32_t* tree_tok_dev, const int32_t* amax_dev,
+                                  int32_t* n_acc_dev, int32_t* path_dev, int32_t* out_tok_dev, void* stream);
+
+/* draft + (optional planting) + verify + accept_compact on the library's own buffers. */
+hydra_status hydra_step(hydra_ctx*, int32_t* n_acc_dev, int32_t* out_tok_dev, void* stream);
+
+/* Accept-exercise mode: plant_dev [batch][n_rows], -1 keeps the drafted token; applied between draft
+ * and verify inside hydra_step.  NULL disables.  The buffer is read at every step. */
+hydra_status hydra_set_plant(hydra_ctx*, const int32_t* plant_dev);
+
+/* Introspection for parity tests: device pointers into library buffers, valid until destroy. */
+enum {
+  HYDRA_BUF_LEN = 0,        /* int32 [max_batch] committed lengths */
+  HYDRA_BUF_ROOT_TOK = 1,   /* int32 [max_batch] */
+  HYDRA_BUF_H_TREE = 2,     /* float [batch*n_rows][d] post-final-norm hidden of the last verify */
+  HYDRA_BUF_H_NEW = 3,      /* float [max_batch][K+1][d] hidden rows committed by the last step */
+  HYDRA_BUF_KV_BASE = 4,    /* [n_layers][2][max_batch][n_heads][max_seq][head_dim] */
+  HYDRA_BUF_KV_PREFIX = 5,  /* [2][max_batch][n_heads][max_seq][head_dim] */
+  HYDRA_BUF_TREE_MASK = 6,  /* uint64 [n_rows] ancestor-or-self bitmask */
+  HYDRA_BUF_TREE_TOK = 7,   /* int32 [batch][n_rows] tokens of the last hydra_step */
+  HYDRA_BUF_AMAX = 8,       /* int32 [batch][n_rows] */
+  HYDRA_BUF_HEAD_LOGITS = 9,/* float [rows][vocab] logits of the last drafted level, row = b*parents+j */
+  HYDRA_BUF_N_NEW = 10,     /* int32 [max_batch] rows in H_NEW */
+  HYDRA_BUF_H_PRIME = 11,   /* float [max_batch][d] hidden state the heads consumed */
+  HYDRA_BUF_LOGITS = 12     /* float [batch*n_rows][vocab] logits of the last verify */
+};
+hydra_status hydra_get_buffer(hydra_ctx*, int which, void** dev_ptr, size_t* bytes);
+
+/* Synchronises the stream and returns (and clears) the device status word as a hydra_status. */
+hydra_status hydra_poll_status(hydra_ctx*, void* stream);
+
+/* Number of kernels the library has launched for this context since create. */
+long long hydra_launch_count(hydra_ctx*);
+
+/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA (default), 1 = the plain SIMT kernel. */
+hydra_status hydra_set_gemm_mode(hydra_ctx*, int mode);
+
+const char* hydra_status_str(hydra_status);
+const char* hydra_last_error(void); /* text of the last CUDA error seen by this thread, "" if none */
+
+/* Single-kernel entry points for kernel-level parity tests.  No context; the library makes its own
+ * tensor maps.  All pointers are device pointers.
+ * hydra_gemm: out[m][n] = sum_k x[m][k] * w[n][k] (float accumulate, float out), dtype as above;
+ *   n % 128 == 0 and k % 64 == 0 for mode 0.  splits >= 1 partial sums are reduced into out;
+ *   partial_dev needs splits*m*n floats when splits > 1 (may be NULL when splits == 1).
+ *   mode as in hydra_set_gemm_mode; status_dev is an int32 status word (bit 1 bounds, bit 2 timeout).
+ * hydra_tree_attention: q [rows][n_heads][head_dim] float (rows = batch*tc), caches
+ *   [batch][n_heads][max_seq][head_dim] (dtype), pos0 [batch] committed lengths, n_rows [batch] or
+ *   NULL (= tc), mask [tc] ancestor bitmasks; out [rows][n_heads*head_dim] (dtype).  Row i of
+ *   sequence b sees slots < pos0[b] and slot pos0[b]+j when bit j of mask[i] is set.  scratch_dev
+ *   needs hydra_attention_scratch_bytes(...) bytes. */
+hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, float* partial_dev, int m, int n, int k,
+                        int dtype, int splits, int mode, int32_t* status_dev, void* stream);
+size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
+hydra_status hydra_tree_attention(const float* q_dev, const void* k_cache_dev, const void* v_cache_dev,
+                                  const int32_t* pos0_dev, const int32_t* n_rows_dev, const uint64_t* mask_dev,
+                                  void* out_dev, void* scratch_dev, int batch, int tc, int n_heads, int head_dim,
+                                  int max_seq, int dtype, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYDRA_H_ */

@@ -1,0 +1,60 @@
+// Shared device/host helpers of libhydra (internal).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/hydra.h"
+
+namespace hydra {
+
+typedef __nv_bfloat16 bf16;
+
+// Device status word bits (sticky until polled).
+enum : int { ST_BOUNDS = 1, ST_TIMEOUT = 2 };
+
+// Launch bookkeeping: every launcher reports through this so the library can count its kernels.
+extern thread_local long long* g_launch_counter;
+void set_last_error(const char* what, cudaError_t e);
+inline void count_launch() { if (g_launch_counter) ++*g_launch_counter; }
+
+#define HYDRA_CUDA(call)                                                        \
+  do { cudaError_t e_ = (call);                                                 \
+       if (e_ != cudaSuccess) { hydra::set_last_error(#call, e_); return HYDRA_ERR_CUDA; } } while (0)
+
+#define HYDRA_LAUNCH_CHECK()                                                    \
+  do { hydra::count_launch(); cudaError_t e_ = cudaGetLastError();              \
+       if (e_ != cudaSuccess) { hydra::set_last_error("kernel launch", e_); return HYDRA_ERR_CUDA; } } while (0)
+
+#define HYDRA_TRY(call) do { hydra_status s_ = (call); if (s_ != HYDRA_OK) return s_; } while (0)
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
+
+// Rows of one forward call: `batch` sequences with `tc` row slots each; sequence b uses its first
+// n_rows[b] slots (all tc when n_rows is null).  Row i of b has KV slot pos0[b]+i, rotary position
+// pos0[b]+depth[i] and may attend to cache slots < pos0[b] and to slot pos0[b]+j iff bit j of mask[i].
+struct RowSet {
+  int batch, tc;
+  const int* n_rows;      // device [batch] or null
+  const int* pos0;        // device [batch]
+  const int* depth;       // device [tc]
+  const uint64_t* mask;   // device [tc]
+};
+
+}  // namespace hydra

@@ -1,0 +1,742 @@
+// Row-wise, element-wise, attention, draft-head and acceptance kernels of libhydra (everything that is
+// not the tensor-core GEMM).  float or bfloat16 storage, float arithmetic.
+#include "launch.h"
+#include <math.h>
+
+namespace hydra {
+
+// ------------------------------------------------------------------------------------------------
+// SIMT GEMM: out[m][n] = sum_k x[m][k] w[n][k].  One warp per output feature, MR rows per pass.
+// ------------------------------------------------------------------------------------------------
+template <typename T> struct Vec4 { };
+template <> struct Vec4<float> {
+  static __device__ __forceinline__ void load(const float* p, float (&v)[4]) {
+    float4 t = *reinterpret_cast<const float4*>(p); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+};
+template <> struct Vec4<bf16> {
+  static __device__ __forceinline__ void load(const bf16* p, float (&v)[4]) {
+    uint2 t = *reinterpret_cast<const uint2*>(p);
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&t.x), b = *reinterpret_cast<__nv_bfloat162*>(&t.y);
+    v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b); }
+};
+
+template <typename T, int MR>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ w,
+                                                        float* __restrict__ out, int m, int n, int k) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int col = blockIdx.x * 8 + warp;
+  const int m0 = blockIdx.y * MR;
+  if (col >= n) return;
+  float acc[MR];
+#pragma unroll
+  for (int r = 0; r < MR; ++r) acc[r] = 0.f;
+  const T* wr = w + (size_t)col * k;
+  for (int kk = lane * 4; kk < k; kk += 128) {
+    float wv[4];
+    Vec4<T>::load(wr + kk, wv);
+#pragma unroll
+    for (int r = 0; r < MR; ++r) {
+      int row = m0 + r < m ? m0 + r : m - 1;
+      float xv[4];
+      Vec4<T>::load(x + (size_t)row * k + kk, xv);
+      acc[r] += wv[0] * xv[0] + wv[1] * xv[1] + wv[2] * xv[2] + wv[3] * xv[3];
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < MR; ++r) {
+    float s = warp_sum(acc[r]);
+    if (lane == 0 && m0 + r < m) out[(size_t)(m0 + r) * n + col] = s;
+  }
+}
+
+hydra_status gemm_simt(const void* x, const void* w, float* out, int m, int n, int k, int dtype, cudaStream_t st) {
+  if (m <= 0 || n <= 0 || k <= 0 || (k & 3)) return HYDRA_ERR_UNSUPPORTED;
+  constexpr int MR = 16;
+  dim3 grid((n + 7) / 8, (m + MR - 1) / MR);
+  if (dtype == 0) gemm_simt_kernel<float, MR><<<grid, 256, 0, st>>>((const float*)x, (const float*)w, out, m, n, k);
+  else gemm_simt_kernel<bf16, MR><<<grid, 256, 0, st>>>((const bf16*)x, (const bf16*)w, out, m, n, k);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+__global__ void reduce_splits_kernel(const float* __restrict__ part, size_t stride, int splits, float* __restrict__ out,
+                                     size_t count) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  float s = 0.f;
+  for (int p = 0; p < splits; ++p) s += part[p * stride + i];
+  out[i] = s;
+}
+hydra_status reduce_splits(const float* part, size_t stride, int splits, float* out, size_t count, cudaStream_t st) {
+  reduce_splits_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(part, stride, splits, out, count);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Embedding gather
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_rows_kernel(const T* __restrict__ embed, const int* __restrict__ tok, float* __restrict__ x, int d,
+                                  int vocab, int* status) {
+  int r = blockIdx.x;
+  int t = tok[r];
+  if (t < 0 || t >= vocab) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); t = 0; }
+  const T* e = embed + (size_t)t * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)r * d + i] = to_f<T>(e[i]);
+}
+hydra_status embed_rows(const void* embed, const int* tok, float* x, int rows, int d, int vocab, int dtype, int* status,
+                        cudaStream_t st) {
+  if (dtype == 0) embed_rows_kernel<float><<<rows, 256, 0, st>>>((const float*)embed, tok, x, d, vocab, status);
+  else embed_rows_kernel<bf16><<<rows, 256, 0, st>>>((const bf16*)embed, tok, x, d, vocab, status);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Residual add of split-K partial sums + RMSNorm (Llama: x * gain / sqrt(mean(x^2) + eps))
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float block_sum(float v, float* sh) {
+  v = warp_sum(v);
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) sh[warp] = v;
+  __syncthreads();
+  float t = (threadIdx.x < (blockDim.x >> 5)) ? sh[threadIdx.x] : 0.f;
+  if (warp == 0) { t = warp_sum(t); if (lane == 0) sh[0] = t; }
+  __syncthreads();
+  t = sh[0];
+  __syncthreads();
+  return t;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) residual_rmsnorm_kernel(const float* res, const float* __restrict__ part,
+                                                               size_t stride, int splits, float* x_out,
+                                                               const T* __restrict__ gain, T* __restrict__ xn,
+                                                               float* __restrict__ hn, int d, float eps) {
+  __shared__ float sh[32];
+  const size_t base = (size_t)blockIdx.x * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    float v = res ? res[base + i] : 0.f;
+    if (part) for (int p = 0; p < splits; ++p) v += part[p * stride + base + i];
+    x_out[base + i] = v;
+    ss += v * v;
+  }
+  if (!gain) return;
+  float tot = block_sum(ss, sh);
+  float inv = rsqrtf(tot / (float)d + eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    float v = x_out[base + i] * inv * to_f<T>(gain[i]);
+    if (xn) xn[base + i] = from_f<T>(v);
+    if (hn) hn[base + i] = v;
+  }
+}
+hydra_status residual_rmsnorm(const float* res, const float* part, size_t stride, int splits, float* x_out,
+                              const void* gain, void* xn, float* hn, int rows, int d, float eps, int dtype,
+                              cudaStream_t st) {
+  if (dtype == 0)
+    residual_rmsnorm_kernel<float><<<rows, 256, 0, st>>>(res, part, stride, splits, x_out, (const float*)gain, (float*)xn,
+                                                         hn, d, eps);
+  else
+    residual_rmsnorm_kernel<bf16><<<rows, 256, 0, st>>>(res, part, stride, splits, x_out, (const bf16*)gain, (bf16*)xn, hn,
+                                                        d, eps);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rotary table + QKV post-processing (sum partials, rotate q and k, append K,V to the cache)
+// ------------------------------------------------------------------------------------------------
+__global__ void rope_table_kernel(RowSet rs, float2* __restrict__ table, int half, float theta) {
+  int r = blockIdx.x, b = r / rs.tc, i = r % rs.tc;
+  int pos = rs.pos0[b] + rs.depth[i];
+  for (int j = threadIdx.x; j < half; j += blockDim.x) {
+    double inv = exp2(-((double)j / (double)half) * log2((double)theta));
+    double s, c;
+    sincos((double)pos * inv, &s, &c);
+    table[(size_t)r * half + j] = make_float2((float)c, (float)s);
+  }
+}
+hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st) {
+  rope_table_kernel<<<rs.batch * rs.tc, 64, 0, st>>>(rs, table, head_dim / 2, theta);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __restrict__ part, size_t stride, int splits,
+                                                             const float2* __restrict__ table, float* __restrict__ q,
+                                                             T* __restrict__ kc, T* __restrict__ vc, RowSet rs, int H,
+                                                             int hd, int max_seq, int* status) {
+  const int r = blockIdx.x, b = r / rs.tc, i = r % rs.tc;
+  const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
+  if (i >= nr) return;
+  const int d = H * hd, half = hd >> 1;
+  const int slot = rs.pos0[b] + i;
+  if (slot < 0 || slot >= max_seq) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); return; }
+  const float* p0 = part + (size_t)r * 3 * d;
+  for (int e = threadIdx.x; e < H * half; e += blockDim.x) {
+    int h = e / half, j = e % half;
+    int c0 = h * hd + j, c1 = c0 + half;
+    float qa = 0, qb = 0, ka = 0, kb = 0, va = 0, vb = 0;
+    for (int s = 0; s < splits; ++s) {
+      const float* p = p0 + s * stride;
+      qa += p[c0]; qb += p[c1]; ka += p[d + c0]; kb += p[d + c1]; va += p[2 * d + c0]; vb += p[2 * d + c1];
+    }
+    float2 cs = table[(size_t)r * half + j];
+    q[(size_t)r * d + c0] = qa * cs.x - qb * cs.y;
+    q[(size_t)r * d + c1] = qb * cs.x + qa * cs.y;
+    size_t o = (((size_t)b * H + h) * max_seq + slot) * hd;
+    kc[o + j] = from_f<T>(ka * cs.x - kb * cs.y);
+    kc[o + j + half] = from_f<T>(kb * cs.x + ka * cs.y);
+    vc[o + j] = from_f<T>(va);
+    vc[o + j + half] = from_f<T>(vb);
+  }
+}
+hydra_status qkv_rope_store(const float* part, size_t stride, int splits, const float2* table, float* q, void* kcache,
+                            void* vcache, RowSet rs, int H, int hd, int max_seq, int dtype, int* status,
+                            cudaStream_t st) {
+  int rows = rs.batch * rs.tc;
+  if (dtype == 0)
+    qkv_rope_store_kernel<float><<<rows, 256, 0, st>>>(part, stride, splits, table, q, (float*)kcache, (float*)vcache, rs,
+                                                       H, hd, max_seq, status);
+  else
+    qkv_rope_store_kernel<bf16><<<rows, 256, 0, st>>>(part, stride, splits, table, q, (bf16*)kcache, (bf16*)vcache, rs, H,
+                                                      hd, max_seq, status);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Tree attention, split over the KV length.  One CTA per (head, sequence, KV chunk); the chunk's K,V
+// rows are read once; every query row keeps an online softmax (running max, sum, weighted V) per warp.
+// ------------------------------------------------------------------------------------------------
+constexpr int ATT_CHUNK = 128;    // KV rows per CTA
+constexpr int ATT_TILE = 32;      // KV rows staged per iteration
+constexpr int ATT_WARPS = 8;
+
+template <typename T, int HD>
+__global__ void __launch_bounds__(ATT_WARPS * 32) tree_attn_kernel(const float* __restrict__ q, const T* __restrict__ kc,
+                                                                   const T* __restrict__ vc, RowSet rs,
+                                                                   float* __restrict__ part_o, float* __restrict__ part_ml,
+                                                                   int H, int max_seq, int nchunks) {
+  extern __shared__ float smem[];
+  constexpr int RPW = 8;                                  // query rows per warp (tc <= 64)
+  constexpr int KPL = HD / 32;                            // output dims per lane
+  float* qs = smem;                                       // [64][HD]
+  float* ks = qs + 64 * HD;                               // [ATT_TILE][HD+1]
+  float* vs = ks + ATT_TILE * (HD + 1);                   // [ATT_TILE][HD]
+  const int h = blockIdx.x, b = blockIdx.y, c = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
+  const int p0 = rs.pos0[b];
+  const int total = p0 + nr;
+  const int s0 = c * ATT_CHUNK;
+  const int s1 = min(s0 + ATT_CHUNK, total);
+  const int d = H * HD;
+  const float scale = rsqrtf((float)HD);
+
+  for (int e = threadIdx.x; e < nr * HD; e += blockDim.x) {
+    int i = e / HD, k = e % HD;
+    qs[i * HD + k] = q[((size_t)(b * rs.tc + i)) * d + h * HD + k] * scale;
+  }
+  float m[RPW], l[RPW], o[RPW][KPL];
+  uint64_t msk[RPW];
+#pragma unroll
+  for (int j = 0; j < RPW; ++j) {
+    m[j] = -INFINITY; l[j] = 0.f;
+    int r = warp * RPW + j;
+    msk[j] = r < nr ? rs.mask[r] : 0ull;
+#pragma unroll
+    for (int kk = 0; kk < KPL; ++kk) o[j][kk] = 0.f;
+  }
+  const T* kbase = kc + ((size_t)b * H + h) * max_seq * HD;
+  const T* vbase = vc + ((size_t)b * H + h) * max_seq * HD;
+
+  for (int t0 = s0; t0 < s1; t0 += ATT_TILE) {
+    __syncthreads();
+    for (int e = threadIdx.x; e < ATT_TILE * HD; e += blockDim.x) {
+      int j = e / HD, k = e % HD;
+      int slot = t0 + j;
+      float kv = 0.f, vv = 0.f;
+      if (slot < s1) { kv = to_f<T>(kbase[(size_t)slot * HD + k]); vv = to_f<T>(vbase[(size_t)slot * HD + k]); }
+      ks[j * (HD + 1) + k] = kv;
+      vs[j * HD + k] = vv;
+    }
+    __syncthreads();
+    const int slot = t0 + lane;
+#pragma unroll
+    for (int j = 0; j < RPW; ++j) {
+      const int r = warp * RPW + j;
+      if (r >= nr) continue;
+      bool valid = slot < s1 && (slot < p0 || ((msk[j] >> (slot - p0)) & 1ull));
+      float sc = 0.f;
+      const float* qr = qs + r * HD;
+      const float* kr = ks + lane * (HD + 1);
+#pragma unroll 8
+      for (int k = 0; k < HD; ++k) sc += qr[k] * kr[k];
+      sc = valid ? sc : -INFINITY;
+      float mn = fmaxf(m[j], warp_max(sc));
+      if (mn == -INFINITY) continue;
+      float alpha = expf(m[j] - mn);
+      float p = valid ? expf(sc - mn) : 0.f;
+      l[j] = l[j] * alpha + warp_sum(p);
+      float acc[KPL];
+#pragma unroll
+      for (int kk = 0; kk < KPL; ++kk) acc[kk] = o[j][kk] * alpha;
+      for (int jj = 0; jj < ATT_TILE; ++jj) {
+        float pj = __shfl_sync(0xffffffffu, p, jj);
+#pragma unroll
+        for (int kk = 0; kk < KPL; ++kk) acc[kk] += pj * vs[jj * HD + lane + 32 * kk];
+      }
+#pragma unroll
+      for (int kk = 0; kk < KPL; ++kk) o[j][kk] = acc[kk];
+      m[j] = mn;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < RPW; ++j) {
+    const int r = warp * RPW + j;
+    if (r >= nr) continue;
+    size_t idx = ((size_t)(b * rs.tc + r) * H + h) * nchunks + c;
+#pragma unroll
+    for (int kk = 0; kk < KPL; ++kk) part_o[idx * HD + lane + 32 * kk] = o[j][kk];
+    if (lane == 0) { part_ml[idx * 2] = m[j]; part_ml[idx * 2 + 1] = l[j]; }
+  }
+}
+
+template <typename T, int HD>
+__global__ void tree_attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, RowSet rs,
+                                         T* __restrict__ out, int H, int nchunks) {
+  const int r = blockIdx.x, h = blockIdx.y, b = r / rs.tc, i = r % rs.tc;
+  const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
+  const int k = threadIdx.x;
+  T* dst = out + (size_t)r * H * HD + h * HD;
+  if (i >= nr) { dst[k] = from_f<T>(0.f); return; }
+  const int used = min(nchunks, (rs.pos0[b] + nr + ATT_CHUNK - 1) / ATT_CHUNK);
+  size_t idx = ((size_t)r * H + h) * nchunks;
+  float M = -INFINITY;
+  for (int c = 0; c < used; ++c) M = fmaxf(M, part_ml[(idx + c) * 2]);
+  float L = 0.f, acc = 0.f;
+  for (int c = 0; c < used; ++c) {
+    float mc = part_ml[(idx + c) * 2];
+    if (mc == -INFINITY) continue;
+    float w = expf(mc - M);
+    L += part_ml[(idx + c) * 2 + 1] * w;
+    acc += part_o[(idx + c) * HD + k] * w;
+  }
+  dst[k] = from_f<T>(acc / L);
+}
+
+size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq) {
+  size_t nchunks = (size_t)(max_seq + ATT_CHUNK - 1) / ATT_CHUNK;
+  return (size_t)batch * tc * n_heads * nchunks * (head_dim + 2) * sizeof(float);
+}
+
+template <typename T, int HD>
+static hydra_status tree_attention_t(const float* q, const T* kc, const T* vc, RowSet rs, T* out, float* scratch, int H,
+                                     int max_seq, int len_upper, cudaStream_t st) {
+  int nchunks_max = (max_seq + ATT_CHUNK - 1) / ATT_CHUNK;
+  int nchunks = (len_upper + ATT_CHUNK - 1) / ATT_CHUNK;
+  if (nchunks < 1) nchunks = 1;
+  if (nchunks > nchunks_max) nchunks = nchunks_max;
+  size_t rows = (size_t)rs.batch * rs.tc;
+  float* part_o = scratch;
+  float* part_ml = scratch + rows * H * nchunks_max * HD;
+  size_t smem = (size_t)(64 * HD + ATT_TILE * (HD + 1) + ATT_TILE * HD) * sizeof(float);
+  static bool attr_done = false;
+  if (!attr_done) {
+    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_kernel<T, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_done = true;
+  }
+  tree_attn_kernel<T, HD><<<dim3(H, rs.batch, nchunks), ATT_WARPS * 32, smem, st>>>(q, kc, vc, rs, part_o, part_ml, H,
+                                                                                   max_seq, nchunks);
+  HYDRA_LAUNCH_CHECK();
+  tree_attn_combine_kernel<T, HD><<<dim3((unsigned)rows, H), HD, 0, st>>>(part_o, part_ml, rs, out, H, nchunks);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+hydra_status tree_attention(const float* q, const void* kc, const void* vc, RowSet rs, void* out, void* scratch, int H,
+                            int hd, int max_seq, int len_upper, int dtype, cudaStream_t st) {
+  if (rs.tc > 64) return HYDRA_ERR_UNSUPPORTED;
+  if (dtype == 0 && hd == 64)
+    return tree_attention_t<float, 64>(q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
+  if (dtype == 0 && hd == 128)
+    return tree_attention_t<float, 128>(q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
+  if (dtype == 1 && hd == 64)
+    return tree_attention_t<bf16, 64>(q, (const bf16*)kc, (const bf16*)vc, rs, (bf16*)out, (float*)scratch, H, max_seq, len_upper, st);
+  if (dtype == 1 && hd == 128)
+    return tree_attention_t<bf16, 128>(q, (const bf16*)kc, (const bf16*)vc, rs, (bf16*)out, (float*)scratch, H, max_seq, len_upper, st);
+  return HYDRA_ERR_UNSUPPORTED;
+}
+
+// ------------------------------------------------------------------------------------------------
+// SiLU(gate) * up from the gate/up partial sums
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void silu_mul_kernel(const float* __restrict__ part, size_t stride, int splits, T* __restrict__ act, int rows,
+                                int f) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)rows * f) return;
+  size_t r = i / f, c = i % f;
+  float g = 0.f, u = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const float* p = part + s * stride + r * 2 * f;
+    g += p[c]; u += p[f + c];
+  }
+  act[i] = from_f<T>(silu_f(g) * u);
+}
+hydra_status silu_mul(const float* part, size_t stride, int splits, void* act, int rows, int f, int dtype,
+                      cudaStream_t st) {
+  size_t n = (size_t)rows * f;
+  unsigned grid = (unsigned)((n + 255) / 256);
+  if (dtype == 0) silu_mul_kernel<float><<<grid, 256, 0, st>>>(part, stride, splits, (float*)act, rows, f);
+  else silu_mul_kernel<bf16><<<grid, 256, 0, st>>>(part, stride, splits, (bf16*)act, rows, f);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// argmax / top-k with total order (value descending, token id ascending)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
+
+__device__ __forceinline__ void block_best(float& v, int& i, float* shv, int* shi) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, v, o);
+    int oi = __shfl_xor_sync(0xffffffffu, i, o);
+    if (better(ov, oi, v, i)) { v = ov; i = oi; }
+  }
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __syncthreads();
+  if (lane == 0) { shv[warp] = v; shi[warp] = i; }
+  __syncthreads();
+  if (warp == 0) {
+    int nw = blockDim.x >> 5;
+    v = lane < nw ? shv[lane] : -INFINITY;
+    i = lane < nw ? shi[lane] : 0x7fffffff;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, v, o);
+      int oi = __shfl_xor_sync(0xffffffffu, i, o);
+      if (better(ov, oi, v, i)) { v = ov; i = oi; }
+    }
+    if (lane == 0) { shv[0] = v; shi[0] = i; }
+  }
+  __syncthreads();
+  v = shv[0]; i = shi[0];
+}
+
+__global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restrict__ logits, int* __restrict__ amax,
+                                                          int vocab) {
+  __shared__ float shv[32];
+  __shared__ int shi[32];
+  const float* row = logits + (size_t)blockIdx.x * vocab;
+  float bv = -INFINITY; int bi = 0x7fffffff;
+  for (int i = threadIdx.x; i < vocab; i += blockDim.x) { float v = row[i]; if (better(v, i, bv, bi)) { bv = v; bi = i; } }
+  block_best(bv, bi, shv, shi);
+  if (threadIdx.x == 0) amax[blockIdx.x] = bi;
+}
+hydra_status argmax_rows(const float* logits, int* amax, int rows, int vocab, cudaStream_t st) {
+  argmax_rows_kernel<<<rows, 256, 0, st>>>(logits, amax, vocab);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+__global__ void __launch_bounds__(256) topk_children_kernel(const float* __restrict__ logits, LevelDesc lv,
+                                                            const int* __restrict__ first_child,
+                                                            const int* __restrict__ n_child, int* __restrict__ tree_tok,
+                                                            int T, int vocab) {
+  __shared__ float shv[32];
+  __shared__ int shi[32];
+  const int row = blockIdx.x, b = row / lv.n_parents, j = row % lv.n_parents;
+  const int p = lv.parents[j];
+  const int nc = n_child[p], fc = first_child[p];
+  const float* lg = logits + (size_t)row * vocab;
+  float pv = INFINITY; int pi = -1;
+  for (int t = 0; t < nc; ++t) {
+    float bv = -INFINITY; int bi = 0x7fffffff;
+    for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
+      float v = lg[i];
+      bool after = v < pv || (v == pv && i > pi);          // strictly after the previous pick in the order
+      if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
+    }
+    block_best(bv, bi, shv, shi);
+    if (threadIdx.x == 0) tree_tok[b * T + fc + t] = bi;
+    pv = bv; pi = bi;
+  }
+}
+hydra_status topk_children(const float* logits, LevelDesc lv, const int* first_child, const int* n_child, int* tree_tok,
+                           int batch, int T, int vocab, cudaStream_t st) {
+  topk_children_kernel<<<batch * lv.n_parents, 256, 0, st>>>(logits, lv, first_child, n_child, tree_tok, T, vocab);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Hydra heads: input gather and the residual SiLU layer epilogue
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) head_gather_kernel(const float* __restrict__ hprime, const T* __restrict__ embed,
+                                                          const int* __restrict__ root_tok, int* tree_tok,
+                                                          const int* __restrict__ path_tab, LevelDesc lv, T* __restrict__ z,
+                                                          int T_rows, int kp1, int d_model, int vocab, int* status) {
+  const int row = blockIdx.x, b = row / lv.n_parents, j = row % lv.n_parents;
+  const int blk = blockIdx.y;                               // 0: hidden, 1..d: path tokens root..parent
+  const int p = lv.parents[j];
+  T* dst = z + ((size_t)row * (lv.d + 1) + blk) * d_model;
+  if (blk == 0) {
+    for (int i = threadIdx.x; i < d_model; i += blockDim.x) dst[i] = from_f<T>(hprime[(size_t)b * d_model + i]);
+    if (lv.d == 1 && j == 0 && threadIdx.x == 0) tree_tok[b * T_rows] = root_tok[b];
+    return;
+  }
+  int node = path_tab[p * kp1 + (blk - 1)];
+  int t = node == 0 ? root_tok[b] : tree_tok[b * T_rows + node];
+  if (t < 0 || t >= vocab) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); t = 0; }
+  const T* e = embed + (size_t)t * d_model;
+  for (int i = threadIdx.x; i < d_model; i += blockDim.x) dst[i] = e[i];
+}
+hydra_status head_gather(const float* hprime, const void* embed, const int* root_tok, int* tree_tok, const int* path_tab,
+                         LevelDesc lv, void* z, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
+                         cudaStream_t st) {
+  dim3 grid(batch * lv.n_parents, lv.d + 1);
+  if (dtype == 0)
+    head_gather_kernel<float><<<grid, 256, 0, st>>>(hprime, (const float*)embed, root_tok, tree_tok, path_tab, lv, (float*)z,
+                                                    T, kp1, d_model, vocab, status);
+  else
+    head_gather_kernel<bf16><<<grid, 256, 0, st>>>(hprime, (const bf16*)embed, root_tok, tree_tok, path_tab, lv, (bf16*)z,
+                                                   T, kp1, d_model, vocab, status);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+template <typename T>
+__global__ void head_act_kernel(const float* res, int res_is_hprime, int rows_per_b, const float* __restrict__ part,
+                                size_t stride, int splits, const T* __restrict__ bias, float* y_out, T* __restrict__ yb,
+                                int rows, int d) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)rows * d) return;
+  int r = (int)(i / d), c = (int)(i % d);
+  float v = bias ? to_f<T>(bias[c]) : 0.f;
+  for (int s = 0; s < splits; ++s) v += part[s * stride + i];
+  float base = res_is_hprime ? res[(size_t)(r / rows_per_b) * d + c] : res[i];
+  float y = base + silu_f(v);
+  y_out[i] = y;
+  yb[i] = from_f<T>(y);
+}
+hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, size_t stride, int splits,
+                      const void* bias, float* y_out, void* yb, int rows, int d, int dtype, cudaStream_t st) {
+  size_t n = (size_t)rows * d;
+  unsigned grid = (unsigned)((n + 255) / 256);
+  if (dtype == 0)
+    head_act_kernel<float><<<grid, 256, 0, st>>>(res, res_is_hprime, rows_per_b, part, stride, splits, (const float*)bias,
+                                                 y_out, (float*)yb, rows, d);
+  else
+    head_act_kernel<bf16><<<grid, 256, 0, st>>>(res, res_is_hprime, rows_per_b, part, stride, splits, (const bf16*)bias,
+                                                y_out, (bf16*)yb, rows, d);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Greedy acceptance + in-place KV compaction + state update, one kernel.
+// grid (G, batch).  Every CTA recomputes the accepted path of its sequence (cheap), then moves its
+// share of 16-byte KV pieces.  A thread moves its piece for k = 1..n in order: the destination slot k
+// can only be the source of a shallower path position (a row at depth j has index >= j), which that
+// same thread has already read, so the in-place move is hazard-free.  The last CTA of a sequence to
+// finish publishes the new length / root token; all CTAs read the old length before they signal.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
+  __shared__ int s_path[72];
+  __shared__ int s_n, s_best;
+  const int b = blockIdx.y;
+  const int T = a.T;
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    uint64_t bits = 0;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      int i = lane + 32 * half;
+      bool mt = false;
+      if (i >= 1 && i < T) mt = a.tree_tok[b * T + i] == a.amax[b * T + a.parent[i]];
+      bits |= (uint64_t)__ballot_sync(0xffffffffu, mt) << (32 * half);
+    }
+    int key = -1;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      int i = lane + 32 * half;
+      if (i < T) {
+        bool acc = ((a.anc[i] & ~1ull) & ~bits) == 0ull;
+        if (acc) key = max(key, a.depth[i] * 64 + (63 - i));
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
+    if (lane == 0) {
+      int best = 63 - (key & 63), n = key >> 6;
+      s_n = n; s_best = best;
+      int node = best;
+      for (int k = n; k >= 0; --k) { s_path[k] = node; node = a.parent[node]; }
+    }
+  }
+  __syncthreads();
+  const int n = s_n, best = s_best;
+  const int L = a.len[b];
+  const bool in_range = L >= 0 && L + T <= a.max_seq;
+  if (!in_range) {
+    if (threadIdx.x == 0) atomicOr(a.status, ST_BOUNDS);
+  } else {
+    const int row_bytes = a.head_dim * a.esize;
+    const int ppr = row_bytes / 16;                                    // 16-byte pieces per row
+    const long long units = (long long)a.n_layers * 2 * a.n_heads * ppr;
+    for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += (long long)gridDim.x * blockDim.x) {
+      int piece = (int)(u % ppr);
+      long long t = u / ppr;
+      int head = (int)(t % a.n_heads);
+      long long lk = t / a.n_heads;                                    // layer*2 + kv
+      char* base = (char*)a.kv_base + ((((size_t)lk * a.max_batch + b) * a.n_heads + head) * a.max_seq) * row_bytes;
+      for (int k = 1; k <= n; ++k) {
+        int src = s_path[k];
+        if (src != k)
+          *reinterpret_cast<uint4*>(base + (size_t)(L + k) * row_bytes + piece * 16) =
+              *reinterpret_cast<const uint4*>(base + (size_t)(L + src) * row_bytes + piece * 16);
+      }
+    }
+    // hidden rows of the accepted path feed the next draft
+    const int d4 = a.d_model / 4;
+    for (int u = blockIdx.x * blockDim.x + threadIdx.x; u < (n + 1) * d4; u += gridDim.x * blockDim.x) {
+      int k = u / d4, c = u % d4;
+      reinterpret_cast<float4*>(a.h_new + ((size_t)b * (a.K + 1) + k) * a.d_model)[c] =
+          reinterpret_cast<const float4*>(a.h_tree + ((size_t)b * a.h_tree_stride + s_path[k]) * a.d_model)[c];
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x <= a.K) {
+    int k = threadIdx.x;
+    if (a.path) a.path[b * (a.K + 1) + k] = k <= n ? s_path[k] : -1;
+    if (a.out_tok) {
+      int v = -1;
+      if (k < n) v = a.tree_tok[b * T + s_path[k + 1]];
+      else if (k == n) v = a.amax[b * T + best];
+      a.out_tok[b * (a.K + 1) + k] = v;
+    }
+    if (k == 0 && a.n_acc) a.n_acc[b] = n;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned prev = atomicAdd(&a.done_counter[b], 1u);
+    if (prev == gridDim.x - 1) {
+      a.done_counter[b] = 0;
+      if (in_range) {
+        a.len[b] = L + n + 1;
+        a.root_tok[b] = a.amax[b * T + best];
+        a.n_new[b] = n + 1;
+      }
+    }
+  }
+}
+hydra_status accept_compact(const AcceptArgs& a, cudaStream_t st) {
+  long long units = (long long)a.n_layers * 2 * a.n_heads * (a.head_dim * a.esize / 16);
+  int G = (int)((units + 255) / 256);
+  int cap = (148 * 4 + a.batch - 1) / a.batch;
+  if (G > cap) G = cap;
+  if (G < 1) G = 1;
+  accept_compact_kernel<<<dim3(G, a.batch), 256, 0, st>>>(a);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Small state kernels
+// ------------------------------------------------------------------------------------------------
+__global__ void set_chunk_kernel(const int* prompt_len, int chunk, int tc, int* pos0, int* n_rows, int batch) {
+  int b = threadIdx.x;
+  if (b >= batch) return;
+  int rem = prompt_len[b] - chunk * tc;
+  pos0[b] = rem > 0 ? chunk * tc : prompt_len[b];
+  n_rows[b] = rem < 0 ? 0 : (rem > tc ? tc : rem);
+}
+hydra_status set_chunk(const int* prompt_len, int chunk, int tc, int* pos0, int* n_rows, int batch, cudaStream_t st) {
+  set_chunk_kernel<<<1, 64, 0, st>>>(prompt_len, chunk, tc, pos0, n_rows, batch);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+__global__ void gather_chunk_tokens_kernel(const int* tokens, const int* offsets, int chunk, int tc, int* tok_out) {
+  int b = blockIdx.x, i = threadIdx.x;
+  if (i >= tc) return;
+  int n = offsets[b + 1] - offsets[b];
+  int idx = chunk * tc + i;
+  tok_out[b * tc + i] = idx < n ? tokens[offsets[b] + idx] : 0;
+}
+hydra_status gather_chunk_tokens(const int* tokens, const int* offsets, int chunk, int tc, int* tok_out, int batch,
+                                 cudaStream_t st) {
+  gather_chunk_tokens_kernel<<<batch, 64, 0, st>>>(tokens, offsets, chunk, tc, tok_out);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+__global__ void capture_last_kernel(const float* h, const int* prompt_len, int chunk, int tc, float* h_new, int kp1,
+                                    int* n_new, int* len, int d) {
+  int b = blockIdx.x;
+  int last = prompt_len[b] - 1;
+  if (last < chunk * tc || last >= (chunk + 1) * tc) return;
+  int i = last - chunk * tc;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) h_new[(size_t)b * kp1 * d + c] = h[((size_t)b * tc + i) * d + c];
+  if (threadIdx.x == 0) { n_new[b] = 1; len[b] = prompt_len[b]; }
+}
+hydra_status capture_last(const float* h, const int* prompt_len, int chunk, int tc, float* h_new, int kp1, int* n_new,
+                          int* len, int batch, int d, cudaStream_t st) {
+  capture_last_kernel<<<batch, 256, 0, st>>>(h, prompt_len, chunk, tc, h_new, kp1, n_new, len, d);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+__global__ void prefix_rowset_kernel(const int* len, const int* n_new, int* pos0, int* n_rows, int batch) {
+  int b = threadIdx.x;
+  if (b >= batch) return;
+  pos0[b] = len[b] - n_new[b];
+  n_rows[b] = n_new[b];
+}
+hydra_status prefix_rowset(const int* len, const int* n_new, int* pos0, int* n_rows, int batch, cudaStream_t st) {
+  prefix_rowset_kernel<<<1, 64, 0, st>>>(len, n_new, pos0, n_rows, batch);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+__global__ void pick_last_row_kernel(const float* x, const int* n_rows, int tc, float* hprime, int d) {
+  int b = blockIdx.x;
+  int i = n_rows[b] - 1;
+  if (i < 0) i = 0;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) hprime[(size_t)b * d + c] = x[((size_t)b * tc + i) * d + c];
+}
+hydra_status pick_last_row(const float* x, const int* n_rows, int tc, float* hprime, int batch, int d, cudaStream_t st) {
+  pick_last_row_kernel<<<batch, 256, 0, st>>>(x, n_rows, tc, hprime, d);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+__global__ void apply_plant_kernel(int* tree_tok, const int* plant, int count) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count && plant[i] >= 0) tree_tok[i] = plant[i];
+}
+hydra_status apply_plant(int* tree_tok, const int* plant, int count, cudaStream_t st) {
+  apply_plant_kernel<<<(count + 255) / 256, 256, 0, st>>>(tree_tok, plant, count);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+__global__ void copy_i32_kernel(int* dst, const int* src, int count) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) dst[i] = src[i];
+}
+hydra_status copy_i32(int* dst, const int* src, int count, cudaStream_t st) {
+  copy_i32_kernel<<<(count + 255) / 256, 256, 0, st>>>(dst, src, count);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+}  // namespace hydra

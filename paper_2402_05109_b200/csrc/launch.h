@@ -1,0 +1,81 @@
+// Host-side launchers of every kernel (internal).  Each enqueues on `st` and returns a hydra_status.
+#pragma once
+#include "common.cuh"
+
+namespace hydra {
+
+// ---- GEMM: out[split][m][n] = sum over that split's k range of x[m][k] * w[n][k]
+// tcgen05 path (bfloat16 operands).  out rows have stride n; split s is written at out + s*split_stride.
+// x_rows_alloc = rows the x buffer really holds (>= m); rows of the last tile beyond m are computed and dropped.
+hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* out, size_t split_stride, int m, int n,
+                     int k, int splits, int* status, cudaStream_t st);
+bool gemm_tc_available();                 // driver entry point for tensor-map encoding found
+// SIMT path (float or bfloat16 operands), no split.
+hydra_status gemm_simt(const void* x, const void* w, float* out, int m, int n, int k, int dtype, cudaStream_t st);
+// out[i] = sum_s part[s*stride + i]
+hydra_status reduce_splits(const float* part, size_t split_stride, int splits, float* out, size_t count, cudaStream_t st);
+
+// ---- element-wise / row-wise stages of a decoder layer (dtype: 0 float, 1 bfloat16 for the "act" outputs)
+hydra_status embed_rows(const void* embed, const int* tok, float* x, int rows, int d, int vocab, int dtype, int* status,
+                        cudaStream_t st);
+// x_out = (res ? res : 0) + sum_s part[s]; if gain: xn = rmsnorm(x_out)*gain (act dtype, optional) and hn = the same in
+// float (optional).  part may be null.  x_out may alias res.
+hydra_status residual_rmsnorm(const float* res, const float* part, size_t split_stride, int splits, float* x_out,
+                              const void* gain, void* xn, float* hn, int rows, int d, float eps, int dtype,
+                              cudaStream_t st);
+// table[r][j] = (cos, sin) of (pos0[b]+depth[i]) * theta^(-2j/head_dim), evaluated in double
+hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st);
+// q (float [rows][H][hd], rotated), K/V cache rows (rotated K) from the QKV partial sums.
+hydra_status qkv_rope_store(const float* part, size_t split_stride, int splits, const float2* table, float* q,
+                            void* kcache, void* vcache, RowSet rs, int n_heads, int head_dim, int max_seq, int dtype,
+                            int* status, cudaStream_t st);
+size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
+hydra_status tree_attention(const float* q, const void* kcache, const void* vcache, RowSet rs, void* out, void* scratch,
+                            int n_heads, int head_dim, int max_seq, int len_upper, int dtype, cudaStream_t st);
+hydra_status silu_mul(const float* part, size_t split_stride, int splits, void* act, int rows, int f, int dtype,
+                      cudaStream_t st);
+// amax[r] = argmax_v logits[r][v] (lowest id among equal maxima)
+hydra_status argmax_rows(const float* logits, int* amax, int rows, int vocab, cudaStream_t st);
+
+// ---- Hydra heads
+struct LevelDesc {           // one tree level d (1-based): the parents that have children
+  int d, n_parents;
+  const int* parents;        // device [n_parents] row ids
+};
+// z[b*P+j] = [hprime[b] ; E[tok[b][path(parent j)]]] in act dtype; also tree_tok[b][0] = root_tok[b] when d == 1.
+hydra_status head_gather(const float* hprime, const void* embed, const int* root_tok, int* tree_tok, const int* path_tab,
+                         LevelDesc lv, void* z, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
+                         cudaStream_t st);
+// y_out = res + silu(sum_s part[s] + bias); res row = hprime[b] when res_is_hprime else y row.  yb = act-dtype copy.
+hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, size_t split_stride,
+                      int splits, const void* bias, float* y_out, void* yb, int rows, int d, int dtype, cudaStream_t st);
+// children of parent j of sequence b = top n_child tokens of logits row b*P+j, descending (ties: lower id first)
+hydra_status topk_children(const float* logits, LevelDesc lv, const int* first_child, const int* n_child, int* tree_tok,
+                           int batch, int T, int vocab, cudaStream_t st);
+
+// ---- acceptance + compaction (one kernel)
+struct AcceptArgs {
+  const int* tree_tok; const int* amax;
+  const int* parent; const int* depth; const uint64_t* anc;
+  int T, K, batch, n_layers, n_heads, head_dim, max_seq, max_batch, d_model, esize;
+  void* kv_base; const float* h_tree; int h_tree_stride;   // h_tree row = b*h_tree_stride + i
+  float* h_new; int* n_new; int* len; int* root_tok;
+  int* n_acc; int* path; int* out_tok; unsigned int* done_counter; int* status;
+};
+hydra_status accept_compact(const AcceptArgs& a, cudaStream_t st);
+
+// ---- small state kernels
+hydra_status set_chunk(const int* prompt_len, int chunk, int tc, int* pos0, int* n_rows, int batch, cudaStream_t st);
+hydra_status gather_chunk_tokens(const int* tokens, const int* offsets, int chunk, int tc, int* tok_out, int batch,
+                                 cudaStream_t st);
+// for sequences whose last prompt row lies in this chunk: h_new[b][0] = h[b*tc + i], n_new = 1, len = prompt_len
+hydra_status capture_last(const float* h, const int* prompt_len, int chunk, int tc, float* h_new, int kp1, int* n_new,
+                          int* len, int batch, int d, cudaStream_t st);
+// pos0[b] = len[b] - n_new[b]; n_rows[b] = n_new[b]
+hydra_status prefix_rowset(const int* len, const int* n_new, int* pos0, int* n_rows, int batch, cudaStream_t st);
+// hprime[b] = x[b*tc + n_rows[b]-1]
+hydra_status pick_last_row(const float* x, const int* n_rows, int tc, float* hprime, int batch, int d, cudaStream_t st);
+hydra_status apply_plant(int* tree_tok, const int* plant, int count, cudaStream_t st);
+hydra_status copy_i32(int* dst, const int* src, int count, cudaStream_t st);
+
+}  // namespace hydra
