@@ -102,6 +102,14 @@ def silu(x: torch.Tensor) -> torch.Tensor:
     return x / (1.0 + torch.exp(-x))
 
 
+def masked_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, mask: torch.Tensor) -> torch.Tensor:
+    """softmax(q k^T / sqrt(hd) restricted to mask) v per head.  q: [n, H, hd]; k, v: [L, H, hd];
+    mask: [n, L] bool (row i may attend to slot j).  Returns [n, H, hd]."""
+    scores = torch.einsum("nhd,lhd->hnl", q, k) / math.sqrt(q.shape[-1])
+    scores = scores.masked_fill(~mask[None], float("-inf"))
+    return torch.einsum("hnl,lhd->nhd", torch.softmax(scores, dim=-1), v)
+
+
 def topk_desc(logits: torch.Tensor, k: int) -> List[int]:
     """The k most likely tokens in descending order; equal logits ordered by ascending token id."""
     vals = logits.tolist()
@@ -122,16 +130,26 @@ class HydraOracle:
     """State and phases of Hydra decoding for a batch of independent sequences."""
 
     def __init__(self, model, head, parent: Sequence[int], weights: Dict[str, torch.Tensor],
-                 max_seq: int, dtype=torch.float64):
+                 max_seq: int, dtype=torch.float64, cache_weights: bool = False):
         self.m, self.h = model, head
         self.tree = TreeTables(parent, max_depth=head.n_heads)
         self.w = weights
         self.dtype = dtype
         self.max_seq = max_seq
         self.B = 0
+        self._wcache: Dict[str, torch.Tensor] = {}
+        self._cache_weights = cache_weights
+        self.hprime: List[torch.Tensor] = []
 
     def W(self, name: str) -> torch.Tensor:
-        return self.w[name].to(device="cpu", dtype=self.dtype)
+        """Weight `name` widened to the arithmetic dtype (head, embedding and LM-head matrices, which
+        are used many times per step, are kept widened when cache_weights is set; the rest is widened on use)."""
+        if name in self._wcache:
+            return self._wcache[name]
+        t = self.w[name].to(device="cpu", dtype=self.dtype)
+        if self._cache_weights and (name[0] == "H" or name in ("embed", "lm_head")):
+            self._wcache[name] = t
+        return t
 
     # -- one Llama decoder layer over n new rows of one sequence, appending to that layer's cache
     def _layer(self, pre: str, x, pos, allowed_new, kc, vc, cache_len):
@@ -148,10 +166,7 @@ class HydraOracle:
         vc[cache_len:cache_len + n] = v
         L = cache_len + n
         mask = torch.cat([torch.ones(n, cache_len, dtype=torch.bool), allowed_new], dim=1)   # [n, L]
-        scores = torch.einsum("nhd,lhd->hnl", q, kc[:L]) / math.sqrt(hd)
-        scores = scores.masked_fill(~mask[None], float("-inf"))
-        p = torch.softmax(scores, dim=-1)
-        att = torch.einsum("hnl,lhd->nhd", p, vc[:L]).reshape(n, m.d_model)
+        att = masked_attention(q, kc[:L], vc[:L], mask).reshape(n, m.d_model)
         x = x + att @ self.W(pre + "wo").T
         xn = rmsnorm(x, self.W(pre + "ffn_norm"), m.rms_eps)
         gu = xn @ self.W(pre + "w_gate_up").T
@@ -215,8 +230,10 @@ class HydraOracle:
         t = self.tree
         tok = torch.zeros(self.B, t.T, dtype=torch.int64)
         all_logits = [dict() for _ in range(self.B)]
+        self.hprime = []
         for b in range(self.B):
             hp = self._head_input_hidden(b)
+            self.hprime.append(hp)
             tok[b, 0] = self.root_tok[b]
             for d in range(1, t.K + 1):
                 for p in t.level_parents[d - 1]:

@@ -1,0 +1,239 @@
+"""ctypes binding of include/hydra.h.  Names follow the C ABI; arguments are torch CUDA tensors."""
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhydra.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError("libhydra.so is not built: run `python -m paper_2402_05109_b200.build` (needs nvcc)")
+lib = C.CDLL(LIB_PATH)
+
+
+class HydraError(RuntimeError):
+    pass
+
+
+class ModelCfgC(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab")] + \
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("dtype", C.c_int), ("max_batch", C.c_int),
+                ("max_seq", C.c_int)]
+
+
+class HeadCfgC(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("n_heads", "n_mlp_layers", "prefix_attn", "has_bias")]
+
+
+class TreeCfgC(C.Structure):
+    _fields_ = [("n_rows", C.c_int), ("parent", C.POINTER(C.c_int32))]
+
+
+_PP = C.POINTER(C.c_void_p)
+
+
+class WeightsC(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
+                ("attn_norm", _PP), ("wqkv", _PP), ("wo", _PP), ("ffn_norm", _PP), ("w_gate_up", _PP), ("w_down", _PP),
+                ("head_w1", _PP), ("head_b1", _PP), ("head_wr", _PP), ("head_br", _PP)] + \
+               [(n, C.c_void_p) for n in ("pfx_attn_norm", "pfx_wqkv", "pfx_wo", "pfx_ffn_norm", "pfx_w_gate_up",
+                                           "pfx_w_down")]
+
+
+_vp, _i, _sz = C.c_void_p, C.c_int, C.c_size_t
+lib.hydra_workspace_bytes.restype = _sz
+lib.hydra_workspace_bytes.argtypes = [C.POINTER(ModelCfgC), C.POINTER(HeadCfgC), C.POINTER(TreeCfgC)]
+lib.hydra_create.argtypes = [C.POINTER(_vp), C.POINTER(ModelCfgC), C.POINTER(HeadCfgC), C.POINTER(TreeCfgC),
+                             C.POINTER(WeightsC), _vp, _sz]
+lib.hydra_destroy.argtypes = [_vp]
+lib.hydra_prefill.argtypes = [_vp, _i, _vp, C.POINTER(C.c_int32), _vp]
+lib.hydra_draft.argtypes = [_vp, _vp, _vp]
+lib.hydra_verify.argtypes = [_vp, _vp, _vp, _vp, _vp]
+lib.hydra_accept_compact.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.hydra_step.argtypes = [_vp, _vp, _vp, _vp]
+lib.hydra_set_plant.argtypes = [_vp, _vp]
+lib.hydra_get_buffer.argtypes = [_vp, _i, C.POINTER(_vp), C.POINTER(_sz)]
+lib.hydra_poll_status.argtypes = [_vp, _vp]
+lib.hydra_launch_count.restype = C.c_longlong
+lib.hydra_launch_count.argtypes = [_vp]
+lib.hydra_set_gemm_mode.argtypes = [_vp, _i]
+lib.hydra_status_str.restype = C.c_char_p
+lib.hydra_status_str.argtypes = [_i]
+lib.hydra_last_error.restype = C.c_char_p
+lib.hydra_gemm.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]
+lib.hydra_attention_scratch_bytes.restype = _sz
+lib.hydra_attention_scratch_bytes.argtypes = [_i] * 5
+lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 6 + [_vp]
+
+BUF = dict(LEN=0, ROOT_TOK=1, H_TREE=2, H_NEW=3, KV_BASE=4, KV_PREFIX=5, TREE_MASK=6, TREE_TOK=7, AMAX=8,
+           HEAD_LOGITS=9, N_NEW=10, H_PRIME=11, LOGITS=12)
+_BUF_DTYPE = dict(LEN=torch.int32, ROOT_TOK=torch.int32, H_TREE=torch.float32, H_NEW=torch.float32,
+                  TREE_MASK=torch.int64, TREE_TOK=torch.int32, AMAX=torch.int32, HEAD_LOGITS=torch.float32,
+                  N_NEW=torch.int32, H_PRIME=torch.float32, LOGITS=torch.float32)
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise HydraError("%s: %s (%d) %s" % (what, lib.hydra_status_str(code).decode(), code,
+                                             lib.hydra_last_error().decode()))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _ptr_array(tensors: Sequence[Optional[torch.Tensor]]):
+    arr = (C.c_void_p * max(1, len(tensors)))()
+    for i, t in enumerate(tensors):
+        arr[i] = _ptr(t)
+    return arr
+
+
+class Hydra:
+    """One decoding context (hydra_create .. hydra_destroy).  `weights` maps the names of synth.weights
+    (embed, lm_head, final_norm, L{l}.*, P.*, H{i}.*) to CUDA tensors, row-major [out][in]."""
+
+    def __init__(self, model, head, parent: Sequence[int], weights: Dict[str, torch.Tensor], max_batch: int, max_seq: int):
+        self.model, self.head, self.parent = model, head, list(parent)
+        self.T = len(parent)
+        self.K = head.n_heads
+        self.max_batch, self.max_seq = max_batch, max_seq
+        self.dtype = torch.float32 if model.dtype == "fp32" else torch.bfloat16
+        self._w = weights                                   # keep the tensors alive
+        for name, t in weights.items():
+            if not t.is_cuda or not t.is_contiguous() or t.dtype != self.dtype:
+                raise HydraError("weight %s must be a contiguous CUDA tensor of %s" % (name, self.dtype))
+        self._mc = ModelCfgC(model.n_layers, model.d_model, model.n_heads, model.head_dim, model.d_ffn, model.vocab,
+                             model.rms_eps, model.rope_theta, 0 if model.dtype == "fp32" else 1, max_batch, max_seq)
+        self._hc = HeadCfgC(head.n_heads, head.n_mlp_layers, int(head.prefix_attn), int(head.has_bias))
+        self._parent_arr = (C.c_int32 * self.T)(*self.parent)
+        self._tc = TreeCfgC(self.T, self._parent_arr)
+        nbytes = lib.hydra_workspace_bytes(C.byref(self._mc), C.byref(self._hc), C.byref(self._tc))
+        if nbytes == 0:
+            raise HydraError("invalid configuration")
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+        self._ws_off = (-self.workspace.data_ptr()) % 256
+        L = range(model.n_layers)
+        g = weights.get
+        self._arrs = [_ptr_array([g("L%d.%s" % (l, n)) for l in L])
+                      for n in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down")]
+        self._arrs += [_ptr_array([g("H%d.%s" % (i, n)) for i in range(1, head.n_heads + 1)])
+                       for n in ("w1", "b1", "wr", "br")]
+        wc = WeightsC(_ptr(g("embed")), _ptr(g("lm_head")), _ptr(g("final_norm")),
+                      *[C.cast(a, _PP) for a in self._arrs],
+                      *[_ptr(g("P." + n)) for n in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down")])
+        self._ctx = C.c_void_p()
+        _check(lib.hydra_create(C.byref(self._ctx), C.byref(self._mc), C.byref(self._hc), C.byref(self._tc), C.byref(wc),
+                                self.workspace.data_ptr() + self._ws_off, nbytes), "hydra_create")
+        self.batch = 0
+
+    def close(self):
+        if getattr(self, "_ctx", None) is not None and self._ctx.value:
+            lib.hydra_destroy(self._ctx)
+            self._ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- the calls of the C ABI
+    def prefill(self, prompts: List[torch.Tensor]):
+        self.batch = len(prompts)
+        offs = [0]
+        for p in prompts:
+            offs.append(offs[-1] + p.numel())
+        toks = torch.cat([p.to(torch.int32).flatten() for p in prompts]).cuda()
+        arr = (C.c_int32 * len(offs))(*offs)
+        _check(lib.hydra_prefill(self._ctx, self.batch, toks.data_ptr(), arr, _stream()), "hydra_prefill")
+        torch.cuda.current_stream().synchronize()          # toks may be freed after this returns
+
+    def draft(self) -> torch.Tensor:
+        tok = torch.empty(self.batch, self.T, dtype=torch.int32, device="cuda")
+        _check(lib.hydra_draft(self._ctx, tok.data_ptr(), _stream()), "hydra_draft")
+        return tok
+
+    def verify(self, tree_tok: torch.Tensor, want_logits: bool = False):
+        assert tree_tok.dtype == torch.int32 and tree_tok.is_cuda and tree_tok.is_contiguous()
+        amax = torch.empty(self.batch, self.T, dtype=torch.int32, device="cuda")
+        logits = torch.empty(self.batch, self.T, self.model.vocab, dtype=torch.float32, device="cuda") if want_logits else None
+        _check(lib.hydra_verify(self._ctx, tree_tok.data_ptr(), amax.data_ptr(), _ptr(logits), _stream()), "hydra_verify")
+        return (amax, logits) if want_logits else amax
+
+    def accept_compact(self, tree_tok: torch.Tensor, amax: torch.Tensor):
+        n_acc = torch.empty(self.batch, dtype=torch.int32, device="cuda")
+        path = torch.empty(self.batch, self.K + 1, dtype=torch.int32, device="cuda")
+        out = torch.empty(self.batch, self.K + 1, dtype=torch.int32, device="cuda")
+        _check(lib.hydra_accept_compact(self._ctx, tree_tok.data_ptr(), amax.data_ptr(), n_acc.data_ptr(), path.data_ptr(),
+                                        out.data_ptr(), _stream()), "hydra_accept_compact")
+        return n_acc, path, out
+
+    def step(self, n_acc: Optional[torch.Tensor] = None, out_tok: Optional[torch.Tensor] = None):
+        if n_acc is None:
+            n_acc = torch.empty(self.batch, dtype=torch.int32, device="cuda")
+        if out_tok is None:
+            out_tok = torch.empty(self.batch, self.K + 1, dtype=torch.int32, device="cuda")
+        _check(lib.hydra_step(self._ctx, n_acc.data_ptr(), out_tok.data_ptr(), _stream()), "hydra_step")
+        return n_acc, out_tok
+
+    def set_plant(self, plant: Optional[torch.Tensor]):
+        self._plant = plant
+        _check(lib.hydra_set_plant(self._ctx, _ptr(plant)), "hydra_set_plant")
+
+    def set_gemm_mode(self, mode: int):
+        _check(lib.hydra_set_gemm_mode(self._ctx, mode), "hydra_set_gemm_mode")
+
+    def poll_status(self):
+        _check(lib.hydra_poll_status(self._ctx, _stream()), "hydra_poll_status")
+
+    def launch_count(self) -> int:
+        return int(lib.hydra_launch_count(self._ctx))
+
+    def get_buffer(self, name: str) -> torch.Tensor:
+        """A tensor view of a library buffer (flat; KV buffers in the cache dtype)."""
+        p, n = C.c_void_p(), C.c_size_t()
+        _check(lib.hydra_get_buffer(self._ctx, BUF[name], C.byref(p), C.byref(n)), "hydra_get_buffer")
+        off = p.value - self.workspace.data_ptr()
+        return self.workspace[off:off + n.value].view(_BUF_DTYPE.get(name, self.dtype))
+
+    def kv_base(self) -> torch.Tensor:
+        m = self.model
+        return self.get_buffer("KV_BASE").view(m.n_layers, 2, self.max_batch, m.n_heads, self.max_seq, m.head_dim)
+
+    def kv_prefix(self) -> torch.Tensor:
+        m = self.model
+        return self.get_buffer("KV_PREFIX").view(2, self.max_batch, m.n_heads, self.max_seq, m.head_dim)
+
+
+# ---- single-kernel entry points (kernel-level parity tests)
+def gemm(x: torch.Tensor, w: torch.Tensor, splits: int = 1, mode: int = 0) -> torch.Tensor:
+    """out[m][n] = sum_k x[m][k] w[n][k] in float; x, w both float32 or both bfloat16 CUDA tensors."""
+    m, k = x.shape
+    n = w.shape[0]
+    dtype = 0 if x.dtype == torch.float32 else 1
+    out = torch.empty(m, n, dtype=torch.float32, device="cuda")
+    part = torch.empty(splits, m, n, dtype=torch.float32, device="cuda") if splits > 1 else None
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib.hydra_gemm(x.data_ptr(), w.data_ptr(), out.data_ptr(), _ptr(part), m, n, k, dtype, splits, mode,
+                          status.data_ptr(), _stream()), "hydra_gemm")
+    word = int(status.item())
+    if word:
+        raise HydraError("hydra_gemm device status word %d" % word)
+    return out
+
+
+def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int) -> torch.Tensor:
+    batch, n_heads, max_seq, head_dim = k_cache.shape
+    dtype = 0 if k_cache.dtype == torch.float32 else 1
+    out = torch.empty(batch * tc, n_heads * head_dim, dtype=k_cache.dtype, device="cuda")
+    scratch = torch.empty(lib.hydra_attention_scratch_bytes(batch, tc, n_heads, head_dim, max_seq), dtype=torch.uint8,
+                          device="cuda")
+    _check(lib.hydra_tree_attention(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), pos0.data_ptr(), _ptr(n_rows),
+                                    mask.data_ptr(), out.data_ptr(), scratch.data_ptr(), batch, tc, n_heads, head_dim,
+                                    max_seq, dtype, _stream()), "hydra_tree_attention")
+    return out

@@ -1,0 +1,599 @@
+// libhydra: context, workspace carving, host orchestration of the decode step and the C ABI.
+#include "launch.h"
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+namespace hydra {
+
+thread_local long long* g_launch_counter = nullptr;
+static thread_local char g_err[512] = "";
+void set_last_error(const char* what, cudaError_t e) {
+  snprintf(g_err, sizeof(g_err), "%s: %s", what, cudaGetErrorString(e));
+}
+
+namespace {
+
+constexpr int CHUNK = 64;          // rows per sequence of one prefill pass (and the row capacity of a forward call)
+
+struct LayerW { const void *attn_norm, *wqkv, *wo, *ffn_norm, *w_gate_up, *w_down; };
+
+struct Bump {                      // 256-byte aligned bump allocator; base == nullptr only measures
+  char* base; size_t off;
+  template <typename T> T* take(size_t count) {
+    off = (off + 255) & ~(size_t)255;
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+int tile_rows(int m) { return m <= 16 ? 16 : m <= 32 ? 32 : m <= 64 ? 64 : m <= 128 ? 128 : 256; }
+int pad_rows(int m) { int t = tile_rows(m); return (m + t - 1) / t * t; }
+
+// Split-K factor: spread a GEMM with few n-tiles over the SMs.  Cost model: waves x (k-blocks per CTA +
+// a fixed per-CTA ramp), in units of one 64-wide k-block.
+int choose_splits(int m, int n, int k) {
+  int mt = tile_rows(m);
+  int tiles = (n / 128) * ((m + mt - 1) / mt);
+  int kb = k / 64;
+  int best = 1; double best_cost = 1e30;
+  for (int s = 1; s <= 16 && s * 2 <= kb; ++s) {
+    double waves = (double)((tiles * s + 147) / 148);
+    double cost = waves * ((kb + s - 1) / s + 6);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
+enum State { ST_CREATED = 0, ST_READY = 1, ST_DRAFTED = 2, ST_VERIFIED = 3 };
+
+}  // namespace
+}  // namespace hydra
+
+using namespace hydra;
+
+struct hydra_ctx {
+  hydra_model_cfg m; hydra_head_cfg h;
+  int T, Ktree;                                  // tree rows, tree depth
+  std::vector<int> parent, depth, first_child, n_child, path_tab;
+  std::vector<uint64_t> anc;
+  std::vector<std::vector<int>> level_parents;   // [Ktree]
+  std::vector<LayerW> layers; LayerW pfx;
+  std::vector<const void*> head_w1, head_b1, head_wr, head_br;
+  const void *embed, *lm_head, *final_norm;
+  int esize;                                     // bytes per weight / KV element
+  int R;                                         // row capacity of a forward call (padded)
+  int RH;                                        // row capacity of the head buffers (padded)
+  int maxP;
+  // device buffers
+  int *d_parent, *d_depth, *d_first_child, *d_n_child, *d_path_tab, *d_chain_depth;
+  uint64_t *d_anc, *d_chain_mask;
+  std::vector<int*> d_level_parents;
+  int *d_len, *d_n_new, *d_root_tok, *d_status, *d_pos0, *d_nrows, *d_prompt_len, *d_offsets, *d_tok, *d_tree_tok, *d_amax;
+  unsigned int* d_done;
+  char *kv_base, *kv_pfx;
+  float *x, *q, *part, *h_tree, *logits, *h_new, *hprime, *y, *head_logits;
+  float2* rope;
+  void *xn, *attn_out, *act, *z, *yb, *att_scratch;
+  size_t part_floats;
+  // host state
+  int batch, state, gemm_mode;
+  std::vector<int> len_ub;
+  const int* plant;
+  long long launches;
+};
+
+namespace {
+
+size_t kv_layer_elems(const hydra_model_cfg& m) { return (size_t)m.max_batch * m.n_heads * m.max_seq * m.head_dim; }
+
+struct TreeHost {
+  int T = 0, K = 0, maxP = 1;
+  std::vector<int> parent, depth, first_child, n_child, path_tab;
+  std::vector<uint64_t> anc;
+  std::vector<std::vector<int>> level_parents;
+};
+
+// Tables of the static tree: depth, ancestor-or-self bitmask, children ranges, root paths, per-level parents.
+bool build_tree(const hydra_tree_cfg* t, int max_depth, TreeHost& o) {
+  if (!t || !t->parent || t->n_rows < 1 || t->n_rows > 64 || t->parent[0] != -1) return false;
+  int T = t->n_rows;
+  o.T = T; o.parent.assign(t->parent, t->parent + T);
+  o.depth.assign(T, 0); o.anc.assign(T, 0); o.first_child.assign(T, 0); o.n_child.assign(T, 0);
+  o.anc[0] = 1ull;
+  for (int i = 1; i < T; ++i) {
+    int p = o.parent[i];
+    if (p < 0 || p >= i) return false;
+    o.depth[i] = o.depth[p] + 1;
+    o.anc[i] = o.anc[p] | (1ull << i);
+    if (o.n_child[p] == 0) o.first_child[p] = i;
+    else if (o.first_child[p] + o.n_child[p] != i) return false;     // children of a parent must be adjacent rows
+    o.n_child[p]++;
+    if (o.depth[i] < o.depth[i - 1]) return false;                   // rows ordered by depth
+    if (o.depth[i] == o.depth[i - 1] && i > 1 && p < o.parent[i - 1]) return false;   // ... then by rank path
+  }
+  o.K = *std::max_element(o.depth.begin(), o.depth.end());
+  if (o.K > max_depth) return false;
+  int kp1 = max_depth + 1;
+  o.path_tab.assign((size_t)T * kp1, -1);
+  for (int i = 0; i < T; ++i) { int node = i; for (int k = o.depth[i]; k >= 0; --k) { o.path_tab[i * kp1 + k] = node; node = o.parent[node]; } }
+  o.level_parents.assign(o.K, {});
+  for (int d = 1; d <= o.K; ++d)
+    for (int i = 0; i < T; ++i) if (o.depth[i] == d - 1 && o.n_child[i] > 0) o.level_parents[d - 1].push_back(i);
+  o.maxP = 1;
+  for (auto& lv : o.level_parents) o.maxP = std::max(o.maxP, (int)lv.size());
+  return true;
+}
+
+bool valid_cfg(const hydra_model_cfg* m, const hydra_head_cfg* h) {
+  if (!m || !h) return false;
+  if (m->n_layers < 1 || m->d_model < 1 || m->n_heads < 1 || m->d_ffn < 1 || m->vocab < 1 || m->max_batch < 1 || m->max_seq < 1)
+    return false;
+  if (m->n_heads * m->head_dim != m->d_model) return false;
+  if (m->dtype != 0 && m->dtype != 1) return false;
+  if (h->n_heads < 0 || h->n_mlp_layers < 1) return false;
+  return true;
+}
+hydra_status supported_cfg(const hydra_model_cfg* m) {
+  if (m->head_dim != 64 && m->head_dim != 128) return HYDRA_ERR_UNSUPPORTED;
+  if (m->d_model % 4 || m->d_ffn % 4) return HYDRA_ERR_UNSUPPORTED;
+  if (m->max_batch > 64) return HYDRA_ERR_UNSUPPORTED;
+  if (m->dtype == 1 && (m->d_model % 128 || m->d_ffn % 64 || m->vocab % 128)) return HYDRA_ERR_UNSUPPORTED;
+  return HYDRA_OK;
+}
+
+// Lays every library buffer out in the workspace (or just measures it when ws == nullptr).
+size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, const TreeHost& t, char* ws) {
+  Bump b{ws, 0};
+  const int es = m.dtype == 0 ? 4 : 2;
+  const int d = m.d_model, f = m.d_ffn, V = m.vocab, K = h.n_heads, T = t.T;
+  const int R = pad_rows(m.max_batch * CHUNK);
+  const int RH = pad_rows(m.max_batch * t.maxP);
+  // largest split-K partial buffer over every GEMM shape and row count the library issues
+  size_t part_floats = 0;
+  {
+    const int shapes[][2] = {{3 * d, d}, {d, d}, {2 * f, d}, {d, f}};
+    const int row_counts[] = {m.max_batch * CHUNK, m.max_batch * T, m.max_batch * (K + 1)};
+    for (auto& s : shapes)
+      for (int rows : row_counts)
+        for (int bb = 1; bb <= m.max_batch; ++bb) {
+          int mm = rows / m.max_batch * bb;
+          int sp = m.dtype == 1 ? choose_splits(mm, s[0], s[1]) : 1;
+          part_floats = std::max(part_floats, (size_t)sp * mm * s[0]);
+        }
+    for (int i = 1; i <= K; ++i)
+      for (int mm = 1; mm <= m.max_batch * t.maxP; ++mm) {
+        int sp1 = m.dtype == 1 ? choose_splits(mm, d, (i + 1) * d) : 1, sp2 = m.dtype == 1 ? choose_splits(mm, d, d) : 1;
+        part_floats = std::max(part_floats, (size_t)std::max(sp1, sp2) * mm * d);
+      }
+  }
+  auto* parent = b.take<int>(T); auto* depth = b.take<int>(T); auto* fc = b.take<int>(T); auto* nc = b.take<int>(T);
+  auto* path_tab = b.take<int>((size_t)T * (K + 1)); auto* chain_depth = b.take<int>(CHUNK);
+  auto* anc = b.take<uint64_t>(T); auto* chain_mask = b.take<uint64_t>(CHUNK);
+  std::vector<int*> lvl;
+  for (auto& lv : t.level_parents) lvl.push_back(b.take<int>(lv.size()));
+  auto* len = b.take<int>(m.max_batch); auto* n_new = b.take<int>(m.max_batch); auto* root = b.take<int>(m.max_batch);
+  auto* status = b.take<int>(1); auto* pos0 = b.take<int>(m.max_batch); auto* nrows = b.take<int>(m.max_batch);
+  auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
+  auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
+  auto* done = b.take<unsigned int>(m.max_batch);
+  auto* kvb = b.take<char>((size_t)m.n_layers * 2 * kv_layer_elems(m) * es);
+  auto* kvp = b.take<char>(h.prefix_attn ? (size_t)2 * kv_layer_elems(m) * es : 0);
+  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<float>((size_t)R * d);
+  auto* part = b.take<float>(part_floats);
+  auto* h_tree = b.take<float>((size_t)R * d);
+  auto* logits = b.take<float>((size_t)pad_rows(m.max_batch * T) * V);
+  auto* h_new = b.take<float>((size_t)pad_rows(m.max_batch * (K + 1)) * d);
+  auto* hprime = b.take<float>((size_t)m.max_batch * d);
+  auto* y = b.take<float>((size_t)RH * d); auto* head_logits = b.take<float>((size_t)RH * V);
+  auto* rope = b.take<float2>((size_t)R * (m.head_dim / 2));
+  auto* xn = b.take<char>((size_t)R * d * es); auto* attn_out = b.take<char>((size_t)R * d * es);
+  auto* act = b.take<char>((size_t)R * f * es);
+  auto* z = b.take<char>((size_t)RH * (K + 1) * d * es); auto* yb = b.take<char>((size_t)RH * d * es);
+  auto* att = b.take<char>(attention_scratch_bytes(m.max_batch, CHUNK, m.n_heads, m.head_dim, m.max_seq));
+  if (c) {
+    c->R = R; c->RH = RH; c->part_floats = part_floats; c->esize = es;
+    c->d_parent = parent; c->d_depth = depth; c->d_first_child = fc; c->d_n_child = nc; c->d_path_tab = path_tab;
+    c->d_chain_depth = chain_depth; c->d_anc = anc; c->d_chain_mask = chain_mask; c->d_level_parents = lvl;
+    c->d_len = len; c->d_n_new = n_new; c->d_root_tok = root; c->d_status = status; c->d_pos0 = pos0; c->d_nrows = nrows;
+    c->d_prompt_len = plen; c->d_offsets = offs; c->d_tok = tok; c->d_tree_tok = tree_tok; c->d_amax = amax; c->d_done = done;
+    c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits;
+    c->h_new = h_new; c->hprime = hprime; c->y = y; c->head_logits = head_logits; c->rope = rope; c->xn = xn;
+    c->attn_out = attn_out; c->act = act; c->z = z; c->yb = yb; c->att_scratch = att;
+  }
+  return (b.off + 255) & ~(size_t)255;
+}
+
+// out = x @ w^T into c->part (split-K partial sums) or, when direct_out is given, straight into it (no split).
+hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void* w, int m, int n, int k, float* direct_out,
+                      int* splits, size_t* stride, cudaStream_t st) {
+  float* out = direct_out ? direct_out : c->part;
+  *stride = (size_t)m * n;
+  if (c->m.dtype == 1 && c->gemm_mode == 0) {
+    int sp = direct_out ? 1 : choose_splits(m, n, k);
+    if ((size_t)sp * m * n > c->part_floats && !direct_out) sp = 1;
+    *splits = sp;
+    return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, out, *stride, m, n, k, sp, c->d_status, st);
+  }
+  *splits = 1;
+  return gemm_simt(x, w, out, m, n, k, c->m.dtype, st);
+}
+
+// One decoder layer over the rows of `rs`.  Expects the residual rows in c->x and their normed copy in c->xn.
+// Leaves the updated residual in c->x; when next_gain is given also xn = rmsnorm(x)*next_gain (and hn in float).
+hydra_status run_layer(hydra_ctx* c, const LayerW& w, char* kc, char* vc, const RowSet& rs, int len_upper,
+                       const void* next_gain, float* hn, cudaStream_t st) {
+  const hydra_model_cfg& m = c->m;
+  const int rows = rs.batch * rs.tc, d = m.d_model, f = m.d_ffn, dt = m.dtype;
+  int sp; size_t stride;
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.wqkv, rows, 3 * d, d, nullptr, &sp, &stride, st));
+  HYDRA_TRY(qkv_rope_store(c->part, stride, sp, c->rope, c->q, kc, vc, rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
+  HYDRA_TRY(tree_attention(c->q, kc, vc, rs, c->attn_out, c->att_scratch, m.n_heads, m.head_dim, m.max_seq, len_upper, dt, st));
+  HYDRA_TRY(run_gemm(c, c->attn_out, c->R, w.wo, rows, d, d, nullptr, &sp, &stride, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, c->part, stride, sp, c->x, w.ffn_norm, c->xn, nullptr, rows, d, m.rms_eps, dt, st));
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, nullptr, &sp, &stride, st));
+  HYDRA_TRY(silu_mul(c->part, stride, sp, c->act, rows, f, dt, st));
+  HYDRA_TRY(run_gemm(c, c->act, c->R, w.w_down, rows, d, f, nullptr, &sp, &stride, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, c->part, stride, sp, c->x, next_gain, next_gain ? c->xn : nullptr, hn, rows, d, m.rms_eps, dt, st));
+  return HYDRA_OK;
+}
+
+// Base model over the rows of `rs` whose tokens are tok[rows]: leaves post-final-norm hidden rows in c->h_tree
+// (float) and c->xn (operand type).
+hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_upper, cudaStream_t st) {
+  const hydra_model_cfg& m = c->m;
+  const int rows = rs.batch * rs.tc;
+  const size_t kvl = kv_layer_elems(m) * c->esize;
+  HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
+  HYDRA_TRY(embed_rows(c->embed, tok, c->x, rows, m.d_model, m.vocab, m.dtype, c->d_status, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, nullptr, 0, 0, c->x, c->layers[0].attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
+  for (int l = 0; l < m.n_layers; ++l) {
+    bool last = l + 1 == m.n_layers;
+    HYDRA_TRY(run_layer(c, c->layers[l], c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs, len_upper,
+                        last ? c->final_norm : c->layers[l + 1].attn_norm, last ? c->h_tree : nullptr, st));
+  }
+  return HYDRA_OK;
+}
+
+// Prefix-attention layer over rows whose input (post-final-norm hidden) is `src` laid out like rs.
+hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int len_upper, cudaStream_t st) {
+  const hydra_model_cfg& m = c->m;
+  const int rows = rs.batch * rs.tc;
+  const size_t kvl = kv_layer_elems(m) * c->esize;
+  HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
+  HYDRA_TRY(residual_rmsnorm(src, nullptr, 0, 0, c->x, c->pfx.attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
+  return run_layer(c, c->pfx, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, nullptr, nullptr, st);
+}
+
+int max_len_ub(const hydra_ctx* c) { int v = 0; for (int b = 0; b < c->batch; ++b) v = std::max(v, c->len_ub[b]); return v; }
+
+hydra_status do_draft(hydra_ctx* c, int* tree_tok, cudaStream_t st) {
+  const hydra_model_cfg& m = c->m;
+  const int B = c->batch, K = c->h.n_heads, d = m.d_model, dt = m.dtype;
+  if (c->h.prefix_attn) {
+    HYDRA_TRY(prefix_rowset(c->d_len, c->d_n_new, c->d_pos0, c->d_nrows, B, st));
+    RowSet rs{B, K + 1, c->d_nrows, c->d_pos0, c->d_chain_depth, c->d_chain_mask};
+    HYDRA_TRY(run_prefix(c, c->h_new, rs, max_len_ub(c), st));
+    HYDRA_TRY(pick_last_row(c->x, c->d_nrows, K + 1, c->hprime, B, d, st));
+  } else {
+    HYDRA_TRY(pick_last_row(c->h_new, c->d_n_new, K + 1, c->hprime, B, d, st));
+  }
+  if (c->Ktree == 0) return copy_i32(tree_tok, c->d_root_tok, B, st);      // root-only tree (T == 1)
+  for (int lvl = 1; lvl <= c->Ktree; ++lvl) {
+    const int P = (int)c->level_parents[lvl - 1].size();
+    const int rows = B * P;
+    LevelDesc lv{lvl, P, c->d_level_parents[lvl - 1]};
+    HYDRA_TRY(head_gather(c->hprime, c->embed, c->d_root_tok, tree_tok, c->d_path_tab, lv, c->z, B, c->T, K + 1, d, m.vocab, dt, c->d_status, st));
+    int sp; size_t stride;
+    HYDRA_TRY(run_gemm(c, c->z, c->RH, c->head_w1[lvl - 1], rows, d, (lvl + 1) * d, nullptr, &sp, &stride, st));
+    HYDRA_TRY(head_act(c->hprime, 1, P, c->part, stride, sp, c->h.has_bias ? c->head_b1[lvl - 1] : nullptr, c->y, c->yb, rows, d, dt, st));
+    for (int l = 0; l + 1 < c->h.n_mlp_layers; ++l) {
+      const char* wr = (const char*)c->head_wr[lvl - 1] + (size_t)l * d * d * c->esize;
+      const char* br = c->h.has_bias ? (const char*)c->head_br[lvl - 1] + (size_t)l * d * c->esize : nullptr;
+      HYDRA_TRY(run_gemm(c, c->yb, c->RH, wr, rows, d, d, nullptr, &sp, &stride, st));
+      HYDRA_TRY(head_act(c->y, 0, P, c->part, stride, sp, br, c->y, c->yb, rows, d, dt, st));
+    }
+    HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, rows, m.vocab, d, c->head_logits, &sp, &stride, st));
+    HYDRA_TRY(topk_children(c->head_logits, lv, c->d_first_child, c->d_n_child, tree_tok, B, c->T, m.vocab, st));
+  }
+  return HYDRA_OK;
+}
+
+hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logits, cudaStream_t st) {
+  const hydra_model_cfg& m = c->m;
+  const int rows = c->batch * c->T;
+  RowSet rs{c->batch, c->T, nullptr, c->d_len, c->d_depth, c->d_anc};
+  HYDRA_TRY(run_base(c, tree_tok, rs, max_len_ub(c) + c->T, st));
+  int sp; size_t stride;
+  float* lg = logits ? logits : c->logits;
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, lg, &sp, &stride, st));
+  return argmax_rows(lg, amax, rows, m.vocab, st);
+}
+
+hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* n_acc, int* path, int* out_tok, cudaStream_t st) {
+  const hydra_model_cfg& m = c->m;
+  AcceptArgs a{};
+  a.tree_tok = tree_tok; a.amax = amax; a.parent = c->d_parent; a.depth = c->d_depth; a.anc = c->d_anc;
+  a.T = c->T; a.K = c->h.n_heads; a.batch = c->batch; a.n_layers = m.n_layers; a.n_heads = m.n_heads; a.head_dim = m.head_dim;
+  a.max_seq = m.max_seq; a.max_batch = m.max_batch; a.d_model = m.d_model; a.esize = c->esize;
+  a.kv_base = c->kv_base; a.h_tree = c->h_tree; a.h_tree_stride = c->T;
+  a.h_new = c->h_new; a.n_new = c->d_n_new; a.len = c->d_len; a.root_tok = c->d_root_tok;
+  a.n_acc = n_acc; a.path = path; a.out_tok = out_tok; a.done_counter = c->d_done; a.status = c->d_status;
+  HYDRA_TRY(accept_compact(a, st));
+  for (int b = 0; b < c->batch; ++b) c->len_ub[b] += c->Ktree + 1;
+  return HYDRA_OK;
+}
+
+bool capacity_ok(const hydra_ctx* c) {
+  for (int b = 0; b < c->batch; ++b) if (c->len_ub[b] + c->T > c->m.max_seq) return false;
+  return true;
+}
+
+struct CounterScope {
+  explicit CounterScope(hydra_ctx* c) { g_launch_counter = c ? &c->launches : nullptr; }
+  ~CounterScope() { g_launch_counter = nullptr; }
+};
+
+}  // namespace
+
+extern "C" {
+
+size_t hydra_workspace_bytes(const hydra_model_cfg* m, const hydra_head_cfg* h, const hydra_tree_cfg* t) {
+  TreeHost th;
+  if (!valid_cfg(m, h) || !build_tree(t, h->n_heads, th)) return 0;
+  return carve(nullptr, *m, *h, th, nullptr);
+}
+
+hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra_head_cfg* h, const hydra_tree_cfg* t,
+                          const hydra_weights* w, void* ws, size_t ws_bytes) {
+  if (!out || !w || !ws) return HYDRA_ERR_INVALID;
+  *out = nullptr;
+  TreeHost th;
+  if (!valid_cfg(m, h) || !build_tree(t, h->n_heads, th)) return HYDRA_ERR_INVALID;
+  hydra_status sup = supported_cfg(m);
+  if (sup != HYDRA_OK) return sup;
+  if ((uintptr_t)ws & 255) return HYDRA_ERR_INVALID;
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wqkv || !w->wo || !w->ffn_norm || !w->w_gate_up || !w->w_down)
+    return HYDRA_ERR_INVALID;
+  if (th.K > 0 && (!w->head_w1 || (h->has_bias && !w->head_b1))) return HYDRA_ERR_INVALID;
+  if (th.K > 0 && h->n_mlp_layers > 1 && (!w->head_wr || (h->has_bias && !w->head_br))) return HYDRA_ERR_INVALID;
+  if (h->prefix_attn && (!w->pfx_attn_norm || !w->pfx_wqkv || !w->pfx_wo || !w->pfx_ffn_norm || !w->pfx_w_gate_up || !w->pfx_w_down))
+    return HYDRA_ERR_INVALID;
+  size_t need = carve(nullptr, *m, *h, th, nullptr);
+  if (ws_bytes < need) return HYDRA_ERR_CAPACITY;
+  if (m->dtype == 1 && !gemm_tc_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
+  hydra_ctx* c = new (std::nothrow) hydra_ctx();
+  if (!c) return HYDRA_ERR_INVALID;
+  c->m = *m; c->h = *h; c->T = th.T; c->Ktree = th.K; c->maxP = th.maxP;
+  c->parent = th.parent; c->depth = th.depth; c->first_child = th.first_child; c->n_child = th.n_child;
+  c->path_tab = th.path_tab; c->anc = th.anc; c->level_parents = th.level_parents;
+  for (int l = 0; l < m->n_layers; ++l) {
+    LayerW lw{w->attn_norm[l], w->wqkv[l], w->wo[l], w->ffn_norm[l], w->w_gate_up[l], w->w_down[l]};
+    if (!lw.attn_norm || !lw.wqkv || !lw.wo || !lw.ffn_norm || !lw.w_gate_up || !lw.w_down) { delete c; return HYDRA_ERR_INVALID; }
+    c->layers.push_back(lw);
+  }
+  c->pfx = LayerW{w->pfx_attn_norm, w->pfx_wqkv, w->pfx_wo, w->pfx_ffn_norm, w->pfx_w_gate_up, w->pfx_w_down};
+  for (int i = 0; i < th.K; ++i) {
+    c->head_w1.push_back(w->head_w1[i]);
+    c->head_b1.push_back(h->has_bias ? w->head_b1[i] : nullptr);
+    c->head_wr.push_back(h->n_mlp_layers > 1 ? w->head_wr[i] : nullptr);
+    c->head_br.push_back(h->n_mlp_layers > 1 && h->has_bias ? w->head_br[i] : nullptr);
+    if (!c->head_w1[i] || (h->n_mlp_layers > 1 && !c->head_wr[i])) { delete c; return HYDRA_ERR_INVALID; }
+  }
+  c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
+  carve(c, *m, *h, th, (char*)ws);
+  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->plant = nullptr; c->launches = 0;
+  c->len_ub.assign(m->max_batch, 0);
+  // clear the workspace, upload the static tables
+  auto fail = [&](cudaError_t e, const char* what) { set_last_error(what, e); delete c; return HYDRA_ERR_CUDA; };
+  cudaError_t e;
+  if ((e = cudaMemset(ws, 0, need)) != cudaSuccess) return fail(e, "cudaMemset(workspace)");
+  const int T = th.T, K = h->n_heads;
+  std::vector<int> chain_depth(CHUNK); std::vector<uint64_t> chain_mask(CHUNK);
+  for (int i = 0; i < CHUNK; ++i) { chain_depth[i] = i; chain_mask[i] = i == 63 ? ~0ull : ((1ull << (i + 1)) - 1); }
+#define UP(dst, src, bytes) if ((bytes) && (e = cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice)) != cudaSuccess) return fail(e, "cudaMemcpy(tables)")
+  UP(c->d_parent, th.parent.data(), T * sizeof(int)); UP(c->d_depth, th.depth.data(), T * sizeof(int));
+  UP(c->d_first_child, th.first_child.data(), T * sizeof(int)); UP(c->d_n_child, th.n_child.data(), T * sizeof(int));
+  UP(c->d_path_tab, th.path_tab.data(), (size_t)T * (K + 1) * sizeof(int));
+  UP(c->d_chain_depth, chain_depth.data(), CHUNK * sizeof(int)); UP(c->d_chain_mask, chain_mask.data(), CHUNK * sizeof(uint64_t));
+  UP(c->d_anc, th.anc.data(), T * sizeof(uint64_t));
+  for (size_t i = 0; i < th.level_parents.size(); ++i) UP(c->d_level_parents[i], th.level_parents[i].data(), th.level_parents[i].size() * sizeof(int));
+#undef UP
+  if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "cudaDeviceSynchronize");
+  *out = c;
+  return HYDRA_OK;
+}
+
+hydra_status hydra_destroy(hydra_ctx* c) {
+  if (!c) return HYDRA_ERR_INVALID;
+  cudaError_t e = cudaDeviceSynchronize();
+  delete c;
+  if (e != cudaSuccess) { set_last_error("cudaDeviceSynchronize", e); return HYDRA_ERR_CUDA; }
+  return HYDRA_OK;
+}
+
+hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const int32_t* offs, void* stream) {
+  if (!c || !tokens || !offs || batch < 1 || batch > c->m.max_batch) return HYDRA_ERR_INVALID;
+  CounterScope cs(c);
+  cudaStream_t st = (cudaStream_t)stream;
+  const hydra_model_cfg& m = c->m;
+  std::vector<int> plen(batch);
+  int maxlen = 0;
+  for (int b = 0; b < batch; ++b) {
+    plen[b] = offs[b + 1] - offs[b];
+    if (plen[b] < 1) return HYDRA_ERR_INVALID;
+    if (plen[b] + c->T > m.max_seq) return HYDRA_ERR_CAPACITY;
+    maxlen = std::max(maxlen, plen[b]);
+  }
+  c->batch = batch;
+  HYDRA_CUDA(cudaMemcpyAsync(c->d_prompt_len, plen.data(), batch * sizeof(int), cudaMemcpyHostToDevice, st));
+  HYDRA_CUDA(cudaMemcpyAsync(c->d_offsets, offs, (batch + 1) * sizeof(int), cudaMemcpyHostToDevice, st));
+  HYDRA_CUDA(cudaStreamSynchronize(st));           // the host vectors above go out of scope
+  const int nchunks = (maxlen + CHUNK - 1) / CHUNK;
+  RowSet rs{batch, CHUNK, c->d_nrows, c->d_pos0, c->d_chain_depth, c->d_chain_mask};
+  for (int ch = 0; ch < nchunks; ++ch) {
+    HYDRA_TRY(set_chunk(c->d_prompt_len, ch, CHUNK, c->d_pos0, c->d_nrows, batch, st));
+    HYDRA_TRY(gather_chunk_tokens(tokens, c->d_offsets, ch, CHUNK, c->d_tok, batch, st));
+    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * CHUNK, st));
+    HYDRA_TRY(capture_last(c->h_tree, c->d_prompt_len, ch, CHUNK, c->h_new, c->h.n_heads + 1, c->d_n_new, c->d_len, batch, m.d_model, st));
+    if (c->h.prefix_attn) HYDRA_TRY(run_prefix(c, c->h_tree, rs, (ch + 1) * CHUNK, st));
+  }
+  // root token = argmax of the logits of the last prompt row
+  HYDRA_TRY(pick_last_row(c->h_new, c->d_n_new, c->h.n_heads + 1, c->hprime, batch, m.d_model, st));
+  HYDRA_TRY(cast_rows(c->hprime, c->yb, (size_t)batch * m.d_model, m.dtype, st));
+  int sp; size_t stride;
+  HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, batch, m.vocab, m.d_model, c->head_logits, &sp, &stride, st));
+  HYDRA_TRY(argmax_rows(c->head_logits, c->d_root_tok, batch, m.vocab, st));
+  for (int b = 0; b < batch; ++b) c->len_ub[b] = plen[b];
+  c->state = ST_READY;
+  return HYDRA_OK;
+}
+
+hydra_status hydra_draft(hydra_ctx* c, int32_t* tree_tok, void* stream) {
+  if (!c || !tree_tok) return HYDRA_ERR_INVALID;
+  if (c->state != ST_READY && c->state != ST_DRAFTED) return HYDRA_ERR_STATE;
+  if (!capacity_ok(c)) return HYDRA_ERR_CAPACITY;
+  CounterScope cs(c);
+  HYDRA_TRY(do_draft(c, tree_tok, (cudaStream_t)stream));
+  c->state = ST_DRAFTED;
+  return HYDRA_OK;
+}
+
+hydra_status hydra_verify(hydra_ctx* c, const int32_t* tree_tok, int32_t* amax, float* logits, void* stream) {
+  if (!c || !tree_tok || !amax) return HYDRA_ERR_INVALID;
+  if (c->state != ST_READY && c->state != ST_DRAFTED && c->state != ST_VERIFIED) return HYDRA_ERR_STATE;
+  if (!capacity_ok(c)) return HYDRA_ERR_CAPACITY;
+  CounterScope cs(c);
+  HYDRA_TRY(do_verify(c, tree_tok, amax, logits, (cudaStream_t)stream));
+  c->state = ST_VERIFIED;
+  return HYDRA_OK;
+}
+
+hydra_status hydra_accept_compact(hydra_ctx* c, const int32_t* tree_tok, const int32_t* amax, int32_t* n_acc, int32_t* path,
+                                  int32_t* out_tok, void* stream) {
+  if (!c || !tree_tok || !amax) return HYDRA_ERR_INVALID;
+  if (c->state != ST_VERIFIED) return HYDRA_ERR_STATE;
+  CounterScope cs(c);
+  HYDRA_TRY(do_accept(c, tree_tok, amax, n_acc, path, out_tok, (cudaStream_t)stream));
+  c->state = ST_READY;
+  return HYDRA_OK;
+}
+
+hydra_status hydra_step(hydra_ctx* c, int32_t* n_acc, int32_t* out_tok, void* stream) {
+  if (!c) return HYDRA_ERR_INVALID;
+  if (c->state != ST_READY) return HYDRA_ERR_STATE;
+  if (!capacity_ok(c)) return HYDRA_ERR_CAPACITY;
+  CounterScope cs(c);
+  cudaStream_t st = (cudaStream_t)stream;
+  HYDRA_TRY(do_draft(c, c->d_tree_tok, st));
+  if (c->plant) HYDRA_TRY(apply_plant(c->d_tree_tok, c->plant, c->batch * c->T, st));
+  HYDRA_TRY(do_verify(c, c->d_tree_tok, c->d_amax, nullptr, st));
+  HYDRA_TRY(do_accept(c, c->d_tree_tok, c->d_amax, n_acc, nullptr, out_tok, st));
+  return HYDRA_OK;
+}
+
+hydra_status hydra_set_plant(hydra_ctx* c, const int32_t* plant) {
+  if (!c) return HYDRA_ERR_INVALID;
+  c->plant = plant;
+  return HYDRA_OK;
+}
+
+hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes) {
+  if (!c || !ptr) return HYDRA_ERR_INVALID;
+  const hydra_model_cfg& m = c->m;
+  const size_t kvl = kv_layer_elems(m) * c->esize;
+  const int K = c->h.n_heads;
+  void* p = nullptr; size_t n = 0;
+  switch (which) {
+    case HYDRA_BUF_LEN: p = c->d_len; n = m.max_batch * sizeof(int); break;
+    case HYDRA_BUF_ROOT_TOK: p = c->d_root_tok; n = m.max_batch * sizeof(int); break;
+    case HYDRA_BUF_H_TREE: p = c->h_tree; n = (size_t)c->R * m.d_model * sizeof(float); break;
+    case HYDRA_BUF_H_NEW: p = c->h_new; n = (size_t)m.max_batch * (K + 1) * m.d_model * sizeof(float); break;
+    case HYDRA_BUF_KV_BASE: p = c->kv_base; n = (size_t)m.n_layers * 2 * kvl; break;
+    case HYDRA_BUF_KV_PREFIX: p = c->h.prefix_attn ? c->kv_pfx : nullptr; n = c->h.prefix_attn ? 2 * kvl : 0; break;
+    case HYDRA_BUF_TREE_MASK: p = c->d_anc; n = c->T * sizeof(uint64_t); break;
+    case HYDRA_BUF_TREE_TOK: p = c->d_tree_tok; n = (size_t)m.max_batch * c->T * sizeof(int); break;
+    case HYDRA_BUF_AMAX: p = c->d_amax; n = (size_t)m.max_batch * c->T * sizeof(int); break;
+    case HYDRA_BUF_HEAD_LOGITS: p = c->head_logits; n = (size_t)c->RH * m.vocab * sizeof(float); break;
+    case HYDRA_BUF_N_NEW: p = c->d_n_new; n = m.max_batch * sizeof(int); break;
+    case HYDRA_BUF_H_PRIME: p = c->hprime; n = (size_t)m.max_batch * m.d_model * sizeof(float); break;
+    case HYDRA_BUF_LOGITS: p = c->logits; n = (size_t)m.max_batch * c->T * m.vocab * sizeof(float); break;
+    default: return HYDRA_ERR_INVALID;
+  }
+  *ptr = p;
+  if (bytes) *bytes = n;
+  return HYDRA_OK;
+}
+
+hydra_status hydra_poll_status(hydra_ctx* c, void* stream) {
+  if (!c) return HYDRA_ERR_INVALID;
+  cudaStream_t st = (cudaStream_t)stream;
+  int word = 0;
+  HYDRA_CUDA(cudaStreamSynchronize(st));
+  HYDRA_CUDA(cudaMemcpy(&word, c->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (word) HYDRA_CUDA(cudaMemset(c->d_status, 0, sizeof(int)));
+  if (word & ST_TIMEOUT) return HYDRA_ERR_TIMEOUT;
+  if (word & ST_BOUNDS) return HYDRA_ERR_BOUNDS;
+  return HYDRA_OK;
+}
+
+long long hydra_launch_count(hydra_ctx* c) { return c ? c->launches : 0; }
+
+hydra_status hydra_set_gemm_mode(hydra_ctx* c, int mode) {
+  if (!c || (mode != 0 && mode != 1)) return HYDRA_ERR_INVALID;
+  c->gemm_mode = mode;
+  return HYDRA_OK;
+}
+
+const char* hydra_status_str(hydra_status s) {
+  switch (s) {
+    case HYDRA_OK: return "ok";
+    case HYDRA_ERR_INVALID: return "invalid argument";
+    case HYDRA_ERR_CAPACITY: return "capacity exceeded";
+    case HYDRA_ERR_STATE: return "call out of order";
+    case HYDRA_ERR_UNSUPPORTED: return "unsupported shape";
+    case HYDRA_ERR_CUDA: return "CUDA error";
+    case HYDRA_ERR_TIMEOUT: return "device-side wait timed out";
+    case HYDRA_ERR_BOUNDS: return "device-side index out of range";
+  }
+  return "unknown";
+}
+
+const char* hydra_last_error(void) { return g_err; }
+
+hydra_status hydra_gemm(const void* x, const void* w, float* out, float* partial, int m, int n, int k, int dtype, int splits,
+                        int mode, int32_t* status, void* stream) {
+  if (!x || !w || !out || m < 1 || n < 1 || k < 1 || splits < 1 || (dtype != 0 && dtype != 1)) return HYDRA_ERR_INVALID;
+  cudaStream_t st = (cudaStream_t)stream;
+  CounterScope cs(nullptr);
+  if (dtype == 1 && mode == 0) {
+    if (!status) return HYDRA_ERR_INVALID;
+    if (!gemm_tc_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
+    if (splits == 1) return gemm_tc((const bf16*)x, m, (const bf16*)w, out, (size_t)m * n, m, n, k, 1, status, st);
+    if (!partial) return HYDRA_ERR_INVALID;
+    HYDRA_TRY(gemm_tc((const bf16*)x, m, (const bf16*)w, partial, (size_t)m * n, m, n, k, splits, status, st));
+    return reduce_splits(partial, (size_t)m * n, splits, out, (size_t)m * n, st);
+  }
+  if (splits != 1) return HYDRA_ERR_UNSUPPORTED;
+  return gemm_simt(x, w, out, m, n, k, dtype, st);
+}
+
+size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq) {
+  if (batch < 1 || tc < 1 || n_heads < 1 || head_dim < 1 || max_seq < 1) return 0;
+  return attention_scratch_bytes(batch, tc, n_heads, head_dim, max_seq);
+}
+
+hydra_status hydra_tree_attention(const float* q, const void* kc, const void* vc, const int32_t* pos0, const int32_t* n_rows,
+                                  const uint64_t* mask, void* out, void* scratch, int batch, int tc, int n_heads, int head_dim,
+                                  int max_seq, int dtype, void* stream) {
+  if (!q || !kc || !vc || !pos0 || !mask || !out || !scratch || batch < 1 || tc < 1 || tc > 64) return HYDRA_ERR_INVALID;
+  CounterScope cs(nullptr);
+  RowSet rs{batch, tc, n_rows, pos0, nullptr, mask};
+  return tree_attention(q, kc, vc, rs, out, scratch, n_heads, head_dim, max_seq, max_seq, dtype, (cudaStream_t)stream);
+}
+
+}  // extern "C"

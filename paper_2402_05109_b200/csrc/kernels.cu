@@ -729,6 +729,19 @@ hydra_status apply_plant(int* tree_tok, const int* plant, int count, cudaStream_
   return HYDRA_OK;
 }
 
+template <typename T>
+__global__ void cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t count) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) dst[i] = from_f<T>(src[i]);
+}
+hydra_status cast_rows(const float* src, void* dst, size_t count, int dtype, cudaStream_t st) {
+  unsigned grid = (unsigned)((count + 255) / 256);
+  if (dtype == 0) cast_rows_kernel<float><<<grid, 256, 0, st>>>(src, (float*)dst, count);
+  else cast_rows_kernel<bf16><<<grid, 256, 0, st>>>(src, (bf16*)dst, count);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
 __global__ void copy_i32_kernel(int* dst, const int* src, int count) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < count) dst[i] = src[i];

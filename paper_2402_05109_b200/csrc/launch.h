@@ -76,6 +76,8 @@ hydra_status prefix_rowset(const int* len, const int* n_new, int* pos0, int* n_r
 // hprime[b] = x[b*tc + n_rows[b]-1]
 hydra_status pick_last_row(const float* x, const int* n_rows, int tc, float* hprime, int batch, int d, cudaStream_t st);
 hydra_status apply_plant(int* tree_tok, const int* plant, int count, cudaStream_t st);
+// dst = src converted to the operand type
+hydra_status cast_rows(const float* src, void* dst, size_t count, int dtype, cudaStream_t st);
 hydra_status copy_i32(int* dst, const int* src, int count, cudaStream_t st);
 
 }  // namespace hydra

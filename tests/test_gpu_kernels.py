@@ -1,0 +1,64 @@
+"""Kernel-level parity through the C ABI: the tensor-core GEMM, the SIMT GEMM and tree attention against
+their plain definitions evaluated by the oracle's routines / torch CPU float64."""
+import pytest
+import torch
+
+from oracle.hydra_oracle import masked_attention, TreeTables
+from synth import normal_, load_tree
+
+pytestmark = pytest.mark.gpu
+
+
+def rnd(shape, seed, stream, dtype, std=1.0):
+    return normal_(torch.empty(shape, dtype=dtype), seed, stream, std)
+
+
+@pytest.mark.parametrize("m,n,k,splits", [(64, 256, 512, 1), (64, 384, 4096, 3), (5, 128, 256, 1), (11, 256, 1280, 2),
+                                          (16, 128, 64, 1), (100, 512, 704, 4), (256, 256, 1024, 1), (300, 384, 512, 2),
+                                          (64, 128, 11008, 4), (1, 1024, 256, 1)])
+def test_gemm_tensor_core_matches_definition(m, n, k, splits):
+    from paper_2402_05109_b200 import gemm
+    x = rnd((m, k), 11, m + k, torch.bfloat16)
+    w = rnd((n, k), 12, n + k, torch.bfloat16, 0.02)
+    ref = x.double() @ w.double().T
+    out = gemm(x.cuda(), w.cuda(), splits=splits, mode=0).cpu().double()
+    # products of bfloat16 values are exact in float; only the float accumulation order differs
+    tol = 1e-5 * float(ref.abs().max()) + 1e-6 * k ** 0.5
+    assert float((out - ref).abs().max()) <= tol
+    simt = gemm(x.cuda(), w.cuda(), splits=1, mode=1).cpu().double()
+    assert float((simt - ref).abs().max()) <= tol
+
+
+@pytest.mark.parametrize("m,n,k", [(16, 768, 256), (7, 1376, 256), (16, 256, 688), (4, 1024, 1024)])
+def test_gemm_float(m, n, k):
+    from paper_2402_05109_b200 import gemm
+    x = rnd((m, k), 13, 1, torch.float32)
+    w = rnd((n, k), 14, 2, torch.float32, 0.02)
+    ref = x.double() @ w.double().T
+    out = gemm(x.cuda(), w.cuda()).cpu().double()
+    assert float((out - ref).abs().max()) <= 1e-5 * float(ref.abs().max()) + 1e-6
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("hd", [64, 128])
+def test_tree_attention_matches_masked_softmax(dtype, hd):
+    from paper_2402_05109_b200 import tree_attention
+    parent = load_tree("tree63_d4")
+    t = TreeTables(parent)
+    B, H, S, tc = 3, 3, 700, t.T
+    pos0 = [0, 333, 600]                    # empty cache, a cache spanning several KV chunks with a ragged tail, long
+    n_rows = [tc, tc, 17]                   # ragged row counts (rows beyond n_rows are ignored)
+    kc = rnd((B, H, S, hd), 21, 1, dtype)
+    vc = rnd((B, H, S, hd), 21, 2, dtype)
+    q = rnd((B * tc, H, hd), 21, 3, torch.float32)
+    mask = torch.tensor([a - (1 << 64) if a >= (1 << 63) else a for a in t.anc_mask], dtype=torch.int64)
+    out = tree_attention(q.cuda(), kc.cuda(), vc.cuda(), torch.tensor(pos0, dtype=torch.int32).cuda(),
+                         torch.tensor(n_rows, dtype=torch.int32).cuda(), mask.cuda(), tc).float().cpu().view(B, tc, H, hd)
+    for b in range(B):
+        n, L = n_rows[b], pos0[b] + n_rows[b]
+        allowed = torch.cat([torch.ones(n, pos0[b], dtype=torch.bool), t.allowed[:n, :n]], dim=1)
+        k = kc[b, :, :L].permute(1, 0, 2).double()
+        v = vc[b, :, :L].permute(1, 0, 2).double()
+        ref = masked_attention(q.view(B, tc, H, hd)[b, :n].double(), k, v, allowed)
+        err = float((out[b, :n].double() - ref).abs().max())
+        assert err <= (2e-5 if dtype == torch.float32 else 2e-2), err

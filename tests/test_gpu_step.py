@@ -1,0 +1,94 @@
+"""Whole-step parity of the CUDA library against the CPU oracle (lock-step, through the C ABI)."""
+import pytest
+import torch
+
+from oracle.hydra_oracle import HydraOracle
+from synth import get_config, make_weights, make_prompts, load_tree, chain_tree
+from synth.configs import ModelCfg, HeadCfg
+from tests.parity import lockstep
+
+pytestmark = pytest.mark.gpu
+
+
+def run(model, head, parent, prompts_lens, steps, seed, max_seq, oracle_dtype=torch.float64, weights_device="cpu", **kw):
+    from paper_2402_05109_b200 import Hydra
+    w = make_weights(model, head, seed, device=weights_device)
+    wg = {k: v.cuda() for k, v in w.items()}
+    wc = {k: v.cpu() for k, v in w.items()}
+    prompts = make_prompts(seed, prompts_lens, model.vocab)
+    o = HydraOracle(model, head, parent, wc, max_seq, dtype=oracle_dtype, cache_weights=True)
+    g = Hydra(model, head, parent, wg, max_batch=len(prompts), max_seq=max_seq)
+    try:
+        return lockstep(o, g, prompts, steps, seed, **kw), g
+    finally:
+        g.close()
+
+
+def test_c1_tiny_fp32_all_steps_accept_exercise():
+    cfg = get_config("c1")
+    st, _ = run(cfg.model, cfg.head, load_tree(cfg.tree), cfg.prompt_lens, cfg.steps, cfg.seed, cfg.max_seq, kv_layers=(0, 1))
+    assert st.steps == 8
+    seen = {n for step in st.n_acc for n in step}
+    assert seen >= {0, 1, 2, 3}, seen
+    assert st.max_logit_err < 1e-3 and st.max_hidden_err < 1e-4      # float path: far inside the tolerances
+
+
+def test_small_bf16_hydrapp_ragged_batch():
+    """bfloat16 / tensor-core path with the prefix layer, 4-layer heads, the 63-node tree and a ragged batch
+    whose prompts span several prefill chunks with ragged tails."""
+    m = ModelCfg(3, 256, 2, 128, 512, 1024, dtype="bf16")
+    h = HeadCfg(4, 4, True)
+    st, _ = run(m, h, load_tree("tree63_d4"), [37, 130, 64], 6, 5, 256)
+    seen = {n for step in st.n_acc for n in step}
+    assert seen >= {0, 1, 2, 3, 4}, seen
+
+
+def test_small_bf16_simt_gemm_mode_and_root_only_tree():
+    from paper_2402_05109_b200 import Hydra
+    m = ModelCfg(2, 256, 4, 64, 512, 1024, dtype="bf16")
+    h = HeadCfg(2, 1, False)
+    w = make_weights(m, h, 6)
+    prompts = make_prompts(6, [20], m.vocab)
+    o = HydraOracle(m, h, [-1], w, 64)
+    g = Hydra(m, h, [-1], {k: v.cuda() for k, v in w.items()}, 1, 64)
+    g.set_gemm_mode(1)
+    st = lockstep(o, g, prompts, 3, 6, plant=False)
+    assert all(n == [0] for n in st.n_acc)
+    g.close()
+
+
+def test_chain_tree_and_capacity_and_state_errors():
+    from paper_2402_05109_b200 import Hydra, HydraError
+    m = ModelCfg(2, 256, 4, 64, 512, 1024, dtype="fp32")
+    h = HeadCfg(3, 1, False)
+    w = make_weights(m, h, 7)
+    parent = chain_tree(3)
+    o = HydraOracle(m, h, parent, w, 48)
+    g = Hydra(m, h, parent, {k: v.cuda() for k, v in w.items()}, 1, 48)
+    with pytest.raises(HydraError, match="order"):
+        g.batch = 1
+        g.draft()
+    st = lockstep(o, g, make_prompts(7, [30], m.vocab), 3, 7)
+    # capacity: upper bound 30 + 3*4 = 42; 42 + 4 <= 48 passes, then 46 + 4 > 48 must be refused before any launch
+    g.step()
+    before = g.launch_count()
+    with pytest.raises(HydraError, match="capacity"):
+        g.step()
+    assert g.launch_count() == before
+    g.close()
+
+
+def test_out_of_range_token_sets_status_word():
+    from paper_2402_05109_b200 import Hydra, HydraError
+    m = ModelCfg(1, 256, 4, 64, 512, 1024, dtype="fp32")
+    h = HeadCfg(1, 1, False)
+    w = make_weights(m, h, 8)
+    g = Hydra(m, h, [-1, 0], {k: v.cuda() for k, v in w.items()}, 1, 32)
+    g.prefill(make_prompts(8, [5], m.vocab))
+    g.draft()
+    bad = torch.tensor([[3, 5000]], dtype=torch.int32).cuda()
+    g.verify(bad)
+    with pytest.raises(HydraError, match="index"):
+        g.poll_status()
+    g.poll_status()                     # cleared by the poll
+    g.close()
