@@ -105,8 +105,8 @@ def lockstep(o: HydraOracle, g, prompts, steps: int, seed: int, plant: bool = Tr
         if plant:
             for b in range(B):
                 mlen = min(planted_length(s, b, K), o.tree.K)
-                teacher = (teacher_fn or o.greedy_continuation)(b, mlen + 1)[1:] if mlen > 0 else []
-                row = plant_row(o.tree.parent, teacher, mlen, seed, s, b)
+                teacher = (teacher_fn or o.greedy_continuation)(b, mlen + 2)[1:]
+                row = plant_row(o.tree.parent, teacher, mlen, seed, s, b, vocab=m.vocab)
                 for i, v in enumerate(row):
                     if v >= 0:
                         tok[b, i] = v
