@@ -1,0 +1,407 @@
+#!/usr/bin/env python
+"""Benchmark of the Hydra decode step (draft -> verify -> accept+compact) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one batch of synthetic input.  Prints ONE JSON line.
+Multi-GPU runs are independent replicas (the step has no exchange between sequences): every rank runs the
+same workload on its own GPU, the time is the max over ranks, the value the sum of all ranks' tokens.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from synth import get_config, make_weights, make_prompts, load_tree, plant_row, planted_length  # noqa: E402
+
+METRIC = "drafted+verified tokens/s (tree rows through draft+verify+accept per second)"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def verify_bytes(m, B, T, lens):
+    """Algorithmic bytes of one verification: every base weight once, every live KV row once, new rows written."""
+    s = 2 if m.dtype == "bf16" else 4
+    d, f = m.d_model, m.d_ffn
+    w = s * (m.n_layers * (4 * d * d + 3 * d * f) + m.vocab * d)
+    kv = sum(2 * m.n_layers * d * s * (L + T) for L in lens) + B * T * 2 * m.n_layers * d * s
+    return w + kv
+
+
+def draft_bytes(m, h, lens):
+    s = 2 if m.dtype == "bf16" else 4
+    d, f = m.d_model, m.d_ffn
+    heads = sum(((i + 1) + (h.n_mlp_layers - 1)) * d * d for i in range(1, h.n_heads + 1)) + h.n_heads * m.vocab * d
+    pfx = (4 * d * d + 3 * d * f) if h.prefix_attn else 0
+    return s * (heads + pfx) + (sum(2 * d * s * L for L in lens) if h.prefix_attn else 0)
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def teacher_stream(Hydra, cfg, weights, prompts, n_tokens, max_seq):
+    """Greedy continuation of every prompt from the library itself (root-only tree = plain decoding)."""
+    g = Hydra(cfg.model, cfg.head, [-1], weights, len(prompts), max_seq)
+    g.prefill(prompts)
+    B = len(prompts)
+    roots = g.get_buffer("ROOT_TOK")[:B].clone()
+    outs = torch.empty(n_tokens, B, cfg.head.n_heads + 1, dtype=torch.int32, device="cuda")
+    nacc = torch.empty(B, dtype=torch.int32, device="cuda")
+    for i in range(n_tokens):
+        g.step(nacc, outs[i])
+    g.poll_status()
+    seq = torch.cat([roots[None], outs[:, :, 0]]).cpu().T.tolist()       # [B][n_tokens+1], first = root
+    g.close()
+    return seq
+
+
+def plant_schedule(cfg, parent, teacher, n_steps):
+    """plant[s][b][T] assuming every step accepts exactly its planted length."""
+    K, V = cfg.head.n_heads, cfg.model.vocab
+    B = cfg.batch
+    pos = [0] * B
+    plan = torch.full((n_steps, B, len(parent)), -1, dtype=torch.int32)
+    planned = []
+    for s in range(n_steps):
+        row_m = []
+        for b in range(B):
+            mlen = planted_length(s, b, K)
+            t = teacher[b][pos[b] + 1: pos[b] + mlen + 2]
+            plan[s, b] = torch.tensor(plant_row(parent, t, mlen, cfg.seed, s, b, vocab=V), dtype=torch.int32)
+            pos[b] += mlen + 1
+            row_m.append(mlen)
+        planned.append(row_m)
+    return plan, planned
+
+
+def oracle_sample(cfg, weights_cpu, parent, n_steps, threads):
+    """The CPU oracle, as it stands, on a bounded sample of the workload: full draft and acceptance, and the
+    verification forward timed on 1 and on 3 of the decoder layers (plus final norm and LM head) and
+    extrapolated linearly to all layers.  Prompt shortened to 64 tokens.  Returns seconds per step."""
+    import copy
+    from oracle.hydra_oracle import HydraOracle
+    torch.set_num_threads(threads)
+    prompts = make_prompts(cfg.seed, [64] * cfg.batch, cfg.model.vocab)
+    oracles = []
+    for nl in (1, 3):
+        m = copy.copy(cfg.model)
+        m.n_layers = nl
+        o = HydraOracle(m, cfg.head, parent, weights_cpu, 64 + 8 * (cfg.head.n_heads + 1) * (n_steps + 1) + len(parent),
+                        dtype=torch.float32, cache_weights=True)
+        o.prefill(prompts)
+        oracles.append(o)
+    NL = cfg.model.n_layers
+    per_step = []
+    for s in range(n_steps):
+        o1, o3 = oracles
+        t0 = time.perf_counter()
+        tok = o3.draft()
+        t1 = time.perf_counter()
+        amax3, _ = o3.verify(tok)
+        t2 = time.perf_counter()
+        o3.accept_compact(tok, amax3)
+        t3 = time.perf_counter()
+        tok1 = o1.draft()
+        t4 = time.perf_counter()
+        amax1, _ = o1.verify(tok1)
+        t5 = time.perf_counter()
+        o1.accept_compact(tok1, amax1)
+        v3, v1 = t2 - t1, t5 - t4
+        per_layer = max(0.0, (v3 - v1) / 2.0)
+        per_step.append((t1 - t0) + (t3 - t2) + v1 + (NL - 1) * per_layer)
+    return per_step
+
+
+def run_reference(args, cfg, parent):
+    """Reference arm: the CPU oracle timed on the host cores (a deliberately plain program)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    threads = os.cpu_count() or 1
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = make_weights(cfg.model, cfg.head, cfg.seed, device=dev)
+    w = {k: v.cpu() for k, v in w.items()}
+    per_step = oracle_sample(cfg, w, parent, args.warmup + args.steps, threads)[args.warmup:]
+    sec = sum(per_step) / len(per_step)
+    rows = cfg.batch * len(parent)
+    val = rows / sec
+    sample = ("oracle decode step at the workload's shapes with the prompt shortened to 64 tokens; verification timed "
+              "on 1 and 3 decoder layers and extrapolated linearly to %d layers" % cfg.model.n_layers)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": {"workload": cfg.name},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    cfg = get_config(args.workload)
+    parent = load_tree(cfg.tree)
+    if args.impl == "reference":
+        return run_reference(args, cfg, parent)
+
+    from paper_2402_05109_b200 import Hydra           # raises if libhydra.so is missing: no fallback
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    m, h = cfg.model, cfg.head
+    B, T, K = cfg.batch, len(parent), cfg.head.n_heads
+    n_total = args.warmup + args.steps
+    max_seq = max(cfg.prompt_lens) + (n_total + 1) * (K + 1) + T + 8
+    weights = make_weights(m, h, cfg.seed, device="cuda")
+    prompts = make_prompts(cfg.seed, cfg.prompt_lens, m.vocab)
+    teacher = teacher_stream(Hydra, cfg, weights, prompts, n_total * (K + 1) + K + 2, max_seq + n_total * (K + 1))
+    plan, planned = plant_schedule(cfg, parent, teacher, n_total)
+    plan_dev = plan.cuda()
+    g = Hydra(m, h, parent, weights, B, max_seq)
+    stream = torch.cuda.current_stream()
+
+    def fresh():
+        g.prefill(prompts)
+        g.poll_status()
+
+    # ---- device-resident timed run: K whole steps back to back
+    fresh()
+    nacc = torch.zeros(n_total, B, dtype=torch.int32, device="cuda")
+    outs = torch.empty(n_total, B, K + 1, dtype=torch.int32, device="cuda")
+    for s in range(args.warmup):
+        g.set_plant(plan_dev[s])
+        g.step(nacc[s], outs[s])
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = g.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s in range(args.warmup, n_total):
+        g.set_plant(plan_dev[s])
+        g.step(nacc[s], outs[s])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    launches = g.launch_count() - launches0
+    g.poll_status()
+    ms_total = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    acc = nacc[args.warmup:].float().mean().item()
+    lens_end = g.get_buffer("LEN")[:B].cpu().tolist()
+
+    # ---- per-phase times (split API, events around each phase)
+    fresh()
+    ph = {"draft": [], "verify": [], "accept": []}
+    lens_mid = []
+    for s in range(n_total):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        ev[0].record(stream)
+        tok = g.draft()
+        ev[1].record(stream)
+        tok = torch.where(plan_dev[s] >= 0, plan_dev[s], tok).contiguous()
+        torch.cuda.synchronize()
+        ev[1].record(stream)
+        amax = g.verify(tok)
+        ev[2].record(stream)
+        g.accept_compact(tok, amax)
+        ev[3].record(stream)
+        torch.cuda.synchronize()
+        if s >= args.warmup:
+            ph["verify"].append(ev[1].elapsed_time(ev[2]))
+            ph["accept"].append(ev[2].elapsed_time(ev[3]))
+            lens_mid.append(g.get_buffer("LEN")[:B].cpu().tolist())
+    # draft timed separately so that the host-side overlay does not sit inside it
+    fresh()
+    for s in range(n_total):
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        tok = g.draft()
+        b_.record(stream)
+        tok = torch.where(plan_dev[s] >= 0, plan_dev[s], tok).contiguous()
+        amax = g.verify(tok)
+        g.accept_compact(tok, amax)
+        torch.cuda.synchronize()
+        if s >= args.warmup:
+            ph["draft"].append(a.elapsed_time(b_))
+    med = lambda v: sorted(v)[len(v) // 2]
+    t_draft, t_verify, t_accept = med(ph["draft"]), med(ph["verify"]), med(ph["accept"])
+    mean_lens = [sum(l[b] for l in lens_mid) / len(lens_mid) for b in range(B)]
+    vbytes = verify_bytes(m, B, T, mean_lens)
+    dbytes = draft_bytes(m, h, mean_lens)
+    hbm_peak, peak_kind = peaks()
+    verify_gbs = vbytes / (t_verify * 1e-3) / 1e9
+
+    # ---- dominant kernel (the weight-streaming GEMM): event-bracketed launches over K steps
+    fresh()
+    for s in range(args.warmup):
+        g.set_plant(plan_dev[s]); g.step(nacc[s], outs[s])
+    g.set_timing(True)
+    for s in range(args.warmup, n_total):
+        g.set_plant(plan_dev[s]); g.step(nacc[s], outs[s])
+    gemm_ms, gemm_n, gemm_bytes = g.get_timing(0)
+    att_ms, att_n, _ = g.get_timing(1)
+    acc_ms, acc_n, _ = g.get_timing(2)
+    g.set_timing(False)
+    gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
+
+    # ---- end to end: host buffers, copies inside the timed region, one synchronisation per step
+    fresh()
+    h_plan = torch.empty(B, T, dtype=torch.int32).pin_memory()
+    h_nacc = torch.empty(B, dtype=torch.int32).pin_memory()
+    h_out = torch.empty(B, K + 1, dtype=torch.int32).pin_memory()
+    d_plan = torch.empty(B, T, dtype=torch.int32, device="cuda")
+    d_nacc = torch.empty(B, dtype=torch.int32, device="cuda")
+    d_out = torch.empty(B, K + 1, dtype=torch.int32, device="cuda")
+    g.set_plant(d_plan)
+    pos = [0] * B
+    emitted = 0
+    t_e2e = 0.0
+    for s in range(n_total):
+        for b in range(B):                       # the host plants from the tokens actually emitted so far
+            mlen = planted_length(s, b, K)
+            tch = teacher[b][pos[b] + 1: pos[b] + mlen + 2]
+            h_plan[b] = torch.tensor(plant_row(parent, tch, mlen, cfg.seed, s, b, vocab=m.vocab), dtype=torch.int32)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        d_plan.copy_(h_plan, non_blocking=True)
+        g.step(d_nacc, d_out)
+        h_nacc.copy_(d_nacc, non_blocking=True)
+        h_out.copy_(d_out, non_blocking=True)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        for b in range(B):
+            pos[b] += int(h_nacc[b]) + 1
+        if s >= args.warmup:
+            t_e2e += dt
+            emitted += int(h_nacc.sum()) + B
+    if dist is not None:
+        t = torch.tensor([t_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_e2e = float(t.item())
+    e2e_val = world * B * T * args.steps / t_e2e
+
+    # ---- CPU baseline: the oracle on the host cores (rank 0, single-GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        threads = os.cpu_count() or 1
+        wc = {k: v.cpu() for k, v in weights.items()}
+        per = oracle_sample(cfg, wc, parent, 3, threads)[1:]
+        sec = sum(per) / len(per)
+        cpu = {"value": B * T / sec, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+               "sample": "2 timed oracle decode steps (after 1 warm-up) at the workload's shapes, prompt shortened to 64 "
+                         "tokens, verification timed on 1 and 3 decoder layers and extrapolated linearly to %d layers; "
+                         "%.2f s per full step" % (m.n_layers, sec)}
+    g.close()
+    if rank != 0:
+        return
+    value = world * B * T / (ms_step * 1e-3)
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if m.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": "%s: %d-layer d=%d Llama-shape decoder, %d Hydra heads x %d MLP layers, prefix layer=%s, "
+                               "%d-row tree (root + %d candidates), batch %d, prompts %s, accept-exercise planting"
+                               % (cfg.name, m.n_layers, m.d_model, K, h.n_mlp_layers, h.prefix_attn, T, T - 1, B,
+                                  cfg.prompt_lens),
+                   "l2": "every step streams %.1f GB of weights, far above the 126 MB L2; no flush needed" % (vbytes / 1e9),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "verify_ms": t_verify, "draft_ms": t_draft, "accept_compact_ms": t_accept,
+        "verify_bytes": vbytes, "draft_bytes": dbytes,
+        "verify_hbm_gbs": verify_gbs, "verify_frac_of_8TBs": verify_gbs / NOMINAL_HBM_GBS,
+        "verify_frac_of_%s" % peak_kind: verify_gbs / hbm_peak,
+        "emitted_tokens_per_s": world * (acc + 1) * B / (ms_step * 1e-3), "mean_accepted": acc,
+        "planned_mean_accepted": sum(sum(r) for r in planned[args.warmup:]) / (args.steps * B),
+        "final_lens": lens_end,
+        "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel (weight-streaming bf16 GEMM, all shapes of a step)",
+                     "achieved": gemm_gbs, "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": gemm_gbs / hbm_peak, "frac_of_8TBs": gemm_gbs / NOMINAL_HBM_GBS, "traffic": None,
+                     "launches": gemm_n, "avg_launch_us": gemm_ms * 1e3 / max(1, gemm_n),
+                     "bytes_per_launch": gemm_bytes / max(1, gemm_n),
+                     "gemm_ms_per_step": gemm_ms / args.steps, "attention_ms_per_step": att_ms / args.steps,
+                     "accept_ms_per_step": acc_ms / args.steps},
+        "e2e": {"value": e2e_val, "unit": "tokens/s", "h2d_bytes_per_step": B * T * 4, "d2h_bytes_per_step": B * (K + 2) * 4,
+                "ms_per_step": t_e2e / args.steps * 1e3, "emitted_tokens_per_s": world * emitted / t_e2e},
+        "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

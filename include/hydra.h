@@ -146,6 +146,15 @@ hydra_status hydra_poll_status(hydra_ctx*, void* stream);
 /* Number of kernels the library has launched for this context since create. */
 long long hydra_launch_count(hydra_ctx*);
 
+/* Per-kernel-class device timing for benchmarks.  While on, every launch of a class is bracketed by a pair
+ * of CUDA events on the call's stream (this separates back-to-back kernels, so whole-step times taken
+ * with timing on are slightly longer).  hydra_get_timing synchronises the device, returns the summed
+ * event time (ms), the number of bracketed launches and, for GEMMs, their summed algorithmic bytes
+ * (weight matrix + activation slab read once, output written once), then forgets those records. */
+enum { HYDRA_TIME_GEMM = 0, HYDRA_TIME_ATTENTION = 1, HYDRA_TIME_ACCEPT = 2 };
+hydra_status hydra_set_timing(hydra_ctx*, int on);
+hydra_status hydra_get_timing(hydra_ctx*, int kclass, double* ms_total, long long* launches, double* bytes_total);
+
 /* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA (default), 1 = the plain SIMT kernel. */
 hydra_status hydra_set_gemm_mode(hydra_ctx*, int mode);
 

@@ -130,7 +130,7 @@ class HydraOracle:
     """State and phases of Hydra decoding for a batch of independent sequences."""
 
     def __init__(self, model, head, parent: Sequence[int], weights: Dict[str, torch.Tensor],
-                 max_seq: int, dtype=torch.float64, cache_weights: bool = False):
+                 max_seq: int, dtype=torch.float64, cache_weights=False):
         self.m, self.h = model, head
         self.tree = TreeTables(parent, max_depth=head.n_heads)
         self.w = weights
@@ -143,11 +143,12 @@ class HydraOracle:
 
     def W(self, name: str) -> torch.Tensor:
         """Weight `name` widened to the arithmetic dtype (head, embedding and LM-head matrices, which
-        are used many times per step, are kept widened when cache_weights is set; the rest is widened on use)."""
+        are used many times per step, are kept widened when cache_weights is True, everything when it is "all";
+        the rest is widened on use)."""
         if name in self._wcache:
             return self._wcache[name]
         t = self.w[name].to(device="cpu", dtype=self.dtype)
-        if self._cache_weights and (name[0] == "H" or name in ("embed", "lm_head")):
+        if self._cache_weights == "all" or (self._cache_weights and (name[0] == "H" or name in ("embed", "lm_head"))):
             self._wcache[name] = t
         return t
 

@@ -57,6 +57,8 @@ lib.hydra_poll_status.argtypes = [_vp, _vp]
 lib.hydra_launch_count.restype = C.c_longlong
 lib.hydra_launch_count.argtypes = [_vp]
 lib.hydra_set_gemm_mode.argtypes = [_vp, _i]
+lib.hydra_set_timing.argtypes = [_vp, _i]
+lib.hydra_get_timing.argtypes = [_vp, _i, C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
 lib.hydra_status_str.restype = C.c_char_p
 lib.hydra_status_str.argtypes = [_i]
 lib.hydra_last_error.restype = C.c_char_p
@@ -187,6 +189,15 @@ class Hydra:
 
     def set_gemm_mode(self, mode: int):
         _check(lib.hydra_set_gemm_mode(self._ctx, mode), "hydra_set_gemm_mode")
+
+    def set_timing(self, on: bool):
+        _check(lib.hydra_set_timing(self._ctx, int(on)), "hydra_set_timing")
+
+    def get_timing(self, kclass: int):
+        """(ms_total, launches, algorithmic_bytes) of a kernel class: 0 GEMM, 1 tree attention, 2 accept+compact."""
+        ms, n, by = C.c_double(), C.c_longlong(), C.c_double()
+        _check(lib.hydra_get_timing(self._ctx, kclass, C.byref(ms), C.byref(n), C.byref(by)), "hydra_get_timing")
+        return ms.value, n.value, by.value
 
     def poll_status(self):
         _check(lib.hydra_poll_status(self._ctx, _stream()), "hydra_poll_status")

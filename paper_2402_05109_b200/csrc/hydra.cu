@@ -85,6 +85,11 @@ struct hydra_ctx {
   std::vector<int> len_ub;
   const int* plant;
   long long launches;
+  // optional per-kernel-class timing (benchmarks): event pairs recorded around launches of a class
+  struct Timed { cudaEvent_t a, b; int cls; double bytes; };
+  int timing;
+  std::vector<Timed> timed;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
 };
 
 namespace {
@@ -208,14 +213,30 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   return (b.off + 255) & ~(size_t)255;
 }
 
+struct TimeScope {                // brackets the launches issued during its lifetime with an event pair
+  hydra_ctx* c; cudaStream_t st; cudaEvent_t a = nullptr, b = nullptr; int cls; double bytes;
+  TimeScope(hydra_ctx* c_, int cls_, double bytes_, cudaStream_t st_) : c(c_), st(st_), cls(cls_), bytes(bytes_) {
+    if (!c->timing) return;
+    if (!c->event_pool.empty()) { a = c->event_pool.back().first; b = c->event_pool.back().second; c->event_pool.pop_back(); }
+    else if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { a = b = nullptr; return; }
+    cudaEventRecord(a, st);
+  }
+  ~TimeScope() { if (a) { cudaEventRecord(b, st); c->timed.push_back({a, b, cls, bytes}); } }
+};
+
 // out = x @ w^T into c->part (split-K partial sums) or, when direct_out is given, straight into it (no split).
 hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void* w, int m, int n, int k, float* direct_out,
                       int* splits, size_t* stride, cudaStream_t st) {
   float* out = direct_out ? direct_out : c->part;
   *stride = (size_t)m * n;
+  int sp = 1;
+  if (c->m.dtype == 1 && c->gemm_mode == 0 && !direct_out) {
+    sp = choose_splits(m, n, k);
+    if ((size_t)sp * m * n > c->part_floats) sp = 1;
+  }
+  // algorithmic bytes of the launch: the weight matrix and the activation slab read once, the output written once
+  TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * sp * m * n, st);
   if (c->m.dtype == 1 && c->gemm_mode == 0) {
-    int sp = direct_out ? 1 : choose_splits(m, n, k);
-    if ((size_t)sp * m * n > c->part_floats && !direct_out) sp = 1;
     *splits = sp;
     return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, out, *stride, m, n, k, sp, c->d_status, st);
   }
@@ -232,7 +253,10 @@ hydra_status run_layer(hydra_ctx* c, const LayerW& w, char* kc, char* vc, const 
   int sp; size_t stride;
   HYDRA_TRY(run_gemm(c, c->xn, c->R, w.wqkv, rows, 3 * d, d, nullptr, &sp, &stride, st));
   HYDRA_TRY(qkv_rope_store(c->part, stride, sp, c->rope, c->q, kc, vc, rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
-  HYDRA_TRY(tree_attention(c->q, kc, vc, rs, c->attn_out, c->att_scratch, m.n_heads, m.head_dim, m.max_seq, len_upper, dt, st));
+  {
+    TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
+    HYDRA_TRY(tree_attention(c->q, kc, vc, rs, c->attn_out, c->att_scratch, m.n_heads, m.head_dim, m.max_seq, len_upper, dt, st));
+  }
   HYDRA_TRY(run_gemm(c, c->attn_out, c->R, w.wo, rows, d, d, nullptr, &sp, &stride, st));
   HYDRA_TRY(residual_rmsnorm(c->x, c->part, stride, sp, c->x, w.ffn_norm, c->xn, nullptr, rows, d, m.rms_eps, dt, st));
   HYDRA_TRY(run_gemm(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, nullptr, &sp, &stride, st));
@@ -323,7 +347,10 @@ hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* 
   a.kv_base = c->kv_base; a.h_tree = c->h_tree; a.h_tree_stride = c->T;
   a.h_new = c->h_new; a.n_new = c->d_n_new; a.len = c->d_len; a.root_tok = c->d_root_tok;
   a.n_acc = n_acc; a.path = path; a.out_tok = out_tok; a.done_counter = c->d_done; a.status = c->d_status;
-  HYDRA_TRY(accept_compact(a, st));
+  {
+    TimeScope ts(c, HYDRA_TIME_ACCEPT, 0.0, st);
+    HYDRA_TRY(accept_compact(a, st));
+  }
   for (int b = 0; b < c->batch; ++b) c->len_ub[b] += c->Ktree + 1;
   return HYDRA_OK;
 }
@@ -386,7 +413,7 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
   }
   c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
   carve(c, *m, *h, th, (char*)ws);
-  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->plant = nullptr; c->launches = 0;
+  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->plant = nullptr; c->launches = 0; c->timing = 0;
   c->len_ub.assign(m->max_batch, 0);
   // clear the workspace, upload the static tables
   auto fail = [&](cudaError_t e, const char* what) { set_last_error(what, e); delete c; return HYDRA_ERR_CUDA; };
@@ -411,6 +438,8 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
 hydra_status hydra_destroy(hydra_ctx* c) {
   if (!c) return HYDRA_ERR_INVALID;
   cudaError_t e = cudaDeviceSynchronize();
+  for (auto& t : c->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+  for (auto& p : c->event_pool) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
   delete c;
   if (e != cudaSuccess) { set_last_error("cudaDeviceSynchronize", e); return HYDRA_ERR_CUDA; }
   return HYDRA_OK;
@@ -542,6 +571,31 @@ hydra_status hydra_poll_status(hydra_ctx* c, void* stream) {
 }
 
 long long hydra_launch_count(hydra_ctx* c) { return c ? c->launches : 0; }
+
+hydra_status hydra_set_timing(hydra_ctx* c, int on) {
+  if (!c) return HYDRA_ERR_INVALID;
+  c->timing = on ? 1 : 0;
+  return HYDRA_OK;
+}
+
+hydra_status hydra_get_timing(hydra_ctx* c, int kclass, double* ms_total, long long* launches, double* bytes_total) {
+  if (!c || kclass < 0 || kclass > HYDRA_TIME_ACCEPT) return HYDRA_ERR_INVALID;
+  HYDRA_CUDA(cudaDeviceSynchronize());
+  double ms = 0, bytes = 0; long long n = 0;
+  std::vector<hydra_ctx::Timed> keep;
+  for (auto& t : c->timed) {
+    if (t.cls != kclass) { keep.push_back(t); continue; }
+    float dt = 0.f;
+    HYDRA_CUDA(cudaEventElapsedTime(&dt, t.a, t.b));
+    ms += dt; bytes += t.bytes; ++n;
+    c->event_pool.push_back({t.a, t.b});
+  }
+  c->timed.swap(keep);
+  if (ms_total) *ms_total = ms;
+  if (launches) *launches = n;
+  if (bytes_total) *bytes_total = bytes;
+  return HYDRA_OK;
+}
 
 hydra_status hydra_set_gemm_mode(hydra_ctx* c, int mode) {
   if (!c || (mode != 0 && mode != 1)) return HYDRA_ERR_INVALID;

@@ -59,10 +59,12 @@ def uniform_ids(seed: int, stream: int, count: int, high: int, device="cpu") -> 
     return ((bits * high) >> 31).to(torch.int32)
 
 
-def normal_(out: torch.Tensor, seed: int, stream: int, std: float, chunk: int = 1 << 22) -> torch.Tensor:
+def normal_(out: torch.Tensor, seed: int, stream: int, std: float, chunk: int = 0) -> torch.Tensor:
     """Fill `out` (any float dtype, contiguous) with std * N(0,1), element i = f(seed, stream, i)."""
     flat = out.view(-1)
     n = flat.numel()
+    if chunk <= 0:
+        chunk = (1 << 25) if out.is_cuda else (1 << 22)
     two_pi = 2.0 * math.pi
     for s in range(0, n, chunk):
         c = min(chunk, n - s)
