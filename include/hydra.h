@@ -174,6 +174,24 @@ const char* hydra_last_error(void); /* text of the last CUDA error seen by this 
  *   needs hydra_attention_scratch_bytes(...) bytes. */
 hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, float* partial_dev, int m, int n, int k,
                         int dtype, int splits, int mode, int32_t* status_dev, void* stream);
+/* hydra_gemm_noalloc: the bfloat16 tensor-core split-K GEMM of hydra_gemm (dtype 1, mode 0) for callers that
+ * may not allocate device memory.  (The paper has no counterpart; this is a convenience of the library.)
+ * Serving loops that must stay clear of the allocator's locks and implicit synchronisation, plugins living
+ * inside a host's fixed memory budget, and processes whose free memory already belongs to a pool cannot
+ * supply hydra_gemm's partial_dev buffer; here the partial sums live in an 8 MiB array that is part of the
+ * library image (every GPU that loads the library holds it until the process exits).
+ *   - x [m][k], w [n][k] bfloat16, out [m][n] float, status_dev as in hydra_gemm: all caller-owned device
+ *     memory; n % 128 == 0, k % 64 == 0, 1 <= splits <= k/64.
+ *   - splits*m*n*4 bytes must fit in the 8 MiB array, otherwise HYDRA_ERR_CAPACITY (text in
+ *     hydra_last_error) and nothing is launched.
+ *   - The call allocates nothing on the device.  The first call on each device looks up the array's device
+ *     address (cudaGetSymbolAddress, with that device current); make that first call outside any stream
+ *     capture.
+ *   - All calls on a GPU share the one array and it keeps the previous call's partial sums; the GEMM
+ *     overwrites every element it later reads, so no clearing is needed, but two calls whose kernels overlap
+ *     on the GPU (different streams, different threads) race on it: serialise them. */
+hydra_status hydra_gemm_noalloc(const void* x_dev, const void* w_dev, float* out_dev, int m, int n, int k, int splits,
+                                int32_t* status_dev, void* stream);
 size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
 hydra_status hydra_tree_attention(const float* q_dev, const void* k_cache_dev, const void* v_cache_dev,
                                   const int32_t* pos0_dev, const int32_t* n_rows_dev, const uint64_t* mask_dev,

@@ -63,6 +63,7 @@ lib.hydra_status_str.restype = C.c_char_p
 lib.hydra_status_str.argtypes = [_i]
 lib.hydra_last_error.restype = C.c_char_p
 lib.hydra_gemm.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]
+lib.hydra_gemm_noalloc.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp]
 lib.hydra_attention_scratch_bytes.restype = _sz
 lib.hydra_attention_scratch_bytes.argtypes = [_i] * 5
 lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 6 + [_vp]
@@ -236,6 +237,16 @@ def gemm(x: torch.Tensor, w: torch.Tensor, splits: int = 1, mode: int = 0) -> to
     if word:
         raise HydraError("hydra_gemm device status word %d" % word)
     return out
+
+
+def gemm_noalloc(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor, status: torch.Tensor, splits: int):
+    """hydra_gemm_noalloc: split-K bfloat16 GEMM whose partial sums live in the library's built-in 8 MiB scratch.
+    The caller passes every tensor (nothing is allocated here, on the host side either): x [m][k], w [n][k]
+    bfloat16, out [m][n] float32, status int32[1].  Calls that overlap on the GPU race on the scratch."""
+    m, k = x.shape
+    n = w.shape[0]
+    _check(lib.hydra_gemm_noalloc(x.data_ptr(), w.data_ptr(), out.data_ptr(), m, n, k, splits, status.data_ptr(), _stream()),
+           "hydra_gemm_noalloc")
 
 
 def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int) -> torch.Tensor:
