@@ -54,6 +54,8 @@ def get_config(name: str) -> RunCfg:
                       "tree15_d3", 1, [32], 8, 0, 128)
     if name == "c2":
         return RunCfg("c2", ModelCfg(**_7B), HeadCfg(**_PP), "tree63_d4", 1, [512], 128, 1, 512 + 128 * 5 + 64)
+    if name == "c2s":          # c2 cut to 4 layers (1.9 GB of weights): the small case for profiler captures
+        return RunCfg("c2s", ModelCfg(**dict(_7B, n_layers=4)), HeadCfg(**_PP), "tree63_d4", 1, [512], 16, 1, 512 + 16 * 5 + 64)
     if name.startswith("c3"):
         b = int(name[3:]) if len(name) > 2 else 8          # "c3b1", "c3b2", "c3b4", "c3b8"
         return RunCfg(name, ModelCfg(**_7B), HeadCfg(**_PP), "tree63_d4", b, _ragged(2, b, 128, 1024), 64, 2,
