@@ -167,7 +167,7 @@ const char* hydra_last_error(void); /* text of the last CUDA error seen by this 
  *   n % 128 == 0 and k % 64 == 0 for mode 0.  splits >= 1 partial sums are reduced into out;
  *   partial_dev needs splits*m*n floats when splits > 1 (may be NULL when splits == 1).
  *   mode as in hydra_set_gemm_mode; status_dev is an int32 status word (bit 1 bounds, bit 2 timeout).
- * hydra_tree_attention: q [rows][n_heads][head_dim] float (rows = batch*tc), caches
+ * hydra_tree_attention: q [rows][n_heads][head_dim] (dtype; rows = batch*tc), caches
  *   [batch][n_heads][max_seq][head_dim] (dtype), pos0 [batch] committed lengths, n_rows [batch] or
  *   NULL (= tc), mask [tc] ancestor bitmasks; out [rows][n_heads*head_dim] (dtype).  Row i of
  *   sequence b sees slots < pos0[b] and slot pos0[b]+j when bit j of mask[i] is set.  scratch_dev
@@ -193,7 +193,7 @@ hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, fl
 hydra_status hydra_gemm_noalloc(const void* x_dev, const void* w_dev, float* out_dev, int m, int n, int k, int splits,
                                 int32_t* status_dev, void* stream);
 size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
-hydra_status hydra_tree_attention(const float* q_dev, const void* k_cache_dev, const void* v_cache_dev,
+hydra_status hydra_tree_attention(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev,
                                   const int32_t* pos0_dev, const int32_t* n_rows_dev, const uint64_t* mask_dev,
                                   void* out_dev, void* scratch_dev, int batch, int tc, int n_heads, int head_dim,
                                   int max_seq, int dtype, void* stream);

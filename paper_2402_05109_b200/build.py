@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhydra.so")
 OBJ = os.path.join(HERE, "_build")
-SOURCES = ["kernels.cu", "gemm_tc.cu", "hydra.cu", "noalloc.cu"]
+SOURCES = ["kernels.cu", "gemm_tc.cu", "attention_tc.cu", "hydra.cu", "noalloc.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 
 

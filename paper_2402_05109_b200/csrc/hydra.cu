@@ -76,9 +76,9 @@ struct hydra_ctx {
   int *d_len, *d_n_new, *d_root_tok, *d_status, *d_pos0, *d_nrows, *d_prompt_len, *d_offsets, *d_tok, *d_tree_tok, *d_amax;
   unsigned int* d_done;
   char *kv_base, *kv_pfx;
-  float *x, *q, *part, *h_tree, *logits, *h_new, *hprime, *y, *head_logits;
+  float *x, *part, *h_tree, *logits, *h_new, *hprime, *y, *head_logits;
   float2* rope;
-  void *xn, *attn_out, *act, *z, *yb, *att_scratch;
+  void *q, *xn, *attn_out, *act, *z, *yb, *att_scratch;
   size_t part_floats;
   // host state
   int batch, state, gemm_mode;
@@ -188,7 +188,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* done = b.take<unsigned int>(m.max_batch);
   auto* kvb = b.take<char>((size_t)m.n_layers * 2 * kv_layer_elems(m) * es);
   auto* kvp = b.take<char>(h.prefix_attn ? (size_t)2 * kv_layer_elems(m) * es : 0);
-  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<float>((size_t)R * d);
+  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)R * d * es);
   auto* part = b.take<float>(part_floats);
   auto* h_tree = b.take<float>((size_t)R * d);
   auto* logits = b.take<float>((size_t)pad_rows(m.max_batch * T) * V);
@@ -641,7 +641,7 @@ size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_di
   return attention_scratch_bytes(batch, tc, n_heads, head_dim, max_seq);
 }
 
-hydra_status hydra_tree_attention(const float* q, const void* kc, const void* vc, const int32_t* pos0, const int32_t* n_rows,
+hydra_status hydra_tree_attention(const void* q, const void* kc, const void* vc, const int32_t* pos0, const int32_t* n_rows,
                                   const uint64_t* mask, void* out, void* scratch, int batch, int tc, int n_heads, int head_dim,
                                   int max_seq, int dtype, void* stream) {
   if (!q || !kc || !vc || !pos0 || !mask || !out || !scratch || batch < 1 || tc < 1 || tc > 64) return HYDRA_ERR_INVALID;

@@ -109,38 +109,59 @@ __device__ __forceinline__ float block_sum(float v, float* sh) {
   return t;
 }
 
+template <typename T> __device__ __forceinline__ void store4(T* p, float4 v);
+template <> __device__ __forceinline__ void store4<float>(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+template <> __device__ __forceinline__ void store4<bf16>(bf16* p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u; u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+template <typename T> __device__ __forceinline__ float4 load4(const T* p);
+template <> __device__ __forceinline__ float4 load4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
+template <> __device__ __forceinline__ float4 load4<bf16>(const bf16* p) {
+  float v[4]; Vec4<bf16>::load(p, v); return make_float4(v[0], v[1], v[2], v[3]);
+}
+
+constexpr int NORM_THREADS = 512;
 template <typename T>
-__global__ void __launch_bounds__(256) residual_rmsnorm_kernel(const float* res, const float* __restrict__ part,
-                                                               size_t stride, int splits, float* x_out,
-                                                               const T* __restrict__ gain, T* __restrict__ xn,
-                                                               float* __restrict__ hn, int d, float eps) {
+__global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const float* res, const float* __restrict__ part,
+                                                                        size_t stride, int splits, float* x_out,
+                                                                        const T* __restrict__ gain, T* __restrict__ xn,
+                                                                        float* __restrict__ hn, int d, float eps) {
   __shared__ float sh[32];
   const size_t base = (size_t)blockIdx.x * d;
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = res ? res[base + i] : 0.f;
-    if (part) for (int p = 0; p < splits; ++p) v += part[p * stride + base + i];
-    x_out[base + i] = v;
-    ss += v * v;
+  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
+    float4 v = res ? *reinterpret_cast<const float4*>(res + base + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (part)
+      for (int p = 0; p < splits; ++p) {
+        float4 a = *reinterpret_cast<const float4*>(part + p * stride + base + i);
+        v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+      }
+    *reinterpret_cast<float4*>(x_out + base + i) = v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   if (!gain) return;
   float tot = block_sum(ss, sh);
   float inv = rsqrtf(tot / (float)d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = x_out[base + i] * inv * to_f<T>(gain[i]);
-    if (xn) xn[base + i] = from_f<T>(v);
-    if (hn) hn[base + i] = v;
+  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
+    float4 v = *reinterpret_cast<const float4*>(x_out + base + i);
+    float4 gn = load4<T>(gain + i);
+    v.x *= inv * gn.x; v.y *= inv * gn.y; v.z *= inv * gn.z; v.w *= inv * gn.w;
+    if (xn) store4<T>(xn + base + i, v);
+    if (hn) *reinterpret_cast<float4*>(hn + base + i) = v;
   }
 }
 hydra_status residual_rmsnorm(const float* res, const float* part, size_t stride, int splits, float* x_out,
                               const void* gain, void* xn, float* hn, int rows, int d, float eps, int dtype,
                               cudaStream_t st) {
+  if (d & 3) return HYDRA_ERR_UNSUPPORTED;
   if (dtype == 0)
-    residual_rmsnorm_kernel<float><<<rows, 256, 0, st>>>(res, part, stride, splits, x_out, (const float*)gain, (float*)xn,
-                                                         hn, d, eps);
+    residual_rmsnorm_kernel<float><<<rows, NORM_THREADS, 0, st>>>(res, part, stride, splits, x_out, (const float*)gain,
+                                                                  (float*)xn, hn, d, eps);
   else
-    residual_rmsnorm_kernel<bf16><<<rows, 256, 0, st>>>(res, part, stride, splits, x_out, (const bf16*)gain, (bf16*)xn, hn,
-                                                        d, eps);
+    residual_rmsnorm_kernel<bf16><<<rows, NORM_THREADS, 0, st>>>(res, part, stride, splits, x_out, (const bf16*)gain,
+                                                                 (bf16*)xn, hn, d, eps);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -165,45 +186,44 @@ hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cud
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __restrict__ part, size_t stride, int splits,
-                                                             const float2* __restrict__ table, float* __restrict__ q,
-                                                             T* __restrict__ kc, T* __restrict__ vc, RowSet rs, int H,
-                                                             int hd, int max_seq, int* status) {
-  const int r = blockIdx.x, b = r / rs.tc, i = r % rs.tc;
+__global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restrict__ part, size_t stride, int splits,
+                                                            const float2* __restrict__ table, T* __restrict__ q,
+                                                            T* __restrict__ kc, T* __restrict__ vc, RowSet rs, int H,
+                                                            int hd, int max_seq, int* status) {
+  const int r = blockIdx.x, h = blockIdx.y, b = r / rs.tc, i = r % rs.tc;
   const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
   if (i >= nr) return;
   const int d = H * hd, half = hd >> 1;
   const int slot = rs.pos0[b] + i;
-  if (slot < 0 || slot >= max_seq) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); return; }
+  if (slot < 0 || slot >= max_seq) { if (threadIdx.x == 0 && h == 0) atomicOr(status, ST_BOUNDS); return; }
+  const int j = threadIdx.x;                                       // rotation pair (j, j + half) of this head
+  if (j >= half) return;
   const float* p0 = part + (size_t)r * 3 * d;
-  for (int e = threadIdx.x; e < H * half; e += blockDim.x) {
-    int h = e / half, j = e % half;
-    int c0 = h * hd + j, c1 = c0 + half;
-    float qa = 0, qb = 0, ka = 0, kb = 0, va = 0, vb = 0;
-    for (int s = 0; s < splits; ++s) {
-      const float* p = p0 + s * stride;
-      qa += p[c0]; qb += p[c1]; ka += p[d + c0]; kb += p[d + c1]; va += p[2 * d + c0]; vb += p[2 * d + c1];
-    }
-    float2 cs = table[(size_t)r * half + j];
-    q[(size_t)r * d + c0] = qa * cs.x - qb * cs.y;
-    q[(size_t)r * d + c1] = qb * cs.x + qa * cs.y;
-    size_t o = (((size_t)b * H + h) * max_seq + slot) * hd;
-    kc[o + j] = from_f<T>(ka * cs.x - kb * cs.y);
-    kc[o + j + half] = from_f<T>(kb * cs.x + ka * cs.y);
-    vc[o + j] = from_f<T>(va);
-    vc[o + j + half] = from_f<T>(vb);
+  const int c0 = h * hd + j, c1 = c0 + half;
+  float qa = 0, qb = 0, ka = 0, kb = 0, va = 0, vb = 0;
+  for (int s = 0; s < splits; ++s) {
+    const float* p = p0 + s * stride;
+    qa += p[c0]; qb += p[c1]; ka += p[d + c0]; kb += p[d + c1]; va += p[2 * d + c0]; vb += p[2 * d + c1];
   }
+  const float2 cs = table[(size_t)r * half + j];
+  q[(size_t)r * d + c0] = from_f<T>(qa * cs.x - qb * cs.y);
+  q[(size_t)r * d + c1] = from_f<T>(qb * cs.x + qa * cs.y);
+  const size_t o = (((size_t)b * H + h) * max_seq + slot) * hd;
+  kc[o + j] = from_f<T>(ka * cs.x - kb * cs.y);
+  kc[o + j + half] = from_f<T>(kb * cs.x + ka * cs.y);
+  vc[o + j] = from_f<T>(va);
+  vc[o + j + half] = from_f<T>(vb);
 }
-hydra_status qkv_rope_store(const float* part, size_t stride, int splits, const float2* table, float* q, void* kcache,
+hydra_status qkv_rope_store(const float* part, size_t stride, int splits, const float2* table, void* q, void* kcache,
                             void* vcache, RowSet rs, int H, int hd, int max_seq, int dtype, int* status,
                             cudaStream_t st) {
-  int rows = rs.batch * rs.tc;
+  dim3 grid(rs.batch * rs.tc, H);
   if (dtype == 0)
-    qkv_rope_store_kernel<float><<<rows, 256, 0, st>>>(part, stride, splits, table, q, (float*)kcache, (float*)vcache, rs,
-                                                       H, hd, max_seq, status);
+    qkv_rope_store_kernel<float><<<grid, 64, 0, st>>>(part, stride, splits, table, (float*)q, (float*)kcache, (float*)vcache,
+                                                      rs, H, hd, max_seq, status);
   else
-    qkv_rope_store_kernel<bf16><<<rows, 256, 0, st>>>(part, stride, splits, table, q, (bf16*)kcache, (bf16*)vcache, rs, H,
-                                                      hd, max_seq, status);
+    qkv_rope_store_kernel<bf16><<<grid, 64, 0, st>>>(part, stride, splits, table, (bf16*)q, (bf16*)kcache, (bf16*)vcache, rs,
+                                                     H, hd, max_seq, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -212,12 +232,12 @@ hydra_status qkv_rope_store(const float* part, size_t stride, int splits, const 
 // Tree attention, split over the KV length.  One CTA per (head, sequence, KV chunk); the chunk's K,V
 // rows are read once; every query row keeps an online softmax (running max, sum, weighted V) per warp.
 // ------------------------------------------------------------------------------------------------
-constexpr int ATT_CHUNK = 128;    // KV rows per CTA
+constexpr int ATT_CHUNK = ATT_CHUNK_ROWS;
 constexpr int ATT_TILE = 32;      // KV rows staged per iteration
 constexpr int ATT_WARPS = 8;
 
 template <typename T, int HD>
-__global__ void __launch_bounds__(ATT_WARPS * 32) tree_attn_kernel(const float* __restrict__ q, const T* __restrict__ kc,
+__global__ void __launch_bounds__(ATT_WARPS * 32) tree_attn_kernel(const T* __restrict__ q, const T* __restrict__ kc,
                                                                    const T* __restrict__ vc, RowSet rs,
                                                                    float* __restrict__ part_o, float* __restrict__ part_ml,
                                                                    int H, int max_seq, int nchunks) {
@@ -239,7 +259,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) tree_attn_kernel(const float* 
 
   for (int e = threadIdx.x; e < nr * HD; e += blockDim.x) {
     int i = e / HD, k = e % HD;
-    qs[i * HD + k] = q[((size_t)(b * rs.tc + i)) * d + h * HD + k] * scale;
+    qs[i * HD + k] = to_f<T>(q[((size_t)(b * rs.tc + i)) * d + h * HD + k]) * scale;
   }
   float m[RPW], l[RPW], o[RPW][KPL];
   uint64_t msk[RPW];
@@ -335,7 +355,7 @@ size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int
 }
 
 template <typename T, int HD>
-static hydra_status tree_attention_t(const float* q, const T* kc, const T* vc, RowSet rs, T* out, float* scratch, int H,
+static hydra_status tree_attention_t(const T* q, const T* kc, const T* vc, RowSet rs, T* out, float* scratch, int H,
                                      int max_seq, int len_upper, cudaStream_t st) {
   int nchunks_max = (max_seq + ATT_CHUNK - 1) / ATT_CHUNK;
   int nchunks = (len_upper + ATT_CHUNK - 1) / ATT_CHUNK;
@@ -358,17 +378,15 @@ static hydra_status tree_attention_t(const float* q, const T* kc, const T* vc, R
   return HYDRA_OK;
 }
 
-hydra_status tree_attention(const float* q, const void* kc, const void* vc, RowSet rs, void* out, void* scratch, int H,
+hydra_status tree_attention(const void* q, const void* kc, const void* vc, RowSet rs, void* out, void* scratch, int H,
                             int hd, int max_seq, int len_upper, int dtype, cudaStream_t st) {
   if (rs.tc > 64) return HYDRA_ERR_UNSUPPORTED;
+  if (dtype == 1)
+    return tree_attention_tc((const bf16*)q, (const bf16*)kc, (const bf16*)vc, rs, (bf16*)out, scratch, H, hd, max_seq, len_upper, st);
   if (dtype == 0 && hd == 64)
-    return tree_attention_t<float, 64>(q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
+    return tree_attention_t<float, 64>((const float*)q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
   if (dtype == 0 && hd == 128)
-    return tree_attention_t<float, 128>(q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
-  if (dtype == 1 && hd == 64)
-    return tree_attention_t<bf16, 64>(q, (const bf16*)kc, (const bf16*)vc, rs, (bf16*)out, (float*)scratch, H, max_seq, len_upper, st);
-  if (dtype == 1 && hd == 128)
-    return tree_attention_t<bf16, 128>(q, (const bf16*)kc, (const bf16*)vc, rs, (bf16*)out, (float*)scratch, H, max_seq, len_upper, st);
+    return tree_attention_t<float, 128>((const float*)q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
   return HYDRA_ERR_UNSUPPORTED;
 }
 

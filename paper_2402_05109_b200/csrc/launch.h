@@ -25,12 +25,16 @@ hydra_status residual_rmsnorm(const float* res, const float* part, size_t split_
                               cudaStream_t st);
 // table[r][j] = (cos, sin) of (pos0[b]+depth[i]) * theta^(-2j/head_dim), evaluated in double
 hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st);
-// q (float [rows][H][hd], rotated), K/V cache rows (rotated K) from the QKV partial sums.
-hydra_status qkv_rope_store(const float* part, size_t split_stride, int splits, const float2* table, float* q,
+// q (operand dtype, [rows][H][hd], rotated), K/V cache rows (rotated K) from the QKV partial sums.
+hydra_status qkv_rope_store(const float* part, size_t split_stride, int splits, const float2* table, void* q,
                             void* kcache, void* vcache, RowSet rs, int n_heads, int head_dim, int max_seq, int dtype,
                             int* status, cudaStream_t st);
+constexpr int ATT_CHUNK_ROWS = 128;     // KV rows per attention CTA (split-KV granularity)
 size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
-hydra_status tree_attention(const float* q, const void* kcache, const void* vcache, RowSet rs, void* out, void* scratch,
+// bfloat16 caches: tensor-core kernel (attention_tc.cu); float caches: SIMT kernel.  q is in the cache dtype.
+hydra_status tree_attention_tc(const bf16* q, const bf16* kc, const bf16* vc, RowSet rs, bf16* out, void* scratch, int n_heads,
+                               int head_dim, int max_seq, int len_upper, cudaStream_t st);
+hydra_status tree_attention(const void* q, const void* kcache, const void* vcache, RowSet rs, void* out, void* scratch,
                             int n_heads, int head_dim, int max_seq, int len_upper, int dtype, cudaStream_t st);
 hydra_status silu_mul(const float* part, size_t split_stride, int splits, void* act, int rows, int f, int dtype,
                       cudaStream_t st);

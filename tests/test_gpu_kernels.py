@@ -50,7 +50,7 @@ def test_tree_attention_matches_masked_softmax(dtype, hd):
     n_rows = [tc, tc, 17]                   # ragged row counts (rows beyond n_rows are ignored)
     kc = rnd((B, H, S, hd), 21, 1, dtype)
     vc = rnd((B, H, S, hd), 21, 2, dtype)
-    q = rnd((B * tc, H, hd), 21, 3, torch.float32)
+    q = rnd((B * tc, H, hd), 21, 3, dtype)
     mask = torch.tensor([a - (1 << 64) if a >= (1 << 63) else a for a in t.anc_mask], dtype=torch.int64)
     out = tree_attention(q.cuda(), kc.cuda(), vc.cuda(), torch.tensor(pos0, dtype=torch.int32).cuda(),
                          torch.tensor(n_rows, dtype=torch.int32).cuda(), mask.cuda(), tc).float().cpu().view(B, tc, H, hd)
@@ -59,6 +59,6 @@ def test_tree_attention_matches_masked_softmax(dtype, hd):
         allowed = torch.cat([torch.ones(n, pos0[b], dtype=torch.bool), t.allowed[:n, :n]], dim=1)
         k = kc[b, :, :L].permute(1, 0, 2).double()
         v = vc[b, :, :L].permute(1, 0, 2).double()
-        ref = masked_attention(q.view(B, tc, H, hd)[b, :n].double(), k, v, allowed)
+        ref = masked_attention(q.view(B, tc, H, hd)[b, :n].double(), k, v, allowed)   # q, k, v hold the rounded values
         err = float((out[b, :n].double() - ref).abs().max())
         assert err <= (2e-5 if dtype == torch.float32 else 2e-2), err
