@@ -135,8 +135,7 @@ enum {
   HYDRA_BUF_AMAX = 8,       /* int32 [batch][n_rows] */
   HYDRA_BUF_HEAD_LOGITS = 9,/* float [rows][vocab] logits of the last drafted level, row = b*parents+j */
   HYDRA_BUF_N_NEW = 10,     /* int32 [max_batch] rows in H_NEW */
-  HYDRA_BUF_H_PRIME = 11,   /* float [max_batch][d] hidden state the heads consumed */
-  HYDRA_BUF_LOGITS = 12     /* float [batch*n_rows][vocab] logits of the last verify */
+  HYDRA_BUF_H_PRIME = 11    /* float [max_batch][d] hidden state the heads consumed */
 };
 hydra_status hydra_get_buffer(hydra_ctx*, int which, void** dev_ptr, size_t* bytes);
 
@@ -164,25 +163,26 @@ const char* hydra_last_error(void); /* text of the last CUDA error seen by this 
 /* Single-kernel entry points for kernel-level parity tests.  No context; the library makes its own
  * tensor maps.  All pointers are device pointers.
  * hydra_gemm: out[m][n] = sum_k x[m][k] * w[n][k] (float accumulate, float out), dtype as above;
- *   n % 128 == 0 and k % 64 == 0 for mode 0.  splits >= 1 partial sums are reduced into out;
- *   partial_dev needs splits*m*n floats when splits > 1 (may be NULL when splits == 1).
+ *   n % 128 == 0 and k % 64 == 0 for mode 0.  partial_dev needs hydra_gemm_partial_floats(m, n, k, dtype, mode)
+ *   floats: the tensor-core GEMM leaves per-CTA partial sums there, which a second kernel adds in fixed order.
  *   mode as in hydra_set_gemm_mode; status_dev is an int32 status word (bit 1 bounds, bit 2 timeout).
  * hydra_tree_attention: q [rows][n_heads][head_dim] (dtype; rows = batch*tc), caches
  *   [batch][n_heads][max_seq][head_dim] (dtype), pos0 [batch] committed lengths, n_rows [batch] or
  *   NULL (= tc), mask [tc] ancestor bitmasks; out [rows][n_heads*head_dim] (dtype).  Row i of
  *   sequence b sees slots < pos0[b] and slot pos0[b]+j when bit j of mask[i] is set.  scratch_dev
  *   needs hydra_attention_scratch_bytes(...) bytes. */
+size_t hydra_gemm_partial_floats(int m, int n, int k, int dtype, int mode);
 hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, float* partial_dev, int m, int n, int k,
-                        int dtype, int splits, int mode, int32_t* status_dev, void* stream);
-/* hydra_gemm_noalloc: the bfloat16 tensor-core split-K GEMM of hydra_gemm (dtype 1, mode 0) for callers that
+                        int dtype, int mode, int32_t* status_dev, void* stream);
+/* hydra_gemm_noalloc: the bfloat16 tensor-core GEMM of hydra_gemm (dtype 1, mode 0) for callers that
  * may not allocate device memory.  (The paper has no counterpart; this is a convenience of the library.)
  * Serving loops that must stay clear of the allocator's locks and implicit synchronisation, plugins living
  * inside a host's fixed memory budget, and processes whose free memory already belongs to a pool cannot
  * supply hydra_gemm's partial_dev buffer; here the partial sums live in an 8 MiB array that is part of the
  * library image (every GPU that loads the library holds it until the process exits).
  *   - x [m][k], w [n][k] bfloat16, out [m][n] float, status_dev as in hydra_gemm: all caller-owned device
- *     memory; n % 128 == 0, k % 64 == 0, 1 <= splits <= k/64.
- *   - splits*m*n*4 bytes must fit in the 8 MiB array, otherwise HYDRA_ERR_CAPACITY (text in
+ *     memory; n % 128 == 0, k % 64 == 0.
+ *   - hydra_gemm_partial_floats(m, n, k, 1, 0) * 4 bytes must fit in the 8 MiB array, otherwise HYDRA_ERR_CAPACITY (text in
  *     hydra_last_error) and nothing is launched.
  *   - The call allocates nothing on the device.  The first call on each device looks up the array's device
  *     address (cudaGetSymbolAddress, with that device current); make that first call outside any stream
@@ -190,7 +190,7 @@ hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, fl
  *   - All calls on a GPU share the one array and it keeps the previous call's partial sums; the GEMM
  *     overwrites every element it later reads, so no clearing is needed, but two calls whose kernels overlap
  *     on the GPU (different streams, different threads) race on it: serialise them. */
-hydra_status hydra_gemm_noalloc(const void* x_dev, const void* w_dev, float* out_dev, int m, int n, int k, int splits,
+hydra_status hydra_gemm_noalloc(const void* x_dev, const void* w_dev, float* out_dev, int m, int n, int k,
                                 int32_t* status_dev, void* stream);
 size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
 hydra_status hydra_tree_attention(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev,

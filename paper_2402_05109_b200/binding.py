@@ -62,17 +62,19 @@ lib.hydra_get_timing.argtypes = [_vp, _i, C.POINTER(C.c_double), C.POINTER(C.c_l
 lib.hydra_status_str.restype = C.c_char_p
 lib.hydra_status_str.argtypes = [_i]
 lib.hydra_last_error.restype = C.c_char_p
-lib.hydra_gemm.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]
-lib.hydra_gemm_noalloc.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp]
+lib.hydra_gemm_partial_floats.restype = _sz
+lib.hydra_gemm_partial_floats.argtypes = [_i] * 5
+lib.hydra_gemm.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
+lib.hydra_gemm_noalloc.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]
 lib.hydra_attention_scratch_bytes.restype = _sz
 lib.hydra_attention_scratch_bytes.argtypes = [_i] * 5
 lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 6 + [_vp]
 
 BUF = dict(LEN=0, ROOT_TOK=1, H_TREE=2, H_NEW=3, KV_BASE=4, KV_PREFIX=5, TREE_MASK=6, TREE_TOK=7, AMAX=8,
-           HEAD_LOGITS=9, N_NEW=10, H_PRIME=11, LOGITS=12)
+           HEAD_LOGITS=9, N_NEW=10, H_PRIME=11)
 _BUF_DTYPE = dict(LEN=torch.int32, ROOT_TOK=torch.int32, H_TREE=torch.float32, H_NEW=torch.float32,
                   TREE_MASK=torch.int64, TREE_TOK=torch.int32, AMAX=torch.int32, HEAD_LOGITS=torch.float32,
-                  N_NEW=torch.int32, H_PRIME=torch.float32, LOGITS=torch.float32)
+                  N_NEW=torch.int32, H_PRIME=torch.float32)
 
 
 def _check(code: int, what: str):
@@ -223,15 +225,15 @@ class Hydra:
 
 
 # ---- single-kernel entry points (kernel-level parity tests)
-def gemm(x: torch.Tensor, w: torch.Tensor, splits: int = 1, mode: int = 0) -> torch.Tensor:
+def gemm(x: torch.Tensor, w: torch.Tensor, mode: int = 0) -> torch.Tensor:
     """out[m][n] = sum_k x[m][k] w[n][k] in float; x, w both float32 or both bfloat16 CUDA tensors."""
     m, k = x.shape
     n = w.shape[0]
     dtype = 0 if x.dtype == torch.float32 else 1
     out = torch.empty(m, n, dtype=torch.float32, device="cuda")
-    part = torch.empty(splits, m, n, dtype=torch.float32, device="cuda") if splits > 1 else None
+    part = torch.empty(lib.hydra_gemm_partial_floats(m, n, k, dtype, mode), dtype=torch.float32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    _check(lib.hydra_gemm(x.data_ptr(), w.data_ptr(), out.data_ptr(), _ptr(part), m, n, k, dtype, splits, mode,
+    _check(lib.hydra_gemm(x.data_ptr(), w.data_ptr(), out.data_ptr(), part.data_ptr(), m, n, k, dtype, mode,
                           status.data_ptr(), _stream()), "hydra_gemm")
     word = int(status.item())
     if word:
@@ -239,13 +241,13 @@ def gemm(x: torch.Tensor, w: torch.Tensor, splits: int = 1, mode: int = 0) -> to
     return out
 
 
-def gemm_noalloc(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor, status: torch.Tensor, splits: int):
-    """hydra_gemm_noalloc: split-K bfloat16 GEMM whose partial sums live in the library's built-in 8 MiB scratch.
+def gemm_noalloc(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor, status: torch.Tensor):
+    """hydra_gemm_noalloc: bfloat16 tensor-core GEMM whose partial sums live in the library's built-in 8 MiB scratch.
     The caller passes every tensor (nothing is allocated here, on the host side either): x [m][k], w [n][k]
     bfloat16, out [m][n] float32, status int32[1].  Calls that overlap on the GPU race on the scratch."""
     m, k = x.shape
     n = w.shape[0]
-    _check(lib.hydra_gemm_noalloc(x.data_ptr(), w.data_ptr(), out.data_ptr(), m, n, k, splits, status.data_ptr(), _stream()),
+    _check(lib.hydra_gemm_noalloc(x.data_ptr(), w.data_ptr(), out.data_ptr(), m, n, k, status.data_ptr(), _stream()),
            "hydra_gemm_noalloc")
 
 

@@ -46,6 +46,17 @@ __device__ __forceinline__ float warp_max(float v) {
 }
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
 
+// Where the partial sums of a GEMM output element live.  The tensor-core GEMM cuts the (tile, k-block) line
+// into ranges of q units per CTA; tile t = (m / mt) * n_tiles + n / 128 owns units [t*kb, (t+1)*kb), so its
+// partial sums sit in slots 0 .. split_count-1 (slot s at part + s*stride + m*N + n), one per CTA that
+// touched the tile, in CTA order.  A single-slot output is described by q = kb = 1.
+struct SplitDesc { int q, kb, n_tiles, mt; size_t stride; };
+__host__ __device__ __forceinline__ int split_count(const SplitDesc& sd, int m, int n) {
+  long long u0 = ((long long)(m / sd.mt) * sd.n_tiles + (n >> 7)) * sd.kb;
+  return (int)((u0 + sd.kb - 1) / sd.q - u0 / sd.q) + 1;
+}
+inline SplitDesc single_slot(size_t stride) { return SplitDesc{1, 1, 1, 1 << 30, stride}; }
+
 // Rows of one forward call: `batch` sequences with `tc` row slots each; sequence b uses its first
 // n_rows[b] slots (all tc when n_rows is null).  Row i of b has KV slot pos0[b]+i, rotary position
 // pos0[b]+depth[i] and may attend to cache slots < pos0[b] and to slot pos0[b]+j iff bit j of mask[i].

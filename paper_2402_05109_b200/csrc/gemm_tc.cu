@@ -1,18 +1,27 @@
-// Weight-streaming bfloat16 GEMM on the sm_100a tensor cores.
+// Weight-streaming bfloat16 GEMM on the sm_100a tensor cores: persistent, stream-K, TMA + tcgen05 + TMEM.
 //
-//   out[split][m][n] = sum_{k in split} x[m][k] * w[n][k]        (float accumulate, float out)
+//   part[slot][m][n] = sum over one K range of x[m][k] * w[n][k]        (float accumulate, float out)
 //
-// The weight matrix is the large operand (read once from HBM), the activation slab is small (tree rows
-// x batch) and L2 resident, so the roles are swapped with respect to the usual GEMM: a 128-row weight
-// tile [128 n][64 k] is the MMA "A" operand (M = 128 TMEM lanes), the activation tile [MT rows][64 k] is
-// the "B" operand (N = MT columns).  Both are K-major and land in shared memory through TMA with the
-// 128-byte swizzle; accumulators live in tensor memory.  One CTA computes one [128 n] x [MT m] tile for
-// one K range (split-K; partial sums are reduced by the consumer kernel, in fixed order).
+// The weight matrix is the large operand (read once from HBM); the activation slab is small (tree rows x
+// batch) and L2 resident.  So the roles are swapped with respect to the usual GEMM: a 128-row weight tile
+// [128 n][64 k] is the MMA "A" operand (M = 128 TMEM lanes), the activation tile [MT rows][64 k] is the "B"
+// operand (N = MT columns).  Both are K-major and land in shared memory through TMA with the 128-byte
+// swizzle; accumulators live in tensor memory.
 //
-// Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocation + MMA issue
-// (one lane), warps 2..5 = epilogue (TMEM -> registers -> global, coalesced along n).
-// Every mbarrier wait is bounded: when it runs out the CTA raises ST_TIMEOUT in the status word,
-// skips its stores, lets its copies settle, frees its tensor memory and returns.
+// Work decomposition (stream-K): the (tile, k-block) pairs of the whole GEMM are laid out in one line,
+// tile-major, and cut into equal contiguous ranges, one per CTA (at most one CTA per SM), so that every SM
+// streams the same number of weight bytes without interruption.  A CTA's range covers the tail of one tile,
+// possibly whole tiles, and the head of another; each such run is a "segment" whose partial sum goes to
+// slot (cta - first cta of the tile) of the partial buffer.  The consumer kernel adds the slots of a tile in
+// fixed order (SplitDesc), so results are deterministic.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocation + MMA issue (one
+// lane), warps 2..5 = epilogue (TMEM -> registers -> global, coalesced along n).  Two accumulator buffers in
+// TMEM let the epilogue of one segment overlap the main loop of the next.  The kernel is launched with
+// programmatic stream serialisation: weight tiles (which never depend on the preceding kernel) are requested
+// before griddepcontrol.wait, activations and all global writes after it.
+// Every mbarrier wait is bounded: when one runs out the CTA raises ST_TIMEOUT in the status word, stops
+// storing, lets its copies settle, frees its tensor memory and returns.
 #include "launch.h"
 #include <cuda.h>
 #include <map>
@@ -37,6 +46,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
     uint32_t ok;
@@ -51,10 +63,20 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   }
   return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
@@ -77,6 +99,8 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
@@ -108,36 +132,41 @@ template <int MT> struct TileCfg {
   static constexpr int B_BYTES = MT * BLOCK_K * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 10 ? 10 : (SMEM_BUDGET / STAGE_BYTES);
-  static constexpr int TMEM_COLS = MT < 32 ? 32 : MT;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int ACC_COLS = MT < 32 ? 32 : MT;             // columns of one accumulator buffer
+  static constexpr int TMEM_COLS = 2 * ACC_COLS;                  // two buffers (power of two, <= 512)
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/;
+};
+
+struct GemmArgs {
+  float* part; size_t slot_stride;
+  int m, n, kb, n_tiles, total_units, q;
+  int* status;
 };
 
 template <int MT>
 __global__ void __launch_bounds__(192, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, float* __restrict__ out,
-               size_t split_stride, int m, int n, int kblocks, int splits, int* status) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const GemmArgs a) {
   using C = TileCfg<MT>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bars = tiles + C::STAGES * C::STAGE_BYTES;          // full[S], empty[S], tmem_full, tmem slot
-  auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (C::STAGES + s); };
-  const uint32_t tmem_full_bar = bars + 8u * (2 * C::STAGES);
-  const uint32_t tmem_slot = bars + 8u * (2 * C::STAGES + 1);
+  const uint32_t bars = tiles + C::STAGES * C::STAGE_BYTES;
+  auto fullw_bar = [&](int s) { return bars + 8u * s; };
+  auto fullx_bar = [&](int s) { return bars + 8u * (C::STAGES + s); };
+  auto empty_bar = [&](int s) { return bars + 8u * (2 * C::STAGES + s); };
+  auto accfull_bar = [&](int i) { return bars + 8u * (3 * C::STAGES + i); };
+  auto accempty_bar = [&](int i) { return bars + 8u * (3 * C::STAGES + 2 + i); };
+  const uint32_t tmem_slot = bars + 8u * (3 * C::STAGES + 4);
   __shared__ int s_abort;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * BLOCK_N;
-  const int split = blockIdx.y;
-  const int m0 = blockIdx.z * MT;
-  const int kb_begin = (int)(((long long)split * kblocks) / splits);
-  const int kb_end = (int)(((long long)(split + 1) * kblocks) / splits);
-  const int nkb = kb_end - kb_begin;
+  const int u_begin = blockIdx.x * a.q;
+  const int u_end = min(u_begin + a.q, a.total_units);
+  const int n_units = u_end - u_begin;
 
   if (threadIdx.x == 0) {
     s_abort = 0;
-    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    mbar_init(tmem_full_bar, 1);
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(fullw_bar(s), 1); mbar_init(fullx_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(accfull_bar(i), 1); mbar_init(accempty_bar(i), 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
@@ -146,56 +175,105 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  grid_dep_launch();                       // all CTAs of this grid are resident: let the next kernel get ready
   uint32_t tmem_base;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 
   if (warp == 0) {
     if (lane == 0) {
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % C::STAGES;
-        const uint32_t ph = (kb / C::STAGES) & 1;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u)) { atomicOr(status, ST_TIMEOUT); s_abort = 1; break; }
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      auto coords = [&](int u, int& kcol, int& nrow, int& mrow) {
+        const int tile = u / a.kb;
+        kcol = (u - tile * a.kb) * BLOCK_K;
+        nrow = (tile % a.n_tiles) * BLOCK_N;
+        mrow = (tile / a.n_tiles) * MT;
+      };
+      // weights do not depend on the preceding kernel: request the first ring of weight tiles right away
+      const int pre = n_units < C::STAGES ? n_units : C::STAGES;
+      for (int i = 0; i < pre; ++i) {
+        int kcol, nrow, mrow;
+        coords(u_begin + i, kcol, nrow, mrow);
+        mbar_arrive_expect_tx(fullw_bar(i), A_BYTES);
+        tma_load_2d(tiles + i * C::STAGE_BYTES, &tmW, kcol, nrow, fullw_bar(i), pol_w);
+      }
+      grid_dep_wait();                     // activations are the preceding kernel's output
+      for (int i = 0; i < n_units; ++i) {
+        const int s = i % C::STAGES;
+        const uint32_t ph = (i / C::STAGES) & 1;
+        int kcol, nrow, mrow;
+        coords(u_begin + i, kcol, nrow, mrow);
         const uint32_t a_dst = tiles + s * C::STAGE_BYTES;
-        mbar_arrive_expect_tx(full_bar(s), C::STAGE_BYTES);
-        tma_load_2d(a_dst, &tmW, (kb_begin + kb) * BLOCK_K, n0, full_bar(s));
-        tma_load_2d(a_dst + A_BYTES, &tmX, (kb_begin + kb) * BLOCK_K, m0, full_bar(s));
+        if (i >= pre) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u)) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
+          mbar_arrive_expect_tx(fullw_bar(s), A_BYTES);
+          tma_load_2d(a_dst, &tmW, kcol, nrow, fullw_bar(s), pol_w);
+        }
+        mbar_arrive_expect_tx(fullx_bar(s), C::B_BYTES);
+        tma_load_2d(a_dst + A_BYTES, &tmX, kcol, mrow, fullx_bar(s), pol_x);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc(MT);
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % C::STAGES;
-        const uint32_t ph = (kb / C::STAGES) & 1;
-        if (!mbar_wait(full_bar(s), ph)) { atomicOr(status, ST_TIMEOUT); s_abort = 1; break; }
+      int seg = 0;
+      bool ok = true;
+      for (int i = 0; i < n_units && ok;) {
+        const int u = u_begin + i;
+        const int tile = u / a.kb;
+        const int seg_len = min((tile + 1) * a.kb, u_end) - u;
+        const int acc = seg & 1;
+        const uint32_t acc_ph = (seg >> 1) & 1;
+        if (!mbar_wait(accempty_bar(acc), acc_ph ^ 1u)) { ok = false; break; }      // epilogue has drained this buffer
         tc_fence_after();
-        const uint32_t a_addr = tiles + s * C::STAGE_BYTES;
-        const uint64_t adesc = smem_desc_sw128(a_addr);
-        const uint64_t bdesc = smem_desc_sw128(a_addr + A_BYTES);
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * C::ACC_COLS);
+        for (int j = 0; j < seg_len; ++j, ++i) {
+          const int s = i % C::STAGES;
+          const uint32_t ph = (i / C::STAGES) & 1;
+          if (!mbar_wait(fullw_bar(s), ph) || !mbar_wait(fullx_bar(s), ph)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = tiles + s * C::STAGE_BYTES;
+          const uint64_t adesc = smem_desc_sw128(a_addr);
+          const uint64_t bdesc = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
-        for (int k = 0; k < BLOCK_K / 16; ++k)           // 16 bf16 = 32 bytes per MMA: +2 in 16-byte units
-          umma_bf16(tmem_base, adesc + 2u * k, bdesc + 2u * k, idesc, (uint32_t)((kb | k) != 0));
-        umma_commit(empty_bar(s));                       // frees the stage once these MMAs have read it
+          for (int k = 0; k < BLOCK_K / 16; ++k)         // 16 bf16 = 32 bytes per MMA: +2 in 16-byte units
+            umma_bf16(tmem_d, adesc + 2u * k, bdesc + 2u * k, idesc, (uint32_t)((j | k) != 0));
+          umma_commit(empty_bar(s));                     // frees the stage once these MMAs have read it
+        }
+        if (!ok) break;
+        umma_commit(accfull_bar(acc));                   // segment complete: hand the accumulator to the epilogue
+        ++seg;
       }
-      umma_commit(tmem_full_bar);
+      if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
     }
   } else {
     const int quarter = warp & 3;                        // TMEM lanes this warp may read
-    bool ok = nkb > 0 && mbar_wait(tmem_full_bar, 0);
-    if (!ok && lane == 0) atomicOr(status, ST_TIMEOUT);
-    tc_fence_after();
-    if (ok && !s_abort) {
-      const int col_n = n0 + quarter * 32 + lane;
-      float* dst = out + (size_t)split * split_stride + col_n;
+    grid_dep_wait();                                     // the partial buffer may still be read by the preceding kernel
+    int seg = 0;
+    for (int i = 0; i < n_units;) {
+      const int u = u_begin + i;
+      const int tile = u / a.kb;
+      const int seg_len = min((tile + 1) * a.kb, u_end) - u;
+      const int acc = seg & 1;
+      const uint32_t acc_ph = (seg >> 1) & 1;
+      if (!mbar_wait(accfull_bar(acc), acc_ph)) { if (lane == 0) atomicOr(a.status, ST_TIMEOUT); break; }
+      tc_fence_after();
+      const int slot = blockIdx.x - (int)(((long long)tile * a.kb) / a.q);
+      const int n0 = (tile % a.n_tiles) * BLOCK_N, m0 = (tile / a.n_tiles) * MT;
+      float* dst = a.part + (size_t)slot * a.slot_stride + n0 + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * C::ACC_COLS);
 #pragma unroll 1
       for (int c = 0; c < MT; c += 16) {
-        if (m0 + c >= m) break;
+        if (m0 + c >= a.m) break;
         uint32_t r[16];
-        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, r);
+        tmem_ld16(taddr + (uint32_t)c, r);
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-          if (m0 + c + j < m) dst[(size_t)(m0 + c + j) * n] = __uint_as_float(r[j]);
+          if (m0 + c + j < a.m) dst[(size_t)(m0 + c + j) * a.n] = __uint_as_float(r[j]);
       }
+      tc_fence_before();
+      if (lane == 0) mbar_arrive(accempty_bar(acc));
+      i += seg_len;
+      ++seg;
     }
   }
   tc_fence_before();
@@ -249,17 +327,31 @@ bool get_tensor_map(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_
   return true;
 }
 
+int sm_count() {
+  static int n = []() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1)
+      return 148;
+    return v;
+  }();
+  return n;
+}
+
 template <int MT>
-hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, float* out, size_t split_stride, int m, int n, int k,
-                    int splits, int* status, cudaStream_t st) {
+hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs& a, int grid, cudaStream_t st) {
   using C = TileCfg<MT>;
   static bool attr_done = false;
   if (!attr_done) {
     HYDRA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_done = true;
   }
-  dim3 grid(n / BLOCK_N, splits, (m + MT - 1) / MT);
-  gemm_tc_kernel<MT><<<grid, 192, C::SMEM_BYTES, st>>>(tw, tx, out, split_stride, m, n, k / BLOCK_K, splits, status);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = C::SMEM_BYTES; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<MT>, tw, tx, a));
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -268,25 +360,52 @@ hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, float* out, si
 
 bool gemm_tc_available() { return encode_fn() != nullptr; }
 
-hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* out, size_t split_stride, int m, int n, int k,
-                     int splits, int* status, cudaStream_t st) {
-  if (m <= 0 || n <= 0 || k <= 0 || n % BLOCK_N || k % BLOCK_K || splits < 1) return HYDRA_ERR_UNSUPPORTED;
+int gemm_tile_rows(int m) { return m <= 16 ? 16 : m <= 32 ? 32 : m <= 64 ? 64 : m <= 128 ? 128 : 256; }
+
+// Stream-K plan: equal contiguous unit ranges, one per CTA, at most one CTA per SM and at least 4 k-blocks each.
+SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots) {
+  SplitDesc sd{};
+  const int mt = gemm_tile_rows(m);
+  sd.mt = mt; sd.n_tiles = n / BLOCK_N; sd.kb = k / BLOCK_K; sd.stride = (size_t)m * n;
+  const int tiles = sd.n_tiles * ((m + mt - 1) / mt);
+  const long long total = (long long)tiles * sd.kb;
+  long long g = sm_count();
+  if (g > total / 4) g = total / 4 > 0 ? total / 4 : 1;
+  sd.q = (int)((total + g - 1) / g);
+  if (grid) *grid = (int)((total + sd.q - 1) / sd.q);
+  if (max_slots) {
+    int mx = 1;
+    for (int t = 0; t < tiles; ++t) {
+      long long u0 = (long long)t * sd.kb;
+      int ns = (int)((u0 + sd.kb - 1) / sd.q - u0 / sd.q) + 1;
+      mx = ns > mx ? ns : mx;
+    }
+    *max_slots = mx;
+  }
+  return sd;
+}
+
+hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part, int m, int n, int k, SplitDesc* sd_out,
+                     int* status, cudaStream_t st) {
+  if (m <= 0 || n <= 0 || k <= 0 || n % BLOCK_N || k % BLOCK_K) return HYDRA_ERR_UNSUPPORTED;
   if (((uintptr_t)x | (uintptr_t)w) & 15) return HYDRA_ERR_INVALID;
-  if (splits > k / BLOCK_K) return HYDRA_ERR_INVALID;
-  int mt = m <= 16 ? 16 : m <= 32 ? 32 : m <= 64 ? 64 : m <= 128 ? 128 : 256;
+  int grid = 1;
+  SplitDesc sd = gemm_tc_plan(m, n, k, &grid, nullptr);
   if (x_rows_alloc < m) x_rows_alloc = m;
   CUtensorMap tw, tx;
   if (!get_tensor_map(w, (uint64_t)n, (uint64_t)k, BLOCK_N, &tw) ||
-      !get_tensor_map(x, (uint64_t)x_rows_alloc, (uint64_t)k, (uint32_t)mt, &tx)) {
+      !get_tensor_map(x, (uint64_t)x_rows_alloc, (uint64_t)k, (uint32_t)sd.mt, &tx)) {
     set_last_error("cuTensorMapEncodeTiled", cudaErrorUnknown);
     return HYDRA_ERR_CUDA;
   }
-  switch (mt) {
-    case 16: return launch<16>(tw, tx, out, split_stride, m, n, k, splits, status, st);
-    case 32: return launch<32>(tw, tx, out, split_stride, m, n, k, splits, status, st);
-    case 64: return launch<64>(tw, tx, out, split_stride, m, n, k, splits, status, st);
-    case 128: return launch<128>(tw, tx, out, split_stride, m, n, k, splits, status, st);
-    default: return launch<256>(tw, tx, out, split_stride, m, n, k, splits, status, st);
+  GemmArgs a{part, sd.stride, m, n, sd.kb, sd.n_tiles, sd.n_tiles * ((m + sd.mt - 1) / sd.mt) * sd.kb, sd.q, status};
+  if (sd_out) *sd_out = sd;
+  switch (sd.mt) {
+    case 16: return launch<16>(tw, tx, a, grid, st);
+    case 32: return launch<32>(tw, tx, a, grid, st);
+    case 64: return launch<64>(tw, tx, a, grid, st);
+    case 128: return launch<128>(tw, tx, a, grid, st);
+    default: return launch<256>(tw, tx, a, grid, st);
   }
 }
 

@@ -31,23 +31,7 @@ struct Bump {                      // 256-byte aligned bump allocator; base == n
   }
 };
 
-int tile_rows(int m) { return m <= 16 ? 16 : m <= 32 ? 32 : m <= 64 ? 64 : m <= 128 ? 128 : 256; }
-int pad_rows(int m) { int t = tile_rows(m); return (m + t - 1) / t * t; }
-
-// Split-K factor: spread a GEMM with few n-tiles over the SMs.  Cost model: waves x (k-blocks per CTA +
-// a fixed per-CTA ramp), in units of one 64-wide k-block.
-int choose_splits(int m, int n, int k) {
-  int mt = tile_rows(m);
-  int tiles = (n / 128) * ((m + mt - 1) / mt);
-  int kb = k / 64;
-  int best = 1; double best_cost = 1e30;
-  for (int s = 1; s <= 16 && s * 2 <= kb; ++s) {
-    double waves = (double)((tiles * s + 147) / 148);
-    double cost = waves * ((kb + s - 1) / s + 6);
-    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
-  }
-  return best;
-}
+int pad_rows(int m) { int t = gemm_tile_rows(m); return (m + t - 1) / t * t; }
 
 enum State { ST_CREATED = 0, ST_READY = 1, ST_DRAFTED = 2, ST_VERIFIED = 3 };
 
@@ -76,7 +60,7 @@ struct hydra_ctx {
   int *d_len, *d_n_new, *d_root_tok, *d_status, *d_pos0, *d_nrows, *d_prompt_len, *d_offsets, *d_tok, *d_tree_tok, *d_amax;
   unsigned int* d_done;
   char *kv_base, *kv_pfx;
-  float *x, *part, *h_tree, *logits, *h_new, *hprime, *y, *head_logits;
+  float *x, *part, *h_tree, *h_new, *hprime, *y, *head_logits;
   float2* rope;
   void *q, *xn, *attn_out, *act, *z, *yb, *att_scratch;
   size_t part_floats;
@@ -158,23 +142,24 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   const int d = m.d_model, f = m.d_ffn, V = m.vocab, K = h.n_heads, T = t.T;
   const int R = pad_rows(m.max_batch * CHUNK);
   const int RH = pad_rows(m.max_batch * t.maxP);
-  // largest split-K partial buffer over every GEMM shape and row count the library issues
+  // largest partial-sum buffer over every GEMM shape and row count the library issues
   size_t part_floats = 0;
   {
-    const int shapes[][2] = {{3 * d, d}, {d, d}, {2 * f, d}, {d, f}};
-    const int row_counts[] = {m.max_batch * CHUNK, m.max_batch * T, m.max_batch * (K + 1)};
-    for (auto& s : shapes)
-      for (int rows : row_counts)
-        for (int bb = 1; bb <= m.max_batch; ++bb) {
-          int mm = rows / m.max_batch * bb;
-          int sp = m.dtype == 1 ? choose_splits(mm, s[0], s[1]) : 1;
-          part_floats = std::max(part_floats, (size_t)sp * mm * s[0]);
-        }
-    for (int i = 1; i <= K; ++i)
-      for (int mm = 1; mm <= m.max_batch * t.maxP; ++mm) {
-        int sp1 = m.dtype == 1 ? choose_splits(mm, d, (i + 1) * d) : 1, sp2 = m.dtype == 1 ? choose_splits(mm, d, d) : 1;
-        part_floats = std::max(part_floats, (size_t)std::max(sp1, sp2) * mm * d);
-      }
+    auto need = [&](int mm, int n, int k) {
+      int slots = 1;
+      if (m.dtype == 1) gemm_tc_plan(mm, n, k, nullptr, &slots);
+      part_floats = std::max(part_floats, (size_t)slots * mm * n);
+    };
+    const int shapes[][2] = {{3 * d, d}, {d, d}, {2 * f, d}, {d, f}, {V, d}};
+    const int per_seq[] = {CHUNK, T, K + 1, 1};
+    for (auto& sh : shapes)
+      for (int rows : per_seq)
+        for (int bb = 1; bb <= m.max_batch; ++bb) need(rows * bb, sh[0], sh[1]);
+    for (int mm = 1; mm <= m.max_batch * t.maxP; ++mm) {
+      for (int i = 1; i <= K; ++i) need(mm, d, (i + 1) * d);
+      need(mm, d, d);
+      need(mm, V, d);
+    }
   }
   auto* parent = b.take<int>(T); auto* depth = b.take<int>(T); auto* fc = b.take<int>(T); auto* nc = b.take<int>(T);
   auto* path_tab = b.take<int>((size_t)T * (K + 1)); auto* chain_depth = b.take<int>(CHUNK);
@@ -191,7 +176,6 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)R * d * es);
   auto* part = b.take<float>(part_floats);
   auto* h_tree = b.take<float>((size_t)R * d);
-  auto* logits = b.take<float>((size_t)pad_rows(m.max_batch * T) * V);
   auto* h_new = b.take<float>((size_t)pad_rows(m.max_batch * (K + 1)) * d);
   auto* hprime = b.take<float>((size_t)m.max_batch * d);
   auto* y = b.take<float>((size_t)RH * d); auto* head_logits = b.take<float>((size_t)RH * V);
@@ -206,7 +190,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
     c->d_chain_depth = chain_depth; c->d_anc = anc; c->d_chain_mask = chain_mask; c->d_level_parents = lvl;
     c->d_len = len; c->d_n_new = n_new; c->d_root_tok = root; c->d_status = status; c->d_pos0 = pos0; c->d_nrows = nrows;
     c->d_prompt_len = plen; c->d_offsets = offs; c->d_tok = tok; c->d_tree_tok = tree_tok; c->d_amax = amax; c->d_done = done;
-    c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits;
+    c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree;
     c->h_new = h_new; c->hprime = hprime; c->y = y; c->head_logits = head_logits; c->rope = rope; c->xn = xn;
     c->attn_out = attn_out; c->act = act; c->z = z; c->yb = yb; c->att_scratch = att;
   }
@@ -224,24 +208,21 @@ struct TimeScope {                // brackets the launches issued during its lif
   ~TimeScope() { if (a) { cudaEventRecord(b, st); c->timed.push_back({a, b, cls, bytes}); } }
 };
 
-// out = x @ w^T into c->part (split-K partial sums) or, when direct_out is given, straight into it (no split).
-hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void* w, int m, int n, int k, float* direct_out,
-                      int* splits, size_t* stride, cudaStream_t st) {
-  float* out = direct_out ? direct_out : c->part;
-  *stride = (size_t)m * n;
-  int sp = 1;
-  if (c->m.dtype == 1 && c->gemm_mode == 0 && !direct_out) {
-    sp = choose_splits(m, n, k);
-    if ((size_t)sp * m * n > c->part_floats) sp = 1;
-  }
-  // algorithmic bytes of the launch: the weight matrix and the activation slab read once, the output written once
-  TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * sp * m * n, st);
+// Partial sums of x @ w^T into c->part; *sd says where the slots of each output tile are.
+hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void* w, int m, int n, int k, SplitDesc* sd,
+                      cudaStream_t st) {
   if (c->m.dtype == 1 && c->gemm_mode == 0) {
-    *splits = sp;
-    return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, out, *stride, m, n, k, sp, c->d_status, st);
+    int slots = 1;
+    SplitDesc plan = gemm_tc_plan(m, n, k, nullptr, &slots);
+    if ((size_t)slots * m * n > c->part_floats) return HYDRA_ERR_CAPACITY;
+    // algorithmic bytes of the launch: the weight matrix and the activation slab read once, the partial sums written once
+    TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * m * n, st);
+    (void)plan;
+    return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, c->part, m, n, k, sd, c->d_status, st);
   }
-  *splits = 1;
-  return gemm_simt(x, w, out, m, n, k, c->m.dtype, st);
+  TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * m * n, st);
+  *sd = single_slot((size_t)m * n);
+  return gemm_simt(x, w, c->part, m, n, k, c->m.dtype, st);
 }
 
 // One decoder layer over the rows of `rs`.  Expects the residual rows in c->x and their normed copy in c->xn.
@@ -250,19 +231,19 @@ hydra_status run_layer(hydra_ctx* c, const LayerW& w, char* kc, char* vc, const 
                        const void* next_gain, float* hn, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int rows = rs.batch * rs.tc, d = m.d_model, f = m.d_ffn, dt = m.dtype;
-  int sp; size_t stride;
-  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.wqkv, rows, 3 * d, d, nullptr, &sp, &stride, st));
-  HYDRA_TRY(qkv_rope_store(c->part, stride, sp, c->rope, c->q, kc, vc, rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
+  SplitDesc sd;
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.wqkv, rows, 3 * d, d, &sd, st));
+  HYDRA_TRY(qkv_rope_store(c->part, sd, c->rope, c->q, kc, vc, rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
   {
     TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
     HYDRA_TRY(tree_attention(c->q, kc, vc, rs, c->attn_out, c->att_scratch, m.n_heads, m.head_dim, m.max_seq, len_upper, dt, st));
   }
-  HYDRA_TRY(run_gemm(c, c->attn_out, c->R, w.wo, rows, d, d, nullptr, &sp, &stride, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, c->part, stride, sp, c->x, w.ffn_norm, c->xn, nullptr, rows, d, m.rms_eps, dt, st));
-  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, nullptr, &sp, &stride, st));
-  HYDRA_TRY(silu_mul(c->part, stride, sp, c->act, rows, f, dt, st));
-  HYDRA_TRY(run_gemm(c, c->act, c->R, w.w_down, rows, d, f, nullptr, &sp, &stride, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, c->part, stride, sp, c->x, next_gain, next_gain ? c->xn : nullptr, hn, rows, d, m.rms_eps, dt, st));
+  HYDRA_TRY(run_gemm(c, c->attn_out, c->R, w.wo, rows, d, d, &sd, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, c->part, sd, c->x, w.ffn_norm, c->xn, nullptr, rows, d, m.rms_eps, dt, st));
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, &sd, st));
+  HYDRA_TRY(silu_mul(c->part, sd, c->act, rows, f, dt, st));
+  HYDRA_TRY(run_gemm(c, c->act, c->R, w.w_down, rows, d, f, &sd, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, c->part, sd, c->x, next_gain, next_gain ? c->xn : nullptr, hn, rows, d, m.rms_eps, dt, st));
   return HYDRA_OK;
 }
 
@@ -274,7 +255,7 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
   const size_t kvl = kv_layer_elems(m) * c->esize;
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
   HYDRA_TRY(embed_rows(c->embed, tok, c->x, rows, m.d_model, m.vocab, m.dtype, c->d_status, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, nullptr, 0, 0, c->x, c->layers[0].attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, nullptr, single_slot(0), c->x, c->layers[0].attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
   for (int l = 0; l < m.n_layers; ++l) {
     bool last = l + 1 == m.n_layers;
     HYDRA_TRY(run_layer(c, c->layers[l], c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs, len_upper,
@@ -289,7 +270,7 @@ hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int le
   const int rows = rs.batch * rs.tc;
   const size_t kvl = kv_layer_elems(m) * c->esize;
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
-  HYDRA_TRY(residual_rmsnorm(src, nullptr, 0, 0, c->x, c->pfx.attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
+  HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
   return run_layer(c, c->pfx, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, nullptr, nullptr, st);
 }
 
@@ -312,17 +293,17 @@ hydra_status do_draft(hydra_ctx* c, int* tree_tok, cudaStream_t st) {
     const int rows = B * P;
     LevelDesc lv{lvl, P, c->d_level_parents[lvl - 1]};
     HYDRA_TRY(head_gather(c->hprime, c->embed, c->d_root_tok, tree_tok, c->d_path_tab, lv, c->z, B, c->T, K + 1, d, m.vocab, dt, c->d_status, st));
-    int sp; size_t stride;
-    HYDRA_TRY(run_gemm(c, c->z, c->RH, c->head_w1[lvl - 1], rows, d, (lvl + 1) * d, nullptr, &sp, &stride, st));
-    HYDRA_TRY(head_act(c->hprime, 1, P, c->part, stride, sp, c->h.has_bias ? c->head_b1[lvl - 1] : nullptr, c->y, c->yb, rows, d, dt, st));
+    SplitDesc sd;
+    HYDRA_TRY(run_gemm(c, c->z, c->RH, c->head_w1[lvl - 1], rows, d, (lvl + 1) * d, &sd, st));
+    HYDRA_TRY(head_act(c->hprime, 1, P, c->part, sd, c->h.has_bias ? c->head_b1[lvl - 1] : nullptr, c->y, c->yb, rows, d, dt, st));
     for (int l = 0; l + 1 < c->h.n_mlp_layers; ++l) {
       const char* wr = (const char*)c->head_wr[lvl - 1] + (size_t)l * d * d * c->esize;
       const char* br = c->h.has_bias ? (const char*)c->head_br[lvl - 1] + (size_t)l * d * c->esize : nullptr;
-      HYDRA_TRY(run_gemm(c, c->yb, c->RH, wr, rows, d, d, nullptr, &sp, &stride, st));
-      HYDRA_TRY(head_act(c->y, 0, P, c->part, stride, sp, br, c->y, c->yb, rows, d, dt, st));
+      HYDRA_TRY(run_gemm(c, c->yb, c->RH, wr, rows, d, d, &sd, st));
+      HYDRA_TRY(head_act(c->y, 0, P, c->part, sd, br, c->y, c->yb, rows, d, dt, st));
     }
-    HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, rows, m.vocab, d, c->head_logits, &sp, &stride, st));
-    HYDRA_TRY(topk_children(c->head_logits, lv, c->d_first_child, c->d_n_child, tree_tok, B, c->T, m.vocab, st));
+    HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, rows, m.vocab, d, &sd, st));
+    HYDRA_TRY(topk_children(c->part, sd, c->head_logits, lv, c->d_first_child, c->d_n_child, tree_tok, B, c->T, m.vocab, st));
   }
   return HYDRA_OK;
 }
@@ -332,10 +313,9 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
   const int rows = c->batch * c->T;
   RowSet rs{c->batch, c->T, nullptr, c->d_len, c->d_depth, c->d_anc};
   HYDRA_TRY(run_base(c, tree_tok, rs, max_len_ub(c) + c->T, st));
-  int sp; size_t stride;
-  float* lg = logits ? logits : c->logits;
-  HYDRA_TRY(run_gemm(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, lg, &sp, &stride, st));
-  return argmax_rows(lg, amax, rows, m.vocab, st);
+  SplitDesc sd;
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, &sd, st));
+  return argmax_rows(c->part, sd, logits, amax, rows, m.vocab, st);
 }
 
 hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* n_acc, int* path, int* out_tok, cudaStream_t st) {
@@ -474,9 +454,9 @@ hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const
   // root token = argmax of the logits of the last prompt row
   HYDRA_TRY(pick_last_row(c->h_new, c->d_n_new, c->h.n_heads + 1, c->hprime, batch, m.d_model, st));
   HYDRA_TRY(cast_rows(c->hprime, c->yb, (size_t)batch * m.d_model, m.dtype, st));
-  int sp; size_t stride;
-  HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, batch, m.vocab, m.d_model, c->head_logits, &sp, &stride, st));
-  HYDRA_TRY(argmax_rows(c->head_logits, c->d_root_tok, batch, m.vocab, st));
+  SplitDesc sd;
+  HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, batch, m.vocab, m.d_model, &sd, st));
+  HYDRA_TRY(argmax_rows(c->part, sd, nullptr, c->d_root_tok, batch, m.vocab, st));
   for (int b = 0; b < batch; ++b) c->len_ub[b] = plen[b];
   c->state = ST_READY;
   return HYDRA_OK;
@@ -550,7 +530,6 @@ hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes
     case HYDRA_BUF_HEAD_LOGITS: p = c->head_logits; n = (size_t)c->RH * m.vocab * sizeof(float); break;
     case HYDRA_BUF_N_NEW: p = c->d_n_new; n = m.max_batch * sizeof(int); break;
     case HYDRA_BUF_H_PRIME: p = c->hprime; n = (size_t)m.max_batch * m.d_model * sizeof(float); break;
-    case HYDRA_BUF_LOGITS: p = c->logits; n = (size_t)m.max_batch * c->T * m.vocab * sizeof(float); break;
     default: return HYDRA_ERR_INVALID;
   }
   *ptr = p;
@@ -619,20 +598,26 @@ const char* hydra_status_str(hydra_status s) {
 
 const char* hydra_last_error(void) { return g_err; }
 
-hydra_status hydra_gemm(const void* x, const void* w, float* out, float* partial, int m, int n, int k, int dtype, int splits,
-                        int mode, int32_t* status, void* stream) {
-  if (!x || !w || !out || m < 1 || n < 1 || k < 1 || splits < 1 || (dtype != 0 && dtype != 1)) return HYDRA_ERR_INVALID;
+size_t hydra_gemm_partial_floats(int m, int n, int k, int dtype, int mode) {
+  if (m < 1 || n < 1 || k < 1) return 0;
+  if (dtype != 1 || mode != 0 || n % 128 || k % 64) return (size_t)m * n;
+  int slots = 1;
+  gemm_tc_plan(m, n, k, nullptr, &slots);
+  return (size_t)slots * m * n;
+}
+
+hydra_status hydra_gemm(const void* x, const void* w, float* out, float* partial, int m, int n, int k, int dtype, int mode,
+                        int32_t* status, void* stream) {
+  if (!x || !w || !out || !partial || m < 1 || n < 1 || k < 1 || (dtype != 0 && dtype != 1)) return HYDRA_ERR_INVALID;
   cudaStream_t st = (cudaStream_t)stream;
   CounterScope cs(nullptr);
   if (dtype == 1 && mode == 0) {
     if (!status) return HYDRA_ERR_INVALID;
     if (!gemm_tc_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
-    if (splits == 1) return gemm_tc((const bf16*)x, m, (const bf16*)w, out, (size_t)m * n, m, n, k, 1, status, st);
-    if (!partial) return HYDRA_ERR_INVALID;
-    HYDRA_TRY(gemm_tc((const bf16*)x, m, (const bf16*)w, partial, (size_t)m * n, m, n, k, splits, status, st));
-    return reduce_splits(partial, (size_t)m * n, splits, out, (size_t)m * n, st);
+    SplitDesc sd;
+    HYDRA_TRY(gemm_tc((const bf16*)x, m, (const bf16*)w, partial, m, n, k, &sd, status, st));
+    return reduce_splits(partial, sd, out, m, n, st);
   }
-  if (splits != 1) return HYDRA_ERR_UNSUPPORTED;
   return gemm_simt(x, w, out, m, n, k, dtype, st);
 }
 

@@ -59,16 +59,16 @@ hydra_status gemm_simt(const void* x, const void* w, float* out, int m, int n, i
   return HYDRA_OK;
 }
 
-__global__ void reduce_splits_kernel(const float* __restrict__ part, size_t stride, int splits, float* __restrict__ out,
-                                     size_t count) {
+__global__ void reduce_splits_kernel(const float* __restrict__ part, SplitDesc sd, float* __restrict__ out, int m, int n) {
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= count) return;
+  if (i >= (size_t)m * n) return;
+  const int ns = split_count(sd, (int)(i / n), (int)(i % n));
   float s = 0.f;
-  for (int p = 0; p < splits; ++p) s += part[p * stride + i];
+  for (int p = 0; p < ns; ++p) s += part[p * sd.stride + i];
   out[i] = s;
 }
-hydra_status reduce_splits(const float* part, size_t stride, int splits, float* out, size_t count, cudaStream_t st) {
-  reduce_splits_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(part, stride, splits, out, count);
+hydra_status reduce_splits(const float* part, SplitDesc sd, float* out, int m, int n, cudaStream_t st) {
+  reduce_splits_kernel<<<(unsigned)(((size_t)m * n + 255) / 256), 256, 0, st>>>(part, sd, out, m, n);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -125,7 +125,7 @@ template <> __device__ __forceinline__ float4 load4<bf16>(const bf16* p) {
 constexpr int NORM_THREADS = 512;
 template <typename T>
 __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const float* res, const float* __restrict__ part,
-                                                                        size_t stride, int splits, float* x_out,
+                                                                        SplitDesc sd, float* x_out,
                                                                         const T* __restrict__ gain, T* __restrict__ xn,
                                                                         float* __restrict__ hn, int d, float eps) {
   __shared__ float sh[32];
@@ -133,11 +133,13 @@ __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const fl
   float ss = 0.f;
   for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
     float4 v = res ? *reinterpret_cast<const float4*>(res + base + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-    if (part)
-      for (int p = 0; p < splits; ++p) {
-        float4 a = *reinterpret_cast<const float4*>(part + p * stride + base + i);
+    if (part) {
+      const int ns = split_count(sd, (int)blockIdx.x, i);
+      for (int p = 0; p < ns; ++p) {
+        float4 a = *reinterpret_cast<const float4*>(part + p * sd.stride + base + i);
         v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
       }
+    }
     *reinterpret_cast<float4*>(x_out + base + i) = v;
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
@@ -152,15 +154,15 @@ __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const fl
     if (hn) *reinterpret_cast<float4*>(hn + base + i) = v;
   }
 }
-hydra_status residual_rmsnorm(const float* res, const float* part, size_t stride, int splits, float* x_out,
+hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd, float* x_out,
                               const void* gain, void* xn, float* hn, int rows, int d, float eps, int dtype,
                               cudaStream_t st) {
   if (d & 3) return HYDRA_ERR_UNSUPPORTED;
   if (dtype == 0)
-    residual_rmsnorm_kernel<float><<<rows, NORM_THREADS, 0, st>>>(res, part, stride, splits, x_out, (const float*)gain,
+    residual_rmsnorm_kernel<float><<<rows, NORM_THREADS, 0, st>>>(res, part, sd, x_out, (const float*)gain,
                                                                   (float*)xn, hn, d, eps);
   else
-    residual_rmsnorm_kernel<bf16><<<rows, NORM_THREADS, 0, st>>>(res, part, stride, splits, x_out, (const bf16*)gain,
+    residual_rmsnorm_kernel<bf16><<<rows, NORM_THREADS, 0, st>>>(res, part, sd, x_out, (const bf16*)gain,
                                                                  (bf16*)xn, hn, d, eps);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -186,7 +188,7 @@ hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cud
 }
 
 template <typename T>
-__global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restrict__ part, size_t stride, int splits,
+__global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restrict__ part, SplitDesc sd,
                                                             const float2* __restrict__ table, T* __restrict__ q,
                                                             T* __restrict__ kc, T* __restrict__ vc, RowSet rs, int H,
                                                             int hd, int max_seq, int* status) {
@@ -200,11 +202,16 @@ __global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restr
   if (j >= half) return;
   const float* p0 = part + (size_t)r * 3 * d;
   const int c0 = h * hd + j, c1 = c0 + half;
-  float qa = 0, qb = 0, ka = 0, kb = 0, va = 0, vb = 0;
-  for (int s = 0; s < splits; ++s) {
-    const float* p = p0 + s * stride;
-    qa += p[c0]; qb += p[c1]; ka += p[d + c0]; kb += p[d + c1]; va += p[2 * d + c0]; vb += p[2 * d + c1];
+  float v6[6];
+  const int cols[6] = {c0, c1, d + c0, d + c1, 2 * d + c0, 2 * d + c1};
+#pragma unroll
+  for (int e = 0; e < 6; ++e) {
+    const int ns = split_count(sd, r, cols[e]);
+    float acc = 0.f;
+    for (int s = 0; s < ns; ++s) acc += p0[s * sd.stride + cols[e]];
+    v6[e] = acc;
   }
+  const float qa = v6[0], qb = v6[1], ka = v6[2], kb = v6[3], va = v6[4], vb = v6[5];
   const float2 cs = table[(size_t)r * half + j];
   q[(size_t)r * d + c0] = from_f<T>(qa * cs.x - qb * cs.y);
   q[(size_t)r * d + c1] = from_f<T>(qb * cs.x + qa * cs.y);
@@ -214,15 +221,15 @@ __global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restr
   vc[o + j] = from_f<T>(va);
   vc[o + j + half] = from_f<T>(vb);
 }
-hydra_status qkv_rope_store(const float* part, size_t stride, int splits, const float2* table, void* q, void* kcache,
+hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, void* kcache,
                             void* vcache, RowSet rs, int H, int hd, int max_seq, int dtype, int* status,
                             cudaStream_t st) {
   dim3 grid(rs.batch * rs.tc, H);
   if (dtype == 0)
-    qkv_rope_store_kernel<float><<<grid, 64, 0, st>>>(part, stride, splits, table, (float*)q, (float*)kcache, (float*)vcache,
+    qkv_rope_store_kernel<float><<<grid, 64, 0, st>>>(part, sd, table, (float*)q, (float*)kcache, (float*)vcache,
                                                       rs, H, hd, max_seq, status);
   else
-    qkv_rope_store_kernel<bf16><<<grid, 64, 0, st>>>(part, stride, splits, table, (bf16*)q, (bf16*)kcache, (bf16*)vcache, rs,
+    qkv_rope_store_kernel<bf16><<<grid, 64, 0, st>>>(part, sd, table, (bf16*)q, (bf16*)kcache, (bf16*)vcache, rs,
                                                      H, hd, max_seq, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -394,24 +401,23 @@ hydra_status tree_attention(const void* q, const void* kc, const void* vc, RowSe
 // SiLU(gate) * up from the gate/up partial sums
 // ------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void silu_mul_kernel(const float* __restrict__ part, size_t stride, int splits, T* __restrict__ act, int rows,
-                                int f) {
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+__global__ void silu_mul_kernel(const float* __restrict__ part, SplitDesc sd, T* __restrict__ act, int rows, int f) {
+  size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= (size_t)rows * f) return;
-  size_t r = i / f, c = i % f;
-  float g = 0.f, u = 0.f;
-  for (int s = 0; s < splits; ++s) {
-    const float* p = part + s * stride + r * 2 * f;
-    g += p[c]; u += p[f + c];
-  }
-  act[i] = from_f<T>(silu_f(g) * u);
+  const int r = (int)(i / f), c = (int)(i % f);
+  const float* p = part + (size_t)r * 2 * f;
+  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+  const int ng = split_count(sd, r, c), nu = split_count(sd, r, f + c);
+  for (int s = 0; s < ng; ++s) { float4 a = *reinterpret_cast<const float4*>(p + s * sd.stride + c); g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w; }
+  for (int s = 0; s < nu; ++s) { float4 a = *reinterpret_cast<const float4*>(p + s * sd.stride + f + c); u.x += a.x; u.y += a.y; u.z += a.z; u.w += a.w; }
+  store4<T>(act + i, make_float4(silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w));
 }
-hydra_status silu_mul(const float* part, size_t stride, int splits, void* act, int rows, int f, int dtype,
-                      cudaStream_t st) {
-  size_t n = (size_t)rows * f;
+hydra_status silu_mul(const float* part, SplitDesc sd, void* act, int rows, int f, int dtype, cudaStream_t st) {
+  if (f & 3) return HYDRA_ERR_UNSUPPORTED;
+  size_t n = (size_t)rows * f / 4;
   unsigned grid = (unsigned)((n + 255) / 256);
-  if (dtype == 0) silu_mul_kernel<float><<<grid, 256, 0, st>>>(part, stride, splits, (float*)act, rows, f);
-  else silu_mul_kernel<bf16><<<grid, 256, 0, st>>>(part, stride, splits, (bf16*)act, rows, f);
+  if (dtype == 0) silu_mul_kernel<float><<<grid, 256, 0, st>>>(part, sd, (float*)act, rows, f);
+  else silu_mul_kernel<bf16><<<grid, 256, 0, st>>>(part, sd, (bf16*)act, rows, f);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -448,23 +454,35 @@ __device__ __forceinline__ void block_best(float& v, int& i, float* shv, int* sh
   v = shv[0]; i = shi[0];
 }
 
-__global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restrict__ logits, int* __restrict__ amax,
-                                                          int vocab) {
+__device__ __forceinline__ float summed(const float* part, const SplitDesc& sd, int row, int col, int n) {
+  const int ns = split_count(sd, row, col);
+  float v = 0.f;
+  for (int s = 0; s < ns; ++s) v += part[s * sd.stride + (size_t)row * n + col];
+  return v;
+}
+
+__global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restrict__ part, SplitDesc sd,
+                                                          float* __restrict__ logits_out, int* __restrict__ amax, int vocab) {
   __shared__ float shv[32];
   __shared__ int shi[32];
-  const float* row = logits + (size_t)blockIdx.x * vocab;
+  const int row = blockIdx.x;
   float bv = -INFINITY; int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < vocab; i += blockDim.x) { float v = row[i]; if (better(v, i, bv, bi)) { bv = v; bi = i; } }
+  for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
+    float v = summed(part, sd, row, i, vocab);
+    if (logits_out) logits_out[(size_t)row * vocab + i] = v;
+    if (better(v, i, bv, bi)) { bv = v; bi = i; }
+  }
   block_best(bv, bi, shv, shi);
-  if (threadIdx.x == 0) amax[blockIdx.x] = bi;
+  if (threadIdx.x == 0) amax[row] = bi;
 }
-hydra_status argmax_rows(const float* logits, int* amax, int rows, int vocab, cudaStream_t st) {
-  argmax_rows_kernel<<<rows, 256, 0, st>>>(logits, amax, vocab);
+hydra_status argmax_rows(const float* part, SplitDesc sd, float* logits_out, int* amax, int rows, int vocab, cudaStream_t st) {
+  argmax_rows_kernel<<<rows, 256, 0, st>>>(part, sd, logits_out, amax, vocab);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
-__global__ void __launch_bounds__(256) topk_children_kernel(const float* __restrict__ logits, LevelDesc lv,
+__global__ void __launch_bounds__(256) topk_children_kernel(const float* __restrict__ part, SplitDesc sd, float* __restrict__ logits,
+                                                            LevelDesc lv,
                                                             const int* __restrict__ first_child,
                                                             const int* __restrict__ n_child, int* __restrict__ tree_tok,
                                                             int T, int vocab) {
@@ -473,7 +491,8 @@ __global__ void __launch_bounds__(256) topk_children_kernel(const float* __restr
   const int row = blockIdx.x, b = row / lv.n_parents, j = row % lv.n_parents;
   const int p = lv.parents[j];
   const int nc = n_child[p], fc = first_child[p];
-  const float* lg = logits + (size_t)row * vocab;
+  float* lg = logits + (size_t)row * vocab;
+  for (int i = threadIdx.x; i < vocab; i += blockDim.x) lg[i] = summed(part, sd, row, i, vocab);   // each thread re-reads its own
   float pv = INFINITY; int pi = -1;
   for (int t = 0; t < nc; ++t) {
     float bv = -INFINITY; int bi = 0x7fffffff;
@@ -487,9 +506,9 @@ __global__ void __launch_bounds__(256) topk_children_kernel(const float* __restr
     pv = bv; pi = bi;
   }
 }
-hydra_status topk_children(const float* logits, LevelDesc lv, const int* first_child, const int* n_child, int* tree_tok,
-                           int batch, int T, int vocab, cudaStream_t st) {
-  topk_children_kernel<<<batch * lv.n_parents, 256, 0, st>>>(logits, lv, first_child, n_child, tree_tok, T, vocab);
+hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, const int* first_child,
+                           const int* n_child, int* tree_tok, int batch, int T, int vocab, cudaStream_t st) {
+  topk_children_kernel<<<batch * lv.n_parents, 256, 0, st>>>(part, sd, logits, lv, first_child, n_child, tree_tok, T, vocab);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -533,27 +552,28 @@ hydra_status head_gather(const float* hprime, const void* embed, const int* root
 
 template <typename T>
 __global__ void head_act_kernel(const float* res, int res_is_hprime, int rows_per_b, const float* __restrict__ part,
-                                size_t stride, int splits, const T* __restrict__ bias, float* y_out, T* __restrict__ yb,
+                                SplitDesc sd, const T* __restrict__ bias, float* y_out, T* __restrict__ yb,
                                 int rows, int d) {
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (size_t)rows * d) return;
   int r = (int)(i / d), c = (int)(i % d);
   float v = bias ? to_f<T>(bias[c]) : 0.f;
-  for (int s = 0; s < splits; ++s) v += part[s * stride + i];
+  const int ns = split_count(sd, r, c);
+  for (int s = 0; s < ns; ++s) v += part[s * sd.stride + i];
   float base = res_is_hprime ? res[(size_t)(r / rows_per_b) * d + c] : res[i];
   float y = base + silu_f(v);
   y_out[i] = y;
   yb[i] = from_f<T>(y);
 }
-hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, size_t stride, int splits,
+hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, SplitDesc sd,
                       const void* bias, float* y_out, void* yb, int rows, int d, int dtype, cudaStream_t st) {
   size_t n = (size_t)rows * d;
   unsigned grid = (unsigned)((n + 255) / 256);
   if (dtype == 0)
-    head_act_kernel<float><<<grid, 256, 0, st>>>(res, res_is_hprime, rows_per_b, part, stride, splits, (const float*)bias,
+    head_act_kernel<float><<<grid, 256, 0, st>>>(res, res_is_hprime, rows_per_b, part, sd, (const float*)bias,
                                                  y_out, (float*)yb, rows, d);
   else
-    head_act_kernel<bf16><<<grid, 256, 0, st>>>(res, res_is_hprime, rows_per_b, part, stride, splits, (const bf16*)bias,
+    head_act_kernel<bf16><<<grid, 256, 0, st>>>(res, res_is_hprime, rows_per_b, part, sd, (const bf16*)bias,
                                                 y_out, (bf16*)yb, rows, d);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;

@@ -4,29 +4,31 @@
 
 namespace hydra {
 
-// ---- GEMM: out[split][m][n] = sum over that split's k range of x[m][k] * w[n][k]
-// tcgen05 path (bfloat16 operands).  out rows have stride n; split s is written at out + s*split_stride.
-// x_rows_alloc = rows the x buffer really holds (>= m); rows of the last tile beyond m are computed and dropped.
-hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* out, size_t split_stride, int m, int n,
-                     int k, int splits, int* status, cudaStream_t st);
+// ---- GEMM: partial sums of x[m][k] * w[n][k] (see SplitDesc for where they land)
+// tcgen05 path (bfloat16 operands).  x_rows_alloc = rows the x buffer really holds (>= m); rows of the last
+// tile beyond m are computed and dropped.  part needs gemm_tc_plan(...)'s max_slots * m * n floats.
+hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part, int m, int n, int k, SplitDesc* sd_out,
+                     int* status, cudaStream_t st);
+SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots);
+int gemm_tile_rows(int m);                // activation rows per MMA tile for an m-row GEMM: 16, 32, 64, 128 or 256
 bool gemm_tc_available();                 // driver entry point for tensor-map encoding found
-// SIMT path (float or bfloat16 operands), no split.
+// SIMT path (float or bfloat16 operands), single slot.
 hydra_status gemm_simt(const void* x, const void* w, float* out, int m, int n, int k, int dtype, cudaStream_t st);
-// out[i] = sum_s part[s*stride + i]
-hydra_status reduce_splits(const float* part, size_t split_stride, int splits, float* out, size_t count, cudaStream_t st);
+// out[m][n] = sum of the slots of part
+hydra_status reduce_splits(const float* part, SplitDesc sd, float* out, int m, int n, cudaStream_t st);
 
 // ---- element-wise / row-wise stages of a decoder layer (dtype: 0 float, 1 bfloat16 for the "act" outputs)
 hydra_status embed_rows(const void* embed, const int* tok, float* x, int rows, int d, int vocab, int dtype, int* status,
                         cudaStream_t st);
 // x_out = (res ? res : 0) + sum_s part[s]; if gain: xn = rmsnorm(x_out)*gain (act dtype, optional) and hn = the same in
 // float (optional).  part may be null.  x_out may alias res.
-hydra_status residual_rmsnorm(const float* res, const float* part, size_t split_stride, int splits, float* x_out,
+hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd, float* x_out,
                               const void* gain, void* xn, float* hn, int rows, int d, float eps, int dtype,
                               cudaStream_t st);
 // table[r][j] = (cos, sin) of (pos0[b]+depth[i]) * theta^(-2j/head_dim), evaluated in double
 hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st);
 // q (operand dtype, [rows][H][hd], rotated), K/V cache rows (rotated K) from the QKV partial sums.
-hydra_status qkv_rope_store(const float* part, size_t split_stride, int splits, const float2* table, void* q,
+hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q,
                             void* kcache, void* vcache, RowSet rs, int n_heads, int head_dim, int max_seq, int dtype,
                             int* status, cudaStream_t st);
 constexpr int ATT_CHUNK_ROWS = 128;     // KV rows per attention CTA (split-KV granularity)
@@ -36,10 +38,10 @@ hydra_status tree_attention_tc(const bf16* q, const bf16* kc, const bf16* vc, Ro
                                int head_dim, int max_seq, int len_upper, cudaStream_t st);
 hydra_status tree_attention(const void* q, const void* kcache, const void* vcache, RowSet rs, void* out, void* scratch,
                             int n_heads, int head_dim, int max_seq, int len_upper, int dtype, cudaStream_t st);
-hydra_status silu_mul(const float* part, size_t split_stride, int splits, void* act, int rows, int f, int dtype,
+hydra_status silu_mul(const float* part, SplitDesc sd, void* act, int rows, int f, int dtype,
                       cudaStream_t st);
-// amax[r] = argmax_v logits[r][v] (lowest id among equal maxima)
-hydra_status argmax_rows(const float* logits, int* amax, int rows, int vocab, cudaStream_t st);
+// amax[r] = argmax_v of the summed partial logits (lowest id among equal maxima); the sums go to logits_out if given
+hydra_status argmax_rows(const float* part, SplitDesc sd, float* logits_out, int* amax, int rows, int vocab, cudaStream_t st);
 
 // ---- Hydra heads
 struct LevelDesc {           // one tree level d (1-based): the parents that have children
@@ -51,10 +53,11 @@ hydra_status head_gather(const float* hprime, const void* embed, const int* root
                          LevelDesc lv, void* z, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
                          cudaStream_t st);
 // y_out = res + silu(sum_s part[s] + bias); res row = hprime[b] when res_is_hprime else y row.  yb = act-dtype copy.
-hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, size_t split_stride,
-                      int splits, const void* bias, float* y_out, void* yb, int rows, int d, int dtype, cudaStream_t st);
-// children of parent j of sequence b = top n_child tokens of logits row b*P+j, descending (ties: lower id first)
-hydra_status topk_children(const float* logits, LevelDesc lv, const int* first_child, const int* n_child, int* tree_tok,
+hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, SplitDesc sd,
+                      const void* bias, float* y_out, void* yb, int rows, int d, int dtype, cudaStream_t st);
+// children of parent j of sequence b = top n_child tokens of logits row b*P+j, descending (ties: lower id first);
+// the logits are the summed partials, also written to `logits` [rows][vocab]
+hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, const int* first_child, const int* n_child, int* tree_tok,
                            int batch, int T, int vocab, cudaStream_t st);
 
 // ---- acceptance + compaction (one kernel)

@@ -13,19 +13,19 @@ def rnd(shape, seed, stream, dtype, std=1.0):
     return normal_(torch.empty(shape, dtype=dtype), seed, stream, std)
 
 
-@pytest.mark.parametrize("m,n,k,splits", [(64, 256, 512, 1), (64, 384, 4096, 3), (5, 128, 256, 1), (11, 256, 1280, 2),
-                                          (16, 128, 64, 1), (100, 512, 704, 4), (256, 256, 1024, 1), (300, 384, 512, 2),
-                                          (64, 128, 11008, 4), (1, 1024, 256, 1)])
-def test_gemm_tensor_core_matches_definition(m, n, k, splits):
+@pytest.mark.parametrize("m,n,k", [(64, 256, 512), (64, 12288, 4096), (5, 128, 256), (11, 256, 1280), (16, 128, 64),
+                                   (100, 512, 704), (256, 256, 1024), (300, 384, 512), (64, 4096, 11008),
+                                   (1, 1024, 256), (64, 32000, 1024), (512, 1024, 512)])
+def test_gemm_tensor_core_matches_definition(m, n, k):
     from paper_2402_05109_b200 import gemm
     x = rnd((m, k), 11, m + k, torch.bfloat16)
     w = rnd((n, k), 12, n + k, torch.bfloat16, 0.02)
     ref = x.double() @ w.double().T
-    out = gemm(x.cuda(), w.cuda(), splits=splits, mode=0).cpu().double()
+    out = gemm(x.cuda(), w.cuda(), mode=0).cpu().double()
     # products of bfloat16 values are exact in float; only the float accumulation order differs
     tol = 1e-5 * float(ref.abs().max()) + 1e-6 * k ** 0.5
     assert float((out - ref).abs().max()) <= tol
-    simt = gemm(x.cuda(), w.cuda(), splits=1, mode=1).cpu().double()
+    simt = gemm(x.cuda(), w.cuda(), mode=1).cpu().double()
     assert float((simt - ref).abs().max()) <= tol
 
 
