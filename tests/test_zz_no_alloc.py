@@ -32,8 +32,8 @@ def test_noalloc_gemm_matches_gemm_on_two_calls_in_a_row():
         assert float((out.double().cpu() - exact).abs().max()) <= tol
         assert torch.equal(out, ref)          # same kernels, same split order: bit-identical
     # a problem whose partial sums exceed the built-in scratch is refused with a clear error, nothing launched
-    x, w = _operands(256, 8192, 256, 33)
-    out = torch.zeros(256, 8192, dtype=torch.float32, device="cuda")
+    x, w = _operands(256, 16384, 256, 33)
+    out = torch.zeros(256, 16384, dtype=torch.float32, device="cuda")
     with pytest.raises(HydraError, match="8 MiB"):
         gemm_noalloc(x, w, out, status)
     assert float(out.abs().max()) == 0.0
