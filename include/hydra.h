@@ -154,7 +154,8 @@ enum { HYDRA_TIME_GEMM = 0, HYDRA_TIME_ATTENTION = 1, HYDRA_TIME_ACCEPT = 2 };
 hydra_status hydra_set_timing(hydra_ctx*, int on);
 hydra_status hydra_get_timing(hydra_ctx*, int kclass, double* ms_total, long long* launches, double* bytes_total);
 
-/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA (default), 1 = the plain SIMT kernel. */
+/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA with fused epilogues (default), 1 = the plain SIMT
+ * kernel, 2 = tcgen05/TMA with the consumer operations in separate kernels. */
 hydra_status hydra_set_gemm_mode(hydra_ctx*, int mode);
 
 const char* hydra_status_str(hydra_status);

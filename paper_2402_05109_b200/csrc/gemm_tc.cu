@@ -20,6 +20,12 @@
 // TMEM let the epilogue of one segment overlap the main loop of the next.  The kernel is launched with
 // programmatic stream serialisation: weight tiles (which never depend on the preceding kernel) are requested
 // before griddepcontrol.wait, activations and all global writes after it.
+// Fused epilogues: after writing its slot a CTA bumps the tile's arrival counter; the CTA that completes the
+// tile ("last arriver") adds the slots in slot order and applies the consumer operation right there -- rotary
+// embedding + KV-cache append (QKV), residual add + next-norm operand + row sums of squares (O and down
+// projections), SiLU(gate)*up (gate/up pairs), or a plain scaled store (LM head).  RMSNorm is factored as
+// (x*gain) W^T * inv_rms[row]: the producer stores x*gain in bfloat16 and per-tile sums of squares, the
+// consuming GEMM scales its reduced output rows by inv_rms.
 // Every mbarrier wait is bounded: when one runs out the CTA raises ST_TIMEOUT in the status word, stops
 // storing, lets its copies settle, frees its tensor memory and returns.
 #include "launch.h"
@@ -35,7 +41,7 @@ namespace {
 constexpr int BLOCK_N = 128;             // weight rows per tile (MMA M)
 constexpr int BLOCK_K = 64;              // 64 bf16 = 128 bytes = one swizzle row
 constexpr int A_BYTES = BLOCK_N * BLOCK_K * 2;
-constexpr int SMEM_BUDGET = 200 * 1024;
+constexpr int SMEM_BUDGET = 100 * 1024;    // per CTA: two CTAs of consecutive (PDL-overlapped) kernels fit one SM
 constexpr uint32_t WAIT_LIMIT = 1u << 24;   // try_wait attempts before giving up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -131,7 +137,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int mt) {
 template <int MT> struct TileCfg {
   static constexpr int B_BYTES = MT * BLOCK_K * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 10 ? 10 : (SMEM_BUDGET / STAGE_BYTES);
+  static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 10 ? 10 : ((SMEM_BUDGET / STAGE_BYTES) < 3 ? 3 : (SMEM_BUDGET / STAGE_BYTES));
   static constexpr int ACC_COLS = MT < 32 ? 32 : MT;             // columns of one accumulator buffer
   static constexpr int TMEM_COLS = 2 * ACC_COLS;                  // two buffers (power of two, <= 512)
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/;
@@ -141,7 +147,93 @@ struct GemmArgs {
   float* part; size_t slot_stride;
   int m, n, kb, n_tiles, total_units, q;
   int* status;
+  int epi;                       // GemmEpilogue::kind
+  unsigned int* counters;        // [tiles], zero at rest
+  const float* ss_in; int ss_in_tiles; int ss_ld; float inv_d, eps;     // RMSNorm factor of the operand rows (null: none)
+  RowSet rs; const float2* rope; void* q_out; void* kc; void* vc; int H, hd, max_seq;   // EPI_QKV
+  float* x; void* xg; const void* gain; float* ss_out;                                   // EPI_RESID
+  void* act; int f;                                                                      // EPI_GATEUP
+  float* out;                                                                            // EPI_OUT
 };
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the 4 epilogue warps
+
+__device__ __forceinline__ int tile_slots(const GemmArgs& a, int tile) {
+  const long long u0 = (long long)tile * a.kb;
+  return (int)((u0 + a.kb - 1) / a.q - u0 / a.q) + 1;
+}
+// Sum of a tile's partial slots for output element (m, n), in slot order (read past L1: other SMs wrote them).
+__device__ __forceinline__ float slot_sum(const GemmArgs& a, int ns, int m, int n) {
+  const float* p = a.part + (size_t)m * a.n + n;
+  float v = 0.f;
+  for (int s = 0; s < ns; ++s) v += __ldcg(p + (size_t)s * a.slot_stride);
+  return v;
+}
+
+// Consumer operation applied by the last arriver of a tile (or of a gate/up tile pair).  tid = column within
+// the tile (0..127); all 128 epilogue threads call it.
+template <int MT>
+__device__ void apply_epilogue(const GemmArgs& a, int tile, int tid, const float* s_inv, float (*s_ex)[128], float (*s_ss)[MT]) {
+  const int tn = tile % a.n_tiles, tm = tile / a.n_tiles;
+  const int m0 = tm * MT, m1 = min(m0 + MT, a.m);
+  const int warp4 = tid >> 5, lane = tid & 31;
+  if (a.epi == EPI_OUT) {
+    const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
+    for (int m = m0; m < m1; ++m) a.out[(size_t)m * a.n + n] = slot_sum(a, ns, m, n) * s_inv[m];
+  } else if (a.epi == EPI_RESID) {
+    const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
+    const float gn = a.gain ? __bfloat162float(reinterpret_cast<const bf16*>(a.gain)[n]) : 0.f;
+    for (int m = m0; m < m1; ++m) {
+      const size_t idx = (size_t)m * a.n + n;
+      const float xv = a.x[idx] + slot_sum(a, ns, m, n);
+      a.x[idx] = xv;
+      if (a.gain) reinterpret_cast<bf16*>(a.xg)[idx] = __float2bfloat16_rn(xv * gn);
+      const float ss = warp_sum(xv * xv);
+      if (lane == 0) s_ss[warp4][m - m0] = ss;
+    }
+    epi_bar();
+    for (int r = tid; r < m1 - m0; r += 128)
+      a.ss_out[(size_t)tn * a.ss_ld + m0 + r] = s_ss[0][r] + s_ss[1][r] + s_ss[2][r] + s_ss[3][r];
+  } else if (a.epi == EPI_GATEUP) {
+    const int half_tiles = a.n_tiles >> 1;
+    const int p = tn % half_tiles;
+    const int tg = tm * a.n_tiles + p, tu = tg + half_tiles;
+    const int nsg = tile_slots(a, tg), nsu = tile_slots(a, tu);
+    const int c = p * BLOCK_N + tid;
+    for (int m = m0; m < m1; ++m) {
+      const float sc = s_inv[m];
+      const float g = slot_sum(a, nsg, m, c) * sc, u = slot_sum(a, nsu, m, a.f + c) * sc;
+      reinterpret_cast<bf16*>(a.act)[(size_t)m * a.f + c] = __float2bfloat16_rn(silu_f(g) * u);
+    }
+  } else if (a.epi == EPI_QKV) {
+    const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
+    const int d = a.H * a.hd, half = a.hd >> 1;
+    const int which = n / d, within = n % d, head = within / a.hd, jl = within % a.hd;
+    const int partner = jl < half ? tid + half : tid - half;
+    bf16* kv = reinterpret_cast<bf16*>(which == 1 ? a.kc : a.vc);
+    for (int m = m0; m < m1; ++m) {
+      const int b = m / a.rs.tc, i = m % a.rs.tc;
+      const int nr = a.rs.n_rows ? a.rs.n_rows[b] : a.rs.tc;
+      const int slot = a.rs.pos0[b] + i;
+      const bool row_ok = i < nr && slot >= 0 && slot < a.max_seq;       // uniform over the 128 threads
+      if (i < nr && !row_ok && tid == 0) atomicOr(a.status, ST_BOUNDS);
+      const float v = row_ok ? slot_sum(a, ns, m, n) * s_inv[m] : 0.f;
+      float outv = v;
+      if (which < 2) {                                                   // rotate q and k (half-split pairing)
+        float* ex = s_ex[m & 1];
+        ex[tid] = v;
+        epi_bar();
+        const float pv = ex[partner];
+        const float2 cs = row_ok ? a.rope[(size_t)m * half + (jl % half)] : make_float2(1.f, 0.f);
+        outv = jl < half ? v * cs.x - pv * cs.y : v * cs.x + pv * cs.y;
+      }
+      if (row_ok) {
+        if (which == 0) reinterpret_cast<bf16*>(a.q_out)[(size_t)m * d + within] = __float2bfloat16_rn(outv);
+        else kv[(((size_t)b * a.H + head) * a.max_seq + slot) * a.hd + jl] = __float2bfloat16_rn(outv);
+      }
+    }
+  }
+}
 
 template <int MT>
 __global__ void __launch_bounds__(192, 1)
@@ -156,7 +248,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   auto accfull_bar = [&](int i) { return bars + 8u * (3 * C::STAGES + i); };
   auto accempty_bar = [&](int i) { return bars + 8u * (3 * C::STAGES + 2 + i); };
   const uint32_t tmem_slot = bars + 8u * (3 * C::STAGES + 4);
-  __shared__ int s_abort;
+  __shared__ int s_abort, s_last;
+  __shared__ float s_inv[512];               // inv_rms of the operand rows (fused epilogues need m <= 512)
+  __shared__ float s_ex[2][128];
+  __shared__ float s_ss[4][MT];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_begin = blockIdx.x * a.q;
@@ -247,7 +342,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else {
     const int quarter = warp & 3;                        // TMEM lanes this warp may read
-    grid_dep_wait();                                     // the partial buffer may still be read by the preceding kernel
+    const int epi_tid = quarter * 32 + lane;             // column of the tile this thread owns
+    grid_dep_wait();                                     // partial buffer / operand statistics belong to the preceding kernel
+    if (a.epi != EPI_PARTIAL) {
+      for (int m = epi_tid; m < a.m && m < 512; m += 128) {
+        float ss = 0.f;
+        for (int t = 0; t < a.ss_in_tiles; ++t) ss += a.ss_in[(size_t)t * a.ss_ld + m];
+        s_inv[m] = a.ss_in ? rsqrtf(ss * a.inv_d + a.eps) : 1.f;
+      }
+      epi_bar();
+    }
     int seg = 0;
     for (int i = 0; i < n_units;) {
       const int u = u_begin + i;
@@ -259,7 +363,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       tc_fence_after();
       const int slot = blockIdx.x - (int)(((long long)tile * a.kb) / a.q);
       const int n0 = (tile % a.n_tiles) * BLOCK_N, m0 = (tile / a.n_tiles) * MT;
-      float* dst = a.part + (size_t)slot * a.slot_stride + n0 + quarter * 32 + lane;
+      float* dst = a.part + (size_t)slot * a.slot_stride + n0 + epi_tid;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * C::ACC_COLS);
 #pragma unroll 1
       for (int c = 0; c < MT; c += 16) {
@@ -271,7 +375,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           if (m0 + c + j < a.m) dst[(size_t)(m0 + c + j) * a.n] = __uint_as_float(r[j]);
       }
       tc_fence_before();
-      if (lane == 0) mbar_arrive(accempty_bar(acc));
+      if (lane == 0) mbar_arrive(accempty_bar(acc));     // the MMA warp may reuse this accumulator
+      if (a.epi != EPI_PARTIAL) {
+        int cidx = tile, expected;
+        if (a.epi == EPI_GATEUP) {
+          const int half_tiles = a.n_tiles >> 1;
+          const int tm = tile / a.n_tiles, p = (tile % a.n_tiles) % half_tiles;
+          cidx = tm * half_tiles + p;
+          expected = tile_slots(a, tm * a.n_tiles + p) + tile_slots(a, tm * a.n_tiles + p + half_tiles);
+        } else {
+          expected = tile_slots(a, tile);
+        }
+        __threadfence();                                 // this thread's slot stores before the arrival
+        epi_bar();
+        if (epi_tid == 0) {
+          const unsigned prev = atomicAdd(&a.counters[cidx], 1u);
+          const int last = (int)(prev + 1u) == expected;
+          if (last) a.counters[cidx] = 0u;               // back to rest for the next launch
+          s_last = last;
+        }
+        epi_bar();
+        if (s_last) {
+          __threadfence();
+          apply_epilogue<MT>(a, tile, epi_tid, s_inv, s_ex, s_ss);
+        }
+      }
       i += seg_len;
       ++seg;
     }
@@ -386,7 +514,7 @@ SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots) {
 }
 
 hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part, int m, int n, int k, SplitDesc* sd_out,
-                     int* status, cudaStream_t st) {
+                     const GemmEpilogue* epi, int* status, cudaStream_t st) {
   if (m <= 0 || n <= 0 || k <= 0 || n % BLOCK_N || k % BLOCK_K) return HYDRA_ERR_UNSUPPORTED;
   if (((uintptr_t)x | (uintptr_t)w) & 15) return HYDRA_ERR_INVALID;
   int grid = 1;
@@ -398,7 +526,19 @@ hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part
     set_last_error("cuTensorMapEncodeTiled", cudaErrorUnknown);
     return HYDRA_ERR_CUDA;
   }
-  GemmArgs a{part, sd.stride, m, n, sd.kb, sd.n_tiles, sd.n_tiles * ((m + sd.mt - 1) / sd.mt) * sd.kb, sd.q, status};
+  GemmArgs a{};
+  a.part = part; a.slot_stride = sd.stride; a.m = m; a.n = n; a.kb = sd.kb; a.n_tiles = sd.n_tiles;
+  a.total_units = sd.n_tiles * ((m + sd.mt - 1) / sd.mt) * sd.kb; a.q = sd.q; a.status = status; a.epi = EPI_PARTIAL;
+  if (epi && epi->kind != EPI_PARTIAL) {
+    if (m > 512 || !epi->counters) return HYDRA_ERR_UNSUPPORTED;
+    if (epi->kind == EPI_GATEUP && ((sd.n_tiles & 1) || epi->f != n / 2)) return HYDRA_ERR_UNSUPPORTED;
+    if (epi->kind == EPI_QKV && ((epi->H * epi->hd) % BLOCK_N || (epi->hd != 64 && epi->hd != 128))) return HYDRA_ERR_UNSUPPORTED;
+    a.epi = epi->kind; a.counters = epi->counters;
+    a.ss_in = epi->ss_in; a.ss_in_tiles = epi->ss_in_tiles; a.ss_ld = epi->ss_ld; a.inv_d = epi->inv_d; a.eps = epi->eps;
+    a.rs = epi->rs; a.rope = epi->rope; a.q_out = epi->q_out; a.kc = epi->kc; a.vc = epi->vc; a.H = epi->H; a.hd = epi->hd;
+    a.max_seq = epi->max_seq; a.x = epi->x; a.xg = epi->xg; a.gain = epi->gain; a.ss_out = epi->ss_out; a.act = epi->act;
+    a.f = epi->f; a.out = epi->out;
+  }
   if (sd_out) *sd_out = sd;
   switch (sd.mt) {
     case 16: return launch<16>(tw, tx, a, grid, st);

@@ -17,6 +17,7 @@ void set_last_error(const char* what, cudaError_t e) {
 
 namespace {
 
+constexpr int COUNTERS = 8192;     // tile arrival counters of the fused GEMM epilogues (>= tiles of any GEMM)
 constexpr int CHUNK = 64;          // rows per sequence of one prefill pass (and the row capacity of a forward call)
 
 struct LayerW { const void *attn_norm, *wqkv, *wo, *ffn_norm, *w_gate_up, *w_down; };
@@ -58,14 +59,15 @@ struct hydra_ctx {
   uint64_t *d_anc, *d_chain_mask;
   std::vector<int*> d_level_parents;
   int *d_len, *d_n_new, *d_root_tok, *d_status, *d_pos0, *d_nrows, *d_prompt_len, *d_offsets, *d_tok, *d_tree_tok, *d_amax;
-  unsigned int* d_done;
+  unsigned int *d_done, *d_counters;
+  int ss_tiles;                                  // per-tile sums of squares describing the rows in x (fused path)
   char *kv_base, *kv_pfx;
-  float *x, *part, *h_tree, *h_new, *hprime, *y, *head_logits;
+  float *x, *part, *h_tree, *logits, *ss, *h_new, *hprime, *y, *head_logits;
   float2* rope;
   void *q, *xn, *attn_out, *act, *z, *yb, *att_scratch;
   size_t part_floats;
   // host state
-  int batch, state, gemm_mode;
+  int batch, state, gemm_mode, fused;
   std::vector<int> len_ub;
   const int* plant;
   long long launches;
@@ -171,11 +173,14 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
   auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
   auto* done = b.take<unsigned int>(m.max_batch);
+  auto* counters = b.take<unsigned int>(COUNTERS);
   auto* kvb = b.take<char>((size_t)m.n_layers * 2 * kv_layer_elems(m) * es);
   auto* kvp = b.take<char>(h.prefix_attn ? (size_t)2 * kv_layer_elems(m) * es : 0);
   auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)R * d * es);
   auto* part = b.take<float>(part_floats);
   auto* h_tree = b.take<float>((size_t)R * d);
+  auto* logits = b.take<float>((size_t)pad_rows(m.max_batch * T) * V);
+  auto* ss = b.take<float>((size_t)(d / 128 + 1) * R);
   auto* h_new = b.take<float>((size_t)pad_rows(m.max_batch * (K + 1)) * d);
   auto* hprime = b.take<float>((size_t)m.max_batch * d);
   auto* y = b.take<float>((size_t)RH * d); auto* head_logits = b.take<float>((size_t)RH * V);
@@ -190,7 +195,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
     c->d_chain_depth = chain_depth; c->d_anc = anc; c->d_chain_mask = chain_mask; c->d_level_parents = lvl;
     c->d_len = len; c->d_n_new = n_new; c->d_root_tok = root; c->d_status = status; c->d_pos0 = pos0; c->d_nrows = nrows;
     c->d_prompt_len = plen; c->d_offsets = offs; c->d_tok = tok; c->d_tree_tok = tree_tok; c->d_amax = amax; c->d_done = done;
-    c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree;
+    c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits; c->ss = ss; c->d_counters = counters;
     c->h_new = h_new; c->hprime = hprime; c->y = y; c->head_logits = head_logits; c->rope = rope; c->xn = xn;
     c->attn_out = attn_out; c->act = act; c->z = z; c->yb = yb; c->att_scratch = att;
   }
@@ -218,11 +223,55 @@ hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void*
     // algorithmic bytes of the launch: the weight matrix and the activation slab read once, the partial sums written once
     TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * m * n, st);
     (void)plan;
-    return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, c->part, m, n, k, sd, c->d_status, st);
+    return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, c->part, m, n, k, sd, nullptr, c->d_status, st);
   }
   TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * m * n, st);
   *sd = single_slot((size_t)m * n);
   return gemm_simt(x, w, c->part, m, n, k, c->m.dtype, st);
+}
+
+// The fused path: bfloat16 tensor-core GEMMs whose epilogues do the RoPE/KV append, residual adds, norm
+// statistics and SiLU*up, so a layer is five kernels (QKV, attention, O, gate/up, down).
+bool fused_ok(const hydra_ctx* c, int rows) {
+  const hydra_model_cfg& m = c->m;
+  long long tiles = (long long)std::max(std::max(3 * m.d_model, 2 * m.d_ffn), m.vocab) / 128 * ((rows + 255) / 256 + 1);
+  return m.dtype == 1 && c->gemm_mode == 0 && c->fused && rows <= 512 && m.d_model % 128 == 0 && m.d_ffn % 128 == 0 &&
+         tiles <= COUNTERS;
+}
+
+hydra_status run_gemm_fused(hydra_ctx* c, const void* x, int x_rows_alloc, const void* w, int m, int n, int k, GemmEpilogue& e,
+                            cudaStream_t st) {
+  int slots = 1;
+  gemm_tc_plan(m, n, k, nullptr, &slots);
+  if ((size_t)slots * m * n > c->part_floats) return HYDRA_ERR_CAPACITY;
+  e.counters = c->d_counters;
+  TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * m * n, st);
+  return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, c->part, m, n, k, nullptr, &e, c->d_status, st);
+}
+
+void norm_in(const hydra_ctx* c, GemmEpilogue& e) {
+  e.ss_in = c->ss; e.ss_in_tiles = c->ss_tiles; e.ss_ld = c->R; e.inv_d = 1.0f / (float)c->m.d_model; e.eps = c->m.rms_eps;
+}
+
+hydra_status run_layer_fused(hydra_ctx* c, const LayerW& w, char* kc, char* vc, const RowSet& rs, int len_upper,
+                             const void* next_gain, cudaStream_t st) {
+  const hydra_model_cfg& m = c->m;
+  const int rows = rs.batch * rs.tc, d = m.d_model, f = m.d_ffn;
+  GemmEpilogue q; q.kind = EPI_QKV; norm_in(c, q);
+  q.rs = rs; q.rope = c->rope; q.q_out = c->q; q.kc = kc; q.vc = vc; q.H = m.n_heads; q.hd = m.head_dim; q.max_seq = m.max_seq;
+  HYDRA_TRY(run_gemm_fused(c, c->xn, c->R, w.wqkv, rows, 3 * d, d, q, st));
+  {
+    TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
+    HYDRA_TRY(tree_attention(c->q, kc, vc, rs, c->attn_out, c->att_scratch, m.n_heads, m.head_dim, m.max_seq, len_upper, 1, st));
+  }
+  GemmEpilogue o; o.kind = EPI_RESID; o.x = c->x; o.xg = c->xn; o.gain = w.ffn_norm; o.ss_out = c->ss; o.ss_ld = c->R;
+  HYDRA_TRY(run_gemm_fused(c, c->attn_out, c->R, w.wo, rows, d, d, o, st));
+  c->ss_tiles = d / 128;
+  GemmEpilogue g; g.kind = EPI_GATEUP; norm_in(c, g); g.act = c->act; g.f = f;
+  HYDRA_TRY(run_gemm_fused(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, g, st));
+  GemmEpilogue dn; dn.kind = EPI_RESID; dn.x = c->x; dn.xg = c->xn; dn.gain = next_gain; dn.ss_out = c->ss; dn.ss_ld = c->R;
+  HYDRA_TRY(run_gemm_fused(c, c->act, c->R, w.w_down, rows, d, f, dn, st));
+  return HYDRA_OK;
 }
 
 // One decoder layer over the rows of `rs`.  Expects the residual rows in c->x and their normed copy in c->xn.
@@ -254,6 +303,16 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
   const int rows = rs.batch * rs.tc;
   const size_t kvl = kv_layer_elems(m) * c->esize;
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
+  if (fused_ok(c, rows)) {
+    HYDRA_TRY(rows_prepare(nullptr, c->embed, tok, m.vocab, c->layers[0].attn_norm, c->x, c->xn, c->ss, rows, m.d_model, c->d_status, st));
+    c->ss_tiles = 1;
+    for (int l = 0; l < m.n_layers; ++l) {
+      bool last = l + 1 == m.n_layers;
+      HYDRA_TRY(run_layer_fused(c, c->layers[l], c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs,
+                                len_upper, last ? c->final_norm : c->layers[l + 1].attn_norm, st));
+    }
+    return finalize_hidden(c->x, c->ss, c->ss_tiles, c->R, c->final_norm, m.rms_eps, c->h_tree, rows, m.d_model, st);
+  }
   HYDRA_TRY(embed_rows(c->embed, tok, c->x, rows, m.d_model, m.vocab, m.dtype, c->d_status, st));
   HYDRA_TRY(residual_rmsnorm(c->x, nullptr, single_slot(0), c->x, c->layers[0].attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
   for (int l = 0; l < m.n_layers; ++l) {
@@ -270,6 +329,11 @@ hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int le
   const int rows = rs.batch * rs.tc;
   const size_t kvl = kv_layer_elems(m) * c->esize;
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
+  if (fused_ok(c, rows)) {
+    HYDRA_TRY(rows_prepare(src, nullptr, nullptr, 0, c->pfx.attn_norm, c->x, c->xn, c->ss, rows, m.d_model, c->d_status, st));
+    c->ss_tiles = 1;
+    return run_layer_fused(c, c->pfx, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, nullptr, st);
+  }
   HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
   return run_layer(c, c->pfx, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, nullptr, nullptr, st);
 }
@@ -313,6 +377,12 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
   const int rows = c->batch * c->T;
   RowSet rs{c->batch, c->T, nullptr, c->d_len, c->d_depth, c->d_anc};
   HYDRA_TRY(run_base(c, tree_tok, rs, max_len_ub(c) + c->T, st));
+  if (fused_ok(c, rows)) {                 // c->xn holds x * final_norm gain; the LM head scales its rows by inv_rms
+    float* lg = logits ? logits : c->logits;
+    GemmEpilogue e; e.kind = EPI_OUT; norm_in(c, e); e.out = lg;
+    HYDRA_TRY(run_gemm_fused(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, e, st));
+    return argmax_rows(lg, single_slot(0), nullptr, amax, rows, m.vocab, st);
+  }
   SplitDesc sd;
   HYDRA_TRY(run_gemm(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, &sd, st));
   return argmax_rows(c->part, sd, logits, amax, rows, m.vocab, st);
@@ -393,7 +463,7 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
   }
   c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
   carve(c, *m, *h, th, (char*)ws);
-  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->plant = nullptr; c->launches = 0; c->timing = 0;
+  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->fused = 1; c->ss_tiles = 1; c->plant = nullptr; c->launches = 0; c->timing = 0;
   c->len_ub.assign(m->max_batch, 0);
   // clear the workspace, upload the static tables
   auto fail = [&](cudaError_t e, const char* what) { set_last_error(what, e); delete c; return HYDRA_ERR_CUDA; };
@@ -577,8 +647,9 @@ hydra_status hydra_get_timing(hydra_ctx* c, int kclass, double* ms_total, long l
 }
 
 hydra_status hydra_set_gemm_mode(hydra_ctx* c, int mode) {
-  if (!c || (mode != 0 && mode != 1)) return HYDRA_ERR_INVALID;
-  c->gemm_mode = mode;
+  if (!c || mode < 0 || mode > 2) return HYDRA_ERR_INVALID;
+  c->gemm_mode = mode == 1 ? 1 : 0;
+  c->fused = mode == 0;
   return HYDRA_OK;
 }
 
@@ -615,7 +686,7 @@ hydra_status hydra_gemm(const void* x, const void* w, float* out, float* partial
     if (!status) return HYDRA_ERR_INVALID;
     if (!gemm_tc_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
     SplitDesc sd;
-    HYDRA_TRY(gemm_tc((const bf16*)x, m, (const bf16*)w, partial, m, n, k, &sd, status, st));
+    HYDRA_TRY(gemm_tc((const bf16*)x, m, (const bf16*)w, partial, m, n, k, &sd, nullptr, status, st));
     return reduce_splits(partial, sd, out, m, n, st);
   }
   return gemm_simt(x, w, out, m, n, k, dtype, st);

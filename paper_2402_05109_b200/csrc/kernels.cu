@@ -168,6 +168,60 @@ hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd,
   return HYDRA_OK;
 }
 
+// Rows entering a fused layer stack: x = src row (or the embedding of tok), xg = bf16(x * gain), ss[m] = sum x^2.
+__global__ void __launch_bounds__(NORM_THREADS) rows_prepare_kernel(const float* __restrict__ src, const bf16* __restrict__ embed,
+                                                                    const int* __restrict__ tok, int vocab,
+                                                                    const bf16* __restrict__ gain, float* __restrict__ x,
+                                                                    bf16* __restrict__ xg, float* __restrict__ ss, int d, int* status) {
+  __shared__ float sh[32];
+  const int r = blockIdx.x;
+  const size_t base = (size_t)r * d;
+  const bf16* e = nullptr;
+  if (embed) {
+    int t = tok[r];
+    if (t < 0 || t >= vocab) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); t = 0; }
+    e = embed + (size_t)t * d;
+  }
+  float acc = 0.f;
+  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
+    float4 v = e ? load4<bf16>(e + i) : *reinterpret_cast<const float4*>(src + base + i);
+    float4 gn = load4<bf16>(gain + i);
+    *reinterpret_cast<float4*>(x + base + i) = v;
+    store4<bf16>(xg + base + i, make_float4(v.x * gn.x, v.y * gn.y, v.z * gn.z, v.w * gn.w));
+    acc += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  float tot = block_sum(acc, sh);
+  if (threadIdx.x == 0) ss[r] = tot;
+}
+hydra_status rows_prepare(const float* src, const void* embed, const int* tok, int vocab, const void* gain, float* x, void* xg,
+                          float* ss, int rows, int d, int* status, cudaStream_t st) {
+  rows_prepare_kernel<<<rows, NORM_THREADS, 0, st>>>(src, (const bf16*)embed, tok, vocab, (const bf16*)gain, x, (bf16*)xg, ss, d, status);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
+// h[m] = x[m] * gain * rsqrt(sum_t ss[t*ld + m] / d + eps)   (the normalised hidden rows, float)
+__global__ void __launch_bounds__(NORM_THREADS) finalize_hidden_kernel(const float* __restrict__ x, const float* __restrict__ ss,
+                                                                       int ss_tiles, int ld, const bf16* __restrict__ gain,
+                                                                       float eps, float* __restrict__ h, int d) {
+  const int r = blockIdx.x;
+  float tot = 0.f;
+  for (int t = 0; t < ss_tiles; ++t) tot += ss[(size_t)t * ld + r];
+  const float inv = rsqrtf(tot / (float)d + eps);
+  const size_t base = (size_t)r * d;
+  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
+    float4 v = *reinterpret_cast<const float4*>(x + base + i);
+    float4 gn = load4<bf16>(gain + i);
+    *reinterpret_cast<float4*>(h + base + i) = make_float4(v.x * inv * gn.x, v.y * inv * gn.y, v.z * inv * gn.z, v.w * inv * gn.w);
+  }
+}
+hydra_status finalize_hidden(const float* x, const float* ss, int ss_tiles, int ld, const void* gain, float eps, float* h,
+                             int rows, int d, cudaStream_t st) {
+  finalize_hidden_kernel<<<rows, NORM_THREADS, 0, st>>>(x, ss, ss_tiles, ld, (const bf16*)gain, eps, h, d);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Rotary table + QKV post-processing (sum partials, rotate q and k, append K,V to the cache)
 // ------------------------------------------------------------------------------------------------

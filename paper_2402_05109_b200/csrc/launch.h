@@ -7,8 +7,25 @@ namespace hydra {
 // ---- GEMM: partial sums of x[m][k] * w[n][k] (see SplitDesc for where they land)
 // tcgen05 path (bfloat16 operands).  x_rows_alloc = rows the x buffer really holds (>= m); rows of the last
 // tile beyond m are computed and dropped.  part needs gemm_tc_plan(...)'s max_slots * m * n floats.
+// Optional fused consumer: the CTA that completes a tile adds its slots and applies one of these right away.
+enum { EPI_PARTIAL = 0,   // none: the caller's next kernel reduces the slots
+       EPI_OUT = 1,       // out[m][n] = sum * inv_rms[m]
+       EPI_RESID = 2,     // x += sum; xg = bf16(x * gain[n]); ss_out[n_tile][m] = sum over the tile of x^2
+       EPI_GATEUP = 3,    // act[m][c] = bf16(silu(g) * u), g/u = scaled sums of gate tile c/128 and up tile (f + c)/128
+       EPI_QKV = 4 };     // rotate q,k (table), q -> q_out, k,v -> cache rows pos0[b]+i; all scaled by inv_rms[m]
+struct GemmEpilogue {
+  int kind = EPI_PARTIAL;
+  unsigned int* counters = nullptr;                 // device, one per tile, zero at rest (the kernel restores zero)
+  // RMSNorm factor of the operand rows: inv_rms[m] = rsqrt(sum_t ss_in[t*ss_ld + m] * inv_d + eps); null = 1
+  const float* ss_in = nullptr; int ss_in_tiles = 0; int ss_ld = 0; float inv_d = 0.f, eps = 0.f;
+  RowSet rs{}; const float2* rope = nullptr; void* q_out = nullptr; void* kc = nullptr; void* vc = nullptr;
+  int H = 0, hd = 0, max_seq = 0;
+  float* x = nullptr; void* xg = nullptr; const void* gain = nullptr; float* ss_out = nullptr;
+  void* act = nullptr; int f = 0;
+  float* out = nullptr;
+};
 hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part, int m, int n, int k, SplitDesc* sd_out,
-                     int* status, cudaStream_t st);
+                     const GemmEpilogue* epi, int* status, cudaStream_t st);
 SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots);
 int gemm_tile_rows(int m);                // activation rows per MMA tile for an m-row GEMM: 16, 32, 64, 128 or 256
 bool gemm_tc_available();                 // driver entry point for tensor-map encoding found
@@ -25,6 +42,11 @@ hydra_status embed_rows(const void* embed, const int* tok, float* x, int rows, i
 hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd, float* x_out,
                               const void* gain, void* xn, float* hn, int rows, int d, float eps, int dtype,
                               cudaStream_t st);
+// Fused (bfloat16) layer stack: rows entering it and the normalised hidden rows leaving it (see GemmEpilogue).
+hydra_status rows_prepare(const float* src, const void* embed, const int* tok, int vocab, const void* gain, float* x, void* xg,
+                          float* ss, int rows, int d, int* status, cudaStream_t st);
+hydra_status finalize_hidden(const float* x, const float* ss, int ss_tiles, int ld, const void* gain, float eps, float* h,
+                             int rows, int d, cudaStream_t st);
 // table[r][j] = (cos, sin) of (pos0[b]+depth[i]) * theta^(-2j/head_dim), evaluated in double
 hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st);
 // q (operand dtype, [rows][H][hd], rotated), K/V cache rows (rotated K) from the QKV partial sums.

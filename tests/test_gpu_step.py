@@ -43,7 +43,9 @@ def test_small_bf16_hydrapp_ragged_batch():
     assert seen >= {0, 1, 2, 3, 4}, seen
 
 
-def test_small_bf16_simt_gemm_mode_and_root_only_tree():
+@pytest.mark.parametrize("mode", [1, 2])
+def test_small_bf16_other_gemm_modes_and_root_only_tree(mode):
+    """mode 1: SIMT GEMM; mode 2: tensor-core GEMM with the consumer operations in separate kernels."""
     from paper_2402_05109_b200 import Hydra
     m = ModelCfg(2, 256, 4, 64, 512, 1024, dtype="bf16")
     h = HeadCfg(2, 1, False)
@@ -51,7 +53,7 @@ def test_small_bf16_simt_gemm_mode_and_root_only_tree():
     prompts = make_prompts(6, [20], m.vocab)
     o = HydraOracle(m, h, [-1], w, 64)
     g = Hydra(m, h, [-1], {k: v.cuda() for k, v in w.items()}, 1, 64)
-    g.set_gemm_mode(1)
+    g.set_gemm_mode(mode)
     st = lockstep(o, g, prompts, 3, 6, plant=False)
     assert all(n == [0] for n in st.n_acc)
     g.close()
