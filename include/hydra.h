@@ -115,7 +115,9 @@ hydra_status hydra_verify(hydra_ctx*, const int32_t* tree_tok_dev, int32_t* amax
 hydra_status hydra_accept_compact(hydra_ctx*, const int32_t* tree_tok_dev, const int32_t* amax_dev,
                                   int32_t* n_acc_dev, int32_t* path_dev, int32_t* out_tok_dev, void* stream);
 
-/* draft + (optional planting) + verify + accept_compact on the library's own buffers. */
+/* draft + (optional planting) + verify + accept_compact on the library's own buffers.  From the second step
+ * after a prefill on, the step is captured into a CUDA graph (re-captured when an attention grid must grow
+ * or a pointer argument changes) and replayed with one launch; set HYDRA_NO_GRAPH=1 to launch kernel by kernel. */
 hydra_status hydra_step(hydra_ctx*, int32_t* n_acc_dev, int32_t* out_tok_dev, void* stream);
 
 /* Accept-exercise mode: plant_dev [batch][n_rows], -1 keeps the drafted token; applied between draft
@@ -154,8 +156,9 @@ enum { HYDRA_TIME_GEMM = 0, HYDRA_TIME_ATTENTION = 1, HYDRA_TIME_ACCEPT = 2 };
 hydra_status hydra_set_timing(hydra_ctx*, int on);
 hydra_status hydra_get_timing(hydra_ctx*, int kclass, double* ms_total, long long* launches, double* bytes_total);
 
-/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA with fused epilogues (default), 1 = the plain SIMT
- * kernel, 2 = tcgen05/TMA with the consumer operations in separate kernels. */
+/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA, consumer operations in their own kernels (default);
+ * 1 = the plain SIMT kernel; 2 = tcgen05/TMA with the consumer operations fused into the GEMM epilogues
+ * (applied by the CTA that completes a tile). */
 hydra_status hydra_set_gemm_mode(hydra_ctx*, int mode);
 
 const char* hydra_status_str(hydra_status);

@@ -43,6 +43,8 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
                                                                   const bf16* __restrict__ vc, RowSet rs,
                                                                   float* __restrict__ part_o, float* __restrict__ part_ml,
                                                                   int H, int max_seq, int nchunks, int chunk) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int LDS = HD + 8;                         // padded row (bf16 elements): conflict-free ldmatrix
   constexpr int KSTEPS = HD / 16;
   constexpr int NB = HD / 8;                          // output n-blocks
@@ -212,6 +214,8 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
 template <int HD>
 __global__ void __launch_bounds__(HD) tree_attn_tc_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                                                   RowSet rs, bf16* __restrict__ out, int H, int nchunks, int chunk) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x, h = blockIdx.y, b = r / rs.tc, i = r % rs.tc;
   const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
   const int k = threadIdx.x;
@@ -248,9 +252,9 @@ hydra_status run(const bf16* q, const bf16* kc, const bf16* vc, RowSet rs, bf16*
     HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_done = true;
   }
-  tree_attn_tc_kernel<HD><<<dim3(H, rs.batch, nchunks), NWARP * 32, smem, st>>>(q, kc, vc, rs, part_o, part_ml, H, max_seq, nchunks, chunk);
+  launch_pdl(tree_attn_tc_kernel<HD>, dim3(dim3(H, rs.batch, nchunks)), dim3(NWARP * 32), smem, st, q, kc, vc, rs, part_o, part_ml, H, max_seq, nchunks, chunk);
   HYDRA_LAUNCH_CHECK();
-  tree_attn_tc_combine_kernel<HD><<<dim3((unsigned)rows, H), HD, 0, st>>>(part_o, part_ml, rs, out, H, nchunks, chunk);
+  launch_pdl(tree_attn_tc_combine_kernel<HD>, dim3(dim3((unsigned)rows, H)), dim3(HD), 0, st, part_o, part_ml, rs, out, H, nchunks, chunk);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }

@@ -44,6 +44,12 @@ __device__ __forceinline__ float warp_max(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
+// Programmatic dependent launch: every kernel of the library starts with pdl_trigger() (lets the next kernel
+// in the stream get resident early) and pdl_wait() (blocks until the preceding kernel has completed and its
+// writes are visible) before it touches memory, so dependencies stay transitive along the stream.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
 
 // Where the partial sums of a GEMM output element live.  The tensor-core GEMM cuts the (tile, k-block) line
@@ -56,6 +62,18 @@ __host__ __device__ __forceinline__ int split_count(const SplitDesc& sd, int m, 
   return (int)((u0 + sd.kb - 1) / sd.q - u0 / sd.q) + 1;
 }
 inline SplitDesc single_slot(size_t stride) { return SplitDesc{1, 1, 1, 1 << 30, stride}; }
+
+// Launch with programmatic stream serialisation allowed (see pdl_wait).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 // Rows of one forward call: `batch` sequences with `tc` row slots each; sequence b uses its first
 // n_rows[b] slots (all tc when n_rows is null).  Row i of b has KV slot pos0[b]+i, rotary position

@@ -30,6 +30,7 @@
 // storing, lets its copies settle, frees its tensor memory and returns.
 #include "launch.h"
 #include <cuda.h>
+#include <cstdlib>
 #include <map>
 #include <mutex>
 #include <tuple>
@@ -41,7 +42,6 @@ namespace {
 constexpr int BLOCK_N = 128;             // weight rows per tile (MMA M)
 constexpr int BLOCK_K = 64;              // 64 bf16 = 128 bytes = one swizzle row
 constexpr int A_BYTES = BLOCK_N * BLOCK_K * 2;
-constexpr int SMEM_BUDGET = 100 * 1024;    // per CTA: two CTAs of consecutive (PDL-overlapped) kernels fit one SM
 constexpr uint32_t WAIT_LIMIT = 1u << 24;   // try_wait attempts before giving up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -134,7 +134,8 @@ __host__ __device__ constexpr uint32_t instr_desc(int mt) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mt >> 3) << 17) | ((uint32_t)(BLOCK_N >> 4) << 24);
 }
 
-template <int MT> struct TileCfg {
+template <int MT, int BUDGET_KB> struct TileCfg {
+  static constexpr int SMEM_BUDGET = BUDGET_KB * 1024;
   static constexpr int B_BYTES = MT * BLOCK_K * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 10 ? 10 : ((SMEM_BUDGET / STAGE_BYTES) < 3 ? 3 : (SMEM_BUDGET / STAGE_BYTES));
@@ -154,7 +155,11 @@ struct GemmArgs {
   float* x; void* xg; const void* gain; float* ss_out;                                   // EPI_RESID
   void* act; int f;                                                                      // EPI_GATEUP
   float* out;                                                                            // EPI_OUT
+  long long* trace;              // optional [grid][8] nanosecond timestamps of each CTA's phases (tuning aid), or null
 };
+
+__device__ __forceinline__ long long global_ns() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define TRACE(slot) do { if (a.trace) a.trace[blockIdx.x * 8 + (slot)] = global_ns(); } while (0)
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the 4 epilogue warps
 
@@ -162,34 +167,56 @@ __device__ __forceinline__ int tile_slots(const GemmArgs& a, int tile) {
   const long long u0 = (long long)tile * a.kb;
   return (int)((u0 + a.kb - 1) / a.q - u0 / a.q) + 1;
 }
-// Sum of a tile's partial slots for output element (m, n), in slot order (read past L1: other SMs wrote them).
-__device__ __forceinline__ float slot_sum(const GemmArgs& a, int ns, int m, int n) {
-  const float* p = a.part + (size_t)m * a.n + n;
-  float v = 0.f;
-  for (int s = 0; s < ns; ++s) v += __ldcg(p + (size_t)s * a.slot_stride);
-  return v;
+// Sums of a tile's partial slots for RB consecutive rows of one column, in slot order.  Loads of the RB rows are
+// independent so they overlap (the slots were written by other SMs: read past L1).  Rows >= m1 give 0.
+constexpr int RB = 32;
+__device__ __forceinline__ void slot_sums(const GemmArgs& a, int ns, int mb, int m1, int n, float (&v)[RB]) {
+  const float* p = a.part + (size_t)mb * a.n + n;
+#pragma unroll
+  for (int r = 0; r < RB; ++r) v[r] = 0.f;
+  for (int s = 0; s < ns; ++s) {
+    const float* ps = p + (size_t)s * a.slot_stride;
+#pragma unroll
+    for (int r = 0; r < RB; ++r)
+      if (mb + r < m1) v[r] += __ldcg(ps + (size_t)r * a.n);
+  }
 }
 
 // Consumer operation applied by the last arriver of a tile (or of a gate/up tile pair).  tid = column within
-// the tile (0..127); all 128 epilogue threads call it.
+// the tile (0..127); all 128 epilogue threads call it.  Rows are processed RB at a time.
 template <int MT>
-__device__ void apply_epilogue(const GemmArgs& a, int tile, int tid, const float* s_inv, float (*s_ex)[128], float (*s_ss)[MT]) {
+__device__ void apply_epilogue(const GemmArgs& a, int tile, int tid, const float* s_inv, float (*s_ss)[MT]) {
   const int tn = tile % a.n_tiles, tm = tile / a.n_tiles;
   const int m0 = tm * MT, m1 = min(m0 + MT, a.m);
   const int warp4 = tid >> 5, lane = tid & 31;
   if (a.epi == EPI_OUT) {
     const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
-    for (int m = m0; m < m1; ++m) a.out[(size_t)m * a.n + n] = slot_sum(a, ns, m, n) * s_inv[m];
+    for (int mb = m0; mb < m1; mb += RB) {
+      float v[RB];
+      slot_sums(a, ns, mb, m1, n, v);
+#pragma unroll
+      for (int r = 0; r < RB; ++r)
+        if (mb + r < m1) a.out[(size_t)(mb + r) * a.n + n] = v[r] * s_inv[mb + r];
+    }
   } else if (a.epi == EPI_RESID) {
     const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
     const float gn = a.gain ? __bfloat162float(reinterpret_cast<const bf16*>(a.gain)[n]) : 0.f;
-    for (int m = m0; m < m1; ++m) {
-      const size_t idx = (size_t)m * a.n + n;
-      const float xv = a.x[idx] + slot_sum(a, ns, m, n);
-      a.x[idx] = xv;
-      if (a.gain) reinterpret_cast<bf16*>(a.xg)[idx] = __float2bfloat16_rn(xv * gn);
-      const float ss = warp_sum(xv * xv);
-      if (lane == 0) s_ss[warp4][m - m0] = ss;
+    for (int mb = m0; mb < m1; mb += RB) {
+      float v[RB], xv[RB];
+#pragma unroll
+      for (int r = 0; r < RB; ++r) xv[r] = mb + r < m1 ? a.x[(size_t)(mb + r) * a.n + n] : 0.f;
+      slot_sums(a, ns, mb, m1, n, v);
+#pragma unroll
+      for (int r = 0; r < RB; ++r) {
+        xv[r] += v[r];
+        if (mb + r < m1) {
+          const size_t idx = (size_t)(mb + r) * a.n + n;
+          a.x[idx] = xv[r];
+          if (a.gain) reinterpret_cast<bf16*>(a.xg)[idx] = __float2bfloat16_rn(xv[r] * gn);
+        }
+        const float ss = warp_sum(xv[r] * xv[r]);
+        if (lane == 0 && mb + r < m1) s_ss[warp4][mb + r - m0] = ss;
+      }
     }
     epi_bar();
     for (int r = tid; r < m1 - m0; r += 128)
@@ -200,45 +227,57 @@ __device__ void apply_epilogue(const GemmArgs& a, int tile, int tid, const float
     const int tg = tm * a.n_tiles + p, tu = tg + half_tiles;
     const int nsg = tile_slots(a, tg), nsu = tile_slots(a, tu);
     const int c = p * BLOCK_N + tid;
-    for (int m = m0; m < m1; ++m) {
-      const float sc = s_inv[m];
-      const float g = slot_sum(a, nsg, m, c) * sc, u = slot_sum(a, nsu, m, a.f + c) * sc;
-      reinterpret_cast<bf16*>(a.act)[(size_t)m * a.f + c] = __float2bfloat16_rn(silu_f(g) * u);
+    for (int mb = m0; mb < m1; mb += RB) {
+      float g[RB], u[RB];
+      slot_sums(a, nsg, mb, m1, c, g);
+      slot_sums(a, nsu, mb, m1, a.f + c, u);
+#pragma unroll
+      for (int r = 0; r < RB; ++r)
+        if (mb + r < m1) {
+          const float sc = s_inv[mb + r];
+          reinterpret_cast<bf16*>(a.act)[(size_t)(mb + r) * a.f + c] = __float2bfloat16_rn(silu_f(g[r] * sc) * (u[r] * sc));
+        }
     }
   } else if (a.epi == EPI_QKV) {
     const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
     const int d = a.H * a.hd, half = a.hd >> 1;
     const int which = n / d, within = n % d, head = within / a.hd, jl = within % a.hd;
-    const int partner = jl < half ? tid + half : tid - half;
     bf16* kv = reinterpret_cast<bf16*>(which == 1 ? a.kc : a.vc);
-    for (int m = m0; m < m1; ++m) {
-      const int b = m / a.rs.tc, i = m % a.rs.tc;
-      const int nr = a.rs.n_rows ? a.rs.n_rows[b] : a.rs.tc;
-      const int slot = a.rs.pos0[b] + i;
-      const bool row_ok = i < nr && slot >= 0 && slot < a.max_seq;       // uniform over the 128 threads
-      if (i < nr && !row_ok && tid == 0) atomicOr(a.status, ST_BOUNDS);
-      const float v = row_ok ? slot_sum(a, ns, m, n) * s_inv[m] : 0.f;
-      float outv = v;
-      if (which < 2) {                                                   // rotate q and k (half-split pairing)
-        float* ex = s_ex[m & 1];
-        ex[tid] = v;
-        epi_bar();
-        const float pv = ex[partner];
-        const float2 cs = row_ok ? a.rope[(size_t)m * half + (jl % half)] : make_float2(1.f, 0.f);
-        outv = jl < half ? v * cs.x - pv * cs.y : v * cs.x + pv * cs.y;
+    const int n_partner = n + (jl < half ? half : -half);
+    for (int mb = m0; mb < m1; mb += RB) {
+      float v[RB], pv[RB];
+      slot_sums(a, ns, mb, m1, n, v);
+      if (which < 2) slot_sums(a, ns, mb, m1, n_partner, pv);            // the other element of the rotation pair
+      bool row_ok[RB]; int bq[RB], slot[RB];
+#pragma unroll
+      for (int r = 0; r < RB; ++r) {
+        const int m = mb + r < m1 ? mb + r : m1 - 1;
+        const int b = m / a.rs.tc, i = m % a.rs.tc;
+        const int nr = a.rs.n_rows ? a.rs.n_rows[b] : a.rs.tc;
+        bq[r] = b; slot[r] = a.rs.pos0[b] + i;
+        const bool in_rows = mb + r < m1 && i < nr;
+        row_ok[r] = in_rows && slot[r] >= 0 && slot[r] < a.max_seq;
+        if (in_rows && !row_ok[r] && tid == 0) atomicOr(a.status, ST_BOUNDS);
+        if (which < 2 && row_ok[r]) {                                    // rotate q and k (half-split pairing)
+          const float2 cs = a.rope[(size_t)m * half + (jl % half)];
+          v[r] = jl < half ? v[r] * cs.x - pv[r] * cs.y : v[r] * cs.x + pv[r] * cs.y;
+        }
+        v[r] *= s_inv[m];
       }
-      if (row_ok) {
-        if (which == 0) reinterpret_cast<bf16*>(a.q_out)[(size_t)m * d + within] = __float2bfloat16_rn(outv);
-        else kv[(((size_t)b * a.H + head) * a.max_seq + slot) * a.hd + jl] = __float2bfloat16_rn(outv);
-      }
+#pragma unroll
+      for (int r = 0; r < RB; ++r)
+        if (row_ok[r]) {
+          if (which == 0) reinterpret_cast<bf16*>(a.q_out)[(size_t)(mb + r) * d + within] = __float2bfloat16_rn(v[r]);
+          else kv[(((size_t)bq[r] * a.H + head) * a.max_seq + slot[r]) * a.hd + jl] = __float2bfloat16_rn(v[r]);
+        }
     }
   }
 }
 
-template <int MT>
+template <int MT, int BUDGET_KB>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const GemmArgs a) {
-  using C = TileCfg<MT>;
+  using C = TileCfg<MT, BUDGET_KB>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = tiles + C::STAGES * C::STAGE_BYTES;
@@ -250,7 +289,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const uint32_t tmem_slot = bars + 8u * (3 * C::STAGES + 4);
   __shared__ int s_abort, s_last;
   __shared__ float s_inv[512];               // inv_rms of the operand rows (fused epilogues need m <= 512)
-  __shared__ float s_ex[2][128];
   __shared__ float s_ss[4][MT];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -259,6 +297,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int n_units = u_end - u_begin;
 
   if (threadIdx.x == 0) {
+    TRACE(0);
     s_abort = 0;
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(fullw_bar(s), 1); mbar_init(fullx_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(accfull_bar(i), 1); mbar_init(accempty_bar(i), 4); }
@@ -270,6 +309,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (threadIdx.x == 0) TRACE(1);
   grid_dep_launch();                       // all CTAs of this grid are resident: let the next kernel get ready
   uint32_t tmem_base;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
@@ -291,6 +331,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         mbar_arrive_expect_tx(fullw_bar(i), A_BYTES);
         tma_load_2d(tiles + i * C::STAGE_BYTES, &tmW, kcol, nrow, fullw_bar(i), pol_w);
       }
+      TRACE(2);
       grid_dep_wait();                     // activations are the preceding kernel's output
       for (int i = 0; i < n_units; ++i) {
         const int s = i % C::STAGES;
@@ -325,6 +366,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           const int s = i % C::STAGES;
           const uint32_t ph = (i / C::STAGES) & 1;
           if (!mbar_wait(fullw_bar(s), ph) || !mbar_wait(fullx_bar(s), ph)) { ok = false; break; }
+          if (i == 0) TRACE(3);
           tc_fence_after();
           const uint32_t a_addr = tiles + s * C::STAGE_BYTES;
           const uint64_t adesc = smem_desc_sw128(a_addr);
@@ -338,6 +380,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         umma_commit(accfull_bar(acc));                   // segment complete: hand the accumulator to the epilogue
         ++seg;
       }
+      TRACE(4);
       if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
     }
   } else {
@@ -360,6 +403,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int acc = seg & 1;
       const uint32_t acc_ph = (seg >> 1) & 1;
       if (!mbar_wait(accfull_bar(acc), acc_ph)) { if (lane == 0) atomicOr(a.status, ST_TIMEOUT); break; }
+      if (epi_tid == 0 && i + seg_len >= n_units) TRACE(5);
       tc_fence_after();
       const int slot = blockIdx.x - (int)(((long long)tile * a.kb) / a.q);
       const int n0 = (tile % a.n_tiles) * BLOCK_N, m0 = (tile / a.n_tiles) * MT;
@@ -397,12 +441,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         epi_bar();
         if (s_last) {
           __threadfence();
-          apply_epilogue<MT>(a, tile, epi_tid, s_inv, s_ex, s_ss);
+          apply_epilogue<MT>(a, tile, epi_tid, s_inv, s_ss);
         }
       }
       i += seg_len;
       ++seg;
     }
+    if (epi_tid == 0) TRACE(6);
   }
   tc_fence_before();
   __syncthreads();
@@ -410,6 +455,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     for (int i = 0; i < 2000; ++i) __nanosleep(100);
   }
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, C::TMEM_COLS); }
+  if (threadIdx.x == 32) TRACE(7);
 }
 
 // ---- tensor maps -------------------------------------------------------------------------------
@@ -465,12 +511,12 @@ int sm_count() {
   return n;
 }
 
-template <int MT>
-hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs& a, int grid, cudaStream_t st) {
-  using C = TileCfg<MT>;
+template <int MT, int BUDGET_KB>
+hydra_status launch_b(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs& a, int grid, cudaStream_t st) {
+  using C = TileCfg<MT, BUDGET_KB>;
   static bool attr_done = false;
   if (!attr_done) {
-    HYDRA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    HYDRA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<MT, BUDGET_KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_done = true;
   }
   cudaLaunchConfig_t cfg = {};
@@ -479,9 +525,18 @@ hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
-  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<MT>, tw, tx, a));
+  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<MT, BUDGET_KB>, tw, tx, a));
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
+}
+
+// Shared memory per CTA: 100 KB lets the CTAs of two consecutive (programmatically overlapped) GEMMs share an SM;
+// HYDRA_GEMM_SMEM_KB=200 selects a deeper ring with one CTA per SM.
+template <int MT>
+hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs& a, int grid, cudaStream_t st) {
+  static const int kb = []() { const char* e = getenv("HYDRA_GEMM_SMEM_KB"); return e ? atoi(e) : 100; }();
+  if (kb >= 200) return launch_b<MT, 200>(tw, tx, a, grid, st);
+  return launch_b<MT, 100>(tw, tx, a, grid, st);
 }
 
 }  // namespace
@@ -539,6 +594,7 @@ hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part
     a.max_seq = epi->max_seq; a.x = epi->x; a.xg = epi->xg; a.gain = epi->gain; a.ss_out = epi->ss_out; a.act = epi->act;
     a.f = epi->f; a.out = epi->out;
   }
+  a.trace = epi ? epi->trace : nullptr;
   if (sd_out) *sd_out = sd;
   switch (sd.mt) {
     case 16: return launch<16>(tw, tx, a, grid, st);

@@ -2,7 +2,10 @@
 #include "launch.h"
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
+#include <map>
+#include <tuple>
 #include <new>
 #include <string>
 #include <vector>
@@ -73,6 +76,16 @@ struct hydra_ctx {
   long long launches;
   // optional per-kernel-class timing (benchmarks): event pairs recorded around launches of a class
   struct Timed { cudaEvent_t a, b; int cls; double bytes; };
+  // whole-step CUDA graphs, keyed by everything a captured step freezes (attention grid sizes, buffer pointers)
+  struct GraphKey {
+    int len_verify, len_prefix; const void *plant, *n_acc, *out_tok;
+    bool operator<(const GraphKey& o) const {
+      return std::tie(len_verify, len_prefix, plant, n_acc, out_tok) < std::tie(o.len_verify, o.len_prefix, o.plant, o.n_acc, o.out_tok);
+    }
+  };
+  struct StepGraph { cudaGraphExec_t exec; long long launches; };
+  std::map<GraphKey, StepGraph> graphs;
+  int use_graph; long long steps_done;
   int timing;
   std::vector<Timed> timed;
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
@@ -339,6 +352,9 @@ hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int le
 }
 
 int max_len_ub(const hydra_ctx* c) { int v = 0; for (int b = 0; b < c->batch; ++b) v = std::max(v, c->len_ub[b]); return v; }
+// Upper bound of the KV length used to size attention grids, rounded up so that it (and a captured step graph)
+// stays valid for many steps; CTAs beyond the real length exit at once.
+int len_bucket(const hydra_ctx* c, int v) { v = (v + 511) / 512 * 512; return std::min(v, c->m.max_seq); }
 
 hydra_status do_draft(hydra_ctx* c, int* tree_tok, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
@@ -346,7 +362,7 @@ hydra_status do_draft(hydra_ctx* c, int* tree_tok, cudaStream_t st) {
   if (c->h.prefix_attn) {
     HYDRA_TRY(prefix_rowset(c->d_len, c->d_n_new, c->d_pos0, c->d_nrows, B, st));
     RowSet rs{B, K + 1, c->d_nrows, c->d_pos0, c->d_chain_depth, c->d_chain_mask};
-    HYDRA_TRY(run_prefix(c, c->h_new, rs, max_len_ub(c), st));
+    HYDRA_TRY(run_prefix(c, c->h_new, rs, len_bucket(c, max_len_ub(c)), st));
     HYDRA_TRY(pick_last_row(c->x, c->d_nrows, K + 1, c->hprime, B, d, st));
   } else {
     HYDRA_TRY(pick_last_row(c->h_new, c->d_n_new, K + 1, c->hprime, B, d, st));
@@ -376,7 +392,7 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
   const hydra_model_cfg& m = c->m;
   const int rows = c->batch * c->T;
   RowSet rs{c->batch, c->T, nullptr, c->d_len, c->d_depth, c->d_anc};
-  HYDRA_TRY(run_base(c, tree_tok, rs, max_len_ub(c) + c->T, st));
+  HYDRA_TRY(run_base(c, tree_tok, rs, len_bucket(c, max_len_ub(c) + c->T), st));
   if (fused_ok(c, rows)) {                 // c->xn holds x * final_norm gain; the LM head scales its rows by inv_rms
     float* lg = logits ? logits : c->logits;
     GemmEpilogue e; e.kind = EPI_OUT; norm_in(c, e); e.out = lg;
@@ -401,8 +417,21 @@ hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* 
     TimeScope ts(c, HYDRA_TIME_ACCEPT, 0.0, st);
     HYDRA_TRY(accept_compact(a, st));
   }
-  for (int b = 0; b < c->batch; ++b) c->len_ub[b] += c->Ktree + 1;
   return HYDRA_OK;
+}
+
+void bump_len_ub(hydra_ctx* c) { for (int b = 0; b < c->batch; ++b) c->len_ub[b] += c->Ktree + 1; }
+
+hydra_status enqueue_step(hydra_ctx* c, int* n_acc, int* out_tok, cudaStream_t st) {
+  HYDRA_TRY(do_draft(c, c->d_tree_tok, st));
+  if (c->plant) HYDRA_TRY(apply_plant(c->d_tree_tok, c->plant, c->batch * c->T, st));
+  HYDRA_TRY(do_verify(c, c->d_tree_tok, c->d_amax, nullptr, st));
+  return do_accept(c, c->d_tree_tok, c->d_amax, n_acc, nullptr, out_tok, st);
+}
+
+void drop_graphs(hydra_ctx* c) {
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second.exec);
+  c->graphs.clear();
 }
 
 bool capacity_ok(const hydra_ctx* c) {
@@ -463,7 +492,8 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
   }
   c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
   carve(c, *m, *h, th, (char*)ws);
-  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->fused = 1; c->ss_tiles = 1; c->plant = nullptr; c->launches = 0; c->timing = 0;
+  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->fused = 0; c->ss_tiles = 1; c->plant = nullptr; c->launches = 0; c->timing = 0; c->steps_done = 0;
+  { const char* e = getenv("HYDRA_NO_GRAPH"); c->use_graph = !(e && e[0] == '1'); }
   c->len_ub.assign(m->max_batch, 0);
   // clear the workspace, upload the static tables
   auto fail = [&](cudaError_t e, const char* what) { set_last_error(what, e); delete c; return HYDRA_ERR_CUDA; };
@@ -488,6 +518,7 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
 hydra_status hydra_destroy(hydra_ctx* c) {
   if (!c) return HYDRA_ERR_INVALID;
   cudaError_t e = cudaDeviceSynchronize();
+  drop_graphs(c);
   for (auto& t : c->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
   for (auto& p : c->event_pool) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
   delete c;
@@ -528,6 +559,7 @@ hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const
   HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, batch, m.vocab, m.d_model, &sd, st));
   HYDRA_TRY(argmax_rows(c->part, sd, nullptr, c->d_root_tok, batch, m.vocab, st));
   for (int b = 0; b < batch; ++b) c->len_ub[b] = plen[b];
+  drop_graphs(c);
   c->state = ST_READY;
   return HYDRA_OK;
 }
@@ -558,6 +590,7 @@ hydra_status hydra_accept_compact(hydra_ctx* c, const int32_t* tree_tok, const i
   if (c->state != ST_VERIFIED) return HYDRA_ERR_STATE;
   CounterScope cs(c);
   HYDRA_TRY(do_accept(c, tree_tok, amax, n_acc, path, out_tok, (cudaStream_t)stream));
+  bump_len_ub(c);
   c->state = ST_READY;
   return HYDRA_OK;
 }
@@ -568,10 +601,34 @@ hydra_status hydra_step(hydra_ctx* c, int32_t* n_acc, int32_t* out_tok, void* st
   if (!capacity_ok(c)) return HYDRA_ERR_CAPACITY;
   CounterScope cs(c);
   cudaStream_t st = (cudaStream_t)stream;
-  HYDRA_TRY(do_draft(c, c->d_tree_tok, st));
-  if (c->plant) HYDRA_TRY(apply_plant(c->d_tree_tok, c->plant, c->batch * c->T, st));
-  HYDRA_TRY(do_verify(c, c->d_tree_tok, c->d_amax, nullptr, st));
-  HYDRA_TRY(do_accept(c, c->d_tree_tok, c->d_amax, n_acc, nullptr, out_tok, st));
+  if (!c->use_graph || c->timing || c->steps_done == 0) {      // the first step runs uncaptured (one-time lazy set-up)
+    HYDRA_TRY(enqueue_step(c, n_acc, out_tok, st));
+  } else {
+    const int lu = max_len_ub(c);
+    hydra_ctx::GraphKey key{len_bucket(c, lu + c->T), len_bucket(c, lu), c->plant, n_acc, out_tok};
+    auto it = c->graphs.find(key);
+    if (it == c->graphs.end()) {
+      if (c->graphs.size() >= 8) drop_graphs(c);
+      const long long before = c->launches;
+      HYDRA_CUDA(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+      hydra_status es = enqueue_step(c, n_acc, out_tok, st);
+      cudaGraph_t graph = nullptr;
+      cudaError_t ce = cudaStreamEndCapture(st, &graph);
+      const long long captured = c->launches - before;
+      c->launches = before;
+      if (es != HYDRA_OK) { if (graph) cudaGraphDestroy(graph); return es; }
+      if (ce != cudaSuccess) { set_last_error("cudaStreamEndCapture", ce); return HYDRA_ERR_CUDA; }
+      cudaGraphExec_t exec = nullptr;
+      ce = cudaGraphInstantiate(&exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (ce != cudaSuccess) { set_last_error("cudaGraphInstantiate", ce); return HYDRA_ERR_CUDA; }
+      it = c->graphs.emplace(key, hydra_ctx::StepGraph{exec, captured}).first;
+    }
+    HYDRA_CUDA(cudaGraphLaunch(it->second.exec, st));
+    c->launches += it->second.launches;
+  }
+  bump_len_ub(c);
+  ++c->steps_done;
   return HYDRA_OK;
 }
 
@@ -649,7 +706,8 @@ hydra_status hydra_get_timing(hydra_ctx* c, int kclass, double* ms_total, long l
 hydra_status hydra_set_gemm_mode(hydra_ctx* c, int mode) {
   if (!c || mode < 0 || mode > 2) return HYDRA_ERR_INVALID;
   c->gemm_mode = mode == 1 ? 1 : 0;
-  c->fused = mode == 0;
+  c->fused = mode == 2;
+  drop_graphs(c);
   return HYDRA_OK;
 }
 

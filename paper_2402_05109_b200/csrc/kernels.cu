@@ -23,6 +23,8 @@ template <> struct Vec4<bf16> {
 template <typename T, int MR>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ w,
                                                         float* __restrict__ out, int m, int n, int k) {
+  pdl_trigger();
+  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int col = blockIdx.x * 8 + warp;
   const int m0 = blockIdx.y * MR;
@@ -53,13 +55,15 @@ hydra_status gemm_simt(const void* x, const void* w, float* out, int m, int n, i
   if (m <= 0 || n <= 0 || k <= 0 || (k & 3)) return HYDRA_ERR_UNSUPPORTED;
   constexpr int MR = 16;
   dim3 grid((n + 7) / 8, (m + MR - 1) / MR);
-  if (dtype == 0) gemm_simt_kernel<float, MR><<<grid, 256, 0, st>>>((const float*)x, (const float*)w, out, m, n, k);
-  else gemm_simt_kernel<bf16, MR><<<grid, 256, 0, st>>>((const bf16*)x, (const bf16*)w, out, m, n, k);
+  if (dtype == 0) launch_pdl(gemm_simt_kernel<float, MR>, dim3(grid), dim3(256), 0, st, (const float*)x, (const float*)w, out, m, n, k);
+  else launch_pdl(gemm_simt_kernel<bf16, MR>, dim3(grid), dim3(256), 0, st, (const bf16*)x, (const bf16*)w, out, m, n, k);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 __global__ void reduce_splits_kernel(const float* __restrict__ part, SplitDesc sd, float* __restrict__ out, int m, int n) {
+  pdl_trigger();
+  pdl_wait();
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (size_t)m * n) return;
   const int ns = split_count(sd, (int)(i / n), (int)(i % n));
@@ -68,7 +72,7 @@ __global__ void reduce_splits_kernel(const float* __restrict__ part, SplitDesc s
   out[i] = s;
 }
 hydra_status reduce_splits(const float* part, SplitDesc sd, float* out, int m, int n, cudaStream_t st) {
-  reduce_splits_kernel<<<(unsigned)(((size_t)m * n + 255) / 256), 256, 0, st>>>(part, sd, out, m, n);
+  launch_pdl(reduce_splits_kernel, dim3((unsigned)(((size_t)m * n + 255) / 256)), dim3(256), 0, st, part, sd, out, m, n);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -79,6 +83,8 @@ hydra_status reduce_splits(const float* part, SplitDesc sd, float* out, int m, i
 template <typename T>
 __global__ void embed_rows_kernel(const T* __restrict__ embed, const int* __restrict__ tok, float* __restrict__ x, int d,
                                   int vocab, int* status) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x;
   int t = tok[r];
   if (t < 0 || t >= vocab) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); t = 0; }
@@ -87,8 +93,8 @@ __global__ void embed_rows_kernel(const T* __restrict__ embed, const int* __rest
 }
 hydra_status embed_rows(const void* embed, const int* tok, float* x, int rows, int d, int vocab, int dtype, int* status,
                         cudaStream_t st) {
-  if (dtype == 0) embed_rows_kernel<float><<<rows, 256, 0, st>>>((const float*)embed, tok, x, d, vocab, status);
-  else embed_rows_kernel<bf16><<<rows, 256, 0, st>>>((const bf16*)embed, tok, x, d, vocab, status);
+  if (dtype == 0) launch_pdl(embed_rows_kernel<float>, dim3(rows), dim3(256), 0, st, (const float*)embed, tok, x, d, vocab, status);
+  else launch_pdl(embed_rows_kernel<bf16>, dim3(rows), dim3(256), 0, st, (const bf16*)embed, tok, x, d, vocab, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -128,6 +134,8 @@ __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const fl
                                                                         SplitDesc sd, float* x_out,
                                                                         const T* __restrict__ gain, T* __restrict__ xn,
                                                                         float* __restrict__ hn, int d, float eps) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const size_t base = (size_t)blockIdx.x * d;
   float ss = 0.f;
@@ -159,10 +167,10 @@ hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd,
                               cudaStream_t st) {
   if (d & 3) return HYDRA_ERR_UNSUPPORTED;
   if (dtype == 0)
-    residual_rmsnorm_kernel<float><<<rows, NORM_THREADS, 0, st>>>(res, part, sd, x_out, (const float*)gain,
+    launch_pdl(residual_rmsnorm_kernel<float>, dim3(rows), dim3(NORM_THREADS), 0, st, res, part, sd, x_out, (const float*)gain,
                                                                   (float*)xn, hn, d, eps);
   else
-    residual_rmsnorm_kernel<bf16><<<rows, NORM_THREADS, 0, st>>>(res, part, sd, x_out, (const bf16*)gain,
+    launch_pdl(residual_rmsnorm_kernel<bf16>, dim3(rows), dim3(NORM_THREADS), 0, st, res, part, sd, x_out, (const bf16*)gain,
                                                                  (bf16*)xn, hn, d, eps);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -173,6 +181,8 @@ __global__ void __launch_bounds__(NORM_THREADS) rows_prepare_kernel(const float*
                                                                     const int* __restrict__ tok, int vocab,
                                                                     const bf16* __restrict__ gain, float* __restrict__ x,
                                                                     bf16* __restrict__ xg, float* __restrict__ ss, int d, int* status) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sh[32];
   const int r = blockIdx.x;
   const size_t base = (size_t)r * d;
@@ -195,7 +205,7 @@ __global__ void __launch_bounds__(NORM_THREADS) rows_prepare_kernel(const float*
 }
 hydra_status rows_prepare(const float* src, const void* embed, const int* tok, int vocab, const void* gain, float* x, void* xg,
                           float* ss, int rows, int d, int* status, cudaStream_t st) {
-  rows_prepare_kernel<<<rows, NORM_THREADS, 0, st>>>(src, (const bf16*)embed, tok, vocab, (const bf16*)gain, x, (bf16*)xg, ss, d, status);
+  launch_pdl(rows_prepare_kernel, dim3(rows), dim3(NORM_THREADS), 0, st, src, (const bf16*)embed, tok, vocab, (const bf16*)gain, x, (bf16*)xg, ss, d, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -204,6 +214,8 @@ hydra_status rows_prepare(const float* src, const void* embed, const int* tok, i
 __global__ void __launch_bounds__(NORM_THREADS) finalize_hidden_kernel(const float* __restrict__ x, const float* __restrict__ ss,
                                                                        int ss_tiles, int ld, const bf16* __restrict__ gain,
                                                                        float eps, float* __restrict__ h, int d) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x;
   float tot = 0.f;
   for (int t = 0; t < ss_tiles; ++t) tot += ss[(size_t)t * ld + r];
@@ -217,7 +229,7 @@ __global__ void __launch_bounds__(NORM_THREADS) finalize_hidden_kernel(const flo
 }
 hydra_status finalize_hidden(const float* x, const float* ss, int ss_tiles, int ld, const void* gain, float eps, float* h,
                              int rows, int d, cudaStream_t st) {
-  finalize_hidden_kernel<<<rows, NORM_THREADS, 0, st>>>(x, ss, ss_tiles, ld, (const bf16*)gain, eps, h, d);
+  launch_pdl(finalize_hidden_kernel, dim3(rows), dim3(NORM_THREADS), 0, st, x, ss, ss_tiles, ld, (const bf16*)gain, eps, h, d);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -226,6 +238,8 @@ hydra_status finalize_hidden(const float* x, const float* ss, int ss_tiles, int 
 // Rotary table + QKV post-processing (sum partials, rotate q and k, append K,V to the cache)
 // ------------------------------------------------------------------------------------------------
 __global__ void rope_table_kernel(RowSet rs, float2* __restrict__ table, int half, float theta) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x, b = r / rs.tc, i = r % rs.tc;
   int pos = rs.pos0[b] + rs.depth[i];
   for (int j = threadIdx.x; j < half; j += blockDim.x) {
@@ -236,7 +250,7 @@ __global__ void rope_table_kernel(RowSet rs, float2* __restrict__ table, int hal
   }
 }
 hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st) {
-  rope_table_kernel<<<rs.batch * rs.tc, 64, 0, st>>>(rs, table, head_dim / 2, theta);
+  launch_pdl(rope_table_kernel, dim3(rs.batch * rs.tc), dim3(64), 0, st, rs, table, head_dim / 2, theta);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -246,6 +260,8 @@ __global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restr
                                                             const float2* __restrict__ table, T* __restrict__ q,
                                                             T* __restrict__ kc, T* __restrict__ vc, RowSet rs, int H,
                                                             int hd, int max_seq, int* status) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x, h = blockIdx.y, b = r / rs.tc, i = r % rs.tc;
   const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
   if (i >= nr) return;
@@ -280,10 +296,10 @@ hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table
                             cudaStream_t st) {
   dim3 grid(rs.batch * rs.tc, H);
   if (dtype == 0)
-    qkv_rope_store_kernel<float><<<grid, 64, 0, st>>>(part, sd, table, (float*)q, (float*)kcache, (float*)vcache,
+    launch_pdl(qkv_rope_store_kernel<float>, dim3(grid), dim3(64), 0, st, part, sd, table, (float*)q, (float*)kcache, (float*)vcache,
                                                       rs, H, hd, max_seq, status);
   else
-    qkv_rope_store_kernel<bf16><<<grid, 64, 0, st>>>(part, sd, table, (bf16*)q, (bf16*)kcache, (bf16*)vcache, rs,
+    launch_pdl(qkv_rope_store_kernel<bf16>, dim3(grid), dim3(64), 0, st, part, sd, table, (bf16*)q, (bf16*)kcache, (bf16*)vcache, rs,
                                                      H, hd, max_seq, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -302,6 +318,8 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) tree_attn_kernel(const T* __re
                                                                    const T* __restrict__ vc, RowSet rs,
                                                                    float* __restrict__ part_o, float* __restrict__ part_ml,
                                                                    int H, int max_seq, int nchunks) {
+  pdl_trigger();
+  pdl_wait();
   extern __shared__ float smem[];
   constexpr int RPW = 8;                                  // query rows per warp (tc <= 64)
   constexpr int KPL = HD / 32;                            // output dims per lane
@@ -390,6 +408,8 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) tree_attn_kernel(const T* __re
 template <typename T, int HD>
 __global__ void tree_attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, RowSet rs,
                                          T* __restrict__ out, int H, int nchunks) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x, h = blockIdx.y, b = r / rs.tc, i = r % rs.tc;
   const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
   const int k = threadIdx.x;
@@ -431,10 +451,10 @@ static hydra_status tree_attention_t(const T* q, const T* kc, const T* vc, RowSe
     HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_kernel<T, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_done = true;
   }
-  tree_attn_kernel<T, HD><<<dim3(H, rs.batch, nchunks), ATT_WARPS * 32, smem, st>>>(q, kc, vc, rs, part_o, part_ml, H,
+  launch_pdl(tree_attn_kernel<T, HD>, dim3(dim3(H, rs.batch, nchunks)), dim3(ATT_WARPS * 32), smem, st, q, kc, vc, rs, part_o, part_ml, H,
                                                                                    max_seq, nchunks);
   HYDRA_LAUNCH_CHECK();
-  tree_attn_combine_kernel<T, HD><<<dim3((unsigned)rows, H), HD, 0, st>>>(part_o, part_ml, rs, out, H, nchunks);
+  launch_pdl(tree_attn_combine_kernel<T, HD>, dim3(dim3((unsigned)rows, H)), dim3(HD), 0, st, part_o, part_ml, rs, out, H, nchunks);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -456,6 +476,8 @@ hydra_status tree_attention(const void* q, const void* kc, const void* vc, RowSe
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void silu_mul_kernel(const float* __restrict__ part, SplitDesc sd, T* __restrict__ act, int rows, int f) {
+  pdl_trigger();
+  pdl_wait();
   size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= (size_t)rows * f) return;
   const int r = (int)(i / f), c = (int)(i % f);
@@ -470,8 +492,8 @@ hydra_status silu_mul(const float* part, SplitDesc sd, void* act, int rows, int 
   if (f & 3) return HYDRA_ERR_UNSUPPORTED;
   size_t n = (size_t)rows * f / 4;
   unsigned grid = (unsigned)((n + 255) / 256);
-  if (dtype == 0) silu_mul_kernel<float><<<grid, 256, 0, st>>>(part, sd, (float*)act, rows, f);
-  else silu_mul_kernel<bf16><<<grid, 256, 0, st>>>(part, sd, (bf16*)act, rows, f);
+  if (dtype == 0) launch_pdl(silu_mul_kernel<float>, dim3(grid), dim3(256), 0, st, part, sd, (float*)act, rows, f);
+  else launch_pdl(silu_mul_kernel<bf16>, dim3(grid), dim3(256), 0, st, part, sd, (bf16*)act, rows, f);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -517,6 +539,8 @@ __device__ __forceinline__ float summed(const float* part, const SplitDesc& sd, 
 
 __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restrict__ part, SplitDesc sd,
                                                           float* __restrict__ logits_out, int* __restrict__ amax, int vocab) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float shv[32];
   __shared__ int shi[32];
   const int row = blockIdx.x;
@@ -530,7 +554,7 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restric
   if (threadIdx.x == 0) amax[row] = bi;
 }
 hydra_status argmax_rows(const float* part, SplitDesc sd, float* logits_out, int* amax, int rows, int vocab, cudaStream_t st) {
-  argmax_rows_kernel<<<rows, 256, 0, st>>>(part, sd, logits_out, amax, vocab);
+  launch_pdl(argmax_rows_kernel, dim3(rows), dim3(256), 0, st, part, sd, logits_out, amax, vocab);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -540,6 +564,8 @@ __global__ void __launch_bounds__(256) topk_children_kernel(const float* __restr
                                                             const int* __restrict__ first_child,
                                                             const int* __restrict__ n_child, int* __restrict__ tree_tok,
                                                             int T, int vocab) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float shv[32];
   __shared__ int shi[32];
   const int row = blockIdx.x, b = row / lv.n_parents, j = row % lv.n_parents;
@@ -562,7 +588,7 @@ __global__ void __launch_bounds__(256) topk_children_kernel(const float* __restr
 }
 hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, const int* first_child,
                            const int* n_child, int* tree_tok, int batch, int T, int vocab, cudaStream_t st) {
-  topk_children_kernel<<<batch * lv.n_parents, 256, 0, st>>>(part, sd, logits, lv, first_child, n_child, tree_tok, T, vocab);
+  launch_pdl(topk_children_kernel, dim3(batch * lv.n_parents), dim3(256), 0, st, part, sd, logits, lv, first_child, n_child, tree_tok, T, vocab);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -575,6 +601,8 @@ __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restric
                                                           const int* __restrict__ root_tok, int* tree_tok,
                                                           const int* __restrict__ path_tab, LevelDesc lv, T* __restrict__ z,
                                                           int T_rows, int kp1, int d_model, int vocab, int* status) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.x, b = row / lv.n_parents, j = row % lv.n_parents;
   const int blk = blockIdx.y;                               // 0: hidden, 1..d: path tokens root..parent
   const int p = lv.parents[j];
@@ -595,10 +623,10 @@ hydra_status head_gather(const float* hprime, const void* embed, const int* root
                          cudaStream_t st) {
   dim3 grid(batch * lv.n_parents, lv.d + 1);
   if (dtype == 0)
-    head_gather_kernel<float><<<grid, 256, 0, st>>>(hprime, (const float*)embed, root_tok, tree_tok, path_tab, lv, (float*)z,
+    launch_pdl(head_gather_kernel<float>, dim3(grid), dim3(256), 0, st, hprime, (const float*)embed, root_tok, tree_tok, path_tab, lv, (float*)z,
                                                     T, kp1, d_model, vocab, status);
   else
-    head_gather_kernel<bf16><<<grid, 256, 0, st>>>(hprime, (const bf16*)embed, root_tok, tree_tok, path_tab, lv, (bf16*)z,
+    launch_pdl(head_gather_kernel<bf16>, dim3(grid), dim3(256), 0, st, hprime, (const bf16*)embed, root_tok, tree_tok, path_tab, lv, (bf16*)z,
                                                    T, kp1, d_model, vocab, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -608,6 +636,8 @@ template <typename T>
 __global__ void head_act_kernel(const float* res, int res_is_hprime, int rows_per_b, const float* __restrict__ part,
                                 SplitDesc sd, const T* __restrict__ bias, float* y_out, T* __restrict__ yb,
                                 int rows, int d) {
+  pdl_trigger();
+  pdl_wait();
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (size_t)rows * d) return;
   int r = (int)(i / d), c = (int)(i % d);
@@ -624,10 +654,10 @@ hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const
   size_t n = (size_t)rows * d;
   unsigned grid = (unsigned)((n + 255) / 256);
   if (dtype == 0)
-    head_act_kernel<float><<<grid, 256, 0, st>>>(res, res_is_hprime, rows_per_b, part, sd, (const float*)bias,
+    launch_pdl(head_act_kernel<float>, dim3(grid), dim3(256), 0, st, res, res_is_hprime, rows_per_b, part, sd, (const float*)bias,
                                                  y_out, (float*)yb, rows, d);
   else
-    head_act_kernel<bf16><<<grid, 256, 0, st>>>(res, res_is_hprime, rows_per_b, part, sd, (const bf16*)bias,
+    launch_pdl(head_act_kernel<bf16>, dim3(grid), dim3(256), 0, st, res, res_is_hprime, rows_per_b, part, sd, (const bf16*)bias,
                                                 y_out, (bf16*)yb, rows, d);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -642,6 +672,8 @@ hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const
 // finish publishes the new length / root token; all CTAs read the old length before they signal.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ int s_path[72];
   __shared__ int s_n, s_best;
   const int b = blockIdx.y;
@@ -736,7 +768,7 @@ hydra_status accept_compact(const AcceptArgs& a, cudaStream_t st) {
   int cap = (148 * 4 + a.batch - 1) / a.batch;
   if (G > cap) G = cap;
   if (G < 1) G = 1;
-  accept_compact_kernel<<<dim3(G, a.batch), 256, 0, st>>>(a);
+  launch_pdl(accept_compact_kernel, dim3(dim3(G, a.batch)), dim3(256), 0, st, a);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -745,6 +777,8 @@ hydra_status accept_compact(const AcceptArgs& a, cudaStream_t st) {
 // Small state kernels
 // ------------------------------------------------------------------------------------------------
 __global__ void set_chunk_kernel(const int* prompt_len, int chunk, int tc, int* pos0, int* n_rows, int batch) {
+  pdl_trigger();
+  pdl_wait();
   int b = threadIdx.x;
   if (b >= batch) return;
   int rem = prompt_len[b] - chunk * tc;
@@ -752,12 +786,14 @@ __global__ void set_chunk_kernel(const int* prompt_len, int chunk, int tc, int* 
   n_rows[b] = rem < 0 ? 0 : (rem > tc ? tc : rem);
 }
 hydra_status set_chunk(const int* prompt_len, int chunk, int tc, int* pos0, int* n_rows, int batch, cudaStream_t st) {
-  set_chunk_kernel<<<1, 64, 0, st>>>(prompt_len, chunk, tc, pos0, n_rows, batch);
+  launch_pdl(set_chunk_kernel, dim3(1), dim3(64), 0, st, prompt_len, chunk, tc, pos0, n_rows, batch);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 __global__ void gather_chunk_tokens_kernel(const int* tokens, const int* offsets, int chunk, int tc, int* tok_out) {
+  pdl_trigger();
+  pdl_wait();
   int b = blockIdx.x, i = threadIdx.x;
   if (i >= tc) return;
   int n = offsets[b + 1] - offsets[b];
@@ -766,13 +802,15 @@ __global__ void gather_chunk_tokens_kernel(const int* tokens, const int* offsets
 }
 hydra_status gather_chunk_tokens(const int* tokens, const int* offsets, int chunk, int tc, int* tok_out, int batch,
                                  cudaStream_t st) {
-  gather_chunk_tokens_kernel<<<batch, 64, 0, st>>>(tokens, offsets, chunk, tc, tok_out);
+  launch_pdl(gather_chunk_tokens_kernel, dim3(batch), dim3(64), 0, st, tokens, offsets, chunk, tc, tok_out);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 __global__ void capture_last_kernel(const float* h, const int* prompt_len, int chunk, int tc, float* h_new, int kp1,
                                     int* n_new, int* len, int d) {
+  pdl_trigger();
+  pdl_wait();
   int b = blockIdx.x;
   int last = prompt_len[b] - 1;
   if (last < chunk * tc || last >= (chunk + 1) * tc) return;
@@ -782,64 +820,74 @@ __global__ void capture_last_kernel(const float* h, const int* prompt_len, int c
 }
 hydra_status capture_last(const float* h, const int* prompt_len, int chunk, int tc, float* h_new, int kp1, int* n_new,
                           int* len, int batch, int d, cudaStream_t st) {
-  capture_last_kernel<<<batch, 256, 0, st>>>(h, prompt_len, chunk, tc, h_new, kp1, n_new, len, d);
+  launch_pdl(capture_last_kernel, dim3(batch), dim3(256), 0, st, h, prompt_len, chunk, tc, h_new, kp1, n_new, len, d);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 __global__ void prefix_rowset_kernel(const int* len, const int* n_new, int* pos0, int* n_rows, int batch) {
+  pdl_trigger();
+  pdl_wait();
   int b = threadIdx.x;
   if (b >= batch) return;
   pos0[b] = len[b] - n_new[b];
   n_rows[b] = n_new[b];
 }
 hydra_status prefix_rowset(const int* len, const int* n_new, int* pos0, int* n_rows, int batch, cudaStream_t st) {
-  prefix_rowset_kernel<<<1, 64, 0, st>>>(len, n_new, pos0, n_rows, batch);
+  launch_pdl(prefix_rowset_kernel, dim3(1), dim3(64), 0, st, len, n_new, pos0, n_rows, batch);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 __global__ void pick_last_row_kernel(const float* x, const int* n_rows, int tc, float* hprime, int d) {
+  pdl_trigger();
+  pdl_wait();
   int b = blockIdx.x;
   int i = n_rows[b] - 1;
   if (i < 0) i = 0;
   for (int c = threadIdx.x; c < d; c += blockDim.x) hprime[(size_t)b * d + c] = x[((size_t)b * tc + i) * d + c];
 }
 hydra_status pick_last_row(const float* x, const int* n_rows, int tc, float* hprime, int batch, int d, cudaStream_t st) {
-  pick_last_row_kernel<<<batch, 256, 0, st>>>(x, n_rows, tc, hprime, d);
+  launch_pdl(pick_last_row_kernel, dim3(batch), dim3(256), 0, st, x, n_rows, tc, hprime, d);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 __global__ void apply_plant_kernel(int* tree_tok, const int* plant, int count) {
+  pdl_trigger();
+  pdl_wait();
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < count && plant[i] >= 0) tree_tok[i] = plant[i];
 }
 hydra_status apply_plant(int* tree_tok, const int* plant, int count, cudaStream_t st) {
-  apply_plant_kernel<<<(count + 255) / 256, 256, 0, st>>>(tree_tok, plant, count);
+  launch_pdl(apply_plant_kernel, dim3((count + 255) / 256), dim3(256), 0, st, tree_tok, plant, count);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 template <typename T>
 __global__ void cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t count) {
+  pdl_trigger();
+  pdl_wait();
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < count) dst[i] = from_f<T>(src[i]);
 }
 hydra_status cast_rows(const float* src, void* dst, size_t count, int dtype, cudaStream_t st) {
   unsigned grid = (unsigned)((count + 255) / 256);
-  if (dtype == 0) cast_rows_kernel<float><<<grid, 256, 0, st>>>(src, (float*)dst, count);
-  else cast_rows_kernel<bf16><<<grid, 256, 0, st>>>(src, (bf16*)dst, count);
+  if (dtype == 0) launch_pdl(cast_rows_kernel<float>, dim3(grid), dim3(256), 0, st, src, (float*)dst, count);
+  else launch_pdl(cast_rows_kernel<bf16>, dim3(grid), dim3(256), 0, st, src, (bf16*)dst, count);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 __global__ void copy_i32_kernel(int* dst, const int* src, int count) {
+  pdl_trigger();
+  pdl_wait();
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < count) dst[i] = src[i];
 }
 hydra_status copy_i32(int* dst, const int* src, int count, cudaStream_t st) {
-  copy_i32_kernel<<<(count + 255) / 256, 256, 0, st>>>(dst, src, count);
+  launch_pdl(copy_i32_kernel, dim3((count + 255) / 256), dim3(256), 0, st, dst, src, count);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }

@@ -23,6 +23,7 @@ struct GemmEpilogue {
   float* x = nullptr; void* xg = nullptr; const void* gain = nullptr; float* ss_out = nullptr;
   void* act = nullptr; int f = 0;
   float* out = nullptr;
+  long long* trace = nullptr;                       // optional [grid][8] per-CTA phase timestamps in ns (tuning aid)
 };
 hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part, int m, int n, int k, SplitDesc* sd_out,
                      const GemmEpilogue* epi, int* status, cudaStream_t st);
