@@ -210,6 +210,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
+    torch.cuda.set_stream(torch.cuda.Stream())           # a real stream: the library captures its steps into CUDA graphs
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -253,11 +254,13 @@ def main():
     sampler = ClockSampler(local) if rank == 0 else None
     launches0 = g.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()                 # lets a profiler restrict itself to the timed region (--profile-from-start off)
     e0.record(stream)
     for s in range(args.warmup, n_total):
         one_step(s)
     e1.record(stream)
     torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()

@@ -601,7 +601,8 @@ hydra_status hydra_step(hydra_ctx* c, int32_t* n_acc, int32_t* out_tok, void* st
   if (!capacity_ok(c)) return HYDRA_ERR_CAPACITY;
   CounterScope cs(c);
   cudaStream_t st = (cudaStream_t)stream;
-  if (!c->use_graph || c->timing || c->steps_done == 0) {      // the first step runs uncaptured (one-time lazy set-up)
+  const bool capturable = st != nullptr && st != cudaStreamLegacy && st != cudaStreamPerThread;   // default streams cannot be captured
+  if (!c->use_graph || !capturable || c->timing || c->steps_done == 0) {      // the first step runs uncaptured (one-time lazy set-up)
     HYDRA_TRY(enqueue_step(c, n_acc, out_tok, st));
   } else {
     const int lu = max_len_ub(c);

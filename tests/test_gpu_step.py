@@ -94,3 +94,32 @@ def test_out_of_range_token_sets_status_word():
         g.poll_status()
     g.poll_status()                     # cleared by the poll
     g.close()
+
+
+def test_step_graph_replay_matches_kernel_by_kernel_launches():
+    """hydra_step on a non-default stream replays a captured CUDA graph from the second step on; the emitted
+    tokens must equal those of a context that launches kernel by kernel (default stream)."""
+    from paper_2402_05109_b200 import Hydra
+    m = ModelCfg(2, 256, 2, 128, 512, 1024, dtype="bf16")
+    h = HeadCfg(4, 2, True)
+    parent = load_tree("tree63_d4")
+    w = {k: v.cuda() for k, v in make_weights(m, h, 9).items()}
+    prompts = make_prompts(9, [40, 75], m.vocab)
+    outs = []
+    for use_stream in (False, True):
+        g = Hydra(m, h, parent, w, 2, 704)
+        stream = torch.cuda.Stream() if use_stream else torch.cuda.current_stream()
+        with torch.cuda.stream(stream):
+            g.prefill(prompts)
+            n_acc = torch.empty(2, dtype=torch.int32, device="cuda")
+            out = torch.empty(2, 5, dtype=torch.int32, device="cuda")
+            seq = []
+            for s in range(100):                      # long enough for the attention grid to grow (re-capture)
+                g.step(n_acc, out)
+                seq.append(out.clone())
+            g.poll_status()
+            stream.synchronize()
+        outs.append(torch.stack(seq).cpu())
+        assert g.launch_count() > 100 * 50
+        g.close()
+    assert torch.equal(outs[0], outs[1])
