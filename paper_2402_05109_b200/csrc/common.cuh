@@ -58,8 +58,8 @@ __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)
 // touched the tile, in CTA order.  A single-slot output is described by q = kb = 1.
 struct SplitDesc { int q, kb, n_tiles, mt; size_t stride; };
 __host__ __device__ __forceinline__ int split_count(const SplitDesc& sd, int m, int n) {
-  long long u0 = ((long long)(m / sd.mt) * sd.n_tiles + (n >> 7)) * sd.kb;
-  return (int)((u0 + sd.kb - 1) / sd.q - u0 / sd.q) + 1;
+  const int u0 = ((m / sd.mt) * sd.n_tiles + (n >> 7)) * sd.kb;        // tiles * kb stays far below 2^31
+  return (u0 + sd.kb - 1) / sd.q - u0 / sd.q + 1;
 }
 inline SplitDesc single_slot(size_t stride) { return SplitDesc{1, 1, 1, 1 << 30, stride}; }
 

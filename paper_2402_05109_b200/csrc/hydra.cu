@@ -67,6 +67,7 @@ struct hydra_ctx {
   char *kv_base, *kv_pfx;
   float *x, *part, *h_tree, *logits, *ss, *h_new, *hprime, *y, *head_logits;
   float2* rope;
+  void *topk_scratch; int topk_rows_cap;
   void *q, *xn, *attn_out, *act, *z, *yb, *att_scratch;
   size_t part_floats;
   // host state
@@ -201,6 +202,8 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* xn = b.take<char>((size_t)R * d * es); auto* attn_out = b.take<char>((size_t)R * d * es);
   auto* act = b.take<char>((size_t)R * f * es);
   auto* z = b.take<char>((size_t)RH * (K + 1) * d * es); auto* yb = b.take<char>((size_t)RH * d * es);
+  const int topk_cap = std::max(R, RH);
+  auto* topk_s = b.take<char>(topk_scratch_bytes(topk_cap, V));
   auto* att = b.take<char>(attention_scratch_bytes(m.max_batch, CHUNK, m.n_heads, m.head_dim, m.max_seq));
   if (c) {
     c->R = R; c->RH = RH; c->part_floats = part_floats; c->esize = es;
@@ -210,7 +213,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
     c->d_prompt_len = plen; c->d_offsets = offs; c->d_tok = tok; c->d_tree_tok = tree_tok; c->d_amax = amax; c->d_done = done;
     c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits; c->ss = ss; c->d_counters = counters;
     c->h_new = h_new; c->hprime = hprime; c->y = y; c->head_logits = head_logits; c->rope = rope; c->xn = xn;
-    c->attn_out = attn_out; c->act = act; c->z = z; c->yb = yb; c->att_scratch = att;
+    c->attn_out = attn_out; c->act = act; c->z = z; c->yb = yb; c->att_scratch = att; c->topk_scratch = topk_s; c->topk_rows_cap = topk_cap;
   }
   return (b.off + 255) & ~(size_t)255;
 }
@@ -383,7 +386,10 @@ hydra_status do_draft(hydra_ctx* c, int* tree_tok, cudaStream_t st) {
       HYDRA_TRY(head_act(c->y, 0, P, c->part, sd, br, c->y, c->yb, rows, d, dt, st));
     }
     HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, rows, m.vocab, d, &sd, st));
-    HYDRA_TRY(topk_children(c->part, sd, c->head_logits, lv, c->d_first_child, c->d_n_child, tree_tok, B, c->T, m.vocab, st));
+    int max_children = 1;
+    for (int p : c->level_parents[lvl - 1]) max_children = std::max(max_children, c->n_child[p]);
+    HYDRA_TRY(topk_children(c->part, sd, c->head_logits, lv, max_children, c->d_first_child, c->d_n_child, tree_tok, c->topk_scratch,
+                            c->topk_rows_cap, B, c->T, m.vocab, st));
   }
   return HYDRA_OK;
 }
@@ -397,11 +403,11 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
     float* lg = logits ? logits : c->logits;
     GemmEpilogue e; e.kind = EPI_OUT; norm_in(c, e); e.out = lg;
     HYDRA_TRY(run_gemm_fused(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, e, st));
-    return argmax_rows(lg, single_slot(0), nullptr, amax, rows, m.vocab, st);
+    return argmax_rows(lg, single_slot(0), nullptr, amax, c->topk_scratch, c->topk_rows_cap, rows, m.vocab, st);
   }
   SplitDesc sd;
   HYDRA_TRY(run_gemm(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, &sd, st));
-  return argmax_rows(c->part, sd, logits, amax, rows, m.vocab, st);
+  return argmax_rows(c->part, sd, logits, amax, c->topk_scratch, c->topk_rows_cap, rows, m.vocab, st);
 }
 
 hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* n_acc, int* path, int* out_tok, cudaStream_t st) {
@@ -557,7 +563,7 @@ hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const
   HYDRA_TRY(cast_rows(c->hprime, c->yb, (size_t)batch * m.d_model, m.dtype, st));
   SplitDesc sd;
   HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, batch, m.vocab, m.d_model, &sd, st));
-  HYDRA_TRY(argmax_rows(c->part, sd, nullptr, c->d_root_tok, batch, m.vocab, st));
+  HYDRA_TRY(argmax_rows(c->part, sd, nullptr, c->d_root_tok, c->topk_scratch, c->topk_rows_cap, batch, m.vocab, st));
   for (int b = 0; b < batch; ++b) c->len_ub[b] = plen[b];
   drop_graphs(c);
   c->state = ST_READY;

@@ -537,60 +537,106 @@ __device__ __forceinline__ float summed(const float* part, const SplitDesc& sd, 
   return v;
 }
 
-__global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restrict__ part, SplitDesc sd,
-                                                          float* __restrict__ logits_out, int* __restrict__ amax, int vocab) {
+// Top-c of every logits row in two stages.  Stage 1: grid (rows, blocks of TOPK_SPAN columns); each block sums the
+// partial slots of its columns (optionally storing the sums as the row's logits), then picks its c best in c
+// rounds of a block-wide reduction over register-resident values.  Stage 2: one block per row merges the
+// candidates of all column blocks the same way and writes the winners (children of a tree node, or the argmax).
+constexpr int TOPK_SPAN = 2048;           // columns per stage-1 block (8 per thread)
+constexpr int TOPK_MAX = 64;              // a tree node has at most 63 children
+
+__global__ void __launch_bounds__(256) topk_stage1_kernel(const float* __restrict__ part, SplitDesc sd,
+                                                          float* __restrict__ logits_out, float* __restrict__ cand_v,
+                                                          int* __restrict__ cand_i, int vocab, int c) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ float shv[32];
+  __shared__ int shi[32];
+  const int row = blockIdx.x, blk = blockIdx.y, nblk = gridDim.y;
+  float v[8]; int idx[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int col = blk * TOPK_SPAN + j * 256 + threadIdx.x;
+    idx[j] = col;
+    v[j] = -INFINITY;
+    if (col < vocab) {
+      v[j] = summed(part, sd, row, col, vocab);
+      if (logits_out) logits_out[(size_t)row * vocab + col] = v[j];
+    } else {
+      idx[j] = 0x7fffffff;
+    }
+  }
+  for (int t = 0; t < c; ++t) {
+    float bv = -INFINITY; int bi = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) if (better(v[j], idx[j], bv, bi)) { bv = v[j]; bi = idx[j]; }
+    block_best(bv, bi, shv, shi);
+    if (threadIdx.x == 0) {
+      cand_v[((size_t)row * nblk + blk) * TOPK_MAX + t] = bv;
+      cand_i[((size_t)row * nblk + blk) * TOPK_MAX + t] = bi;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) if (idx[j] == bi) { v[j] = -INFINITY; idx[j] = 0x7fffffff; }    // taken
+  }
+}
+
+// out_of(row) and count_of(row): where the winners go.  lv.parents == null: argmax (one winner per row to amax[row]).
+__global__ void __launch_bounds__(256) topk_stage2_kernel(const float* __restrict__ cand_v, const int* __restrict__ cand_i,
+                                                          int nblk, int c, LevelDesc lv, const int* __restrict__ first_child,
+                                                          const int* __restrict__ n_child, int* __restrict__ out, int T) {
   pdl_trigger();
   pdl_wait();
   __shared__ float shv[32];
   __shared__ int shi[32];
   const int row = blockIdx.x;
-  float bv = -INFINITY; int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
-    float v = summed(part, sd, row, i, vocab);
-    if (logits_out) logits_out[(size_t)row * vocab + i] = v;
-    if (better(v, i, bv, bi)) { bv = v; bi = i; }
+  int* dst = out + row;
+  int count = 1;
+  if (lv.parents) {
+    const int b = row / lv.n_parents, p = lv.parents[row % lv.n_parents];
+    dst = out + b * T + first_child[p];
+    count = n_child[p];
   }
-  block_best(bv, bi, shv, shi);
-  if (threadIdx.x == 0) amax[row] = bi;
+  float pv = INFINITY; int pi = -1;
+  for (int t = 0; t < count; ++t) {
+    float bv = -INFINITY; int bi = 0x7fffffff;
+    for (int e = threadIdx.x; e < nblk * c; e += blockDim.x) {
+      const size_t at = ((size_t)row * nblk + e / c) * TOPK_MAX + e % c;
+      const float v = cand_v[at]; const int i = cand_i[at];
+      const bool after = v < pv || (v == pv && i > pi);          // strictly after the previous pick in the order
+      if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
+    }
+    block_best(bv, bi, shv, shi);
+    if (threadIdx.x == 0) dst[t] = bi;
+    pv = bv; pi = bi;
+  }
 }
-hydra_status argmax_rows(const float* part, SplitDesc sd, float* logits_out, int* amax, int rows, int vocab, cudaStream_t st) {
-  launch_pdl(argmax_rows_kernel, dim3(rows), dim3(256), 0, st, part, sd, logits_out, amax, vocab);
+
+size_t topk_scratch_bytes(int rows, int vocab) {
+  const size_t nblk = (size_t)(vocab + TOPK_SPAN - 1) / TOPK_SPAN;
+  return (size_t)rows * nblk * TOPK_MAX * (sizeof(float) + sizeof(int));
+}
+
+static hydra_status topk_rows(const float* part, SplitDesc sd, float* logits_out, void* scratch, int rows_cap, int rows, int vocab,
+                              int c, LevelDesc lv, const int* first_child, const int* n_child, int* out, int T, cudaStream_t st) {
+  if (c < 1 || c > TOPK_MAX || rows > rows_cap) return HYDRA_ERR_UNSUPPORTED;
+  const int nblk = (vocab + TOPK_SPAN - 1) / TOPK_SPAN;
+  float* cand_v = (float*)scratch;
+  int* cand_i = (int*)(cand_v + (size_t)rows_cap * nblk * TOPK_MAX);
+  launch_pdl(topk_stage1_kernel, dim3(rows, nblk), dim3(256), 0, st, part, sd, logits_out, cand_v, cand_i, vocab, c);
+  HYDRA_LAUNCH_CHECK();
+  launch_pdl(topk_stage2_kernel, dim3(rows), dim3(256), 0, st, (const float*)cand_v, (const int*)cand_i, nblk, c, lv, first_child, n_child, out, T);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
-__global__ void __launch_bounds__(256) topk_children_kernel(const float* __restrict__ part, SplitDesc sd, float* __restrict__ logits,
-                                                            LevelDesc lv,
-                                                            const int* __restrict__ first_child,
-                                                            const int* __restrict__ n_child, int* __restrict__ tree_tok,
-                                                            int T, int vocab) {
-  pdl_trigger();
-  pdl_wait();
-  __shared__ float shv[32];
-  __shared__ int shi[32];
-  const int row = blockIdx.x, b = row / lv.n_parents, j = row % lv.n_parents;
-  const int p = lv.parents[j];
-  const int nc = n_child[p], fc = first_child[p];
-  float* lg = logits + (size_t)row * vocab;
-  for (int i = threadIdx.x; i < vocab; i += blockDim.x) lg[i] = summed(part, sd, row, i, vocab);   // each thread re-reads its own
-  float pv = INFINITY; int pi = -1;
-  for (int t = 0; t < nc; ++t) {
-    float bv = -INFINITY; int bi = 0x7fffffff;
-    for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
-      float v = lg[i];
-      bool after = v < pv || (v == pv && i > pi);          // strictly after the previous pick in the order
-      if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
-    }
-    block_best(bv, bi, shv, shi);
-    if (threadIdx.x == 0) tree_tok[b * T + fc + t] = bi;
-    pv = bv; pi = bi;
-  }
+hydra_status argmax_rows(const float* part, SplitDesc sd, float* logits_out, int* amax, void* scratch, int rows_cap, int rows,
+                         int vocab, cudaStream_t st) {
+  return topk_rows(part, sd, logits_out, scratch, rows_cap, rows, vocab, 1, LevelDesc{0, 0, nullptr}, nullptr, nullptr, amax, 0, st);
 }
-hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, const int* first_child,
-                           const int* n_child, int* tree_tok, int batch, int T, int vocab, cudaStream_t st) {
-  launch_pdl(topk_children_kernel, dim3(batch * lv.n_parents), dim3(256), 0, st, part, sd, logits, lv, first_child, n_child, tree_tok, T, vocab);
-  HYDRA_LAUNCH_CHECK();
-  return HYDRA_OK;
+
+hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, int max_children, const int* first_child,
+                           const int* n_child, int* tree_tok, void* scratch, int rows_cap, int batch, int T, int vocab,
+                           cudaStream_t st) {
+  return topk_rows(part, sd, logits, scratch, rows_cap, batch * lv.n_parents, vocab, max_children, lv, first_child, n_child, tree_tok, T, st);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -64,7 +64,10 @@ hydra_status tree_attention(const void* q, const void* kcache, const void* vcach
 hydra_status silu_mul(const float* part, SplitDesc sd, void* act, int rows, int f, int dtype,
                       cudaStream_t st);
 // amax[r] = argmax_v of the summed partial logits (lowest id among equal maxima); the sums go to logits_out if given
-hydra_status argmax_rows(const float* part, SplitDesc sd, float* logits_out, int* amax, int rows, int vocab, cudaStream_t st);
+// scratch: topk_scratch_bytes(rows_cap, vocab) bytes of candidate storage
+size_t topk_scratch_bytes(int rows, int vocab);
+hydra_status argmax_rows(const float* part, SplitDesc sd, float* logits_out, int* amax, void* scratch, int rows_cap, int rows,
+                         int vocab, cudaStream_t st);
 
 // ---- Hydra heads
 struct LevelDesc {           // one tree level d (1-based): the parents that have children
@@ -80,8 +83,9 @@ hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const
                       const void* bias, float* y_out, void* yb, int rows, int d, int dtype, cudaStream_t st);
 // children of parent j of sequence b = top n_child tokens of logits row b*P+j, descending (ties: lower id first);
 // the logits are the summed partials, also written to `logits` [rows][vocab]
-hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, const int* first_child, const int* n_child, int* tree_tok,
-                           int batch, int T, int vocab, cudaStream_t st);
+hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, int max_children, const int* first_child,
+                           const int* n_child, int* tree_tok, void* scratch, int rows_cap, int batch, int T, int vocab,
+                           cudaStream_t st);
 
 // ---- acceptance + compaction (one kernel)
 struct AcceptArgs {
