@@ -10,8 +10,10 @@
  * Conventions
  *  - Every call returns a hydra_status; nothing throws, aborts or exits.
  *  - "dev" pointers are device pointers, "host" pointers are host pointers.  All matrices are
- *    row-major [out][in].  dtype 0: weights, KV cache and GEMM operands are float; dtype 1: they
- *    are bfloat16, while accumulation, residual stream, norms and softmax stay float.
+ *    row-major [out][in].  dtype 0: weights, KV cache and GEMM operands are float; dtype 1: weights are
+ *    bfloat16; activations that feed a GEMM or the attention, and the KV cache, are stored as TWO bfloat16
+ *    planes (hi = bf16(v), lo = bf16(v - hi), about 16 mantissa bits together), while accumulation, residual
+ *    stream, norms and softmax stay float.
  *  - The caller owns the weights, the workspace and every in/out buffer and keeps them alive until
  *    hydra_destroy.  The library owns only the opaque context; KV caches, tables and scratch are
  *    carved out of the caller's workspace (hydra_workspace_bytes, 256-byte aligned base).
@@ -130,8 +132,8 @@ enum {
   HYDRA_BUF_ROOT_TOK = 1,   /* int32 [max_batch] */
   HYDRA_BUF_H_TREE = 2,     /* float [batch*n_rows][d] post-final-norm hidden of the last verify */
   HYDRA_BUF_H_NEW = 3,      /* float [max_batch][K+1][d] hidden rows committed by the last step */
-  HYDRA_BUF_KV_BASE = 4,    /* [n_layers][2][max_batch][n_heads][max_seq][head_dim] */
-  HYDRA_BUF_KV_PREFIX = 5,  /* [2][max_batch][n_heads][max_seq][head_dim] */
+  HYDRA_BUF_KV_BASE = 4,    /* [n_layers][k,v][planes][max_batch][n_heads][max_seq][head_dim]; planes = 2 (hi, lo) for dtype 1, else 1 */
+  HYDRA_BUF_KV_PREFIX = 5,  /* [k,v][planes][max_batch][n_heads][max_seq][head_dim] */
   HYDRA_BUF_TREE_MASK = 6,  /* uint64 [n_rows] ancestor-or-self bitmask */
   HYDRA_BUF_TREE_TOK = 7,   /* int32 [batch][n_rows] tokens of the last hydra_step */
   HYDRA_BUF_AMAX = 8,       /* int32 [batch][n_rows] */
@@ -156,9 +158,8 @@ enum { HYDRA_TIME_GEMM = 0, HYDRA_TIME_ATTENTION = 1, HYDRA_TIME_ACCEPT = 2 };
 hydra_status hydra_set_timing(hydra_ctx*, int on);
 hydra_status hydra_get_timing(hydra_ctx*, int kclass, double* ms_total, long long* launches, double* bytes_total);
 
-/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA, consumer operations in their own kernels (default);
- * 1 = the plain SIMT kernel; 2 = tcgen05/TMA with the consumer operations fused into the GEMM epilogues
- * (applied by the CTA that completes a tile). */
+/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA (default); 1 = the plain SIMT kernel (debugging; it
+ * reads only the hi plane of the activations). */
 hydra_status hydra_set_gemm_mode(hydra_ctx*, int mode);
 
 const char* hydra_status_str(hydra_status);
@@ -167,18 +168,20 @@ const char* hydra_last_error(void); /* text of the last CUDA error seen by this 
 /* Single-kernel entry points for kernel-level parity tests.  No context; the library makes its own
  * tensor maps.  All pointers are device pointers.
  * hydra_gemm: out[m][n] = sum_k x[m][k] * w[n][k] (float accumulate, float out), dtype as above;
- *   n % 128 == 0 and k % 64 == 0 for mode 0.  partial_dev needs hydra_gemm_partial_floats(m, n, k, dtype, mode)
- *   floats: the tensor-core GEMM leaves per-CTA partial sums there, which a second kernel adds in fixed order.
- *   mode as in hydra_set_gemm_mode; status_dev is an int32 status word (bit 1 bounds, bit 2 timeout).
- * hydra_tree_attention: q [rows][n_heads][head_dim] (dtype; rows = batch*tc), caches
- *   [batch][n_heads][max_seq][head_dim] (dtype), pos0 [batch] committed lengths, n_rows [batch] or
- *   NULL (= tc), mask [tc] ancestor bitmasks; out [rows][n_heads*head_dim] (dtype).  Row i of
- *   sequence b sees slots < pos0[b] and slot pos0[b]+j when bit j of mask[i] is set.  scratch_dev
- *   needs hydra_attention_scratch_bytes(...) bytes. */
+ *   n % 128 == 0 and k % 64 == 0 for mode 0.  x_planes = 1: x is [m][k]; x_planes = 2 (dtype 1, mode 0 only): x is
+ *   [2][m][k], the hi and lo bfloat16 planes of the activations, and the product uses both.  partial_dev needs
+ *   hydra_gemm_partial_floats(m, n, k, dtype, mode) floats: the tensor-core GEMM leaves per-CTA partial sums
+ *   there, which a second kernel adds in fixed order.  mode as in hydra_set_gemm_mode; status_dev is an int32
+ *   status word (bit 1 bounds, bit 2 timeout).
+ * hydra_tree_attention: q [planes][rows][n_heads][head_dim] (dtype; rows = batch*tc), caches
+ *   [planes][batch][n_heads][max_seq][head_dim] (dtype), pos0 [batch] committed lengths, n_rows [batch] or
+ *   NULL (= tc), mask [tc] ancestor bitmasks; out [planes][rows][n_heads*head_dim] (dtype).  planes = 2 (dtype 1
+ *   only) means hi/lo bfloat16 planes.  Row i of sequence b sees slots < pos0[b] and slot pos0[b]+j when bit j of
+ *   mask[i] is set.  scratch_dev needs hydra_attention_scratch_bytes(...) bytes. */
 size_t hydra_gemm_partial_floats(int m, int n, int k, int dtype, int mode);
 hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, float* partial_dev, int m, int n, int k,
-                        int dtype, int mode, int32_t* status_dev, void* stream);
-/* hydra_gemm_noalloc: the bfloat16 tensor-core GEMM of hydra_gemm (dtype 1, mode 0) for callers that
+                        int dtype, int mode, int x_planes, int32_t* status_dev, void* stream);
+/* hydra_gemm_noalloc: the bfloat16 tensor-core GEMM of hydra_gemm (dtype 1, mode 0, x_planes 1) for callers that
  * may not allocate device memory.  (The paper has no counterpart; this is a convenience of the library.)
  * Serving loops that must stay clear of the allocator's locks and implicit synchronisation, plugins living
  * inside a host's fixed memory budget, and processes whose free memory already belongs to a pool cannot
@@ -200,7 +203,7 @@ size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_di
 hydra_status hydra_tree_attention(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev,
                                   const int32_t* pos0_dev, const int32_t* n_rows_dev, const uint64_t* mask_dev,
                                   void* out_dev, void* scratch_dev, int batch, int tc, int n_heads, int head_dim,
-                                  int max_seq, int dtype, void* stream);
+                                  int max_seq, int dtype, int planes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -64,11 +64,11 @@ lib.hydra_status_str.argtypes = [_i]
 lib.hydra_last_error.restype = C.c_char_p
 lib.hydra_gemm_partial_floats.restype = _sz
 lib.hydra_gemm_partial_floats.argtypes = [_i] * 5
-lib.hydra_gemm.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
+lib.hydra_gemm.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]
 lib.hydra_gemm_noalloc.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]
 lib.hydra_attention_scratch_bytes.restype = _sz
 lib.hydra_attention_scratch_bytes.argtypes = [_i] * 5
-lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 6 + [_vp]
+lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 7 + [_vp]
 
 BUF = dict(LEN=0, ROOT_TOK=1, H_TREE=2, H_NEW=3, KV_BASE=4, KV_PREFIX=5, TREE_MASK=6, TREE_TOK=7, AMAX=8,
            HEAD_LOGITS=9, N_NEW=10, H_PRIME=11)
@@ -217,23 +217,36 @@ class Hydra:
 
     def kv_base(self) -> torch.Tensor:
         m = self.model
-        return self.get_buffer("KV_BASE").view(m.n_layers, 2, self.max_batch, m.n_heads, self.max_seq, m.head_dim)
+        planes = 1 if self.dtype == torch.float32 else 2
+        kv = self.get_buffer("KV_BASE").view(m.n_layers, 2, planes, self.max_batch, m.n_heads, self.max_seq, m.head_dim)
+        return kv.float().sum(dim=2) if planes == 2 else kv[:, :, 0]          # hi + lo
 
     def kv_prefix(self) -> torch.Tensor:
         m = self.model
-        return self.get_buffer("KV_PREFIX").view(2, self.max_batch, m.n_heads, self.max_seq, m.head_dim)
+        planes = 1 if self.dtype == torch.float32 else 2
+        kv = self.get_buffer("KV_PREFIX").view(2, planes, self.max_batch, m.n_heads, self.max_seq, m.head_dim)
+        return kv.float().sum(dim=1) if planes == 2 else kv[:, 0]
 
 
 # ---- single-kernel entry points (kernel-level parity tests)
+def split_hi_lo(x: torch.Tensor) -> torch.Tensor:
+    """[2, ...] bfloat16: hi = bf16(x), lo = bf16(x - hi) of a float tensor (the library's operand format)."""
+    hi = x.to(torch.bfloat16)
+    lo = (x.float() - hi.float()).to(torch.bfloat16)
+    return torch.stack([hi, lo]).contiguous()
+
+
 def gemm(x: torch.Tensor, w: torch.Tensor, mode: int = 0) -> torch.Tensor:
-    """out[m][n] = sum_k x[m][k] w[n][k] in float; x, w both float32 or both bfloat16 CUDA tensors."""
-    m, k = x.shape
+    """out[m][n] = sum_k x[m][k] w[n][k] in float; x, w both float32 or both bfloat16 CUDA tensors.
+    x may be [2][m][k] bfloat16 (hi/lo planes, see split_hi_lo)."""
+    planes = 2 if x.dim() == 3 else 1
+    m, k = x.shape[-2:]
     n = w.shape[0]
     dtype = 0 if x.dtype == torch.float32 else 1
     out = torch.empty(m, n, dtype=torch.float32, device="cuda")
     part = torch.empty(lib.hydra_gemm_partial_floats(m, n, k, dtype, mode), dtype=torch.float32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    _check(lib.hydra_gemm(x.data_ptr(), w.data_ptr(), out.data_ptr(), part.data_ptr(), m, n, k, dtype, mode,
+    _check(lib.hydra_gemm(x.data_ptr(), w.data_ptr(), out.data_ptr(), part.data_ptr(), m, n, k, dtype, mode, planes,
                           status.data_ptr(), _stream()), "hydra_gemm")
     word = int(status.item())
     if word:
@@ -252,12 +265,15 @@ def gemm_noalloc(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor, status: to
 
 
 def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int) -> torch.Tensor:
-    batch, n_heads, max_seq, head_dim = k_cache.shape
+    """Caches [batch][H][S][hd] (one plane) or [2][batch][H][S][hd] (hi/lo planes, bfloat16); q and the result likewise."""
+    planes = 2 if k_cache.dim() == 5 else 1
+    batch, n_heads, max_seq, head_dim = k_cache.shape[-4:]
     dtype = 0 if k_cache.dtype == torch.float32 else 1
-    out = torch.empty(batch * tc, n_heads * head_dim, dtype=k_cache.dtype, device="cuda")
+    shape = (batch * tc, n_heads * head_dim)
+    out = torch.empty((planes,) + shape if planes == 2 else shape, dtype=k_cache.dtype, device="cuda")
     scratch = torch.empty(lib.hydra_attention_scratch_bytes(batch, tc, n_heads, head_dim, max_seq), dtype=torch.uint8,
                           device="cuda")
     _check(lib.hydra_tree_attention(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), pos0.data_ptr(), _ptr(n_rows),
                                     mask.data_ptr(), out.data_ptr(), scratch.data_ptr(), batch, tc, n_heads, head_dim,
-                                    max_seq, dtype, _stream()), "hydra_tree_attention")
+                                    max_seq, dtype, planes, _stream()), "hydra_tree_attention")
     return out

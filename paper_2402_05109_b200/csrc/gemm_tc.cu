@@ -20,12 +20,12 @@
 // TMEM let the epilogue of one segment overlap the main loop of the next.  The kernel is launched with
 // programmatic stream serialisation: weight tiles (which never depend on the preceding kernel) are requested
 // before griddepcontrol.wait, activations and all global writes after it.
-// Fused epilogues: after writing its slot a CTA bumps the tile's arrival counter; the CTA that completes the
-// tile ("last arriver") adds the slots in slot order and applies the consumer operation right there -- rotary
-// embedding + KV-cache append (QKV), residual add + next-norm operand + row sums of squares (O and down
-// projections), SiLU(gate)*up (gate/up pairs), or a plain scaled store (LM head).  RMSNorm is factored as
-// (x*gain) W^T * inv_rms[row]: the producer stores x*gain in bfloat16 and per-tile sums of squares, the
-// consuming GEMM scales its reduced output rows by inv_rms.
+// Precision: weights are bfloat16 (exact: the reference model's weights are the same bfloat16 values).  The
+// activation operand comes as TWO bfloat16 planes, hi = bf16(v) and lo = bf16(v - hi), i.e. about 16 mantissa
+// bits; each weight tile is multiplied with both planes into the same accumulator.  This doubles the MMA work
+// (irrelevant while the kernel is HBM-bound) and the L2-resident activation traffic, not the HBM traffic, and
+// keeps the hidden states within 1e-2 of a float reference over 32+ layers (plain bfloat16 operands drift to
+// 4e-2).  x_lo_rows = 0 selects a single plane.
 // Every mbarrier wait is bounded: when one runs out the CTA raises ST_TIMEOUT in the status word, stops
 // storing, lets its copies settle, frees its tensor memory and returns.
 #include "launch.h"
@@ -136,9 +136,10 @@ __host__ __device__ constexpr uint32_t instr_desc(int mt) {
 
 template <int MT, int BUDGET_KB> struct TileCfg {
   static constexpr int SMEM_BUDGET = BUDGET_KB * 1024;
-  static constexpr int B_BYTES = MT * BLOCK_K * 2;
+  static constexpr int B_PLANE = MT * BLOCK_K * 2;               // one activation plane of a stage
+  static constexpr int B_BYTES = 2 * B_PLANE;                    // hi + lo
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 10 ? 10 : ((SMEM_BUDGET / STAGE_BYTES) < 3 ? 3 : (SMEM_BUDGET / STAGE_BYTES));
+  static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 10 ? 10 : ((SMEM_BUDGET / STAGE_BYTES) < 2 ? 2 : (SMEM_BUDGET / STAGE_BYTES));
   static constexpr int ACC_COLS = MT < 32 ? 32 : MT;             // columns of one accumulator buffer
   static constexpr int TMEM_COLS = 2 * ACC_COLS;                  // two buffers (power of two, <= 512)
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/;
@@ -147,132 +148,13 @@ template <int MT, int BUDGET_KB> struct TileCfg {
 struct GemmArgs {
   float* part; size_t slot_stride;
   int m, n, kb, n_tiles, total_units, q;
+  int x_lo_rows;                 // row offset of the lo plane inside the activation tensor map (0: single plane)
   int* status;
-  int epi;                       // GemmEpilogue::kind
-  unsigned int* counters;        // [tiles], zero at rest
-  const float* ss_in; int ss_in_tiles; int ss_ld; float inv_d, eps;     // RMSNorm factor of the operand rows (null: none)
-  RowSet rs; const float2* rope; void* q_out; void* kc; void* vc; int H, hd, max_seq;   // EPI_QKV
-  float* x; void* xg; const void* gain; float* ss_out;                                   // EPI_RESID
-  void* act; int f;                                                                      // EPI_GATEUP
-  float* out;                                                                            // EPI_OUT
   long long* trace;              // optional [grid][8] nanosecond timestamps of each CTA's phases (tuning aid), or null
 };
 
 __device__ __forceinline__ long long global_ns() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define TRACE(slot) do { if (a.trace) a.trace[blockIdx.x * 8 + (slot)] = global_ns(); } while (0)
-
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the 4 epilogue warps
-
-__device__ __forceinline__ int tile_slots(const GemmArgs& a, int tile) {
-  const long long u0 = (long long)tile * a.kb;
-  return (int)((u0 + a.kb - 1) / a.q - u0 / a.q) + 1;
-}
-// Sums of a tile's partial slots for RB consecutive rows of one column, in slot order.  Loads of the RB rows are
-// independent so they overlap (the slots were written by other SMs: read past L1).  Rows >= m1 give 0.
-constexpr int RB = 32;
-__device__ __forceinline__ void slot_sums(const GemmArgs& a, int ns, int mb, int m1, int n, float (&v)[RB]) {
-  const float* p = a.part + (size_t)mb * a.n + n;
-#pragma unroll
-  for (int r = 0; r < RB; ++r) v[r] = 0.f;
-  for (int s = 0; s < ns; ++s) {
-    const float* ps = p + (size_t)s * a.slot_stride;
-#pragma unroll
-    for (int r = 0; r < RB; ++r)
-      if (mb + r < m1) v[r] += __ldcg(ps + (size_t)r * a.n);
-  }
-}
-
-// Consumer operation applied by the last arriver of a tile (or of a gate/up tile pair).  tid = column within
-// the tile (0..127); all 128 epilogue threads call it.  Rows are processed RB at a time.
-template <int MT>
-__device__ void apply_epilogue(const GemmArgs& a, int tile, int tid, const float* s_inv, float (*s_ss)[MT]) {
-  const int tn = tile % a.n_tiles, tm = tile / a.n_tiles;
-  const int m0 = tm * MT, m1 = min(m0 + MT, a.m);
-  const int warp4 = tid >> 5, lane = tid & 31;
-  if (a.epi == EPI_OUT) {
-    const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
-    for (int mb = m0; mb < m1; mb += RB) {
-      float v[RB];
-      slot_sums(a, ns, mb, m1, n, v);
-#pragma unroll
-      for (int r = 0; r < RB; ++r)
-        if (mb + r < m1) a.out[(size_t)(mb + r) * a.n + n] = v[r] * s_inv[mb + r];
-    }
-  } else if (a.epi == EPI_RESID) {
-    const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
-    const float gn = a.gain ? __bfloat162float(reinterpret_cast<const bf16*>(a.gain)[n]) : 0.f;
-    for (int mb = m0; mb < m1; mb += RB) {
-      float v[RB], xv[RB];
-#pragma unroll
-      for (int r = 0; r < RB; ++r) xv[r] = mb + r < m1 ? a.x[(size_t)(mb + r) * a.n + n] : 0.f;
-      slot_sums(a, ns, mb, m1, n, v);
-#pragma unroll
-      for (int r = 0; r < RB; ++r) {
-        xv[r] += v[r];
-        if (mb + r < m1) {
-          const size_t idx = (size_t)(mb + r) * a.n + n;
-          a.x[idx] = xv[r];
-          if (a.gain) reinterpret_cast<bf16*>(a.xg)[idx] = __float2bfloat16_rn(xv[r] * gn);
-        }
-        const float ss = warp_sum(xv[r] * xv[r]);
-        if (lane == 0 && mb + r < m1) s_ss[warp4][mb + r - m0] = ss;
-      }
-    }
-    epi_bar();
-    for (int r = tid; r < m1 - m0; r += 128)
-      a.ss_out[(size_t)tn * a.ss_ld + m0 + r] = s_ss[0][r] + s_ss[1][r] + s_ss[2][r] + s_ss[3][r];
-  } else if (a.epi == EPI_GATEUP) {
-    const int half_tiles = a.n_tiles >> 1;
-    const int p = tn % half_tiles;
-    const int tg = tm * a.n_tiles + p, tu = tg + half_tiles;
-    const int nsg = tile_slots(a, tg), nsu = tile_slots(a, tu);
-    const int c = p * BLOCK_N + tid;
-    for (int mb = m0; mb < m1; mb += RB) {
-      float g[RB], u[RB];
-      slot_sums(a, nsg, mb, m1, c, g);
-      slot_sums(a, nsu, mb, m1, a.f + c, u);
-#pragma unroll
-      for (int r = 0; r < RB; ++r)
-        if (mb + r < m1) {
-          const float sc = s_inv[mb + r];
-          reinterpret_cast<bf16*>(a.act)[(size_t)(mb + r) * a.f + c] = __float2bfloat16_rn(silu_f(g[r] * sc) * (u[r] * sc));
-        }
-    }
-  } else if (a.epi == EPI_QKV) {
-    const int ns = tile_slots(a, tile), n = tn * BLOCK_N + tid;
-    const int d = a.H * a.hd, half = a.hd >> 1;
-    const int which = n / d, within = n % d, head = within / a.hd, jl = within % a.hd;
-    bf16* kv = reinterpret_cast<bf16*>(which == 1 ? a.kc : a.vc);
-    const int n_partner = n + (jl < half ? half : -half);
-    for (int mb = m0; mb < m1; mb += RB) {
-      float v[RB], pv[RB];
-      slot_sums(a, ns, mb, m1, n, v);
-      if (which < 2) slot_sums(a, ns, mb, m1, n_partner, pv);            // the other element of the rotation pair
-      bool row_ok[RB]; int bq[RB], slot[RB];
-#pragma unroll
-      for (int r = 0; r < RB; ++r) {
-        const int m = mb + r < m1 ? mb + r : m1 - 1;
-        const int b = m / a.rs.tc, i = m % a.rs.tc;
-        const int nr = a.rs.n_rows ? a.rs.n_rows[b] : a.rs.tc;
-        bq[r] = b; slot[r] = a.rs.pos0[b] + i;
-        const bool in_rows = mb + r < m1 && i < nr;
-        row_ok[r] = in_rows && slot[r] >= 0 && slot[r] < a.max_seq;
-        if (in_rows && !row_ok[r] && tid == 0) atomicOr(a.status, ST_BOUNDS);
-        if (which < 2 && row_ok[r]) {                                    // rotate q and k (half-split pairing)
-          const float2 cs = a.rope[(size_t)m * half + (jl % half)];
-          v[r] = jl < half ? v[r] * cs.x - pv[r] * cs.y : v[r] * cs.x + pv[r] * cs.y;
-        }
-        v[r] *= s_inv[m];
-      }
-#pragma unroll
-      for (int r = 0; r < RB; ++r)
-        if (row_ok[r]) {
-          if (which == 0) reinterpret_cast<bf16*>(a.q_out)[(size_t)(mb + r) * d + within] = __float2bfloat16_rn(v[r]);
-          else kv[(((size_t)bq[r] * a.H + head) * a.max_seq + slot[r]) * a.hd + jl] = __float2bfloat16_rn(v[r]);
-        }
-    }
-  }
-}
 
 template <int MT, int BUDGET_KB>
 __global__ void __launch_bounds__(192, 1)
@@ -287,9 +169,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   auto accfull_bar = [&](int i) { return bars + 8u * (3 * C::STAGES + i); };
   auto accempty_bar = [&](int i) { return bars + 8u * (3 * C::STAGES + 2 + i); };
   const uint32_t tmem_slot = bars + 8u * (3 * C::STAGES + 4);
-  __shared__ int s_abort, s_last;
-  __shared__ float s_inv[512];               // inv_rms of the operand rows (fused epilogues need m <= 512)
-  __shared__ float s_ss[4][MT];
+  __shared__ int s_abort;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_begin = blockIdx.x * a.q;
@@ -344,8 +224,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           mbar_arrive_expect_tx(fullw_bar(s), A_BYTES);
           tma_load_2d(a_dst, &tmW, kcol, nrow, fullw_bar(s), pol_w);
         }
-        mbar_arrive_expect_tx(fullx_bar(s), C::B_BYTES);
+        mbar_arrive_expect_tx(fullx_bar(s), a.x_lo_rows ? C::B_BYTES : C::B_PLANE);
         tma_load_2d(a_dst + A_BYTES, &tmX, kcol, mrow, fullx_bar(s), pol_x);
+        if (a.x_lo_rows) tma_load_2d(a_dst + A_BYTES + C::B_PLANE, &tmX, kcol, a.x_lo_rows + mrow, fullx_bar(s), pol_x);
       }
     }
   } else if (warp == 1) {
@@ -374,6 +255,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
           for (int k = 0; k < BLOCK_K / 16; ++k)         // 16 bf16 = 32 bytes per MMA: +2 in 16-byte units
             umma_bf16(tmem_d, adesc + 2u * k, bdesc + 2u * k, idesc, (uint32_t)((j | k) != 0));
+          if (a.x_lo_rows) {                             // the low-order plane of the activations, same weights
+            const uint64_t ldesc = smem_desc_sw128(a_addr + A_BYTES + C::B_PLANE);
+#pragma unroll
+            for (int k = 0; k < BLOCK_K / 16; ++k) umma_bf16(tmem_d, adesc + 2u * k, ldesc + 2u * k, idesc, 1u);
+          }
           umma_commit(empty_bar(s));                     // frees the stage once these MMAs have read it
         }
         if (!ok) break;
@@ -386,15 +272,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   } else {
     const int quarter = warp & 3;                        // TMEM lanes this warp may read
     const int epi_tid = quarter * 32 + lane;             // column of the tile this thread owns
-    grid_dep_wait();                                     // partial buffer / operand statistics belong to the preceding kernel
-    if (a.epi != EPI_PARTIAL) {
-      for (int m = epi_tid; m < a.m && m < 512; m += 128) {
-        float ss = 0.f;
-        for (int t = 0; t < a.ss_in_tiles; ++t) ss += a.ss_in[(size_t)t * a.ss_ld + m];
-        s_inv[m] = a.ss_in ? rsqrtf(ss * a.inv_d + a.eps) : 1.f;
-      }
-      epi_bar();
-    }
+    grid_dep_wait();                                     // the partial buffer may still be read by the preceding kernel
     int seg = 0;
     for (int i = 0; i < n_units;) {
       const int u = u_begin + i;
@@ -420,30 +298,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
       tc_fence_before();
       if (lane == 0) mbar_arrive(accempty_bar(acc));     // the MMA warp may reuse this accumulator
-      if (a.epi != EPI_PARTIAL) {
-        int cidx = tile, expected;
-        if (a.epi == EPI_GATEUP) {
-          const int half_tiles = a.n_tiles >> 1;
-          const int tm = tile / a.n_tiles, p = (tile % a.n_tiles) % half_tiles;
-          cidx = tm * half_tiles + p;
-          expected = tile_slots(a, tm * a.n_tiles + p) + tile_slots(a, tm * a.n_tiles + p + half_tiles);
-        } else {
-          expected = tile_slots(a, tile);
-        }
-        __threadfence();                                 // this thread's slot stores before the arrival
-        epi_bar();
-        if (epi_tid == 0) {
-          const unsigned prev = atomicAdd(&a.counters[cidx], 1u);
-          const int last = (int)(prev + 1u) == expected;
-          if (last) a.counters[cidx] = 0u;               // back to rest for the next launch
-          s_last = last;
-        }
-        epi_bar();
-        if (s_last) {
-          __threadfence();
-          apply_epilogue<MT>(a, tile, epi_tid, s_inv, s_ss);
-        }
-      }
       i += seg_len;
       ++seg;
     }
@@ -530,11 +384,11 @@ hydra_status launch_b(const CUtensorMap& tw, const CUtensorMap& tx, const GemmAr
   return HYDRA_OK;
 }
 
-// Shared memory per CTA: 100 KB lets the CTAs of two consecutive (programmatically overlapped) GEMMs share an SM;
-// HYDRA_GEMM_SMEM_KB=200 selects a deeper ring with one CTA per SM.
+// Shared memory per CTA: a deep ring (one CTA per SM) by default; HYDRA_GEMM_SMEM_KB=100 selects a ring that lets
+// the CTAs of two consecutive (programmatically overlapped) GEMMs share an SM (measured: no faster).
 template <int MT>
 hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs& a, int grid, cudaStream_t st) {
-  static const int kb = []() { const char* e = getenv("HYDRA_GEMM_SMEM_KB"); return e ? atoi(e) : 100; }();
+  static const int kb = []() { const char* e = getenv("HYDRA_GEMM_SMEM_KB"); return e ? atoi(e) : 200; }();
   if (kb >= 200) return launch_b<MT, 200>(tw, tx, a, grid, st);
   return launch_b<MT, 100>(tw, tx, a, grid, st);
 }
@@ -568,33 +422,23 @@ SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots) {
   return sd;
 }
 
-hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part, int m, int n, int k, SplitDesc* sd_out,
-                     const GemmEpilogue* epi, int* status, cudaStream_t st) {
-  if (m <= 0 || n <= 0 || k <= 0 || n % BLOCK_N || k % BLOCK_K) return HYDRA_ERR_UNSUPPORTED;
+hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* w, float* part, int m, int n, int k,
+                     SplitDesc* sd_out, int* status, long long* trace, cudaStream_t st) {
+  if (m <= 0 || n <= 0 || k <= 0 || n % BLOCK_N || k % BLOCK_K || (x_planes != 1 && x_planes != 2)) return HYDRA_ERR_UNSUPPORTED;
   if (((uintptr_t)x | (uintptr_t)w) & 15) return HYDRA_ERR_INVALID;
   int grid = 1;
   SplitDesc sd = gemm_tc_plan(m, n, k, &grid, nullptr);
   if (x_rows_alloc < m) x_rows_alloc = m;
   CUtensorMap tw, tx;
   if (!get_tensor_map(w, (uint64_t)n, (uint64_t)k, BLOCK_N, &tw) ||
-      !get_tensor_map(x, (uint64_t)x_rows_alloc, (uint64_t)k, (uint32_t)sd.mt, &tx)) {
+      !get_tensor_map(x, (uint64_t)x_rows_alloc * x_planes, (uint64_t)k, (uint32_t)sd.mt, &tx)) {
     set_last_error("cuTensorMapEncodeTiled", cudaErrorUnknown);
     return HYDRA_ERR_CUDA;
   }
   GemmArgs a{};
   a.part = part; a.slot_stride = sd.stride; a.m = m; a.n = n; a.kb = sd.kb; a.n_tiles = sd.n_tiles;
-  a.total_units = sd.n_tiles * ((m + sd.mt - 1) / sd.mt) * sd.kb; a.q = sd.q; a.status = status; a.epi = EPI_PARTIAL;
-  if (epi && epi->kind != EPI_PARTIAL) {
-    if (m > 512 || !epi->counters) return HYDRA_ERR_UNSUPPORTED;
-    if (epi->kind == EPI_GATEUP && ((sd.n_tiles & 1) || epi->f != n / 2)) return HYDRA_ERR_UNSUPPORTED;
-    if (epi->kind == EPI_QKV && ((epi->H * epi->hd) % BLOCK_N || (epi->hd != 64 && epi->hd != 128))) return HYDRA_ERR_UNSUPPORTED;
-    a.epi = epi->kind; a.counters = epi->counters;
-    a.ss_in = epi->ss_in; a.ss_in_tiles = epi->ss_in_tiles; a.ss_ld = epi->ss_ld; a.inv_d = epi->inv_d; a.eps = epi->eps;
-    a.rs = epi->rs; a.rope = epi->rope; a.q_out = epi->q_out; a.kc = epi->kc; a.vc = epi->vc; a.H = epi->H; a.hd = epi->hd;
-    a.max_seq = epi->max_seq; a.x = epi->x; a.xg = epi->xg; a.gain = epi->gain; a.ss_out = epi->ss_out; a.act = epi->act;
-    a.f = epi->f; a.out = epi->out;
-  }
-  a.trace = epi ? epi->trace : nullptr;
+  a.total_units = sd.n_tiles * ((m + sd.mt - 1) / sd.mt) * sd.kb; a.q = sd.q; a.status = status;
+  a.x_lo_rows = x_planes == 2 ? x_rows_alloc : 0; a.trace = trace;
   if (sd_out) *sd_out = sd;
   switch (sd.mt) {
     case 16: return launch<16>(tw, tx, a, grid, st);

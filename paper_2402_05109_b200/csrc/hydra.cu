@@ -20,7 +20,6 @@ void set_last_error(const char* what, cudaError_t e) {
 
 namespace {
 
-constexpr int COUNTERS = 8192;     // tile arrival counters of the fused GEMM epilogues (>= tiles of any GEMM)
 constexpr int CHUNK = 64;          // rows per sequence of one prefill pass (and the row capacity of a forward call)
 
 struct LayerW { const void *attn_norm, *wqkv, *wo, *ffn_norm, *w_gate_up, *w_down; };
@@ -54,6 +53,7 @@ struct hydra_ctx {
   std::vector<const void*> head_w1, head_b1, head_wr, head_br;
   const void *embed, *lm_head, *final_norm;
   int esize;                                     // bytes per weight / KV element
+  int planes;                                    // planes of every operand / cache buffer: 2 (hi, lo) for bfloat16, 1 for float
   int R;                                         // row capacity of a forward call (padded)
   int RH;                                        // row capacity of the head buffers (padded)
   int maxP;
@@ -62,16 +62,15 @@ struct hydra_ctx {
   uint64_t *d_anc, *d_chain_mask;
   std::vector<int*> d_level_parents;
   int *d_len, *d_n_new, *d_root_tok, *d_status, *d_pos0, *d_nrows, *d_prompt_len, *d_offsets, *d_tok, *d_tree_tok, *d_amax;
-  unsigned int *d_done, *d_counters;
-  int ss_tiles;                                  // per-tile sums of squares describing the rows in x (fused path)
+  unsigned int* d_done;
   char *kv_base, *kv_pfx;
-  float *x, *part, *h_tree, *logits, *ss, *h_new, *hprime, *y, *head_logits;
+  float *x, *part, *h_tree, *logits, *h_new, *hprime, *y, *head_logits;
   float2* rope;
   void *topk_scratch; int topk_rows_cap;
   void *q, *xn, *attn_out, *act, *z, *yb, *att_scratch;
   size_t part_floats;
   // host state
-  int batch, state, gemm_mode, fused;
+  int batch, state, gemm_mode;
   std::vector<int> len_ub;
   const int* plant;
   long long launches;
@@ -155,6 +154,7 @@ hydra_status supported_cfg(const hydra_model_cfg* m) {
 size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, const TreeHost& t, char* ws) {
   Bump b{ws, 0};
   const int es = m.dtype == 0 ? 4 : 2;
+  const int np = m.dtype == 0 ? 1 : 2;          // bfloat16 operands and caches are stored as hi + lo planes
   const int d = m.d_model, f = m.d_ffn, V = m.vocab, K = h.n_heads, T = t.T;
   const int R = pad_rows(m.max_batch * CHUNK);
   const int RH = pad_rows(m.max_batch * t.maxP);
@@ -187,31 +187,29 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
   auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
   auto* done = b.take<unsigned int>(m.max_batch);
-  auto* counters = b.take<unsigned int>(COUNTERS);
-  auto* kvb = b.take<char>((size_t)m.n_layers * 2 * kv_layer_elems(m) * es);
-  auto* kvp = b.take<char>(h.prefix_attn ? (size_t)2 * kv_layer_elems(m) * es : 0);
-  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)R * d * es);
+  auto* kvb = b.take<char>((size_t)m.n_layers * 2 * np * kv_layer_elems(m) * es);
+  auto* kvp = b.take<char>(h.prefix_attn ? (size_t)2 * np * kv_layer_elems(m) * es : 0);
+  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)np * R * d * es);
   auto* part = b.take<float>(part_floats);
   auto* h_tree = b.take<float>((size_t)R * d);
   auto* logits = b.take<float>((size_t)pad_rows(m.max_batch * T) * V);
-  auto* ss = b.take<float>((size_t)(d / 128 + 1) * R);
   auto* h_new = b.take<float>((size_t)pad_rows(m.max_batch * (K + 1)) * d);
   auto* hprime = b.take<float>((size_t)m.max_batch * d);
   auto* y = b.take<float>((size_t)RH * d); auto* head_logits = b.take<float>((size_t)RH * V);
   auto* rope = b.take<float2>((size_t)R * (m.head_dim / 2));
-  auto* xn = b.take<char>((size_t)R * d * es); auto* attn_out = b.take<char>((size_t)R * d * es);
-  auto* act = b.take<char>((size_t)R * f * es);
-  auto* z = b.take<char>((size_t)RH * (K + 1) * d * es); auto* yb = b.take<char>((size_t)RH * d * es);
+  auto* xn = b.take<char>((size_t)np * R * d * es); auto* attn_out = b.take<char>((size_t)np * R * d * es);
+  auto* act = b.take<char>((size_t)np * R * f * es);
+  auto* z = b.take<char>((size_t)np * RH * (K + 1) * d * es); auto* yb = b.take<char>((size_t)np * RH * d * es);
   const int topk_cap = std::max(R, RH);
   auto* topk_s = b.take<char>(topk_scratch_bytes(topk_cap, V));
   auto* att = b.take<char>(attention_scratch_bytes(m.max_batch, CHUNK, m.n_heads, m.head_dim, m.max_seq));
   if (c) {
-    c->R = R; c->RH = RH; c->part_floats = part_floats; c->esize = es;
+    c->R = R; c->RH = RH; c->part_floats = part_floats; c->esize = es; c->planes = np;
     c->d_parent = parent; c->d_depth = depth; c->d_first_child = fc; c->d_n_child = nc; c->d_path_tab = path_tab;
     c->d_chain_depth = chain_depth; c->d_anc = anc; c->d_chain_mask = chain_mask; c->d_level_parents = lvl;
     c->d_len = len; c->d_n_new = n_new; c->d_root_tok = root; c->d_status = status; c->d_pos0 = pos0; c->d_nrows = nrows;
     c->d_prompt_len = plen; c->d_offsets = offs; c->d_tok = tok; c->d_tree_tok = tree_tok; c->d_amax = amax; c->d_done = done;
-    c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits; c->ss = ss; c->d_counters = counters;
+    c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits;
     c->h_new = h_new; c->hprime = hprime; c->y = y; c->head_logits = head_logits; c->rope = rope; c->xn = xn;
     c->attn_out = attn_out; c->act = act; c->z = z; c->yb = yb; c->att_scratch = att; c->topk_scratch = topk_s; c->topk_rows_cap = topk_cap;
   }
@@ -232,63 +230,21 @@ struct TimeScope {                // brackets the launches issued during its lif
 // Partial sums of x @ w^T into c->part; *sd says where the slots of each output tile are.
 hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void* w, int m, int n, int k, SplitDesc* sd,
                       cudaStream_t st) {
+  // algorithmic bytes of the launch: the weight matrix and the activation slab read once, the output written once
+  TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)c->planes * m * k) + 4.0 * m * n, st);
   if (c->m.dtype == 1 && c->gemm_mode == 0) {
     int slots = 1;
-    SplitDesc plan = gemm_tc_plan(m, n, k, nullptr, &slots);
+    gemm_tc_plan(m, n, k, nullptr, &slots);
     if ((size_t)slots * m * n > c->part_floats) return HYDRA_ERR_CAPACITY;
-    // algorithmic bytes of the launch: the weight matrix and the activation slab read once, the partial sums written once
-    TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * m * n, st);
-    (void)plan;
-    return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, c->part, m, n, k, sd, nullptr, c->d_status, st);
+    return gemm_tc((const bf16*)x, x_rows_alloc, c->planes, (const bf16*)w, c->part, m, n, k, sd, c->d_status, nullptr, st);
   }
-  TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * m * n, st);
   *sd = single_slot((size_t)m * n);
-  return gemm_simt(x, w, c->part, m, n, k, c->m.dtype, st);
+  return gemm_simt(x, w, c->part, m, n, k, c->m.dtype, st);      // bfloat16: the hi plane only (debug mode)
 }
 
-// The fused path: bfloat16 tensor-core GEMMs whose epilogues do the RoPE/KV append, residual adds, norm
-// statistics and SiLU*up, so a layer is five kernels (QKV, attention, O, gate/up, down).
-bool fused_ok(const hydra_ctx* c, int rows) {
-  const hydra_model_cfg& m = c->m;
-  long long tiles = (long long)std::max(std::max(3 * m.d_model, 2 * m.d_ffn), m.vocab) / 128 * ((rows + 255) / 256 + 1);
-  return m.dtype == 1 && c->gemm_mode == 0 && c->fused && rows <= 512 && m.d_model % 128 == 0 && m.d_ffn % 128 == 0 &&
-         tiles <= COUNTERS;
-}
-
-hydra_status run_gemm_fused(hydra_ctx* c, const void* x, int x_rows_alloc, const void* w, int m, int n, int k, GemmEpilogue& e,
-                            cudaStream_t st) {
-  int slots = 1;
-  gemm_tc_plan(m, n, k, nullptr, &slots);
-  if ((size_t)slots * m * n > c->part_floats) return HYDRA_ERR_CAPACITY;
-  e.counters = c->d_counters;
-  TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)m * k) + 4.0 * m * n, st);
-  return gemm_tc((const bf16*)x, x_rows_alloc, (const bf16*)w, c->part, m, n, k, nullptr, &e, c->d_status, st);
-}
-
-void norm_in(const hydra_ctx* c, GemmEpilogue& e) {
-  e.ss_in = c->ss; e.ss_in_tiles = c->ss_tiles; e.ss_ld = c->R; e.inv_d = 1.0f / (float)c->m.d_model; e.eps = c->m.rms_eps;
-}
-
-hydra_status run_layer_fused(hydra_ctx* c, const LayerW& w, char* kc, char* vc, const RowSet& rs, int len_upper,
-                             const void* next_gain, cudaStream_t st) {
-  const hydra_model_cfg& m = c->m;
-  const int rows = rs.batch * rs.tc, d = m.d_model, f = m.d_ffn;
-  GemmEpilogue q; q.kind = EPI_QKV; norm_in(c, q);
-  q.rs = rs; q.rope = c->rope; q.q_out = c->q; q.kc = kc; q.vc = vc; q.H = m.n_heads; q.hd = m.head_dim; q.max_seq = m.max_seq;
-  HYDRA_TRY(run_gemm_fused(c, c->xn, c->R, w.wqkv, rows, 3 * d, d, q, st));
-  {
-    TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
-    HYDRA_TRY(tree_attention(c->q, kc, vc, rs, c->attn_out, c->att_scratch, m.n_heads, m.head_dim, m.max_seq, len_upper, 1, st));
-  }
-  GemmEpilogue o; o.kind = EPI_RESID; o.x = c->x; o.xg = c->xn; o.gain = w.ffn_norm; o.ss_out = c->ss; o.ss_ld = c->R;
-  HYDRA_TRY(run_gemm_fused(c, c->attn_out, c->R, w.wo, rows, d, d, o, st));
-  c->ss_tiles = d / 128;
-  GemmEpilogue g; g.kind = EPI_GATEUP; norm_in(c, g); g.act = c->act; g.f = f;
-  HYDRA_TRY(run_gemm_fused(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, g, st));
-  GemmEpilogue dn; dn.kind = EPI_RESID; dn.x = c->x; dn.xg = c->xn; dn.gain = next_gain; dn.ss_out = c->ss; dn.ss_ld = c->R;
-  HYDRA_TRY(run_gemm_fused(c, c->act, c->R, w.w_down, rows, d, f, dn, st));
-  return HYDRA_OK;
-}
+// element distance between the hi and lo planes of an operand buffer of `rows_alloc` rows of `cols` (0 for float)
+size_t ps(const hydra_ctx* c, int rows_alloc, size_t cols) { return c->planes == 2 ? (size_t)rows_alloc * cols : 0; }
+size_t kv_ps(const hydra_ctx* c) { return c->planes == 2 ? kv_layer_elems(c->m) : 0; }
 
 // One decoder layer over the rows of `rs`.  Expects the residual rows in c->x and their normed copy in c->xn.
 // Leaves the updated residual in c->x; when next_gain is given also xn = rmsnorm(x)*next_gain (and hn in float).
@@ -298,17 +254,18 @@ hydra_status run_layer(hydra_ctx* c, const LayerW& w, char* kc, char* vc, const 
   const int rows = rs.batch * rs.tc, d = m.d_model, f = m.d_ffn, dt = m.dtype;
   SplitDesc sd;
   HYDRA_TRY(run_gemm(c, c->xn, c->R, w.wqkv, rows, 3 * d, d, &sd, st));
-  HYDRA_TRY(qkv_rope_store(c->part, sd, c->rope, c->q, kc, vc, rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
+  HYDRA_TRY(qkv_rope_store(c->part, sd, c->rope, c->q, ps(c, c->R, d), kc, vc, kv_ps(c), rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
   {
     TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
-    HYDRA_TRY(tree_attention(c->q, kc, vc, rs, c->attn_out, c->att_scratch, m.n_heads, m.head_dim, m.max_seq, len_upper, dt, st));
+    HYDRA_TRY(tree_attention(c->q, ps(c, c->R, d), kc, vc, kv_ps(c), rs, c->attn_out, ps(c, c->R, d), c->att_scratch, m.n_heads, m.head_dim,
+                             m.max_seq, len_upper, dt, st));
   }
   HYDRA_TRY(run_gemm(c, c->attn_out, c->R, w.wo, rows, d, d, &sd, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, c->part, sd, c->x, w.ffn_norm, c->xn, nullptr, rows, d, m.rms_eps, dt, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, c->part, sd, c->x, w.ffn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, dt, st));
   HYDRA_TRY(run_gemm(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, &sd, st));
-  HYDRA_TRY(silu_mul(c->part, sd, c->act, rows, f, dt, st));
+  HYDRA_TRY(silu_mul(c->part, sd, c->act, ps(c, c->R, f), rows, f, dt, st));
   HYDRA_TRY(run_gemm(c, c->act, c->R, w.w_down, rows, d, f, &sd, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, c->part, sd, c->x, next_gain, next_gain ? c->xn : nullptr, hn, rows, d, m.rms_eps, dt, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, c->part, sd, c->x, next_gain, next_gain ? c->xn : nullptr, ps(c, c->R, d), hn, rows, d, m.rms_eps, dt, st));
   return HYDRA_OK;
 }
 
@@ -317,20 +274,10 @@ hydra_status run_layer(hydra_ctx* c, const LayerW& w, char* kc, char* vc, const 
 hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_upper, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int rows = rs.batch * rs.tc;
-  const size_t kvl = kv_layer_elems(m) * c->esize;
+  const size_t kvl = kv_layer_elems(m) * c->esize * c->planes;      // bytes of one layer's K (or V) cache, all planes
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
-  if (fused_ok(c, rows)) {
-    HYDRA_TRY(rows_prepare(nullptr, c->embed, tok, m.vocab, c->layers[0].attn_norm, c->x, c->xn, c->ss, rows, m.d_model, c->d_status, st));
-    c->ss_tiles = 1;
-    for (int l = 0; l < m.n_layers; ++l) {
-      bool last = l + 1 == m.n_layers;
-      HYDRA_TRY(run_layer_fused(c, c->layers[l], c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs,
-                                len_upper, last ? c->final_norm : c->layers[l + 1].attn_norm, st));
-    }
-    return finalize_hidden(c->x, c->ss, c->ss_tiles, c->R, c->final_norm, m.rms_eps, c->h_tree, rows, m.d_model, st);
-  }
   HYDRA_TRY(embed_rows(c->embed, tok, c->x, rows, m.d_model, m.vocab, m.dtype, c->d_status, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, nullptr, single_slot(0), c->x, c->layers[0].attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, nullptr, single_slot(0), c->x, c->layers[0].attn_norm, c->xn, ps(c, c->R, m.d_model), nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
   for (int l = 0; l < m.n_layers; ++l) {
     bool last = l + 1 == m.n_layers;
     HYDRA_TRY(run_layer(c, c->layers[l], c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs, len_upper,
@@ -343,14 +290,9 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
 hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int len_upper, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int rows = rs.batch * rs.tc;
-  const size_t kvl = kv_layer_elems(m) * c->esize;
+  const size_t kvl = kv_layer_elems(m) * c->esize * c->planes;      // bytes of one layer's K (or V) cache, all planes
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
-  if (fused_ok(c, rows)) {
-    HYDRA_TRY(rows_prepare(src, nullptr, nullptr, 0, c->pfx.attn_norm, c->x, c->xn, c->ss, rows, m.d_model, c->d_status, st));
-    c->ss_tiles = 1;
-    return run_layer_fused(c, c->pfx, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, nullptr, st);
-  }
-  HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
+  HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, ps(c, c->R, m.d_model), nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
   return run_layer(c, c->pfx, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, nullptr, nullptr, st);
 }
 
@@ -375,15 +317,16 @@ hydra_status do_draft(hydra_ctx* c, int* tree_tok, cudaStream_t st) {
     const int P = (int)c->level_parents[lvl - 1].size();
     const int rows = B * P;
     LevelDesc lv{lvl, P, c->d_level_parents[lvl - 1]};
-    HYDRA_TRY(head_gather(c->hprime, c->embed, c->d_root_tok, tree_tok, c->d_path_tab, lv, c->z, B, c->T, K + 1, d, m.vocab, dt, c->d_status, st));
+    HYDRA_TRY(head_gather(c->hprime, c->embed, c->d_root_tok, tree_tok, c->d_path_tab, lv, c->z, ps(c, c->RH, (size_t)(lvl + 1) * d), B, c->T, K + 1, d, m.vocab, dt,
+                          c->d_status, st));
     SplitDesc sd;
     HYDRA_TRY(run_gemm(c, c->z, c->RH, c->head_w1[lvl - 1], rows, d, (lvl + 1) * d, &sd, st));
-    HYDRA_TRY(head_act(c->hprime, 1, P, c->part, sd, c->h.has_bias ? c->head_b1[lvl - 1] : nullptr, c->y, c->yb, rows, d, dt, st));
+    HYDRA_TRY(head_act(c->hprime, 1, P, c->part, sd, c->h.has_bias ? c->head_b1[lvl - 1] : nullptr, c->y, c->yb, ps(c, c->RH, d), rows, d, dt, st));
     for (int l = 0; l + 1 < c->h.n_mlp_layers; ++l) {
       const char* wr = (const char*)c->head_wr[lvl - 1] + (size_t)l * d * d * c->esize;
       const char* br = c->h.has_bias ? (const char*)c->head_br[lvl - 1] + (size_t)l * d * c->esize : nullptr;
       HYDRA_TRY(run_gemm(c, c->yb, c->RH, wr, rows, d, d, &sd, st));
-      HYDRA_TRY(head_act(c->y, 0, P, c->part, sd, br, c->y, c->yb, rows, d, dt, st));
+      HYDRA_TRY(head_act(c->y, 0, P, c->part, sd, br, c->y, c->yb, ps(c, c->RH, d), rows, d, dt, st));
     }
     HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, rows, m.vocab, d, &sd, st));
     int max_children = 1;
@@ -399,12 +342,6 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
   const int rows = c->batch * c->T;
   RowSet rs{c->batch, c->T, nullptr, c->d_len, c->d_depth, c->d_anc};
   HYDRA_TRY(run_base(c, tree_tok, rs, len_bucket(c, max_len_ub(c) + c->T), st));
-  if (fused_ok(c, rows)) {                 // c->xn holds x * final_norm gain; the LM head scales its rows by inv_rms
-    float* lg = logits ? logits : c->logits;
-    GemmEpilogue e; e.kind = EPI_OUT; norm_in(c, e); e.out = lg;
-    HYDRA_TRY(run_gemm_fused(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, e, st));
-    return argmax_rows(lg, single_slot(0), nullptr, amax, c->topk_scratch, c->topk_rows_cap, rows, m.vocab, st);
-  }
   SplitDesc sd;
   HYDRA_TRY(run_gemm(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, &sd, st));
   return argmax_rows(c->part, sd, logits, amax, c->topk_scratch, c->topk_rows_cap, rows, m.vocab, st);
@@ -415,7 +352,7 @@ hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* 
   AcceptArgs a{};
   a.tree_tok = tree_tok; a.amax = amax; a.parent = c->d_parent; a.depth = c->d_depth; a.anc = c->d_anc;
   a.T = c->T; a.K = c->h.n_heads; a.batch = c->batch; a.n_layers = m.n_layers; a.n_heads = m.n_heads; a.head_dim = m.head_dim;
-  a.max_seq = m.max_seq; a.max_batch = m.max_batch; a.d_model = m.d_model; a.esize = c->esize;
+  a.max_seq = m.max_seq; a.max_batch = m.max_batch; a.d_model = m.d_model; a.esize = c->esize; a.kv_planes = c->planes;
   a.kv_base = c->kv_base; a.h_tree = c->h_tree; a.h_tree_stride = c->T;
   a.h_new = c->h_new; a.n_new = c->d_n_new; a.len = c->d_len; a.root_tok = c->d_root_tok;
   a.n_acc = n_acc; a.path = path; a.out_tok = out_tok; a.done_counter = c->d_done; a.status = c->d_status;
@@ -498,7 +435,7 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
   }
   c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
   carve(c, *m, *h, th, (char*)ws);
-  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->fused = 0; c->ss_tiles = 1; c->plant = nullptr; c->launches = 0; c->timing = 0; c->steps_done = 0;
+  c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->plant = nullptr; c->launches = 0; c->timing = 0; c->steps_done = 0;
   { const char* e = getenv("HYDRA_NO_GRAPH"); c->use_graph = !(e && e[0] == '1'); }
   c->len_ub.assign(m->max_batch, 0);
   // clear the workspace, upload the static tables
@@ -560,7 +497,7 @@ hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const
   }
   // root token = argmax of the logits of the last prompt row
   HYDRA_TRY(pick_last_row(c->h_new, c->d_n_new, c->h.n_heads + 1, c->hprime, batch, m.d_model, st));
-  HYDRA_TRY(cast_rows(c->hprime, c->yb, (size_t)batch * m.d_model, m.dtype, st));
+  HYDRA_TRY(cast_rows(c->hprime, c->yb, ps(c, c->RH, m.d_model), (size_t)batch * m.d_model, m.dtype, st));
   SplitDesc sd;
   HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, batch, m.vocab, m.d_model, &sd, st));
   HYDRA_TRY(argmax_rows(c->part, sd, nullptr, c->d_root_tok, c->topk_scratch, c->topk_rows_cap, batch, m.vocab, st));
@@ -648,7 +585,7 @@ hydra_status hydra_set_plant(hydra_ctx* c, const int32_t* plant) {
 hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes) {
   if (!c || !ptr) return HYDRA_ERR_INVALID;
   const hydra_model_cfg& m = c->m;
-  const size_t kvl = kv_layer_elems(m) * c->esize;
+  const size_t kvl = kv_layer_elems(m) * c->esize * c->planes;      // bytes of one layer's K (or V) cache, all planes
   const int K = c->h.n_heads;
   void* p = nullptr; size_t n = 0;
   switch (which) {
@@ -656,7 +593,7 @@ hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes
     case HYDRA_BUF_ROOT_TOK: p = c->d_root_tok; n = m.max_batch * sizeof(int); break;
     case HYDRA_BUF_H_TREE: p = c->h_tree; n = (size_t)c->R * m.d_model * sizeof(float); break;
     case HYDRA_BUF_H_NEW: p = c->h_new; n = (size_t)m.max_batch * (K + 1) * m.d_model * sizeof(float); break;
-    case HYDRA_BUF_KV_BASE: p = c->kv_base; n = (size_t)m.n_layers * 2 * kvl; break;
+    case HYDRA_BUF_KV_BASE: p = c->kv_base; n = (size_t)m.n_layers * 2 * kvl; break;          // kvl covers all planes
     case HYDRA_BUF_KV_PREFIX: p = c->h.prefix_attn ? c->kv_pfx : nullptr; n = c->h.prefix_attn ? 2 * kvl : 0; break;
     case HYDRA_BUF_TREE_MASK: p = c->d_anc; n = c->T * sizeof(uint64_t); break;
     case HYDRA_BUF_TREE_TOK: p = c->d_tree_tok; n = (size_t)m.max_batch * c->T * sizeof(int); break;
@@ -711,9 +648,8 @@ hydra_status hydra_get_timing(hydra_ctx* c, int kclass, double* ms_total, long l
 }
 
 hydra_status hydra_set_gemm_mode(hydra_ctx* c, int mode) {
-  if (!c || mode < 0 || mode > 2) return HYDRA_ERR_INVALID;
-  c->gemm_mode = mode == 1 ? 1 : 0;
-  c->fused = mode == 2;
+  if (!c || (mode != 0 && mode != 1)) return HYDRA_ERR_INVALID;
+  c->gemm_mode = mode;
   drop_graphs(c);
   return HYDRA_OK;
 }
@@ -743,15 +679,16 @@ size_t hydra_gemm_partial_floats(int m, int n, int k, int dtype, int mode) {
 }
 
 hydra_status hydra_gemm(const void* x, const void* w, float* out, float* partial, int m, int n, int k, int dtype, int mode,
-                        int32_t* status, void* stream) {
+                        int x_planes, int32_t* status, void* stream) {
   if (!x || !w || !out || !partial || m < 1 || n < 1 || k < 1 || (dtype != 0 && dtype != 1)) return HYDRA_ERR_INVALID;
+  if (x_planes != 1 && !(x_planes == 2 && dtype == 1 && mode == 0)) return HYDRA_ERR_INVALID;
   cudaStream_t st = (cudaStream_t)stream;
   CounterScope cs(nullptr);
   if (dtype == 1 && mode == 0) {
     if (!status) return HYDRA_ERR_INVALID;
     if (!gemm_tc_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
     SplitDesc sd;
-    HYDRA_TRY(gemm_tc((const bf16*)x, m, (const bf16*)w, partial, m, n, k, &sd, nullptr, status, st));
+    HYDRA_TRY(gemm_tc((const bf16*)x, m, x_planes, (const bf16*)w, partial, m, n, k, &sd, status, nullptr, st));
     return reduce_splits(partial, sd, out, m, n, st);
   }
   return gemm_simt(x, w, out, m, n, k, dtype, st);
@@ -764,11 +701,14 @@ size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_di
 
 hydra_status hydra_tree_attention(const void* q, const void* kc, const void* vc, const int32_t* pos0, const int32_t* n_rows,
                                   const uint64_t* mask, void* out, void* scratch, int batch, int tc, int n_heads, int head_dim,
-                                  int max_seq, int dtype, void* stream) {
+                                  int max_seq, int dtype, int planes, void* stream) {
   if (!q || !kc || !vc || !pos0 || !mask || !out || !scratch || batch < 1 || tc < 1 || tc > 64) return HYDRA_ERR_INVALID;
+  if (planes != 1 && !(planes == 2 && dtype == 1)) return HYDRA_ERR_INVALID;
   CounterScope cs(nullptr);
   RowSet rs{batch, tc, n_rows, pos0, nullptr, mask};
-  return tree_attention(q, kc, vc, rs, out, scratch, n_heads, head_dim, max_seq, max_seq, dtype, (cudaStream_t)stream);
+  const size_t d = (size_t)n_heads * head_dim;
+  const size_t qp = planes == 2 ? (size_t)batch * tc * d : 0, kvp = planes == 2 ? (size_t)batch * n_heads * max_seq * head_dim : 0;
+  return tree_attention(q, qp, kc, vc, kvp, rs, out, qp, scratch, n_heads, head_dim, max_seq, max_seq, dtype, (cudaStream_t)stream);
 }
 
 }  // extern "C"

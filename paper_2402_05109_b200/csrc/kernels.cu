@@ -128,11 +128,29 @@ template <> __device__ __forceinline__ float4 load4<bf16>(const bf16* p) {
   float v[4]; Vec4<bf16>::load(p, v); return make_float4(v[0], v[1], v[2], v[3]);
 }
 
+// Operand storage.  float buffers hold one plane.  bfloat16 operand buffers hold two planes `ps` elements apart:
+// hi = bf16(v) and lo = bf16(v - hi), together about 16 mantissa bits (ps = 0 stores hi only).
+template <typename T> __device__ __forceinline__ void put(T* p, size_t ps, float v);
+template <> __device__ __forceinline__ void put<float>(float* p, size_t, float v) { *p = v; }
+template <> __device__ __forceinline__ void put<bf16>(bf16* p, size_t ps, float v) {
+  const bf16 h = __float2bfloat16_rn(v);
+  *p = h;
+  if (ps) p[ps] = __float2bfloat16_rn(v - __bfloat162float(h));
+}
+template <typename T> __device__ __forceinline__ void put4(T* p, size_t ps, float4 v);
+template <> __device__ __forceinline__ void put4<float>(float* p, size_t, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+template <> __device__ __forceinline__ void put4<bf16>(bf16* p, size_t ps, float4 v) {
+  const float4 h = make_float4(__bfloat162float(__float2bfloat16_rn(v.x)), __bfloat162float(__float2bfloat16_rn(v.y)),
+                               __bfloat162float(__float2bfloat16_rn(v.z)), __bfloat162float(__float2bfloat16_rn(v.w)));
+  store4<bf16>(p, h);
+  if (ps) store4<bf16>(p + ps, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
+}
+
 constexpr int NORM_THREADS = 512;
 template <typename T>
 __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const float* res, const float* __restrict__ part,
                                                                         SplitDesc sd, float* x_out,
-                                                                        const T* __restrict__ gain, T* __restrict__ xn,
+                                                                        const T* __restrict__ gain, T* __restrict__ xn, size_t xn_ps,
                                                                         float* __restrict__ hn, int d, float eps) {
   pdl_trigger();
   pdl_wait();
@@ -158,78 +176,20 @@ __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const fl
     float4 v = *reinterpret_cast<const float4*>(x_out + base + i);
     float4 gn = load4<T>(gain + i);
     v.x *= inv * gn.x; v.y *= inv * gn.y; v.z *= inv * gn.z; v.w *= inv * gn.w;
-    if (xn) store4<T>(xn + base + i, v);
+    if (xn) put4<T>(xn + base + i, xn_ps, v);
     if (hn) *reinterpret_cast<float4*>(hn + base + i) = v;
   }
 }
 hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd, float* x_out,
-                              const void* gain, void* xn, float* hn, int rows, int d, float eps, int dtype,
+                              const void* gain, void* xn, size_t xn_ps, float* hn, int rows, int d, float eps, int dtype,
                               cudaStream_t st) {
   if (d & 3) return HYDRA_ERR_UNSUPPORTED;
   if (dtype == 0)
     launch_pdl(residual_rmsnorm_kernel<float>, dim3(rows), dim3(NORM_THREADS), 0, st, res, part, sd, x_out, (const float*)gain,
-                                                                  (float*)xn, hn, d, eps);
+                                                                  (float*)xn, xn_ps, hn, d, eps);
   else
     launch_pdl(residual_rmsnorm_kernel<bf16>, dim3(rows), dim3(NORM_THREADS), 0, st, res, part, sd, x_out, (const bf16*)gain,
-                                                                 (bf16*)xn, hn, d, eps);
-  HYDRA_LAUNCH_CHECK();
-  return HYDRA_OK;
-}
-
-// Rows entering a fused layer stack: x = src row (or the embedding of tok), xg = bf16(x * gain), ss[m] = sum x^2.
-__global__ void __launch_bounds__(NORM_THREADS) rows_prepare_kernel(const float* __restrict__ src, const bf16* __restrict__ embed,
-                                                                    const int* __restrict__ tok, int vocab,
-                                                                    const bf16* __restrict__ gain, float* __restrict__ x,
-                                                                    bf16* __restrict__ xg, float* __restrict__ ss, int d, int* status) {
-  pdl_trigger();
-  pdl_wait();
-  __shared__ float sh[32];
-  const int r = blockIdx.x;
-  const size_t base = (size_t)r * d;
-  const bf16* e = nullptr;
-  if (embed) {
-    int t = tok[r];
-    if (t < 0 || t >= vocab) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); t = 0; }
-    e = embed + (size_t)t * d;
-  }
-  float acc = 0.f;
-  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
-    float4 v = e ? load4<bf16>(e + i) : *reinterpret_cast<const float4*>(src + base + i);
-    float4 gn = load4<bf16>(gain + i);
-    *reinterpret_cast<float4*>(x + base + i) = v;
-    store4<bf16>(xg + base + i, make_float4(v.x * gn.x, v.y * gn.y, v.z * gn.z, v.w * gn.w));
-    acc += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-  }
-  float tot = block_sum(acc, sh);
-  if (threadIdx.x == 0) ss[r] = tot;
-}
-hydra_status rows_prepare(const float* src, const void* embed, const int* tok, int vocab, const void* gain, float* x, void* xg,
-                          float* ss, int rows, int d, int* status, cudaStream_t st) {
-  launch_pdl(rows_prepare_kernel, dim3(rows), dim3(NORM_THREADS), 0, st, src, (const bf16*)embed, tok, vocab, (const bf16*)gain, x, (bf16*)xg, ss, d, status);
-  HYDRA_LAUNCH_CHECK();
-  return HYDRA_OK;
-}
-
-// h[m] = x[m] * gain * rsqrt(sum_t ss[t*ld + m] / d + eps)   (the normalised hidden rows, float)
-__global__ void __launch_bounds__(NORM_THREADS) finalize_hidden_kernel(const float* __restrict__ x, const float* __restrict__ ss,
-                                                                       int ss_tiles, int ld, const bf16* __restrict__ gain,
-                                                                       float eps, float* __restrict__ h, int d) {
-  pdl_trigger();
-  pdl_wait();
-  const int r = blockIdx.x;
-  float tot = 0.f;
-  for (int t = 0; t < ss_tiles; ++t) tot += ss[(size_t)t * ld + r];
-  const float inv = rsqrtf(tot / (float)d + eps);
-  const size_t base = (size_t)r * d;
-  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
-    float4 v = *reinterpret_cast<const float4*>(x + base + i);
-    float4 gn = load4<bf16>(gain + i);
-    *reinterpret_cast<float4*>(h + base + i) = make_float4(v.x * inv * gn.x, v.y * inv * gn.y, v.z * inv * gn.z, v.w * inv * gn.w);
-  }
-}
-hydra_status finalize_hidden(const float* x, const float* ss, int ss_tiles, int ld, const void* gain, float eps, float* h,
-                             int rows, int d, cudaStream_t st) {
-  launch_pdl(finalize_hidden_kernel, dim3(rows), dim3(NORM_THREADS), 0, st, x, ss, ss_tiles, ld, (const bf16*)gain, eps, h, d);
+                                                                 (bf16*)xn, xn_ps, hn, d, eps);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -258,8 +218,9 @@ hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cud
 template <typename T>
 __global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restrict__ part, SplitDesc sd,
                                                             const float2* __restrict__ table, T* __restrict__ q,
-                                                            T* __restrict__ kc, T* __restrict__ vc, RowSet rs, int H,
-                                                            int hd, int max_seq, int* status) {
+                                                            size_t q_ps, T* __restrict__ kc, T* __restrict__ vc,
+                                                            size_t kv_ps, RowSet rs, int H, int hd, int max_seq,
+                                                            int* status) {
   pdl_trigger();
   pdl_wait();
   const int r = blockIdx.x, h = blockIdx.y, b = r / rs.tc, i = r % rs.tc;
@@ -283,23 +244,23 @@ __global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restr
   }
   const float qa = v6[0], qb = v6[1], ka = v6[2], kb = v6[3], va = v6[4], vb = v6[5];
   const float2 cs = table[(size_t)r * half + j];
-  q[(size_t)r * d + c0] = from_f<T>(qa * cs.x - qb * cs.y);
-  q[(size_t)r * d + c1] = from_f<T>(qb * cs.x + qa * cs.y);
+  put<T>(q + (size_t)r * d + c0, q_ps, qa * cs.x - qb * cs.y);
+  put<T>(q + (size_t)r * d + c1, q_ps, qb * cs.x + qa * cs.y);
   const size_t o = (((size_t)b * H + h) * max_seq + slot) * hd;
-  kc[o + j] = from_f<T>(ka * cs.x - kb * cs.y);
-  kc[o + j + half] = from_f<T>(kb * cs.x + ka * cs.y);
-  vc[o + j] = from_f<T>(va);
-  vc[o + j + half] = from_f<T>(vb);
+  put<T>(kc + o + j, kv_ps, ka * cs.x - kb * cs.y);
+  put<T>(kc + o + j + half, kv_ps, kb * cs.x + ka * cs.y);
+  put<T>(vc + o + j, kv_ps, va);
+  put<T>(vc + o + j + half, kv_ps, vb);
 }
-hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, void* kcache,
-                            void* vcache, RowSet rs, int H, int hd, int max_seq, int dtype, int* status,
+hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, size_t q_ps, void* kcache,
+                            void* vcache, size_t kv_ps, RowSet rs, int H, int hd, int max_seq, int dtype, int* status,
                             cudaStream_t st) {
   dim3 grid(rs.batch * rs.tc, H);
   if (dtype == 0)
-    launch_pdl(qkv_rope_store_kernel<float>, dim3(grid), dim3(64), 0, st, part, sd, table, (float*)q, (float*)kcache, (float*)vcache,
-                                                      rs, H, hd, max_seq, status);
+    launch_pdl(qkv_rope_store_kernel<float>, dim3(grid), dim3(64), 0, st, part, sd, table, (float*)q, q_ps, (float*)kcache, (float*)vcache,
+                                                      kv_ps, rs, H, hd, max_seq, status);
   else
-    launch_pdl(qkv_rope_store_kernel<bf16>, dim3(grid), dim3(64), 0, st, part, sd, table, (bf16*)q, (bf16*)kcache, (bf16*)vcache, rs,
+    launch_pdl(qkv_rope_store_kernel<bf16>, dim3(grid), dim3(64), 0, st, part, sd, table, (bf16*)q, q_ps, (bf16*)kcache, (bf16*)vcache, kv_ps, rs,
                                                      H, hd, max_seq, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -459,11 +420,12 @@ static hydra_status tree_attention_t(const T* q, const T* kc, const T* vc, RowSe
   return HYDRA_OK;
 }
 
-hydra_status tree_attention(const void* q, const void* kc, const void* vc, RowSet rs, void* out, void* scratch, int H,
-                            int hd, int max_seq, int len_upper, int dtype, cudaStream_t st) {
+hydra_status tree_attention(const void* q, size_t q_ps, const void* kc, const void* vc, size_t kv_ps, RowSet rs, void* out,
+                            size_t out_ps, void* scratch, int H, int hd, int max_seq, int len_upper, int dtype, cudaStream_t st) {
   if (rs.tc > 64) return HYDRA_ERR_UNSUPPORTED;
   if (dtype == 1)
-    return tree_attention_tc((const bf16*)q, (const bf16*)kc, (const bf16*)vc, rs, (bf16*)out, scratch, H, hd, max_seq, len_upper, st);
+    return tree_attention_tc((const bf16*)q, q_ps, (const bf16*)kc, (const bf16*)vc, kv_ps, rs, (bf16*)out, out_ps, scratch, H, hd,
+                             max_seq, len_upper, st);
   if (dtype == 0 && hd == 64)
     return tree_attention_t<float, 64>((const float*)q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
   if (dtype == 0 && hd == 128)
@@ -475,7 +437,7 @@ hydra_status tree_attention(const void* q, const void* kc, const void* vc, RowSe
 // SiLU(gate) * up from the gate/up partial sums
 // ------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void silu_mul_kernel(const float* __restrict__ part, SplitDesc sd, T* __restrict__ act, int rows, int f) {
+__global__ void silu_mul_kernel(const float* __restrict__ part, SplitDesc sd, T* __restrict__ act, size_t act_ps, int rows, int f) {
   pdl_trigger();
   pdl_wait();
   size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
@@ -486,14 +448,14 @@ __global__ void silu_mul_kernel(const float* __restrict__ part, SplitDesc sd, T*
   const int ng = split_count(sd, r, c), nu = split_count(sd, r, f + c);
   for (int s = 0; s < ng; ++s) { float4 a = *reinterpret_cast<const float4*>(p + s * sd.stride + c); g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w; }
   for (int s = 0; s < nu; ++s) { float4 a = *reinterpret_cast<const float4*>(p + s * sd.stride + f + c); u.x += a.x; u.y += a.y; u.z += a.z; u.w += a.w; }
-  store4<T>(act + i, make_float4(silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w));
+  put4<T>(act + i, act_ps, make_float4(silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w));
 }
-hydra_status silu_mul(const float* part, SplitDesc sd, void* act, int rows, int f, int dtype, cudaStream_t st) {
+hydra_status silu_mul(const float* part, SplitDesc sd, void* act, size_t act_ps, int rows, int f, int dtype, cudaStream_t st) {
   if (f & 3) return HYDRA_ERR_UNSUPPORTED;
   size_t n = (size_t)rows * f / 4;
   unsigned grid = (unsigned)((n + 255) / 256);
-  if (dtype == 0) launch_pdl(silu_mul_kernel<float>, dim3(grid), dim3(256), 0, st, part, sd, (float*)act, rows, f);
-  else launch_pdl(silu_mul_kernel<bf16>, dim3(grid), dim3(256), 0, st, part, sd, (bf16*)act, rows, f);
+  if (dtype == 0) launch_pdl(silu_mul_kernel<float>, dim3(grid), dim3(256), 0, st, part, sd, (float*)act, act_ps, rows, f);
+  else launch_pdl(silu_mul_kernel<bf16>, dim3(grid), dim3(256), 0, st, part, sd, (bf16*)act, act_ps, rows, f);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -645,7 +607,7 @@ hydra_status topk_children(const float* part, SplitDesc sd, float* logits, Level
 template <typename T>
 __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restrict__ hprime, const T* __restrict__ embed,
                                                           const int* __restrict__ root_tok, int* tree_tok,
-                                                          const int* __restrict__ path_tab, LevelDesc lv, T* __restrict__ z,
+                                                          const int* __restrict__ path_tab, LevelDesc lv, T* __restrict__ z, size_t z_ps,
                                                           int T_rows, int kp1, int d_model, int vocab, int* status) {
   pdl_trigger();
   pdl_wait();
@@ -654,7 +616,7 @@ __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restric
   const int p = lv.parents[j];
   T* dst = z + ((size_t)row * (lv.d + 1) + blk) * d_model;
   if (blk == 0) {
-    for (int i = threadIdx.x; i < d_model; i += blockDim.x) dst[i] = from_f<T>(hprime[(size_t)b * d_model + i]);
+    for (int i = threadIdx.x; i < d_model; i += blockDim.x) put<T>(dst + i, z_ps, hprime[(size_t)b * d_model + i]);
     if (lv.d == 1 && j == 0 && threadIdx.x == 0) tree_tok[b * T_rows] = root_tok[b];
     return;
   }
@@ -662,17 +624,17 @@ __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restric
   int t = node == 0 ? root_tok[b] : tree_tok[b * T_rows + node];
   if (t < 0 || t >= vocab) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); t = 0; }
   const T* e = embed + (size_t)t * d_model;
-  for (int i = threadIdx.x; i < d_model; i += blockDim.x) dst[i] = e[i];
+  for (int i = threadIdx.x; i < d_model; i += blockDim.x) put<T>(dst + i, z_ps, to_f<T>(e[i]));      // embeddings are exact: lo = 0
 }
 hydra_status head_gather(const float* hprime, const void* embed, const int* root_tok, int* tree_tok, const int* path_tab,
-                         LevelDesc lv, void* z, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
+                         LevelDesc lv, void* z, size_t z_ps, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
                          cudaStream_t st) {
   dim3 grid(batch * lv.n_parents, lv.d + 1);
   if (dtype == 0)
-    launch_pdl(head_gather_kernel<float>, dim3(grid), dim3(256), 0, st, hprime, (const float*)embed, root_tok, tree_tok, path_tab, lv, (float*)z,
+    launch_pdl(head_gather_kernel<float>, dim3(grid), dim3(256), 0, st, hprime, (const float*)embed, root_tok, tree_tok, path_tab, lv, (float*)z, z_ps,
                                                     T, kp1, d_model, vocab, status);
   else
-    launch_pdl(head_gather_kernel<bf16>, dim3(grid), dim3(256), 0, st, hprime, (const bf16*)embed, root_tok, tree_tok, path_tab, lv, (bf16*)z,
+    launch_pdl(head_gather_kernel<bf16>, dim3(grid), dim3(256), 0, st, hprime, (const bf16*)embed, root_tok, tree_tok, path_tab, lv, (bf16*)z, z_ps,
                                                    T, kp1, d_model, vocab, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -680,7 +642,7 @@ hydra_status head_gather(const float* hprime, const void* embed, const int* root
 
 template <typename T>
 __global__ void head_act_kernel(const float* res, int res_is_hprime, int rows_per_b, const float* __restrict__ part,
-                                SplitDesc sd, const T* __restrict__ bias, float* y_out, T* __restrict__ yb,
+                                SplitDesc sd, const T* __restrict__ bias, float* y_out, T* __restrict__ yb, size_t yb_ps,
                                 int rows, int d) {
   pdl_trigger();
   pdl_wait();
@@ -693,18 +655,18 @@ __global__ void head_act_kernel(const float* res, int res_is_hprime, int rows_pe
   float base = res_is_hprime ? res[(size_t)(r / rows_per_b) * d + c] : res[i];
   float y = base + silu_f(v);
   y_out[i] = y;
-  yb[i] = from_f<T>(y);
+  put<T>(yb + i, yb_ps, y);
 }
 hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, SplitDesc sd,
-                      const void* bias, float* y_out, void* yb, int rows, int d, int dtype, cudaStream_t st) {
+                      const void* bias, float* y_out, void* yb, size_t yb_ps, int rows, int d, int dtype, cudaStream_t st) {
   size_t n = (size_t)rows * d;
   unsigned grid = (unsigned)((n + 255) / 256);
   if (dtype == 0)
     launch_pdl(head_act_kernel<float>, dim3(grid), dim3(256), 0, st, res, res_is_hprime, rows_per_b, part, sd, (const float*)bias,
-                                                 y_out, (float*)yb, rows, d);
+                                                 y_out, (float*)yb, yb_ps, rows, d);
   else
     launch_pdl(head_act_kernel<bf16>, dim3(grid), dim3(256), 0, st, res, res_is_hprime, rows_per_b, part, sd, (const bf16*)bias,
-                                                y_out, (bf16*)yb, rows, d);
+                                                y_out, (bf16*)yb, yb_ps, rows, d);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -761,12 +723,12 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
   } else {
     const int row_bytes = a.head_dim * a.esize;
     const int ppr = row_bytes / 16;                                    // 16-byte pieces per row
-    const long long units = (long long)a.n_layers * 2 * a.n_heads * ppr;
+    const long long units = (long long)a.n_layers * 2 * a.kv_planes * a.n_heads * ppr;
     for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += (long long)gridDim.x * blockDim.x) {
       int piece = (int)(u % ppr);
       long long t = u / ppr;
       int head = (int)(t % a.n_heads);
-      long long lk = t / a.n_heads;                                    // layer*2 + kv
+      long long lk = t / a.n_heads;                                    // (layer*2 + kv)*planes + plane
       char* base = (char*)a.kv_base + ((((size_t)lk * a.max_batch + b) * a.n_heads + head) * a.max_seq) * row_bytes;
       for (int k = 1; k <= n; ++k) {
         int src = s_path[k];
@@ -809,7 +771,7 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
   }
 }
 hydra_status accept_compact(const AcceptArgs& a, cudaStream_t st) {
-  long long units = (long long)a.n_layers * 2 * a.n_heads * (a.head_dim * a.esize / 16);
+  long long units = (long long)a.n_layers * 2 * a.kv_planes * a.n_heads * (a.head_dim * a.esize / 16);
   int G = (int)((units + 255) / 256);
   int cap = (148 * 4 + a.batch - 1) / a.batch;
   if (G > cap) G = cap;
@@ -912,16 +874,16 @@ hydra_status apply_plant(int* tree_tok, const int* plant, int count, cudaStream_
 }
 
 template <typename T>
-__global__ void cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t count) {
+__global__ void cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t dst_ps, size_t count) {
   pdl_trigger();
   pdl_wait();
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < count) dst[i] = from_f<T>(src[i]);
+  if (i < count) put<T>(dst + i, dst_ps, src[i]);
 }
-hydra_status cast_rows(const float* src, void* dst, size_t count, int dtype, cudaStream_t st) {
+hydra_status cast_rows(const float* src, void* dst, size_t dst_ps, size_t count, int dtype, cudaStream_t st) {
   unsigned grid = (unsigned)((count + 255) / 256);
-  if (dtype == 0) launch_pdl(cast_rows_kernel<float>, dim3(grid), dim3(256), 0, st, src, (float*)dst, count);
-  else launch_pdl(cast_rows_kernel<bf16>, dim3(grid), dim3(256), 0, st, src, (bf16*)dst, count);
+  if (dtype == 0) launch_pdl(cast_rows_kernel<float>, dim3(grid), dim3(256), 0, st, src, (float*)dst, dst_ps, count);
+  else launch_pdl(cast_rows_kernel<bf16>, dim3(grid), dim3(256), 0, st, src, (bf16*)dst, dst_ps, count);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }

@@ -7,26 +7,9 @@ namespace hydra {
 // ---- GEMM: partial sums of x[m][k] * w[n][k] (see SplitDesc for where they land)
 // tcgen05 path (bfloat16 operands).  x_rows_alloc = rows the x buffer really holds (>= m); rows of the last
 // tile beyond m are computed and dropped.  part needs gemm_tc_plan(...)'s max_slots * m * n floats.
-// Optional fused consumer: the CTA that completes a tile adds its slots and applies one of these right away.
-enum { EPI_PARTIAL = 0,   // none: the caller's next kernel reduces the slots
-       EPI_OUT = 1,       // out[m][n] = sum * inv_rms[m]
-       EPI_RESID = 2,     // x += sum; xg = bf16(x * gain[n]); ss_out[n_tile][m] = sum over the tile of x^2
-       EPI_GATEUP = 3,    // act[m][c] = bf16(silu(g) * u), g/u = scaled sums of gate tile c/128 and up tile (f + c)/128
-       EPI_QKV = 4 };     // rotate q,k (table), q -> q_out, k,v -> cache rows pos0[b]+i; all scaled by inv_rms[m]
-struct GemmEpilogue {
-  int kind = EPI_PARTIAL;
-  unsigned int* counters = nullptr;                 // device, one per tile, zero at rest (the kernel restores zero)
-  // RMSNorm factor of the operand rows: inv_rms[m] = rsqrt(sum_t ss_in[t*ss_ld + m] * inv_d + eps); null = 1
-  const float* ss_in = nullptr; int ss_in_tiles = 0; int ss_ld = 0; float inv_d = 0.f, eps = 0.f;
-  RowSet rs{}; const float2* rope = nullptr; void* q_out = nullptr; void* kc = nullptr; void* vc = nullptr;
-  int H = 0, hd = 0, max_seq = 0;
-  float* x = nullptr; void* xg = nullptr; const void* gain = nullptr; float* ss_out = nullptr;
-  void* act = nullptr; int f = 0;
-  float* out = nullptr;
-  long long* trace = nullptr;                       // optional [grid][8] per-CTA phase timestamps in ns (tuning aid)
-};
-hydra_status gemm_tc(const bf16* x, int x_rows_alloc, const bf16* w, float* part, int m, int n, int k, SplitDesc* sd_out,
-                     const GemmEpilogue* epi, int* status, cudaStream_t st);
+// x holds x_planes (1 or 2) planes of x_rows_alloc rows each: plane 0 = bf16(v), plane 1 = bf16(v - plane 0).
+hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* w, float* part, int m, int n, int k,
+                     SplitDesc* sd_out, int* status, long long* trace, cudaStream_t st);
 SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots);
 int gemm_tile_rows(int m);                // activation rows per MMA tile for an m-row GEMM: 16, 32, 64, 128 or 256
 bool gemm_tc_available();                 // driver entry point for tensor-map encoding found
@@ -41,27 +24,24 @@ hydra_status embed_rows(const void* embed, const int* tok, float* x, int rows, i
 // x_out = (res ? res : 0) + sum_s part[s]; if gain: xn = rmsnorm(x_out)*gain (act dtype, optional) and hn = the same in
 // float (optional).  part may be null.  x_out may alias res.
 hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd, float* x_out,
-                              const void* gain, void* xn, float* hn, int rows, int d, float eps, int dtype,
+                              const void* gain, void* xn, size_t xn_ps, float* hn, int rows, int d, float eps, int dtype,
                               cudaStream_t st);
-// Fused (bfloat16) layer stack: rows entering it and the normalised hidden rows leaving it (see GemmEpilogue).
-hydra_status rows_prepare(const float* src, const void* embed, const int* tok, int vocab, const void* gain, float* x, void* xg,
-                          float* ss, int rows, int d, int* status, cudaStream_t st);
-hydra_status finalize_hidden(const float* x, const float* ss, int ss_tiles, int ld, const void* gain, float eps, float* h,
-                             int rows, int d, cudaStream_t st);
 // table[r][j] = (cos, sin) of (pos0[b]+depth[i]) * theta^(-2j/head_dim), evaluated in double
 hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st);
 // q (operand dtype, [rows][H][hd], rotated), K/V cache rows (rotated K) from the QKV partial sums.
-hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q,
-                            void* kcache, void* vcache, RowSet rs, int n_heads, int head_dim, int max_seq, int dtype,
+hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, size_t q_ps,
+                            void* kcache, void* vcache, size_t kv_ps, RowSet rs, int n_heads, int head_dim, int max_seq, int dtype,
                             int* status, cudaStream_t st);
 constexpr int ATT_CHUNK_ROWS = 128;     // KV rows per attention CTA (split-KV granularity)
 size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
 // bfloat16 caches: tensor-core kernel (attention_tc.cu); float caches: SIMT kernel.  q is in the cache dtype.
-hydra_status tree_attention_tc(const bf16* q, const bf16* kc, const bf16* vc, RowSet rs, bf16* out, void* scratch, int n_heads,
-                               int head_dim, int max_seq, int len_upper, cudaStream_t st);
-hydra_status tree_attention(const void* q, const void* kcache, const void* vcache, RowSet rs, void* out, void* scratch,
-                            int n_heads, int head_dim, int max_seq, int len_upper, int dtype, cudaStream_t st);
-hydra_status silu_mul(const float* part, SplitDesc sd, void* act, int rows, int f, int dtype,
+// "_ps" arguments: element distance between the hi and lo planes of a bfloat16 operand (0 = hi only; unused for float).
+hydra_status tree_attention_tc(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out,
+                               size_t out_ps, void* scratch, int n_heads, int head_dim, int max_seq, int len_upper, cudaStream_t st);
+hydra_status tree_attention(const void* q, size_t q_ps, const void* kcache, const void* vcache, size_t kv_ps, RowSet rs, void* out,
+                            size_t out_ps, void* scratch, int n_heads, int head_dim, int max_seq, int len_upper, int dtype,
+                            cudaStream_t st);
+hydra_status silu_mul(const float* part, SplitDesc sd, void* act, size_t act_ps, int rows, int f, int dtype,
                       cudaStream_t st);
 // amax[r] = argmax_v of the summed partial logits (lowest id among equal maxima); the sums go to logits_out if given
 // scratch: topk_scratch_bytes(rows_cap, vocab) bytes of candidate storage
@@ -76,11 +56,11 @@ struct LevelDesc {           // one tree level d (1-based): the parents that hav
 };
 // z[b*P+j] = [hprime[b] ; E[tok[b][path(parent j)]]] in act dtype; also tree_tok[b][0] = root_tok[b] when d == 1.
 hydra_status head_gather(const float* hprime, const void* embed, const int* root_tok, int* tree_tok, const int* path_tab,
-                         LevelDesc lv, void* z, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
+                         LevelDesc lv, void* z, size_t z_ps, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
                          cudaStream_t st);
 // y_out = res + silu(sum_s part[s] + bias); res row = hprime[b] when res_is_hprime else y row.  yb = act-dtype copy.
 hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, SplitDesc sd,
-                      const void* bias, float* y_out, void* yb, int rows, int d, int dtype, cudaStream_t st);
+                      const void* bias, float* y_out, void* yb, size_t yb_ps, int rows, int d, int dtype, cudaStream_t st);
 // children of parent j of sequence b = top n_child tokens of logits row b*P+j, descending (ties: lower id first);
 // the logits are the summed partials, also written to `logits` [rows][vocab]
 hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, int max_children, const int* first_child,
@@ -91,7 +71,7 @@ hydra_status topk_children(const float* part, SplitDesc sd, float* logits, Level
 struct AcceptArgs {
   const int* tree_tok; const int* amax;
   const int* parent; const int* depth; const uint64_t* anc;
-  int T, K, batch, n_layers, n_heads, head_dim, max_seq, max_batch, d_model, esize;
+  int T, K, batch, n_layers, n_heads, head_dim, max_seq, max_batch, d_model, esize, kv_planes;
   void* kv_base; const float* h_tree; int h_tree_stride;   // h_tree row = b*h_tree_stride + i
   float* h_new; int* n_new; int* len; int* root_tok;
   int* n_acc; int* path; int* out_tok; unsigned int* done_counter; int* status;
@@ -111,7 +91,7 @@ hydra_status prefix_rowset(const int* len, const int* n_new, int* pos0, int* n_r
 hydra_status pick_last_row(const float* x, const int* n_rows, int tc, float* hprime, int batch, int d, cudaStream_t st);
 hydra_status apply_plant(int* tree_tok, const int* plant, int count, cudaStream_t st);
 // dst = src converted to the operand type
-hydra_status cast_rows(const float* src, void* dst, size_t count, int dtype, cudaStream_t st);
+hydra_status cast_rows(const float* src, void* dst, size_t dst_ps, size_t count, int dtype, cudaStream_t st);
 hydra_status copy_i32(int* dst, const int* src, int count, cudaStream_t st);
 
 }  // namespace hydra

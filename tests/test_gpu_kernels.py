@@ -29,6 +29,20 @@ def test_gemm_tensor_core_matches_definition(m, n, k):
     assert float((simt - ref).abs().max()) <= tol
 
 
+@pytest.mark.parametrize("m,n,k", [(64, 512, 4096), (11, 256, 1280), (300, 384, 704)])
+def test_gemm_hi_lo_activation_planes(m, n, k):
+    """Float activations passed as hi/lo bfloat16 planes: the product must match the float activations to ~2^-16."""
+    from paper_2402_05109_b200 import gemm, split_hi_lo
+    x = rnd((m, k), 15, m + k, torch.float32)
+    w = rnd((n, k), 16, n + k, torch.bfloat16, 0.02)
+    ref = x.double() @ w.double().T
+    out = gemm(split_hi_lo(x.cuda()), w.cuda(), mode=0).cpu().double()
+    scale = float(ref.abs().max())
+    assert float((out - ref).abs().max()) <= 3e-5 * scale
+    single = gemm(x.to(torch.bfloat16).cuda(), w.cuda(), mode=0).cpu().double()
+    assert float((single - ref).abs().max()) > 10 * float((out - ref).abs().max())       # the lo plane matters
+
+
 @pytest.mark.parametrize("m,n,k", [(16, 768, 256), (7, 1376, 256), (16, 256, 688), (4, 1024, 1024)])
 def test_gemm_float(m, n, k):
     from paper_2402_05109_b200 import gemm
@@ -39,26 +53,30 @@ def test_gemm_float(m, n, k):
     assert float((out - ref).abs().max()) <= 1e-5 * float(ref.abs().max()) + 1e-6
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("dtype,planes", [(torch.float32, 1), (torch.bfloat16, 1), (torch.bfloat16, 2)])
 @pytest.mark.parametrize("hd", [64, 128])
-def test_tree_attention_matches_masked_softmax(dtype, hd):
-    from paper_2402_05109_b200 import tree_attention
+def test_tree_attention_matches_masked_softmax(dtype, planes, hd):
+    from paper_2402_05109_b200 import tree_attention, split_hi_lo
     parent = load_tree("tree63_d4")
     t = TreeTables(parent)
     B, H, S, tc = 3, 3, 700, t.T
     pos0 = [0, 333, 600]                    # empty cache, a cache spanning several KV chunks with a ragged tail, long
     n_rows = [tc, tc, 17]                   # ragged row counts (rows beyond n_rows are ignored)
-    kc = rnd((B, H, S, hd), 21, 1, dtype)
-    vc = rnd((B, H, S, hd), 21, 2, dtype)
-    q = rnd((B * tc, H, hd), 21, 3, dtype)
+    src = torch.float32 if planes == 2 else dtype
+    kc = rnd((B, H, S, hd), 21, 1, src)
+    vc = rnd((B, H, S, hd), 21, 2, src)
+    q = rnd((B * tc, H, hd), 21, 3, src)
+    dev = (lambda x: split_hi_lo(x.cuda())) if planes == 2 else (lambda x: x.cuda())
     mask = torch.tensor([a - (1 << 64) if a >= (1 << 63) else a for a in t.anc_mask], dtype=torch.int64)
-    out = tree_attention(q.cuda(), kc.cuda(), vc.cuda(), torch.tensor(pos0, dtype=torch.int32).cuda(),
-                         torch.tensor(n_rows, dtype=torch.int32).cuda(), mask.cuda(), tc).float().cpu().view(B, tc, H, hd)
+    out = tree_attention(dev(q), dev(kc), dev(vc), torch.tensor(pos0, dtype=torch.int32).cuda(),
+                         torch.tensor(n_rows, dtype=torch.int32).cuda(), mask.cuda(), tc).float().cpu()
+    out = (out.sum(0) if planes == 2 else out).view(B, tc, H, hd)
     for b in range(B):
         n, L = n_rows[b], pos0[b] + n_rows[b]
         allowed = torch.cat([torch.ones(n, pos0[b], dtype=torch.bool), t.allowed[:n, :n]], dim=1)
         k = kc[b, :, :L].permute(1, 0, 2).double()
         v = vc[b, :, :L].permute(1, 0, 2).double()
-        ref = masked_attention(q.view(B, tc, H, hd)[b, :n].double(), k, v, allowed)   # q, k, v hold the rounded values
+        ref = masked_attention(q.view(B, tc, H, hd)[b, :n].double(), k, v, allowed)   # q, k, v hold the stored values
         err = float((out[b, :n].double() - ref).abs().max())
-        assert err <= (2e-5 if dtype == torch.float32 else 2e-2), err
+        tol = 2e-5 if dtype == torch.float32 else (2e-4 if planes == 2 else 2e-2)
+        assert err <= tol, err

@@ -43,9 +43,9 @@ def test_small_bf16_hydrapp_ragged_batch():
     assert seen >= {0, 1, 2, 3, 4}, seen
 
 
-@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("mode", [1])
 def test_small_bf16_other_gemm_modes_and_root_only_tree(mode):
-    """mode 1: SIMT GEMM; mode 2: tensor-core GEMM with the consumer operations fused into its epilogues."""
+    """mode 1: the SIMT GEMM (reads only the hi plane of the activations)."""
     from paper_2402_05109_b200 import Hydra
     m = ModelCfg(2, 256, 4, 64, 512, 1024, dtype="bf16")
     h = HeadCfg(2, 1, False)
