@@ -38,7 +38,8 @@ def verify_bytes(m, B, T, lens):
     s = 2 if m.dtype == "bf16" else 4
     d, f = m.d_model, m.d_ffn
     w = s * (m.n_layers * (4 * d * d + 3 * d * f) + m.vocab * d)
-    kv = sum(2 * m.n_layers * d * s * (L + T) for L in lens) + B * T * 2 * m.n_layers * d * s
+    skv = 4                      # cache element: float, or two bfloat16 planes (hi + lo)
+    kv = sum(2 * m.n_layers * d * skv * (L + T) for L in lens) + B * T * 2 * m.n_layers * d * skv
     return w + kv
 
 
@@ -47,7 +48,7 @@ def draft_bytes(m, h, lens):
     d, f = m.d_model, m.d_ffn
     heads = sum(((i + 1) + (h.n_mlp_layers - 1)) * d * d for i in range(1, h.n_heads + 1)) + h.n_heads * m.vocab * d
     pfx = (4 * d * d + 3 * d * f) if h.prefix_attn else 0
-    return s * (heads + pfx) + (sum(2 * d * s * L for L in lens) if h.prefix_attn else 0)
+    return s * (heads + pfx) + (sum(2 * d * 4 * L for L in lens) if h.prefix_attn else 0)
 
 
 class ClockSampler:
