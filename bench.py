@@ -166,6 +166,14 @@ def oracle_sample(cfg, weights_cpu, parent, n_steps, threads):
     return per_step
 
 
+def workload_name(cfg, parent):
+    m, h = cfg.model, cfg.head
+    return ("%s: %d-layer d=%d Llama-shape decoder, %d Hydra heads x %d MLP layers, prefix layer=%s, %d-row tree "
+            "(root + %d candidates), batch %d, prompts %s, accept-exercise planting"
+            % (cfg.name, m.n_layers, m.d_model, h.n_heads, h.n_mlp_layers, h.prefix_attn, len(parent), len(parent) - 1,
+               cfg.batch, cfg.prompt_lens))
+
+
 def run_reference(args, cfg, parent):
     """Reference arm: the CPU oracle timed on the host cores (a deliberately plain program)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -184,7 +192,7 @@ def run_reference(args, cfg, parent):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": {"workload": cfg.name},
+        "dtype": "f32", "data": "synthetic", "config": {"workload": workload_name(cfg, parent)},
         "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
@@ -388,10 +396,7 @@ def main():
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if m.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": "%s: %d-layer d=%d Llama-shape decoder, %d Hydra heads x %d MLP layers, prefix layer=%s, "
-                               "%d-row tree (root + %d candidates), batch %d, prompts %s, accept-exercise planting"
-                               % (cfg.name, m.n_layers, m.d_model, K, h.n_mlp_layers, h.prefix_attn, T, T - 1, B,
-                                  cfg.prompt_lens),
+        "config": {"workload": workload_name(cfg, parent),
                    "l2": "every step streams %.1f GB of weights, far above the 126 MB L2; no flush needed" % (vbytes / 1e9),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "verify_ms": t_verify, "draft_ms": t_draft, "accept_compact_ms": t_accept,
