@@ -150,10 +150,15 @@ struct GemmArgs {
   int m, n, kb, n_tiles, total_units, q;
   int x_lo_rows;                 // row offset of the lo plane inside the activation tensor map (0: single plane)
   int* status;
+  int* diag;                     // optional int[8]: where the first bounded wait gave up (site, cta, unit, units, grid, m, n, kb)
   long long* trace;              // optional [grid][8] nanosecond timestamps of each CTA's phases (tuning aid), or null
 };
 
 __device__ __forceinline__ long long global_ns() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+// Records the first wait that ran out (site: 1 producer/empty, 2 mma/acc-empty, 3 mma/full-w, 4 mma/full-x, 5 epilogue/acc-full).
+#define GIVE_UP(site, unit) do { atomicOr(a.status, ST_TIMEOUT); \
+    if (a.diag && atomicCAS(a.diag, 0, (site)) == 0) { a.diag[1] = blockIdx.x; a.diag[2] = (unit); a.diag[3] = n_units; \
+      a.diag[4] = gridDim.x; a.diag[5] = a.m; a.diag[6] = a.n; a.diag[7] = a.kb; } } while (0)
 #define TRACE(slot) do { if (a.trace) a.trace[blockIdx.x * 8 + (slot)] = global_ns(); } while (0)
 
 template <int MT, int BUDGET_KB>
@@ -220,7 +225,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         coords(u_begin + i, kcol, nrow, mrow);
         const uint32_t a_dst = tiles + s * C::STAGE_BYTES;
         if (i >= pre) {
-          if (!mbar_wait(empty_bar(s), ph ^ 1u)) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
+          if (!mbar_wait(empty_bar(s), ph ^ 1u)) { GIVE_UP(1, i); s_abort = 1; break; }
           mbar_arrive_expect_tx(fullw_bar(s), A_BYTES);
           tma_load_2d(a_dst, &tmW, kcol, nrow, fullw_bar(s), pol_w);
         }
@@ -240,13 +245,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int seg_len = min((tile + 1) * a.kb, u_end) - u;
         const int acc = seg & 1;
         const uint32_t acc_ph = (seg >> 1) & 1;
-        if (!mbar_wait(accempty_bar(acc), acc_ph ^ 1u)) { ok = false; break; }      // epilogue has drained this buffer
+        if (!mbar_wait(accempty_bar(acc), acc_ph ^ 1u)) { GIVE_UP(2, i); ok = false; break; }      // epilogue has drained this buffer
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * C::ACC_COLS);
         for (int j = 0; j < seg_len; ++j, ++i) {
           const int s = i % C::STAGES;
           const uint32_t ph = (i / C::STAGES) & 1;
-          if (!mbar_wait(fullw_bar(s), ph) || !mbar_wait(fullx_bar(s), ph)) { ok = false; break; }
+          if (!mbar_wait(fullw_bar(s), ph)) { GIVE_UP(3, i); ok = false; break; }
+          if (!mbar_wait(fullx_bar(s), ph)) { GIVE_UP(4, i); ok = false; break; }
           if (i == 0) TRACE(3);
           tc_fence_after();
           const uint32_t a_addr = tiles + s * C::STAGE_BYTES;
@@ -280,7 +286,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int seg_len = min((tile + 1) * a.kb, u_end) - u;
       const int acc = seg & 1;
       const uint32_t acc_ph = (seg >> 1) & 1;
-      if (!mbar_wait(accfull_bar(acc), acc_ph)) { if (lane == 0) atomicOr(a.status, ST_TIMEOUT); break; }
+      if (!mbar_wait(accfull_bar(acc), acc_ph)) { if (lane == 0) GIVE_UP(5, i); break; }
       if (epi_tid == 0 && i + seg_len >= n_units) TRACE(5);
       tc_fence_after();
       const int slot = blockIdx.x - (int)(((long long)tile * a.kb) / a.q);
@@ -423,7 +429,7 @@ SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots) {
 }
 
 hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* w, float* part, int m, int n, int k,
-                     SplitDesc* sd_out, int* status, long long* trace, cudaStream_t st) {
+                     SplitDesc* sd_out, int* status, int* diag, long long* trace, cudaStream_t st) {
   if (m <= 0 || n <= 0 || k <= 0 || n % BLOCK_N || k % BLOCK_K || (x_planes != 1 && x_planes != 2)) return HYDRA_ERR_UNSUPPORTED;
   if (((uintptr_t)x | (uintptr_t)w) & 15) return HYDRA_ERR_INVALID;
   int grid = 1;
@@ -438,7 +444,7 @@ hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* 
   GemmArgs a{};
   a.part = part; a.slot_stride = sd.stride; a.m = m; a.n = n; a.kb = sd.kb; a.n_tiles = sd.n_tiles;
   a.total_units = sd.n_tiles * ((m + sd.mt - 1) / sd.mt) * sd.kb; a.q = sd.q; a.status = status;
-  a.x_lo_rows = x_planes == 2 ? x_rows_alloc : 0; a.trace = trace;
+  a.x_lo_rows = x_planes == 2 ? x_rows_alloc : 0; a.diag = diag; a.trace = trace;
   if (sd_out) *sd_out = sd;
   switch (sd.mt) {
     case 16: return launch<16>(tw, tx, a, grid, st);

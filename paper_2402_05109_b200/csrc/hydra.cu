@@ -183,7 +183,8 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   std::vector<int*> lvl;
   for (auto& lv : t.level_parents) lvl.push_back(b.take<int>(lv.size()));
   auto* len = b.take<int>(m.max_batch); auto* n_new = b.take<int>(m.max_batch); auto* root = b.take<int>(m.max_batch);
-  auto* status = b.take<int>(1); auto* pos0 = b.take<int>(m.max_batch); auto* nrows = b.take<int>(m.max_batch);
+  auto* status = b.take<int>(16);          // [0] status word, [8..15] where a bounded wait gave up
+  auto* pos0 = b.take<int>(m.max_batch); auto* nrows = b.take<int>(m.max_batch);
   auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
   auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
   auto* done = b.take<unsigned int>(m.max_batch);
@@ -236,7 +237,7 @@ hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void*
     int slots = 1;
     gemm_tc_plan(m, n, k, nullptr, &slots);
     if ((size_t)slots * m * n > c->part_floats) return HYDRA_ERR_CAPACITY;
-    return gemm_tc((const bf16*)x, x_rows_alloc, c->planes, (const bf16*)w, c->part, m, n, k, sd, c->d_status, nullptr, st);
+    return gemm_tc((const bf16*)x, x_rows_alloc, c->planes, (const bf16*)w, c->part, m, n, k, sd, c->d_status, c->d_status + 8, nullptr, st);
   }
   *sd = single_slot((size_t)m * n);
   return gemm_simt(x, w, c->part, m, n, k, c->m.dtype, st);      // bfloat16: the hi plane only (debug mode)
@@ -614,7 +615,12 @@ hydra_status hydra_poll_status(hydra_ctx* c, void* stream) {
   int word = 0;
   HYDRA_CUDA(cudaStreamSynchronize(st));
   HYDRA_CUDA(cudaMemcpy(&word, c->d_status, sizeof(int), cudaMemcpyDeviceToHost));
-  if (word) HYDRA_CUDA(cudaMemset(c->d_status, 0, sizeof(int)));
+  if (word & ST_TIMEOUT) {
+    int d[8] = {0};
+    cudaMemcpy(d, c->d_status + 8, sizeof(d), cudaMemcpyDeviceToHost);
+    snprintf(g_err, sizeof(g_err), "GEMM wait gave up: site %d cta %d unit %d/%d grid %d m %d n %d kb %d", d[0], d[1], d[2], d[3], d[4], d[5], d[6], d[7]);
+  }
+  if (word) HYDRA_CUDA(cudaMemset(c->d_status, 0, 16 * sizeof(int)));
   if (word & ST_TIMEOUT) return HYDRA_ERR_TIMEOUT;
   if (word & ST_BOUNDS) return HYDRA_ERR_BOUNDS;
   return HYDRA_OK;
@@ -688,7 +694,7 @@ hydra_status hydra_gemm(const void* x, const void* w, float* out, float* partial
     if (!status) return HYDRA_ERR_INVALID;
     if (!gemm_tc_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
     SplitDesc sd;
-    HYDRA_TRY(gemm_tc((const bf16*)x, m, x_planes, (const bf16*)w, partial, m, n, k, &sd, status, nullptr, st));
+    HYDRA_TRY(gemm_tc((const bf16*)x, m, x_planes, (const bf16*)w, partial, m, n, k, &sd, status, nullptr, nullptr, st));
     return reduce_splits(partial, sd, out, m, n, st);
   }
   return gemm_simt(x, w, out, m, n, k, dtype, st);

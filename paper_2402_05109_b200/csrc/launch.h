@@ -9,7 +9,7 @@ namespace hydra {
 // tile beyond m are computed and dropped.  part needs gemm_tc_plan(...)'s max_slots * m * n floats.
 // x holds x_planes (1 or 2) planes of x_rows_alloc rows each: plane 0 = bf16(v), plane 1 = bf16(v - plane 0).
 hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* w, float* part, int m, int n, int k,
-                     SplitDesc* sd_out, int* status, long long* trace, cudaStream_t st);
+                     SplitDesc* sd_out, int* status, int* diag /*int[8] or null*/, long long* trace, cudaStream_t st);
 SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots);
 int gemm_tile_rows(int m);                // activation rows per MMA tile for an m-row GEMM: 16, 32, 64, 128 or 256
 bool gemm_tc_available();                 // driver entry point for tensor-map encoding found

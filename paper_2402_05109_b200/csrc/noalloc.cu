@@ -46,6 +46,6 @@ extern "C" hydra_status hydra_gemm_noalloc(const void* x, const void* w, float* 
   float* part = g_scratch_ptr[dev];
   // every partial element the reduction reads is written by the GEMM first, so nothing has to be cleared
   SplitDesc sd;
-  HYDRA_TRY(gemm_tc((const bf16*)x, m, 1, (const bf16*)w, part, m, n, k, &sd, status, nullptr, st));
+  HYDRA_TRY(gemm_tc((const bf16*)x, m, 1, (const bf16*)w, part, m, n, k, &sd, status, nullptr, nullptr, st));
   return reduce_splits(part, sd, out, m, n, st);
 }
