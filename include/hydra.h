@@ -89,7 +89,8 @@ typedef struct {
 size_t hydra_workspace_bytes(const hydra_model_cfg*, const hydra_head_cfg*, const hydra_tree_cfg*);
 
 /* Validate the configs, build and upload the tree tables (depth, ancestor bitmask, paths, levels),
- * carve the workspace (256-byte aligned; it is cleared by this call). */
+ * carve the workspace (256-byte aligned; it is cleared by this call).  Synchronises the whole device before
+ * and after, so the workspace may be memory that earlier work on any stream was still using. */
 hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg*, const hydra_head_cfg*, const hydra_tree_cfg*,
                           const hydra_weights*, void* workspace_dev, size_t workspace_bytes);
 hydra_status hydra_destroy(hydra_ctx*);

@@ -442,6 +442,8 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
   // clear the workspace, upload the static tables
   auto fail = [&](cudaError_t e, const char* what) { set_last_error(what, e); delete c; return HYDRA_ERR_CUDA; };
   cudaError_t e;
+  // the workspace may be memory that work still queued on some (non-blocking) stream is using: drain the device first
+  if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "cudaDeviceSynchronize");
   if ((e = cudaMemset(ws, 0, need)) != cudaSuccess) return fail(e, "cudaMemset(workspace)");
   const int T = th.T, K = h->n_heads;
   std::vector<int> chain_depth(CHUNK); std::vector<uint64_t> chain_mask(CHUNK);
