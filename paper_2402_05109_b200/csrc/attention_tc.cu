@@ -11,12 +11,12 @@
 // softmax weights are split the same way before the P V product.  A plane distance of 0 selects hi-only operands.
 #include "launch.h"
 #include <math.h>
+#include <cstdlib>
 
 namespace hydra {
 
 namespace {
 
-constexpr int TILE = 64;           // KV rows per pipeline stage
 constexpr int NWARP = 4;           // 16 query rows each
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -41,7 +41,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int HD, bool HL>
+template <int HD, bool HL, int TILE>
 __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __restrict__ q, size_t q_ps, const bf16* __restrict__ kc,
                                                                   const bf16* __restrict__ vc, size_t kv_ps, RowSet rs,
                                                                   float* __restrict__ part_o, float* __restrict__ part_ml,
@@ -261,8 +261,8 @@ __global__ void __launch_bounds__(HD) tree_attn_tc_combine_kernel(const float* _
   if (out_ps) dst[out_ps + k] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
-template <int HD, bool HL>
-hydra_status run(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
+template <int HD, bool HL, int TILE>
+hydra_status run_t(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
                  float* scratch, int H, int max_seq, int len_upper, int chunk, cudaStream_t st) {
   const int nchunks_max = (max_seq + chunk - 1) / chunk;
   int nchunks = (len_upper + chunk - 1) / chunk;
@@ -275,16 +275,25 @@ hydra_status run(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, siz
   const size_t smem = (size_t)NP * (64 + 4 * TILE) * LDS * sizeof(bf16);
   static bool attr_done = false;
   if (!attr_done) {
-    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_done = true;
   }
-  launch_pdl(tree_attn_tc_kernel<HD, HL>, dim3(H, rs.batch, nchunks), dim3(NWARP * 32), smem, st, q, q_ps, kc, vc, kv_ps, rs, part_o, part_ml, H,
+  launch_pdl(tree_attn_tc_kernel<HD, HL, TILE>, dim3(H, rs.batch, nchunks), dim3(NWARP * 32), smem, st, q, q_ps, kc, vc, kv_ps, rs, part_o, part_ml, H,
              max_seq, nchunks, chunk);
   HYDRA_LAUNCH_CHECK();
   launch_pdl(tree_attn_tc_combine_kernel<HD>, dim3((unsigned)rows, H), dim3(HD), 0, st, (const float*)part_o, (const float*)part_ml, rs, out, out_ps, H,
              nchunks, chunk);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
+}
+
+// KV rows per pipeline stage: 32 lets two CTAs share an SM with two-plane operands (HYDRA_ATT_TILE=64: one CTA, fewer syncs).
+template <int HD, bool HL>
+hydra_status run(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
+                 float* scratch, int H, int max_seq, int len_upper, int chunk, cudaStream_t st) {
+  static const int tile = []() { const char* e = getenv("HYDRA_ATT_TILE"); return e ? atoi(e) : 32; }();
+  if (tile == 64) return run_t<HD, HL, 64>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, chunk, st);
+  return run_t<HD, HL, 32>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, chunk, st);
 }
 
 }  // namespace
