@@ -215,53 +215,73 @@ hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cud
   return HYDRA_OK;
 }
 
+// One thread rotates four consecutive pairs (j..j+3, j+half..j+half+3) of one head of q and k and copies the
+// matching v elements; all loads and stores are 16 bytes wide.
 template <typename T>
-__global__ void __launch_bounds__(64) qkv_rope_store_kernel(const float* __restrict__ part, SplitDesc sd,
-                                                            const float2* __restrict__ table, T* __restrict__ q,
-                                                            size_t q_ps, T* __restrict__ kc, T* __restrict__ vc,
-                                                            size_t kv_ps, RowSet rs, int H, int hd, int max_seq,
-                                                            int* status) {
+__global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __restrict__ part, SplitDesc sd,
+                                                             const float2* __restrict__ table, T* __restrict__ q,
+                                                             size_t q_ps, T* __restrict__ kc, T* __restrict__ vc,
+                                                             size_t kv_ps, RowSet rs, int H, int hd, int max_seq,
+                                                             int* status) {
   pdl_trigger();
   pdl_wait();
-  const int r = blockIdx.x, h = blockIdx.y, b = r / rs.tc, i = r % rs.tc;
+  const int r = blockIdx.x, b = r / rs.tc, i = r % rs.tc;
   const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
   if (i >= nr) return;
   const int d = H * hd, half = hd >> 1;
   const int slot = rs.pos0[b] + i;
-  if (slot < 0 || slot >= max_seq) { if (threadIdx.x == 0 && h == 0) atomicOr(status, ST_BOUNDS); return; }
-  const int j = threadIdx.x;                                       // rotation pair (j, j + half) of this head
-  if (j >= half) return;
+  if (slot < 0 || slot >= max_seq) { if (threadIdx.x == 0 && blockIdx.y == 0) atomicOr(status, ST_BOUNDS); return; }
+  const int tph = half >> 2;                                       // threads per head
+  const int h = blockIdx.y * (256 / tph) + threadIdx.x / tph;
+  if (h >= H) return;
+  const int j = (threadIdx.x % tph) * 4;
   const float* p0 = part + (size_t)r * 3 * d;
   const int c0 = h * hd + j, c1 = c0 + half;
-  float v6[6];
   const int cols[6] = {c0, c1, d + c0, d + c1, 2 * d + c0, 2 * d + c1};
+  float4 v6[6];
 #pragma unroll
   for (int e = 0; e < 6; ++e) {
     const int ns = split_count(sd, r, cols[e]);
-    float acc = 0.f;
-    for (int s = 0; s < ns; ++s) acc += p0[s * sd.stride + cols[e]];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < ns; ++s) {
+      const float4 a = *reinterpret_cast<const float4*>(p0 + s * sd.stride + cols[e]);
+      acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+    }
     v6[e] = acc;
   }
-  const float qa = v6[0], qb = v6[1], ka = v6[2], kb = v6[3], va = v6[4], vb = v6[5];
-  const float2 cs = table[(size_t)r * half + j];
-  put<T>(q + (size_t)r * d + c0, q_ps, qa * cs.x - qb * cs.y);
-  put<T>(q + (size_t)r * d + c1, q_ps, qb * cs.x + qa * cs.y);
+  const float4 t01 = *reinterpret_cast<const float4*>(table + (size_t)r * half + j);        // (cos, sin) of j, j+1
+  const float4 t23 = *reinterpret_cast<const float4*>(table + (size_t)r * half + j + 2);    // (cos, sin) of j+2, j+3
+  const float cs[4] = {t01.x, t01.z, t23.x, t23.z}, sn[4] = {t01.y, t01.w, t23.y, t23.w};
+  auto rot = [&](const float4& a, const float4& bq, float4& lo, float4& hi) {
+    const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {bq.x, bq.y, bq.z, bq.w};
+    float l[4], hh[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { l[e] = av[e] * cs[e] - bv[e] * sn[e]; hh[e] = bv[e] * cs[e] + av[e] * sn[e]; }
+    lo = make_float4(l[0], l[1], l[2], l[3]); hi = make_float4(hh[0], hh[1], hh[2], hh[3]);
+  };
+  float4 qlo, qhi, klo, khi;
+  rot(v6[0], v6[1], qlo, qhi);
+  rot(v6[2], v6[3], klo, khi);
+  put4<T>(q + (size_t)r * d + c0, q_ps, qlo);
+  put4<T>(q + (size_t)r * d + c1, q_ps, qhi);
   const size_t o = (((size_t)b * H + h) * max_seq + slot) * hd;
-  put<T>(kc + o + j, kv_ps, ka * cs.x - kb * cs.y);
-  put<T>(kc + o + j + half, kv_ps, kb * cs.x + ka * cs.y);
-  put<T>(vc + o + j, kv_ps, va);
-  put<T>(vc + o + j + half, kv_ps, vb);
+  put4<T>(kc + o + j, kv_ps, klo);
+  put4<T>(kc + o + j + half, kv_ps, khi);
+  put4<T>(vc + o + j, kv_ps, v6[4]);
+  put4<T>(vc + o + j + half, kv_ps, v6[5]);
 }
 hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, size_t q_ps, void* kcache,
                             void* vcache, size_t kv_ps, RowSet rs, int H, int hd, int max_seq, int dtype, int* status,
                             cudaStream_t st) {
-  dim3 grid(rs.batch * rs.tc, H);
+  if (hd % 8) return HYDRA_ERR_UNSUPPORTED;
+  const int heads_per_block = 256 / (hd / 8);
+  dim3 grid(rs.batch * rs.tc, (H + heads_per_block - 1) / heads_per_block);
   if (dtype == 0)
-    launch_pdl(qkv_rope_store_kernel<float>, dim3(grid), dim3(64), 0, st, part, sd, table, (float*)q, q_ps, (float*)kcache, (float*)vcache,
-                                                      kv_ps, rs, H, hd, max_seq, status);
+    launch_pdl(qkv_rope_store_kernel<float>, grid, dim3(256), 0, st, part, sd, table, (float*)q, q_ps, (float*)kcache, (float*)vcache,
+               kv_ps, rs, H, hd, max_seq, status);
   else
-    launch_pdl(qkv_rope_store_kernel<bf16>, dim3(grid), dim3(64), 0, st, part, sd, table, (bf16*)q, q_ps, (bf16*)kcache, (bf16*)vcache, kv_ps, rs,
-                                                     H, hd, max_seq, status);
+    launch_pdl(qkv_rope_store_kernel<bf16>, grid, dim3(256), 0, st, part, sd, table, (bf16*)q, q_ps, (bf16*)kcache, (bf16*)vcache,
+               kv_ps, rs, H, hd, max_seq, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
