@@ -140,7 +140,11 @@ template <int MT, int BUDGET_KB> struct TileCfg {
   static constexpr int B_BYTES = 2 * B_PLANE;                    // hi + lo
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 10 ? 10 : ((SMEM_BUDGET / STAGE_BYTES) < 2 ? 2 : (SMEM_BUDGET / STAGE_BYTES));
-  static constexpr int ACC_COLS = MT < 32 ? 32 : MT;             // columns of one accumulator buffer
+  // Two planes, MT <= 128: the hi and lo activation tiles sit back to back in shared memory and form ONE MMA B
+  // operand of 2*MT rows, so each weight tile is read from shared memory once; accumulator columns [0, MT) hold
+  // W*hi, [MT, 2MT) hold W*lo and the epilogue adds them.  MT = 256: two accumulating passes over the weight tile.
+  static constexpr bool CAT = MT <= 128;
+  static constexpr int ACC_COLS = CAT ? (2 * MT < 32 ? 32 : 2 * MT) : MT;   // columns of one accumulator buffer
   static constexpr int TMEM_COLS = 2 * ACC_COLS;                  // two buffers (power of two, <= 512)
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/;
 };
@@ -148,6 +152,7 @@ template <int MT, int BUDGET_KB> struct TileCfg {
 struct GemmArgs {
   float* part; size_t slot_stride;
   int m, n, kb, n_tiles, total_units, q;
+  int flags;                     // bit 0: no L2 eviction hints on the TMA loads (tuning)
   int x_lo_rows;                 // row offset of the lo plane inside the activation tensor map (0: single plane)
   int* status;
   int* diag;                     // optional int[8]: where the first bounded wait gave up (site, cta, unit, units, grid, m, n, kb)
@@ -201,7 +206,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
   if (warp == 0) {
     if (lane == 0) {
-      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      if (a.flags & 1) { asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol_w)); pol_x = pol_w; }
       auto coords = [&](int u, int& kcol, int& nrow, int& mrow) {
         const int tile = u / a.kb;
         kcol = (u - tile * a.kb) * BLOCK_K;
@@ -236,7 +242,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(MT);
+      const bool cat = C::CAT && a.x_lo_rows != 0;
+      const uint32_t idesc = cat ? instr_desc(2 * MT) : instr_desc(MT);
       int seg = 0;
       bool ok = true;
       for (int i = 0; i < n_units && ok;) {
@@ -261,7 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
           for (int k = 0; k < BLOCK_K / 16; ++k)         // 16 bf16 = 32 bytes per MMA: +2 in 16-byte units
             umma_bf16(tmem_d, adesc + 2u * k, bdesc + 2u * k, idesc, (uint32_t)((j | k) != 0));
-          if (a.x_lo_rows) {                             // the low-order plane of the activations, same weights
+          if (a.x_lo_rows && !cat) {                     // the low-order plane of the activations, same weights
             const uint64_t ldesc = smem_desc_sw128(a_addr + A_BYTES + C::B_PLANE);
 #pragma unroll
             for (int k = 0; k < BLOCK_K / 16; ++k) umma_bf16(tmem_d, adesc + 2u * k, ldesc + 2u * k, idesc, 1u);
@@ -293,11 +300,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int n0 = (tile % a.n_tiles) * BLOCK_N, m0 = (tile / a.n_tiles) * MT;
       float* dst = a.part + (size_t)slot * a.slot_stride + n0 + epi_tid;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * C::ACC_COLS);
+      const bool cat = C::CAT && a.x_lo_rows != 0;
 #pragma unroll 1
       for (int c = 0; c < MT; c += 16) {
         if (m0 + c >= a.m) break;
         uint32_t r[16];
         tmem_ld16(taddr + (uint32_t)c, r);
+        if (cat) {                                       // add the W*lo columns
+          uint32_t r2[16];
+          tmem_ld16(taddr + (uint32_t)(MT + c), r2);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+        }
 #pragma unroll
         for (int j = 0; j < 16; ++j)
           if (m0 + c + j < a.m) dst[(size_t)(m0 + c + j) * a.n] = __uint_as_float(r[j]);
@@ -445,6 +459,7 @@ hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* 
   a.part = part; a.slot_stride = sd.stride; a.m = m; a.n = n; a.kb = sd.kb; a.n_tiles = sd.n_tiles;
   a.total_units = sd.n_tiles * ((m + sd.mt - 1) / sd.mt) * sd.kb; a.q = sd.q; a.status = status;
   a.x_lo_rows = x_planes == 2 ? x_rows_alloc : 0; a.diag = diag; a.trace = trace;
+  { static const int f = []() { const char* e = getenv("HYDRA_GEMM_NOHINT"); return e && e[0] == '1' ? 1 : 0; }(); a.flags = f; }
   if (sd_out) *sd_out = sd;
   switch (sd.mt) {
     case 16: return launch<16>(tw, tx, a, grid, st);
