@@ -194,6 +194,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
+    // weights do not depend on the preceding kernel: request the first ring of weight tiles right away, before the
+    // CTA-wide set-up (TMEM allocation, barrier hand-over) and before griddepcontrol.wait
+    const uint64_t pol_w0 = policy_evict_first();
+    const int pre0 = n_units < C::STAGES ? n_units : C::STAGES;
+    for (int i = 0; i < pre0; ++i) {
+      const int u = u_begin + i, tile = u / a.kb;
+      mbar_arrive_expect_tx(fullw_bar(i), A_BYTES);
+      tma_load_2d(tiles + i * C::STAGE_BYTES, &tmW, (u - tile * a.kb) * BLOCK_K, (tile % a.n_tiles) * BLOCK_N, fullw_bar(i), pol_w0);
+    }
   }
   if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
   tc_fence_before();
@@ -214,14 +223,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         nrow = (tile % a.n_tiles) * BLOCK_N;
         mrow = (tile / a.n_tiles) * MT;
       };
-      // weights do not depend on the preceding kernel: request the first ring of weight tiles right away
-      const int pre = n_units < C::STAGES ? n_units : C::STAGES;
-      for (int i = 0; i < pre; ++i) {
-        int kcol, nrow, mrow;
-        coords(u_begin + i, kcol, nrow, mrow);
-        mbar_arrive_expect_tx(fullw_bar(i), A_BYTES);
-        tma_load_2d(tiles + i * C::STAGE_BYTES, &tmW, kcol, nrow, fullw_bar(i), pol_w);
-      }
+      const int pre = n_units < C::STAGES ? n_units : C::STAGES;      // weight tiles already requested in the prologue
       TRACE(2);
       grid_dep_wait();                     // activations are the preceding kernel's output
       for (int i = 0; i < n_units; ++i) {
