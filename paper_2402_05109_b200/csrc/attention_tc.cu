@@ -1,11 +1,15 @@
 // Tree attention for bfloat16 caches on the tensor cores (mma.sync m16n8k16, float accumulate).
 //
-// One CTA per (head, sequence, KV chunk): the chunk's K and V rows are streamed once from HBM through a
-// double-buffered cp.async ring of 64-row tiles; the (at most 64) query rows of the call stay in registers
-// as MMA fragments, 16 rows per warp.  Scores of committed slots are unmasked; a tree slot j is visible to
+// One CTA per (head, sequence, KV chunk).  A sequence's KV rows are cut into TILE-row tiles and the tiles are dealt
+// to the grid's chunks in equal contiguous runs (computed on the device from the real length, so every chunk of
+// the launch has work whatever the length); the chunk's K and V tiles are streamed once from HBM through a
+// five-stage cp.async ring (four tiles in flight per CTA: the walk is bound by HBM latency otherwise).  Eight warps: warp w owns query rows 16 (w & 3) .. +15 (as MMA fragments) and
+// the keys of half (w >> 2) of every tile.  Scores of committed slots are unmasked; a tree slot j is visible to
 // row i iff bit j of the row's ancestor bitmask is set.  Each warp keeps a running (max, sum, weighted V)
 // per query row in the exp2 domain (online softmax, reductions by warp shuffles over the 4 lanes that share
-// a row); per-chunk partial results are merged by the combine kernel in fixed order.
+// a row); the two key halves are merged through shared memory at the end.  Per-chunk partial results go to a
+// scratch buffer; the CTA that reports in last for a (head, sequence) pair (an arrival counter that it resets)
+// merges the pair's chunks in chunk order and writes the output rows.
 // Precision: q, K, V and the attention output are stored as two bfloat16 planes (hi = bf16(v), lo = bf16(v - hi),
 // about 16 mantissa bits together).  Products use the three significant cross terms (hi*hi + lo*hi + hi*lo); the
 // softmax weights are split the same way before the P V product.  A plane distance of 0 selects hi-only operands.
@@ -17,7 +21,10 @@ namespace hydra {
 
 namespace {
 
-constexpr int NWARP = 4;           // 16 query rows each
+constexpr int NWARP = 8;           // warp w: query rows 16 (w & 3) .. +15, key half w >> 2 of every tile
+
+// First tile of chunk c when nt tiles are dealt to nch chunks in equal contiguous runs.
+__device__ __forceinline__ int chunk_first_tile(int c, int nt, int nch) { return (int)(((unsigned)c * (unsigned)nt) / (unsigned)nch); }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -41,11 +48,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int HD, bool HL, int TILE>
+template <int HD, bool HL, int TILE, int NS>
 __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __restrict__ q, size_t q_ps, const bf16* __restrict__ kc,
                                                                   const bf16* __restrict__ vc, size_t kv_ps, RowSet rs,
                                                                   float* __restrict__ part_o, float* __restrict__ part_ml,
-                                                                  int H, int max_seq, int nchunks, int chunk) {
+                                                                  int* __restrict__ arrived, bf16* __restrict__ out, size_t out_ps,
+                                                                  int H, int max_seq, int nchunks) {
   pdl_trigger();
   pdl_wait();
   constexpr int LDS = HD + 8;                         // padded row (bf16 elements): conflict-free ldmatrix
@@ -55,7 +63,8 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
   constexpr int TSZ = TILE * LDS;                     // elements of one staged tile
   extern __shared__ __align__(16) unsigned char smem_raw[];
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);       // [NP][64][LDS]
-  bf16* KVs = Qs + NP * 64 * LDS;                     // [2 stages][K planes, V planes][TILE][LDS]
+  bf16* KVs = Qs + NP * 64 * LDS;                     // [NS stages][K planes, V planes][TILE][LDS]
+  __shared__ int s_last;
 
   const int h = blockIdx.x, b = blockIdx.y, c = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -63,10 +72,11 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
   const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
   const int p0 = rs.pos0[b];
   const int total = p0 + nr;
-  const int s0 = c * chunk;
-  const int s1 = min(s0 + chunk, total);
+  const int nt = (total + TILE - 1) / TILE;
+  const int s0 = chunk_first_tile(c, nt, nchunks) * TILE;
+  const int s1 = min(chunk_first_tile(c + 1, nt, nchunks) * TILE, total);
   const int d = H * HD;
-  if (s0 >= s1 || nr <= 0) return;                    // nothing in this chunk: the combine kernel skips it
+  const bool has_work = s0 < s1 && nr > 0;            // a chunk that got no tile only reports in (see the end)
   const size_t head_off = ((size_t)b * H + h) * max_seq * HD;
   constexpr int PIECES = HD / 8;                       // 16-byte pieces per row
 
@@ -86,8 +96,14 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
     }
   };
 
-  // stage Q (rows past nr are zero) and the first KV tile
-  for (int e = tid; e < 64 * PIECES; e += NWARP * 32) {
+  const int ntiles = has_work ? (s1 - s0 + TILE - 1) / TILE : 0;
+  // request the first NS-1 KV tiles (one cp.async group each), then stage Q (rows past nr are zero)
+#pragma unroll
+  for (int i = 0; i < NS - 1; ++i) {
+    if (i < ntiles) load_tile(i, s0 + i * TILE);
+    cp_async_commit();
+  }
+  for (int e = tid; has_work && e < 64 * PIECES; e += NWARP * 32) {
     const int r = e / PIECES, pc = e % PIECES;
 #pragma unroll
     for (int pl = 0; pl < NP; ++pl) {
@@ -96,12 +112,9 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
       *reinterpret_cast<uint4*>(Qs + (pl * 64 + r) * LDS + pc * 8) = v;
     }
   }
-  load_tile(0, s0);
-  cp_async_commit();
-  __syncthreads();
-
-  const int row0 = warp * 16;
-  const bool warp_active = row0 < nr;
+  const int row0 = (warp & 3) * 16, khalf = warp >> 2;
+  constexpr int HT = TILE / 2;                           // keys of a tile per warp
+  const bool warp_active = has_work && row0 < nr;
   const int ra = row0 + g, rb = row0 + g + 8;            // the two query rows this thread owns
   const uint64_t mask_a = ra < nr ? rs.mask[ra] : 0ull, mask_b = rb < nr ? rs.mask[rb] : 0ull;
   float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
@@ -111,19 +124,18 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
   const float sc = rsqrtf((float)HD) * 1.4426950408889634f;   // 1/sqrt(hd) * log2(e)
   const uint32_t q_addr = (uint32_t)__cvta_generic_to_shared(Qs + (row0 + (lane & 15)) * LDS + (lane >> 4) * 8);
 
-  const int ntiles = (s1 - s0 + TILE - 1) / TILE;
   for (int it = 0; it < ntiles; ++it) {
     const int t0 = s0 + it * TILE;
-    const int buf = it & 1;
-    if (it + 1 < ntiles) load_tile(buf ^ 1, t0 + TILE);
+    const int buf = it % NS;
+    if (it + NS - 1 < ntiles) load_tile((it + NS - 1) % NS, t0 + (NS - 1) * TILE);      // the buffer read in iteration it - 1
     cp_async_commit();
-    cp_async_wait<1>();
+    cp_async_wait<NS - 1>();                             // tile `it` (and Q, stored before the first barrier) has landed
     __syncthreads();
     if (warp_active) {
-      float s[TILE / 8][4];
+      float s[HT / 8][4];
 #pragma unroll
-      for (int n = 0; n < TILE / 8; ++n) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
-      const uint32_t k_off = (uint32_t)((((lane & 7) + (lane >> 4) * 8) * LDS + ((lane >> 3) & 1) * 8) * 2);
+      for (int n = 0; n < HT / 8; ++n) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
+      const uint32_t k_off = (uint32_t)(((khalf * HT + (lane & 7) + (lane >> 4) * 8) * LDS + ((lane >> 3) & 1) * 8) * 2);
       const uint32_t kh_addr = (uint32_t)__cvta_generic_to_shared(tile_ptr(buf, 0, 0)) + k_off;
 #pragma unroll
       for (int kk = 0; kk < KSTEPS; ++kk) {
@@ -131,7 +143,7 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
         ldsm_x4(q_addr + kk * 32, qh[0], qh[1], qh[2], qh[3]);
         if (HL) ldsm_x4(q_addr + 64 * LDS * 2 + kk * 32, ql[0], ql[1], ql[2], ql[3]);
 #pragma unroll
-        for (int np = 0; np < TILE / 16; ++np) {       // 16 keys per ldmatrix.x4
+        for (int np = 0; np < HT / 16; ++np) {         // 16 keys per ldmatrix.x4
           uint32_t b0, b1, b2, b3;
           const uint32_t addr = kh_addr + (uint32_t)((np * 16 * LDS + kk * 16) * 2);
           ldsm_x4(addr, b0, b1, b2, b3);
@@ -147,15 +159,16 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
         }
       }
       // scale, mask, running max
-      const bool need_mask = t0 + TILE > p0 || t0 + TILE > s1;
+      const int k0 = t0 + khalf * HT;                    // first key of this warp's half
+      const bool need_mask = k0 + HT > p0 || k0 + HT > s1;
       float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
-      for (int n = 0; n < TILE / 8; ++n) {
+      for (int n = 0; n < HT / 8; ++n) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           float v = s[n][e] * sc;
           if (need_mask) {
-            int key = t0 + n * 8 + 2 * t + (e & 1);
+            int key = k0 + n * 8 + 2 * t + (e & 1);
             uint64_t mk = (e < 2) ? mask_a : mask_b;
             bool ok = key < s1 && (key < p0 || ((mk >> (key - p0)) & 1ull));
             v = ok ? v : -INFINITY;
@@ -172,7 +185,7 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
       m_a = mn_a; m_b = mn_b;
       float sum_a = 0.f, sum_b = 0.f;
 #pragma unroll
-      for (int n = 0; n < TILE / 8; ++n) {
+      for (int n = 0; n < HT / 8; ++n) {
         s[n][0] = exp2f(s[n][0] - base_a); s[n][1] = exp2f(s[n][1] - base_a);
         s[n][2] = exp2f(s[n][2] - base_b); s[n][3] = exp2f(s[n][3] - base_b);
         sum_a += s[n][0] + s[n][1]; sum_b += s[n][2] + s[n][3];
@@ -181,10 +194,10 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
 #pragma unroll
       for (int n = 0; n < NB; ++n) { o[n][0] *= al_a; o[n][1] *= al_a; o[n][2] *= al_b; o[n][3] *= al_b; }
       // O += P V
-      const uint32_t v_off = (uint32_t)((((lane & 7) + ((lane >> 3) & 1) * 8) * LDS + (lane >> 4) * 8) * 2);
+      const uint32_t v_off = (uint32_t)(((khalf * HT + (lane & 7) + ((lane >> 3) & 1) * 8) * LDS + (lane >> 4) * 8) * 2);
       const uint32_t vh_addr = (uint32_t)__cvta_generic_to_shared(tile_ptr(buf, 1, 0)) + v_off;
 #pragma unroll
-      for (int kp = 0; kp < TILE / 16; ++kp) {         // 16 keys per k-step
+      for (int kp = 0; kp < HT / 16; ++kp) {           // 16 keys per k-step
         uint32_t ah[4], al[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -214,86 +227,157 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
     }
     __syncthreads();
   }
-  if (!warp_active) return;
   l_a += __shfl_xor_sync(0xffffffffu, l_a, 1); l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
   l_b += __shfl_xor_sync(0xffffffffu, l_b, 1); l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
-  // partials: o (un-normalised), m (log2 domain), l
-  if (ra < nr) {
-    size_t idx = ((size_t)(b * rs.tc + ra) * H + h) * nchunks + c;
+  // merge the two key halves: the upper warps hand (m, l, o) to their partner through the (now idle) tile ring
+  float* xch = reinterpret_cast<float*>(KVs) + ((warp & 3) * 32 + lane) * (NB * 4 + 4);
+  if (khalf == 1 && warp_active) {
 #pragma unroll
-    for (int n = 0; n < NB; ++n) *reinterpret_cast<float2*>(part_o + idx * HD + n * 8 + 2 * t) = make_float2(o[n][0], o[n][1]);
-    if (t == 0) { part_ml[idx * 2] = m_a; part_ml[idx * 2 + 1] = l_a; }
+    for (int n = 0; n < NB; ++n) *reinterpret_cast<float4*>(xch + n * 4) = make_float4(o[n][0], o[n][1], o[n][2], o[n][3]);
+    *reinterpret_cast<float4*>(xch + NB * 4) = make_float4(m_a, m_b, l_a, l_b);
   }
-  if (rb < nr) {
-    size_t idx = ((size_t)(b * rs.tc + rb) * H + h) * nchunks + c;
+  __syncthreads();
+  if (khalf == 0 && warp_active) {
+    const float4 ml = *reinterpret_cast<const float4*>(xch + NB * 4);
+    const float mn_a = fmaxf(m_a, ml.x), mn_b = fmaxf(m_b, ml.y);
+    const float base_a = mn_a == -INFINITY ? 0.f : mn_a, base_b = mn_b == -INFINITY ? 0.f : mn_b;
+    const float w0a = exp2f(m_a - base_a), w1a = exp2f(ml.x - base_a), w0b = exp2f(m_b - base_b), w1b = exp2f(ml.y - base_b);
+    m_a = mn_a; m_b = mn_b;
+    l_a = l_a * w0a + ml.z * w1a; l_b = l_b * w0b + ml.w * w1b;
+    // partials: o (un-normalised), m (log2 domain), l
+    const size_t idx_a = ((size_t)(b * rs.tc + ra) * H + h) * nchunks + c, idx_b = ((size_t)(b * rs.tc + rb) * H + h) * nchunks + c;
 #pragma unroll
-    for (int n = 0; n < NB; ++n) *reinterpret_cast<float2*>(part_o + idx * HD + n * 8 + 2 * t) = make_float2(o[n][2], o[n][3]);
-    if (t == 0) { part_ml[idx * 2] = m_b; part_ml[idx * 2 + 1] = l_b; }
+    for (int n = 0; n < NB; ++n) {
+      const float4 v = *reinterpret_cast<const float4*>(xch + n * 4);
+      if (ra < nr) __stcg(reinterpret_cast<float2*>(part_o + idx_a * HD + n * 8 + 2 * t), make_float2(o[n][0] * w0a + v.x * w1a, o[n][1] * w0a + v.y * w1a));
+      if (rb < nr) __stcg(reinterpret_cast<float2*>(part_o + idx_b * HD + n * 8 + 2 * t), make_float2(o[n][2] * w0b + v.z * w1b, o[n][3] * w0b + v.w * w1b));
+    }
+    if (t == 0 && ra < nr) __stcg(reinterpret_cast<float2*>(part_ml + idx_a * 2), make_float2(m_a, l_a));
+    if (t == 0 && rb < nr) __stcg(reinterpret_cast<float2*>(part_ml + idx_b * 2), make_float2(m_b, l_b));
+  }
+  // The last of the (head, sequence)'s chunks to report in merges them:
+  // out[r][h][:] = sum_c o_c 2^(m_c - M) / sum_c l_c 2^(m_c - M) over the chunks that were dealt tiles, in chunk order.
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int prev = atomicAdd(arrived + b * H + h, 1);
+    s_last = prev == nchunks - 1;
+    if (s_last) arrived[b * H + h] = 0;                  // ready for the next launch
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // weights first (one (row, chunk) pair per thread), then the rows: every thread owns up to 8 float4 pieces and
+  // walks the chunks with all of its loads of a chunk in flight together
+  float* sm_m = reinterpret_cast<float*>(KVs);         // [tc][nchunks] chunk maxima, then the normalised chunk weights
+  float* sm_l = sm_m + rs.tc * nchunks;
+  for (int e = tid; e < rs.tc * nchunks; e += NWARP * 32) {
+    const int i = e / nchunks, cc = e % nchunks;
+    float2 ml = make_float2(-INFINITY, 0.f);
+    if (i < nr && chunk_first_tile(cc, nt, nchunks) != chunk_first_tile(cc + 1, nt, nchunks))       // else: dealt no tile, wrote nothing
+      ml = __ldcg(reinterpret_cast<const float2*>(part_ml + (((size_t)b * rs.tc + i) * H + h) * nchunks * 2 + cc * 2));
+    sm_m[e] = ml.x; sm_l[e] = ml.y;
+  }
+  __syncthreads();
+  for (int i = tid; i < rs.tc; i += NWARP * 32) {
+    float M = -INFINITY, L = 0.f;
+    for (int cc = 0; cc < nchunks; ++cc) M = fmaxf(M, sm_m[i * nchunks + cc]);
+    for (int cc = 0; cc < nchunks; ++cc) {
+      const float mc = sm_m[i * nchunks + cc];
+      const float w = mc == -INFINITY ? 0.f : exp2f(mc - M);
+      L += sm_l[i * nchunks + cc] * w;
+      sm_m[i * nchunks + cc] = w;
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    for (int cc = 0; cc < nchunks; ++cc) sm_m[i * nchunks + cc] *= inv;
+  }
+  __syncthreads();
+  constexpr int V4 = HD / 4, PER = (64 * V4 + NWARP * 32 - 1) / (NWARP * 32);
+  float4 acc[PER];
+#pragma unroll
+  for (int j = 0; j < PER; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int cc = 0; cc < nchunks; ++cc) {
+    float4 v[PER];
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const int e = tid + j * NWARP * 32, i = e / V4, k4 = e % V4;
+      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < nr && sm_m[i * nchunks + cc] != 0.f)
+        v[j] = __ldcg(reinterpret_cast<const float4*>(part_o + ((((size_t)b * rs.tc + i) * H + h) * nchunks + cc) * HD + k4 * 4));
+    }
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const int i = (tid + j * NWARP * 32) / V4;
+      const float w = i < rs.tc ? sm_m[i * nchunks + cc] : 0.f;
+      acc[j].x += v[j].x * w; acc[j].y += v[j].y * w; acc[j].z += v[j].z * w; acc[j].w += v[j].w * w;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int e = tid + j * NWARP * 32, i = e / V4, k4 = e % V4;
+    if (i >= rs.tc) continue;
+    bf16* dst = out + ((size_t)b * rs.tc + i) * d + h * HD + k4 * 4;      // rows past nr get zeros
+    const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[j].x, acc[j].y), h1 = __floats2bfloat162_rn(acc[j].z, acc[j].w);
+    *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+    if (out_ps) {
+      const __nv_bfloat162 l0 = __floats2bfloat162_rn(acc[j].x - __low2float(h0), acc[j].y - __high2float(h0));
+      const __nv_bfloat162 l1 = __floats2bfloat162_rn(acc[j].z - __low2float(h1), acc[j].w - __high2float(h1));
+      *reinterpret_cast<uint2*>(dst + out_ps) = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+    }
   }
 }
 
-// out[r][h][:] = sum_c o_c 2^(m_c - M) / sum_c l_c 2^(m_c - M) over the chunks that hold slots of sequence b.
-template <int HD>
-__global__ void __launch_bounds__(HD) tree_attn_tc_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                                                  RowSet rs, bf16* __restrict__ out, size_t out_ps, int H, int nchunks, int chunk) {
-  pdl_trigger();
-  pdl_wait();
-  const int r = blockIdx.x, h = blockIdx.y, b = r / rs.tc, i = r % rs.tc;
-  const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
-  const int k = threadIdx.x;
-  bf16* dst = out + (size_t)r * H * HD + h * HD;
-  if (i >= nr) { dst[k] = __float2bfloat16_rn(0.f); if (out_ps) dst[out_ps + k] = __float2bfloat16_rn(0.f); return; }
-  const int used = min(nchunks, (rs.pos0[b] + nr + chunk - 1) / chunk);
-  const size_t idx = ((size_t)r * H + h) * nchunks;
-  float M = -INFINITY;
-  for (int c = 0; c < used; ++c) M = fmaxf(M, part_ml[(idx + c) * 2]);
-  float L = 0.f, acc = 0.f;
-  for (int c = 0; c < used; ++c) {
-    float mc = part_ml[(idx + c) * 2];
-    if (mc == -INFINITY) continue;
-    float w = exp2f(mc - M);
-    L += part_ml[(idx + c) * 2 + 1] * w;
-    acc += part_o[(idx + c) * HD + k] * w;
+// Number of KV chunks per (head, sequence) for lengths up to len_upper.  Few (head, sequence) pairs: one CTA per SM
+// at most and chunks as long as that allows (the kernel is bound by the MMA rate of an SM, so what counts is the
+// largest number of tiles any SM walks, plus about one tile of set-up per CTA); many pairs: chunks of about
+// 128 rows, which the block scheduler balances.
+int pick_chunks(int pairs, int len_upper, int tile, int nchunks_max, int sms) {
+  const int nt = (len_upper + tile - 1) / tile;
+  int hi = (len_upper + ATT_CHUNK_ROWS - 1) / ATT_CHUNK_ROWS;
+  hi = hi < 1 ? 1 : (hi > nchunks_max ? nchunks_max : hi);
+  int best = hi; long best_cost = -1;
+  for (int n = 1; n <= hi; ++n) {
+    const long per_sm = ((long)pairs * n + sms - 1) / sms, tiles = (nt + n - 1) / n;
+    const long cost = per_sm * (tiles + 1) + 1;
+    if (best_cost < 0 || cost <= best_cost) { best = n; best_cost = cost; }
   }
-  const float v = acc / L;
-  const bf16 hi = __float2bfloat16_rn(v);
-  dst[k] = hi;
-  if (out_ps) dst[out_ps + k] = __float2bfloat16_rn(v - __bfloat162float(hi));
+  return best;
 }
 
-template <int HD, bool HL, int TILE>
-hydra_status run_t(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
-                 float* scratch, int H, int max_seq, int len_upper, int chunk, cudaStream_t st) {
-  const int nchunks_max = (max_seq + chunk - 1) / chunk;
-  int nchunks = (len_upper + chunk - 1) / chunk;
-  nchunks = nchunks < 1 ? 1 : (nchunks > nchunks_max ? nchunks_max : nchunks);
+template <int HD, bool HL, int NS>
+hydra_status run_ns(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
+                 float* scratch, int H, int max_seq, int len_upper, cudaStream_t st) {
+  constexpr int TILE = 32;                    // 32-row tiles, four of them in flight: hides the HBM latency of a chunk's walk
+  const int nchunks_max = (max_seq + ATT_CHUNK_ROWS - 1) / ATT_CHUNK_ROWS;     // what the scratch is sized for
+  static int sms = 0;
+  if (!sms) { int dev = 0; HYDRA_CUDA(cudaGetDevice(&dev)); HYDRA_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)); }
+  if ((size_t)H * rs.batch * sizeof(int) > ATT_SCRATCH_HEADER) return HYDRA_ERR_UNSUPPORTED;
+  const int nchunks = pick_chunks(H * rs.batch, len_upper, TILE, nchunks_max, sms);
   const size_t rows = (size_t)rs.batch * rs.tc;
-  float* part_o = scratch;
-  float* part_ml = scratch + rows * H * nchunks_max * HD;
+  int* arrived = reinterpret_cast<int*>(scratch);     // one counter per (sequence, head): zero between launches
+  float* part_o = scratch + ATT_SCRATCH_HEADER / sizeof(float);
+  float* part_ml = part_o + rows * H * nchunks_max * HD;
   constexpr int LDS = HD + 8;
   constexpr int NP = HL ? 2 : 1;
-  const size_t smem = (size_t)NP * (64 + 4 * TILE) * LDS * sizeof(bf16);
+  const size_t smem = (size_t)NP * (64 + 2 * NS * TILE) * LDS * sizeof(bf16);
   static bool attr_done = false;
   if (!attr_done) {
-    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_done = true;
   }
-  launch_pdl(tree_attn_tc_kernel<HD, HL, TILE>, dim3(H, rs.batch, nchunks), dim3(NWARP * 32), smem, st, q, q_ps, kc, vc, kv_ps, rs, part_o, part_ml, H,
-             max_seq, nchunks, chunk);
-  HYDRA_LAUNCH_CHECK();
-  launch_pdl(tree_attn_tc_combine_kernel<HD>, dim3((unsigned)rows, H), dim3(HD), 0, st, (const float*)part_o, (const float*)part_ml, rs, out, out_ps, H,
-             nchunks, chunk);
+  launch_pdl(tree_attn_tc_kernel<HD, HL, TILE, NS>, dim3(H, rs.batch, nchunks), dim3(NWARP * 32), smem, st, q, q_ps, kc, vc, kv_ps, rs, part_o, part_ml,
+             arrived, out, out_ps, H, max_seq, nchunks);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
-// KV rows per pipeline stage: 32 lets two CTAs share an SM with two-plane operands (HYDRA_ATT_TILE=64: one CTA, fewer syncs).
 template <int HD, bool HL>
 hydra_status run(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
-                 float* scratch, int H, int max_seq, int len_upper, int chunk, cudaStream_t st) {
-  static const int tile = []() { const char* e = getenv("HYDRA_ATT_TILE"); return e ? atoi(e) : 32; }();
-  if (tile == 64) return run_t<HD, HL, 64>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, chunk, st);
-  return run_t<HD, HL, 32>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, chunk, st);
+                 float* scratch, int H, int max_seq, int len_upper, cudaStream_t st) {
+  static const int ns = []() { const char* e = getenv("HYDRA_ATT_NS"); return e ? atoi(e) : 5; }();
+  if (ns == 2) return run_ns<HD, HL, 2>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, st);
+  if (ns == 3) return run_ns<HD, HL, 3>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, st);
+  return run_ns<HD, HL, 5>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, st);
 }
 
 }  // namespace
@@ -302,12 +386,11 @@ hydra_status tree_attention_tc(const bf16* q, size_t q_ps, const bf16* kc, const
                                size_t out_ps, void* scratch, int H, int hd, int max_seq, int len_upper, cudaStream_t st) {
   if (rs.tc > 64) return HYDRA_ERR_UNSUPPORTED;
   if ((q_ps == 0) != (kv_ps == 0)) return HYDRA_ERR_UNSUPPORTED;           // q and the caches split the same way
-  const int chunk = ATT_CHUNK_ROWS;
   const bool hl = q_ps != 0;
-  if (hd == 128 && hl) return run<128, true>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, chunk, st);
-  if (hd == 128) return run<128, false>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, chunk, st);
-  if (hd == 64 && hl) return run<64, true>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, chunk, st);
-  if (hd == 64) return run<64, false>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, chunk, st);
+  if (hd == 128 && hl) return run<128, true>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, st);
+  if (hd == 128) return run<128, false>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, st);
+  if (hd == 64 && hl) return run<64, true>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, st);
+  if (hd == 64) return run<64, false>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, st);
   return HYDRA_ERR_UNSUPPORTED;
 }
 

@@ -716,6 +716,7 @@ hydra_status hydra_tree_attention(const void* q, const void* kc, const void* vc,
   RowSet rs{batch, tc, n_rows, pos0, nullptr, mask};
   const size_t d = (size_t)n_heads * head_dim;
   const size_t qp = planes == 2 ? (size_t)batch * tc * d : 0, kvp = planes == 2 ? (size_t)batch * n_heads * max_seq * head_dim : 0;
+  HYDRA_CUDA(cudaMemsetAsync(scratch, 0, ATT_SCRATCH_HEADER, (cudaStream_t)stream));     // arrival counters start at zero
   return tree_attention(q, qp, kc, vc, kvp, rs, out, qp, scratch, n_heads, head_dim, max_seq, max_seq, dtype, (cudaStream_t)stream);
 }
 

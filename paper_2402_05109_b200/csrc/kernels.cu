@@ -413,7 +413,7 @@ __global__ void tree_attn_combine_kernel(const float* __restrict__ part_o, const
 
 size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq) {
   size_t nchunks = (size_t)(max_seq + ATT_CHUNK - 1) / ATT_CHUNK;
-  return (size_t)batch * tc * n_heads * nchunks * (head_dim + 2) * sizeof(float);
+  return ATT_SCRATCH_HEADER + (size_t)batch * tc * n_heads * nchunks * (head_dim + 2) * sizeof(float);
 }
 
 template <typename T, int HD>

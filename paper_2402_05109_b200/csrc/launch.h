@@ -33,6 +33,7 @@ hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table
                             void* kcache, void* vcache, size_t kv_ps, RowSet rs, int n_heads, int head_dim, int max_seq, int dtype,
                             int* status, cudaStream_t st);
 constexpr int ATT_CHUNK_ROWS = 128;     // KV rows per attention CTA (split-KV granularity)
+constexpr size_t ATT_SCRATCH_HEADER = 65536; // bytes at the head of the attention scratch: per-(sequence, head) arrival counters
 size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
 // bfloat16 caches: tensor-core kernel (attention_tc.cu); float caches: SIMT kernel.  q is in the cache dtype.
 // "_ps" arguments: element distance between the hi and lo planes of a bfloat16 operand (0 = hi only; unused for float).
