@@ -205,7 +205,7 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--gemm-mode", type=int, default=0, help="0 tcgen05 + separate consumer kernels (default), 1 SIMT, 2 tcgen05 with fused epilogues")
+    ap.add_argument("--gemm-mode", type=int, default=0, help="0 tcgen05, one launch per GEMM (default), 1 SIMT, 2 tcgen05 with one persistent kernel per layer tail")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

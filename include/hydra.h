@@ -159,8 +159,12 @@ enum { HYDRA_TIME_GEMM = 0, HYDRA_TIME_ATTENTION = 1, HYDRA_TIME_ACCEPT = 2 };
 hydra_status hydra_set_timing(hydra_ctx*, int on);
 hydra_status hydra_get_timing(hydra_ctx*, int kclass, double* ms_total, long long* launches, double* bytes_total);
 
-/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA (default); 1 = the plain SIMT kernel (debugging; it
- * reads only the hi plane of the activations). */
+/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA, one launch per GEMM and per row-wise kernel (default);
+ * 1 = the plain SIMT kernel (debugging; it reads only the hi plane of the activations); 2 = tcgen05/TMA with
+ * everything of a layer after its attention (O projection, residual + norm, gate/up, SiLU * up, down, residual +
+ * norm, the next layer's QKV projection or the LM head) in ONE persistent, cooperatively launched kernel whose
+ * CTAs hand over between GEMMs through grid-wide counters (same results as mode 0; currently slower, because a
+ * hand-over costs more than a launch boundary; calls of two contexts in this mode must not overlap on the GPU). */
 hydra_status hydra_set_gemm_mode(hydra_ctx*, int mode);
 
 const char* hydra_status_str(hydra_status);

@@ -117,6 +117,26 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 64 consecutive accumulator columns of this thread's lane (one wait for the whole batch)
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr)
+      : "memory");
+}
+// the same for two column ranges at once (the W*hi and W*lo halves of a concatenated accumulator)
+__device__ __forceinline__ void tmem_ld64x2(uint32_t taddr0, uint32_t taddr1, uint32_t (&r)[64], uint32_t (&q)[64]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%128];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%64,%65,%66,%67,%68,%69,%70,%71,%72,%73,%74,%75,%76,%77,%78,%79,%80,%81,%82,%83,%84,%85,%86,%87,%88,%89,%90,%91,%92,%93,%94,%95,%96,%97,%98,%99,%100,%101,%102,%103,%104,%105,%106,%107,%108,%109,%110,%111,%112,%113,%114,%115,%116,%117,%118,%119,%120,%121,%122,%123,%124,%125,%126,%127}, [%129];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]), "=r"(q[0]), "=r"(q[1]), "=r"(q[2]), "=r"(q[3]), "=r"(q[4]), "=r"(q[5]), "=r"(q[6]), "=r"(q[7]), "=r"(q[8]), "=r"(q[9]), "=r"(q[10]), "=r"(q[11]), "=r"(q[12]), "=r"(q[13]), "=r"(q[14]), "=r"(q[15]), "=r"(q[16]), "=r"(q[17]), "=r"(q[18]), "=r"(q[19]), "=r"(q[20]), "=r"(q[21]), "=r"(q[22]), "=r"(q[23]), "=r"(q[24]), "=r"(q[25]), "=r"(q[26]), "=r"(q[27]), "=r"(q[28]), "=r"(q[29]), "=r"(q[30]), "=r"(q[31]), "=r"(q[32]), "=r"(q[33]), "=r"(q[34]), "=r"(q[35]), "=r"(q[36]), "=r"(q[37]), "=r"(q[38]), "=r"(q[39]), "=r"(q[40]), "=r"(q[41]), "=r"(q[42]), "=r"(q[43]), "=r"(q[44]), "=r"(q[45]), "=r"(q[46]), "=r"(q[47]), "=r"(q[48]), "=r"(q[49]), "=r"(q[50]), "=r"(q[51]), "=r"(q[52]), "=r"(q[53]), "=r"(q[54]), "=r"(q[55]), "=r"(q[56]), "=r"(q[57]), "=r"(q[58]), "=r"(q[59]), "=r"(q[60]), "=r"(q[61]), "=r"(q[62]), "=r"(q[63])
+      : "r"(taddr0), "r"(taddr1)
+      : "memory");
+}
+
 // Shared-memory matrix descriptor of a K-major tile stored with the 128-byte swizzle: rows are 128 bytes,
 // groups of 8 rows are 1024 bytes apart (stride byte offset), descriptor version 1, layout type 2.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
@@ -132,6 +152,46 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
 // Instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = MT.
 __host__ __device__ constexpr uint32_t instr_desc(int mt) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mt >> 3) << 17) | ((uint32_t)(BLOCK_N >> 4) << 24);
+}
+
+// One accumulator buffer (MT columns, plus MT more holding W*lo when `cat`) of this thread's lane -> partial-sum rows
+// m0.. of column dst; 64 columns per batch of tensor-memory loads when the tile has that many.
+template <int MT>
+__device__ __forceinline__ void store_accumulator(uint32_t taddr, bool cat, float* dst, int m0, int m, int n) {
+  if constexpr (MT >= 64) {
+#pragma unroll 1
+    for (int c = 0; c < MT; c += 64) {
+      if (m0 + c >= m) break;
+      uint32_t r[64];
+      if (cat) {
+        uint32_t r2[64];
+        tmem_ld64x2(taddr + (uint32_t)c, taddr + (uint32_t)(MT + c), r, r2);
+#pragma unroll
+        for (int j = 0; j < 64; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+      } else {
+        tmem_ld64(taddr + (uint32_t)c, r);
+      }
+#pragma unroll
+      for (int j = 0; j < 64; ++j)
+        if (m0 + c + j < m) __stcg(dst + (size_t)(m0 + c + j) * n, __uint_as_float(r[j]));
+    }
+  } else {
+#pragma unroll 1
+    for (int c = 0; c < MT; c += 16) {
+      if (m0 + c >= m) break;
+      uint32_t r[16];
+      tmem_ld16(taddr + (uint32_t)c, r);
+      if (cat) {                                         // add the W*lo columns
+        uint32_t r2[16];
+        tmem_ld16(taddr + (uint32_t)(MT + c), r2);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (m0 + c + j < m) __stcg(dst + (size_t)(m0 + c + j) * n, __uint_as_float(r[j]));
+    }
+  }
 }
 
 template <int MT, int BUDGET_KB> struct TileCfg {
@@ -217,49 +277,48 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (lane == 0) {
       uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       if (a.flags & 1) { asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol_w)); pol_x = pol_w; }
-      auto coords = [&](int u, int& kcol, int& nrow, int& mrow) {
-        const int tile = u / a.kb;
-        kcol = (u - tile * a.kb) * BLOCK_K;
-        nrow = (tile % a.n_tiles) * BLOCK_N;
-        mrow = (tile / a.n_tiles) * MT;
-      };
       const int pre = n_units < C::STAGES ? n_units : C::STAGES;      // weight tiles already requested in the prologue
+      // (k column, weight row, activation row) of the unit being issued, advanced without divisions
+      int kcol = 0, nrow = 0, mrow = 0;
+      if (n_units > 0) {
+        const int tile = u_begin / a.kb;
+        kcol = (u_begin - tile * a.kb) * BLOCK_K; nrow = (tile % a.n_tiles) * BLOCK_N; mrow = (tile / a.n_tiles) * MT;
+      }
+      const int kend = a.kb * BLOCK_K, nend = a.n_tiles * BLOCK_N, lo_rows = a.x_lo_rows;
+      const uint32_t x_bytes = lo_rows ? C::B_BYTES : C::B_PLANE;
+      int s = 0; uint32_t eph = 1;                       // ring stage, parity of its empty barrier
       TRACE(2);
       grid_dep_wait();                     // activations are the preceding kernel's output
       for (int i = 0; i < n_units; ++i) {
-        const int s = i % C::STAGES;
-        const uint32_t ph = (i / C::STAGES) & 1;
-        int kcol, nrow, mrow;
-        coords(u_begin + i, kcol, nrow, mrow);
         const uint32_t a_dst = tiles + s * C::STAGE_BYTES;
         if (i >= pre) {
-          if (!mbar_wait(empty_bar(s), ph ^ 1u)) { GIVE_UP(1, i); s_abort = 1; break; }
+          if (!mbar_wait(empty_bar(s), eph)) { GIVE_UP(1, i); s_abort = 1; break; }
           mbar_arrive_expect_tx(fullw_bar(s), A_BYTES);
           tma_load_2d(a_dst, &tmW, kcol, nrow, fullw_bar(s), pol_w);
         }
-        mbar_arrive_expect_tx(fullx_bar(s), a.x_lo_rows ? C::B_BYTES : C::B_PLANE);
+        mbar_arrive_expect_tx(fullx_bar(s), x_bytes);
         tma_load_2d(a_dst + A_BYTES, &tmX, kcol, mrow, fullx_bar(s), pol_x);
-        if (a.x_lo_rows) tma_load_2d(a_dst + A_BYTES + C::B_PLANE, &tmX, kcol, a.x_lo_rows + mrow, fullx_bar(s), pol_x);
+        if (lo_rows) tma_load_2d(a_dst + A_BYTES + C::B_PLANE, &tmX, kcol, lo_rows + mrow, fullx_bar(s), pol_x);
+        if (++s == C::STAGES) { s = 0; eph ^= 1u; }
+        if ((kcol += BLOCK_K) == kend) { kcol = 0; if ((nrow += BLOCK_N) == nend) { nrow = 0; mrow += MT; } }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       const bool cat = C::CAT && a.x_lo_rows != 0;
       const uint32_t idesc = cat ? instr_desc(2 * MT) : instr_desc(MT);
-      int seg = 0;
+      int seg = 0, s = 0;
+      uint32_t ph = 0;                                   // ring stage, parity of its full barriers
       bool ok = true;
+      const bool two_pass = a.x_lo_rows && !cat;
+      int seg_len = n_units > 0 ? min((u_begin / a.kb + 1) * a.kb, u_end) - u_begin : 0;      // first segment: the tail of a tile
       for (int i = 0; i < n_units && ok;) {
-        const int u = u_begin + i;
-        const int tile = u / a.kb;
-        const int seg_len = min((tile + 1) * a.kb, u_end) - u;
         const int acc = seg & 1;
         const uint32_t acc_ph = (seg >> 1) & 1;
         if (!mbar_wait(accempty_bar(acc), acc_ph ^ 1u)) { GIVE_UP(2, i); ok = false; break; }      // epilogue has drained this buffer
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * C::ACC_COLS);
         for (int j = 0; j < seg_len; ++j, ++i) {
-          const int s = i % C::STAGES;
-          const uint32_t ph = (i / C::STAGES) & 1;
           if (!mbar_wait(fullw_bar(s), ph)) { GIVE_UP(3, i); ok = false; break; }
           if (!mbar_wait(fullx_bar(s), ph)) { GIVE_UP(4, i); ok = false; break; }
           if (i == 0) TRACE(3);
@@ -270,16 +329,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
           for (int k = 0; k < BLOCK_K / 16; ++k)         // 16 bf16 = 32 bytes per MMA: +2 in 16-byte units
             umma_bf16(tmem_d, adesc + 2u * k, bdesc + 2u * k, idesc, (uint32_t)((j | k) != 0));
-          if (a.x_lo_rows && !cat) {                     // the low-order plane of the activations, same weights
+          if (two_pass) {                                // the low-order plane of the activations, same weights
             const uint64_t ldesc = smem_desc_sw128(a_addr + A_BYTES + C::B_PLANE);
 #pragma unroll
             for (int k = 0; k < BLOCK_K / 16; ++k) umma_bf16(tmem_d, adesc + 2u * k, ldesc + 2u * k, idesc, 1u);
           }
           umma_commit(empty_bar(s));                     // frees the stage once these MMAs have read it
+          if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
         umma_commit(accfull_bar(acc));                   // segment complete: hand the accumulator to the epilogue
         ++seg;
+        seg_len = min(a.kb, n_units - i);                // every later segment starts a tile
       }
       TRACE(4);
       if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
@@ -302,22 +363,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int n0 = (tile % a.n_tiles) * BLOCK_N, m0 = (tile / a.n_tiles) * MT;
       float* dst = a.part + (size_t)slot * a.slot_stride + n0 + epi_tid;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * C::ACC_COLS);
-      const bool cat = C::CAT && a.x_lo_rows != 0;
-#pragma unroll 1
-      for (int c = 0; c < MT; c += 16) {
-        if (m0 + c >= a.m) break;
-        uint32_t r[16];
-        tmem_ld16(taddr + (uint32_t)c, r);
-        if (cat) {                                       // add the W*lo columns
-          uint32_t r2[16];
-          tmem_ld16(taddr + (uint32_t)(MT + c), r2);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
-        }
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (m0 + c + j < a.m) dst[(size_t)(m0 + c + j) * a.n] = __uint_as_float(r[j]);
-      }
+      store_accumulator<MT>(taddr, C::CAT && a.x_lo_rows != 0, dst, m0, a.m, a.n);
       tc_fence_before();
       if (lane == 0) mbar_arrive(accempty_bar(acc));     // the MMA warp may reuse this accumulator
       i += seg_len;
@@ -332,6 +378,338 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   }
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, C::TMEM_COLS); }
   if (threadIdx.x == 32) TRACE(7);
+}
+
+// ---- GEMM chain ----------------------------------------------------------------------------------
+// Several GEMMs over the same rows run as ONE persistent kernel: job j's activations are produced from job j-1's
+// partial sums by a row-wise step (residual + RMSNorm, or SiLU(gate) * up) that the epilogue warps of all CTAs share
+// out among themselves between two grid-wide counters.  The producer warp keeps requesting the next job's weight
+// tiles (which depend on nothing) while that step runs, so HBM does not idle across the boundary, and the ramp and
+// tail of a separate launch per GEMM and per row-wise kernel disappear.
+//   done[j]  (sync[j])      counts CTAs whose partial sums of job j are in memory
+//   ready[j] (sync[8 + j])  counts CTAs that finished their share of the step that makes job j's activations
+//   sync[16]                counts CTAs at the exit; the last one clears all counters for the next launch
+// The grid is launched cooperatively with one CTA per SM, so every CTA is resident and the counters fill;
+// every spin is bounded all the same (ST_TIMEOUT + the usual unwinding through the bounded barrier waits).
+constexpr int MAX_JOBS = 4;
+constexpr uint32_t SPIN_LIMIT = 1u << 22;
+struct ChainJob {
+  int n, kb, n_tiles, total_units, q, x_lo_rows;
+  int op, cols;                  // row-wise step after this job (CHAIN_NONE / CHAIN_RESID_NORM / CHAIN_SILU_MUL), its output width
+  size_t slot_stride;
+  float* resid; const bf16* gain; bf16* out; size_t out_ps; float* hn; float eps;
+};
+struct ChainArgs {
+  CUtensorMap tmW[MAX_JOBS];
+  CUtensorMap tmX[MAX_JOBS];
+  ChainJob job[MAX_JOBS];
+  float* part; int m, n_jobs; int* status; int* diag; int* sync;
+};
+
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ bool spin_until(const int* p, int target) {
+  for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+    if (ld_acquire(p) >= target) return true;
+    __nanosleep(40);
+  }
+  return false;
+}
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// acc[u] = sum over the ns[u] slots of the four floats at element offset off[u] of a slot (all loads of a round in flight together)
+template <int U>
+__device__ __forceinline__ void sum_slots_multi(const float* part, size_t stride, const size_t (&off)[U], const int (&ns)[U], float4 (&acc)[U]) {
+  constexpr int PMAX = 6;
+  int mx = 0;
+#pragma unroll
+  for (int u = 0; u < U; ++u) { acc[u] = make_float4(0.f, 0.f, 0.f, 0.f); mx = max(mx, ns[u]); }
+#pragma unroll
+  for (int p = 0; p < PMAX; ++p) {
+    float4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = p < ns[u] ? __ldcg(reinterpret_cast<const float4*>(part + p * stride + off[u])) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < U; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
+  }
+  for (int p = PMAX; p < mx; ++p)
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (p < ns[u]) {
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(part + p * stride + off[u]));
+        acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
+      }
+}
+__device__ __forceinline__ void store_hl4(bf16* dst, size_t lo_off, const float4& v) {
+  const __nv_bfloat162 h0 = __floats2bfloat162_rn(v.x, v.y), h1 = __floats2bfloat162_rn(v.z, v.w);
+  *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+  if (lo_off) {
+    const __nv_bfloat162 l0 = __floats2bfloat162_rn(v.x - __low2float(h0), v.y - __high2float(h0));
+    const __nv_bfloat162 l1 = __floats2bfloat162_rn(v.z - __low2float(h1), v.w - __high2float(h1));
+    *reinterpret_cast<uint2*>(dst + lo_off) = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+  }
+}
+
+// act[r][c] = SiLU(gate[r][c]) * up[r][c] from the gate/up partial sums ([r][2 f] per slot): this CTA's share, 128 threads
+__device__ void chain_silu_mul(const ChainArgs& a, const ChainJob& J, const SplitDesc& sd, int et) {
+  const int f = J.cols;
+  const long long items = (long long)a.m * f / 4, step = (long long)gridDim.x * 128;
+  for (long long it0 = (long long)blockIdx.x * 128 + et; it0 < items; it0 += 2 * step) {
+    size_t off[4]; int ns[4]; float4 acc[4];
+    long long e[2] = {it0 * 4, (it0 + step) * 4};
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const bool valid = e[k] < (long long)a.m * f;
+      const int r = valid ? (int)(e[k] / f) : 0, c = valid ? (int)(e[k] % f) : 0;
+      off[2 * k] = (size_t)r * 2 * f + c; off[2 * k + 1] = off[2 * k] + f;
+      ns[2 * k] = valid ? split_count(sd, r, c) : 0; ns[2 * k + 1] = valid ? split_count(sd, r, f + c) : 0;
+    }
+    sum_slots_multi<4>(a.part, sd.stride, off, ns, acc);
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+      if (e[k] < (long long)a.m * f) {
+        const float4 g = acc[2 * k], u = acc[2 * k + 1];
+        store_hl4(J.out + e[k], J.out_ps, make_float4(silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w));
+      }
+  }
+}
+
+// resid[r] += sum of the partial slots; then (with a gain) out[r] = resid[r] * rsqrt(mean(resid[r]^2) + eps) * gain as hi/lo
+// planes (and as float in hn): rows r = cta, cta + grid, ...; 128 threads per row
+__device__ void chain_resid_norm(const ChainArgs& a, const ChainJob& J, const SplitDesc& sd, int et, float* red /* smem [4] */) {
+  const int d = J.cols;
+  for (int r = blockIdx.x; r < a.m; r += gridDim.x) {
+    float* xr = J.resid + (size_t)r * d;
+    float ss = 0.f;
+    for (int c0 = et * 4; c0 < d; c0 += 4 * 512) {
+      size_t off[4]; int ns[4]; float4 acc[4], v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + u * 512;
+        const bool valid = c < d;
+        off[u] = (size_t)r * d + (valid ? c : 0); ns[u] = valid ? split_count(sd, r, c) : 0;
+        v[u] = valid ? *reinterpret_cast<const float4*>(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      sum_slots_multi<4>(a.part, sd.stride, off, ns, acc);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + u * 512;
+        if (c < d) {
+          v[u].x += acc[u].x; v[u].y += acc[u].y; v[u].z += acc[u].z; v[u].w += acc[u].w;
+          *reinterpret_cast<float4*>(xr + c) = v[u];
+          ss += v[u].x * v[u].x + v[u].y * v[u].y + v[u].z * v[u].z + v[u].w * v[u].w;
+        }
+      }
+    }
+    if (!J.gain) continue;
+    ss = warp_sum(ss);
+    epi_bar();                                           // red[] free again (previous row's readers are done)
+    if ((et & 31) == 0) red[et >> 5] = ss;
+    epi_bar();
+    const float inv = rsqrtf((red[0] + red[1] + red[2] + red[3]) / (float)d + J.eps);
+    for (int c = et * 4; c < d; c += 512) {
+      float4 v = *reinterpret_cast<const float4*>(xr + c);           // this thread's own stores above
+      const uint2 gr = *reinterpret_cast<const uint2*>(J.gain + c);
+      const __nv_bfloat162 g0 = *reinterpret_cast<const __nv_bfloat162*>(&gr.x), g1 = *reinterpret_cast<const __nv_bfloat162*>(&gr.y);
+      v.x *= inv * __low2float(g0); v.y *= inv * __high2float(g0); v.z *= inv * __low2float(g1); v.w *= inv * __high2float(g1);
+      if (J.out) store_hl4(J.out + (size_t)r * d + c, J.out_ps, v);
+      if (J.hn) *reinterpret_cast<float4*>(J.hn + (size_t)r * d + c) = v;
+    }
+  }
+}
+
+#define CHAIN_GIVE_UP(site, jj, ii) do { atomicOr(a.status, ST_TIMEOUT); \
+    if (a.diag && atomicCAS(a.diag, 0, (site)) == 0) { a.diag[1] = blockIdx.x; a.diag[2] = (ii); a.diag[3] = (jj); \
+      a.diag[4] = gridDim.x; a.diag[5] = a.m; a.diag[6] = a.job[jj].n; a.diag[7] = a.job[jj].kb; } } while (0)
+
+template <int MT>
+__global__ void __launch_bounds__(192, 1) gemm_chain_kernel(const __grid_constant__ ChainArgs a) {
+  using C = TileCfg<MT, 200>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = tiles + C::STAGES * C::STAGE_BYTES;
+  auto fullw_bar = [&](int s) { return bars + 8u * s; };
+  auto fullx_bar = [&](int s) { return bars + 8u * (C::STAGES + s); };
+  auto empty_bar = [&](int s) { return bars + 8u * (2 * C::STAGES + s); };
+  auto accfull_bar = [&](int i) { return bars + 8u * (3 * C::STAGES + i); };
+  auto accempty_bar = [&](int i) { return bars + 8u * (3 * C::STAGES + 2 + i); };
+  const uint32_t tmem_slot = bars + 8u * (3 * C::STAGES + 4);
+  __shared__ int s_abort, s_flag;
+  __shared__ float s_red[4];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = gridDim.x;
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(fullw_bar(s), 1); mbar_init(fullx_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(accfull_bar(i), 1); mbar_init(accempty_bar(i), 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    for (int j = 0; j < a.n_jobs; ++j) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&a.tmW[j]) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&a.tmX[j]) : "memory");
+    }
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  grid_dep_launch();
+  uint32_t tmem_base;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+  const bool cat = C::CAT && a.job[0].x_lo_rows != 0;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      int ws = 0; uint32_t wph = 1;                      // ring stage and empty-barrier parity of the next weight tile (all jobs)
+      bool ok = true;
+      for (int j = 0; j < a.n_jobs && ok; ++j) {
+        const ChainJob& J = a.job[j];
+        const CUtensorMap* tw = &a.tmW[j];
+        const CUtensorMap* tx = &a.tmX[j];
+        const int kb = J.kb, n_tiles = J.n_tiles, lo_rows = J.x_lo_rows;
+        const int ub = blockIdx.x * J.q, nu = max(min(ub + J.q, J.total_units) - ub, 0);
+        const int pre = nu < C::STAGES ? nu : C::STAGES;
+        // (k-block, weight-tile row, activation-tile row) of the next weight / activation load, advanced without divisions
+        int wk = 0, wn = 0, xk = 0, xn = 0, xm = 0, xs = ws;
+        if (nu > 0) {
+          const int tile = ub / kb;
+          wk = xk = (ub - tile * kb) * BLOCK_K;
+          wn = xn = (tile % n_tiles) * BLOCK_N;
+          xm = (tile / n_tiles) * MT;
+        }
+        const int kend = kb * BLOCK_K, nend = n_tiles * BLOCK_N;
+        auto issue_w = [&](int i) {
+          if (!mbar_wait(empty_bar(ws), wph)) { CHAIN_GIVE_UP(1, j, i); return false; }
+          mbar_arrive_expect_tx(fullw_bar(ws), A_BYTES);
+          tma_load_2d(tiles + ws * C::STAGE_BYTES, tw, wk, wn, fullw_bar(ws), pol_w);
+          if (++ws == C::STAGES) { ws = 0; wph ^= 1u; }
+          if ((wk += BLOCK_K) == kend) { wk = 0; if ((wn += BLOCK_N) == nend) wn = 0; }
+          return true;
+        };
+        for (int i = 0; i < pre && ok; ++i) ok = issue_w(i);       // weights first: they wait for nothing but ring space
+        if (!ok) break;
+        if (j == 0) grid_dep_wait();                     // the first job's activations are the preceding kernel's output
+        else {
+          if (!spin_until(a.sync + 8 + j, G)) { CHAIN_GIVE_UP(6, j, 0); ok = false; break; }
+          fence_async_proxy();                           // the rows were written with ordinary stores, TMA reads them
+        }
+        const uint32_t x_bytes = lo_rows ? C::B_BYTES : C::B_PLANE;
+        for (int i = 0; i < nu; ++i) {
+          if (i >= pre && !(ok = issue_w(i))) break;
+          const uint32_t b_dst = tiles + xs * C::STAGE_BYTES + A_BYTES;
+          mbar_arrive_expect_tx(fullx_bar(xs), x_bytes);
+          tma_load_2d(b_dst, tx, xk, xm, fullx_bar(xs), pol_x);
+          if (lo_rows) tma_load_2d(b_dst + C::B_PLANE, tx, xk, lo_rows + xm, fullx_bar(xs), pol_x);
+          if (++xs == C::STAGES) xs = 0;
+          if ((xk += BLOCK_K) == kend) { xk = 0; if ((xn += BLOCK_N) == nend) { xn = 0; xm += MT; } }
+        }
+      }
+      if (!ok) s_abort = 1;
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = cat ? instr_desc(2 * MT) : instr_desc(MT);
+      int seg = 0, st_ = 0;
+      uint32_t ph = 0;                                   // ring stage and full-barrier parity of the next unit (all jobs)
+      bool ok = true;
+      for (int j = 0; j < a.n_jobs && ok; ++j) {
+        const ChainJob& J = a.job[j];
+        const int kb = J.kb;
+        const bool two_pass = J.x_lo_rows && !cat;
+        const int ub = blockIdx.x * J.q, ue = min(ub + J.q, J.total_units), nu = max(ue - ub, 0);
+        int seg_len = nu > 0 ? min((ub / kb + 1) * kb, ue) - ub : 0;       // the first segment: the tail of a tile
+        for (int i = 0; i < nu && ok;) {
+          const int acc = seg & 1;
+          if (!mbar_wait(accempty_bar(acc), ((seg >> 1) & 1) ^ 1u)) { CHAIN_GIVE_UP(2, j, i); ok = false; break; }
+          tc_fence_after();
+          const uint32_t tmem_d = tmem_base + (uint32_t)(acc * C::ACC_COLS);
+          for (int k2 = 0; k2 < seg_len; ++k2, ++i) {
+            if (!mbar_wait(fullw_bar(st_), ph)) { CHAIN_GIVE_UP(3, j, i); ok = false; break; }
+            if (!mbar_wait(fullx_bar(st_), ph)) { CHAIN_GIVE_UP(4, j, i); ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = tiles + st_ * C::STAGE_BYTES;
+            const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+            for (int k = 0; k < BLOCK_K / 16; ++k) umma_bf16(tmem_d, adesc + 2u * k, bdesc + 2u * k, idesc, (uint32_t)((k2 | k) != 0));
+            if (two_pass) {
+              const uint64_t ldesc = smem_desc_sw128(a_addr + A_BYTES + C::B_PLANE);
+#pragma unroll
+              for (int k = 0; k < BLOCK_K / 16; ++k) umma_bf16(tmem_d, adesc + 2u * k, ldesc + 2u * k, idesc, 1u);
+            }
+            umma_commit(empty_bar(st_));
+            if (++st_ == C::STAGES) { st_ = 0; ph ^= 1u; }
+          }
+          if (!ok) break;
+          umma_commit(accfull_bar(acc));
+          ++seg;
+          seg_len = min(kb, nu - i);                     // every later segment starts a tile
+        }
+      }
+      if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int et = quarter * 32 + lane;
+    grid_dep_wait();
+    int seg = 0;
+    bool ok = true;
+    for (int j = 0; j < a.n_jobs && ok; ++j) {
+      const ChainJob& J = a.job[j];
+      const int ub = blockIdx.x * J.q, ue = min(ub + J.q, J.total_units), nu = max(ue - ub, 0);
+      for (int i = 0; i < nu;) {
+        const int u = ub + i, tile = u / J.kb;
+        const int seg_len = min((tile + 1) * J.kb, ue) - u;
+        const int acc = seg & 1;
+        if (!mbar_wait(accfull_bar(acc), (seg >> 1) & 1)) { if (lane == 0) CHAIN_GIVE_UP(5, j, i); ok = false; break; }
+        tc_fence_after();
+        const int slot = blockIdx.x - (int)(((long long)tile * J.kb) / J.q);
+        const int n0 = (tile % J.n_tiles) * BLOCK_N, m0 = (tile / J.n_tiles) * MT;
+        float* dst = a.part + (size_t)slot * J.slot_stride + n0 + et;
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * C::ACC_COLS);
+        store_accumulator<MT>(taddr, cat, dst, m0, a.m, J.n);
+        tc_fence_before();
+        if (lane == 0) mbar_arrive(accempty_bar(acc));
+        i += seg_len;
+        ++seg;
+      }
+      if (!ok || J.op == CHAIN_NONE) continue;
+      // every CTA's partial sums of this job in memory -> this CTA's share of the row-wise step -> next job's rows ready
+      __threadfence();
+      epi_bar();
+      if (et == 0) {
+        atomicAdd(a.sync + j, 1);
+        s_flag = spin_until(a.sync + j, G) ? 1 : 0;
+        if (!s_flag) CHAIN_GIVE_UP(7, j, 0);
+      }
+      epi_bar();
+      if (!s_flag) { ok = false; break; }
+      const SplitDesc sd{J.q, J.kb, J.n_tiles, MT, J.slot_stride};
+      if (J.op == CHAIN_SILU_MUL) chain_silu_mul(a, J, sd, et);
+      else chain_resid_norm(a, J, sd, et, s_red);
+      __threadfence();
+      fence_async_proxy();
+      epi_bar();
+      if (et == 0) atomicAdd(a.sync + 8 + j + 1, 1);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (s_abort) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(100);
+  }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, C::TMEM_COLS); }
+  if (threadIdx.x == 0) {                                // the last CTA out clears the counters for the next launch
+    __threadfence();
+    if (atomicAdd(a.sync + 16, 1) == G - 1) {
+      for (int k = 0; k <= 16; ++k) a.sync[k] = 0;
+      __threadfence();
+    }
+  }
 }
 
 // ---- tensor maps -------------------------------------------------------------------------------
@@ -415,6 +793,27 @@ hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs
   return launch_b<MT, 100>(tw, tx, a, grid, st);
 }
 
+template <int MT>
+hydra_status launch_chain(const ChainArgs& a, int grid, cudaStream_t st) {
+  using C = TileCfg<MT, 200>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    HYDRA_CUDA(cudaFuncSetAttribute(gemm_chain_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    attr_done = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = C::SMEM_BYTES; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeCooperative;           // all CTAs resident at once: the grid-wide counters need it
+  attr[0].val.cooperative = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, gemm_chain_kernel<MT>, a));
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
 }  // namespace
 
 bool gemm_tc_available() { return encode_fn() != nullptr; }
@@ -469,6 +868,43 @@ hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* 
     case 64: return launch<64>(tw, tx, a, grid, st);
     case 128: return launch<128>(tw, tx, a, grid, st);
     default: return launch<256>(tw, tx, a, grid, st);
+  }
+}
+
+hydra_status gemm_chain(const ChainStep* steps, int n_steps, int m, int x_planes, float* part, size_t part_floats, SplitDesc* last_sd,
+                        int* status, int* diag, int* sync, cudaStream_t st) {
+  if (n_steps < 1 || n_steps > MAX_JOBS || m <= 0 || (x_planes != 1 && x_planes != 2)) return HYDRA_ERR_UNSUPPORTED;
+  ChainArgs a{};
+  a.part = part; a.m = m; a.n_jobs = n_steps; a.status = status; a.diag = diag; a.sync = sync;
+  const int mt = gemm_tile_rows(m);
+  for (int j = 0; j < n_steps; ++j) {
+    const ChainStep& s = steps[j];
+    if (s.n <= 0 || s.k <= 0 || s.n % BLOCK_N || s.k % BLOCK_K) return HYDRA_ERR_UNSUPPORTED;
+    if (((uintptr_t)s.x | (uintptr_t)s.w) & 15) return HYDRA_ERR_INVALID;
+    if (s.op != CHAIN_NONE && (s.cols & 3)) return HYDRA_ERR_UNSUPPORTED;
+    if (s.op == CHAIN_NONE && j + 1 < n_steps) return HYDRA_ERR_INVALID;       // only the last job may leave raw partial sums
+    int slots = 1;
+    const SplitDesc sd = gemm_tc_plan(m, s.n, s.k, nullptr, &slots);
+    if ((size_t)slots * m * s.n > part_floats) return HYDRA_ERR_CAPACITY;
+    const int rows_alloc = s.x_rows_alloc < m ? m : s.x_rows_alloc;
+    if (!get_tensor_map(s.w, (uint64_t)s.n, (uint64_t)s.k, BLOCK_N, &a.tmW[j]) ||
+        !get_tensor_map(s.x, (uint64_t)rows_alloc * x_planes, (uint64_t)s.k, (uint32_t)mt, &a.tmX[j])) {
+      set_last_error("cuTensorMapEncodeTiled", cudaErrorUnknown);
+      return HYDRA_ERR_CUDA;
+    }
+    ChainJob& J = a.job[j];
+    J.n = s.n; J.kb = sd.kb; J.n_tiles = sd.n_tiles; J.total_units = sd.n_tiles * ((m + mt - 1) / mt) * sd.kb; J.q = sd.q;
+    J.x_lo_rows = x_planes == 2 ? rows_alloc : 0; J.op = s.op; J.cols = s.cols; J.slot_stride = sd.stride;
+    J.resid = s.resid; J.gain = s.gain; J.out = s.out; J.out_ps = s.out_ps; J.hn = s.hn; J.eps = s.eps;
+    if (j + 1 == n_steps && last_sd) *last_sd = sd;
+  }
+  const int grid = sm_count();
+  switch (mt) {
+    case 16: return launch_chain<16>(a, grid, st);
+    case 32: return launch_chain<32>(a, grid, st);
+    case 64: return launch_chain<64>(a, grid, st);
+    case 128: return launch_chain<128>(a, grid, st);
+    default: return launch_chain<256>(a, grid, st);
   }
 }
 

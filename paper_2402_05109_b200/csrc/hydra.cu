@@ -183,7 +183,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   std::vector<int*> lvl;
   for (auto& lv : t.level_parents) lvl.push_back(b.take<int>(lv.size()));
   auto* len = b.take<int>(m.max_batch); auto* n_new = b.take<int>(m.max_batch); auto* root = b.take<int>(m.max_batch);
-  auto* status = b.take<int>(16);          // [0] status word, [8..15] where a bounded wait gave up
+  auto* status = b.take<int>(64);          // [0] status word, [8..15] where a bounded wait gave up, [32..48] the GEMM chain's counters
   auto* pos0 = b.take<int>(m.max_batch); auto* nrows = b.take<int>(m.max_batch);
   auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
   auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
@@ -233,7 +233,7 @@ hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void*
                       cudaStream_t st) {
   // algorithmic bytes of the launch: the weight matrix and the activation slab read once, the output written once
   TimeScope ts(c, HYDRA_TIME_GEMM, (double)c->esize * ((double)n * k + (double)c->planes * m * k) + 4.0 * m * n, st);
-  if (c->m.dtype == 1 && c->gemm_mode == 0) {
+  if (c->m.dtype == 1 && c->gemm_mode != 1) {
     int slots = 1;
     gemm_tc_plan(m, n, k, nullptr, &slots);
     if ((size_t)slots * m * n > c->part_floats) return HYDRA_ERR_CAPACITY;
@@ -247,42 +247,73 @@ hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void*
 size_t ps(const hydra_ctx* c, int rows_alloc, size_t cols) { return c->planes == 2 ? (size_t)rows_alloc * cols : 0; }
 size_t kv_ps(const hydra_ctx* c) { return c->planes == 2 ? kv_layer_elems(c->m) : 0; }
 
-// One decoder layer over the rows of `rs`.  Expects the residual rows in c->x and their normed copy in c->xn.
-// Leaves the updated residual in c->x; when next_gain is given also xn = rmsnorm(x)*next_gain (and hn in float).
-hydra_status run_layer(hydra_ctx* c, const LayerW& w, char* kc, char* vc, const RowSet& rs, int len_upper,
-                       const void* next_gain, float* hn, cudaStream_t st) {
+// RoPE + KV append + tree attention of one layer from the QKV partial sums (*sd) in c->part; result in c->attn_out.
+hydra_status attention_block(hydra_ctx* c, char* kc, char* vc, const RowSet& rs, int len_upper, const SplitDesc& sd, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
-  const int rows = rs.batch * rs.tc, d = m.d_model, f = m.d_ffn, dt = m.dtype;
-  SplitDesc sd;
-  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.wqkv, rows, 3 * d, d, &sd, st));
+  const int d = m.d_model, dt = m.dtype;
   HYDRA_TRY(qkv_rope_store(c->part, sd, c->rope, c->q, ps(c, c->R, d), kc, vc, kv_ps(c), rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
-  {
-    TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
-    HYDRA_TRY(tree_attention(c->q, ps(c, c->R, d), kc, vc, kv_ps(c), rs, c->attn_out, ps(c, c->R, d), c->att_scratch, m.n_heads, m.head_dim,
-                             m.max_seq, len_upper, dt, st));
+  TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
+  return tree_attention(c->q, ps(c, c->R, d), kc, vc, kv_ps(c), rs, c->attn_out, ps(c, c->R, d), c->att_scratch, m.n_heads, m.head_dim,
+                        m.max_seq, len_upper, dt, st);
+}
+
+double gemm_bytes(const hydra_ctx* c, int m, int n, int k) {        // weights + activation slab read once, output written once
+  return (double)c->esize * ((double)n * k + (double)c->planes * m * k) + 4.0 * m * n;
+}
+
+// The rest of a layer after its attention: O projection, + residual, RMSNorm, gate/up, SiLU * up, down, + residual and,
+// when next_gain is given, xn = rmsnorm(x) * next_gain (hn: the same in float); when next_w is given, also the
+// GEMM xn @ next_w^T (the next layer's QKV projection, or the LM head), whose partial sums stay in c->part (*sd).
+// Kernel by kernel, or (GEMM mode 2, bfloat16) all of it as ONE persistent kernel (gemm_chain).
+hydra_status mlp_block(hydra_ctx* c, const LayerW& w, int rows, const void* next_gain, float* hn, const void* next_w, int next_n,
+                       SplitDesc* sd, cudaStream_t st) {
+  const hydra_model_cfg& m = c->m;
+  const int d = m.d_model, f = m.d_ffn, dt = m.dtype;
+  if (dt == 1 && c->gemm_mode == 2) {
+    ChainStep steps[4] = {};
+    steps[0] = ChainStep{(const bf16*)c->attn_out, c->R, (const bf16*)w.wo, d, d, CHAIN_RESID_NORM, d, c->x, (const bf16*)w.ffn_norm,
+                         (bf16*)c->xn, ps(c, c->R, d), nullptr, m.rms_eps};
+    steps[1] = ChainStep{(const bf16*)c->xn, c->R, (const bf16*)w.w_gate_up, 2 * f, d, CHAIN_SILU_MUL, f, nullptr, nullptr,
+                         (bf16*)c->act, ps(c, c->R, f), nullptr, 0.f};
+    steps[2] = ChainStep{(const bf16*)c->act, c->R, (const bf16*)w.w_down, d, f, CHAIN_RESID_NORM, d, c->x, (const bf16*)next_gain,
+                         next_gain ? (bf16*)c->xn : nullptr, ps(c, c->R, d), hn, m.rms_eps};
+    int n = 3;
+    double bytes = gemm_bytes(c, rows, d, d) + gemm_bytes(c, rows, 2 * f, d) + gemm_bytes(c, rows, d, f);
+    if (next_w) {
+      steps[n++] = ChainStep{(const bf16*)c->xn, c->R, (const bf16*)next_w, next_n, d, CHAIN_NONE, 0, nullptr, nullptr, nullptr, 0, nullptr, 0.f};
+      bytes += gemm_bytes(c, rows, next_n, d);
+    }
+    TimeScope ts(c, HYDRA_TIME_GEMM, bytes, st);
+    return gemm_chain(steps, n, rows, c->planes, c->part, c->part_floats, sd, c->d_status, c->d_status + 8, c->d_status + 32, st);
   }
-  HYDRA_TRY(run_gemm(c, c->attn_out, c->R, w.wo, rows, d, d, &sd, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, c->part, sd, c->x, w.ffn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, dt, st));
-  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, &sd, st));
-  HYDRA_TRY(silu_mul(c->part, sd, c->act, ps(c, c->R, f), rows, f, dt, st));
-  HYDRA_TRY(run_gemm(c, c->act, c->R, w.w_down, rows, d, f, &sd, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, c->part, sd, c->x, next_gain, next_gain ? c->xn : nullptr, ps(c, c->R, d), hn, rows, d, m.rms_eps, dt, st));
+  SplitDesc s1;
+  HYDRA_TRY(run_gemm(c, c->attn_out, c->R, w.wo, rows, d, d, &s1, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, c->part, s1, c->x, w.ffn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, dt, st));
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, w.w_gate_up, rows, 2 * f, d, &s1, st));
+  HYDRA_TRY(silu_mul(c->part, s1, c->act, ps(c, c->R, f), rows, f, dt, st));
+  HYDRA_TRY(run_gemm(c, c->act, c->R, w.w_down, rows, d, f, &s1, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, c->part, s1, c->x, next_gain, next_gain ? c->xn : nullptr, ps(c, c->R, d), hn, rows, d, m.rms_eps, dt, st));
+  if (next_w) HYDRA_TRY(run_gemm(c, c->xn, c->R, next_w, rows, next_n, d, sd, st));
   return HYDRA_OK;
 }
 
 // Base model over the rows of `rs` whose tokens are tok[rows]: leaves post-final-norm hidden rows in c->h_tree
-// (float) and c->xn (operand type).
-hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_upper, cudaStream_t st) {
+// (float) and c->xn (operand type); with tail_w also the partial sums of xn @ tail_w^T (the LM head) in c->part (*tail_sd).
+hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_upper, const void* tail_w, int tail_n, SplitDesc* tail_sd,
+                      cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
-  const int rows = rs.batch * rs.tc;
+  const int rows = rs.batch * rs.tc, d = m.d_model;
   const size_t kvl = kv_layer_elems(m) * c->esize * c->planes;      // bytes of one layer's K (or V) cache, all planes
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
-  HYDRA_TRY(embed_rows(c->embed, tok, c->x, rows, m.d_model, m.vocab, m.dtype, c->d_status, st));
-  HYDRA_TRY(residual_rmsnorm(c->x, nullptr, single_slot(0), c->x, c->layers[0].attn_norm, c->xn, ps(c, c->R, m.d_model), nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
+  HYDRA_TRY(embed_rows(c->embed, tok, c->x, rows, d, m.vocab, m.dtype, c->d_status, st));
+  HYDRA_TRY(residual_rmsnorm(c->x, nullptr, single_slot(0), c->x, c->layers[0].attn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, m.dtype, st));
+  SplitDesc sd;
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, c->layers[0].wqkv, rows, 3 * d, d, &sd, st));
   for (int l = 0; l < m.n_layers; ++l) {
-    bool last = l + 1 == m.n_layers;
-    HYDRA_TRY(run_layer(c, c->layers[l], c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs, len_upper,
-                        last ? c->final_norm : c->layers[l + 1].attn_norm, last ? c->h_tree : nullptr, st));
+    const bool last = l + 1 == m.n_layers;
+    HYDRA_TRY(attention_block(c, c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs, len_upper, sd, st));
+    HYDRA_TRY(mlp_block(c, c->layers[l], rows, last ? c->final_norm : c->layers[l + 1].attn_norm, last ? c->h_tree : nullptr,
+                        last ? tail_w : c->layers[l + 1].wqkv, last ? tail_n : 3 * d, last ? tail_sd : &sd, st));
   }
   return HYDRA_OK;
 }
@@ -290,11 +321,14 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
 // Prefix-attention layer over rows whose input (post-final-norm hidden) is `src` laid out like rs.
 hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int len_upper, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
-  const int rows = rs.batch * rs.tc;
+  const int rows = rs.batch * rs.tc, d = m.d_model;
   const size_t kvl = kv_layer_elems(m) * c->esize * c->planes;      // bytes of one layer's K (or V) cache, all planes
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
-  HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, ps(c, c->R, m.d_model), nullptr, rows, m.d_model, m.rms_eps, m.dtype, st));
-  return run_layer(c, c->pfx, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, nullptr, nullptr, st);
+  HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, m.dtype, st));
+  SplitDesc sd;
+  HYDRA_TRY(run_gemm(c, c->xn, c->R, c->pfx.wqkv, rows, 3 * d, d, &sd, st));
+  HYDRA_TRY(attention_block(c, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, sd, st));
+  return mlp_block(c, c->pfx, rows, nullptr, nullptr, nullptr, 0, nullptr, st);
 }
 
 int max_len_ub(const hydra_ctx* c) { int v = 0; for (int b = 0; b < c->batch; ++b) v = std::max(v, c->len_ub[b]); return v; }
@@ -342,9 +376,8 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
   const hydra_model_cfg& m = c->m;
   const int rows = c->batch * c->T;
   RowSet rs{c->batch, c->T, nullptr, c->d_len, c->d_depth, c->d_anc};
-  HYDRA_TRY(run_base(c, tree_tok, rs, len_bucket(c, max_len_ub(c) + c->T), st));
   SplitDesc sd;
-  HYDRA_TRY(run_gemm(c, c->xn, c->R, c->lm_head, rows, m.vocab, m.d_model, &sd, st));
+  HYDRA_TRY(run_base(c, tree_tok, rs, len_bucket(c, max_len_ub(c) + c->T), c->lm_head, m.vocab, &sd, st));
   return argmax_rows(c->part, sd, logits, amax, c->topk_scratch, c->topk_rows_cap, rows, m.vocab, st);
 }
 
@@ -494,7 +527,7 @@ hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const
   for (int ch = 0; ch < nchunks; ++ch) {
     HYDRA_TRY(set_chunk(c->d_prompt_len, ch, CHUNK, c->d_pos0, c->d_nrows, batch, st));
     HYDRA_TRY(gather_chunk_tokens(tokens, c->d_offsets, ch, CHUNK, c->d_tok, batch, st));
-    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * CHUNK, st));
+    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * CHUNK, nullptr, 0, nullptr, st));
     HYDRA_TRY(capture_last(c->h_tree, c->d_prompt_len, ch, CHUNK, c->h_new, c->h.n_heads + 1, c->d_n_new, c->d_len, batch, m.d_model, st));
     if (c->h.prefix_attn) HYDRA_TRY(run_prefix(c, c->h_tree, rs, (ch + 1) * CHUNK, st));
   }
@@ -622,7 +655,7 @@ hydra_status hydra_poll_status(hydra_ctx* c, void* stream) {
     cudaMemcpy(d, c->d_status + 8, sizeof(d), cudaMemcpyDeviceToHost);
     snprintf(g_err, sizeof(g_err), "GEMM wait gave up: site %d cta %d unit %d/%d grid %d m %d n %d kb %d", d[0], d[1], d[2], d[3], d[4], d[5], d[6], d[7]);
   }
-  if (word) HYDRA_CUDA(cudaMemset(c->d_status, 0, 16 * sizeof(int)));
+  if (word) HYDRA_CUDA(cudaMemset(c->d_status, 0, 64 * sizeof(int)));
   if (word & ST_TIMEOUT) return HYDRA_ERR_TIMEOUT;
   if (word & ST_BOUNDS) return HYDRA_ERR_BOUNDS;
   return HYDRA_OK;
@@ -656,7 +689,7 @@ hydra_status hydra_get_timing(hydra_ctx* c, int kclass, double* ms_total, long l
 }
 
 hydra_status hydra_set_gemm_mode(hydra_ctx* c, int mode) {
-  if (!c || (mode != 0 && mode != 1)) return HYDRA_ERR_INVALID;
+  if (!c || mode < 0 || mode > 2) return HYDRA_ERR_INVALID;
   c->gemm_mode = mode;
   drop_graphs(c);
   return HYDRA_OK;

@@ -43,9 +43,9 @@ def test_small_bf16_hydrapp_ragged_batch():
     assert seen >= {0, 1, 2, 3, 4}, seen
 
 
-@pytest.mark.parametrize("mode", [1])
+@pytest.mark.parametrize("mode", [1, 2])
 def test_small_bf16_other_gemm_modes_and_root_only_tree(mode):
-    """mode 1: the SIMT GEMM (reads only the hi plane of the activations)."""
+    """mode 1: the SIMT GEMM (reads only the hi plane of the activations); mode 2: one persistent kernel per layer tail."""
     from paper_2402_05109_b200 import Hydra
     m = ModelCfg(2, 256, 4, 64, 512, 1024, dtype="bf16")
     h = HeadCfg(2, 1, False)
@@ -123,3 +123,20 @@ def test_step_graph_replay_matches_kernel_by_kernel_launches():
         assert g.launch_count() > 100 * 50
         g.close()
     assert torch.equal(outs[0], outs[1])
+
+
+def test_small_bf16_hydra_pp_gemm_chain_mode():
+    """GEMM mode 2 (layer tail as one persistent kernel with grid-wide hand-overs) against the oracle: prefix layer,
+    63-node tree, ragged batch of 3, graph replay from the second step on."""
+    from paper_2402_05109_b200 import Hydra
+    m = ModelCfg(3, 256, 2, 128, 512, 1024, dtype="bf16")
+    h = HeadCfg(4, 2, True)
+    parent = load_tree("tree63_d4")
+    w = make_weights(m, h, 11)
+    prompts = make_prompts(11, [37, 130, 64], m.vocab)
+    o = HydraOracle(m, h, parent, w, 256, cache_weights=True)
+    g = Hydra(m, h, parent, {k: v.cuda() for k, v in w.items()}, 3, 256)
+    g.set_gemm_mode(2)
+    st = lockstep(o, g, prompts, 4, 11)
+    assert st.steps == 4
+    g.close()
