@@ -61,6 +61,29 @@ __host__ __device__ __forceinline__ int split_count(const SplitDesc& sd, int m, 
   const int u0 = ((m / sd.mt) * sd.n_tiles + (n >> 7)) * sd.kb;        // tiles * kb stays far below 2^31
   return (u0 + sd.kb - 1) / sd.q - u0 / sd.q + 1;
 }
+// acc[u] = sum over the ns[u] slots of the four floats at element offset off[u] of a slot (all loads of a round in flight together)
+template <int U>
+__device__ __forceinline__ void sum_slots_multi(const float* part, size_t stride, const size_t (&off)[U], const int (&ns)[U], float4 (&acc)[U]) {
+  constexpr int PMAX = 6;
+  int mx = 0;
+#pragma unroll
+  for (int u = 0; u < U; ++u) { acc[u] = make_float4(0.f, 0.f, 0.f, 0.f); mx = max(mx, ns[u]); }
+#pragma unroll
+  for (int p = 0; p < PMAX; ++p) {
+    float4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = p < ns[u] ? __ldcg(reinterpret_cast<const float4*>(part + p * stride + off[u])) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < U; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
+  }
+  for (int p = PMAX; p < mx; ++p)
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (p < ns[u]) {
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(part + p * stride + off[u]));
+        acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
+      }
+}
 inline SplitDesc single_slot(size_t stride) { return SplitDesc{1, 1, 1, 1 << 30, stride}; }
 
 // Launch with programmatic stream serialisation allowed (see pdl_wait).

@@ -421,29 +421,6 @@ __device__ __forceinline__ bool spin_until(const int* p, int target) {
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// acc[u] = sum over the ns[u] slots of the four floats at element offset off[u] of a slot (all loads of a round in flight together)
-template <int U>
-__device__ __forceinline__ void sum_slots_multi(const float* part, size_t stride, const size_t (&off)[U], const int (&ns)[U], float4 (&acc)[U]) {
-  constexpr int PMAX = 6;
-  int mx = 0;
-#pragma unroll
-  for (int u = 0; u < U; ++u) { acc[u] = make_float4(0.f, 0.f, 0.f, 0.f); mx = max(mx, ns[u]); }
-#pragma unroll
-  for (int p = 0; p < PMAX; ++p) {
-    float4 v[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) v[u] = p < ns[u] ? __ldcg(reinterpret_cast<const float4*>(part + p * stride + off[u])) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int u = 0; u < U; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
-  }
-  for (int p = PMAX; p < mx; ++p)
-#pragma unroll
-    for (int u = 0; u < U; ++u)
-      if (p < ns[u]) {
-        const float4 v = __ldcg(reinterpret_cast<const float4*>(part + p * stride + off[u]));
-        acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
-      }
-}
 __device__ __forceinline__ void store_hl4(bf16* dst, size_t lo_off, const float4& v) {
   const __nv_bfloat162 h0 = __floats2bfloat162_rn(v.x, v.y), h1 = __floats2bfloat162_rn(v.z, v.w);
   *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));

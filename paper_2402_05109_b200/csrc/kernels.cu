@@ -157,17 +157,26 @@ __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const fl
   __shared__ float sh[32];
   const size_t base = (size_t)blockIdx.x * d;
   float ss = 0.f;
-  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
-    float4 v = res ? *reinterpret_cast<const float4*>(res + base + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-    if (part) {
-      const int ns = split_count(sd, (int)blockIdx.x, i);
-      for (int p = 0; p < ns; ++p) {
-        float4 a = *reinterpret_cast<const float4*>(part + p * sd.stride + base + i);
-        v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+  for (int i0 = threadIdx.x * 4; i0 < d; i0 += NORM_THREADS * 4 * 2) {       // two pieces per round, all their slot loads in flight together
+    size_t off[2]; int ns[2]; float4 acc[2], v[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = i0 + u * NORM_THREADS * 4;
+      const bool valid = i < d;
+      off[u] = base + (valid ? i : 0);
+      ns[u] = valid && part ? split_count(sd, (int)blockIdx.x, i) : 0;
+      v[u] = valid && res ? *reinterpret_cast<const float4*>(res + base + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    sum_slots_multi<2>(part, sd.stride, off, ns, acc);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = i0 + u * NORM_THREADS * 4;
+      if (i < d) {
+        v[u].x += acc[u].x; v[u].y += acc[u].y; v[u].z += acc[u].z; v[u].w += acc[u].w;
+        *reinterpret_cast<float4*>(x_out + base + i) = v[u];
+        ss += v[u].x * v[u].x + v[u].y * v[u].y + v[u].z * v[u].z + v[u].w * v[u].w;
       }
     }
-    *reinterpret_cast<float4*>(x_out + base + i) = v;
-    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   if (!gain) return;
   float tot = block_sum(ss, sh);
@@ -235,19 +244,14 @@ __global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __rest
   const int h = blockIdx.y * (256 / tph) + threadIdx.x / tph;
   if (h >= H) return;
   const int j = (threadIdx.x % tph) * 4;
-  const float* p0 = part + (size_t)r * 3 * d;
   const int c0 = h * hd + j, c1 = c0 + half;
   const int cols[6] = {c0, c1, d + c0, d + c1, 2 * d + c0, 2 * d + c1};
   float4 v6[6];
+  {
+    size_t off[6]; int ns[6];
 #pragma unroll
-  for (int e = 0; e < 6; ++e) {
-    const int ns = split_count(sd, r, cols[e]);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < ns; ++s) {
-      const float4 a = *reinterpret_cast<const float4*>(p0 + s * sd.stride + cols[e]);
-      acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
-    }
-    v6[e] = acc;
+    for (int e = 0; e < 6; ++e) { off[e] = (size_t)r * 3 * d + cols[e]; ns[e] = split_count(sd, r, cols[e]); }
+    sum_slots_multi<6>(part, sd.stride, off, ns, v6);
   }
   const float4 t01 = *reinterpret_cast<const float4*>(table + (size_t)r * half + j);        // (cos, sin) of j, j+1
   const float4 t23 = *reinterpret_cast<const float4*>(table + (size_t)r * half + j + 2);    // (cos, sin) of j+2, j+3
@@ -463,11 +467,11 @@ __global__ void silu_mul_kernel(const float* __restrict__ part, SplitDesc sd, T*
   size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= (size_t)rows * f) return;
   const int r = (int)(i / f), c = (int)(i % f);
-  const float* p = part + (size_t)r * 2 * f;
-  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
-  const int ng = split_count(sd, r, c), nu = split_count(sd, r, f + c);
-  for (int s = 0; s < ng; ++s) { float4 a = *reinterpret_cast<const float4*>(p + s * sd.stride + c); g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w; }
-  for (int s = 0; s < nu; ++s) { float4 a = *reinterpret_cast<const float4*>(p + s * sd.stride + f + c); u.x += a.x; u.y += a.y; u.z += a.z; u.w += a.w; }
+  size_t off[2] = {(size_t)r * 2 * f + c, (size_t)r * 2 * f + f + c};
+  int ns[2] = {split_count(sd, r, c), split_count(sd, r, f + c)};
+  float4 gu[2];
+  sum_slots_multi<2>(part, sd.stride, off, ns, gu);
+  const float4 g = gu[0], u = gu[1];
   put4<T>(act + i, act_ps, make_float4(silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w));
 }
 hydra_status silu_mul(const float* part, SplitDesc sd, void* act, size_t act_ps, int rows, int f, int dtype, cudaStream_t st) {
