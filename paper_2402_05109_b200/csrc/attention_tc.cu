@@ -48,7 +48,30 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int HD, bool HL, int TILE, int NS>
+// thread-block cluster helpers (the chunks of one (head, sequence) pair form a cluster along z)
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t peer_smem(uint32_t saddr, uint32_t rank) {     // the same offset in CTA `rank`'s shared memory
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_peer4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 ld_peer2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+
+// CLUSTER: the nchunks (<= 8) CTAs of a (head, sequence) pair are one thread-block cluster; they leave their partial
+// rows in their own shared memory and every CTA merges its share of the rows out of its peers' shared memory
+// (no scratch, no counters).  Otherwise: partial rows in scratch, merged by the CTA that reports in last.
+template <int HD, bool HL, int TILE, int NS, bool CLUSTER>
 __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __restrict__ q, size_t q_ps, const bf16* __restrict__ kc,
                                                                   const bf16* __restrict__ vc, size_t kv_ps, RowSet rs,
                                                                   float* __restrict__ part_o, float* __restrict__ part_ml,
@@ -97,20 +120,20 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
   };
 
   const int ntiles = has_work ? (s1 - s0 + TILE - 1) / TILE : 0;
-  // request the first NS-1 KV tiles (one cp.async group each), then stage Q (rows past nr are zero)
-#pragma unroll
-  for (int i = 0; i < NS - 1; ++i) {
-    if (i < ntiles) load_tile(i, s0 + i * TILE);
-    cp_async_commit();
-  }
+  // request Q (rows past nr are zero) and the first NS-1 KV tiles: one cp.async group per tile, Q rides with the first
   for (int e = tid; has_work && e < 64 * PIECES; e += NWARP * 32) {
     const int r = e / PIECES, pc = e % PIECES;
 #pragma unroll
     for (int pl = 0; pl < NP; ++pl) {
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (r < nr) v = *reinterpret_cast<const uint4*>(q + pl * q_ps + (size_t)(b * rs.tc + r) * d + h * HD + pc * 8);
-      *reinterpret_cast<uint4*>(Qs + (pl * 64 + r) * LDS + pc * 8) = v;
+      bf16* dst = Qs + (pl * 64 + r) * LDS + pc * 8;
+      if (r < nr) cp_async16((uint32_t)__cvta_generic_to_shared(dst), q + pl * q_ps + (size_t)(b * rs.tc + r) * d + h * HD + pc * 8);
+      else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
     }
+  }
+#pragma unroll
+  for (int i = 0; i < NS - 1; ++i) {
+    if (i < ntiles) load_tile(i, s0 + i * TILE);
+    cp_async_commit();
   }
   const int row0 = (warp & 3) * 16, khalf = warp >> 2;
   constexpr int HT = TILE / 2;                           // keys of a tile per warp
@@ -237,6 +260,12 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
     *reinterpret_cast<float4*>(xch + NB * 4) = make_float4(m_a, m_b, l_a, l_b);
   }
   __syncthreads();
+  constexpr int XCH_FLOATS = 4 * 32 * (NB * 4 + 4);     // the hand-over area above
+  float* xo = reinterpret_cast<float*>(KVs) + XCH_FLOATS;    // CLUSTER: this chunk's partial rows [64][HD], then (m, l) [64][2]
+  float* xml = xo + 64 * HD;
+  if (CLUSTER && !warp_active && khalf == 0) {           // rows this CTA has nothing for: weight zero
+    if (t == 0) { *reinterpret_cast<float2*>(xml + ra * 2) = make_float2(-INFINITY, 0.f); *reinterpret_cast<float2*>(xml + rb * 2) = make_float2(-INFINITY, 0.f); }
+  }
   if (khalf == 0 && warp_active) {
     const float4 ml = *reinterpret_cast<const float4*>(xch + NB * 4);
     const float mn_a = fmaxf(m_a, ml.x), mn_b = fmaxf(m_b, ml.y);
@@ -245,15 +274,71 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
     m_a = mn_a; m_b = mn_b;
     l_a = l_a * w0a + ml.z * w1a; l_b = l_b * w0b + ml.w * w1b;
     // partials: o (un-normalised), m (log2 domain), l
-    const size_t idx_a = ((size_t)(b * rs.tc + ra) * H + h) * nchunks + c, idx_b = ((size_t)(b * rs.tc + rb) * H + h) * nchunks + c;
+    if (CLUSTER) {
 #pragma unroll
-    for (int n = 0; n < NB; ++n) {
-      const float4 v = *reinterpret_cast<const float4*>(xch + n * 4);
-      if (ra < nr) __stcg(reinterpret_cast<float2*>(part_o + idx_a * HD + n * 8 + 2 * t), make_float2(o[n][0] * w0a + v.x * w1a, o[n][1] * w0a + v.y * w1a));
-      if (rb < nr) __stcg(reinterpret_cast<float2*>(part_o + idx_b * HD + n * 8 + 2 * t), make_float2(o[n][2] * w0b + v.z * w1b, o[n][3] * w0b + v.w * w1b));
+      for (int n = 0; n < NB; ++n) {
+        const float4 v = *reinterpret_cast<const float4*>(xch + n * 4);
+        *reinterpret_cast<float2*>(xo + ra * HD + n * 8 + 2 * t) = make_float2(o[n][0] * w0a + v.x * w1a, o[n][1] * w0a + v.y * w1a);
+        *reinterpret_cast<float2*>(xo + rb * HD + n * 8 + 2 * t) = make_float2(o[n][2] * w0b + v.z * w1b, o[n][3] * w0b + v.w * w1b);
+      }
+      if (t == 0) {
+        *reinterpret_cast<float2*>(xml + ra * 2) = ra < nr ? make_float2(m_a, l_a) : make_float2(-INFINITY, 0.f);
+        *reinterpret_cast<float2*>(xml + rb * 2) = rb < nr ? make_float2(m_b, l_b) : make_float2(-INFINITY, 0.f);
+      }
+    } else {
+      const size_t idx_a = ((size_t)(b * rs.tc + ra) * H + h) * nchunks + c, idx_b = ((size_t)(b * rs.tc + rb) * H + h) * nchunks + c;
+#pragma unroll
+      for (int n = 0; n < NB; ++n) {
+        const float4 v = *reinterpret_cast<const float4*>(xch + n * 4);
+        if (ra < nr) __stcg(reinterpret_cast<float2*>(part_o + idx_a * HD + n * 8 + 2 * t), make_float2(o[n][0] * w0a + v.x * w1a, o[n][1] * w0a + v.y * w1a));
+        if (rb < nr) __stcg(reinterpret_cast<float2*>(part_o + idx_b * HD + n * 8 + 2 * t), make_float2(o[n][2] * w0b + v.z * w1b, o[n][3] * w0b + v.w * w1b));
+      }
+      if (t == 0 && ra < nr) __stcg(reinterpret_cast<float2*>(part_ml + idx_a * 2), make_float2(m_a, l_a));
+      if (t == 0 && rb < nr) __stcg(reinterpret_cast<float2*>(part_ml + idx_b * 2), make_float2(m_b, l_b));
     }
-    if (t == 0 && ra < nr) __stcg(reinterpret_cast<float2*>(part_ml + idx_a * 2), make_float2(m_a, l_a));
-    if (t == 0 && rb < nr) __stcg(reinterpret_cast<float2*>(part_ml + idx_b * 2), make_float2(m_b, l_b));
+  }
+  if (CLUSTER) {
+    // out[r][h][:] = sum_c o_c 2^(m_c - M) / sum_c l_c 2^(m_c - M), chunks in order; this CTA takes rows c, c + nchunks, ...
+    cluster_sync_all();                                  // every chunk's rows are in its shared memory
+    constexpr int V4 = HD / 4;
+    const uint32_t xo_s = (uint32_t)__cvta_generic_to_shared(xo), xml_s = (uint32_t)__cvta_generic_to_shared(xml);
+    const int my_rows = (rs.tc - c + nchunks - 1) / nchunks;
+    for (int e = tid; e < my_rows * V4; e += NWARP * 32) {
+      const int i = c + (e / V4) * nchunks, k4 = e % V4;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < nr) {
+        float mc[8], lc[8];
+        float M = -INFINITY;
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc) {
+          mc[cc] = -INFINITY; lc[cc] = 0.f;
+          if (cc < nchunks) { const float2 ml = ld_peer2(peer_smem(xml_s + (uint32_t)i * 8u, (uint32_t)cc)); mc[cc] = ml.x; lc[cc] = ml.y; }
+          M = fmaxf(M, mc[cc]);
+        }
+        float L = 0.f;
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc) {
+          if (cc < nchunks && mc[cc] != -INFINITY) {
+            const float w = exp2f(mc[cc] - M);
+            const float4 v = ld_peer4(peer_smem(xo_s + (uint32_t)(i * HD + k4 * 4) * 4u, (uint32_t)cc));
+            L += lc[cc] * w;
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+          }
+        }
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+      }
+      bf16* dst = out + ((size_t)b * rs.tc + i) * d + h * HD + k4 * 4;      // rows past nr get zeros
+      const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x, acc.y), h1 = __floats2bfloat162_rn(acc.z, acc.w);
+      *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+      if (out_ps) {
+        const __nv_bfloat162 l0 = __floats2bfloat162_rn(acc.x - __low2float(h0), acc.y - __high2float(h0));
+        const __nv_bfloat162 l1 = __floats2bfloat162_rn(acc.z - __low2float(h1), acc.w - __high2float(h1));
+        *reinterpret_cast<uint2*>(dst + out_ps) = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+      }
+    }
+    cluster_sync_all();                                  // peers may still be reading this CTA's rows
+    return;
   }
   // The last of the (head, sequence)'s chunks to report in merges them:
   // out[r][h][:] = sum_c o_c 2^(m_c - M) / sum_c l_c 2^(m_c - M) over the chunks that were dealt tiles, in chunk order.
@@ -267,15 +352,32 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // weights first (one (row, chunk) pair per thread), then the rows: every thread owns up to 8 float4 pieces and
-  // walks the chunks with all of its loads of a chunk in flight together
+  // Every thread owns up to PER float4 pieces of the output rows.  The partial rows of the first four chunks are
+  // requested before anything else, so that they travel while the chunk weights are worked out (one (row, chunk)
+  // pair per thread, through shared memory); further chunks follow four at a time.
+  constexpr int V4 = HD / 4, PER = (64 * V4 + NWARP * 32 - 1) / (NWARP * 32), CB = 4;
+  float4 v[CB][PER];
+  auto dealt = [&](int cc) { return chunk_first_tile(cc, nt, nchunks) != chunk_first_tile(cc + 1, nt, nchunks); };   // else it wrote nothing
+  auto load_batch = [&](int c0) {
+#pragma unroll
+    for (int cb = 0; cb < CB; ++cb) {
+      const int cc = c0 + cb;
+      const bool live = cc < nchunks && dealt(cc);
+#pragma unroll
+      for (int j = 0; j < PER; ++j) {
+        const int e = tid + j * NWARP * 32, i = e / V4, k4 = e % V4;
+        v[cb][j] = live && i < nr ? __ldcg(reinterpret_cast<const float4*>(part_o + ((((size_t)b * rs.tc + i) * H + h) * nchunks + cc) * HD + k4 * 4))
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+  };
+  load_batch(0);
   float* sm_m = reinterpret_cast<float*>(KVs);         // [tc][nchunks] chunk maxima, then the normalised chunk weights
   float* sm_l = sm_m + rs.tc * nchunks;
   for (int e = tid; e < rs.tc * nchunks; e += NWARP * 32) {
     const int i = e / nchunks, cc = e % nchunks;
     float2 ml = make_float2(-INFINITY, 0.f);
-    if (i < nr && chunk_first_tile(cc, nt, nchunks) != chunk_first_tile(cc + 1, nt, nchunks))       // else: dealt no tile, wrote nothing
-      ml = __ldcg(reinterpret_cast<const float2*>(part_ml + (((size_t)b * rs.tc + i) * H + h) * nchunks * 2 + cc * 2));
+    if (i < nr && dealt(cc)) ml = __ldcg(reinterpret_cast<const float2*>(part_ml + (((size_t)b * rs.tc + i) * H + h) * nchunks * 2 + cc * 2));
     sm_m[e] = ml.x; sm_l[e] = ml.y;
   }
   __syncthreads();
@@ -292,24 +394,20 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
     for (int cc = 0; cc < nchunks; ++cc) sm_m[i * nchunks + cc] *= inv;
   }
   __syncthreads();
-  constexpr int V4 = HD / 4, PER = (64 * V4 + NWARP * 32 - 1) / (NWARP * 32);
   float4 acc[PER];
 #pragma unroll
   for (int j = 0; j < PER; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int cc = 0; cc < nchunks; ++cc) {
-    float4 v[PER];
+  for (int c0 = 0; c0 < nchunks; c0 += CB) {
+    if (c0 > 0) load_batch(c0);
 #pragma unroll
-    for (int j = 0; j < PER; ++j) {
-      const int e = tid + j * NWARP * 32, i = e / V4, k4 = e % V4;
-      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (i < nr && sm_m[i * nchunks + cc] != 0.f)
-        v[j] = __ldcg(reinterpret_cast<const float4*>(part_o + ((((size_t)b * rs.tc + i) * H + h) * nchunks + cc) * HD + k4 * 4));
-    }
+    for (int cb = 0; cb < CB; ++cb) {
+      const int cc = c0 + cb;
 #pragma unroll
-    for (int j = 0; j < PER; ++j) {
-      const int i = (tid + j * NWARP * 32) / V4;
-      const float w = i < rs.tc ? sm_m[i * nchunks + cc] : 0.f;
-      acc[j].x += v[j].x * w; acc[j].y += v[j].y * w; acc[j].z += v[j].z * w; acc[j].w += v[j].w * w;
+      for (int j = 0; j < PER; ++j) {
+        const int i = (tid + j * NWARP * 32) / V4;
+        const float w = cc < nchunks && i < rs.tc ? sm_m[i * nchunks + cc] : 0.f;
+        acc[j].x += v[cb][j].x * w; acc[j].y += v[cb][j].y * w; acc[j].z += v[cb][j].z * w; acc[j].w += v[cb][j].w * w;
+      }
     }
   }
 #pragma unroll
@@ -331,16 +429,18 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
 // at most and chunks as long as that allows (the kernel is bound by the MMA rate of an SM, so what counts is the
 // largest number of tiles any SM walks, plus about one tile of set-up per CTA); many pairs: chunks of about
 // 128 rows, which the block scheduler balances.
-int pick_chunks(int pairs, int len_upper, int tile, int nchunks_max, int sms) {
+int pick_chunks(int pairs, int len_upper, int tile, int nchunks_max, int sms, bool* cluster) {
   const int nt = (len_upper + tile - 1) / tile;
   int hi = (len_upper + ATT_CHUNK_ROWS - 1) / ATT_CHUNK_ROWS;
   hi = hi < 1 ? 1 : (hi > nchunks_max ? nchunks_max : hi);
-  int best = hi; long best_cost = -1;
-  for (int n = 1; n <= hi; ++n) {
+  auto cost = [&](int n) {
     const long per_sm = ((long)pairs * n + sms - 1) / sms, tiles = (nt + n - 1) / n;
-    const long cost = per_sm * (tiles + 1) + 1;
-    if (best_cost < 0 || cost <= best_cost) { best = n; best_cost = cost; }
-  }
+    return per_sm * (tiles + 1) + 1;
+  };
+  int best = hi; long best_cost = -1;
+  for (int n = 1; n <= hi; ++n)
+    if (best_cost < 0 || cost(n) <= best_cost) { best = n; best_cost = cost(n); }
+  *cluster = best <= 8;        // up to 8 chunks: the pair's CTAs form a cluster and merge through shared memory
   return best;
 }
 
@@ -352,21 +452,39 @@ hydra_status run_ns(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, 
   static int sms = 0;
   if (!sms) { int dev = 0; HYDRA_CUDA(cudaGetDevice(&dev)); HYDRA_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)); }
   if ((size_t)H * rs.batch * sizeof(int) > ATT_SCRATCH_HEADER) return HYDRA_ERR_UNSUPPORTED;
-  const int nchunks = pick_chunks(H * rs.batch, len_upper, TILE, nchunks_max, sms);
+  bool cluster = false;
+  const int nchunks = pick_chunks(H * rs.batch, len_upper, TILE, nchunks_max, sms, &cluster);
   const size_t rows = (size_t)rs.batch * rs.tc;
   int* arrived = reinterpret_cast<int*>(scratch);     // one counter per (sequence, head): zero between launches
   float* part_o = scratch + ATT_SCRATCH_HEADER / sizeof(float);
   float* part_ml = part_o + rows * H * nchunks_max * HD;
   constexpr int LDS = HD + 8;
   constexpr int NP = HL ? 2 : 1;
-  const size_t smem = (size_t)NP * (64 + 2 * NS * TILE) * LDS * sizeof(bf16);
+  const size_t ring = (size_t)NP * 2 * NS * TILE * LDS * sizeof(bf16);
+  const size_t xchg = (size_t)(4 * 32 * (HD / 2 + 4) + 64 * HD + 128) * sizeof(float);      // hand-over area + a chunk's partial rows + (m, l)
+  const size_t smem = (size_t)NP * 64 * LDS * sizeof(bf16) + (ring > xchg ? ring : xchg);
   static bool attr_done = false;
   if (!attr_done) {
-    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE, NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE, NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_done = true;
   }
-  launch_pdl(tree_attn_tc_kernel<HD, HL, TILE, NS>, dim3(H, rs.batch, nchunks), dim3(NWARP * 32), smem, st, q, q_ps, kc, vc, kv_ps, rs, part_o, part_ml,
-             arrived, out, out_ps, H, max_seq, nchunks);
+  if (!cluster) {
+    launch_pdl(tree_attn_tc_kernel<HD, HL, TILE, NS, false>, dim3(H, rs.batch, nchunks), dim3(NWARP * 32), smem, st, q, q_ps, kc, vc, kv_ps, rs, part_o,
+               part_ml, arrived, out, out_ps, H, max_seq, nchunks);
+    HYDRA_LAUNCH_CHECK();
+    return HYDRA_OK;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(H, rs.batch, nchunks); cfg.blockDim = dim3(NWARP * 32); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = (unsigned)nchunks;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<HD, HL, TILE, NS, true>, q, q_ps, kc, vc, kv_ps, rs, part_o, part_ml, arrived, out, out_ps, H,
+                                max_seq, nchunks));
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -374,9 +492,6 @@ hydra_status run_ns(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, 
 template <int HD, bool HL>
 hydra_status run(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
                  float* scratch, int H, int max_seq, int len_upper, cudaStream_t st) {
-  static const int ns = []() { const char* e = getenv("HYDRA_ATT_NS"); return e ? atoi(e) : 5; }();
-  if (ns == 2) return run_ns<HD, HL, 2>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, st);
-  if (ns == 3) return run_ns<HD, HL, 3>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, st);
   return run_ns<HD, HL, 5>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, st);
 }
 

@@ -55,13 +55,22 @@ def test_gemm_float(m, n, k):
 
 @pytest.mark.parametrize("dtype,planes", [(torch.float32, 1), (torch.bfloat16, 1), (torch.bfloat16, 2)])
 @pytest.mark.parametrize("hd", [64, 128])
-def test_tree_attention_matches_masked_softmax(dtype, planes, hd):
+@pytest.mark.parametrize("case", ["few_chunks", "many_chunks"])
+def test_tree_attention_matches_masked_softmax(dtype, planes, hd, case):
+    """few_chunks: at most 8 KV chunks per (head, sequence), which the bfloat16 kernel merges inside a thread-block
+    cluster; many_chunks: one long sequence with two heads, 12 chunks, merged through scratch by the last CTA."""
     from paper_2402_05109_b200 import tree_attention, split_hi_lo
     parent = load_tree("tree63_d4")
     t = TreeTables(parent)
-    B, H, S, tc = 3, 3, 700, t.T
-    pos0 = [0, 333, 600]                    # empty cache, a cache spanning several KV chunks with a ragged tail, long
-    n_rows = [tc, tc, 17]                   # ragged row counts (rows beyond n_rows are ignored)
+    tc = t.T
+    if case == "few_chunks":
+        B, H, S = 3, 3, 700
+        pos0 = [0, 333, 600]                # empty cache, a cache spanning several KV chunks with a ragged tail, long
+        n_rows = [tc, tc, 17]               # ragged row counts (rows beyond n_rows are ignored)
+    else:
+        B, H, S = 1, 2, 1500
+        pos0 = [1391]
+        n_rows = [tc]
     src = torch.float32 if planes == 2 else dtype
     kc = rnd((B, H, S, hd), 21, 1, src)
     vc = rnd((B, H, S, hd), 21, 2, src)
