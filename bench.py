@@ -23,6 +23,10 @@ from synth import get_config, make_weights, make_prompts, load_tree, plant_row, 
 
 METRIC = "drafted+verified tokens/s (tree rows through draft+verify+accept per second)"
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + write) per algorithmic byte of the tensor-core GEMM kernel, from the ncu capture summarised in
+# profiles/gemm_tc_kernel_c2s.md (three launches: 389.2 MB moved for 386.0 MB algorithmic).  Only valid for the bf16
+# tensor-core path (gemm mode 0); set to None whenever that kernel changes until the counters are taken again.
+GEMM_TRAFFIC_RATIO = 1.008
 
 
 def peaks():
@@ -130,21 +134,22 @@ def plant_schedule(cfg, parent, teacher, n_steps):
 
 def oracle_sample(cfg, weights_cpu, parent, n_steps, threads):
     """The CPU oracle, as it stands, on a bounded sample of the workload: full draft and acceptance, and the
-    verification forward timed on 1 and on 3 of the decoder layers (plus final norm and LM head) and
+    verification forward timed on 1 and on min(3, all) of the decoder layers (plus final norm and LM head) and
     extrapolated linearly to all layers.  Prompt shortened to 64 tokens.  Returns seconds per step."""
     import copy
     from oracle.hydra_oracle import HydraOracle
     torch.set_num_threads(threads)
     prompts = make_prompts(cfg.seed, [64] * cfg.batch, cfg.model.vocab)
     oracles = []
-    for nl in (1, 3):
+    NL = cfg.model.n_layers
+    nl_hi = min(3, NL)
+    for nl in (1, nl_hi):
         m = copy.copy(cfg.model)
         m.n_layers = nl
         o = HydraOracle(m, cfg.head, parent, weights_cpu, 64 + 8 * (cfg.head.n_heads + 1) * (n_steps + 1) + len(parent),
                         dtype=torch.float32, cache_weights=True)
         o.prefill(prompts)
         oracles.append(o)
-    NL = cfg.model.n_layers
     per_step = []
     for s in range(n_steps):
         o1, o3 = oracles
@@ -161,7 +166,7 @@ def oracle_sample(cfg, weights_cpu, parent, n_steps, threads):
         t5 = time.perf_counter()
         o1.accept_compact(tok1, amax1)
         v3, v1 = t2 - t1, t5 - t4
-        per_layer = max(0.0, (v3 - v1) / 2.0)
+        per_layer = max(0.0, (v3 - v1) / (nl_hi - 1)) if nl_hi > 1 else 0.0
         per_step.append((t1 - t0) + (t3 - t2) + v1 + (NL - 1) * per_layer)
     return per_step
 
@@ -188,7 +193,7 @@ def run_reference(args, cfg, parent):
     rows = cfg.batch * len(parent)
     val = rows / sec
     sample = ("oracle decode step at the workload's shapes with the prompt shortened to 64 tokens; verification timed "
-              "on 1 and 3 decoder layers and extrapolated linearly to %d layers" % cfg.model.n_layers)
+              "on 1 and %d decoder layers and extrapolated linearly to %d layers" % (min(3, cfg.model.n_layers), cfg.model.n_layers))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -386,12 +391,15 @@ def main():
         sec = sum(per) / len(per)
         cpu = {"value": B * T / sec, "unit": "tokens/s", "cores": threads, "kind": "oracle",
                "sample": "2 timed oracle decode steps (after 1 warm-up) at the workload's shapes, prompt shortened to 64 "
-                         "tokens, verification timed on 1 and 3 decoder layers and extrapolated linearly to %d layers; "
+                         "tokens, verification timed on 1 and min(3, all) decoder layers and extrapolated linearly to %d layers; "
                          "%.2f s per full step" % (m.n_layers, sec)}
     g.close()
     if rank != 0:
         return
     value = world * B * T / (ms_step * 1e-3)
+    traffic = None
+    if GEMM_TRAFFIC_RATIO is not None and m.dtype == "bf16" and args.gemm_mode == 0 and gemm_n:
+        traffic = GEMM_TRAFFIC_RATIO * gemm_bytes / gemm_n        # bytes per launch, like `achieved`
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -408,7 +416,7 @@ def main():
         "final_lens": lens_end,
         "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel (weight-streaming bf16 GEMM, all shapes of a step)",
                      "achieved": gemm_gbs, "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": gemm_gbs / hbm_peak, "frac_of_8TBs": gemm_gbs / NOMINAL_HBM_GBS, "traffic": None,
+                     "frac": gemm_gbs / hbm_peak, "frac_of_8TBs": gemm_gbs / NOMINAL_HBM_GBS, "traffic": traffic,
                      "launches": gemm_n, "avg_launch_us": gemm_ms * 1e3 / max(1, gemm_n),
                      "bytes_per_launch": gemm_bytes / max(1, gemm_n),
                      "gemm_ms_per_step": gemm_ms / args.steps, "attention_ms_per_step": att_ms / args.steps,
