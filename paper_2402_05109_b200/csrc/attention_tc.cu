@@ -2,14 +2,16 @@
 //
 // One CTA per (head, sequence, KV chunk).  A sequence's KV rows are cut into TILE-row tiles and the tiles are dealt
 // to the grid's chunks in equal contiguous runs (computed on the device from the real length, so every chunk of
-// the launch has work whatever the length); the chunk's K and V tiles are streamed once from HBM through a
-// five-stage cp.async ring (four tiles in flight per CTA: the walk is bound by HBM latency otherwise).  Eight warps: warp w owns query rows 16 (w & 3) .. +15 (as MMA fragments) and
-// the keys of half (w >> 2) of every tile.  Scores of committed slots are unmasked; a tree slot j is visible to
-// row i iff bit j of the row's ancestor bitmask is set.  Each warp keeps a running (max, sum, weighted V)
-// per query row in the exp2 domain (online softmax, reductions by warp shuffles over the 4 lanes that share
-// a row); the two key halves are merged through shared memory at the end.  Per-chunk partial results go to a
-// scratch buffer; the CTA that reports in last for a (head, sequence) pair (an arrival counter that it resets)
-// merges the pair's chunks in chunk order and writes the output rows.
+// the launch has work whatever the length); Q and the chunk's K and V tiles are streamed once through a five-stage
+// cp.async ring (four tiles in flight per CTA: the walk is bound by HBM latency otherwise).  Eight warps: warp w
+// owns query rows 16 (w & 3) .. +15 (as MMA fragments) and the keys of half (w >> 2) of every tile.  Scores of
+// committed slots are unmasked; a tree slot j is visible to row i iff bit j of the row's ancestor bitmask is set.
+// Each warp keeps a running (max, sum, weighted V) per query row in the exp2 domain (online softmax, reductions by
+// warp shuffles over the 4 lanes that share a row); the two key halves are merged through shared memory at the end.
+// Merging the chunks of a (head, sequence) pair, in chunk order either way: with up to 8 chunks the pair's CTAs
+// form a thread-block cluster, leave their partial rows in their own shared memory and each merges a share of the
+// rows out of its peers' shared memory; with more chunks the partial rows go to a scratch buffer and the CTA that
+// reports in last (an arrival counter that it resets) merges them.
 // Precision: q, K, V and the attention output are stored as two bfloat16 planes (hi = bf16(v), lo = bf16(v - hi),
 // about 16 mantissa bits together).  Products use the three significant cross terms (hi*hi + lo*hi + hi*lo); the
 // softmax weights are split the same way before the P V product.  A plane distance of 0 selects hi-only operands.
