@@ -171,6 +171,21 @@ def oracle_sample(cfg, weights_cpu, parent, n_steps, threads):
     return per_step
 
 
+def max_over_ranks(value, dist, device):
+    """Slowest rank's time: what a replica job's wall clock is.  `dist` is torch.distributed (initialised) or None."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(units_per_rank, world, seconds):
+    """Whole-job units per second of `world` independent replicas that each process units_per_rank in `seconds`
+    (the max over ranks)."""
+    return world * units_per_rank / seconds
+
+
 def workload_name(cfg, parent):
     m, h = cfg.model, cfg.head
     return ("%s: %d-layer d=%d Llama-shape decoder, %d Hydra heads x %d MLP layers, prefix layer=%s, %d-row tree "
@@ -282,10 +297,7 @@ def main():
     launches = g.launch_count() - launches0
     g.poll_status()
     ms_total = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, "cuda")
     ms_step = ms_total / args.steps
     acc = nacc[args.warmup:].float().mean().item()
     lens_end = g.get_buffer("LEN")[:B].cpu().tolist()
@@ -376,11 +388,8 @@ def main():
         if s >= args.warmup:
             t_e2e += dt
             emitted += int(h_nacc.sum()) + B
-    if dist is not None:
-        t = torch.tensor([t_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_e2e = float(t.item())
-    e2e_val = world * B * T * args.steps / t_e2e
+    t_e2e = max_over_ranks(t_e2e, dist, "cuda")
+    e2e_val = job_throughput(B * T * args.steps, world, t_e2e)
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, single-GPU runs only)
     cpu = None
@@ -396,7 +405,7 @@ def main():
     g.close()
     if rank != 0:
         return
-    value = world * B * T / (ms_step * 1e-3)
+    value = job_throughput(B * T, world, ms_step * 1e-3)
     traffic = None
     if GEMM_TRAFFIC_RATIO is not None and m.dtype == "bf16" and args.gemm_mode == 0 and gemm_n:
         traffic = GEMM_TRAFFIC_RATIO * gemm_bytes / gemm_n        # bytes per launch, like `achieved`
