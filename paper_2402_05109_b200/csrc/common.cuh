@@ -53,12 +53,13 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
 
 // Where the partial sums of a GEMM output element live.  The tensor-core GEMM cuts the (tile, k-block) line
-// into ranges of q units per CTA; tile t = (m / mt) * n_tiles + n / 128 owns units [t*kb, (t+1)*kb), so its
+// into ranges of q units per CTA; tile t = (m / mt) * n_tiles + (n >> bn_shift) (weight tiles of 128 or 256 rows)
+// owns units [t*kb, (t+1)*kb), so its
 // partial sums sit in slots 0 .. split_count-1 (slot s at part + s*stride + m*N + n), one per CTA that
 // touched the tile, in CTA order.  A single-slot output is described by q = kb = 1.
-struct SplitDesc { int q, kb, n_tiles, mt; size_t stride; };
+struct SplitDesc { int q, kb, n_tiles, mt, bn_shift; size_t stride; };
 __host__ __device__ __forceinline__ int split_count(const SplitDesc& sd, int m, int n) {
-  const int u0 = ((m / sd.mt) * sd.n_tiles + (n >> 7)) * sd.kb;        // tiles * kb stays far below 2^31
+  const int u0 = ((m / sd.mt) * sd.n_tiles + (n >> sd.bn_shift)) * sd.kb;   // tiles * kb stays far below 2^31
   return (u0 + sd.kb - 1) / sd.q - u0 / sd.q + 1;
 }
 // acc[u] = sum over the ns[u] slots of the four floats at element offset off[u] of a slot (all loads of a round in flight together)
@@ -84,7 +85,7 @@ __device__ __forceinline__ void sum_slots_multi(const float* part, size_t stride
         acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
       }
 }
-inline SplitDesc single_slot(size_t stride) { return SplitDesc{1, 1, 1, 1 << 30, stride}; }
+inline SplitDesc single_slot(size_t stride) { return SplitDesc{1, 1, 1, 1 << 30, 7, stride}; }
 
 // Launch with programmatic stream serialisation allowed (see pdl_wait).
 template <typename... KArgs, typename... Args>

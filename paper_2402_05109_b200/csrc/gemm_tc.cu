@@ -15,9 +15,12 @@
 // slot (cta - first cta of the tile) of the partial buffer.  The consumer kernel adds the slots of a tile in
 // fixed order (SplitDesc), so results are deterministic.
 //
+// A unit carries NH = 1 or 2 such weight tiles (256 weight rows in one TMA box) that share the unit's activation
+// tile and accumulate side by side in tensor memory: wide outputs use 2.
+//
 // Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocation + MMA issue (one
-// lane), warps 2..5 = epilogue (TMEM -> registers -> global, coalesced along n).  Two accumulator buffers in
-// TMEM let the epilogue of one segment overlap the main loop of the next.  The kernel is launched with
+// lane), warps 2..5 = epilogue (TMEM -> registers -> global, coalesced along n).  Two accumulator sets in
+// TMEM (where 512 columns allow) let the epilogue of one segment overlap the main loop of the next.  The kernel is launched with
 // programmatic stream serialisation: weight tiles (which never depend on the preceding kernel) are requested
 // before griddepcontrol.wait, activations and all global writes after it.
 // Precision: weights are bfloat16 (exact: the reference model's weights are the same bfloat16 values).  The
@@ -194,18 +197,20 @@ __device__ __forceinline__ void store_accumulator(uint32_t taddr, bool cat, floa
   }
 }
 
-template <int MT, int BUDGET_KB> struct TileCfg {
+template <int MT, int BUDGET_KB, int NH = 1> struct TileCfg {        // NH: 128-row weight tiles per unit (they share the activation tile)
   static constexpr int SMEM_BUDGET = BUDGET_KB * 1024;
   static constexpr int B_PLANE = MT * BLOCK_K * 2;               // one activation plane of a stage
   static constexpr int B_BYTES = 2 * B_PLANE;                    // hi + lo
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int W_BYTES = NH * A_BYTES;                   // weight rows of a unit: NH * 128
+  static constexpr int STAGE_BYTES = W_BYTES + B_BYTES;
   static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 10 ? 10 : ((SMEM_BUDGET / STAGE_BYTES) < 2 ? 2 : (SMEM_BUDGET / STAGE_BYTES));
   // Two planes, MT <= 128: the hi and lo activation tiles sit back to back in shared memory and form ONE MMA B
   // operand of 2*MT rows, so each weight tile is read from shared memory once; accumulator columns [0, MT) hold
   // W*hi, [MT, 2MT) hold W*lo and the epilogue adds them.  MT = 256: two accumulating passes over the weight tile.
   static constexpr bool CAT = MT <= 128;
   static constexpr int ACC_COLS = CAT ? (2 * MT < 32 ? 32 : 2 * MT) : MT;   // columns of one accumulator buffer
-  static constexpr int TMEM_COLS = 2 * ACC_COLS;                  // two buffers (power of two, <= 512)
+  static constexpr int NBUF = 2 * NH * ACC_COLS <= 512 ? 2 : 1;   // accumulator sets: two when tensor memory allows
+  static constexpr int TMEM_COLS = NBUF * NH * ACC_COLS;          // power of two, <= 512
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers*/;
 };
 
@@ -226,10 +231,11 @@ __device__ __forceinline__ long long global_ns() { long long t; asm volatile("mo
       a.diag[4] = gridDim.x; a.diag[5] = a.m; a.diag[6] = a.n; a.diag[7] = a.kb; } } while (0)
 #define TRACE(slot) do { if (a.trace) a.trace[blockIdx.x * 8 + (slot)] = global_ns(); } while (0)
 
-template <int MT, int BUDGET_KB>
+template <int MT, int BUDGET_KB, int NH>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const GemmArgs a) {
-  using C = TileCfg<MT, BUDGET_KB>;
+  using C = TileCfg<MT, BUDGET_KB, NH>;
+  constexpr int BN = NH * BLOCK_N;                       // weight rows of a unit
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = tiles + C::STAGES * C::STAGE_BYTES;
@@ -260,8 +266,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int pre0 = n_units < C::STAGES ? n_units : C::STAGES;
     for (int i = 0; i < pre0; ++i) {
       const int u = u_begin + i, tile = u / a.kb;
-      mbar_arrive_expect_tx(fullw_bar(i), A_BYTES);
-      tma_load_2d(tiles + i * C::STAGE_BYTES, &tmW, (u - tile * a.kb) * BLOCK_K, (tile % a.n_tiles) * BLOCK_N, fullw_bar(i), pol_w0);
+      mbar_arrive_expect_tx(fullw_bar(i), C::W_BYTES);
+      tma_load_2d(tiles + i * C::STAGE_BYTES, &tmW, (u - tile * a.kb) * BLOCK_K, (tile % a.n_tiles) * BN, fullw_bar(i), pol_w0);
     }
   }
   if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
@@ -282,9 +288,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       int kcol = 0, nrow = 0, mrow = 0;
       if (n_units > 0) {
         const int tile = u_begin / a.kb;
-        kcol = (u_begin - tile * a.kb) * BLOCK_K; nrow = (tile % a.n_tiles) * BLOCK_N; mrow = (tile / a.n_tiles) * MT;
+        kcol = (u_begin - tile * a.kb) * BLOCK_K; nrow = (tile % a.n_tiles) * BN; mrow = (tile / a.n_tiles) * MT;
       }
-      const int kend = a.kb * BLOCK_K, nend = a.n_tiles * BLOCK_N, lo_rows = a.x_lo_rows;
+      const int kend = a.kb * BLOCK_K, nend = a.n_tiles * BN, lo_rows = a.x_lo_rows;
       const uint32_t x_bytes = lo_rows ? C::B_BYTES : C::B_PLANE;
       int s = 0; uint32_t eph = 1;                       // ring stage, parity of its empty barrier
       TRACE(2);
@@ -293,14 +299,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const uint32_t a_dst = tiles + s * C::STAGE_BYTES;
         if (i >= pre) {
           if (!mbar_wait(empty_bar(s), eph)) { GIVE_UP(1, i); s_abort = 1; break; }
-          mbar_arrive_expect_tx(fullw_bar(s), A_BYTES);
+          mbar_arrive_expect_tx(fullw_bar(s), C::W_BYTES);
           tma_load_2d(a_dst, &tmW, kcol, nrow, fullw_bar(s), pol_w);
         }
         mbar_arrive_expect_tx(fullx_bar(s), x_bytes);
-        tma_load_2d(a_dst + A_BYTES, &tmX, kcol, mrow, fullx_bar(s), pol_x);
-        if (lo_rows) tma_load_2d(a_dst + A_BYTES + C::B_PLANE, &tmX, kcol, lo_rows + mrow, fullx_bar(s), pol_x);
+        tma_load_2d(a_dst + C::W_BYTES, &tmX, kcol, mrow, fullx_bar(s), pol_x);
+        if (lo_rows) tma_load_2d(a_dst + C::W_BYTES + C::B_PLANE, &tmX, kcol, lo_rows + mrow, fullx_bar(s), pol_x);
         if (++s == C::STAGES) { s = 0; eph ^= 1u; }
-        if ((kcol += BLOCK_K) == kend) { kcol = 0; if ((nrow += BLOCK_N) == nend) { nrow = 0; mrow += MT; } }
+        if ((kcol += BLOCK_K) == kend) { kcol = 0; if ((nrow += BN) == nend) { nrow = 0; mrow += MT; } }
       }
     }
   } else if (warp == 1) {
@@ -313,26 +319,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const bool two_pass = a.x_lo_rows && !cat;
       int seg_len = n_units > 0 ? min((u_begin / a.kb + 1) * a.kb, u_end) - u_begin : 0;      // first segment: the tail of a tile
       for (int i = 0; i < n_units && ok;) {
-        const int acc = seg & 1;
-        const uint32_t acc_ph = (seg >> 1) & 1;
+        const int acc = seg % C::NBUF;
+        const uint32_t acc_ph = (seg / C::NBUF) & 1;
         if (!mbar_wait(accempty_bar(acc), acc_ph ^ 1u)) { GIVE_UP(2, i); ok = false; break; }      // epilogue has drained this buffer
         tc_fence_after();
-        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * C::ACC_COLS);
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * NH * C::ACC_COLS);
         for (int j = 0; j < seg_len; ++j, ++i) {
           if (!mbar_wait(fullw_bar(s), ph)) { GIVE_UP(3, i); ok = false; break; }
           if (!mbar_wait(fullx_bar(s), ph)) { GIVE_UP(4, i); ok = false; break; }
           if (i == 0) TRACE(3);
           tc_fence_after();
           const uint32_t a_addr = tiles + s * C::STAGE_BYTES;
-          const uint64_t adesc = smem_desc_sw128(a_addr);
-          const uint64_t bdesc = smem_desc_sw128(a_addr + A_BYTES);
+          const uint64_t bdesc = smem_desc_sw128(a_addr + C::W_BYTES);
 #pragma unroll
-          for (int k = 0; k < BLOCK_K / 16; ++k)         // 16 bf16 = 32 bytes per MMA: +2 in 16-byte units
-            umma_bf16(tmem_d, adesc + 2u * k, bdesc + 2u * k, idesc, (uint32_t)((j | k) != 0));
-          if (two_pass) {                                // the low-order plane of the activations, same weights
-            const uint64_t ldesc = smem_desc_sw128(a_addr + A_BYTES + C::B_PLANE);
+          for (int hh = 0; hh < NH; ++hh) {              // the unit's weight tiles, one accumulator each, same activation tile
+            const uint64_t adesc = smem_desc_sw128(a_addr + hh * A_BYTES);
+            const uint32_t d_h = tmem_d + (uint32_t)(hh * C::ACC_COLS);
 #pragma unroll
-            for (int k = 0; k < BLOCK_K / 16; ++k) umma_bf16(tmem_d, adesc + 2u * k, ldesc + 2u * k, idesc, 1u);
+            for (int k = 0; k < BLOCK_K / 16; ++k)       // 16 bf16 = 32 bytes per MMA: +2 in 16-byte units
+              umma_bf16(d_h, adesc + 2u * k, bdesc + 2u * k, idesc, (uint32_t)((j | k) != 0));
+            if (two_pass) {                              // the low-order plane of the activations, same weights
+              const uint64_t ldesc = smem_desc_sw128(a_addr + C::W_BYTES + C::B_PLANE);
+#pragma unroll
+              for (int k = 0; k < BLOCK_K / 16; ++k) umma_bf16(d_h, adesc + 2u * k, ldesc + 2u * k, idesc, 1u);
+            }
           }
           umma_commit(empty_bar(s));                     // frees the stage once these MMAs have read it
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
@@ -354,16 +364,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int u = u_begin + i;
       const int tile = u / a.kb;
       const int seg_len = min((tile + 1) * a.kb, u_end) - u;
-      const int acc = seg & 1;
-      const uint32_t acc_ph = (seg >> 1) & 1;
+      const int acc = seg % C::NBUF;
+      const uint32_t acc_ph = (seg / C::NBUF) & 1;
       if (!mbar_wait(accfull_bar(acc), acc_ph)) { if (lane == 0) GIVE_UP(5, i); break; }
       if (epi_tid == 0 && i + seg_len >= n_units) TRACE(5);
       tc_fence_after();
       const int slot = blockIdx.x - (int)(((long long)tile * a.kb) / a.q);
-      const int n0 = (tile % a.n_tiles) * BLOCK_N, m0 = (tile / a.n_tiles) * MT;
+      const int n0 = (tile % a.n_tiles) * BN, m0 = (tile / a.n_tiles) * MT;
       float* dst = a.part + (size_t)slot * a.slot_stride + n0 + epi_tid;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * C::ACC_COLS);
-      store_accumulator<MT>(taddr, C::CAT && a.x_lo_rows != 0, dst, m0, a.m, a.n);
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * NH * C::ACC_COLS);
+#pragma unroll
+      for (int hh = 0; hh < NH; ++hh)
+        store_accumulator<MT>(taddr + (uint32_t)(hh * C::ACC_COLS), C::CAT && a.x_lo_rows != 0, dst + hh * BLOCK_N, m0, a.m, a.n);
       tc_fence_before();
       if (lane == 0) mbar_arrive(accempty_bar(acc));     // the MMA warp may reuse this accumulator
       i += seg_len;
@@ -665,7 +677,7 @@ __global__ void __launch_bounds__(192, 1) gemm_chain_kernel(const __grid_constan
       }
       epi_bar();
       if (!s_flag) { ok = false; break; }
-      const SplitDesc sd{J.q, J.kb, J.n_tiles, MT, J.slot_stride};
+      const SplitDesc sd{J.q, J.kb, J.n_tiles, MT, 7, J.slot_stride};
       if (J.op == CHAIN_SILU_MUL) chain_silu_mul(a, J, sd, et);
       else chain_resid_norm(a, J, sd, et, s_red);
       __threadfence();
@@ -742,12 +754,12 @@ int sm_count() {
   return n;
 }
 
-template <int MT, int BUDGET_KB>
+template <int MT, int BUDGET_KB, int NH>
 hydra_status launch_b(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs& a, int grid, cudaStream_t st) {
-  using C = TileCfg<MT, BUDGET_KB>;
+  using C = TileCfg<MT, BUDGET_KB, NH>;
   static bool attr_done = false;
   if (!attr_done) {
-    HYDRA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<MT, BUDGET_KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    HYDRA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<MT, BUDGET_KB, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_done = true;
   }
   cudaLaunchConfig_t cfg = {};
@@ -756,18 +768,18 @@ hydra_status launch_b(const CUtensorMap& tw, const CUtensorMap& tx, const GemmAr
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
-  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<MT, BUDGET_KB>, tw, tx, a));
+  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<MT, BUDGET_KB, NH>, tw, tx, a));
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 // Shared memory per CTA: a deep ring (one CTA per SM) by default; HYDRA_GEMM_SMEM_KB=100 selects a ring that lets
 // the CTAs of two consecutive (programmatically overlapped) GEMMs share an SM (measured: no faster).
-template <int MT>
+template <int MT, int NH>
 hydra_status launch(const CUtensorMap& tw, const CUtensorMap& tx, const GemmArgs& a, int grid, cudaStream_t st) {
   static const int kb = []() { const char* e = getenv("HYDRA_GEMM_SMEM_KB"); return e ? atoi(e) : 200; }();
-  if (kb >= 200) return launch_b<MT, 200>(tw, tx, a, grid, st);
-  return launch_b<MT, 100>(tw, tx, a, grid, st);
+  if (kb >= 200 || NH > 1) return launch_b<MT, 200, NH>(tw, tx, a, grid, st);
+  return launch_b<MT, 100, NH>(tw, tx, a, grid, st);
 }
 
 template <int MT>
@@ -798,10 +810,21 @@ bool gemm_tc_available() { return encode_fn() != nullptr; }
 int gemm_tile_rows(int m) { return m <= 16 ? 16 : m <= 32 ? 32 : m <= 64 ? 64 : m <= 128 ? 128 : 256; }
 
 // Stream-K plan: equal contiguous unit ranges, one per CTA, at most one CTA per SM and at least 4 k-blocks each.
-SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots) {
+// 128-row weight tiles per unit: outputs of 4096 columns and more take two (half the activation-tile traffic and half
+// the issue work per weight byte, a third more weight bytes in flight: -5 % step time at the 7B shape).  Above 64
+// activation rows tensor memory holds one set of two accumulators only (the epilogue no longer overlaps the next
+// segment), still a small gain.  HYDRA_GEMM_NH=1 forces single tiles.
+int gemm_tile_halves(int m, int n) {
+  static const int force = []() { const char* e = getenv("HYDRA_GEMM_NH"); return e ? atoi(e) : 0; }();
+  if (force == 1) return 1;
+  return n % (2 * BLOCK_N) == 0 && n >= 4096 ? 2 : 1;
+}
+
+SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots, int force_nh) {
   SplitDesc sd{};
   const int mt = gemm_tile_rows(m);
-  sd.mt = mt; sd.n_tiles = n / BLOCK_N; sd.kb = k / BLOCK_K; sd.stride = (size_t)m * n;
+  const int nh = force_nh ? force_nh : gemm_tile_halves(m, n);
+  sd.mt = mt; sd.n_tiles = n / (nh * BLOCK_N); sd.bn_shift = nh == 2 ? 8 : 7; sd.kb = k / BLOCK_K; sd.stride = (size_t)m * n;
   const int tiles = sd.n_tiles * ((m + mt - 1) / mt);
   const long long total = (long long)tiles * sd.kb;
   long long g = sm_count();
@@ -825,10 +848,11 @@ hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* 
   if (m <= 0 || n <= 0 || k <= 0 || n % BLOCK_N || k % BLOCK_K || (x_planes != 1 && x_planes != 2)) return HYDRA_ERR_UNSUPPORTED;
   if (((uintptr_t)x | (uintptr_t)w) & 15) return HYDRA_ERR_INVALID;
   int grid = 1;
-  SplitDesc sd = gemm_tc_plan(m, n, k, &grid, nullptr);
+  SplitDesc sd = gemm_tc_plan(m, n, k, &grid, nullptr, 0);
   if (x_rows_alloc < m) x_rows_alloc = m;
   CUtensorMap tw, tx;
-  if (!get_tensor_map(w, (uint64_t)n, (uint64_t)k, BLOCK_N, &tw) ||
+  const int nh = sd.bn_shift == 8 ? 2 : 1;
+  if (!get_tensor_map(w, (uint64_t)n, (uint64_t)k, (uint32_t)(nh * BLOCK_N), &tw) ||
       !get_tensor_map(x, (uint64_t)x_rows_alloc * x_planes, (uint64_t)k, (uint32_t)sd.mt, &tx)) {
     set_last_error("cuTensorMapEncodeTiled", cudaErrorUnknown);
     return HYDRA_ERR_CUDA;
@@ -839,12 +863,21 @@ hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* 
   a.x_lo_rows = x_planes == 2 ? x_rows_alloc : 0; a.diag = diag; a.trace = trace;
   { static const int f = []() { const char* e = getenv("HYDRA_GEMM_NOHINT"); return e && e[0] == '1' ? 1 : 0; }(); a.flags = f; }
   if (sd_out) *sd_out = sd;
+  if (nh == 2) {
+    switch (sd.mt) {
+      case 16: return launch<16, 2>(tw, tx, a, grid, st);
+      case 32: return launch<32, 2>(tw, tx, a, grid, st);
+      case 64: return launch<64, 2>(tw, tx, a, grid, st);
+      case 128: return launch<128, 2>(tw, tx, a, grid, st);
+      default: return launch<256, 2>(tw, tx, a, grid, st);
+    }
+  }
   switch (sd.mt) {
-    case 16: return launch<16>(tw, tx, a, grid, st);
-    case 32: return launch<32>(tw, tx, a, grid, st);
-    case 64: return launch<64>(tw, tx, a, grid, st);
-    case 128: return launch<128>(tw, tx, a, grid, st);
-    default: return launch<256>(tw, tx, a, grid, st);
+    case 16: return launch<16, 1>(tw, tx, a, grid, st);
+    case 32: return launch<32, 1>(tw, tx, a, grid, st);
+    case 64: return launch<64, 1>(tw, tx, a, grid, st);
+    case 128: return launch<128, 1>(tw, tx, a, grid, st);
+    default: return launch<256, 1>(tw, tx, a, grid, st);
   }
 }
 
@@ -861,7 +894,7 @@ hydra_status gemm_chain(const ChainStep* steps, int n_steps, int m, int x_planes
     if (s.op != CHAIN_NONE && (s.cols & 3)) return HYDRA_ERR_UNSUPPORTED;
     if (s.op == CHAIN_NONE && j + 1 < n_steps) return HYDRA_ERR_INVALID;       // only the last job may leave raw partial sums
     int slots = 1;
-    const SplitDesc sd = gemm_tc_plan(m, s.n, s.k, nullptr, &slots);
+    const SplitDesc sd = gemm_tc_plan(m, s.n, s.k, nullptr, &slots, 1);       // the chain kernel works on single weight tiles
     if ((size_t)slots * m * s.n > part_floats) return HYDRA_ERR_CAPACITY;
     const int rows_alloc = s.x_rows_alloc < m ? m : s.x_rows_alloc;
     if (!get_tensor_map(s.w, (uint64_t)s.n, (uint64_t)s.k, BLOCK_N, &a.tmW[j]) ||

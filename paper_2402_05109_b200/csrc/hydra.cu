@@ -162,9 +162,9 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   size_t part_floats = 0;
   {
     auto need = [&](int mm, int n, int k) {
-      int slots = 1;
-      if (m.dtype == 1) gemm_tc_plan(mm, n, k, nullptr, &slots);
-      part_floats = std::max(part_floats, (size_t)slots * mm * n);
+      int slots = 1, slots1 = 1;
+      if (m.dtype == 1) { gemm_tc_plan(mm, n, k, nullptr, &slots); gemm_tc_plan(mm, n, k, nullptr, &slots1, 1); }      // stand-alone and chain plans
+      part_floats = std::max(part_floats, (size_t)std::max(slots, slots1) * mm * n);
     };
     const int shapes[][2] = {{3 * d, d}, {d, d}, {2 * f, d}, {d, f}, {V, d}};
     const int per_seq[] = {CHUNK, T, K + 1, 1};

@@ -24,7 +24,7 @@ hydra_status gemm_chain(const ChainStep* steps, int n_steps, int m, int x_planes
                         int* status, int* diag, int* sync, cudaStream_t st);
 hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* w, float* part, int m, int n, int k,
                      SplitDesc* sd_out, int* status, int* diag /*int[8] or null*/, long long* trace, cudaStream_t st);
-SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots);
+SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots, int force_nh = 0);   // force_nh: 128-row weight tiles per unit (0: the kernel's own choice)
 int gemm_tile_rows(int m);                // activation rows per MMA tile for an m-row GEMM: 16, 32, 64, 128 or 256
 bool gemm_tc_available();                 // driver entry point for tensor-map encoding found
 // SIMT path (float or bfloat16 operands), single slot.
