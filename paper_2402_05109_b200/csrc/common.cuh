@@ -63,9 +63,8 @@ __host__ __device__ __forceinline__ int split_count(const SplitDesc& sd, int m, 
   return (u0 + sd.kb - 1) / sd.q - u0 / sd.q + 1;
 }
 // acc[u] = sum over the ns[u] slots of the four floats at element offset off[u] of a slot (all loads of a round in flight together)
-template <int U>
+template <int U, int PMAX = 6>
 __device__ __forceinline__ void sum_slots_multi(const float* part, size_t stride, const size_t (&off)[U], const int (&ns)[U], float4 (&acc)[U]) {
-  constexpr int PMAX = 6;
   int mx = 0;
 #pragma unroll
   for (int u = 0; u < U; ++u) { acc[u] = make_float4(0.f, 0.f, 0.f, 0.f); mx = max(mx, ns[u]); }
@@ -84,6 +83,18 @@ __device__ __forceinline__ void sum_slots_multi(const float* part, size_t stride
         const float4 v = __ldcg(reinterpret_cast<const float4*>(part + p * stride + off[u]));
         acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
       }
+}
+// one float: the slots of element `idx` summed in slot order, the first PMAX loads in flight together
+template <int PMAX = 12>
+__device__ __forceinline__ float sum_slots_scalar(const float* part, size_t stride, size_t idx, int ns) {
+  float v[PMAX];
+#pragma unroll
+  for (int p = 0; p < PMAX; ++p) v[p] = p < ns ? __ldcg(part + p * stride + idx) : 0.f;
+  float acc = 0.f;
+#pragma unroll
+  for (int p = 0; p < PMAX; ++p) acc += v[p];
+  for (int p = PMAX; p < ns; ++p) acc += __ldcg(part + p * stride + idx);
+  return acc;
 }
 inline SplitDesc single_slot(size_t stride) { return SplitDesc{1, 1, 1, 1 << 30, 7, stride}; }
 

@@ -517,10 +517,7 @@ __device__ __forceinline__ void block_best(float& v, int& i, float* shv, int* sh
 }
 
 __device__ __forceinline__ float summed(const float* part, const SplitDesc& sd, int row, int col, int n) {
-  const int ns = split_count(sd, row, col);
-  float v = 0.f;
-  for (int s = 0; s < ns; ++s) v += part[s * sd.stride + (size_t)row * n + col];
-  return v;
+  return sum_slots_scalar<4>(part, sd.stride, (size_t)row * n + col, split_count(sd, row, col));
 }
 
 // Top-c of every logits row in two stages.  Stage 1: grid (rows, blocks of TOPK_SPAN columns); each block sums the
@@ -674,8 +671,7 @@ __global__ void head_act_kernel(const float* res, int res_is_hprime, int rows_pe
   if (i >= (size_t)rows * d) return;
   int r = (int)(i / d), c = (int)(i % d);
   float v = bias ? to_f<T>(bias[c]) : 0.f;
-  const int ns = split_count(sd, r, c);
-  for (int s = 0; s < ns; ++s) v += part[s * sd.stride + i];
+  v += sum_slots_scalar<12>(part, sd.stride, i, split_count(sd, r, c));
   float base = res_is_hprime ? res[(size_t)(r / rows_per_b) * d + c] : res[i];
   float y = base + silu_f(v);
   y_out[i] = y;
