@@ -146,7 +146,7 @@ template <> __device__ __forceinline__ void put4<bf16>(bf16* p, size_t ps, float
   if (ps) store4<bf16>(p + ps, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
 }
 
-constexpr int NORM_THREADS = 512;
+constexpr int NORM_THREADS = 1024;
 template <typename T>
 __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const float* res, const float* __restrict__ part,
                                                                         SplitDesc sd, float* x_out,
@@ -157,26 +157,15 @@ __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const fl
   __shared__ float sh[32];
   const size_t base = (size_t)blockIdx.x * d;
   float ss = 0.f;
-  for (int i0 = threadIdx.x * 4; i0 < d; i0 += NORM_THREADS * 4 * 2) {       // two pieces per round, all their slot loads in flight together
-    size_t off[2]; int ns[2]; float4 acc[2], v[2];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int i = i0 + u * NORM_THREADS * 4;
-      const bool valid = i < d;
-      off[u] = base + (valid ? i : 0);
-      ns[u] = valid && part ? split_count(sd, (int)blockIdx.x, i) : 0;
-      v[u] = valid && res ? *reinterpret_cast<const float4*>(res + base + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    sum_slots_multi<2>(part, sd.stride, off, ns, acc);
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int i = i0 + u * NORM_THREADS * 4;
-      if (i < d) {
-        v[u].x += acc[u].x; v[u].y += acc[u].y; v[u].z += acc[u].z; v[u].w += acc[u].w;
-        *reinterpret_cast<float4*>(x_out + base + i) = v[u];
-        ss += v[u].x * v[u].x + v[u].y * v[u].y + v[u].z * v[u].z + v[u].w * v[u].w;
-      }
-    }
+  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {       // one 16-byte piece per thread and round, all its slot loads in flight together
+    size_t off[1] = {base + i};
+    int ns[1] = {part ? split_count(sd, (int)blockIdx.x, i) : 0};
+    float4 acc[1];
+    float4 v = res ? *reinterpret_cast<const float4*>(res + base + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    sum_slots_multi<1, 12>(part, sd.stride, off, ns, acc);             // narrow outputs are cut into up to ~11 slots per tile
+    v.x += acc[0].x; v.y += acc[0].y; v.z += acc[0].z; v.w += acc[0].w;
+    *reinterpret_cast<float4*>(x_out + base + i) = v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   if (!gain) return;
   float tot = block_sum(ss, sh);
