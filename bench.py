@@ -24,9 +24,9 @@ from synth import get_config, make_weights, make_prompts, load_tree, plant_row, 
 METRIC = "drafted+verified tokens/s (tree rows through draft+verify+accept per second)"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per algorithmic byte of the tensor-core GEMM kernel, from the ncu capture summarised in
-# profiles/gemm_tc_kernel_c2s.md (three launches: 389.2 MB moved for 386.0 MB algorithmic).  Only valid for the bf16
+# profiles/gemm_tc_kernel_c2s.md (three launches: 392.4 MB moved for 386.1 MB algorithmic).  Only valid for the bf16
 # tensor-core path (gemm mode 0); set to None whenever that kernel changes until the counters are taken again.
-GEMM_TRAFFIC_RATIO = 1.008
+GEMM_TRAFFIC_RATIO = 1.016
 
 
 def peaks():
