@@ -57,9 +57,10 @@ def get_config(name: str) -> RunCfg:
     if name == "c2s":          # c2 cut to 4 layers (1.9 GB of weights): the small case for profiler captures
         return RunCfg("c2s", ModelCfg(**dict(_7B, n_layers=4)), HeadCfg(**_PP), "tree63_d4", 1, [512], 16, 1, 512 + 16 * 5 + 64)
     if name.startswith("c3"):
-        b = int(name[3:]) if len(name) > 2 else 8          # "c3b1", "c3b2", "c3b4", "c3b8"
-        return RunCfg(name, ModelCfg(**_7B), HeadCfg(**_PP), "tree63_d4", b, _ragged(2, b, 128, 1024), 64, 2,
-                      1024 + 64 * 5 + 64)
+        small = name.endswith("s")                         # "c3b8s": cut to 4 layers, the small case for profiler captures
+        b = int(name[3:].rstrip("s")) if len(name) > 2 else 8          # "c3b1", "c3b2", "c3b4", "c3b8"
+        return RunCfg(name, ModelCfg(**dict(_7B, n_layers=4 if small else 32)), HeadCfg(**_PP), "tree63_d4", b, _ragged(2, b, 128, 1024),
+                      16 if small else 64, 2, 1024 + 64 * 5 + 64)
     if name == "c4":
         return RunCfg("c4", ModelCfg(**_13B), HeadCfg(**_PP), "tree63_d4", 1, [2048], 64, 3, 2048 + 64 * 5 + 64)
     if name == "c5":
