@@ -23,9 +23,10 @@ from synth import get_config, make_weights, make_prompts, load_tree, plant_row, 
 
 METRIC = "drafted+verified tokens/s (tree rows through draft+verify+accept per second)"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) per algorithmic byte of the tensor-core GEMM kernel, from the ncu capture summarised in
-# profiles/gemm_tc_kernel_c2s.md (three launches: 392.4 MB moved for 386.1 MB algorithmic).  Only valid for the bf16
-# tensor-core path (gemm mode 0); set to None whenever that kernel changes until the counters are taken again.
+# DRAM bytes (read + write) per algorithmic byte of the tensor-core GEMM kernel, from an ncu capture of three launches
+# on the 4-layer cut of this workload (392.4 MB moved for 386.1 MB algorithmic; traffic is proportional to the weight
+# bytes, so the ratio carries to the full-size step).  Only valid for the bf16 tensor-core path (gemm mode 0); set to
+# None whenever that kernel changes until the counters are taken again.
 GEMM_TRAFFIC_RATIO = 1.016
 
 
@@ -37,12 +38,15 @@ def peaks():
     return 6650.0, "fallback"
 
 
-def verify_bytes(m, B, T, lens):
-    """Algorithmic bytes of one verification: every base weight once, every live KV row once, new rows written."""
+def verify_bytes(m, B, T, lens, skv=None):
+    """Algorithmic bytes of one verification: every base weight once, every live KV row once, new rows written.
+    skv = bytes per cache element: the method's own (one element of the weight type) by default; 4 is what this
+    library's cache really holds (float, or two bfloat16 planes)."""
     s = 2 if m.dtype == "bf16" else 4
+    if skv is None:
+        skv = s
     d, f = m.d_model, m.d_ffn
     w = s * (m.n_layers * (4 * d * d + 3 * d * f) + m.vocab * d)
-    skv = 4                      # cache element: float, or two bfloat16 planes (hi + lo)
     kv = sum(2 * m.n_layers * d * skv * (L + T) for L in lens) + B * T * 2 * m.n_layers * d * skv
     return w + kv
 
@@ -132,10 +136,42 @@ def plant_schedule(cfg, parent, teacher, n_steps):
     return plan, planned
 
 
-def oracle_sample(cfg, weights_cpu, parent, n_steps, threads):
-    """The CPU oracle, as it stands, on a bounded sample of the workload: full draft and acceptance, and the
-    verification forward timed on 1 and on min(3, all) of the decoder layers (plus final norm and LM head) and
-    extrapolated linearly to all layers.  Prompt shortened to 64 tokens.  Returns seconds per step."""
+ORACLE_PREFILL_BUDGET_FLOP = 12e12      # a real prompt pass on the host is affordable below this (c2: 6.8e12)
+
+
+def oracle_can_run_full(cfg):
+    m = cfg.model
+    params = m.n_layers * (4 * m.d_model ** 2 + 3 * m.d_model * m.d_ffn) + m.vocab * m.d_model
+    host_bytes = 4.0 * params * 1.15
+    return 2.0 * params * sum(cfg.prompt_lens) <= ORACLE_PREFILL_BUDGET_FLOP and host_bytes <= 64e9
+
+
+def oracle_full(cfg, weights_cpu, parent, n_steps, threads):
+    """The CPU oracle, as it stands, on the workload itself: a real prompt pass at the workload's prompt lengths,
+    then n_steps whole decode steps (draft, verify, accept + compact), each timed by wall clock.  Returns
+    (seconds per step list, seconds of the prompt pass)."""
+    from oracle.hydra_oracle import HydraOracle
+    torch.set_num_threads(threads)
+    prompts = make_prompts(cfg.seed, cfg.prompt_lens, cfg.model.vocab)
+    K = cfg.head.n_heads
+    o = HydraOracle(cfg.model, cfg.head, parent, weights_cpu, max(cfg.prompt_lens) + (n_steps + 1) * (K + 1) + len(parent),
+                    dtype=torch.float32, cache_weights=True)
+    t0 = time.perf_counter()
+    o.prefill(prompts)
+    t_prefill = time.perf_counter() - t0
+    per_step = []
+    for s in range(n_steps):
+        t0 = time.perf_counter()
+        o.step()
+        per_step.append(time.perf_counter() - t0)
+    return per_step, t_prefill
+
+
+def oracle_projected(cfg, weights_cpu, parent, n_steps, threads):
+    """Fallback for shapes whose prompt pass alone would take the host many minutes (13B at 2048 tokens, 33B): full draft
+    and acceptance, the verification forward timed on 1 and on min(3, all) of the decoder layers (plus final norm and
+    LM head) and extrapolated linearly to all layers; prompt shortened to 64 tokens.  A PROJECTION, labelled as such.
+    Returns seconds per step."""
     import copy
     from oracle.hydra_oracle import HydraOracle
     torch.set_num_threads(threads)
@@ -171,6 +207,24 @@ def oracle_sample(cfg, weights_cpu, parent, n_steps, threads):
     return per_step
 
 
+def oracle_timed(cfg, weights, parent, warmup, steps, threads):
+    """(seconds per step, description of the sample) of the CPU oracle on this workload.  weights: name -> tensor
+    (any device); widened to float32 on the host one tensor at a time."""
+    wc = {k: v.float().cpu() for k, v in weights.items()}
+    if oracle_can_run_full(cfg):
+        per, t_prefill = oracle_full(cfg, wc, parent, warmup + steps, threads)
+        per = per[warmup:]
+        sec = sum(per) / len(per)
+        return sec, ("%d whole oracle decode steps (after %d warm-up) at the workload's full shape, measured by wall clock "
+                     "after a real %d-token prompt pass (%.1f s, untimed); %.2f s per step"
+                     % (steps, warmup, sum(cfg.prompt_lens), t_prefill, sec))
+    per = oracle_projected(cfg, wc, parent, warmup + steps, threads)[warmup:]
+    sec = sum(per) / len(per)
+    return sec, ("PROJECTION (the prompt pass alone would take the host many minutes at this shape): oracle decode steps with "
+                 "the prompt shortened to 64 tokens, verification timed on 1 and %d decoder layers and extrapolated linearly "
+                 "to %d layers; %.2f s per step" % (min(3, cfg.model.n_layers), cfg.model.n_layers, sec))
+
+
 def max_over_ranks(value, dist, device):
     """Slowest rank's time: what a replica job's wall clock is.  `dist` is torch.distributed (initialised) or None."""
     if dist is None:
@@ -202,13 +256,9 @@ def run_reference(args, cfg, parent):
     threads = os.cpu_count() or 1
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     w = make_weights(cfg.model, cfg.head, cfg.seed, device=dev)
-    w = {k: v.cpu() for k, v in w.items()}
-    per_step = oracle_sample(cfg, w, parent, args.warmup + args.steps, threads)[args.warmup:]
-    sec = sum(per_step) / len(per_step)
+    sec, sample = oracle_timed(cfg, w, parent, args.warmup, args.steps, threads)
     rows = cfg.batch * len(parent)
     val = rows / sec
-    sample = ("oracle decode step at the workload's shapes with the prompt shortened to 64 tokens; verification timed "
-              "on 1 and %d decoder layers and extrapolated linearly to %d layers" % (min(3, cfg.model.n_layers), cfg.model.n_layers))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -225,7 +275,9 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--gemm-mode", type=int, default=0, help="0 tcgen05, one launch per GEMM (default), 1 SIMT, 2 tcgen05 with one persistent kernel per layer tail")
+    ap.add_argument("--gemm-mode", type=int, default=0, help="0 tcgen05 (default), 1 SIMT")
+    ap.add_argument("--blocks", type=int, default=5, help="timed blocks of --steps steps each; the median block is reported")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel of a step separately (profilers' launch lists)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -255,49 +307,57 @@ def main():
     plan_dev = plan.cuda()
     g = Hydra(m, h, parent, weights, B, max_seq)
     g.set_gemm_mode(args.gemm_mode)
+    g.set_step_graph(not args.no_graph)
     stream = torch.cuda.current_stream()
 
     def fresh():
         g.prefill(prompts)
         g.poll_status()
 
-    # ---- device-resident timed run: K whole steps back to back
-    fresh()
+    # ---- device-resident timed runs: `blocks` identical blocks (prompt pass, W warm-up steps, then K whole steps back
+    # to back between two events); the median block is the reported one
     nacc = torch.zeros(n_total, B, dtype=torch.int32, device="cuda")
     cur_plan = torch.empty(B, T, dtype=torch.int32, device="cuda")        # fixed buffers: the captured step graph keeps
     cur_nacc = torch.empty(B, dtype=torch.int32, device="cuda")           # their addresses
     cur_out = torch.empty(B, K + 1, dtype=torch.int32, device="cuda")
-    g.set_plant(cur_plan)
 
     def one_step(s):
         cur_plan.copy_(plan_dev[s], non_blocking=True)
         g.step(cur_nacc, cur_out)
         nacc[s].copy_(cur_nacc, non_blocking=True)
 
-    for s in range(args.warmup):
-        one_step(s)
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(local) if rank == 0 else None
-    launches0 = g.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.profiler.start()                 # lets a profiler restrict itself to the timed region (--profile-from-start off)
-    e0.record(stream)
-    for s in range(args.warmup, n_total):
-        one_step(s)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    torch.cuda.profiler.stop()
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
+    sampler = None
+    block_ms, launches = [], 0
+    for blk in range(max(1, args.blocks)):
+        fresh()
+        g.set_plant(cur_plan)
+        for s in range(args.warmup):
+            one_step(s)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if blk == 0 and rank == 0:
+            sampler = ClockSampler(local)
+        launches0 = g.launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if blk == 0:
+            torch.cuda.profiler.start()             # lets a profiler restrict itself to one timed block (--profile-from-start off)
+        e0.record(stream)
+        for s in range(args.warmup, n_total):
+            one_step(s)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if blk == 0:
+            torch.cuda.profiler.stop()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        launches = g.launch_count() - launches0
+        block_ms.append(max_over_ranks(e0.elapsed_time(e1), dist, "cuda"))
     clocks = sampler.stop() if sampler else None
-    launches = g.launch_count() - launches0
     g.poll_status()
-    ms_total = e0.elapsed_time(e1)
-    ms_total = max_over_ranks(ms_total, dist, "cuda")
+    ms_total = sorted(block_ms)[len(block_ms) // 2]
     ms_step = ms_total / args.steps
     acc = nacc[args.warmup:].float().mean().item()
     lens_end = g.get_buffer("LEN")[:B].cpu().tolist()
@@ -339,7 +399,8 @@ def main():
     med = lambda v: sorted(v)[len(v) // 2]
     t_draft, t_verify, t_accept = med(ph["draft"]), med(ph["verify"]), med(ph["accept"])
     mean_lens = [sum(l[b] for l in lens_mid) / len(lens_mid) for b in range(B)]
-    vbytes = verify_bytes(m, B, T, mean_lens)
+    vbytes = verify_bytes(m, B, T, mean_lens)                 # the method's bytes: one cache element = one weight element
+    vbytes_read = verify_bytes(m, B, T, mean_lens, skv=4)     # what this library's two-plane (or float) cache really moves
     dbytes = draft_bytes(m, h, mean_lens)
     hbm_peak, peak_kind = peaks()
     verify_gbs = vbytes / (t_verify * 1e-3) / 1e9
@@ -395,13 +456,8 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         threads = os.cpu_count() or 1
-        wc = {k: v.cpu() for k, v in weights.items()}
-        per = oracle_sample(cfg, wc, parent, 3, threads)[1:]
-        sec = sum(per) / len(per)
-        cpu = {"value": B * T / sec, "unit": "tokens/s", "cores": threads, "kind": "oracle",
-               "sample": "2 timed oracle decode steps (after 1 warm-up) at the workload's shapes, prompt shortened to 64 "
-                         "tokens, verification timed on 1 and min(3, all) decoder layers and extrapolated linearly to %d layers; "
-                         "%.2f s per full step" % (m.n_layers, sec)}
+        sec, sample = oracle_timed(cfg, weights, parent, 1, 2, threads)
+        cpu = {"value": B * T / sec, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample}
     g.close()
     if rank != 0:
         return
@@ -417,7 +473,8 @@ def main():
                    "l2": "every step streams %.1f GB of weights, far above the 126 MB L2; no flush needed" % (vbytes / 1e9),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "verify_ms": t_verify, "draft_ms": t_draft, "accept_compact_ms": t_accept,
-        "verify_bytes": vbytes, "draft_bytes": dbytes,
+        "verify_bytes": vbytes, "verify_bytes_moved_by_this_cache_format": vbytes_read, "draft_bytes": dbytes,
+        "block_ms_per_step": [t / args.steps for t in block_ms],
         "verify_hbm_gbs": verify_gbs, "verify_frac_of_8TBs": verify_gbs / NOMINAL_HBM_GBS,
         "verify_frac_of_%s" % peak_kind: verify_gbs / hbm_peak,
         "emitted_tokens_per_s": world * (acc + 1) * B / (ms_step * 1e-3), "mean_accepted": acc,

@@ -18,10 +18,14 @@
  *    hydra_destroy.  The library owns only the opaque context; KV caches, tables and scratch are
  *    carved out of the caller's workspace (hydra_workspace_bytes, 256-byte aligned base).
  *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and do not synchronise, except
- *    hydra_create (uploads tables), hydra_poll_status and hydra_destroy.
+ *    hydra_create (uploads tables; synchronises the device), hydra_prefill (synchronises the stream once,
+ *    after uploading the prompt offsets, before its first kernel), hydra_poll_status, hydra_get_timing and
+ *    hydra_destroy.
  *  - Order: create -> prefill -> (draft -> verify -> accept_compact | step)*.  A call out of order
  *    returns HYDRA_ERR_STATE.  The host keeps an upper bound of every sequence length (it grows by
- *    K+1 per step); a step that could exceed max_seq returns HYDRA_ERR_CAPACITY before any launch.
+ *    K+1 per step, as if every step accepted a full path); a step whose bound could exceed max_seq returns
+ *    HYDRA_ERR_CAPACITY before any launch.  hydra_poll_status replaces the bounds by the real lengths, so a
+ *    caller that polls now and then can use the whole cache.
  *  - Device-side problems (token id / slot out of range, a bounded wait that ran out) set a status
  *    word that hydra_poll_status returns; kernels skip the offending access and never trap.
  */
@@ -95,33 +99,50 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg*, const hydra_h
                           const hydra_weights*, void* workspace_dev, size_t workspace_bytes);
 hydra_status hydra_destroy(hydra_ctx*);
 
-/* Base-model forward over the prompts (ordinary causal attention) filling the KV caches; leaves, per
- * sequence, the committed length, the root token (argmax after the last prompt token) and the last
- * hidden state.  tokens_dev holds the prompts back to back; seq_offsets_host has batch+1 entries. */
+/* Set-up of speculative decoding (Background, "Speculative decoding": the base model has processed the
+ * sequence so far and proposes the next token).  Base-model forward over the prompts (ordinary causal
+ * attention) filling the KV caches, and, with prefix_attn, the extra layer's cache (Section "Hydra++",
+ * "Prefix Attention"); leaves, per sequence, the committed length, the root token (argmax after the last
+ * prompt token) and the last hidden state.  tokens_dev holds the prompts back to back; seq_offsets_host
+ * has batch+1 entries (read before the call returns).  Synchronises the stream once (see Conventions).
+ * Errors: INVALID (null pointer, batch outside 1..max_batch, empty prompt), CAPACITY (prompt + tree rows
+ * exceed max_seq). */
 hydra_status hydra_prefill(hydra_ctx*, int batch, const int32_t* tokens_dev, const int32_t* seq_offsets_host,
                            void* stream);
 
-/* Populate the candidate tree level by level: children of a node = its head's top tokens in
- * descending order (ties: lower token id first).  tree_tok_dev [batch][n_rows] out, row 0 = root. */
+/* Drafting (Section "Hydra Heads", second displayed equation: head i sees the last hidden state and the
+ * tokens speculated before it; Section "Hydra++": deeper MLPs and the extra decoder layer queried once per
+ * step; Background, "Tree decoding": children of a node = the top tokens of its head in descending order).
+ * Populates the candidate tree level by level; ties: lower token id first.  tree_tok_dev [batch][n_rows]
+ * int32 out, row 0 = root.  Errors: STATE, CAPACITY. */
 hydra_status hydra_draft(hydra_ctx*, int32_t* tree_tok_dev, void* stream);
 
-/* One base forward over all tree rows of all sequences with the ancestor mask; K,V of row i land in
- * cache slot len+i.  amax_dev [batch][n_rows] out: argmax of each row's logits (ties: lowest id).
- * logits_dev [batch][n_rows][vocab] float out, or NULL.  tree_tok_dev may be edited by the caller. */
+/* Verification (Background, "Tree decoding": all candidates packed into one input, a token attends only
+ * to its ancestors).  One base forward over all tree rows of all sequences with the ancestor mask; K,V of
+ * row i land in cache slot len+i, its rotary position is len+depth(i).  amax_dev [batch][n_rows] int32 out:
+ * argmax of each row's logits (ties: lowest id).  logits_dev [batch][n_rows][vocab] float out, or NULL.
+ * tree_tok_dev [batch][n_rows] int32 in; the caller may have edited it since hydra_draft.  A token id outside
+ * [0, vocab) raises the BOUNDS bit of the status word (the row is computed for token 0).  Errors: STATE, CAPACITY. */
 hydra_status hydra_verify(hydra_ctx*, const int32_t* tree_tok_dev, int32_t* amax_dev, float* logits_dev, void* stream);
 
-/* Greedy acceptance and in-place cache compaction in one kernel.  A candidate is accepted when it
+/* Acceptance and compaction (Background, verification criteria: the greedy criterion keeps a candidate
+ * that equals the base model's most likely token; Background, "Speculative decoding": the accepted tokens
+ * are appended to the sequence, the rest is discarded).  One kernel.  A candidate is accepted when it
  * equals amax of its parent and its parent is accepted; the deepest accepted row wins (lowest row
- * among equals).  n_acc_dev [batch]: accepted candidates (0..K); path_dev [batch][K+1]: accepted rows
+ * among equals); the accepted rows' K,V move to cache slots len+1..len+n in place.  n_acc_dev [batch]: accepted candidates (0..K); path_dev [batch][K+1]: accepted rows
  * root..best, -1 padded; out_tok_dev [batch][K+1]: accepted tokens then the bonus token, -1 padded.
  * Any of the three outputs may be NULL.  Updates the committed lengths, root tokens and hidden rows. */
 hydra_status hydra_accept_compact(hydra_ctx*, const int32_t* tree_tok_dev, const int32_t* amax_dev,
                                   int32_t* n_acc_dev, int32_t* path_dev, int32_t* out_tok_dev, void* stream);
 
-/* draft + (optional planting) + verify + accept_compact on the library's own buffers.  From the second step
- * after a prefill on, the step is captured into a CUDA graph (re-captured when an attention grid must grow
- * or a pointer argument changes) and replayed with one launch; set HYDRA_NO_GRAPH=1 to launch kernel by kernel. */
+/* One whole decoding step (the three passages above): draft + (optional planting) + verify + accept_compact
+ * on the library's own buffers.  n_acc_dev [batch], out_tok_dev [batch][K+1] as in hydra_accept_compact (either
+ * may be NULL).  From the second step after a prefill on, the step is captured into a CUDA graph (re-captured
+ * when an attention grid must grow or a pointer argument changes) and replayed with one launch, unless the stream
+ * is a default stream (not capturable) or hydra_set_step_graph switched graphs off.  Errors: STATE, CAPACITY. */
 hydra_status hydra_step(hydra_ctx*, int32_t* n_acc_dev, int32_t* out_tok_dev, void* stream);
+/* on = 0: hydra_step launches kernel by kernel (for profilers that list kernels); on = 1 (default): graph replay. */
+hydra_status hydra_set_step_graph(hydra_ctx*, int on);
 
 /* Accept-exercise mode: plant_dev [batch][n_rows], -1 keeps the drafted token; applied between draft
  * and verify inside hydra_step.  NULL disables.  The buffer is read at every step. */
@@ -140,7 +161,9 @@ enum {
   HYDRA_BUF_AMAX = 8,       /* int32 [batch][n_rows] */
   HYDRA_BUF_HEAD_LOGITS = 9,/* float [rows][vocab] logits of the last drafted level, row = b*parents+j */
   HYDRA_BUF_N_NEW = 10,     /* int32 [max_batch] rows in H_NEW */
-  HYDRA_BUF_H_PRIME = 11    /* float [max_batch][d] hidden state the heads consumed */
+  HYDRA_BUF_H_PRIME = 11,   /* float [max_batch][d] hidden state the heads consumed */
+  HYDRA_BUF_STATUS = 12     /* int32 [64]: [0] the device status word (bit 1 bounds, bit 2 timeout) that hydra_poll_status
+                               reads and clears, [8..15] where a bounded wait gave up (site, cta, unit, units, grid, m, n, k-blocks) */
 };
 hydra_status hydra_get_buffer(hydra_ctx*, int which, void** dev_ptr, size_t* bytes);
 
@@ -159,12 +182,8 @@ enum { HYDRA_TIME_GEMM = 0, HYDRA_TIME_ATTENTION = 1, HYDRA_TIME_ACCEPT = 2 };
 hydra_status hydra_set_timing(hydra_ctx*, int on);
 hydra_status hydra_get_timing(hydra_ctx*, int kclass, double* ms_total, long long* launches, double* bytes_total);
 
-/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA, one launch per GEMM and per row-wise kernel (default);
- * 1 = the plain SIMT kernel (debugging; it reads only the hi plane of the activations); 2 = tcgen05/TMA with
- * everything of a layer after its attention (O projection, residual + norm, gate/up, SiLU * up, down, residual +
- * norm, the next layer's QKV projection or the LM head) in ONE persistent, cooperatively launched kernel whose
- * CTAs hand over between GEMMs through grid-wide counters (same results as mode 0; currently slower, because a
- * hand-over costs more than a launch boundary; calls of two contexts in this mode must not overlap on the GPU). */
+/* Which GEMM the bfloat16 path uses: 0 = tcgen05/TMA (default); 1 = the plain SIMT kernel (debugging; it reads
+ * only the hi plane of the activations). */
 hydra_status hydra_set_gemm_mode(hydra_ctx*, int mode);
 
 const char* hydra_status_str(hydra_status);
@@ -204,6 +223,16 @@ hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, fl
  *     on the GPU (different streams, different threads) race on it: serialise them. */
 hydra_status hydra_gemm_noalloc(const void* x_dev, const void* w_dev, float* out_dev, int m, int n, int k,
                                 int32_t* status_dev, void* stream);
+/* hydra_gemm_bounded_wait_probe: exercises the give-up path of the tensor-core GEMM's bounded waits.  Runs the
+ * GEMM of hydra_gemm (dtype 1, mode 0, x_planes 1) on a problem small enough for ONE CTA (else UNSUPPORTED), with
+ * barrier waits limited to wait_limit polls (1..65536) and with the weight-tile request of k-block `skip_unit` left
+ * out, so the tensor-core lane's wait for that tile runs out: the kernel raises the TIMEOUT bit (2) in status_dev[0],
+ * records where it gave up in diag_dev (int32[8]: site, cta, unit, units, grid, m, n, k-blocks; site 3 = weight tile),
+ * lets its copies land, frees its tensor memory and returns; nothing faults and the context stays usable.
+ * partial_dev as in hydra_gemm; its contents are unspecified afterwards. */
+hydra_status hydra_gemm_bounded_wait_probe(const void* x_dev, const void* w_dev, float* partial_dev, int m, int n, int k,
+                                           int skip_unit, unsigned wait_limit, int32_t* status_dev, int32_t* diag_dev,
+                                           void* stream);
 size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
 hydra_status hydra_tree_attention(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev,
                                   const int32_t* pos0_dev, const int32_t* n_rows_dev, const uint64_t* mask_dev,

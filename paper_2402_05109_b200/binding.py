@@ -57,6 +57,7 @@ lib.hydra_poll_status.argtypes = [_vp, _vp]
 lib.hydra_launch_count.restype = C.c_longlong
 lib.hydra_launch_count.argtypes = [_vp]
 lib.hydra_set_gemm_mode.argtypes = [_vp, _i]
+lib.hydra_set_step_graph.argtypes = [_vp, _i]
 lib.hydra_set_timing.argtypes = [_vp, _i]
 lib.hydra_get_timing.argtypes = [_vp, _i, C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
 lib.hydra_status_str.restype = C.c_char_p
@@ -66,15 +67,16 @@ lib.hydra_gemm_partial_floats.restype = _sz
 lib.hydra_gemm_partial_floats.argtypes = [_i] * 5
 lib.hydra_gemm.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]
 lib.hydra_gemm_noalloc.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]
+lib.hydra_gemm_bounded_wait_probe.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, C.c_uint, _vp, _vp, _vp]
 lib.hydra_attention_scratch_bytes.restype = _sz
 lib.hydra_attention_scratch_bytes.argtypes = [_i] * 5
 lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 7 + [_vp]
 
 BUF = dict(LEN=0, ROOT_TOK=1, H_TREE=2, H_NEW=3, KV_BASE=4, KV_PREFIX=5, TREE_MASK=6, TREE_TOK=7, AMAX=8,
-           HEAD_LOGITS=9, N_NEW=10, H_PRIME=11)
+           HEAD_LOGITS=9, N_NEW=10, H_PRIME=11, STATUS=12)
 _BUF_DTYPE = dict(LEN=torch.int32, ROOT_TOK=torch.int32, H_TREE=torch.float32, H_NEW=torch.float32,
                   TREE_MASK=torch.int64, TREE_TOK=torch.int32, AMAX=torch.int32, HEAD_LOGITS=torch.float32,
-                  N_NEW=torch.int32, H_PRIME=torch.float32)
+                  N_NEW=torch.int32, H_PRIME=torch.float32, STATUS=torch.int32)
 
 
 def _check(code: int, what: str):
@@ -193,6 +195,9 @@ class Hydra:
     def set_gemm_mode(self, mode: int):
         _check(lib.hydra_set_gemm_mode(self._ctx, mode), "hydra_set_gemm_mode")
 
+    def set_step_graph(self, on: bool):
+        _check(lib.hydra_set_step_graph(self._ctx, int(on)), "hydra_set_step_graph")
+
     def set_timing(self, on: bool):
         _check(lib.hydra_set_timing(self._ctx, int(on)), "hydra_set_timing")
 
@@ -215,33 +220,28 @@ class Hydra:
         off = p.value - self.workspace.data_ptr()
         return self.workspace[off:off + n.value].view(_BUF_DTYPE.get(name, self.dtype))
 
-    def kv_base(self) -> torch.Tensor:
-        m = self.model
-        planes = 1 if self.dtype == torch.float32 else 2
-        kv = self.get_buffer("KV_BASE").view(m.n_layers, 2, planes, self.max_batch, m.n_heads, self.max_seq, m.head_dim)
-        return kv.float().sum(dim=2) if planes == 2 else kv[:, :, 0]          # hi + lo
-
-    def kv_prefix(self) -> torch.Tensor:
-        m = self.model
-        planes = 1 if self.dtype == torch.float32 else 2
-        kv = self.get_buffer("KV_PREFIX").view(2, planes, self.max_batch, m.n_heads, self.max_seq, m.head_dim)
-        return kv.float().sum(dim=1) if planes == 2 else kv[:, 0]
-
 
 # ---- single-kernel entry points (kernel-level parity tests)
-def split_hi_lo(x: torch.Tensor) -> torch.Tensor:
-    """[2, ...] bfloat16: hi = bf16(x), lo = bf16(x - hi) of a float tensor (the library's operand format)."""
-    hi = x.to(torch.bfloat16)
-    lo = (x.float() - hi.float()).to(torch.bfloat16)
-    return torch.stack([hi, lo]).contiguous()
+def _need(cond: bool, what: str):
+    if not cond:
+        raise HydraError("bad argument: " + what)
+
+
+def _dense_cuda(t: torch.Tensor, dtype, name: str):
+    _need(isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype,
+          "%s must be a contiguous CUDA tensor of %s" % (name, dtype))
 
 
 def gemm(x: torch.Tensor, w: torch.Tensor, mode: int = 0) -> torch.Tensor:
     """out[m][n] = sum_k x[m][k] w[n][k] in float; x, w both float32 or both bfloat16 CUDA tensors.
-    x may be [2][m][k] bfloat16 (hi/lo planes, see split_hi_lo)."""
+    x may be [2][m][k] bfloat16: the hi = bf16(v) and lo = bf16(v - hi) planes of float activations v."""
     planes = 2 if x.dim() == 3 else 1
     m, k = x.shape[-2:]
     n = w.shape[0]
+    _need(x.dtype in (torch.float32, torch.bfloat16), "x must be float32 or bfloat16")
+    _dense_cuda(x, x.dtype, "x")
+    _dense_cuda(w, x.dtype, "w")
+    _need(w.dim() == 2 and w.shape[1] == k and (planes == 1 or x.shape[0] == 2), "x [m][k] or [2][m][k], w [n][k]")
     dtype = 0 if x.dtype == torch.float32 else 1
     out = torch.empty(m, n, dtype=torch.float32, device="cuda")
     part = torch.empty(lib.hydra_gemm_partial_floats(m, n, k, dtype, mode), dtype=torch.float32, device="cuda")
@@ -258,8 +258,14 @@ def gemm_noalloc(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor, status: to
     """hydra_gemm_noalloc: bfloat16 tensor-core GEMM whose partial sums live in the library's built-in 8 MiB scratch.
     The caller passes every tensor (nothing is allocated here, on the host side either): x [m][k], w [n][k]
     bfloat16, out [m][n] float32, status int32[1].  Calls that overlap on the GPU race on the scratch."""
+    _dense_cuda(x, torch.bfloat16, "x")
+    _dense_cuda(w, torch.bfloat16, "w")
+    _dense_cuda(out, torch.float32, "out")
+    _dense_cuda(status, torch.int32, "status")
+    _need(x.dim() == 2 and w.dim() == 2 and w.shape[1] == x.shape[1], "x [m][k], w [n][k]")
     m, k = x.shape
     n = w.shape[0]
+    _need(tuple(out.shape) == (m, n) and status.numel() >= 1, "out [m][n], status int32[>=1]")
     _check(lib.hydra_gemm_noalloc(x.data_ptr(), w.data_ptr(), out.data_ptr(), m, n, k, status.data_ptr(), _stream()),
            "hydra_gemm_noalloc")
 
@@ -268,6 +274,15 @@ def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int) -> torch.Te
     """Caches [batch][H][S][hd] (one plane) or [2][batch][H][S][hd] (hi/lo planes, bfloat16); q and the result likewise."""
     planes = 2 if k_cache.dim() == 5 else 1
     batch, n_heads, max_seq, head_dim = k_cache.shape[-4:]
+    _need(k_cache.dtype in (torch.float32, torch.bfloat16), "caches must be float32 or bfloat16")
+    for name, t in (("q", q), ("k_cache", k_cache), ("v_cache", v_cache)):
+        _dense_cuda(t, k_cache.dtype, name)
+    _need(v_cache.shape == k_cache.shape and q.numel() == planes * batch * tc * n_heads * head_dim, "q / cache shapes")
+    _dense_cuda(pos0, torch.int32, "pos0")
+    _dense_cuda(mask, torch.int64, "mask")
+    _need(pos0.numel() == batch and mask.numel() == tc and (n_rows is None or n_rows.numel() == batch), "pos0 [batch], mask [tc]")
+    if n_rows is not None:
+        _dense_cuda(n_rows, torch.int32, "n_rows")
     dtype = 0 if k_cache.dtype == torch.float32 else 1
     shape = (batch * tc, n_heads * head_dim)
     out = torch.empty((planes,) + shape if planes == 2 else shape, dtype=k_cache.dtype, device="cuda")
@@ -277,3 +292,25 @@ def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int) -> torch.Te
                                     mask.data_ptr(), out.data_ptr(), scratch.data_ptr(), batch, tc, n_heads, head_dim,
                                     max_seq, dtype, planes, _stream()), "hydra_tree_attention")
     return out
+
+
+def gemm_bounded_wait_probe(x: torch.Tensor, w: torch.Tensor, skip_unit: int, wait_limit: int = 1024,
+                            status_words: Optional[torch.Tensor] = None):
+    """hydra_gemm_bounded_wait_probe: a one-CTA tensor-core GEMM whose weight tile `skip_unit` is never requested,
+    so a bounded wait runs out.  Returns (status word, diag int32[8]) as CPU values.  status_words: an int32[>=16]
+    CUDA tensor to use as status word ([0]) and diagnostics ([8..15]), e.g. a context's STATUS buffer."""
+    _dense_cuda(x, torch.bfloat16, "x")
+    _dense_cuda(w, torch.bfloat16, "w")
+    m, k = x.shape
+    n = w.shape[0]
+    _need(w.shape[1] == k, "w [n][k]")
+    part = torch.empty(lib.hydra_gemm_partial_floats(m, n, k, 1, 0), dtype=torch.float32, device="cuda")
+    if status_words is None:
+        status_words = torch.zeros(16, dtype=torch.int32, device="cuda")
+    _dense_cuda(status_words, torch.int32, "status_words")
+    _need(status_words.numel() >= 16, "status_words int32[>=16]")
+    status, diag = status_words[0:1], status_words[8:16]
+    _check(lib.hydra_gemm_bounded_wait_probe(x.data_ptr(), w.data_ptr(), part.data_ptr(), m, n, k, skip_unit, wait_limit,
+                                             status.data_ptr(), diag.data_ptr(), _stream()), "hydra_gemm_bounded_wait_probe")
+    torch.cuda.current_stream().synchronize()
+    return int(status.item()), diag.cpu().tolist()

@@ -451,8 +451,7 @@ hydra_status run_ns(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, 
                  float* scratch, int H, int max_seq, int len_upper, cudaStream_t st) {
   constexpr int TILE = 32;                    // 32-row tiles, four of them in flight: hides the HBM latency of a chunk's walk
   const int nchunks_max = (max_seq + ATT_CHUNK_ROWS - 1) / ATT_CHUNK_ROWS;     // what the scratch is sized for
-  static int sms = 0;
-  if (!sms) { int dev = 0; HYDRA_CUDA(cudaGetDevice(&dev)); HYDRA_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)); }
+  const int sms = sm_count();
   if ((size_t)H * rs.batch * sizeof(int) > ATT_SCRATCH_HEADER) return HYDRA_ERR_UNSUPPORTED;
   bool cluster = false;
   const int nchunks = pick_chunks(H * rs.batch, len_upper, TILE, nchunks_max, sms, &cluster);
@@ -465,11 +464,11 @@ hydra_status run_ns(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, 
   const size_t ring = (size_t)NP * 2 * NS * TILE * LDS * sizeof(bf16);
   const size_t xchg = (size_t)(4 * 32 * (HD / 2 + 4) + 64 * HD + 128) * sizeof(float);      // hand-over area + a chunk's partial rows + (m, l)
   const size_t smem = (size_t)NP * 64 * LDS * sizeof(bf16) + (ring > xchg ? ring : xchg);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceFlag attr_done;
+  if (!attr_done.get()) {
     HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE, NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE, NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_done = true;
+    attr_done.set();
   }
   if (!cluster) {
     launch_pdl(tree_attn_tc_kernel<HD, HL, TILE, NS, false>, dim3(H, rs.batch, nchunks), dim3(NWARP * 32), smem, st, q, q_ps, kc, vc, kv_ps, rs, part_o,

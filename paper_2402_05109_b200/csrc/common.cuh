@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <atomic>
 #include "../../include/hydra.h"
 
 namespace hydra {
@@ -16,6 +17,25 @@ enum : int { ST_BOUNDS = 1, ST_TIMEOUT = 2 };
 extern thread_local long long* g_launch_counter;
 void set_last_error(const char* what, cudaError_t e);
 inline void count_launch() { if (g_launch_counter) ++*g_launch_counter; }
+
+// Per-device one-time set-up (function attributes, SM counts) is keyed by the current device, so that one process
+// may drive several GPUs; the flags are atomics because any thread may make the first call on a device.
+constexpr int MAX_DEVICES = 64;
+inline int current_device() { int d = 0; return cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < MAX_DEVICES ? d : 0; }
+struct PerDeviceFlag {
+  std::atomic<bool> done[MAX_DEVICES];
+  bool get() const { return done[current_device()].load(std::memory_order_acquire); }
+  void set() { done[current_device()].store(true, std::memory_order_release); }
+};
+inline int sm_count() {
+  static std::atomic<int> n[MAX_DEVICES];
+  const int dev = current_device();
+  int v = n[dev].load(std::memory_order_relaxed);
+  if (v > 0) return v;
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1) v = 148;
+  n[dev].store(v, std::memory_order_relaxed);
+  return v;
+}
 
 #define HYDRA_CUDA(call)                                                        \
   do { cudaError_t e_ = (call);                                                 \

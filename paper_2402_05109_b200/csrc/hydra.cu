@@ -162,9 +162,9 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   size_t part_floats = 0;
   {
     auto need = [&](int mm, int n, int k) {
-      int slots = 1, slots1 = 1;
-      if (m.dtype == 1) { gemm_tc_plan(mm, n, k, nullptr, &slots); gemm_tc_plan(mm, n, k, nullptr, &slots1, 1); }      // stand-alone and chain plans
-      part_floats = std::max(part_floats, (size_t)std::max(slots, slots1) * mm * n);
+      int slots = 1;
+      if (m.dtype == 1) gemm_tc_plan(mm, n, k, nullptr, &slots);
+      part_floats = std::max(part_floats, (size_t)slots * mm * n);
     };
     const int shapes[][2] = {{3 * d, d}, {d, d}, {2 * f, d}, {d, f}, {V, d}};
     const int per_seq[] = {CHUNK, T, K + 1, 1};
@@ -183,7 +183,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   std::vector<int*> lvl;
   for (auto& lv : t.level_parents) lvl.push_back(b.take<int>(lv.size()));
   auto* len = b.take<int>(m.max_batch); auto* n_new = b.take<int>(m.max_batch); auto* root = b.take<int>(m.max_batch);
-  auto* status = b.take<int>(64);          // [0] status word, [8..15] where a bounded wait gave up, [32..48] the GEMM chain's counters
+  auto* status = b.take<int>(64);          // [0] status word, [8..15] where a bounded wait gave up
   auto* pos0 = b.take<int>(m.max_batch); auto* nrows = b.take<int>(m.max_batch);
   auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
   auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
@@ -264,28 +264,10 @@ double gemm_bytes(const hydra_ctx* c, int m, int n, int k) {        // weights +
 // The rest of a layer after its attention: O projection, + residual, RMSNorm, gate/up, SiLU * up, down, + residual and,
 // when next_gain is given, xn = rmsnorm(x) * next_gain (hn: the same in float); when next_w is given, also the
 // GEMM xn @ next_w^T (the next layer's QKV projection, or the LM head), whose partial sums stay in c->part (*sd).
-// Kernel by kernel, or (GEMM mode 2, bfloat16) all of it as ONE persistent kernel (gemm_chain).
 hydra_status mlp_block(hydra_ctx* c, const LayerW& w, int rows, const void* next_gain, float* hn, const void* next_w, int next_n,
                        SplitDesc* sd, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int d = m.d_model, f = m.d_ffn, dt = m.dtype;
-  if (dt == 1 && c->gemm_mode == 2) {
-    ChainStep steps[4] = {};
-    steps[0] = ChainStep{(const bf16*)c->attn_out, c->R, (const bf16*)w.wo, d, d, CHAIN_RESID_NORM, d, c->x, (const bf16*)w.ffn_norm,
-                         (bf16*)c->xn, ps(c, c->R, d), nullptr, m.rms_eps};
-    steps[1] = ChainStep{(const bf16*)c->xn, c->R, (const bf16*)w.w_gate_up, 2 * f, d, CHAIN_SILU_MUL, f, nullptr, nullptr,
-                         (bf16*)c->act, ps(c, c->R, f), nullptr, 0.f};
-    steps[2] = ChainStep{(const bf16*)c->act, c->R, (const bf16*)w.w_down, d, f, CHAIN_RESID_NORM, d, c->x, (const bf16*)next_gain,
-                         next_gain ? (bf16*)c->xn : nullptr, ps(c, c->R, d), hn, m.rms_eps};
-    int n = 3;
-    double bytes = gemm_bytes(c, rows, d, d) + gemm_bytes(c, rows, 2 * f, d) + gemm_bytes(c, rows, d, f);
-    if (next_w) {
-      steps[n++] = ChainStep{(const bf16*)c->xn, c->R, (const bf16*)next_w, next_n, d, CHAIN_NONE, 0, nullptr, nullptr, nullptr, 0, nullptr, 0.f};
-      bytes += gemm_bytes(c, rows, next_n, d);
-    }
-    TimeScope ts(c, HYDRA_TIME_GEMM, bytes, st);
-    return gemm_chain(steps, n, rows, c->planes, c->part, c->part_floats, sd, c->d_status, c->d_status + 8, c->d_status + 32, st);
-  }
   SplitDesc s1;
   HYDRA_TRY(run_gemm(c, c->attn_out, c->R, w.wo, rows, d, d, &s1, st));
   HYDRA_TRY(residual_rmsnorm(c->x, c->part, s1, c->x, w.ffn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, dt, st));
@@ -470,7 +452,7 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
   c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
   carve(c, *m, *h, th, (char*)ws);
   c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->plant = nullptr; c->launches = 0; c->timing = 0; c->steps_done = 0;
-  { const char* e = getenv("HYDRA_NO_GRAPH"); c->use_graph = !(e && e[0] == '1'); }
+  c->use_graph = 1;
   c->len_ub.assign(m->max_batch, 0);
   // clear the workspace, upload the static tables
   auto fail = [&](cudaError_t e, const char* what) { set_last_error(what, e); delete c; return HYDRA_ERR_CUDA; };
@@ -637,6 +619,7 @@ hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes
     case HYDRA_BUF_HEAD_LOGITS: p = c->head_logits; n = (size_t)c->RH * m.vocab * sizeof(float); break;
     case HYDRA_BUF_N_NEW: p = c->d_n_new; n = m.max_batch * sizeof(int); break;
     case HYDRA_BUF_H_PRIME: p = c->hprime; n = (size_t)m.max_batch * m.d_model * sizeof(float); break;
+    case HYDRA_BUF_STATUS: p = c->d_status; n = 64 * sizeof(int); break;
     default: return HYDRA_ERR_INVALID;
   }
   *ptr = p;
@@ -650,6 +633,13 @@ hydra_status hydra_poll_status(hydra_ctx* c, void* stream) {
   int word = 0;
   HYDRA_CUDA(cudaStreamSynchronize(st));
   HYDRA_CUDA(cudaMemcpy(&word, c->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (c->batch > 0 && (c->state == ST_READY || c->state == ST_DRAFTED)) {
+    // the stream is drained: replace the host's upper bounds of the lengths (which assume every step accepted a
+    // full path) by the real ones, so that the capacity check and the attention grids follow the real cache use
+    std::vector<int> len(c->batch);
+    HYDRA_CUDA(cudaMemcpy(len.data(), c->d_len, c->batch * sizeof(int), cudaMemcpyDeviceToHost));
+    for (int b = 0; b < c->batch; ++b) if (len[b] >= 0 && len[b] < c->len_ub[b]) c->len_ub[b] = len[b];
+  }
   if (word & ST_TIMEOUT) {
     int d[8] = {0};
     cudaMemcpy(d, c->d_status + 8, sizeof(d), cudaMemcpyDeviceToHost);
@@ -688,8 +678,14 @@ hydra_status hydra_get_timing(hydra_ctx* c, int kclass, double* ms_total, long l
   return HYDRA_OK;
 }
 
+hydra_status hydra_set_step_graph(hydra_ctx* c, int on) {
+  if (!c) return HYDRA_ERR_INVALID;
+  c->use_graph = on ? 1 : 0;
+  return HYDRA_OK;
+}
+
 hydra_status hydra_set_gemm_mode(hydra_ctx* c, int mode) {
-  if (!c || mode < 0 || mode > 2) return HYDRA_ERR_INVALID;
+  if (!c || mode < 0 || mode > 1) return HYDRA_ERR_INVALID;
   c->gemm_mode = mode;
   drop_graphs(c);
   return HYDRA_OK;
@@ -733,6 +729,19 @@ hydra_status hydra_gemm(const void* x, const void* w, float* out, float* partial
     return reduce_splits(partial, sd, out, m, n, st);
   }
   return gemm_simt(x, w, out, m, n, k, dtype, st);
+}
+
+hydra_status hydra_gemm_bounded_wait_probe(const void* x, const void* w, float* partial, int m, int n, int k, int skip_unit,
+                                           unsigned wait_limit, int32_t* status, int32_t* diag, void* stream) {
+  if (!x || !w || !partial || !status || !diag || m < 1 || n < 1 || k < 1 || wait_limit < 1 || wait_limit > (1u << 16)) return HYDRA_ERR_INVALID;
+  int grid = 0;
+  gemm_tc_plan(m, n, k, &grid, nullptr);
+  if (n % 128 || k % 64 || grid != 1) return HYDRA_ERR_UNSUPPORTED;     // one CTA: nothing else waits on the missing tile
+  if (!gemm_tc_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
+  CounterScope cs(nullptr);
+  GemmDebug dbg{wait_limit, skip_unit};
+  SplitDesc sd;
+  return gemm_tc((const bf16*)x, m, 1, (const bf16*)w, partial, m, n, k, &sd, status, diag, &dbg, (cudaStream_t)stream);
 }
 
 size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq) {

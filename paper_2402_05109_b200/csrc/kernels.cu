@@ -420,10 +420,10 @@ static hydra_status tree_attention_t(const T* q, const T* kc, const T* vc, RowSe
   float* part_o = scratch;
   float* part_ml = scratch + rows * H * nchunks_max * HD;
   size_t smem = (size_t)(64 * HD + ATT_TILE * (HD + 1) + ATT_TILE * HD) * sizeof(float);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceFlag attr_done;
+  if (!attr_done.get()) {
     HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_kernel<T, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_done = true;
+    attr_done.set();
   }
   launch_pdl(tree_attn_kernel<T, HD>, dim3(dim3(H, rs.batch, nchunks)), dim3(ATT_WARPS * 32), smem, st, q, kc, vc, rs, part_o, part_ml, H,
                                                                                    max_seq, nchunks);
@@ -782,7 +782,7 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
 hydra_status accept_compact(const AcceptArgs& a, cudaStream_t st) {
   long long units = (long long)a.n_layers * 2 * a.kv_planes * a.n_heads * (a.head_dim * a.esize / 16);
   int G = (int)((units + 255) / 256);
-  int cap = (148 * 4 + a.batch - 1) / a.batch;
+  int cap = (sm_count() * 4 + a.batch - 1) / a.batch;
   if (G > cap) G = cap;
   if (G < 1) G = 1;
   launch_pdl(accept_compact_kernel, dim3(dim3(G, a.batch)), dim3(256), 0, st, a);

@@ -8,22 +8,10 @@ namespace hydra {
 // tcgen05 path (bfloat16 operands).  x_rows_alloc = rows the x buffer really holds (>= m); rows of the last
 // tile beyond m are computed and dropped.  part needs gemm_tc_plan(...)'s max_slots * m * n floats.
 // x holds x_planes (1 or 2) planes of x_rows_alloc rows each: plane 0 = bf16(v), plane 1 = bf16(v - plane 0).
-// A chain of GEMMs over the same m rows in one persistent kernel.  After each job but (optionally) the last, a row-wise
-// step turns the job's partial sums into the next job's activations:
-//   CHAIN_RESID_NORM: resid[m][cols] += sums; with a gain: out (hi/lo planes, plane distance out_ps) and hn (float, optional)
-//                     = resid * rsqrt(mean(resid^2) + eps) * gain
-//   CHAIN_SILU_MUL:   out[m][cols] = SiLU(sums[:, :cols]) * sums[:, cols:]
-// The last job may be CHAIN_NONE: its partial sums stay in `part` for the caller's consumer kernel (*last_sd).
-// `sync` points to 17 zeroed ints that the kernel leaves zeroed.
-enum { CHAIN_NONE = 0, CHAIN_RESID_NORM = 1, CHAIN_SILU_MUL = 2 };
-struct ChainStep {
-  const bf16* x; int x_rows_alloc; const bf16* w; int n, k;
-  int op, cols; float* resid; const bf16* gain; bf16* out; size_t out_ps; float* hn; float eps;
-};
-hydra_status gemm_chain(const ChainStep* steps, int n_steps, int m, int x_planes, float* part, size_t part_floats, SplitDesc* last_sd,
-                        int* status, int* diag, int* sync, cudaStream_t st);
+// dbg (tests of the bounded waits only): a shorter poll limit and one weight-tile request that CTA 0 leaves out.
+struct GemmDebug { uint32_t wait_limit; int skip_unit; };
 hydra_status gemm_tc(const bf16* x, int x_rows_alloc, int x_planes, const bf16* w, float* part, int m, int n, int k,
-                     SplitDesc* sd_out, int* status, int* diag /*int[8] or null*/, long long* trace, cudaStream_t st);
+                     SplitDesc* sd_out, int* status, int* diag /*int[8] or null*/, const GemmDebug* dbg /*null: defaults*/, cudaStream_t st);
 SplitDesc gemm_tc_plan(int m, int n, int k, int* grid, int* max_slots, int force_nh = 0);   // force_nh: 128-row weight tiles per unit (0: the kernel's own choice)
 int gemm_tile_rows(int m);                // activation rows per MMA tile for an m-row GEMM: 16, 32, 64, 128 or 256
 bool gemm_tc_available();                 // driver entry point for tensor-map encoding found

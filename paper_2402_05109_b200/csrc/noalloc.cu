@@ -14,9 +14,9 @@ namespace {
 constexpr size_t NOALLOC_SCRATCH_BYTES = 8u << 20;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
-constexpr int MAX_DEVICES = 64;
-float* g_scratch_ptr[MAX_DEVICES];          // device address of the array, per device (filled on first use)
-bool g_scratch_ready[MAX_DEVICES];
+// device address of the array, per device; 0 until the first call on that device has looked it up (any thread may
+// make that call: the slot is an atomic, and two threads racing on it store the same address)
+std::atomic<uintptr_t> g_scratch_ptr[hydra::MAX_DEVICES];
 
 }  // namespace
 
@@ -34,16 +34,17 @@ extern "C" hydra_status hydra_gemm_noalloc(const void* x, const void* w, float* 
   int dev = -1;
   HYDRA_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= MAX_DEVICES) return HYDRA_ERR_UNSUPPORTED;
-  if (!g_scratch_ready[dev]) {
+  uintptr_t addr = g_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (!addr) {
     // The array's name is only a host-side handle here; the kernels need its address on the current device.
     void* p = nullptr;
     HYDRA_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
-    g_scratch_ptr[dev] = static_cast<float*>(p);
-    g_scratch_ready[dev] = true;
+    addr = reinterpret_cast<uintptr_t>(p);
+    g_scratch_ptr[dev].store(addr, std::memory_order_release);
   }
   if (!gemm_tc_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
   cudaStream_t st = (cudaStream_t)stream;
-  float* part = g_scratch_ptr[dev];
+  float* part = reinterpret_cast<float*>(addr);
   // every partial element the reduction reads is written by the GEMM first, so nothing has to be cleared
   SplitDesc sd;
   HYDRA_TRY(gemm_tc((const bf16*)x, m, 1, (const bf16*)w, part, m, n, k, &sd, status, nullptr, nullptr, st));

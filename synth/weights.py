@@ -1,4 +1,4 @@
-"""Random-initialised weights: every linear, embedding and bias entry ~ N(0, 0.02), norm gains 1.
+"""Random-initialised weights: every linear, embedding and bias entry ~ N(0, 0.02), norm gains 1 (or, on request, random).
 
 Each tensor is its own random stream (keyed by its name), so single tensors or layers can be
 regenerated on demand without holding a whole model.  All matrices are row-major [out][in].
@@ -41,10 +41,15 @@ def weight_names(m: ModelCfg, h: HeadCfg) -> List[str]:
     return list(weight_shapes(m, h).keys())
 
 
-def make_tensor(m: ModelCfg, h: HeadCfg, seed: int, name: str, device="cpu") -> torch.Tensor:
+def make_tensor(m: ModelCfg, h: HeadCfg, seed: int, name: str, device="cpu", norm_gain_std: float = 0.0) -> torch.Tensor:
+    """norm_gain_std > 0 draws every norm gain as 1 + norm_gain_std * N(0,1) from the tensor's own stream (parity
+    tests use it so that each norm's gain vector is distinguishable); the benchmark shapes keep gains of 1."""
     shape = weight_shapes(m, h)[name]
     dtype = torch.float32 if m.dtype == "fp32" else torch.bfloat16
     if name.endswith("norm"):
+        if norm_gain_std > 0.0:
+            g = normal_(torch.empty(shape, dtype=torch.float64, device=device), seed, zlib.crc32(name.encode()), norm_gain_std)
+            return (1.0 + g).to(dtype)
         return torch.ones(shape, dtype=dtype, device=device)
     out = torch.empty(shape, dtype=dtype, device=device)
     if not h.has_bias and (name.endswith(".b1") or name.endswith(".br")):
@@ -52,6 +57,7 @@ def make_tensor(m: ModelCfg, h: HeadCfg, seed: int, name: str, device="cpu") -> 
     return normal_(out, seed, zlib.crc32(name.encode()), STD)
 
 
-def make_weights(m: ModelCfg, h: HeadCfg, seed: int, device="cpu", names: Optional[List[str]] = None):
+def make_weights(m: ModelCfg, h: HeadCfg, seed: int, device="cpu", names: Optional[List[str]] = None,
+                 norm_gain_std: float = 0.0):
     names = weight_names(m, h) if names is None else names
-    return {n: make_tensor(m, h, seed, n, device) for n in names}
+    return {n: make_tensor(m, h, seed, n, device, norm_gain_std) for n in names}

@@ -19,6 +19,30 @@ LOGIT_TOL = 5e-2
 GAP = 0.1
 
 
+def split_hi_lo(x: torch.Tensor) -> torch.Tensor:
+    """[2, ...] bfloat16: hi = bf16(x), lo = bf16(x - hi) of a float tensor (how the library stores bfloat16-path
+    activations and cache rows)."""
+    hi = x.to(torch.bfloat16)
+    lo = (x.float() - hi.float()).to(torch.bfloat16)
+    return torch.stack([hi, lo]).contiguous()
+
+
+def kv_planes(g, which: str) -> torch.Tensor:
+    """Raw view of a cache buffer: KV_BASE -> [layers][k,v][planes][batch][heads][seq][hd], KV_PREFIX without the
+    layer axis.  planes = 2 (hi, lo) on the bfloat16 path, 1 on the float path."""
+    m = g.model
+    planes = 1 if g.dtype == torch.float32 else 2
+    shape = (2, planes, g.max_batch, m.n_heads, g.max_seq, m.head_dim)
+    if which == "KV_BASE":
+        shape = (m.n_layers,) + shape
+    return g.get_buffer(which).view(shape)
+
+
+def kv_values(g, which: str) -> torch.Tensor:
+    """Cache values as float (hi + lo): KV_BASE -> [layers][k,v][batch][heads][seq][hd]."""
+    return kv_planes(g, which).float().sum(dim=-5)
+
+
 def rel_l2(a: torch.Tensor, b: torch.Tensor) -> float:
     a, b = a.double().flatten(), b.double().flatten()
     return float((a - b).norm() / (b.norm() + 1e-30))
@@ -33,6 +57,8 @@ class Stats:
     max_hidden_err: float = 0.0
     max_head_logit_err: float = 0.0
     max_kv_err: float = 0.0
+    max_hprime_err: float = 0.0
+    max_prefix_kv_err: float = 0.0
     n_acc: List[List[int]] = field(default_factory=list)
 
 
@@ -68,6 +94,9 @@ def lockstep(o: HydraOracle, g, prompts, steps: int, seed: int, plant: bool = Tr
     o.prefill(prompts)
     g.prefill(prompts)
     g.poll_status()
+    # the ancestor-or-self bitmask is an integer output: bit for bit
+    mask_g = g.get_buffer("TREE_MASK")[:T].cpu().tolist()
+    assert [v & ((1 << 64) - 1) for v in mask_g] == o.tree.anc_mask, "tree mask differs"
     lens = g.get_buffer("LEN")[:B].cpu().tolist()
     assert lens == o.len
     hn = g.get_buffer("H_NEW").view(g.max_batch, K + 1, m.d_model)
@@ -87,6 +116,20 @@ def lockstep(o: HydraOracle, g, prompts, steps: int, seed: int, plant: bool = Tr
         tok_g = g.draft()
         g.poll_status()
         assert tok_g[:, 0].cpu().tolist() == o.root_tok
+        # the hidden state the heads consumed, and (Hydra++) the extra layer's cache over the committed rows
+        hp = g.get_buffer("H_PRIME").view(g.max_batch, m.d_model)
+        for b in range(B):
+            e = rel_l2(hp[b].cpu(), o.hprime[b])
+            st.max_hprime_err = max(st.max_hprime_err, e)
+            assert e <= HID_TOL, f"step {s}: h' rel-L2 {e}"
+        if o.h.prefix_attn:
+            pkv = kv_values(g, "KV_PREFIX")
+            for b in range(B):
+                L = o.len[b]
+                for which, ref in ((0, o.pk[b]), (1, o.pv[b])):
+                    e = rel_l2(pkv[which, b, :, :L].permute(1, 0, 2).cpu(), ref[:L])
+                    st.max_prefix_kv_err = max(st.max_prefix_kv_err, e)
+                    assert e <= HID_TOL, f"step {s}: prefix-layer cache rel-L2 {e}"
         if check_heads:
             tg = tok_g.cpu().long()
             for b in range(B):
@@ -137,7 +180,7 @@ def lockstep(o: HydraOracle, g, prompts, steps: int, seed: int, plant: bool = Tr
         assert g.get_buffer("ROOT_TOK")[:B].cpu().tolist() == o.root_tok
         assert g.get_buffer("N_NEW")[:B].cpu().tolist() == [int(n) + 1 for n in n_o]
         st.n_acc.append(n_o.tolist())
-        kv = g.kv_base()
+        kv = kv_values(g, "KV_BASE")
         for l in kv_layers:
             for b in range(B):
                 L = o.len[b]

@@ -65,7 +65,7 @@ def test_c3_7b_ragged_batches():
     wg, wc = weights_both(cfg8)
     for b in (2, 4, 8):
         lens = cfg8.prompt_lens[:b]
-        st = run_cfg(cfg8, wg, wc, lens, 2, max(lens) + 2 * 5 + 64 + 8, kv_layers=(0,), check_heads=(b == 2))
+        st = run_cfg(cfg8, wg, wc, lens, 2, max(lens) + 2 * 5 + 64 + 8, kv_layers=(0,))
         assert len({n for s in st.n_acc for n in s}) >= 2          # accepted lengths differ across the batch
     del wg, wc
     cleanup()
@@ -82,6 +82,6 @@ def test_c4_13b_long_prompt():
 def test_c5_33b_batch4():
     cfg = get_config("c5")
     wg, wc = weights_both(cfg)
-    run_cfg(cfg, wg, wc, [128] * 4, 2, 128 + 2 * 5 + 64 + 8, kv_layers=(0,), check_heads=False)
+    run_cfg(cfg, wg, wc, [128] * 4, 2, 128 + 2 * 5 + 64 + 8, kv_layers=(0,))
     del wg, wc
     cleanup()

@@ -5,6 +5,7 @@ import torch
 
 from oracle.hydra_oracle import masked_attention, TreeTables
 from synth import normal_, load_tree
+from tests.parity import split_hi_lo
 
 pytestmark = pytest.mark.gpu
 
@@ -32,7 +33,7 @@ def test_gemm_tensor_core_matches_definition(m, n, k):
 @pytest.mark.parametrize("m,n,k", [(64, 512, 4096), (11, 256, 1280), (300, 384, 704)])
 def test_gemm_hi_lo_activation_planes(m, n, k):
     """Float activations passed as hi/lo bfloat16 planes: the product must match the float activations to ~2^-16."""
-    from paper_2402_05109_b200 import gemm, split_hi_lo
+    from paper_2402_05109_b200 import gemm
     x = rnd((m, k), 15, m + k, torch.float32)
     w = rnd((n, k), 16, n + k, torch.bfloat16, 0.02)
     ref = x.double() @ w.double().T
@@ -59,7 +60,7 @@ def test_gemm_float(m, n, k):
 def test_tree_attention_matches_masked_softmax(dtype, planes, hd, case):
     """few_chunks: at most 8 KV chunks per (head, sequence), which the bfloat16 kernel merges inside a thread-block
     cluster; many_chunks: one long sequence with two heads, 12 chunks, merged through scratch by the last CTA."""
-    from paper_2402_05109_b200 import tree_attention, split_hi_lo
+    from paper_2402_05109_b200 import tree_attention
     parent = load_tree("tree63_d4")
     t = TreeTables(parent)
     tc = t.T
@@ -89,3 +90,31 @@ def test_tree_attention_matches_masked_softmax(dtype, planes, hd, case):
         err = float((out[b, :n].double() - ref).abs().max())
         tol = 2e-5 if dtype == torch.float32 else (2e-4 if planes == 2 else 2e-2)
         assert err <= tol, err
+
+
+def test_bounded_wait_gives_up_and_the_context_stays_usable():
+    """A one-CTA GEMM whose third weight tile is never requested: the tensor-core lane's bounded wait for it (or the
+    epilogue's wait for the accumulator that then never completes) runs out, the kernel reports TIMEOUT with the place
+    it gave up and returns.  Through a context's status buffer hydra_poll_status turns that into an error and clears
+    it; the next ordinary GEMM is exact."""
+    from paper_2402_05109_b200 import Hydra, HydraError, gemm, gemm_bounded_wait_probe
+    from synth import make_weights
+    from synth.configs import ModelCfg, HeadCfg
+    m, n, k = 16, 128, 256                           # 4 k-blocks: the stream-K plan is a single CTA
+    x = rnd((m, k), 41, 1, torch.bfloat16).cuda()
+    w = rnd((n, k), 41, 2, torch.bfloat16, 0.02).cuda()
+    word, diag = gemm_bounded_wait_probe(x, w, skip_unit=2, wait_limit=1024)
+    assert word & 2, word                            # TIMEOUT bit
+    assert diag[0] in (3, 5), diag                   # gave up waiting for the weight tile / for the accumulator
+    assert diag[1] == 0 and diag[3] == 4 and diag[4] == 1 and diag[5:8] == [m, n, 4], diag
+    mc = ModelCfg(1, 256, 4, 64, 512, 1024, dtype="bf16")
+    hc = HeadCfg(1, 1, False)
+    g = Hydra(mc, hc, [-1, 0], {kk: v.cuda() for kk, v in make_weights(mc, hc, 8).items()}, 1, 32)
+    gemm_bounded_wait_probe(x, w, skip_unit=1, wait_limit=512, status_words=g.get_buffer("STATUS"))
+    with pytest.raises(HydraError, match="timed out"):
+        g.poll_status()
+    g.poll_status()                                  # cleared by the poll
+    g.close()
+    ref = x.double().cpu() @ w.double().cpu().T
+    out = gemm(x, w, mode=0).cpu().double()          # the device and the library are fine afterwards
+    assert float((out - ref).abs().max()) <= 1e-5 * float(ref.abs().max()) + 1e-6 * k ** 0.5

@@ -10,14 +10,16 @@ from tests.parity import lockstep
 pytestmark = pytest.mark.gpu
 
 
-def run(model, head, parent, prompts_lens, steps, seed, max_seq, oracle_dtype=torch.float64, weights_device="cpu", **kw):
+def run(model, head, parent, prompts_lens, steps, seed, max_seq, oracle_dtype=torch.float64, weights_device="cpu",
+        norm_gain_std=0.0, gemm_mode=0, **kw):
     from paper_2402_05109_b200 import Hydra
-    w = make_weights(model, head, seed, device=weights_device)
+    w = make_weights(model, head, seed, device=weights_device, norm_gain_std=norm_gain_std)
     wg = {k: v.cuda() for k, v in w.items()}
     wc = {k: v.cpu() for k, v in w.items()}
     prompts = make_prompts(seed, prompts_lens, model.vocab)
     o = HydraOracle(model, head, parent, wc, max_seq, dtype=oracle_dtype, cache_weights=True)
     g = Hydra(model, head, parent, wg, max_batch=len(prompts), max_seq=max_seq)
+    g.set_gemm_mode(gemm_mode)
     try:
         return lockstep(o, g, prompts, steps, seed, **kw), g
     finally:
@@ -43,9 +45,21 @@ def test_small_bf16_hydrapp_ragged_batch():
     assert seen >= {0, 1, 2, 3, 4}, seen
 
 
-@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("dtype,gemm_mode", [("bf16", 0), ("bf16", 1), ("fp32", 0)])
+def test_random_norm_gains_reach_the_right_norms(dtype, gemm_mode):
+    """Every RMSNorm gain vector (2 per layer, the final norm, the prefix layer's 2) drawn as 1 + 0.1 N(0,1) from its
+    own stream: a kernel that ignored a gain, or read another norm's, would leave the tolerances at once (a 10 %
+    per-channel error).  The benchmark shapes use gains of 1, which cannot show this."""
+    m = ModelCfg(3, 256, 2, 128, 512, 1024, dtype=dtype)
+    h = HeadCfg(4, 2, True)
+    st, _ = run(m, h, load_tree("tree63_d4"), [37, 70], 3, 21, 192, norm_gain_std=0.1, gemm_mode=gemm_mode,
+                kv_layers=(0, 1, 2))
+    assert st.steps == 3
+
+
+@pytest.mark.parametrize("mode", [1])
 def test_small_bf16_other_gemm_modes_and_root_only_tree(mode):
-    """mode 1: the SIMT GEMM (reads only the hi plane of the activations); mode 2: one persistent kernel per layer tail."""
+    """mode 1: the SIMT GEMM (reads only the hi plane of the activations)."""
     from paper_2402_05109_b200 import Hydra
     m = ModelCfg(2, 256, 4, 64, 512, 1024, dtype="bf16")
     h = HeadCfg(2, 1, False)
@@ -77,6 +91,38 @@ def test_chain_tree_and_capacity_and_state_errors():
     with pytest.raises(HydraError, match="capacity"):
         g.step()
     assert g.launch_count() == before
+    g.close()
+
+
+def test_polling_lets_decoding_use_the_whole_cache():
+    """The host's length bounds grow by K+1 per step; hydra_poll_status replaces them by the real lengths.  With
+    root-only acceptance (random candidates are rejected) a sequence grows by one token per step, so a caller
+    that polls must be able to decode until len + T == max_seq, far beyond what the bounds alone allow."""
+    from paper_2402_05109_b200 import Hydra, HydraError
+    m = ModelCfg(1, 256, 4, 64, 512, 1024, dtype="fp32")
+    h = HeadCfg(3, 1, False)
+    parent = chain_tree(3)
+    T, max_seq, plen = len(parent), 64, 20
+    w = make_weights(m, h, 12)
+    g = Hydra(m, h, parent, {k: v.cuda() for k, v in w.items()}, 1, max_seq)
+    g.prefill(make_prompts(12, [plen], m.vocab))
+    never = torch.full((1, T), -1, dtype=torch.int32)
+    never[0, 1] = m.vocab - 1                       # planted first candidate: (almost surely) not the base argmax
+    g.set_plant(never.cuda())
+    n_acc = torch.empty(1, dtype=torch.int32, device="cuda")
+    steps, lens = 0, []
+    while True:
+        try:
+            g.step(n_acc)
+        except HydraError as e:
+            assert "capacity" in str(e)
+            break
+        g.poll_status()
+        steps += 1
+        lens.append(int(g.get_buffer("LEN")[0]))
+        assert steps < 200
+    assert lens[-1] + T > max_seq and lens[-1] <= max_seq          # stopped only when the cache was really full
+    assert steps > (max_seq - T - plen) // (h.n_heads + 1) + 2     # more steps than the un-refreshed bounds allow
     g.close()
 
 
@@ -123,20 +169,3 @@ def test_step_graph_replay_matches_kernel_by_kernel_launches():
         assert g.launch_count() > 100 * 50
         g.close()
     assert torch.equal(outs[0], outs[1])
-
-
-def test_small_bf16_hydra_pp_gemm_chain_mode():
-    """GEMM mode 2 (layer tail as one persistent kernel with grid-wide hand-overs) against the oracle: prefix layer,
-    63-node tree, ragged batch of 3, graph replay from the second step on."""
-    from paper_2402_05109_b200 import Hydra
-    m = ModelCfg(3, 256, 2, 128, 512, 1024, dtype="bf16")
-    h = HeadCfg(4, 2, True)
-    parent = load_tree("tree63_d4")
-    w = make_weights(m, h, 11)
-    prompts = make_prompts(11, [37, 130, 64], m.vocab)
-    o = HydraOracle(m, h, parent, w, 256, cache_weights=True)
-    g = Hydra(m, h, parent, {k: v.cuda() for k, v in w.items()}, 3, 256)
-    g.set_gemm_mode(2)
-    st = lockstep(o, g, prompts, 4, 11)
-    assert st.steps == 4
-    g.close()
