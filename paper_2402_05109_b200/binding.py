@@ -70,7 +70,7 @@ lib.hydra_gemm_noalloc.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]
 lib.hydra_gemm_bounded_wait_probe.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, C.c_uint, _vp, _vp, _vp]
 lib.hydra_attention_scratch_bytes.restype = _sz
 lib.hydra_attention_scratch_bytes.argtypes = [_i] * 5
-lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 7 + [_vp]
+lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 7 + [_vp, _vp]
 
 BUF = dict(LEN=0, ROOT_TOK=1, H_TREE=2, H_NEW=3, KV_BASE=4, KV_PREFIX=5, TREE_MASK=6, TREE_TOK=7, AMAX=8,
            HEAD_LOGITS=9, N_NEW=10, H_PRIME=11, STATUS=12)
@@ -214,11 +214,13 @@ class Hydra:
         return int(lib.hydra_launch_count(self._ctx))
 
     def get_buffer(self, name: str) -> torch.Tensor:
-        """A tensor view of a library buffer (flat; KV buffers in the cache dtype)."""
+        """A tensor view of a library buffer (flat; KV buffers in the cache element type: float32 on the float path,
+        float16 on the bfloat16 path)."""
         p, n = C.c_void_p(), C.c_size_t()
         _check(lib.hydra_get_buffer(self._ctx, BUF[name], C.byref(p), C.byref(n)), "hydra_get_buffer")
         off = p.value - self.workspace.data_ptr()
-        return self.workspace[off:off + n.value].view(_BUF_DTYPE.get(name, self.dtype))
+        cache_dtype = torch.float32 if self.dtype == torch.float32 else torch.float16
+        return self.workspace[off:off + n.value].view(_BUF_DTYPE.get(name, cache_dtype))
 
 
 # ---- single-kernel entry points (kernel-level parity tests)
@@ -270,27 +272,39 @@ def gemm_noalloc(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor, status: to
            "hydra_gemm_noalloc")
 
 
-def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int) -> torch.Tensor:
-    """Caches [batch][H][S][hd] (one plane) or [2][batch][H][S][hd] (hi/lo planes, bfloat16); q and the result likewise."""
-    planes = 2 if k_cache.dim() == 5 else 1
-    batch, n_heads, max_seq, head_dim = k_cache.shape[-4:]
-    _need(k_cache.dtype in (torch.float32, torch.bfloat16), "caches must be float32 or bfloat16")
+def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int, out_planes: int = 1) -> torch.Tensor:
+    """hydra_tree_attention.  q [batch*tc][H][hd], caches [batch][H][S][hd]: all float32, or all float16 (the bfloat16
+    model path, whose result is bfloat16 in out_planes planes: [rows][H*hd] or [2][rows][H*hd] = hi, lo).
+    mask: int64 [tc] ancestor bitmasks, or None for a causal chunk (float16 only)."""
+    batch, n_heads, max_seq, head_dim = k_cache.shape
+    _need(k_cache.dtype in (torch.float32, torch.float16), "caches must be float32 or float16")
     for name, t in (("q", q), ("k_cache", k_cache), ("v_cache", v_cache)):
         _dense_cuda(t, k_cache.dtype, name)
-    _need(v_cache.shape == k_cache.shape and q.numel() == planes * batch * tc * n_heads * head_dim, "q / cache shapes")
+    _need(v_cache.shape == k_cache.shape and q.numel() == batch * tc * n_heads * head_dim, "q / cache shapes")
     _dense_cuda(pos0, torch.int32, "pos0")
-    _dense_cuda(mask, torch.int64, "mask")
-    _need(pos0.numel() == batch and mask.numel() == tc and (n_rows is None or n_rows.numel() == batch), "pos0 [batch], mask [tc]")
+    _need(pos0.numel() == batch and (n_rows is None or n_rows.numel() == batch), "pos0 [batch], n_rows [batch]")
+    if mask is not None:
+        _dense_cuda(mask, torch.int64, "mask")
+        _need(mask.numel() == tc, "mask [tc]")
     if n_rows is not None:
         _dense_cuda(n_rows, torch.int32, "n_rows")
-    dtype = 0 if k_cache.dtype == torch.float32 else 1
     shape = (batch * tc, n_heads * head_dim)
-    out = torch.empty((planes,) + shape if planes == 2 else shape, dtype=k_cache.dtype, device="cuda")
-    scratch = torch.empty(lib.hydra_attention_scratch_bytes(batch, tc, n_heads, head_dim, max_seq), dtype=torch.uint8,
-                          device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    if k_cache.dtype == torch.float32:
+        _need(mask is not None and out_planes == 1, "the float path needs a mask and has one output plane")
+        out = torch.empty(shape, dtype=torch.float32, device="cuda")
+        scratch = torch.empty(lib.hydra_attention_scratch_bytes(batch, tc, n_heads, head_dim, max_seq), dtype=torch.uint8,
+                              device="cuda")
+        dtype = 0
+    else:
+        out = torch.empty((2,) + shape if out_planes == 2 else shape, dtype=torch.bfloat16, device="cuda")
+        scratch, dtype = None, 1
     _check(lib.hydra_tree_attention(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), pos0.data_ptr(), _ptr(n_rows),
-                                    mask.data_ptr(), out.data_ptr(), scratch.data_ptr(), batch, tc, n_heads, head_dim,
-                                    max_seq, dtype, planes, _stream()), "hydra_tree_attention")
+                                    _ptr(mask), out.data_ptr(), _ptr(scratch), batch, tc, n_heads, head_dim,
+                                    max_seq, dtype, out_planes, status.data_ptr(), _stream()), "hydra_tree_attention")
+    word = int(status.item())
+    if word:
+        raise HydraError("hydra_tree_attention device status word %d" % word)
     return out
 
 

@@ -1,56 +1,50 @@
-// Tree attention for bfloat16 caches on the tensor cores (mma.sync m16n8k16, float accumulate).
+// Tree attention for the bfloat16 model path on the sm_100a tensor cores: TMA tile loads, tcgen05.mma with the
+// score and output accumulators in tensor memory, softmax out of tensor memory.
 //
-// One CTA per (head, sequence, KV chunk).  A sequence's KV rows are cut into TILE-row tiles and the tiles are dealt
-// to the grid's chunks in equal contiguous runs (computed on the device from the real length, so every chunk of
-// the launch has work whatever the length); Q and the chunk's K and V tiles are streamed once through a five-stage
-// cp.async ring (four tiles in flight per CTA: the walk is bound by HBM latency otherwise).  Eight warps: warp w
-// owns query rows 16 (w & 3) .. +15 (as MMA fragments) and the keys of half (w >> 2) of every tile.  Scores of
-// committed slots are unmasked; a tree slot j is visible to row i iff bit j of the row's ancestor bitmask is set.
-// Each warp keeps a running (max, sum, weighted V) per query row in the exp2 domain (online softmax, reductions by
-// warp shuffles over the 4 lanes that share a row); the two key halves are merged through shared memory at the end.
-// Merging the chunks of a (head, sequence) pair, in chunk order either way: with up to 8 chunks the pair's CTAs
-// form a thread-block cluster, leave their partial rows in their own shared memory and each merges a share of the
-// rows out of its peers' shared memory; with more chunks the partial rows go to a scratch buffer and the CTA that
-// reports in last (an arrival counter that it resets) merges them.
-// Precision: q, K, V and the attention output are stored as two bfloat16 planes (hi = bf16(v), lo = bf16(v - hi),
-// about 16 mantissa bits together).  Products use the three significant cross terms (hi*hi + lo*hi + hi*lo); the
-// softmax weights are split the same way before the P V product.  A plane distance of 0 selects hi-only operands.
-#include "launch.h"
+// Operand format: q, the K cache (post-RoPE) and the V cache are float16, one plane (11 significant bits; the
+// values are O(1), far inside the float16 range); the softmax weights are rounded to float16 for the P V product;
+// scores, running maxima, sums and the output accumulate in float.  The result leaves as two bfloat16 planes
+// (hi = bf16(v), lo = bf16(v - hi)), the operand format of the GEMM that consumes it.
+//
+// One CTA per (head, sequence, KV chunk).  A sequence's KV rows are cut into 64-row tiles and the tiles are dealt
+// to the launch's chunks in equal contiguous runs, computed on the device from the real length (a captured graph
+// keeps balanced chunks as the sequence grows).  192 threads:
+//   warp 0 (one lane)  TMA producer: Q once, then K and V tiles through a ring of stages (K and V of a stage have
+//                      their own "full" barriers, so the scores of a tile start before its V has landed);
+//   warp 1 (one lane)  MMA issue: S_i = Q K_i^T (M = 128 query lanes, N = 64 keys) into one of two score buffers in
+//                      tensor memory, issued one tile ahead; O += P_i V_i (N = head_dim, V read as an MN-major operand
+//                      straight from its [key][dim] tile) into one accumulator that lives across the chunk;
+//   warps 2..5         softmax: thread = query row.  Reads its score row from tensor memory, applies the scale and
+//                      the mask (committed slots are visible to every row; tree slot j to row i iff bit j of the
+//                      row's ancestor bitmask, or j <= i for a causal chunk), keeps the row's running reference
+//                      maximum and sum in the exp2 domain, writes P_i as float16 into a swizzled shared-memory
+//                      tile for the MMA.  The reference maximum only moves when a tile's maximum exceeds it by
+//                      more than 8 (a factor 256, harmless in float16 and float); only then is the row's output
+//                      accumulator rescaled in tensor memory (load, scale, store), so the common tile needs no
+//                      round trip through registers for O.
+// Query rows beyond the row count of the call ride along as unused lanes of the M = 128 tile.
+// The chunks of a (head, sequence) pair (at most 8) form a thread-block cluster: every CTA leaves its partial rows
+// (un-normalised output, reference maximum, sum) in its own shared memory, and each CTA merges a share of the rows
+// out of its peers' shared memory, in chunk order (deterministic; no scratch traffic, no atomics).
+// Every barrier wait is bounded; when one runs out the CTA raises the time-out bit of the status word, skips its
+// stores, still takes part in the cluster barriers, frees its tensor memory and returns.
+#include "tc.cuh"
+#include <cuda_fp16.h>
 #include <math.h>
-#include <cstdlib>
 
 namespace hydra {
 
 namespace {
 
-constexpr int NWARP = 8;           // warp w: query rows 16 (w & 3) .. +15, key half w >> 2 of every tile
+using namespace tc;
 
-// First tile of chunk c when nt tiles are dealt to nch chunks in equal contiguous runs.
+constexpr int TILE = 64;           // KV rows per tile
+constexpr int NST = 3;             // ring stages (K and V of TILE rows each)
+constexpr int MAX_CHUNKS = 8;      // chunks of a (head, sequence) pair = cluster size
+constexpr float RESCALE_STEP = 8.f;
+
 __device__ __forceinline__ int chunk_first_tile(int c, int nt, int nch) { return (int)(((unsigned)c * (unsigned)nt) / (unsigned)nch); }
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// thread-block cluster helpers (the chunks of one (head, sequence) pair form a cluster along z)
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -69,260 +63,303 @@ __device__ __forceinline__ float2 ld_peer2(uint32_t addr) {
   asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
   return v;
 }
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
 
-// CLUSTER: the nchunks (<= 8) CTAs of a (head, sequence) pair are one thread-block cluster; they leave their partial
-// rows in their own shared memory and every CTA merges its share of the rows out of its peers' shared memory
-// (no scratch, no counters).  Otherwise: partial rows in scratch, merged by the CTA that reports in last.
-template <int HD, bool HL, int TILE, int NS, bool CLUSTER>
-__global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __restrict__ q, size_t q_ps, const bf16* __restrict__ kc,
-                                                                  const bf16* __restrict__ vc, size_t kv_ps, RowSet rs,
-                                                                  float* __restrict__ part_o, float* __restrict__ part_ml,
-                                                                  int* __restrict__ arrived, bf16* __restrict__ out, size_t out_ps,
-                                                                  int H, int max_seq, int nchunks) {
-  pdl_trigger();
-  pdl_wait();
-  constexpr int LDS = HD + 8;                         // padded row (bf16 elements): conflict-free ldmatrix
-  constexpr int KSTEPS = HD / 16;
-  constexpr int NB = HD / 8;                          // output n-blocks
-  constexpr int NP = HL ? 2 : 1;                      // planes
-  constexpr int TSZ = TILE * LDS;                     // elements of one staged tile
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  bf16* Qs = reinterpret_cast<bf16*>(smem_raw);       // [NP][64][LDS]
-  bf16* KVs = Qs + NP * 64 * LDS;                     // [NS stages][K planes, V planes][TILE][LDS]
-  __shared__ int s_last;
+struct AttArgs {
+  RowSet rs;
+  bf16* out; size_t out_ps;
+  int H, max_seq, nchunks;
+  int* status;
+  uint32_t wait_limit;
+};
 
+template <int HD, int QROWS> struct AttCfg {
+  static constexpr int NHALF = HD / 64;                       // 64-column (128-byte) halves of a head row
+  static constexpr int Q_BYTES = NHALF * QROWS * 128;
+  static constexpr int P_BYTES = QROWS * 128;                 // one P tile: [query row][64 keys] float16
+  static constexpr int KV_BYTES = NHALF * TILE * 128;         // K (or V) of one tile
+  static constexpr int STAGE_BYTES = 2 * KV_BYTES;
+  static constexpr int RING_BYTES = NST * STAGE_BYTES;
+  static constexpr int MERGE_BYTES = QROWS * HD * 4 + QROWS * 8;     // a chunk's partial rows + (max, sum); aliases the ring
+  static constexpr int NBAR = 1 + 3 * NST + 8;
+  // The M = 128 operand reads of a 64-row Q or P tile run 8 KB past the tile: Q's into P, P's into the ring
+  // (unused lanes, never read back), so the order Q, P0, P1, ring keeps them inside the allocation.
+  static constexpr int SMEM_BYTES = 1024 + Q_BYTES + 2 * P_BYTES + (RING_BYTES > MERGE_BYTES ? RING_BYTES : MERGE_BYTES) + NBAR * 8 + 16;
+  static constexpr int TMEM_COLS = 256;                       // S0 [0,64), S1 [64,128), O [128, 128+HD)
+  static_assert(RING_BYTES >= MERGE_BYTES, "merge area must fit in the ring");
+};
+
+template <int HD, int QROWS>
+__global__ void __launch_bounds__(192, 1)
+tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, const AttArgs a) {
+  using C = AttCfg<HD, QROWS>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t q_s = base, p_s = q_s + C::Q_BYTES, ring_s = p_s + 2 * C::P_BYTES;
+  const uint32_t bars = ring_s + (C::RING_BYTES > C::MERGE_BYTES ? C::RING_BYTES : C::MERGE_BYTES);
+  const uint32_t q_full = bars;
+  auto k_full = [&](int s) { return bars + 8u * (1 + s); };
+  auto v_full = [&](int s) { return bars + 8u * (1 + NST + s); };
+  auto kv_empty = [&](int s) { return bars + 8u * (1 + 2 * NST + s); };
+  auto s_full = [&](int i) { return bars + 8u * (1 + 3 * NST + i); };
+  auto s_empty = [&](int i) { return bars + 8u * (1 + 3 * NST + 2 + i); };
+  auto p_full = [&](int i) { return bars + 8u * (1 + 3 * NST + 4 + i); };
+  auto pv_done = [&](int i) { return bars + 8u * (1 + 3 * NST + 6 + i); };
+  const uint32_t tmem_slot = bars + 8u * C::NBAR;
+  __shared__ int s_abort;
+
+  const RowSet& rs = a.rs;
   const int h = blockIdx.x, b = blockIdx.y, c = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t = lane & 3;
-  const int nr = rs.n_rows ? rs.n_rows[b] : rs.tc;
+  const int nchunks = a.nchunks, H = a.H;
+
+  if (tid == 0) {
+    s_abort = 0;
+    mbar_init(q_full, 1);
+    for (int s = 0; s < NST; ++s) { mbar_init(k_full(s), 1); mbar_init(v_full(s), 1); mbar_init(kv_empty(s), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(s_empty(i), 4); mbar_init(p_full(i), 4); mbar_init(pv_done(i), 1); }
+    mbar_init_fence();
+    prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  pdl_trigger();
+  pdl_wait();                                           // q and the new cache rows are the preceding kernel's output
+  uint32_t tmem_base;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+  const int nr = min(rs.n_rows ? rs.n_rows[b] : rs.tc, QROWS);
   const int p0 = rs.pos0[b];
   const int total = p0 + nr;
   const int nt = (total + TILE - 1) / TILE;
-  const int s0 = chunk_first_tile(c, nt, nchunks) * TILE;
-  const int s1 = min(chunk_first_tile(c + 1, nt, nchunks) * TILE, total);
-  const int d = H * HD;
-  const bool has_work = s0 < s1 && nr > 0;            // a chunk that got no tile only reports in (see the end)
-  const size_t head_off = ((size_t)b * H + h) * max_seq * HD;
-  constexpr int PIECES = HD / 8;                       // 16-byte pieces per row
+  const int tile0 = chunk_first_tile(c, nt, nchunks), tile1 = chunk_first_tile(c + 1, nt, nchunks);
+  const bool has_work = tile0 < tile1 && nr > 0 && p0 >= 0 && total <= a.max_seq;
+  const int ntiles = has_work ? tile1 - tile0 : 0;
+  const uint32_t limit = a.wait_limit;
 
-  auto tile_ptr = [&](int buf, int kv, int plane) { return KVs + ((buf * 2 + kv) * NP + plane) * TSZ; };
-  auto load_tile = [&](int buf, int t0) {
-    for (int e = tid; e < TILE * PIECES; e += NWARP * 32) {
-      const int r = e / PIECES, pc = e % PIECES;
-      const int slot = t0 + r;
+  if (warp == 0) {
+    if (lane == 0 && has_work) {
+      const uint64_t pol = policy_evict_first(), pol_q = policy_evict_last();
+      mbar_arrive_expect_tx(q_full, C::Q_BYTES);
 #pragma unroll
-      for (int kv = 0; kv < 2; ++kv)
+      for (int hf = 0; hf < C::NHALF; ++hf) tma_load_2d(q_s + hf * QROWS * 128, &tmQ, h * HD + hf * 64, b * rs.tc, q_full, pol_q);
+      const int row0 = (b * H + h) * a.max_seq;
+      for (int i = 0; i < ntiles; ++i) {
+        const int s = i % NST;
+        // stage s was last read by the P V product of tile i - NST, the (i / NST - 1)-th completion of its empty barrier
+        if (i >= NST && !mbar_wait(kv_empty(s), (uint32_t)((i / NST - 1) & 1), limit)) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
+        const uint32_t k_dst = ring_s + s * C::STAGE_BYTES, v_dst = k_dst + C::KV_BYTES;
+        const int r = row0 + (tile0 + i) * TILE;
+        mbar_arrive_expect_tx(k_full(s), C::KV_BYTES);
 #pragma unroll
-        for (int pl = 0; pl < NP; ++pl) {
-          bf16* dst = tile_ptr(buf, kv, pl) + r * LDS + pc * 8;
-          if (slot < s1) cp_async16((uint32_t)__cvta_generic_to_shared(dst), (kv ? vc : kc) + pl * kv_ps + head_off + (size_t)slot * HD + pc * 8);
-          else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);     // rows past the end (their scores are masked)
-        }
-    }
-  };
-
-  const int ntiles = has_work ? (s1 - s0 + TILE - 1) / TILE : 0;
-  // request Q (rows past nr are zero) and the first NS-1 KV tiles: one cp.async group per tile, Q rides with the first
-  for (int e = tid; has_work && e < 64 * PIECES; e += NWARP * 32) {
-    const int r = e / PIECES, pc = e % PIECES;
+        for (int hf = 0; hf < C::NHALF; ++hf) tma_load_2d(k_dst + hf * TILE * 128, &tmK, hf * 64, r, k_full(s), pol);
+        mbar_arrive_expect_tx(v_full(s), C::KV_BYTES);
 #pragma unroll
-    for (int pl = 0; pl < NP; ++pl) {
-      bf16* dst = Qs + (pl * 64 + r) * LDS + pc * 8;
-      if (r < nr) cp_async16((uint32_t)__cvta_generic_to_shared(dst), q + pl * q_ps + (size_t)(b * rs.tc + r) * d + h * HD + pc * 8);
-      else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < NS - 1; ++i) {
-    if (i < ntiles) load_tile(i, s0 + i * TILE);
-    cp_async_commit();
-  }
-  const int row0 = (warp & 3) * 16, khalf = warp >> 2;
-  constexpr int HT = TILE / 2;                           // keys of a tile per warp
-  const bool warp_active = has_work && row0 < nr;
-  const int ra = row0 + g, rb = row0 + g + 8;            // the two query rows this thread owns
-  const uint64_t mask_a = ra < nr ? rs.mask[ra] : 0ull, mask_b = rb < nr ? rs.mask[rb] : 0ull;
-  float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
-  float o[NB][4];
-#pragma unroll
-  for (int n = 0; n < NB; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-  const float sc = rsqrtf((float)HD) * 1.4426950408889634f;   // 1/sqrt(hd) * log2(e)
-  const uint32_t q_addr = (uint32_t)__cvta_generic_to_shared(Qs + (row0 + (lane & 15)) * LDS + (lane >> 4) * 8);
-
-  for (int it = 0; it < ntiles; ++it) {
-    const int t0 = s0 + it * TILE;
-    const int buf = it % NS;
-    if (it + NS - 1 < ntiles) load_tile((it + NS - 1) % NS, t0 + (NS - 1) * TILE);      // the buffer read in iteration it - 1
-    cp_async_commit();
-    cp_async_wait<NS - 1>();                             // tile `it` (and Q, stored before the first barrier) has landed
-    __syncthreads();
-    if (warp_active) {
-      float s[HT / 8][4];
-#pragma unroll
-      for (int n = 0; n < HT / 8; ++n) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
-      const uint32_t k_off = (uint32_t)(((khalf * HT + (lane & 7) + (lane >> 4) * 8) * LDS + ((lane >> 3) & 1) * 8) * 2);
-      const uint32_t kh_addr = (uint32_t)__cvta_generic_to_shared(tile_ptr(buf, 0, 0)) + k_off;
-#pragma unroll
-      for (int kk = 0; kk < KSTEPS; ++kk) {
-        uint32_t qh[4], ql[4];
-        ldsm_x4(q_addr + kk * 32, qh[0], qh[1], qh[2], qh[3]);
-        if (HL) ldsm_x4(q_addr + 64 * LDS * 2 + kk * 32, ql[0], ql[1], ql[2], ql[3]);
-#pragma unroll
-        for (int np = 0; np < HT / 16; ++np) {         // 16 keys per ldmatrix.x4
-          uint32_t b0, b1, b2, b3;
-          const uint32_t addr = kh_addr + (uint32_t)((np * 16 * LDS + kk * 16) * 2);
-          ldsm_x4(addr, b0, b1, b2, b3);
-          mma_bf16(s[2 * np], qh[0], qh[1], qh[2], qh[3], b0, b1);
-          mma_bf16(s[2 * np + 1], qh[0], qh[1], qh[2], qh[3], b2, b3);
-          if (HL) {
-            mma_bf16(s[2 * np], ql[0], ql[1], ql[2], ql[3], b0, b1);
-            mma_bf16(s[2 * np + 1], ql[0], ql[1], ql[2], ql[3], b2, b3);
-            ldsm_x4(addr + TSZ * 2, b0, b1, b2, b3);   // K lo plane
-            mma_bf16(s[2 * np], qh[0], qh[1], qh[2], qh[3], b0, b1);
-            mma_bf16(s[2 * np + 1], qh[0], qh[1], qh[2], qh[3], b2, b3);
-          }
-        }
+        for (int hf = 0; hf < C::NHALF; ++hf) tma_load_2d(v_dst + hf * TILE * 128, &tmV, hf * 64, r, v_full(s), pol);
       }
-      // scale, mask, running max
-      const int k0 = t0 + khalf * HT;                    // first key of this warp's half
-      const bool need_mask = k0 + HT > p0 || k0 + HT > s1;
-      float mx_a = -INFINITY, mx_b = -INFINITY;
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && has_work) {
+      constexpr uint32_t idesc_s = instr_desc_f16(0, 128, TILE, 0);
+      constexpr uint32_t idesc_pv = instr_desc_f16(0, 128, HD, 1);
+      bool ok = mbar_wait(q_full, 0, limit);
+      auto issue_s = [&](int i) {                        // S_i = Q K_i^T into score buffer i & 1
+        const int s = i % NST;
+        if (!mbar_wait(k_full(s), (uint32_t)((i / NST) & 1), limit)) return false;
+        if (i >= 2 && !mbar_wait(s_empty(i & 1), (uint32_t)(((i >> 1) - 1) & 1), limit)) return false;
+        tc_fence_after();
+        const uint32_t k_src = ring_s + s * C::STAGE_BYTES;
 #pragma unroll
-      for (int n = 0; n < HT / 8; ++n) {
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint32_t qa = q_s + (kk >> 2) * QROWS * 128 + (kk & 3) * 32;
+          const uint32_t kb = k_src + (kk >> 2) * TILE * 128 + (kk & 3) * 32;
+          umma_f16(tmem_base + (uint32_t)((i & 1) * TILE), smem_desc_sw128(qa), smem_desc_sw128(kb), idesc_s, (uint32_t)(kk != 0));
+        }
+        umma_commit(s_full(i & 1));
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int i = 0; i < ntiles && ok; ++i) {
+        if (i + 1 < ntiles) ok = issue_s(i + 1);
+        if (!ok) break;
+        const int s = i % NST;
+        if (!mbar_wait(p_full(i & 1), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
+        if (!mbar_wait(v_full(s), (uint32_t)((i / NST) & 1), limit)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t v_src = ring_s + s * C::STAGE_BYTES + C::KV_BYTES;
+        const uint32_t p_src = p_s + (i & 1) * C::P_BYTES;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float v = s[n][e] * sc;
+        for (int kk = 0; kk < TILE / 16; ++kk)
+          umma_f16(tmem_base + 128u, smem_desc_sw128(p_src + kk * 32), smem_desc_sw128_mn(v_src + kk * 2048, TILE * 128), idesc_pv,
+                   (uint32_t)((i | kk) != 0));
+        umma_commit(kv_empty(s));
+        umma_commit(pv_done(i & 1));
+      }
+      if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
+    }
+  } else {
+    // ---- softmax warps: thread = query row (the tensor-memory lane it may read)
+    const int quad = warp & 3, row = quad * 32 + lane;
+    const bool warp_rows = quad * 32 < nr;                // any row of this warp in use
+    const bool row_live = row < nr;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const uint64_t mask = (row_live && rs.mask) ? rs.mask[row] : 0ull;
+    const bool causal = rs.mask == nullptr;
+    const float sc = rsqrtf((float)HD) * 1.4426950408889634f;   // 1/sqrt(hd) * log2(e)
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    const int st = tid - 64;                              // 0..127 among the softmax threads
+    for (int i = 0; i < ntiles && ok; ++i) {
+      const int t0 = (tile0 + i) * TILE;
+      if (!mbar_wait(s_full(i & 1), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
+      tc_fence_after();
+      uint32_t r[64];
+      if (warp_rows) tmem_ld64(lane_addr + (uint32_t)((i & 1) * TILE), r);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_empty(i & 1));
+      float alpha = 1.f;
+      if (warp_rows) {
+        const bool need_mask = t0 + TILE > p0;             // the tile reaches into the new rows (or past the end)
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          float v = __uint_as_float(r[j]) * sc;
           if (need_mask) {
-            int key = k0 + n * 8 + 2 * t + (e & 1);
-            uint64_t mk = (e < 2) ? mask_a : mask_b;
-            bool ok = key < s1 && (key < p0 || ((mk >> (key - p0)) & 1ull));
-            v = ok ? v : -INFINITY;
+            const int key = t0 + j, rel = key - p0;
+            const bool vis = row_live && key < total && (rel < 0 || (causal ? rel <= row : (bool)((mask >> rel) & 1ull)));
+            v = vis ? v : -INFINITY;
+          } else if (!row_live) {
+            v = -INFINITY;
           }
-          s[n][e] = v;
-          if (e < 2) mx_a = fmaxf(mx_a, v); else mx_b = fmaxf(mx_b, v);
+          r[j] = __float_as_uint(v);
+          mx = fmaxf(mx, v);
         }
-      }
-      mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1)); mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
-      mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1)); mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
-      const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
-      const float base_a = mn_a == -INFINITY ? 0.f : mn_a, base_b = mn_b == -INFINITY ? 0.f : mn_b;
-      const float al_a = exp2f(m_a - base_a), al_b = exp2f(m_b - base_b);     // exp2(-inf) = 0 for the first tile
-      m_a = mn_a; m_b = mn_b;
-      float sum_a = 0.f, sum_b = 0.f;
+        float m_new = m_ref;
+        if (mx > m_ref + RESCALE_STEP) m_new = mx;          // also the first finite maximum (m_ref = -inf)
+        const bool rescale = m_ref != -INFINITY && m_new != m_ref;
+        if (rescale) alpha = ex2(m_ref - m_new);
+        m_ref = m_new;
+        const float bse = m_new == -INFINITY ? 0.f : m_new;
+        float sum = 0.f;
+        uint32_t pk[32];
 #pragma unroll
-      for (int n = 0; n < HT / 8; ++n) {
-        s[n][0] = exp2f(s[n][0] - base_a); s[n][1] = exp2f(s[n][1] - base_a);
-        s[n][2] = exp2f(s[n][2] - base_b); s[n][3] = exp2f(s[n][3] - base_b);
-        sum_a += s[n][0] + s[n][1]; sum_b += s[n][2] + s[n][3];
-      }
-      l_a = l_a * al_a + sum_a; l_b = l_b * al_b + sum_b;      // per-thread partial sums; reduced over the quad at the end
-#pragma unroll
-      for (int n = 0; n < NB; ++n) { o[n][0] *= al_a; o[n][1] *= al_a; o[n][2] *= al_b; o[n][3] *= al_b; }
-      // O += P V
-      const uint32_t v_off = (uint32_t)(((khalf * HT + (lane & 7) + ((lane >> 3) & 1) * 8) * LDS + (lane >> 4) * 8) * 2);
-      const uint32_t vh_addr = (uint32_t)__cvta_generic_to_shared(tile_ptr(buf, 1, 0)) + v_off;
-#pragma unroll
-      for (int kp = 0; kp < HT / 16; ++kp) {           // 16 keys per k-step
-        uint32_t ah[4], al[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float x0 = s[2 * kp + (e >> 1)][(e & 1) * 2], x1 = s[2 * kp + (e >> 1)][(e & 1) * 2 + 1];
-          ah[e] = pack_bf16(x0, x1);
-          if (HL) {
-            const __nv_bfloat162 hv = *reinterpret_cast<const __nv_bfloat162*>(&ah[e]);
-            al[e] = pack_bf16(x0 - __low2float(hv), x1 - __high2float(hv));
-          }
+        for (int j = 0; j < 32; ++j) {
+          const float p0v = ex2(__uint_as_float(r[2 * j]) - bse), p1v = ex2(__uint_as_float(r[2 * j + 1]) - bse);
+          pk[j] = pack_half2(p0v, p1v);
+          const __half2 hv = *reinterpret_cast<const __half2*>(&pk[j]);
+          sum += __low2float(hv) + __high2float(hv);       // the sum of what the MMA will really weigh V with
         }
+        l = l * alpha + sum;
+        // P buffer i & 1 was last read by P V of tile i - 2; the row's accumulator by P V of tile i - 1
+        if (i >= 2 && !mbar_wait(pv_done(i & 1), (uint32_t)(((i >> 1) - 1) & 1), limit)) { ok = false; break; }
+        if (__any_sync(0xffffffffu, rescale)) {
+          if (i >= 1 && !mbar_wait(pv_done((i - 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), limit)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int np = 0; np < NB / 2; ++np) {          // 16 output columns per ldmatrix.x4.trans
-          uint32_t b0, b1, b2, b3;
-          const uint32_t addr = vh_addr + (uint32_t)((kp * 16 * LDS + np * 16) * 2);
-          ldsm_x4_trans(addr, b0, b1, b2, b3);
-          mma_bf16(o[2 * np], ah[0], ah[1], ah[2], ah[3], b0, b1);
-          mma_bf16(o[2 * np + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-          if (HL) {
-            mma_bf16(o[2 * np], al[0], al[1], al[2], al[3], b0, b1);
-            mma_bf16(o[2 * np + 1], al[0], al[1], al[2], al[3], b2, b3);
-            ldsm_x4_trans(addr + TSZ * 2, b0, b1, b2, b3);   // V lo plane
-            mma_bf16(o[2 * np], ah[0], ah[1], ah[2], ah[3], b0, b1);
-            mma_bf16(o[2 * np + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+          for (int c0 = 0; c0 < HD; c0 += 32) {
+            uint32_t o[32];
+            tmem_ld32(lane_addr + 128u + (uint32_t)c0, o);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+            tmem_st32(lane_addr + 128u + (uint32_t)c0, o);
           }
         }
+        const uint32_t prow = p_s + (i & 1) * C::P_BYTES + (uint32_t)row * 128u;
+        if (row < QROWS) {
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch) {
+            const uint32_t dst = prow + (uint32_t)((ch ^ (row & 7)) * 16);
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]), "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3]) : "memory");
+          }
+        }
+      } else {
+        if (i >= 2 && !mbar_wait(pv_done(i & 1), (uint32_t)(((i >> 1) - 1) & 1), limit)) { ok = false; break; }
       }
+      if (t0 + TILE > total) {
+        // rows of the V tile past the end of the sequence hold whatever the cache holds: zero them, so that a
+        // zero weight times a non-finite stale value cannot reach the accumulator
+        const int s = i % NST;
+        if (!mbar_wait(v_full(s), (uint32_t)((i / NST) & 1), limit)) { ok = false; break; }
+        const uint32_t v_src = ring_s + s * C::STAGE_BYTES + C::KV_BYTES;
+        const int first = total - t0;                       // first row to clear (>= 1)
+        for (int e = st; e < (TILE - first) * C::NHALF * 8; e += 128) {
+          const int rr = first + e / (C::NHALF * 8), rem = e % (C::NHALF * 8);
+          const uint32_t dst = v_src + (uint32_t)((rem >> 3) * TILE * 128 + rr * 128 + (rem & 7) * 16);
+          asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(dst), "r"(0u) : "memory");
+        }
+      }
+      fence_proxy_async();                                 // P (and the cleared V rows) become visible to the tensor core
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full(i & 1));
     }
-    __syncthreads();
-  }
-  l_a += __shfl_xor_sync(0xffffffffu, l_a, 1); l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
-  l_b += __shfl_xor_sync(0xffffffffu, l_b, 1); l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
-  // merge the two key halves: the upper warps hand (m, l, o) to their partner through the (now idle) tile ring
-  float* xch = reinterpret_cast<float*>(KVs) + ((warp & 3) * 32 + lane) * (NB * 4 + 4);
-  if (khalf == 1 && warp_active) {
+    if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
+    // ---- this chunk's partial rows -> shared memory (the ring is idle once the last P V has completed)
+    if (ok && ntiles > 0 && !mbar_wait(pv_done((ntiles - 1) & 1), (uint32_t)(((ntiles - 1) >> 1) & 1), limit)) {
+      ok = false; atomicOr(a.status, ST_TIMEOUT); s_abort = 1;
+    }
+    tc_fence_after();
+    if (row < QROWS) {
+      const uint32_t xo = ring_s + (uint32_t)row * (HD * 4), xml = ring_s + QROWS * HD * 4 + (uint32_t)row * 8;
+      const bool have = ok && ntiles > 0 && row_live && m_ref != -INFINITY;
+      if (ok && ntiles > 0 && warp_rows) {
 #pragma unroll
-    for (int n = 0; n < NB; ++n) *reinterpret_cast<float4*>(xch + n * 4) = make_float4(o[n][0], o[n][1], o[n][2], o[n][3]);
-    *reinterpret_cast<float4*>(xch + NB * 4) = make_float4(m_a, m_b, l_a, l_b);
+        for (int c0 = 0; c0 < HD; c0 += 32) {
+          uint32_t o[32];
+          tmem_ld32(lane_addr + 128u + (uint32_t)c0, o);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {                    // float4 piece k4 of row i sits at position k4 ^ (i & (HD/4 - 1))
+            const int k4 = c0 / 4 + j;
+            const uint32_t dst = xo + (uint32_t)((k4 ^ (row & (HD / 4 - 1))) * 16);
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(o[4 * j]), "r"(o[4 * j + 1]), "r"(o[4 * j + 2]), "r"(o[4 * j + 3]) : "memory");
+          }
+        }
+      }
+      const float2 ml = have ? make_float2(m_ref, l) : make_float2(-INFINITY, 0.f);
+      asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(xml), "f"(ml.x), "f"(ml.y) : "memory");
+    }
   }
+  tc_fence_before();
   __syncthreads();
-  constexpr int XCH_FLOATS = 4 * 32 * (NB * 4 + 4);     // the hand-over area above
-  float* xo = reinterpret_cast<float*>(KVs) + XCH_FLOATS;    // CLUSTER: this chunk's partial rows [64][HD], then (m, l) [64][2]
-  float* xml = xo + 64 * HD;
-  if (CLUSTER && !warp_active && khalf == 0) {           // rows this CTA has nothing for: weight zero
-    if (t == 0) { *reinterpret_cast<float2*>(xml + ra * 2) = make_float2(-INFINITY, 0.f); *reinterpret_cast<float2*>(xml + rb * 2) = make_float2(-INFINITY, 0.f); }
-  }
-  if (khalf == 0 && warp_active) {
-    const float4 ml = *reinterpret_cast<const float4*>(xch + NB * 4);
-    const float mn_a = fmaxf(m_a, ml.x), mn_b = fmaxf(m_b, ml.y);
-    const float base_a = mn_a == -INFINITY ? 0.f : mn_a, base_b = mn_b == -INFINITY ? 0.f : mn_b;
-    const float w0a = exp2f(m_a - base_a), w1a = exp2f(ml.x - base_a), w0b = exp2f(m_b - base_b), w1b = exp2f(ml.y - base_b);
-    m_a = mn_a; m_b = mn_b;
-    l_a = l_a * w0a + ml.z * w1a; l_b = l_b * w0b + ml.w * w1b;
-    // partials: o (un-normalised), m (log2 domain), l
-    if (CLUSTER) {
-#pragma unroll
-      for (int n = 0; n < NB; ++n) {
-        const float4 v = *reinterpret_cast<const float4*>(xch + n * 4);
-        *reinterpret_cast<float2*>(xo + ra * HD + n * 8 + 2 * t) = make_float2(o[n][0] * w0a + v.x * w1a, o[n][1] * w0a + v.y * w1a);
-        *reinterpret_cast<float2*>(xo + rb * HD + n * 8 + 2 * t) = make_float2(o[n][2] * w0b + v.z * w1b, o[n][3] * w0b + v.w * w1b);
-      }
-      if (t == 0) {
-        *reinterpret_cast<float2*>(xml + ra * 2) = ra < nr ? make_float2(m_a, l_a) : make_float2(-INFINITY, 0.f);
-        *reinterpret_cast<float2*>(xml + rb * 2) = rb < nr ? make_float2(m_b, l_b) : make_float2(-INFINITY, 0.f);
-      }
-    } else {
-      const size_t idx_a = ((size_t)(b * rs.tc + ra) * H + h) * nchunks + c, idx_b = ((size_t)(b * rs.tc + rb) * H + h) * nchunks + c;
-#pragma unroll
-      for (int n = 0; n < NB; ++n) {
-        const float4 v = *reinterpret_cast<const float4*>(xch + n * 4);
-        if (ra < nr) __stcg(reinterpret_cast<float2*>(part_o + idx_a * HD + n * 8 + 2 * t), make_float2(o[n][0] * w0a + v.x * w1a, o[n][1] * w0a + v.y * w1a));
-        if (rb < nr) __stcg(reinterpret_cast<float2*>(part_o + idx_b * HD + n * 8 + 2 * t), make_float2(o[n][2] * w0b + v.z * w1b, o[n][3] * w0b + v.w * w1b));
-      }
-      if (t == 0 && ra < nr) __stcg(reinterpret_cast<float2*>(part_ml + idx_a * 2), make_float2(m_a, l_a));
-      if (t == 0 && rb < nr) __stcg(reinterpret_cast<float2*>(part_ml + idx_b * 2), make_float2(m_b, l_b));
-    }
-  }
-  if (CLUSTER) {
-    // out[r][h][:] = sum_c o_c 2^(m_c - M) / sum_c l_c 2^(m_c - M), chunks in order; this CTA takes rows c, c + nchunks, ...
-    cluster_sync_all();                                  // every chunk's rows are in its shared memory
+  // ---- merge the chunks of this (head, sequence): out[r][h][:] = sum_c o_c 2^(m_c - M) / sum_c l_c 2^(m_c - M),
+  // chunks in order; this CTA takes rows c, c + nchunks, ...
+  cluster_sync_all();                                     // every chunk's rows are in its shared memory
+  {
     constexpr int V4 = HD / 4;
-    const uint32_t xo_s = (uint32_t)__cvta_generic_to_shared(xo), xml_s = (uint32_t)__cvta_generic_to_shared(xml);
-    const int my_rows = (rs.tc - c + nchunks - 1) / nchunks;
-    for (int e = tid; e < my_rows * V4; e += NWARP * 32) {
+    const uint32_t xo_s = ring_s, xml_s = ring_s + QROWS * HD * 4;
+    const int d = H * HD;
+    const int rows_cap = min(rs.tc, QROWS);
+    const int my_rows = rows_cap > c ? (rows_cap - c + nchunks - 1) / nchunks : 0;
+    for (int e = tid; e < my_rows * V4; e += 192) {
       const int i = c + (e / V4) * nchunks, k4 = e % V4;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
       if (i < nr) {
-        float mc[8], lc[8];
+        float mc[MAX_CHUNKS], lc[MAX_CHUNKS];
         float M = -INFINITY;
 #pragma unroll
-        for (int cc = 0; cc < 8; ++cc) {
+        for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
           mc[cc] = -INFINITY; lc[cc] = 0.f;
           if (cc < nchunks) { const float2 ml = ld_peer2(peer_smem(xml_s + (uint32_t)i * 8u, (uint32_t)cc)); mc[cc] = ml.x; lc[cc] = ml.y; }
           M = fmaxf(M, mc[cc]);
         }
         float L = 0.f;
 #pragma unroll
-        for (int cc = 0; cc < 8; ++cc) {
+        for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
           if (cc < nchunks && mc[cc] != -INFINITY) {
             const float w = exp2f(mc[cc] - M);
-            const float4 v = ld_peer4(peer_smem(xo_s + (uint32_t)(i * HD + k4 * 4) * 4u, (uint32_t)cc));
+            const float4 v = ld_peer4(peer_smem(xo_s + (uint32_t)(i * HD * 4 + ((k4 ^ (i & (V4 - 1))) * 16)), (uint32_t)cc));
             L += lc[cc] * w;
             acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
           }
@@ -330,183 +367,86 @@ __global__ void __launch_bounds__(NWARP * 32) tree_attn_tc_kernel(const bf16* __
         const float inv = L > 0.f ? 1.f / L : 0.f;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
       }
-      bf16* dst = out + ((size_t)b * rs.tc + i) * d + h * HD + k4 * 4;      // rows past nr get zeros
-      const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x, acc.y), h1 = __floats2bfloat162_rn(acc.z, acc.w);
-      *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
-      if (out_ps) {
-        const __nv_bfloat162 l0 = __floats2bfloat162_rn(acc.x - __low2float(h0), acc.y - __high2float(h0));
-        const __nv_bfloat162 l1 = __floats2bfloat162_rn(acc.z - __low2float(h1), acc.w - __high2float(h1));
-        *reinterpret_cast<uint2*>(dst + out_ps) = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
-      }
-    }
-    cluster_sync_all();                                  // peers may still be reading this CTA's rows
-    return;
-  }
-  // The last of the (head, sequence)'s chunks to report in merges them:
-  // out[r][h][:] = sum_c o_c 2^(m_c - M) / sum_c l_c 2^(m_c - M) over the chunks that were dealt tiles, in chunk order.
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int prev = atomicAdd(arrived + b * H + h, 1);
-    s_last = prev == nchunks - 1;
-    if (s_last) arrived[b * H + h] = 0;                  // ready for the next launch
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  // Every thread owns up to PER float4 pieces of the output rows.  The partial rows of the first four chunks are
-  // requested before anything else, so that they travel while the chunk weights are worked out (one (row, chunk)
-  // pair per thread, through shared memory); further chunks follow four at a time.
-  constexpr int V4 = HD / 4, PER = (64 * V4 + NWARP * 32 - 1) / (NWARP * 32), CB = 4;
-  float4 v[CB][PER];
-  auto dealt = [&](int cc) { return chunk_first_tile(cc, nt, nchunks) != chunk_first_tile(cc + 1, nt, nchunks); };   // else it wrote nothing
-  auto load_batch = [&](int c0) {
-#pragma unroll
-    for (int cb = 0; cb < CB; ++cb) {
-      const int cc = c0 + cb;
-      const bool live = cc < nchunks && dealt(cc);
-#pragma unroll
-      for (int j = 0; j < PER; ++j) {
-        const int e = tid + j * NWARP * 32, i = e / V4, k4 = e % V4;
-        v[cb][j] = live && i < nr ? __ldcg(reinterpret_cast<const float4*>(part_o + ((((size_t)b * rs.tc + i) * H + h) * nchunks + cc) * HD + k4 * 4))
-                                  : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-    }
-  };
-  load_batch(0);
-  float* sm_m = reinterpret_cast<float*>(KVs);         // [tc][nchunks] chunk maxima, then the normalised chunk weights
-  float* sm_l = sm_m + rs.tc * nchunks;
-  for (int e = tid; e < rs.tc * nchunks; e += NWARP * 32) {
-    const int i = e / nchunks, cc = e % nchunks;
-    float2 ml = make_float2(-INFINITY, 0.f);
-    if (i < nr && dealt(cc)) ml = __ldcg(reinterpret_cast<const float2*>(part_ml + (((size_t)b * rs.tc + i) * H + h) * nchunks * 2 + cc * 2));
-    sm_m[e] = ml.x; sm_l[e] = ml.y;
-  }
-  __syncthreads();
-  for (int i = tid; i < rs.tc; i += NWARP * 32) {
-    float M = -INFINITY, L = 0.f;
-    for (int cc = 0; cc < nchunks; ++cc) M = fmaxf(M, sm_m[i * nchunks + cc]);
-    for (int cc = 0; cc < nchunks; ++cc) {
-      const float mc = sm_m[i * nchunks + cc];
-      const float w = mc == -INFINITY ? 0.f : exp2f(mc - M);
-      L += sm_l[i * nchunks + cc] * w;
-      sm_m[i * nchunks + cc] = w;
-    }
-    const float inv = L > 0.f ? 1.f / L : 0.f;
-    for (int cc = 0; cc < nchunks; ++cc) sm_m[i * nchunks + cc] *= inv;
-  }
-  __syncthreads();
-  float4 acc[PER];
-#pragma unroll
-  for (int j = 0; j < PER; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int c0 = 0; c0 < nchunks; c0 += CB) {
-    if (c0 > 0) load_batch(c0);
-#pragma unroll
-    for (int cb = 0; cb < CB; ++cb) {
-      const int cc = c0 + cb;
-#pragma unroll
-      for (int j = 0; j < PER; ++j) {
-        const int i = (tid + j * NWARP * 32) / V4;
-        const float w = cc < nchunks && i < rs.tc ? sm_m[i * nchunks + cc] : 0.f;
-        acc[j].x += v[cb][j].x * w; acc[j].y += v[cb][j].y * w; acc[j].z += v[cb][j].z * w; acc[j].w += v[cb][j].w * w;
+      if (!s_abort) {
+        bf16* dst = a.out + ((size_t)b * rs.tc + i) * d + h * HD + k4 * 4;      // rows past nr get zeros
+        const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x, acc.y), h1 = __floats2bfloat162_rn(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+        if (a.out_ps) {
+          const __nv_bfloat162 l0 = __floats2bfloat162_rn(acc.x - __low2float(h0), acc.y - __high2float(h0));
+          const __nv_bfloat162 l1 = __floats2bfloat162_rn(acc.z - __low2float(h1), acc.w - __high2float(h1));
+          *reinterpret_cast<uint2*>(dst + a.out_ps) = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+        }
       }
     }
   }
-#pragma unroll
-  for (int j = 0; j < PER; ++j) {
-    const int e = tid + j * NWARP * 32, i = e / V4, k4 = e % V4;
-    if (i >= rs.tc) continue;
-    bf16* dst = out + ((size_t)b * rs.tc + i) * d + h * HD + k4 * 4;      // rows past nr get zeros
-    const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[j].x, acc[j].y), h1 = __floats2bfloat162_rn(acc[j].z, acc[j].w);
-    *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
-    if (out_ps) {
-      const __nv_bfloat162 l0 = __floats2bfloat162_rn(acc[j].x - __low2float(h0), acc[j].y - __high2float(h0));
-      const __nv_bfloat162 l1 = __floats2bfloat162_rn(acc[j].z - __low2float(h1), acc[j].w - __high2float(h1));
-      *reinterpret_cast<uint2*>(dst + out_ps) = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
-    }
+  cluster_sync_all();                                     // peers may still be reading this CTA's rows
+  if (s_abort) {                                          // let copies in flight land before the CTA retires
+    for (int i = 0; i < 2000; ++i) __nanosleep(100);
   }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, C::TMEM_COLS); }
 }
 
-// Number of KV chunks per (head, sequence) for lengths up to len_upper.  Few (head, sequence) pairs: one CTA per SM
-// at most and chunks as long as that allows (the kernel is bound by the MMA rate of an SM, so what counts is the
-// largest number of tiles any SM walks, plus about four tiles' worth of set-up and merging per CTA: measured on the
-// 13B shape at 2048 rows, 3 chunks in one wave beat 7 chunks in two); many pairs: chunks of about 128 rows at most.
-int pick_chunks(int pairs, int len_upper, int tile, int nchunks_max, int sms, bool* cluster) {
-  const int nt = (len_upper + tile - 1) / tile;
-  int hi = (len_upper + ATT_CHUNK_ROWS - 1) / ATT_CHUNK_ROWS;
-  hi = hi < 1 ? 1 : (hi > nchunks_max ? nchunks_max : hi);
+// Number of KV chunks per (head, sequence) for lengths up to len_upper: the count (at most 8) that minimises the
+// largest number of tiles any SM walks, with about three tiles' worth of set-up and merging per CTA; ties go to
+// fewer chunks.  Two CTAs share an SM (shared memory and tensor memory allow it).
+int pick_chunks(int pairs, int len_upper, int sms) {
+  const int nt = (len_upper + TILE - 1) / TILE;
+  int hi = nt < MAX_CHUNKS ? nt : MAX_CHUNKS;
+  if (hi < 1) hi = 1;
   auto cost = [&](int n) {
     const long per_sm = ((long)pairs * n + sms - 1) / sms, tiles = (nt + n - 1) / n;
-    return per_sm * (tiles + 4) + 1;
+    return per_sm * (tiles + 3);
   };
-  int best = hi; long best_cost = -1;
-  for (int n = 1; n <= hi; ++n)
-    if (best_cost < 0 || cost(n) < best_cost) { best = n; best_cost = cost(n); }     // ties: fewer chunks
-  *cluster = best <= 8;        // up to 8 chunks: the pair's CTAs form a cluster and merge through shared memory
+  int best = 1; long best_cost = cost(1);
+  for (int n = 2; n <= hi; ++n)
+    if (cost(n) < best_cost) { best = n; best_cost = cost(n); }
   return best;
 }
 
-template <int HD, bool HL, int NS>
-hydra_status run_ns(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
-                 float* scratch, int H, int max_seq, int len_upper, cudaStream_t st) {
-  constexpr int TILE = 32;                    // 32-row tiles, four of them in flight: hides the HBM latency of a chunk's walk
-  const int nchunks_max = (max_seq + ATT_CHUNK_ROWS - 1) / ATT_CHUNK_ROWS;     // what the scratch is sized for
-  const int sms = sm_count();
-  if ((size_t)H * rs.batch * sizeof(int) > ATT_SCRATCH_HEADER) return HYDRA_ERR_UNSUPPORTED;
-  bool cluster = false;
-  const int nchunks = pick_chunks(H * rs.batch, len_upper, TILE, nchunks_max, sms, &cluster);
-  const size_t rows = (size_t)rs.batch * rs.tc;
-  int* arrived = reinterpret_cast<int*>(scratch);     // one counter per (sequence, head): zero between launches
-  float* part_o = scratch + ATT_SCRATCH_HEADER / sizeof(float);
-  float* part_ml = part_o + rows * H * nchunks_max * HD;
-  constexpr int LDS = HD + 8;
-  constexpr int NP = HL ? 2 : 1;
-  const size_t ring = (size_t)NP * 2 * NS * TILE * LDS * sizeof(bf16);
-  const size_t xchg = (size_t)(4 * 32 * (HD / 2 + 4) + 64 * HD + 128) * sizeof(float);      // hand-over area + a chunk's partial rows + (m, l)
-  const size_t smem = (size_t)NP * 64 * LDS * sizeof(bf16) + (ring > xchg ? ring : xchg);
+template <int HD, int QROWS>
+hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out, size_t out_ps,
+                 int H, int max_seq, int len_upper, int* status, cudaStream_t st) {
+  using C = AttCfg<HD, QROWS>;
+  CUtensorMap tq, tk, tv;
+  const uint64_t cache_rows = (uint64_t)cache_batch * H * max_seq;
+  if (!get_tensor_map(q, (uint64_t)q_rows, (uint64_t)H * HD, QROWS, true, &tq) ||
+      !get_tensor_map(kc, cache_rows, HD, TILE, true, &tk) || !get_tensor_map(vc, cache_rows, HD, TILE, true, &tv)) {
+    set_last_error("cuTensorMapEncodeTiled", cudaErrorUnknown);
+    return HYDRA_ERR_CUDA;
+  }
   static PerDeviceFlag attr_done;
   if (!attr_done.get()) {
-    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE, NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, HL, TILE, NS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, QROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_done.set();
   }
-  if (!cluster) {
-    launch_pdl(tree_attn_tc_kernel<HD, HL, TILE, NS, false>, dim3(H, rs.batch, nchunks), dim3(NWARP * 32), smem, st, q, q_ps, kc, vc, kv_ps, rs, part_o,
-               part_ml, arrived, out, out_ps, H, max_seq, nchunks);
-    HYDRA_LAUNCH_CHECK();
-    return HYDRA_OK;
-  }
+  AttArgs a{};
+  a.rs = rs; a.out = out; a.out_ps = out_ps; a.H = H; a.max_seq = max_seq; a.status = status; a.wait_limit = WAIT_LIMIT;
+  a.nchunks = pick_chunks(H * rs.batch, len_upper, sm_count());
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(H, rs.batch, nchunks); cfg.blockDim = dim3(NWARP * 32); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cfg.gridDim = dim3(H, rs.batch, a.nchunks); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = C::SMEM_BYTES; cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = (unsigned)nchunks;
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = (unsigned)a.nchunks;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
-  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<HD, HL, TILE, NS, true>, q, q_ps, kc, vc, kv_ps, rs, part_o, part_ml, arrived, out, out_ps, H,
-                                max_seq, nchunks));
+  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<HD, QROWS>, tq, tk, tv, a));
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
-template <int HD, bool HL>
-hydra_status run(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out, size_t out_ps,
-                 float* scratch, int H, int max_seq, int len_upper, cudaStream_t st) {
-  return run_ns<HD, HL, 5>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, scratch, H, max_seq, len_upper, st);
-}
-
 }  // namespace
 
-hydra_status tree_attention_tc(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out,
-                               size_t out_ps, void* scratch, int H, int hd, int max_seq, int len_upper, cudaStream_t st) {
-  if (rs.tc > 64) return HYDRA_ERR_UNSUPPORTED;
-  if ((q_ps == 0) != (kv_ps == 0)) return HYDRA_ERR_UNSUPPORTED;           // q and the caches split the same way
-  const bool hl = q_ps != 0;
-  if (hd == 128 && hl) return run<128, true>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, st);
-  if (hd == 128) return run<128, false>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, st);
-  if (hd == 64 && hl) return run<64, true>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, st);
-  if (hd == 64) return run<64, false>(q, q_ps, kc, vc, kv_ps, rs, out, out_ps, (float*)scratch, H, max_seq, len_upper, st);
+hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out,
+                               size_t out_ps, int H, int hd, int max_seq, int len_upper, int* status, cudaStream_t st) {
+  if (rs.tc > 128 || (rs.mask && rs.tc > 64)) return HYDRA_ERR_UNSUPPORTED;
+  if (!tensor_map_encoder_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
+  if (((uintptr_t)q | (uintptr_t)kc | (uintptr_t)vc) & 15) return HYDRA_ERR_INVALID;
+  const bool wide = rs.tc > 64;
+  if (hd == 128) return wide ? run<128, 128>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st)
+                             : run<128, 64>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st);
+  if (hd == 64) return wide ? run<64, 128>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st)
+                            : run<64, 64>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st);
   return HYDRA_ERR_UNSUPPORTED;
 }
 

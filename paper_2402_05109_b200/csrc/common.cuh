@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 #include <atomic>
 #include "../../include/hydra.h"
@@ -138,7 +139,7 @@ struct RowSet {
   const int* n_rows;      // device [batch] or null
   const int* pos0;        // device [batch]
   const int* depth;       // device [tc]
-  const uint64_t* mask;   // device [tc]
+  const uint64_t* mask;   // device [tc]; null: a causal chunk (row i sees new slots 0..i), bfloat16 model path only
 };
 
 }  // namespace hydra

@@ -52,8 +52,9 @@ struct hydra_ctx {
   std::vector<LayerW> layers; LayerW pfx;
   std::vector<const void*> head_w1, head_b1, head_wr, head_br;
   const void *embed, *lm_head, *final_norm;
-  int esize;                                     // bytes per weight / KV element
-  int planes;                                    // planes of every operand / cache buffer: 2 (hi, lo) for bfloat16, 1 for float
+  int esize;                                     // bytes per weight element
+  int planes;                                    // planes of every GEMM operand buffer: 2 (hi, lo) for bfloat16, 1 for float
+  int kv_esize;                                  // bytes per element of q and the KV caches: 4 (float) or 2 (float16)
   int R;                                         // row capacity of a forward call (padded)
   int RH;                                        // row capacity of the head buffers (padded)
   int maxP;
@@ -154,7 +155,8 @@ hydra_status supported_cfg(const hydra_model_cfg* m) {
 size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, const TreeHost& t, char* ws) {
   Bump b{ws, 0};
   const int es = m.dtype == 0 ? 4 : 2;
-  const int np = m.dtype == 0 ? 1 : 2;          // bfloat16 operands and caches are stored as hi + lo planes
+  const int np = m.dtype == 0 ? 1 : 2;          // bfloat16 GEMM operands are stored as hi + lo planes
+  const int ces = m.dtype == 0 ? 4 : 2;         // q and the KV caches: float, or one float16 plane
   const int d = m.d_model, f = m.d_ffn, V = m.vocab, K = h.n_heads, T = t.T;
   const int R = pad_rows(m.max_batch * CHUNK);
   const int RH = pad_rows(m.max_batch * t.maxP);
@@ -188,9 +190,9 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
   auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
   auto* done = b.take<unsigned int>(m.max_batch);
-  auto* kvb = b.take<char>((size_t)m.n_layers * 2 * np * kv_layer_elems(m) * es);
-  auto* kvp = b.take<char>(h.prefix_attn ? (size_t)2 * np * kv_layer_elems(m) * es : 0);
-  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)np * R * d * es);
+  auto* kvb = b.take<char>((size_t)m.n_layers * 2 * kv_layer_elems(m) * ces);
+  auto* kvp = b.take<char>(h.prefix_attn ? (size_t)2 * kv_layer_elems(m) * ces : 0);
+  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)(R + 128) * d * ces);
   auto* part = b.take<float>(part_floats);
   auto* h_tree = b.take<float>((size_t)R * d);
   auto* logits = b.take<float>((size_t)pad_rows(m.max_batch * T) * V);
@@ -203,9 +205,9 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* z = b.take<char>((size_t)np * RH * (K + 1) * d * es); auto* yb = b.take<char>((size_t)np * RH * d * es);
   const int topk_cap = std::max(R, RH);
   auto* topk_s = b.take<char>(topk_scratch_bytes(topk_cap, V));
-  auto* att = b.take<char>(attention_scratch_bytes(m.max_batch, CHUNK, m.n_heads, m.head_dim, m.max_seq));
+  auto* att = b.take<char>(m.dtype == 0 ? attention_scratch_bytes(m.max_batch, CHUNK, m.n_heads, m.head_dim, m.max_seq) : 0);
   if (c) {
-    c->R = R; c->RH = RH; c->part_floats = part_floats; c->esize = es; c->planes = np;
+    c->R = R; c->RH = RH; c->part_floats = part_floats; c->esize = es; c->planes = np; c->kv_esize = ces;
     c->d_parent = parent; c->d_depth = depth; c->d_first_child = fc; c->d_n_child = nc; c->d_path_tab = path_tab;
     c->d_chain_depth = chain_depth; c->d_anc = anc; c->d_chain_mask = chain_mask; c->d_level_parents = lvl;
     c->d_len = len; c->d_n_new = n_new; c->d_root_tok = root; c->d_status = status; c->d_pos0 = pos0; c->d_nrows = nrows;
@@ -245,16 +247,18 @@ hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void*
 
 // element distance between the hi and lo planes of an operand buffer of `rows_alloc` rows of `cols` (0 for float)
 size_t ps(const hydra_ctx* c, int rows_alloc, size_t cols) { return c->planes == 2 ? (size_t)rows_alloc * cols : 0; }
-size_t kv_ps(const hydra_ctx* c) { return c->planes == 2 ? kv_layer_elems(c->m) : 0; }
 
 // RoPE + KV append + tree attention of one layer from the QKV partial sums (*sd) in c->part; result in c->attn_out.
 hydra_status attention_block(hydra_ctx* c, char* kc, char* vc, const RowSet& rs, int len_upper, const SplitDesc& sd, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int d = m.d_model, dt = m.dtype;
-  HYDRA_TRY(qkv_rope_store(c->part, sd, c->rope, c->q, ps(c, c->R, d), kc, vc, kv_ps(c), rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
+  HYDRA_TRY(qkv_rope_store(c->part, sd, c->rope, c->q, kc, vc, rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
   TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
-  return tree_attention(c->q, ps(c, c->R, d), kc, vc, kv_ps(c), rs, c->attn_out, ps(c, c->R, d), c->att_scratch, m.n_heads, m.head_dim,
-                        m.max_seq, len_upper, dt, st);
+  if (dt == 0)
+    return tree_attention_f32((const float*)c->q, (const float*)kc, (const float*)vc, rs, (float*)c->attn_out, c->att_scratch, m.n_heads,
+                              m.head_dim, m.max_seq, len_upper, st);
+  return tree_attention_tc((const __half*)c->q, c->R, (const __half*)kc, (const __half*)vc, m.max_batch, rs, (bf16*)c->attn_out,
+                           ps(c, c->R, d), m.n_heads, m.head_dim, m.max_seq, len_upper, c->d_status, st);
 }
 
 double gemm_bytes(const hydra_ctx* c, int m, int n, int k) {        // weights + activation slab read once, output written once
@@ -285,7 +289,7 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
                       cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int rows = rs.batch * rs.tc, d = m.d_model;
-  const size_t kvl = kv_layer_elems(m) * c->esize * c->planes;      // bytes of one layer's K (or V) cache, all planes
+  const size_t kvl = kv_layer_elems(m) * c->kv_esize;      // bytes of one layer's K (or V) cache
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
   HYDRA_TRY(embed_rows(c->embed, tok, c->x, rows, d, m.vocab, m.dtype, c->d_status, st));
   HYDRA_TRY(residual_rmsnorm(c->x, nullptr, single_slot(0), c->x, c->layers[0].attn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, m.dtype, st));
@@ -304,7 +308,7 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
 hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int len_upper, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int rows = rs.batch * rs.tc, d = m.d_model;
-  const size_t kvl = kv_layer_elems(m) * c->esize * c->planes;      // bytes of one layer's K (or V) cache, all planes
+  const size_t kvl = kv_layer_elems(m) * c->kv_esize;      // bytes of one layer's K (or V) cache
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
   HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, m.dtype, st));
   SplitDesc sd;
@@ -368,7 +372,7 @@ hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* 
   AcceptArgs a{};
   a.tree_tok = tree_tok; a.amax = amax; a.parent = c->d_parent; a.depth = c->d_depth; a.anc = c->d_anc;
   a.T = c->T; a.K = c->h.n_heads; a.batch = c->batch; a.n_layers = m.n_layers; a.n_heads = m.n_heads; a.head_dim = m.head_dim;
-  a.max_seq = m.max_seq; a.max_batch = m.max_batch; a.d_model = m.d_model; a.esize = c->esize; a.kv_planes = c->planes;
+  a.max_seq = m.max_seq; a.max_batch = m.max_batch; a.d_model = m.d_model; a.esize = c->kv_esize; a.kv_planes = 1;
   a.kv_base = c->kv_base; a.h_tree = c->h_tree; a.h_tree_stride = c->T;
   a.h_new = c->h_new; a.n_new = c->d_n_new; a.len = c->d_len; a.root_tok = c->d_root_tok;
   a.n_acc = n_acc; a.path = path; a.out_tok = out_tok; a.done_counter = c->d_done; a.status = c->d_status;
@@ -603,7 +607,7 @@ hydra_status hydra_set_plant(hydra_ctx* c, const int32_t* plant) {
 hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes) {
   if (!c || !ptr) return HYDRA_ERR_INVALID;
   const hydra_model_cfg& m = c->m;
-  const size_t kvl = kv_layer_elems(m) * c->esize * c->planes;      // bytes of one layer's K (or V) cache, all planes
+  const size_t kvl = kv_layer_elems(m) * c->kv_esize;      // bytes of one layer's K (or V) cache
   const int K = c->h.n_heads;
   void* p = nullptr; size_t n = 0;
   switch (which) {
@@ -611,7 +615,7 @@ hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes
     case HYDRA_BUF_ROOT_TOK: p = c->d_root_tok; n = m.max_batch * sizeof(int); break;
     case HYDRA_BUF_H_TREE: p = c->h_tree; n = (size_t)c->R * m.d_model * sizeof(float); break;
     case HYDRA_BUF_H_NEW: p = c->h_new; n = (size_t)m.max_batch * (K + 1) * m.d_model * sizeof(float); break;
-    case HYDRA_BUF_KV_BASE: p = c->kv_base; n = (size_t)m.n_layers * 2 * kvl; break;          // kvl covers all planes
+    case HYDRA_BUF_KV_BASE: p = c->kv_base; n = (size_t)m.n_layers * 2 * kvl; break;
     case HYDRA_BUF_KV_PREFIX: p = c->h.prefix_attn ? c->kv_pfx : nullptr; n = c->h.prefix_attn ? 2 * kvl : 0; break;
     case HYDRA_BUF_TREE_MASK: p = c->d_anc; n = c->T * sizeof(uint64_t); break;
     case HYDRA_BUF_TREE_TOK: p = c->d_tree_tok; n = (size_t)m.max_batch * c->T * sizeof(int); break;
@@ -751,15 +755,19 @@ size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_di
 
 hydra_status hydra_tree_attention(const void* q, const void* kc, const void* vc, const int32_t* pos0, const int32_t* n_rows,
                                   const uint64_t* mask, void* out, void* scratch, int batch, int tc, int n_heads, int head_dim,
-                                  int max_seq, int dtype, int planes, void* stream) {
-  if (!q || !kc || !vc || !pos0 || !mask || !out || !scratch || batch < 1 || tc < 1 || tc > 64) return HYDRA_ERR_INVALID;
-  if (planes != 1 && !(planes == 2 && dtype == 1)) return HYDRA_ERR_INVALID;
+                                  int max_seq, int dtype, int out_planes, int32_t* status, void* stream) {
+  if (!q || !kc || !vc || !pos0 || !out || batch < 1 || tc < 1 || n_heads < 1 || max_seq < 1 || (dtype != 0 && dtype != 1)) return HYDRA_ERR_INVALID;
   CounterScope cs(nullptr);
   RowSet rs{batch, tc, n_rows, pos0, nullptr, mask};
+  if (dtype == 0) {
+    if (!mask || !scratch || out_planes != 1) return HYDRA_ERR_INVALID;
+    return tree_attention_f32((const float*)q, (const float*)kc, (const float*)vc, rs, (float*)out, scratch, n_heads, head_dim, max_seq, max_seq,
+                              (cudaStream_t)stream);
+  }
+  if (!status || (out_planes != 1 && out_planes != 2)) return HYDRA_ERR_INVALID;
   const size_t d = (size_t)n_heads * head_dim;
-  const size_t qp = planes == 2 ? (size_t)batch * tc * d : 0, kvp = planes == 2 ? (size_t)batch * n_heads * max_seq * head_dim : 0;
-  HYDRA_CUDA(cudaMemsetAsync(scratch, 0, ATT_SCRATCH_HEADER, (cudaStream_t)stream));     // arrival counters start at zero
-  return tree_attention(q, qp, kc, vc, kvp, rs, out, qp, scratch, n_heads, head_dim, max_seq, max_seq, dtype, (cudaStream_t)stream);
+  return tree_attention_tc((const __half*)q, batch * tc, (const __half*)kc, (const __half*)vc, batch, rs, (bf16*)out,
+                           out_planes == 2 ? (size_t)batch * tc * d : 0, n_heads, head_dim, max_seq, max_seq, status, (cudaStream_t)stream);
 }
 
 }  // extern "C"

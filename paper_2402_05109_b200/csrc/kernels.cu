@@ -122,6 +122,11 @@ template <> __device__ __forceinline__ void store4<bf16>(bf16* p, float4 v) {
   uint2 u; u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
   *reinterpret_cast<uint2*>(p) = u;
 }
+template <> __device__ __forceinline__ void store4<__half>(__half* p, float4 v) {
+  __half2 a = __floats2half2_rn(v.x, v.y), b = __floats2half2_rn(v.z, v.w);
+  uint2 u; u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
 template <typename T> __device__ __forceinline__ float4 load4(const T* p);
 template <> __device__ __forceinline__ float4 load4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
 template <> __device__ __forceinline__ float4 load4<bf16>(const bf16* p) {
@@ -215,11 +220,12 @@ hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cud
 
 // One thread rotates four consecutive pairs (j..j+3, j+half..j+half+3) of one head of q and k and copies the
 // matching v elements; all loads and stores are 16 bytes wide.
+// T: float (float model path) or float16 (bfloat16 model path: q and the caches are one float16 plane).
 template <typename T>
 __global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __restrict__ part, SplitDesc sd,
                                                              const float2* __restrict__ table, T* __restrict__ q,
-                                                             size_t q_ps, T* __restrict__ kc, T* __restrict__ vc,
-                                                             size_t kv_ps, RowSet rs, int H, int hd, int max_seq,
+                                                             T* __restrict__ kc, T* __restrict__ vc,
+                                                             RowSet rs, int H, int hd, int max_seq,
                                                              int* status) {
   pdl_trigger();
   pdl_wait();
@@ -255,26 +261,25 @@ __global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __rest
   float4 qlo, qhi, klo, khi;
   rot(v6[0], v6[1], qlo, qhi);
   rot(v6[2], v6[3], klo, khi);
-  put4<T>(q + (size_t)r * d + c0, q_ps, qlo);
-  put4<T>(q + (size_t)r * d + c1, q_ps, qhi);
+  store4<T>(q + (size_t)r * d + c0, qlo);
+  store4<T>(q + (size_t)r * d + c1, qhi);
   const size_t o = (((size_t)b * H + h) * max_seq + slot) * hd;
-  put4<T>(kc + o + j, kv_ps, klo);
-  put4<T>(kc + o + j + half, kv_ps, khi);
-  put4<T>(vc + o + j, kv_ps, v6[4]);
-  put4<T>(vc + o + j + half, kv_ps, v6[5]);
+  store4<T>(kc + o + j, klo);
+  store4<T>(kc + o + j + half, khi);
+  store4<T>(vc + o + j, v6[4]);
+  store4<T>(vc + o + j + half, v6[5]);
 }
-hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, size_t q_ps, void* kcache,
-                            void* vcache, size_t kv_ps, RowSet rs, int H, int hd, int max_seq, int dtype, int* status,
-                            cudaStream_t st) {
+hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, void* kcache, void* vcache, RowSet rs,
+                            int H, int hd, int max_seq, int dtype, int* status, cudaStream_t st) {
   if (hd % 8) return HYDRA_ERR_UNSUPPORTED;
   const int heads_per_block = 256 / (hd / 8);
   dim3 grid(rs.batch * rs.tc, (H + heads_per_block - 1) / heads_per_block);
   if (dtype == 0)
-    launch_pdl(qkv_rope_store_kernel<float>, grid, dim3(256), 0, st, part, sd, table, (float*)q, q_ps, (float*)kcache, (float*)vcache,
-               kv_ps, rs, H, hd, max_seq, status);
+    launch_pdl(qkv_rope_store_kernel<float>, grid, dim3(256), 0, st, part, sd, table, (float*)q, (float*)kcache, (float*)vcache,
+               rs, H, hd, max_seq, status);
   else
-    launch_pdl(qkv_rope_store_kernel<bf16>, grid, dim3(256), 0, st, part, sd, table, (bf16*)q, q_ps, (bf16*)kcache, (bf16*)vcache,
-               kv_ps, rs, H, hd, max_seq, status);
+    launch_pdl(qkv_rope_store_kernel<__half>, grid, dim3(256), 0, st, part, sd, table, (__half*)q, (__half*)kcache, (__half*)vcache,
+               rs, H, hd, max_seq, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -406,7 +411,7 @@ __global__ void tree_attn_combine_kernel(const float* __restrict__ part_o, const
 
 size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq) {
   size_t nchunks = (size_t)(max_seq + ATT_CHUNK - 1) / ATT_CHUNK;
-  return ATT_SCRATCH_HEADER + (size_t)batch * tc * n_heads * nchunks * (head_dim + 2) * sizeof(float);
+  return (size_t)batch * tc * n_heads * nchunks * (head_dim + 2) * sizeof(float);
 }
 
 template <typename T, int HD>
@@ -433,16 +438,11 @@ static hydra_status tree_attention_t(const T* q, const T* kc, const T* vc, RowSe
   return HYDRA_OK;
 }
 
-hydra_status tree_attention(const void* q, size_t q_ps, const void* kc, const void* vc, size_t kv_ps, RowSet rs, void* out,
-                            size_t out_ps, void* scratch, int H, int hd, int max_seq, int len_upper, int dtype, cudaStream_t st) {
-  if (rs.tc > 64) return HYDRA_ERR_UNSUPPORTED;
-  if (dtype == 1)
-    return tree_attention_tc((const bf16*)q, q_ps, (const bf16*)kc, (const bf16*)vc, kv_ps, rs, (bf16*)out, out_ps, scratch, H, hd,
-                             max_seq, len_upper, st);
-  if (dtype == 0 && hd == 64)
-    return tree_attention_t<float, 64>((const float*)q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
-  if (dtype == 0 && hd == 128)
-    return tree_attention_t<float, 128>((const float*)q, (const float*)kc, (const float*)vc, rs, (float*)out, (float*)scratch, H, max_seq, len_upper, st);
+hydra_status tree_attention_f32(const float* q, const float* kc, const float* vc, RowSet rs, float* out, void* scratch, int H, int hd,
+                                int max_seq, int len_upper, cudaStream_t st) {
+  if (rs.tc > 64 || !rs.mask) return HYDRA_ERR_UNSUPPORTED;
+  if (hd == 64) return tree_attention_t<float, 64>(q, kc, vc, rs, out, (float*)scratch, H, max_seq, len_upper, st);
+  if (hd == 128) return tree_attention_t<float, 128>(q, kc, vc, rs, out, (float*)scratch, H, max_seq, len_upper, st);
   return HYDRA_ERR_UNSUPPORTED;
 }
 

@@ -30,20 +30,21 @@ hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd,
                               cudaStream_t st);
 // table[r][j] = (cos, sin) of (pos0[b]+depth[i]) * theta^(-2j/head_dim), evaluated in double
 hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st);
-// q (operand dtype, [rows][H][hd], rotated), K/V cache rows (rotated K) from the QKV partial sums.
-hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, size_t q_ps,
-                            void* kcache, void* vcache, size_t kv_ps, RowSet rs, int n_heads, int head_dim, int max_seq, int dtype,
-                            int* status, cudaStream_t st);
-constexpr int ATT_CHUNK_ROWS = 128;     // KV rows per attention CTA (split-KV granularity)
-constexpr size_t ATT_SCRATCH_HEADER = 65536; // bytes at the head of the attention scratch: per-(sequence, head) arrival counters
+// q ([rows][H][hd], rotated) and the K/V cache rows (rotated K) from the QKV partial sums; float for dtype 0, float16
+// (one plane) for dtype 1.
+hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, void* kcache, void* vcache, RowSet rs,
+                            int n_heads, int head_dim, int max_seq, int dtype, int* status, cudaStream_t st);
+// Float model path: SIMT kernel + combine kernel, partial rows of ATT_CHUNK_ROWS-row chunks in `scratch`
+// (attention_scratch_bytes).  q, caches and out are float.
+constexpr int ATT_CHUNK_ROWS = 128;
 size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
-// bfloat16 caches: tensor-core kernel (attention_tc.cu); float caches: SIMT kernel.  q is in the cache dtype.
-// "_ps" arguments: element distance between the hi and lo planes of a bfloat16 operand (0 = hi only; unused for float).
-hydra_status tree_attention_tc(const bf16* q, size_t q_ps, const bf16* kc, const bf16* vc, size_t kv_ps, RowSet rs, bf16* out,
-                               size_t out_ps, void* scratch, int n_heads, int head_dim, int max_seq, int len_upper, cudaStream_t st);
-hydra_status tree_attention(const void* q, size_t q_ps, const void* kcache, const void* vcache, size_t kv_ps, RowSet rs, void* out,
-                            size_t out_ps, void* scratch, int n_heads, int head_dim, int max_seq, int len_upper, int dtype,
-                            cudaStream_t st);
+hydra_status tree_attention_f32(const float* q, const float* kcache, const float* vcache, RowSet rs, float* out, void* scratch,
+                                int n_heads, int head_dim, int max_seq, int len_upper, cudaStream_t st);
+// bfloat16 model path: tensor-core kernel (attention_tc.cu).  q [q_rows][H*hd] and the caches [cache_batch][H][max_seq][hd]
+// are float16, one plane; out is bfloat16 [rows][H*hd] in two planes out_ps elements apart (0: hi only).  rs.mask == null
+// selects a causal chunk (row i sees the committed slots and new slots 0..i) of up to 128 rows; with a mask, up to 64 rows.
+hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out,
+                               size_t out_ps, int n_heads, int head_dim, int max_seq, int len_upper, int* status, cudaStream_t st);
 hydra_status silu_mul(const float* part, SplitDesc sd, void* act, size_t act_ps, int rows, int f, int dtype,
                       cudaStream_t st);
 // amax[r] = argmax_v of the summed partial logits (lowest id among equal maxima); the sums go to logits_out if given

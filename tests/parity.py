@@ -27,20 +27,19 @@ def split_hi_lo(x: torch.Tensor) -> torch.Tensor:
     return torch.stack([hi, lo]).contiguous()
 
 
-def kv_planes(g, which: str) -> torch.Tensor:
-    """Raw view of a cache buffer: KV_BASE -> [layers][k,v][planes][batch][heads][seq][hd], KV_PREFIX without the
-    layer axis.  planes = 2 (hi, lo) on the bfloat16 path, 1 on the float path."""
+def kv_raw(g, which: str) -> torch.Tensor:
+    """Raw view of a cache buffer in its element type (float32 on the float path, float16 on the bfloat16 path):
+    KV_BASE -> [layers][k,v][batch][heads][seq][hd], KV_PREFIX without the layer axis."""
     m = g.model
-    planes = 1 if g.dtype == torch.float32 else 2
-    shape = (2, planes, g.max_batch, m.n_heads, g.max_seq, m.head_dim)
+    shape = (2, g.max_batch, m.n_heads, g.max_seq, m.head_dim)
     if which == "KV_BASE":
         shape = (m.n_layers,) + shape
     return g.get_buffer(which).view(shape)
 
 
 def kv_values(g, which: str) -> torch.Tensor:
-    """Cache values as float (hi + lo): KV_BASE -> [layers][k,v][batch][heads][seq][hd]."""
-    return kv_planes(g, which).float().sum(dim=-5)
+    """Cache values as float."""
+    return kv_raw(g, which).float()
 
 
 def rel_l2(a: torch.Tensor, b: torch.Tensor) -> float:
@@ -62,13 +61,15 @@ class Stats:
     n_acc: List[List[int]] = field(default_factory=list)
 
 
-def check_children(o: HydraOracle, b: int, tok_g: torch.Tensor, st: Stats):
-    """Every drafted child of every parent against the oracle's head evaluated on the GPU's own path
-    tokens (so a legitimate under-gap difference upstream does not cascade)."""
+def check_children(o: HydraOracle, b: int, tok_g: torch.Tensor, hp: torch.Tensor, st: Stats):
+    """Every drafted child of every parent against the oracle's head evaluated on the library's own inputs: its path
+    tokens (so a legitimate under-gap difference upstream does not cascade) and its h' (which is compared with the
+    oracle's on its own; the random-weight head MLPs amplify an input difference several times per layer, so feeding
+    the oracle's h' would test that amplification, not the head kernels)."""
     t = o.tree
     for d in range(1, t.K + 1):
         for p in t.level_parents[d - 1]:
-            lg = o.head_logits(d, o.hprime[b], [int(tok_g[b, j]) for j in t.path[p]])
+            lg = o.head_logits(d, hp, [int(tok_g[b, j]) for j in t.path[p]])
             k = len(t.children[p])
             ref = topk_desc(lg, k + 1)
             vals = [float(lg[r]) for r in ref]
@@ -132,15 +133,16 @@ def lockstep(o: HydraOracle, g, prompts, steps: int, seed: int, plant: bool = Tr
                     assert e <= HID_TOL, f"step {s}: prefix-layer cache rel-L2 {e}"
         if check_heads:
             tg = tok_g.cpu().long()
+            hp_o = [hp[b].cpu().to(o.dtype) for b in range(B)]      # the library's h' as the oracle head's input
             for b in range(B):
-                check_children(o, b, tg, st)
+                check_children(o, b, tg, hp_o[b], st)
             if o.tree.K > 0:                       # logits of the last drafted level, numerically
                 d = o.tree.K
                 P = o.tree.level_parents[d - 1]
                 hl = g.get_buffer("HEAD_LOGITS").view(-1, m.vocab)
                 for b in range(B):
                     for j, p in enumerate(P):
-                        ref = o.head_logits(d, o.hprime[b], [int(tg[b, i]) for i in o.tree.path[p]])
+                        ref = o.head_logits(d, hp_o[b], [int(tg[b, i]) for i in o.tree.path[p]])
                         e = float((hl[b * len(P) + j].cpu().double() - ref.double()).abs().max())
                         st.max_head_logit_err = max(st.max_head_logit_err, e)
                         assert e <= LOGIT_TOL, f"head logits max-abs {e}"

@@ -1,14 +1,14 @@
 """The acceptance + compaction kernel driven directly through hydra_accept_compact with arbitrary candidate and
 argmax arrays: a three-token alphabet makes equal-depth ties and duplicate siblings frequent (the cases the drafted
 and planted trees of the step tests never produce).  Integer outputs are compared bit for bit with the oracle; a
-move is a copy, so every moved cache row of every layer (and plane) must EQUAL the pre-move row."""
+move is a copy, so every moved cache row of every layer must EQUAL the pre-move row."""
 import pytest
 import torch
 
 from oracle.hydra_oracle import HydraOracle
 from synth import make_weights, make_prompts, load_tree
 from synth.configs import ModelCfg, HeadCfg
-from tests.parity import kv_planes
+from tests.parity import kv_raw
 
 pytestmark = pytest.mark.gpu
 
@@ -43,7 +43,7 @@ def test_accept_compact_kernel_on_ties_and_duplicates(dtype, hd):
         # CUDA side: same state every trial
         g.workspace.copy_(snapshot)
         g.verify(tok_real)                          # rewrites the same tree rows; puts the context into the verified state
-        pre = kv_planes(g, "KV_BASE").clone()
+        pre = kv_raw(g, "KV_BASE").clone()
         h_tree = g.get_buffer("H_TREE")[:B * T * m.d_model].view(B, T, m.d_model).clone()
         n_g, path_g, out_g = g.accept_compact(tok.to(torch.int32).cuda(), amax.to(torch.int32).cuda())
         g.poll_status()
@@ -53,16 +53,16 @@ def test_accept_compact_kernel_on_ties_and_duplicates(dtype, hd):
         assert g.get_buffer("LEN")[:B].cpu().tolist() == o.len
         assert g.get_buffer("ROOT_TOK")[:B].cpu().tolist() == o.root_tok
         assert g.get_buffer("N_NEW")[:B].cpu().tolist() == [int(n) + 1 for n in n_o]
-        post = kv_planes(g, "KV_BASE")
+        post = kv_raw(g, "KV_BASE")
         h_new = g.get_buffer("H_NEW").view(g.max_batch, K + 1, m.d_model)
         for b in range(B):
             n, L = int(n_o[b]), lens0[b]
             seen_n.add(n)
             path = path_o[b, :n + 1].tolist()
-            want = pre[:, :, :, b].clone()                                  # [layers][k,v][planes][heads][seq][hd]
+            want = pre[:, :, b].clone()                                     # [layers][k,v][heads][seq][hd]
             for k in range(1, n + 1):
-                want[..., L + k, :] = pre[:, :, :, b, :, L + path[k], :]
-            assert torch.equal(post[:, :, :, b, :, :L + n + 1], want[..., :L + n + 1, :]), (trial, b)
+                want[..., L + k, :] = pre[:, :, b, :, L + path[k], :]
+            assert torch.equal(post[:, :, b, :, :L + n + 1], want[..., :L + n + 1, :]), (trial, b)
             assert torch.equal(h_new[b, :n + 1], h_tree[b, path]), (trial, b)
     assert seen_n == {0, 1, 2, 3}
     g.close()
