@@ -13,7 +13,8 @@
  *    row-major [out][in].  dtype 0: weights, KV cache and GEMM operands are float; dtype 1: weights are
  *    bfloat16; activations that feed a GEMM are stored as TWO bfloat16 planes (hi = bf16(v), lo = bf16(v - hi),
  *    about 16 mantissa bits together); the attention operands (q, the post-rotation K cache, the V cache and the
- *    softmax weights) are float16, one plane; accumulation, residual stream, norms and softmax stay float.
+ *    softmax weights) are float16 in two planes (hi = f16(v), lo = f16(v - hi); hydra_model_cfg.kv_planes = 1 keeps
+ *    hi only); accumulation, residual stream, norms and softmax stay float.
  *  - The caller owns the weights, the workspace and every in/out buffer and keeps them alive until
  *    hydra_destroy.  The library owns only the opaque context; KV caches, tables and scratch are
  *    carved out of the caller's workspace (hydra_workspace_bytes, 256-byte aligned base).
@@ -58,6 +59,9 @@ typedef struct {
   float rms_eps, rope_theta;
   int dtype;               /* 0 = float, 1 = bfloat16 */
   int max_batch, max_seq;  /* capacity of the KV caches */
+  int kv_planes;           /* dtype 1 only: float16 planes of q and the KV caches.  0 or 2: hi + lo (about 22 bits: hidden states
+                              stay within ~1e-4 of a float reference over 60 layers); 1: hi only (half the cache bytes; a few
+                              1e-3 over 32 layers, not enough for the deepest shapes) */
 } hydra_model_cfg;
 
 /* Draft model: K heads, head i an m-layer residual SiLU MLP over [h ; E[x_t] ; E of the i-1 tokens
@@ -154,8 +158,9 @@ enum {
   HYDRA_BUF_ROOT_TOK = 1,   /* int32 [max_batch] */
   HYDRA_BUF_H_TREE = 2,     /* float [batch*n_rows][d] post-final-norm hidden of the last verify */
   HYDRA_BUF_H_NEW = 3,      /* float [max_batch][K+1][d] hidden rows committed by the last step */
-  HYDRA_BUF_KV_BASE = 4,    /* [n_layers][k,v][max_batch][n_heads][max_seq][head_dim]; float for dtype 0, float16 for dtype 1 */
-  HYDRA_BUF_KV_PREFIX = 5,  /* [k,v][max_batch][n_heads][max_seq][head_dim], same element type */
+  HYDRA_BUF_KV_BASE = 4,    /* [n_layers][k,v][planes][max_batch][n_heads][max_seq][head_dim]; float, planes = 1 for dtype 0;
+                               float16, planes = kv_planes (hi, lo) for dtype 1 */
+  HYDRA_BUF_KV_PREFIX = 5,  /* [k,v][planes][max_batch][n_heads][max_seq][head_dim], same element type */
   HYDRA_BUF_TREE_MASK = 6,  /* uint64 [n_rows] ancestor-or-self bitmask */
   HYDRA_BUF_TREE_TOK = 7,   /* int32 [batch][n_rows] tokens of the last hydra_step */
   HYDRA_BUF_AMAX = 8,       /* int32 [batch][n_rows] */
@@ -197,14 +202,15 @@ const char* hydra_last_error(void); /* text of the last CUDA error seen by this 
  *   hydra_gemm_partial_floats(m, n, k, dtype, mode) floats: the tensor-core GEMM leaves per-CTA partial sums
  *   there, which a second kernel adds in fixed order.  mode as in hydra_set_gemm_mode; status_dev is an int32
  *   status word (bit 1 bounds, bit 2 timeout).
- * hydra_tree_attention (Background, "Tree decoding": a token attends only to its ancestors): q [rows][n_heads][head_dim]
- *   (rows = batch*tc), caches [batch][n_heads][max_seq][head_dim], pos0 [batch] committed lengths, n_rows [batch] or
+ * hydra_tree_attention (Background, "Tree decoding": a token attends only to its ancestors): q [planes][rows][n_heads][head_dim]
+ *   (rows = batch*tc), caches [planes][batch][n_heads][max_seq][head_dim], pos0 [batch] committed lengths, n_rows [batch] or
  *   NULL (= tc), mask [tc] ancestor bitmasks.  Row i of sequence b sees slots < pos0[b] and slot pos0[b]+j when bit j
  *   of mask[i] is set; mask NULL (dtype 1 only) means a causal chunk: slot pos0[b]+j is visible when j <= i.
  *   dtype 0: q, caches and out [rows][n_heads*head_dim] are float, tc <= 64, scratch_dev needs
- *   hydra_attention_scratch_bytes(...) bytes, out_planes = 1, status_dev unused.  dtype 1: q and the caches are float16,
- *   out is bfloat16 [out_planes][rows][n_heads*head_dim] (2: hi = bf16(v) and lo = bf16(v - hi)); tc <= 64 with a mask,
- *   <= 128 causal; scratch_dev unused (may be NULL); status_dev is an int32 status word (bit 2: a bounded wait ran out). */
+ *   hydra_attention_scratch_bytes(...) bytes, planes = out_planes = 1, status_dev unused.  dtype 1: q and the caches are
+ *   float16 in `planes` planes (2: hi = f16(v), lo = f16(v - hi)), out is bfloat16 [out_planes][rows][n_heads*head_dim]
+ *   (2: hi = bf16(v) and lo = bf16(v - hi)); tc <= 64 with a mask, <= 128 causal (one plane or head_dim 64 only, else
+ *   UNSUPPORTED); scratch_dev unused (may be NULL); status_dev is an int32 status word (bit 2: a bounded wait ran out). */
 size_t hydra_gemm_partial_floats(int m, int n, int k, int dtype, int mode);
 hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, float* partial_dev, int m, int n, int k,
                         int dtype, int mode, int x_planes, int32_t* status_dev, void* stream);
@@ -240,7 +246,7 @@ size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_di
 hydra_status hydra_tree_attention(const void* q_dev, const void* k_cache_dev, const void* v_cache_dev,
                                   const int32_t* pos0_dev, const int32_t* n_rows_dev, const uint64_t* mask_dev,
                                   void* out_dev, void* scratch_dev, int batch, int tc, int n_heads, int head_dim,
-                                  int max_seq, int dtype, int out_planes, int32_t* status_dev, void* stream);
+                                  int max_seq, int dtype, int planes, int out_planes, int32_t* status_dev, void* stream);
 
 #ifdef __cplusplus
 }

@@ -18,7 +18,7 @@ class HydraError(RuntimeError):
 class ModelCfgC(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("dtype", C.c_int), ("max_batch", C.c_int),
-                ("max_seq", C.c_int)]
+                ("max_seq", C.c_int), ("kv_planes", C.c_int)]
 
 
 class HeadCfgC(C.Structure):
@@ -70,7 +70,7 @@ lib.hydra_gemm_noalloc.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp]
 lib.hydra_gemm_bounded_wait_probe.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, C.c_uint, _vp, _vp, _vp]
 lib.hydra_attention_scratch_bytes.restype = _sz
 lib.hydra_attention_scratch_bytes.argtypes = [_i] * 5
-lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 7 + [_vp, _vp]
+lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 8 + [_vp, _vp]
 
 BUF = dict(LEN=0, ROOT_TOK=1, H_TREE=2, H_NEW=3, KV_BASE=4, KV_PREFIX=5, TREE_MASK=6, TREE_TOK=7, AMAX=8,
            HEAD_LOGITS=9, N_NEW=10, H_PRIME=11, STATUS=12)
@@ -115,7 +115,9 @@ class Hydra:
             if not t.is_cuda or not t.is_contiguous() or t.dtype != self.dtype:
                 raise HydraError("weight %s must be a contiguous CUDA tensor of %s" % (name, self.dtype))
         self._mc = ModelCfgC(model.n_layers, model.d_model, model.n_heads, model.head_dim, model.d_ffn, model.vocab,
-                             model.rms_eps, model.rope_theta, 0 if model.dtype == "fp32" else 1, max_batch, max_seq)
+                             model.rms_eps, model.rope_theta, 0 if model.dtype == "fp32" else 1, max_batch, max_seq,
+                             int(getattr(model, "kv_planes", 2)))
+        self.kv_planes = 1 if model.dtype == "fp32" else (1 if self._mc.kv_planes == 1 else 2)
         self._hc = HeadCfgC(head.n_heads, head.n_mlp_layers, int(head.prefix_attn), int(head.has_bias))
         self._parent_arr = (C.c_int32 * self.T)(*self.parent)
         self._tc = TreeCfgC(self.T, self._parent_arr)
@@ -274,13 +276,16 @@ def gemm_noalloc(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor, status: to
 
 def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int, out_planes: int = 1) -> torch.Tensor:
     """hydra_tree_attention.  q [batch*tc][H][hd], caches [batch][H][S][hd]: all float32, or all float16 (the bfloat16
-    model path, whose result is bfloat16 in out_planes planes: [rows][H*hd] or [2][rows][H*hd] = hi, lo).
+    model path, whose result is bfloat16 in out_planes planes: [rows][H*hd] or [2][rows][H*hd] = hi, lo).  float16 inputs
+    may carry a leading axis of 2: the hi = f16(v) and lo = f16(v - hi) planes.
     mask: int64 [tc] ancestor bitmasks, or None for a causal chunk (float16 only)."""
-    batch, n_heads, max_seq, head_dim = k_cache.shape
+    planes = 2 if k_cache.dim() == 5 else 1
+    batch, n_heads, max_seq, head_dim = k_cache.shape[-4:]
     _need(k_cache.dtype in (torch.float32, torch.float16), "caches must be float32 or float16")
     for name, t in (("q", q), ("k_cache", k_cache), ("v_cache", v_cache)):
         _dense_cuda(t, k_cache.dtype, name)
-    _need(v_cache.shape == k_cache.shape and q.numel() == batch * tc * n_heads * head_dim, "q / cache shapes")
+    _need(v_cache.shape == k_cache.shape and q.numel() == planes * batch * tc * n_heads * head_dim, "q / cache shapes")
+    _need(planes == 1 or k_cache.dtype == torch.float16, "two planes: float16 only")
     _dense_cuda(pos0, torch.int32, "pos0")
     _need(pos0.numel() == batch and (n_rows is None or n_rows.numel() == batch), "pos0 [batch], n_rows [batch]")
     if mask is not None:
@@ -301,7 +306,7 @@ def tree_attention(q, k_cache, v_cache, pos0, n_rows, mask, tc: int, out_planes:
         scratch, dtype = None, 1
     _check(lib.hydra_tree_attention(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), pos0.data_ptr(), _ptr(n_rows),
                                     _ptr(mask), out.data_ptr(), _ptr(scratch), batch, tc, n_heads, head_dim,
-                                    max_seq, dtype, out_planes, status.data_ptr(), _stream()), "hydra_tree_attention")
+                                    max_seq, dtype, planes, out_planes, status.data_ptr(), _stream()), "hydra_tree_attention")
     word = int(status.item())
     if word:
         raise HydraError("hydra_tree_attention device status word %d" % word)

@@ -1,9 +1,13 @@
 // Tree attention for the bfloat16 model path on the sm_100a tensor cores: TMA tile loads, tcgen05.mma with the
 // score and output accumulators in tensor memory, softmax out of tensor memory.
 //
-// Operand format: q, the K cache (post-RoPE) and the V cache are float16, one plane (11 significant bits; the
-// values are O(1), far inside the float16 range); the softmax weights are rounded to float16 for the P V product;
-// scores, running maxima, sums and the output accumulate in float.  The result leaves as two bfloat16 planes
+// Operand format: q, the K cache (post-RoPE), the V cache and the softmax weights are float16 (the values are O(1),
+// far inside the float16 range) in NP planes.  NP = 2: hi = f16(v), lo = f16(v - hi), about 22 significant bits;
+// a product x y is taken as x_hi y_hi + x_hi y_lo + x_lo y_hi.  Stacking the planes of the B operand along its N
+// dimension gives the first two terms in ONE instruction sequence (accumulator columns [0, n) and [n, 2n), added
+// when the accumulator is read); the third is a second sequence into columns [0, n).  NP = 1: hi only, 11 bits
+// (half the cache bytes; hidden states then drift to a few 1e-3 of a float reference over 32 layers).
+// Scores, running maxima, sums and the output accumulate in float.  The result leaves as two bfloat16 planes
 // (hi = bf16(v), lo = bf16(v - hi)), the operand format of the GEMM that consumes it.
 //
 // One CTA per (head, sequence, KV chunk).  A sequence's KV rows are cut into 64-row tiles and the tiles are dealt
@@ -39,7 +43,6 @@ namespace {
 using namespace tc;
 
 constexpr int TILE = 64;           // KV rows per tile
-constexpr int NST = 3;             // ring stages (K and V of TILE rows each)
 constexpr int MAX_CHUNKS = 8;      // chunks of a (head, sequence) pair = cluster size
 constexpr float RESCALE_STEP = 8.f;
 
@@ -75,33 +78,45 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
 
 struct AttArgs {
   RowSet rs;
+  int q_plane_rows, kv_plane_rows;     // rows between the hi and lo planes in the q and cache tensor maps
   bf16* out; size_t out_ps;
   int H, max_seq, nchunks;
   int* status;
   uint32_t wait_limit;
 };
 
-template <int HD, int QROWS> struct AttCfg {
+template <int HD, int QROWS, int NP> struct AttCfg {
   static constexpr int NHALF = HD / 64;                       // 64-column (128-byte) halves of a head row
-  static constexpr int Q_BYTES = NHALF * QROWS * 128;
-  static constexpr int P_BYTES = QROWS * 128;                 // one P tile: [query row][64 keys] float16
-  static constexpr int KV_BYTES = NHALF * TILE * 128;         // K (or V) of one tile
-  static constexpr int STAGE_BYTES = 2 * KV_BYTES;
+  static constexpr int QP_BYTES = NHALF * QROWS * 128;        // one plane of Q: [half][query row][128 bytes]
+  static constexpr int Q_BYTES = NP * QP_BYTES;
+  static constexpr int PP_BYTES = QROWS * 128;                // one plane of a P tile: [query row][64 keys] float16
+  static constexpr int P_BYTES = NP * PP_BYTES;
+  static constexpr int KH_BYTES = NP * TILE * 128;            // one half of a K tile: [plane][key][128 bytes] (the planes stacked along N)
+  static constexpr int K_BYTES = NHALF * KH_BYTES;
+  static constexpr int V_BYTES = NP * NHALF * TILE * 128;     // a V tile: [plane][half][key][128 bytes] (N blocks of 64 output columns)
+  static constexpr int STAGE_BYTES = K_BYTES + V_BYTES;
+  static constexpr int NST = NP == 1 ? 3 : (HD == 64 ? 3 : 2);        // ring stages
   static constexpr int RING_BYTES = NST * STAGE_BYTES;
   static constexpr int MERGE_BYTES = QROWS * HD * 4 + QROWS * 8;     // a chunk's partial rows + (max, sum); aliases the ring
   static constexpr int NBAR = 1 + 3 * NST + 8;
-  // The M = 128 operand reads of a 64-row Q or P tile run 8 KB past the tile: Q's into P, P's into the ring
-  // (unused lanes, never read back), so the order Q, P0, P1, ring keeps them inside the allocation.
+  // The M = 128 operand reads of a 64-row Q or P tile run 8 KB past the tile, into the next piece of Q, of P or of the
+  // ring (unused lanes, never read back), so the order Q, P0, P1, ring keeps them inside the allocation.
   static constexpr int SMEM_BYTES = 1024 + Q_BYTES + 2 * P_BYTES + (RING_BYTES > MERGE_BYTES ? RING_BYTES : MERGE_BYTES) + NBAR * 8 + 16;
-  static constexpr int TMEM_COLS = 256;                       // S0 [0,64), S1 [64,128), O [128, 128+HD)
+  static constexpr int S_COLS = NP * TILE;                    // one score buffer: [Q_hi K_hi + Q_lo K_hi | Q_hi K_lo]
+  static constexpr int O_COLS = NP * HD;                      // the output accumulator: [P_hi V_hi + P_lo V_hi | P_hi V_lo]
+  static constexpr int O_COL0 = 2 * S_COLS;
+  static constexpr int TMEM_COLS = O_COL0 + O_COLS <= 256 ? 256 : 512;
   static_assert(RING_BYTES >= MERGE_BYTES, "merge area must fit in the ring");
+  static_assert(O_COL0 + O_COLS <= 512, "tensor memory");
+  static_assert(SMEM_BYTES <= 232448, "shared memory of one SM");
 };
 
-template <int HD, int QROWS>
+template <int HD, int QROWS, int NP>
 __global__ void __launch_bounds__(192, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const AttArgs a) {
-  using C = AttCfg<HD, QROWS>;
+  using C = AttCfg<HD, QROWS, NP>;
+  constexpr int NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_s = base, p_s = q_s + C::Q_BYTES, ring_s = p_s + 2 * C::P_BYTES;
@@ -153,26 +168,37 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       const uint64_t pol = policy_evict_first(), pol_q = policy_evict_last();
       mbar_arrive_expect_tx(q_full, C::Q_BYTES);
 #pragma unroll
-      for (int hf = 0; hf < C::NHALF; ++hf) tma_load_2d(q_s + hf * QROWS * 128, &tmQ, h * HD + hf * 64, b * rs.tc, q_full, pol_q);
+      for (int pl = 0; pl < NP; ++pl)
+#pragma unroll
+        for (int hf = 0; hf < C::NHALF; ++hf)
+          tma_load_2d(q_s + pl * C::QP_BYTES + hf * QROWS * 128, &tmQ, h * HD + hf * 64, pl * a.q_plane_rows + b * rs.tc, q_full, pol_q);
       const int row0 = (b * H + h) * a.max_seq;
       for (int i = 0; i < ntiles; ++i) {
         const int s = i % NST;
         // stage s was last read by the P V product of tile i - NST, the (i / NST - 1)-th completion of its empty barrier
         if (i >= NST && !mbar_wait(kv_empty(s), (uint32_t)((i / NST - 1) & 1), limit)) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
-        const uint32_t k_dst = ring_s + s * C::STAGE_BYTES, v_dst = k_dst + C::KV_BYTES;
+        const uint32_t k_dst = ring_s + s * C::STAGE_BYTES, v_dst = k_dst + C::K_BYTES;
         const int r = row0 + (tile0 + i) * TILE;
-        mbar_arrive_expect_tx(k_full(s), C::KV_BYTES);
+        mbar_arrive_expect_tx(k_full(s), C::K_BYTES);
 #pragma unroll
-        for (int hf = 0; hf < C::NHALF; ++hf) tma_load_2d(k_dst + hf * TILE * 128, &tmK, hf * 64, r, k_full(s), pol);
-        mbar_arrive_expect_tx(v_full(s), C::KV_BYTES);
+        for (int pl = 0; pl < NP; ++pl)
 #pragma unroll
-        for (int hf = 0; hf < C::NHALF; ++hf) tma_load_2d(v_dst + hf * TILE * 128, &tmV, hf * 64, r, v_full(s), pol);
+          for (int hf = 0; hf < C::NHALF; ++hf)
+            tma_load_2d(k_dst + hf * C::KH_BYTES + pl * TILE * 128, &tmK, hf * 64, pl * a.kv_plane_rows + r, k_full(s), pol);
+        mbar_arrive_expect_tx(v_full(s), C::V_BYTES);
+#pragma unroll
+        for (int pl = 0; pl < NP; ++pl)
+#pragma unroll
+          for (int hf = 0; hf < C::NHALF; ++hf)
+            tma_load_2d(v_dst + (pl * C::NHALF + hf) * TILE * 128, &tmV, hf * 64, pl * a.kv_plane_rows + r, v_full(s), pol);
       }
     }
   } else if (warp == 1) {
     if (lane == 0 && has_work) {
-      constexpr uint32_t idesc_s = instr_desc_f16(0, 128, TILE, 0);
-      constexpr uint32_t idesc_pv = instr_desc_f16(0, 128, HD, 1);
+      constexpr uint32_t idesc_s = instr_desc_f16(0, 128, NP * TILE, 0);      // Q_hi x [K_hi ; K_lo]
+      constexpr uint32_t idesc_s2 = instr_desc_f16(0, 128, TILE, 0);          // Q_lo x K_hi
+      constexpr uint32_t idesc_pv = instr_desc_f16(0, 128, NP * HD, 1);       // P_hi x [V_hi | V_lo]
+      constexpr uint32_t idesc_pv2 = instr_desc_f16(0, 128, HD, 1);           // P_lo x V_hi
       bool ok = mbar_wait(q_full, 0, limit);
       auto issue_s = [&](int i) {                        // S_i = Q K_i^T into score buffer i & 1
         const int s = i % NST;
@@ -183,8 +209,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
           const uint32_t qa = q_s + (kk >> 2) * QROWS * 128 + (kk & 3) * 32;
-          const uint32_t kb = k_src + (kk >> 2) * TILE * 128 + (kk & 3) * 32;
-          umma_f16(tmem_base + (uint32_t)((i & 1) * TILE), smem_desc_sw128(qa), smem_desc_sw128(kb), idesc_s, (uint32_t)(kk != 0));
+          const uint32_t kb = k_src + (kk >> 2) * C::KH_BYTES + (kk & 3) * 32;
+          umma_f16(tmem_base + (uint32_t)((i & 1) * C::S_COLS), smem_desc_sw128(qa), smem_desc_sw128(kb), idesc_s, (uint32_t)(kk != 0));
+        }
+        if (NP == 2) {
+#pragma unroll
+          for (int kk = 0; kk < HD / 16; ++kk) {
+            const uint32_t qa = q_s + C::QP_BYTES + (kk >> 2) * QROWS * 128 + (kk & 3) * 32;
+            const uint32_t kb = k_src + (kk >> 2) * C::KH_BYTES + (kk & 3) * 32;
+            umma_f16(tmem_base + (uint32_t)((i & 1) * C::S_COLS), smem_desc_sw128(qa), smem_desc_sw128(kb), idesc_s2, 1u);
+          }
         }
         umma_commit(s_full(i & 1));
         return true;
@@ -197,12 +231,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (!mbar_wait(p_full(i & 1), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
         if (!mbar_wait(v_full(s), (uint32_t)((i / NST) & 1), limit)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t v_src = ring_s + s * C::STAGE_BYTES + C::KV_BYTES;
+        const uint32_t v_src = ring_s + s * C::STAGE_BYTES + C::K_BYTES;
         const uint32_t p_src = p_s + (i & 1) * C::P_BYTES;
 #pragma unroll
         for (int kk = 0; kk < TILE / 16; ++kk)
-          umma_f16(tmem_base + 128u, smem_desc_sw128(p_src + kk * 32), smem_desc_sw128_mn(v_src + kk * 2048, TILE * 128), idesc_pv,
+          umma_f16(tmem_base + (uint32_t)C::O_COL0, smem_desc_sw128(p_src + kk * 32), smem_desc_sw128_mn(v_src + kk * 2048, TILE * 128), idesc_pv,
                    (uint32_t)((i | kk) != 0));
+        if (NP == 2) {
+#pragma unroll
+          for (int kk = 0; kk < TILE / 16; ++kk)
+            umma_f16(tmem_base + (uint32_t)C::O_COL0, smem_desc_sw128(p_src + C::PP_BYTES + kk * 32), smem_desc_sw128_mn(v_src + kk * 2048, TILE * 128),
+                     idesc_pv2, 1u);
+        }
         umma_commit(kv_empty(s));
         umma_commit(pv_done(i & 1));
       }
@@ -225,7 +265,21 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!mbar_wait(s_full(i & 1), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
       tc_fence_after();
       uint32_t r[64];
-      if (warp_rows) tmem_ld64(lane_addr + (uint32_t)((i & 1) * TILE), r);
+      if (warp_rows) {
+        const uint32_t s_addr = lane_addr + (uint32_t)((i & 1) * C::S_COLS);
+        if (NP == 1) {
+          tmem_ld64(s_addr, r);
+        } else {
+#pragma unroll
+          for (int c0 = 0; c0 < 64; c0 += 32) {            // the two column halves of the score buffer, added
+            uint32_t x[32], y[32];
+            tmem_ld32(s_addr + (uint32_t)c0, x);
+            tmem_ld32(s_addr + (uint32_t)(TILE + c0), y);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[c0 + j] = __float_as_uint(__uint_as_float(x[j]) + __uint_as_float(y[j]));
+          }
+        }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(s_empty(i & 1));
@@ -258,8 +312,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int j = 0; j < 32; ++j) {
           const float p0v = ex2(__uint_as_float(r[2 * j]) - bse), p1v = ex2(__uint_as_float(r[2 * j + 1]) - bse);
           pk[j] = pack_half2(p0v, p1v);
-          const __half2 hv = *reinterpret_cast<const __half2*>(&pk[j]);
-          sum += __low2float(hv) + __high2float(hv);       // the sum of what the MMA will really weigh V with
+          if (NP == 1) {
+            const __half2 hv = *reinterpret_cast<const __half2*>(&pk[j]);
+            sum += __low2float(hv) + __high2float(hv);     // the sum of what the MMA will really weigh V with
+          } else {
+            sum += p0v + p1v;
+            r[2 * j] = __float_as_uint(p0v); r[2 * j + 1] = __float_as_uint(p1v);     // kept for the lo plane
+          }
         }
         l = l * alpha + sum;
         // P buffer i & 1 was last read by P V of tile i - 2; the row's accumulator by P V of tile i - 1
@@ -267,13 +326,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (__any_sync(0xffffffffu, rescale)) {
           if (i >= 1 && !mbar_wait(pv_done((i - 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), limit)) { ok = false; break; }
           tc_fence_after();
-#pragma unroll
-          for (int c0 = 0; c0 < HD; c0 += 32) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < C::O_COLS; c0 += 32) {
             uint32_t o[32];
-            tmem_ld32(lane_addr + 128u + (uint32_t)c0, o);
+            tmem_ld32(lane_addr + (uint32_t)(C::O_COL0 + c0), o);
 #pragma unroll
             for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-            tmem_st32(lane_addr + 128u + (uint32_t)c0, o);
+            tmem_st32(lane_addr + (uint32_t)(C::O_COL0 + c0), o);
           }
         }
         const uint32_t prow = p_s + (i & 1) * C::P_BYTES + (uint32_t)row * 128u;
@@ -282,6 +341,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int ch = 0; ch < 8; ++ch) {
             const uint32_t dst = prow + (uint32_t)((ch ^ (row & 7)) * 16);
             asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]), "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3]) : "memory");
+          }
+          if (NP == 2) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {                 // lo = f16(p - f16(p))
+              const __half2 hv = *reinterpret_cast<const __half2*>(&pk[j]);
+              pk[j] = pack_half2(__uint_as_float(r[2 * j]) - __low2float(hv), __uint_as_float(r[2 * j + 1]) - __high2float(hv));
+            }
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+              const uint32_t dst = prow + (uint32_t)(C::PP_BYTES + (ch ^ (row & 7)) * 16);
+              asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]), "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3]) : "memory");
+            }
           }
         }
       } else {
@@ -292,10 +363,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // zero weight times a non-finite stale value cannot reach the accumulator
         const int s = i % NST;
         if (!mbar_wait(v_full(s), (uint32_t)((i / NST) & 1), limit)) { ok = false; break; }
-        const uint32_t v_src = ring_s + s * C::STAGE_BYTES + C::KV_BYTES;
+        const uint32_t v_src = ring_s + s * C::STAGE_BYTES + C::K_BYTES;
         const int first = total - t0;                       // first row to clear (>= 1)
-        for (int e = st; e < (TILE - first) * C::NHALF * 8; e += 128) {
-          const int rr = first + e / (C::NHALF * 8), rem = e % (C::NHALF * 8);
+        constexpr int BLK = NP * C::NHALF;                  // 64-column blocks of a V tile
+        for (int e = st; e < (TILE - first) * BLK * 8; e += 128) {
+          const int rr = first + e / (BLK * 8), rem = e % (BLK * 8);
           const uint32_t dst = v_src + (uint32_t)((rem >> 3) * TILE * 128 + rr * 128 + (rem & 7) * 16);
           asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(dst), "r"(0u) : "memory");
         }
@@ -315,10 +387,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       const uint32_t xo = ring_s + (uint32_t)row * (HD * 4), xml = ring_s + QROWS * HD * 4 + (uint32_t)row * 8;
       const bool have = ok && ntiles > 0 && row_live && m_ref != -INFINITY;
       if (ok && ntiles > 0 && warp_rows) {
-#pragma unroll
+#pragma unroll 1
         for (int c0 = 0; c0 < HD; c0 += 32) {
           uint32_t o[32];
-          tmem_ld32(lane_addr + 128u + (uint32_t)c0, o);
+          tmem_ld32(lane_addr + (uint32_t)(C::O_COL0 + c0), o);
+          if (NP == 2) {
+            uint32_t o2[32];
+            tmem_ld32(lane_addr + (uint32_t)(C::O_COL0 + HD + c0), o2);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) + __uint_as_float(o2[j]));
+          }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {                    // float4 piece k4 of row i sits at position k4 ^ (i & (HD/4 - 1))
             const int k4 = c0 / 4 + j;
@@ -403,24 +481,26 @@ int pick_chunks(int pairs, int len_upper, int sms) {
   return best;
 }
 
-template <int HD, int QROWS>
+template <int HD, int QROWS, int NP>
 hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out, size_t out_ps,
                  int H, int max_seq, int len_upper, int* status, cudaStream_t st) {
-  using C = AttCfg<HD, QROWS>;
+  using C = AttCfg<HD, QROWS, NP>;
   CUtensorMap tq, tk, tv;
   const uint64_t cache_rows = (uint64_t)cache_batch * H * max_seq;
-  if (!get_tensor_map(q, (uint64_t)q_rows, (uint64_t)H * HD, QROWS, true, &tq) ||
-      !get_tensor_map(kc, cache_rows, HD, TILE, true, &tk) || !get_tensor_map(vc, cache_rows, HD, TILE, true, &tv)) {
+  if (cache_rows * NP > 0x7fffffffull) return HYDRA_ERR_UNSUPPORTED;          // tensor-map row coordinates are 32-bit
+  if (!get_tensor_map(q, (uint64_t)NP * q_rows, (uint64_t)H * HD, QROWS, true, &tq) ||
+      !get_tensor_map(kc, NP * cache_rows, HD, TILE, true, &tk) || !get_tensor_map(vc, NP * cache_rows, HD, TILE, true, &tv)) {
     set_last_error("cuTensorMapEncodeTiled", cudaErrorUnknown);
     return HYDRA_ERR_CUDA;
   }
   static PerDeviceFlag attr_done;
   if (!attr_done.get()) {
-    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, QROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    HYDRA_CUDA(cudaFuncSetAttribute(tree_attn_tc_kernel<HD, QROWS, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_done.set();
   }
   AttArgs a{};
   a.rs = rs; a.out = out; a.out_ps = out_ps; a.H = H; a.max_seq = max_seq; a.status = status; a.wait_limit = WAIT_LIMIT;
+  a.q_plane_rows = q_rows; a.kv_plane_rows = (int)cache_rows;
   a.nchunks = pick_chunks(H * rs.batch, len_upper, sm_count());
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(H, rs.batch, a.nchunks); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = C::SMEM_BYTES; cfg.stream = st;
@@ -430,24 +510,32 @@ hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
-  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<HD, QROWS>, tq, tk, tv, a));
+  HYDRA_CUDA(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<HD, QROWS, NP>, tq, tk, tv, a));
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
+template <int NP>
+hydra_status dispatch(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out, size_t out_ps,
+                      int H, int hd, int max_seq, int len_upper, int* status, cudaStream_t st) {
+  const bool wide = rs.tc > 64;
+  if (hd == 128 && wide && NP == 2) return HYDRA_ERR_UNSUPPORTED;       // Q, P and a two-stage ring of two planes exceed the shared memory of an SM
+  if (hd == 128) return wide ? run<128, 128, 1>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st)
+                             : run<128, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st);
+  if (hd == 64) return wide ? run<64, 128, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st)
+                            : run<64, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st);
+  return HYDRA_ERR_UNSUPPORTED;
+}
+
 }  // namespace
 
-hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out,
-                               size_t out_ps, int H, int hd, int max_seq, int len_upper, int* status, cudaStream_t st) {
-  if (rs.tc > 128 || (rs.mask && rs.tc > 64)) return HYDRA_ERR_UNSUPPORTED;
+hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, int planes, RowSet rs,
+                               bf16* out, size_t out_ps, int H, int hd, int max_seq, int len_upper, int* status, cudaStream_t st) {
+  if (rs.tc > 128 || (rs.mask && rs.tc > 64) || (planes != 1 && planes != 2)) return HYDRA_ERR_UNSUPPORTED;
   if (!tensor_map_encoder_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
   if (((uintptr_t)q | (uintptr_t)kc | (uintptr_t)vc) & 15) return HYDRA_ERR_INVALID;
-  const bool wide = rs.tc > 64;
-  if (hd == 128) return wide ? run<128, 128>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st)
-                             : run<128, 64>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st);
-  if (hd == 64) return wide ? run<64, 128>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st)
-                            : run<64, 64>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st);
-  return HYDRA_ERR_UNSUPPORTED;
+  return planes == 2 ? dispatch<2>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, hd, max_seq, len_upper, status, st)
+                     : dispatch<1>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, hd, max_seq, len_upper, status, st);
 }
 
 }  // namespace hydra

@@ -55,6 +55,7 @@ struct hydra_ctx {
   int esize;                                     // bytes per weight element
   int planes;                                    // planes of every GEMM operand buffer: 2 (hi, lo) for bfloat16, 1 for float
   int kv_esize;                                  // bytes per element of q and the KV caches: 4 (float) or 2 (float16)
+  int kv_planes;                                 // planes of q and the KV caches: 1, or 2 (float16 hi + lo)
   int R;                                         // row capacity of a forward call (padded)
   int RH;                                        // row capacity of the head buffers (padded)
   int maxP;
@@ -140,6 +141,7 @@ bool valid_cfg(const hydra_model_cfg* m, const hydra_head_cfg* h) {
     return false;
   if (m->n_heads * m->head_dim != m->d_model) return false;
   if (m->dtype != 0 && m->dtype != 1) return false;
+  if (m->kv_planes < 0 || m->kv_planes > 2) return false;
   if (h->n_heads < 0 || h->n_mlp_layers < 1) return false;
   return true;
 }
@@ -156,7 +158,8 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   Bump b{ws, 0};
   const int es = m.dtype == 0 ? 4 : 2;
   const int np = m.dtype == 0 ? 1 : 2;          // bfloat16 GEMM operands are stored as hi + lo planes
-  const int ces = m.dtype == 0 ? 4 : 2;         // q and the KV caches: float, or one float16 plane
+  const int ces = m.dtype == 0 ? 4 : 2;         // q and the KV caches: float, or float16 in kvp planes
+  const int kvp = m.dtype == 0 ? 1 : (m.kv_planes == 1 ? 1 : 2);
   const int d = m.d_model, f = m.d_ffn, V = m.vocab, K = h.n_heads, T = t.T;
   const int R = pad_rows(m.max_batch * CHUNK);
   const int RH = pad_rows(m.max_batch * t.maxP);
@@ -190,9 +193,9 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
   auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
   auto* done = b.take<unsigned int>(m.max_batch);
-  auto* kvb = b.take<char>((size_t)m.n_layers * 2 * kv_layer_elems(m) * ces);
-  auto* kvp = b.take<char>(h.prefix_attn ? (size_t)2 * kv_layer_elems(m) * ces : 0);
-  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)(R + 128) * d * ces);
+  auto* kvb = b.take<char>((size_t)m.n_layers * 2 * kvp * kv_layer_elems(m) * ces);
+  auto* kvpfx = b.take<char>(h.prefix_attn ? (size_t)2 * kvp * kv_layer_elems(m) * ces : 0);
+  auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)kvp * R * d * ces);
   auto* part = b.take<float>(part_floats);
   auto* h_tree = b.take<float>((size_t)R * d);
   auto* logits = b.take<float>((size_t)pad_rows(m.max_batch * T) * V);
@@ -207,12 +210,12 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* topk_s = b.take<char>(topk_scratch_bytes(topk_cap, V));
   auto* att = b.take<char>(m.dtype == 0 ? attention_scratch_bytes(m.max_batch, CHUNK, m.n_heads, m.head_dim, m.max_seq) : 0);
   if (c) {
-    c->R = R; c->RH = RH; c->part_floats = part_floats; c->esize = es; c->planes = np; c->kv_esize = ces;
+    c->R = R; c->RH = RH; c->part_floats = part_floats; c->esize = es; c->planes = np; c->kv_esize = ces; c->kv_planes = kvp;
     c->d_parent = parent; c->d_depth = depth; c->d_first_child = fc; c->d_n_child = nc; c->d_path_tab = path_tab;
     c->d_chain_depth = chain_depth; c->d_anc = anc; c->d_chain_mask = chain_mask; c->d_level_parents = lvl;
     c->d_len = len; c->d_n_new = n_new; c->d_root_tok = root; c->d_status = status; c->d_pos0 = pos0; c->d_nrows = nrows;
     c->d_prompt_len = plen; c->d_offsets = offs; c->d_tok = tok; c->d_tree_tok = tree_tok; c->d_amax = amax; c->d_done = done;
-    c->kv_base = kvb; c->kv_pfx = kvp; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits;
+    c->kv_base = kvb; c->kv_pfx = kvpfx; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits;
     c->h_new = h_new; c->hprime = hprime; c->y = y; c->head_logits = head_logits; c->rope = rope; c->xn = xn;
     c->attn_out = attn_out; c->act = act; c->z = z; c->yb = yb; c->att_scratch = att; c->topk_scratch = topk_s; c->topk_rows_cap = topk_cap;
   }
@@ -252,12 +255,13 @@ size_t ps(const hydra_ctx* c, int rows_alloc, size_t cols) { return c->planes ==
 hydra_status attention_block(hydra_ctx* c, char* kc, char* vc, const RowSet& rs, int len_upper, const SplitDesc& sd, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int d = m.d_model, dt = m.dtype;
-  HYDRA_TRY(qkv_rope_store(c->part, sd, c->rope, c->q, kc, vc, rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
+  const size_t q_ps = c->kv_planes == 2 ? (size_t)c->R * d : 0, kv_ps = c->kv_planes == 2 ? kv_layer_elems(m) : 0;
+  HYDRA_TRY(qkv_rope_store(c->part, sd, c->rope, c->q, q_ps, kc, vc, kv_ps, rs, m.n_heads, m.head_dim, m.max_seq, dt, c->d_status, st));
   TimeScope ts(c, HYDRA_TIME_ATTENTION, 0.0, st);
   if (dt == 0)
     return tree_attention_f32((const float*)c->q, (const float*)kc, (const float*)vc, rs, (float*)c->attn_out, c->att_scratch, m.n_heads,
                               m.head_dim, m.max_seq, len_upper, st);
-  return tree_attention_tc((const __half*)c->q, c->R, (const __half*)kc, (const __half*)vc, m.max_batch, rs, (bf16*)c->attn_out,
+  return tree_attention_tc((const __half*)c->q, c->R, (const __half*)kc, (const __half*)vc, m.max_batch, c->kv_planes, rs, (bf16*)c->attn_out,
                            ps(c, c->R, d), m.n_heads, m.head_dim, m.max_seq, len_upper, c->d_status, st);
 }
 
@@ -289,7 +293,7 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
                       cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int rows = rs.batch * rs.tc, d = m.d_model;
-  const size_t kvl = kv_layer_elems(m) * c->kv_esize;      // bytes of one layer's K (or V) cache
+  const size_t kvl = kv_layer_elems(m) * c->kv_esize * c->kv_planes;      // bytes of one layer's K (or V) cache, all planes
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
   HYDRA_TRY(embed_rows(c->embed, tok, c->x, rows, d, m.vocab, m.dtype, c->d_status, st));
   HYDRA_TRY(residual_rmsnorm(c->x, nullptr, single_slot(0), c->x, c->layers[0].attn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, m.dtype, st));
@@ -308,7 +312,7 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
 hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int len_upper, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int rows = rs.batch * rs.tc, d = m.d_model;
-  const size_t kvl = kv_layer_elems(m) * c->kv_esize;      // bytes of one layer's K (or V) cache
+  const size_t kvl = kv_layer_elems(m) * c->kv_esize * c->kv_planes;      // bytes of one layer's K (or V) cache, all planes
   HYDRA_TRY(rope_table(rs, c->rope, m.head_dim, m.rope_theta, st));
   HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, m.dtype, st));
   SplitDesc sd;
@@ -372,7 +376,7 @@ hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* 
   AcceptArgs a{};
   a.tree_tok = tree_tok; a.amax = amax; a.parent = c->d_parent; a.depth = c->d_depth; a.anc = c->d_anc;
   a.T = c->T; a.K = c->h.n_heads; a.batch = c->batch; a.n_layers = m.n_layers; a.n_heads = m.n_heads; a.head_dim = m.head_dim;
-  a.max_seq = m.max_seq; a.max_batch = m.max_batch; a.d_model = m.d_model; a.esize = c->kv_esize; a.kv_planes = 1;
+  a.max_seq = m.max_seq; a.max_batch = m.max_batch; a.d_model = m.d_model; a.esize = c->kv_esize; a.kv_planes = c->kv_planes;
   a.kv_base = c->kv_base; a.h_tree = c->h_tree; a.h_tree_stride = c->T;
   a.h_new = c->h_new; a.n_new = c->d_n_new; a.len = c->d_len; a.root_tok = c->d_root_tok;
   a.n_acc = n_acc; a.path = path; a.out_tok = out_tok; a.done_counter = c->d_done; a.status = c->d_status;
@@ -607,7 +611,7 @@ hydra_status hydra_set_plant(hydra_ctx* c, const int32_t* plant) {
 hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes) {
   if (!c || !ptr) return HYDRA_ERR_INVALID;
   const hydra_model_cfg& m = c->m;
-  const size_t kvl = kv_layer_elems(m) * c->kv_esize;      // bytes of one layer's K (or V) cache
+  const size_t kvl = kv_layer_elems(m) * c->kv_esize * c->kv_planes;      // bytes of one layer's K (or V) cache, all planes
   const int K = c->h.n_heads;
   void* p = nullptr; size_t n = 0;
   switch (which) {
@@ -755,18 +759,18 @@ size_t hydra_attention_scratch_bytes(int batch, int tc, int n_heads, int head_di
 
 hydra_status hydra_tree_attention(const void* q, const void* kc, const void* vc, const int32_t* pos0, const int32_t* n_rows,
                                   const uint64_t* mask, void* out, void* scratch, int batch, int tc, int n_heads, int head_dim,
-                                  int max_seq, int dtype, int out_planes, int32_t* status, void* stream) {
+                                  int max_seq, int dtype, int planes, int out_planes, int32_t* status, void* stream) {
   if (!q || !kc || !vc || !pos0 || !out || batch < 1 || tc < 1 || n_heads < 1 || max_seq < 1 || (dtype != 0 && dtype != 1)) return HYDRA_ERR_INVALID;
   CounterScope cs(nullptr);
   RowSet rs{batch, tc, n_rows, pos0, nullptr, mask};
   if (dtype == 0) {
-    if (!mask || !scratch || out_planes != 1) return HYDRA_ERR_INVALID;
+    if (!mask || !scratch || out_planes != 1 || planes != 1) return HYDRA_ERR_INVALID;
     return tree_attention_f32((const float*)q, (const float*)kc, (const float*)vc, rs, (float*)out, scratch, n_heads, head_dim, max_seq, max_seq,
                               (cudaStream_t)stream);
   }
-  if (!status || (out_planes != 1 && out_planes != 2)) return HYDRA_ERR_INVALID;
+  if (!status || (out_planes != 1 && out_planes != 2) || (planes != 1 && planes != 2)) return HYDRA_ERR_INVALID;
   const size_t d = (size_t)n_heads * head_dim;
-  return tree_attention_tc((const __half*)q, batch * tc, (const __half*)kc, (const __half*)vc, batch, rs, (bf16*)out,
+  return tree_attention_tc((const __half*)q, batch * tc, (const __half*)kc, (const __half*)vc, batch, planes, rs, (bf16*)out,
                            out_planes == 2 ? (size_t)batch * tc * d : 0, n_heads, head_dim, max_seq, max_seq, status, (cudaStream_t)stream);
 }
 

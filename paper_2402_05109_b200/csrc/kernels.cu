@@ -127,6 +127,15 @@ template <> __device__ __forceinline__ void store4<__half>(__half* p, float4 v) 
   uint2 u; u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
   *reinterpret_cast<uint2*>(p) = u;
 }
+// float: one plane.  float16: hi = f16(v) and, ps elements further on, lo = f16(v - hi) (ps = 0: hi only).
+template <typename T> __device__ __forceinline__ void put4h(T* p, size_t ps, float4 v);
+template <> __device__ __forceinline__ void put4h<float>(float* p, size_t, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+template <> __device__ __forceinline__ void put4h<__half>(__half* p, size_t ps, float4 v) {
+  const float4 h = make_float4(__half2float(__float2half_rn(v.x)), __half2float(__float2half_rn(v.y)),
+                               __half2float(__float2half_rn(v.z)), __half2float(__float2half_rn(v.w)));
+  store4<__half>(p, h);
+  if (ps) store4<__half>(p + ps, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
+}
 template <typename T> __device__ __forceinline__ float4 load4(const T* p);
 template <> __device__ __forceinline__ float4 load4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
 template <> __device__ __forceinline__ float4 load4<bf16>(const bf16* p) {
@@ -220,11 +229,11 @@ hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cud
 
 // One thread rotates four consecutive pairs (j..j+3, j+half..j+half+3) of one head of q and k and copies the
 // matching v elements; all loads and stores are 16 bytes wide.
-// T: float (float model path) or float16 (bfloat16 model path: q and the caches are one float16 plane).
+// T: float (float model path) or float16 (bfloat16 model path: q and the caches are float16 in one or two planes).
 template <typename T>
 __global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __restrict__ part, SplitDesc sd,
-                                                             const float2* __restrict__ table, T* __restrict__ q,
-                                                             T* __restrict__ kc, T* __restrict__ vc,
+                                                             const float2* __restrict__ table, T* __restrict__ q, size_t q_ps,
+                                                             T* __restrict__ kc, T* __restrict__ vc, size_t kv_ps,
                                                              RowSet rs, int H, int hd, int max_seq,
                                                              int* status) {
   pdl_trigger();
@@ -261,25 +270,25 @@ __global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __rest
   float4 qlo, qhi, klo, khi;
   rot(v6[0], v6[1], qlo, qhi);
   rot(v6[2], v6[3], klo, khi);
-  store4<T>(q + (size_t)r * d + c0, qlo);
-  store4<T>(q + (size_t)r * d + c1, qhi);
+  put4h<T>(q + (size_t)r * d + c0, q_ps, qlo);
+  put4h<T>(q + (size_t)r * d + c1, q_ps, qhi);
   const size_t o = (((size_t)b * H + h) * max_seq + slot) * hd;
-  store4<T>(kc + o + j, klo);
-  store4<T>(kc + o + j + half, khi);
-  store4<T>(vc + o + j, v6[4]);
-  store4<T>(vc + o + j + half, v6[5]);
+  put4h<T>(kc + o + j, kv_ps, klo);
+  put4h<T>(kc + o + j + half, kv_ps, khi);
+  put4h<T>(vc + o + j, kv_ps, v6[4]);
+  put4h<T>(vc + o + j + half, kv_ps, v6[5]);
 }
-hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, void* kcache, void* vcache, RowSet rs,
-                            int H, int hd, int max_seq, int dtype, int* status, cudaStream_t st) {
+hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, size_t q_ps, void* kcache, void* vcache,
+                            size_t kv_ps, RowSet rs, int H, int hd, int max_seq, int dtype, int* status, cudaStream_t st) {
   if (hd % 8) return HYDRA_ERR_UNSUPPORTED;
   const int heads_per_block = 256 / (hd / 8);
   dim3 grid(rs.batch * rs.tc, (H + heads_per_block - 1) / heads_per_block);
   if (dtype == 0)
-    launch_pdl(qkv_rope_store_kernel<float>, grid, dim3(256), 0, st, part, sd, table, (float*)q, (float*)kcache, (float*)vcache,
-               rs, H, hd, max_seq, status);
+    launch_pdl(qkv_rope_store_kernel<float>, grid, dim3(256), 0, st, part, sd, table, (float*)q, q_ps, (float*)kcache, (float*)vcache,
+               kv_ps, rs, H, hd, max_seq, status);
   else
-    launch_pdl(qkv_rope_store_kernel<__half>, grid, dim3(256), 0, st, part, sd, table, (__half*)q, (__half*)kcache, (__half*)vcache,
-               rs, H, hd, max_seq, status);
+    launch_pdl(qkv_rope_store_kernel<__half>, grid, dim3(256), 0, st, part, sd, table, (__half*)q, q_ps, (__half*)kcache, (__half*)vcache,
+               kv_ps, rs, H, hd, max_seq, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }

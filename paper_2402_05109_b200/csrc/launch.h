@@ -30,21 +30,23 @@ hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd,
                               cudaStream_t st);
 // table[r][j] = (cos, sin) of (pos0[b]+depth[i]) * theta^(-2j/head_dim), evaluated in double
 hydra_status rope_table(RowSet rs, float2* table, int head_dim, float theta, cudaStream_t st);
-// q ([rows][H][hd], rotated) and the K/V cache rows (rotated K) from the QKV partial sums; float for dtype 0, float16
-// (one plane) for dtype 1.
-hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, void* kcache, void* vcache, RowSet rs,
-                            int n_heads, int head_dim, int max_seq, int dtype, int* status, cudaStream_t st);
+// q ([rows][H][hd], rotated) and the K/V cache rows (rotated K) from the QKV partial sums; float for dtype 0; for dtype 1
+// float16 with a lo plane (f16(v - f16(v))) q_ps / kv_ps elements after the hi plane (0: hi only).
+hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, size_t q_ps, void* kcache, void* vcache,
+                            size_t kv_ps, RowSet rs, int n_heads, int head_dim, int max_seq, int dtype, int* status, cudaStream_t st);
 // Float model path: SIMT kernel + combine kernel, partial rows of ATT_CHUNK_ROWS-row chunks in `scratch`
 // (attention_scratch_bytes).  q, caches and out are float.
 constexpr int ATT_CHUNK_ROWS = 128;
 size_t attention_scratch_bytes(int batch, int tc, int n_heads, int head_dim, int max_seq);
 hydra_status tree_attention_f32(const float* q, const float* kcache, const float* vcache, RowSet rs, float* out, void* scratch,
                                 int n_heads, int head_dim, int max_seq, int len_upper, cudaStream_t st);
-// bfloat16 model path: tensor-core kernel (attention_tc.cu).  q [q_rows][H*hd] and the caches [cache_batch][H][max_seq][hd]
-// are float16, one plane; out is bfloat16 [rows][H*hd] in two planes out_ps elements apart (0: hi only).  rs.mask == null
-// selects a causal chunk (row i sees the committed slots and new slots 0..i) of up to 128 rows; with a mask, up to 64 rows.
-hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out,
-                               size_t out_ps, int n_heads, int head_dim, int max_seq, int len_upper, int* status, cudaStream_t st);
+// bfloat16 model path: tensor-core kernel (attention_tc.cu).  q [planes][q_rows][H*hd] and the caches
+// [planes][cache_batch][H][max_seq][hd] are float16 in 1 or 2 planes (hi = f16(v), lo = f16(v - hi)); out is bfloat16
+// [rows][H*hd] in two planes out_ps elements apart (0: hi only).  rs.mask == null selects a causal chunk (row i sees
+// the committed slots and new slots 0..i) of up to 128 rows (one plane, or head_dim 64); with a mask, up to 64 rows.
+hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, int planes, RowSet rs,
+                               bf16* out, size_t out_ps, int n_heads, int head_dim, int max_seq, int len_upper, int* status,
+                               cudaStream_t st);
 hydra_status silu_mul(const float* part, SplitDesc sd, void* act, size_t act_ps, int rows, int f, int dtype,
                       cudaStream_t st);
 // amax[r] = argmax_v of the summed partial logits (lowest id among equal maxima); the sums go to logits_out if given

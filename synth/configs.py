@@ -13,7 +13,8 @@ class ModelCfg:
     vocab: int
     rms_eps: float = 1e-6
     rope_theta: float = 1e4
-    dtype: str = "bf16"            # "fp32" | "bf16": storage type of weights and KV cache
+    dtype: str = "bf16"            # "fp32" | "bf16": storage type of the weights
+    kv_planes: int = 2             # bf16 path: float16 planes of q and the KV caches (2: hi + lo, 1: hi only)
 
 
 @dataclass

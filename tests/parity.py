@@ -27,19 +27,26 @@ def split_hi_lo(x: torch.Tensor) -> torch.Tensor:
     return torch.stack([hi, lo]).contiguous()
 
 
+def split_f16(x: torch.Tensor) -> torch.Tensor:
+    """[2, ...] float16: hi = f16(x), lo = f16(x - hi) of a float tensor (how the library stores q and cache rows)."""
+    hi = x.to(torch.float16)
+    lo = (x.float() - hi.float()).to(torch.float16)
+    return torch.stack([hi, lo]).contiguous()
+
+
 def kv_raw(g, which: str) -> torch.Tensor:
-    """Raw view of a cache buffer in its element type (float32 on the float path, float16 on the bfloat16 path):
-    KV_BASE -> [layers][k,v][batch][heads][seq][hd], KV_PREFIX without the layer axis."""
+    """Raw view of a cache buffer in its element type (float32 on the float path, float16 hi / lo planes on the
+    bfloat16 path): KV_BASE -> [layers][k,v][planes][batch][heads][seq][hd], KV_PREFIX without the layer axis."""
     m = g.model
-    shape = (2, g.max_batch, m.n_heads, g.max_seq, m.head_dim)
+    shape = (2, g.kv_planes, g.max_batch, m.n_heads, g.max_seq, m.head_dim)
     if which == "KV_BASE":
         shape = (m.n_layers,) + shape
     return g.get_buffer(which).view(shape)
 
 
 def kv_values(g, which: str) -> torch.Tensor:
-    """Cache values as float."""
-    return kv_raw(g, which).float()
+    """Cache values as float (the planes added)."""
+    return kv_raw(g, which).float().sum(dim=-5)
 
 
 def rel_l2(a: torch.Tensor, b: torch.Tensor) -> float:

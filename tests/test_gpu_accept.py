@@ -1,7 +1,7 @@
 """The acceptance + compaction kernel driven directly through hydra_accept_compact with arbitrary candidate and
 argmax arrays: a three-token alphabet makes equal-depth ties and duplicate siblings frequent (the cases the drafted
 and planted trees of the step tests never produce).  Integer outputs are compared bit for bit with the oracle; a
-move is a copy, so every moved cache row of every layer must EQUAL the pre-move row."""
+move is a copy, so every moved cache row of every layer (and plane) must EQUAL the pre-move row."""
 import pytest
 import torch
 
@@ -59,10 +59,10 @@ def test_accept_compact_kernel_on_ties_and_duplicates(dtype, hd):
             n, L = int(n_o[b]), lens0[b]
             seen_n.add(n)
             path = path_o[b, :n + 1].tolist()
-            want = pre[:, :, b].clone()                                     # [layers][k,v][heads][seq][hd]
+            want = pre[:, :, :, b].clone()                                  # [layers][k,v][planes][heads][seq][hd]
             for k in range(1, n + 1):
-                want[..., L + k, :] = pre[:, :, b, :, L + path[k], :]
-            assert torch.equal(post[:, :, b, :, :L + n + 1], want[..., :L + n + 1, :]), (trial, b)
+                want[..., L + k, :] = pre[:, :, :, b, :, L + path[k], :]
+            assert torch.equal(post[:, :, :, b, :, :L + n + 1], want[..., :L + n + 1, :]), (trial, b)
             assert torch.equal(h_new[b, :n + 1], h_tree[b, path]), (trial, b)
     assert seen_n == {0, 1, 2, 3}
     g.close()
