@@ -14,11 +14,16 @@ What it follows (Hydra: Sequentially-Dependent Draft Heads for Medusa Decoding):
   * Section "Hydra++": MLP depth 4 and one extra decoder layer queried once per step.
   * Background, verification criteria: greedy acceptance (a candidate is kept when it equals the
     base model's most likely token).
+  * Section "Typical acceptance sampling", paragraph "Typical acceptance criterion": a candidate is
+    kept when its probability under the temperature-tau base distribution at its parent exceeds
+    min(epsilon, alpha * exp(-entropy of that distribution)).
 
 Pinned by tests/test_oracle_*.py: a whole-model comparison against the `transformers` Llama
 implementation, chain-tree == token-by-token decoding, root-only tree == greedy decoding, output
 invariance to the drafted tokens, brute-force acceptance, compaction == sequential decoding,
-closed-form head cases, library sort for top-k, brute-force ancestor masks.
+closed-form head cases, library sort for top-k, brute-force ancestor masks; the typical criterion by its
+limits (tau -> 0 is the greedy criterion, epsilon -> 0 keeps every candidate, a uniform row has
+entropy log V), a library entropy routine and brute force over the tree's paths.
 Parity unpinned: the numeric values of logits for the random models (the paper prints none); they
 are fixed only by the pins above on the operations that produce them.
 """
@@ -123,6 +128,27 @@ def argmax_lowest(logits: torch.Tensor) -> torch.Tensor:
     V = logits.shape[-1]
     idx = torch.arange(V).expand_as(logits)
     return torch.where(logits == mx, idx, torch.full_like(idx, V)).min(dim=-1).values
+
+
+def typical_row(logits: torch.Tensor, tau: float, eps: float, alpha: float):
+    """One parent's side of the typical acceptance criterion (Section "Typical acceptance sampling",
+    displayed inequality): p = softmax(logits / tau), H = -sum p log p, threshold = min(eps, alpha * exp(-H)).
+    Returns (p, threshold); a child token x is accepted when p[x] > threshold."""
+    z = logits.double() / tau
+    z = z - z.max()
+    e = torch.exp(z)
+    p = e / e.sum()
+    logp = z - torch.log(e.sum())
+    H = -(p * logp).sum()                      # p = 0 terms vanish: exp underflow gives 0 * finite
+    return p, min(eps, alpha * math.exp(-float(H)))
+
+
+def inverse_cdf(p: torch.Tensor, u: float) -> int:
+    """The token drawn from p by the uniform number u in [0, 1): the first id whose cumulative probability
+    (in token-id order) exceeds u."""
+    c = torch.cumsum(p.double(), dim=0)
+    idx = int((c > u * float(c[-1])).nonzero()[0])
+    return idx
 
 
 # ----------------------------------------------------------------------------- the oracle
@@ -257,38 +283,87 @@ class HydraOracle:
             amax.append(argmax_lowest(lg))
         return torch.stack(amax), torch.stack(logits)
 
-    # -- greedy acceptance + cache compaction
-    def accept_compact(self, tree_tok: torch.Tensor, amax: torch.Tensor):
-        """A candidate is accepted when it equals the base argmax at its parent and its parent is
-        accepted; the deepest accepted row wins (lowest row index among equals).  The accepted rows'
-        K,V move next to the committed prefix, everything else in the tree is dropped."""
+    # -- acceptance + cache compaction
+    def _commit(self, b: int, best: int, new_root: int, tree_tok: torch.Tensor):
+        """Append the accepted path root..best of sequence b to its state: the accepted rows' K,V move next to the
+        committed prefix (everything else in the tree is dropped), their hidden rows feed the next draft."""
         t = self.tree
+        path = t.path[best]
+        n = len(path) - 1
+        L = self.len[b]
+        for l in range(self.m.n_layers):
+            for cache in (self.kc[l][b], self.vc[l][b]):
+                moved = cache[L + torch.tensor(path)].clone()        # out of place
+                cache[L:L + n + 1] = moved
+        self.h_new[b] = self.h_tree[b][path].clone()
+        self.len[b] = L + n + 1
+        self.root_tok[b] = new_root
         K = self.h.n_heads
+        out = [int(tree_tok[b, j]) for j in path[1:]] + [new_root]
+        return n, path + [-1] * (K + 1 - len(path)), out + [-1] * (K + 1 - len(out))
+
+    def _deepest(self, accepted: List[bool]) -> int:
+        """The deepest accepted row, the lowest row index among equals."""
+        t = self.tree
+        best = 0
+        for i in range(t.T):
+            if accepted[i] and t.depth[i] > t.depth[best]:
+                best = i
+        return best
+
+    def accept_compact(self, tree_tok: torch.Tensor, amax: torch.Tensor):
+        """Greedy criterion: a candidate is accepted when it equals the base argmax at its parent and its parent is
+        accepted; the deepest accepted row wins (lowest row index among equals)."""
+        t = self.tree
         n_acc, paths, outs = [], [], []
         for b in range(self.B):
             accepted = [True] + [False] * (t.T - 1)
             for i in range(1, t.T):                       # parents precede children
                 p = t.parent[i]
                 accepted[i] = accepted[p] and int(tree_tok[b, i]) == int(amax[b, p])
-            best = 0
-            for i in range(t.T):
-                if accepted[i] and t.depth[i] > t.depth[best]:
-                    best = i
-            path = t.path[best]
-            n = len(path) - 1
-            new_root = int(amax[b, best])
-            L = self.len[b]
-            for l in range(self.m.n_layers):
-                for cache in (self.kc[l][b], self.vc[l][b]):
-                    moved = cache[L + torch.tensor(path)].clone()        # out of place
-                    cache[L:L + n + 1] = moved
-            self.h_new[b] = self.h_tree[b][path].clone()
-            self.len[b] = L + n + 1
-            self.root_tok[b] = new_root
-            n_acc.append(n)
-            paths.append(path + [-1] * (K + 1 - len(path)))
-            out = [int(tree_tok[b, j]) for j in path[1:]] + [new_root]
-            outs.append(out + [-1] * (K + 1 - len(out)))
+            best = self._deepest(accepted)
+            n, path, out = self._commit(b, best, int(amax[b, best]), tree_tok)
+            n_acc.append(n); paths.append(path); outs.append(out)
+        return torch.tensor(n_acc), torch.tensor(paths), torch.tensor(outs)
+
+    def typical_pass(self, tree_tok: torch.Tensor, logits: torch.Tensor, tau: float, eps: float, alpha: float):
+        """[B][T] bool: candidate i passes the typical criterion at its parent (row 0 is True).  Also returns the
+        margin log p - log threshold of every candidate (how far the decision is from flipping)."""
+        t = self.tree
+        ok = torch.ones(self.B, t.T, dtype=torch.bool)
+        margin = torch.full((self.B, t.T), float("inf"), dtype=torch.float64)
+        for b in range(self.B):
+            rows = {}
+            for i in range(1, t.T):
+                par = t.parent[i]
+                if par not in rows:
+                    rows[par] = typical_row(logits[b, par], tau, eps, alpha)
+                p, thr = rows[par]
+                px = float(p[int(tree_tok[b, i])])
+                ok[b, i] = px > thr
+                margin[b, i] = (math.log(px) if px > 0 else -1e30) - math.log(thr)
+        return ok, margin
+
+    def typical_accept_compact(self, tree_tok: torch.Tensor, logits: torch.Tensor, tau: float, eps: float, alpha: float,
+                               u: Optional[Sequence[float]] = None):
+        """Typical acceptance (Section "Typical acceptance sampling"): a candidate is accepted when it passes the
+        criterion at its parent and its parent is accepted; the deepest accepted row wins (lowest row index among
+        equals).  The token after the accepted path comes from the temperature-tau base distribution at the best
+        row: drawn by inverse CDF with the uniform number u[b], or its most likely token when u is None."""
+        t = self.tree
+        ok, _ = self.typical_pass(tree_tok, logits, tau, eps, alpha)
+        n_acc, paths, outs = [], [], []
+        for b in range(self.B):
+            accepted = [True] + [False] * (t.T - 1)
+            for i in range(1, t.T):
+                accepted[i] = accepted[t.parent[i]] and bool(ok[b, i])
+            best = self._deepest(accepted)
+            if u is None:
+                new_root = int(argmax_lowest(logits[b, best:best + 1])[0])
+            else:
+                new_root = inverse_cdf(typical_row(logits[b, best], tau, eps, alpha)[0], float(u[b]))
+            n, path, out = self._commit(b, best, new_root, tree_tok)
+            n_acc.append(n); paths.append(path); outs.append(out)
         return torch.tensor(n_acc), torch.tensor(paths), torch.tensor(outs)
 
     def step(self, plant: Optional[torch.Tensor] = None):

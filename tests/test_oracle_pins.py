@@ -363,3 +363,117 @@ def test_sibling_permutation_invariance():
     tok2 = tok[:, perm]
     _, lg2 = o.verify(tok2)
     assert (lg2[0][perm] - lg[0]).abs().max() < 1e-11
+
+
+# ------------------------------------------------------------------ typical acceptance (Section "Typical acceptance sampling")
+def _typical_setup(seed=3):
+    m, h, w = tiny()
+    parent = load_tree("tree15_d3")
+    o = HydraOracle(m, h, parent, w, 64)
+    o.prefill([make_prompts(1, [5], m.vocab)[0]])
+    g = torch.Generator().manual_seed(seed)
+    return m, o, g
+
+
+def _reset(o, m):
+    o.h_tree = [torch.zeros(o.tree.T, m.d_model, dtype=torch.float64)]
+    o.len = [5]
+
+
+def test_typical_row_against_library_entropy_and_closed_forms():
+    from oracle.hydra_oracle import typical_row
+    scipy_special = pytest.importorskip("scipy.special")
+    scipy_stats = pytest.importorskip("scipy.stats")
+    g = torch.Generator().manual_seed(1)
+    for tau in (0.3, 0.7, 1.0, 2.5):
+        lg = torch.randn(97, generator=g, dtype=torch.float64) * 3.0
+        p, thr = typical_row(lg, tau, 0.3, 0.5)
+        p_lib = scipy_special.softmax(lg.numpy() / tau)
+        assert float((p - torch.from_numpy(p_lib)).abs().max()) < 1e-14
+        H = float(scipy_stats.entropy(p_lib))                   # natural logarithm
+        assert abs(thr - min(0.3, 0.5 * math.exp(-H))) < 1e-14
+    # a uniform row: p = 1/V, entropy log V, so the threshold is min(eps, alpha / V)
+    V = 64
+    p, thr = typical_row(torch.full((V,), 1.7, dtype=torch.float64), 0.7, 0.2, 0.4)
+    assert float((p - 1.0 / V).abs().max()) < 1e-15 and abs(thr - min(0.2, 0.4 / V)) < 1e-15
+    # a one-hot row (huge gap): entropy 0, threshold min(eps, alpha)
+    lg = torch.zeros(V, dtype=torch.float64); lg[5] = 1e4
+    p, thr = typical_row(lg, 1.0, 0.25, 0.1)
+    assert float(p[5]) == 1.0 and thr == 0.1
+    # the posterior threshold caps it from above
+    assert typical_row(lg, 1.0, 0.05, 0.9)[1] == 0.05
+
+
+def test_typical_acceptance_limits_and_brute_force():
+    """tau -> 0: the temperature distribution collapses on the argmax, the entropy goes to 0 and the criterion is the
+    greedy one.  eps -> 0 (alpha = sqrt(eps)): every candidate of non-zero probability passes, so the deepest leaf
+    with the lowest row index wins.  In between: brute force over all root-to-leaf paths with the pass bits taken
+    straight from the inequality."""
+    from oracle.hydra_oracle import typical_row
+    m, o, g = _typical_setup()
+    t = o.tree
+    V = m.vocab
+    for trial in range(60):
+        logits = torch.randn(1, t.T, V, generator=g, dtype=torch.float64) * 2.0
+        amax = argmax_lowest(logits[0])[None]
+        tok = torch.randint(0, V, (1, t.T), generator=g)
+        for i in range(1, t.T):                                  # plant the argmax of the parent on about half the rows
+            if torch.rand(1, generator=g).item() < 0.5:
+                tok[0, i] = amax[0, t.parent[i]]
+        # tau -> 0 equals the greedy criterion (bonus token: argmax either way)
+        _reset(o, m)
+        n_t, path_t, out_t = o.typical_accept_compact(tok, logits, 1e-3, 0.3, 0.5)
+        _reset(o, m)
+        n_g, path_g, out_g = o.accept_compact(tok, amax)
+        assert torch.equal(n_t, n_g) and torch.equal(path_t, path_g) and torch.equal(out_t, out_g)
+        # eps -> 0 accepts everything: the first row of the deepest level
+        _reset(o, m)
+        n_e, path_e, _ = o.typical_accept_compact(tok, logits, 0.7, 1e-300, 1e-150)
+        deepest = min(i for i in range(t.T) if t.depth[i] == t.K)
+        assert int(n_e[0]) == t.K and [x for x in path_e[0].tolist() if x >= 0] == t.path[deepest]
+        # brute force at the paper's temperature and a threshold in its range
+        tau, eps = 0.7, 0.15
+        alpha = math.sqrt(eps)
+        bits = [True] * t.T
+        for i in range(1, t.T):
+            z = logits[0, t.parent[i]] / tau
+            p = torch.softmax(z, dim=0)                          # library routine
+            H = float(torch.distributions.Categorical(probs=p).entropy())
+            bits[i] = float(p[int(tok[0, i])]) > min(eps, alpha * math.exp(-H))
+        best, best_len = 0, 0
+        for leaf in range(t.T):                                  # every root-to-node path, longest all-pass prefix
+            path = t.path[leaf]
+            k = 0
+            while k + 1 < len(path) and bits[path[k + 1]]:
+                k += 1
+            if k > best_len or (k == best_len and path[k] < best):
+                best, best_len = path[k], k
+        _reset(o, m)
+        n_b, path_b, out_b = o.typical_accept_compact(tok, logits, tau, eps, alpha)
+        assert int(n_b[0]) == best_len and [x for x in path_b[0].tolist() if x >= 0] == t.path[best]
+        assert out_b[0].tolist()[:best_len + 1] == [int(tok[0, j]) for j in t.path[best][1:]] + [int(amax[0, best])]
+        ok, margin = o.typical_pass(tok, logits, tau, eps, alpha)
+        assert ok[0].tolist() == bits and all((margin[0, i] > 0) == bits[i] for i in range(1, t.T))
+
+
+def test_bonus_token_inverse_cdf():
+    """The sampled token against numpy's cumulative sum and searchsorted, and its frequencies against the distribution."""
+    import numpy as np
+    from oracle.hydra_oracle import inverse_cdf
+    g = torch.Generator().manual_seed(5)
+    p = torch.softmax(torch.randn(50, generator=g, dtype=torch.float64), dim=0)
+    c = np.cumsum(p.numpy())
+    us = torch.rand(4000, generator=g, dtype=torch.float64).tolist() + [0.0, 0.999999999]
+    draws = [inverse_cdf(p, u) for u in us]
+    assert draws == [int(np.searchsorted(c, u * c[-1], side="right")) for u in us]
+    freq = torch.bincount(torch.tensor(draws[:4000]), minlength=50).double() / 4000
+    assert float((freq - p).abs().max()) < 0.03
+    m, o, _ = _typical_setup()
+    t = o.tree
+    logits = torch.randn(1, t.T, m.vocab, generator=g, dtype=torch.float64)
+    tok = torch.zeros(1, t.T, dtype=torch.int64)
+    _reset(o, m)
+    n, path, out = o.typical_accept_compact(tok, logits, 0.7, 1.0, 1.0 - 1e-12, u=[0.37])   # threshold ~ exp(-H) <= max p: mixed
+    best = [x for x in path[0].tolist() if x >= 0][-1]
+    want = inverse_cdf(torch.softmax(logits[0, best] / 0.7, dim=0), 0.37)
+    assert o.root_tok[0] == want == out[0].tolist()[int(n[0])]
