@@ -58,12 +58,12 @@ __device__ __forceinline__ uint32_t peer_smem(uint32_t saddr, uint32_t rank) {  
 }
 __device__ __forceinline__ float4 ld_peer4(uint32_t addr) {
   float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ float2 ld_peer2(uint32_t addr) {
   float2 v;
-  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ float ex2(float x) {
@@ -83,6 +83,8 @@ struct AttArgs {
   int H, max_seq, nchunks;
   int* status;
   uint32_t wait_limit;
+  int early;                           // the lengths (rs.pos0, rs.n_rows) and the committed cache rows were written by kernels that
+                                       // completed before the preceding kernel started (see tree_attention_tc)
 };
 
 template <int HD, int QROWS, int NP> struct AttCfg {
@@ -96,11 +98,14 @@ template <int HD, int QROWS, int NP> struct AttCfg {
   static constexpr int V_BYTES = NP * NHALF * TILE * 128;     // a V tile: [plane][half][key][128 bytes] (N blocks of 64 output columns)
   static constexpr int STAGE_BYTES = K_BYTES + V_BYTES;
   static constexpr int NST = NP == 1 ? 3 : (HD == 64 ? 3 : 2);        // ring stages
+  // MMA M is 128 whatever QROWS is: with 64 query rows the upper 64 accumulator lanes are unused (M = 64 instructions
+  // measured slower per instruction), and the operand reads of a 64-row Q or P tile run 8 KB past the tile, into the next
+  // piece of Q, of P or of the ring (never read back), so the order Q, P0, P1, ring keeps them inside the allocation.
+  static constexpr int MROWS = 128;
+  static constexpr int RPW = MROWS / 4;                       // accumulator rows (tensor-memory lanes) per softmax warp
   static constexpr int RING_BYTES = NST * STAGE_BYTES;
   static constexpr int MERGE_BYTES = QROWS * HD * 4 + QROWS * 8;     // a chunk's partial rows + (max, sum); aliases the ring
   static constexpr int NBAR = 1 + 3 * NST + 8;
-  // The M = 128 operand reads of a 64-row Q or P tile run 8 KB past the tile, into the next piece of Q, of P or of the
-  // ring (unused lanes, never read back), so the order Q, P0, P1, ring keeps them inside the allocation.
   static constexpr int SMEM_BYTES = 1024 + Q_BYTES + 2 * P_BYTES + (RING_BYTES > MERGE_BYTES ? RING_BYTES : MERGE_BYTES) + NBAR * 8 + 16;
   static constexpr int S_COLS = NP * TILE;                    // one score buffer: [Q_hi K_hi + Q_lo K_hi | Q_hi K_lo]
   static constexpr int O_COLS = NP * HD;                      // the output accumulator: [P_hi V_hi + P_lo V_hi | P_hi V_lo]
@@ -131,6 +136,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   auto pv_done = [&](int i) { return bars + 8u * (1 + 3 * NST + 6 + i); };
   const uint32_t tmem_slot = bars + 8u * C::NBAR;
   __shared__ int s_abort;
+  __shared__ float s_w[128 * MAX_CHUNKS];               // normalised chunk weights of the rows this CTA merges
 
   const RowSet& rs = a.rs;
   const int h = blockIdx.x, b = blockIdx.y, c = blockIdx.z;
@@ -150,7 +156,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   __syncthreads();
   tc_fence_after();
   pdl_trigger();
-  pdl_wait();                                           // q and the new cache rows are the preceding kernel's output
+  // q and the new cache rows are the preceding kernel's output.  With a.early the lengths and the committed cache rows
+  // are known to be older than anything still in flight, so the producer requests committed tiles before it waits.
+  if (!a.early) pdl_wait();
   uint32_t tmem_base;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 
@@ -166,17 +174,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (warp == 0) {
     if (lane == 0 && has_work) {
       const uint64_t pol = policy_evict_first(), pol_q = policy_evict_last();
-      mbar_arrive_expect_tx(q_full, C::Q_BYTES);
-#pragma unroll
-      for (int pl = 0; pl < NP; ++pl)
-#pragma unroll
-        for (int hf = 0; hf < C::NHALF; ++hf)
-          tma_load_2d(q_s + pl * C::QP_BYTES + hf * QROWS * 128, &tmQ, h * HD + hf * 64, pl * a.q_plane_rows + b * rs.tc, q_full, pol_q);
       const int row0 = (b * H + h) * a.max_seq;
-      for (int i = 0; i < ntiles; ++i) {
+      auto request_tile = [&](int i) {
         const int s = i % NST;
-        // stage s was last read by the P V product of tile i - NST, the (i / NST - 1)-th completion of its empty barrier
-        if (i >= NST && !mbar_wait(kv_empty(s), (uint32_t)((i / NST - 1) & 1), limit)) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
         const uint32_t k_dst = ring_s + s * C::STAGE_BYTES, v_dst = k_dst + C::K_BYTES;
         const int r = row0 + (tile0 + i) * TILE;
         mbar_arrive_expect_tx(k_full(s), C::K_BYTES);
@@ -191,34 +191,50 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
           for (int hf = 0; hf < C::NHALF; ++hf)
             tma_load_2d(v_dst + (pl * C::NHALF + hf) * TILE * 128, &tmV, hf * 64, pl * a.kv_plane_rows + r, v_full(s), pol);
+      };
+      int i = 0;
+      if (a.early) {
+        for (; i < ntiles && i < NST && (tile0 + i + 1) * TILE <= p0; ++i) request_tile(i);     // committed rows only
+        pdl_wait();
+      }
+      mbar_arrive_expect_tx(q_full, C::Q_BYTES);
+#pragma unroll
+      for (int pl = 0; pl < NP; ++pl)
+#pragma unroll
+        for (int hf = 0; hf < C::NHALF; ++hf)
+          tma_load_2d(q_s + pl * C::QP_BYTES + hf * QROWS * 128, &tmQ, h * HD + hf * 64, pl * a.q_plane_rows + b * rs.tc, q_full, pol_q);
+      for (; i < ntiles; ++i) {
+        // stage i % NST was last read by the P V product of tile i - NST, the (i / NST - 1)-th completion of its empty barrier
+        if (i >= NST && !mbar_wait(kv_empty(i % NST), (uint32_t)((i / NST - 1) & 1), limit)) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
+        request_tile(i);
       }
     }
   } else if (warp == 1) {
     if (lane == 0 && has_work) {
-      constexpr uint32_t idesc_s = instr_desc_f16(0, 128, NP * TILE, 0);      // Q_hi x [K_hi ; K_lo]
-      constexpr uint32_t idesc_s2 = instr_desc_f16(0, 128, TILE, 0);          // Q_lo x K_hi
-      constexpr uint32_t idesc_pv = instr_desc_f16(0, 128, NP * HD, 1);       // P_hi x [V_hi | V_lo]
-      constexpr uint32_t idesc_pv2 = instr_desc_f16(0, 128, HD, 1);           // P_lo x V_hi
+      constexpr uint32_t idesc_s = instr_desc_f16(0, C::MROWS, NP * TILE, 0);      // Q_hi x [K_hi ; K_lo]
+      constexpr uint32_t idesc_s2 = instr_desc_f16(0, C::MROWS, TILE, 0);          // Q_lo x K_hi
+      constexpr uint32_t idesc_pv = instr_desc_f16(0, C::MROWS, NP * HD, 1);       // P_hi x [V_hi | V_lo]
+      constexpr uint32_t idesc_pv2 = instr_desc_f16(0, C::MROWS, HD, 1);           // P_lo x V_hi
+      // operand descriptors: built once; a byte offset inside shared memory adds offset / 16 to the start-address field
+      const uint64_t q_desc = smem_desc_sw128(q_s), p_desc = smem_desc_sw128(p_s), k_desc = smem_desc_sw128(ring_s),
+                     v_desc = smem_desc_sw128_mn(ring_s + C::K_BYTES, TILE * 128);
       bool ok = mbar_wait(q_full, 0, limit);
       auto issue_s = [&](int i) {                        // S_i = Q K_i^T into score buffer i & 1
         const int s = i % NST;
         if (!mbar_wait(k_full(s), (uint32_t)((i / NST) & 1), limit)) return false;
         if (i >= 2 && !mbar_wait(s_empty(i & 1), (uint32_t)(((i >> 1) - 1) & 1), limit)) return false;
         tc_fence_after();
-        const uint32_t k_src = ring_s + s * C::STAGE_BYTES;
+        const uint64_t kd = k_desc + (uint64_t)((s * C::STAGE_BYTES) >> 4);
+        const uint32_t d_s = tmem_base + (uint32_t)((i & 1) * C::S_COLS);
 #pragma unroll
-        for (int kk = 0; kk < HD / 16; ++kk) {
-          const uint32_t qa = q_s + (kk >> 2) * QROWS * 128 + (kk & 3) * 32;
-          const uint32_t kb = k_src + (kk >> 2) * C::KH_BYTES + (kk & 3) * 32;
-          umma_f16(tmem_base + (uint32_t)((i & 1) * C::S_COLS), smem_desc_sw128(qa), smem_desc_sw128(kb), idesc_s, (uint32_t)(kk != 0));
-        }
+        for (int kk = 0; kk < HD / 16; ++kk)
+          umma_f16(d_s, q_desc + (uint64_t)(((kk >> 2) * QROWS * 128 + (kk & 3) * 32) >> 4),
+                   kd + (uint64_t)(((kk >> 2) * C::KH_BYTES + (kk & 3) * 32) >> 4), idesc_s, (uint32_t)(kk != 0));
         if (NP == 2) {
 #pragma unroll
-          for (int kk = 0; kk < HD / 16; ++kk) {
-            const uint32_t qa = q_s + C::QP_BYTES + (kk >> 2) * QROWS * 128 + (kk & 3) * 32;
-            const uint32_t kb = k_src + (kk >> 2) * C::KH_BYTES + (kk & 3) * 32;
-            umma_f16(tmem_base + (uint32_t)((i & 1) * C::S_COLS), smem_desc_sw128(qa), smem_desc_sw128(kb), idesc_s2, 1u);
-          }
+          for (int kk = 0; kk < HD / 16; ++kk)
+            umma_f16(d_s, q_desc + (uint64_t)((C::QP_BYTES + (kk >> 2) * QROWS * 128 + (kk & 3) * 32) >> 4),
+                     kd + (uint64_t)(((kk >> 2) * C::KH_BYTES + (kk & 3) * 32) >> 4), idesc_s2, 1u);
         }
         umma_commit(s_full(i & 1));
         return true;
@@ -231,17 +247,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (!mbar_wait(p_full(i & 1), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
         if (!mbar_wait(v_full(s), (uint32_t)((i / NST) & 1), limit)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t v_src = ring_s + s * C::STAGE_BYTES + C::K_BYTES;
-        const uint32_t p_src = p_s + (i & 1) * C::P_BYTES;
+        const uint64_t vd = v_desc + (uint64_t)((s * C::STAGE_BYTES) >> 4), pd = p_desc + (uint64_t)(((i & 1) * C::P_BYTES) >> 4);
+        const uint32_t d_o = tmem_base + (uint32_t)C::O_COL0;
 #pragma unroll
         for (int kk = 0; kk < TILE / 16; ++kk)
-          umma_f16(tmem_base + (uint32_t)C::O_COL0, smem_desc_sw128(p_src + kk * 32), smem_desc_sw128_mn(v_src + kk * 2048, TILE * 128), idesc_pv,
-                   (uint32_t)((i | kk) != 0));
+          umma_f16(d_o, pd + (uint64_t)((kk * 32) >> 4), vd + (uint64_t)((kk * 2048) >> 4), idesc_pv, (uint32_t)((i | kk) != 0));
         if (NP == 2) {
 #pragma unroll
           for (int kk = 0; kk < TILE / 16; ++kk)
-            umma_f16(tmem_base + (uint32_t)C::O_COL0, smem_desc_sw128(p_src + C::PP_BYTES + kk * 32), smem_desc_sw128_mn(v_src + kk * 2048, TILE * 128),
-                     idesc_pv2, 1u);
+            umma_f16(d_o, pd + (uint64_t)((C::PP_BYTES + kk * 32) >> 4), vd + (uint64_t)((kk * 2048) >> 4), idesc_pv2, 1u);
         }
         umma_commit(kv_empty(s));
         umma_commit(pv_done(i & 1));
@@ -249,10 +263,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
     }
   } else {
-    // ---- softmax warps: thread = query row (the tensor-memory lane it may read)
-    const int quad = warp & 3, row = quad * 32 + lane;
-    const bool warp_rows = quad * 32 < nr;                // any row of this warp in use
-    const bool row_live = row < nr;
+    // ---- softmax warps: thread = accumulator row = a tensor-memory lane of the warp's quadrant
+    const int quad = warp & 3, row = quad * C::RPW + lane;
+    const bool row_valid = row < QROWS;
+    const bool warp_rows = quad * C::RPW < nr;            // any row of this warp in use
+    const bool row_live = row_valid && row < nr;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const uint64_t mask = (row_live && rs.mask) ? rs.mask[row] : 0ull;
     const bool causal = rs.mask == nullptr;
@@ -260,7 +275,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const int st = tid - 64;                              // 0..127 among the softmax threads
-    for (int i = 0; i < ntiles && ok; ++i) {
+    for (int i = 0; i < ntiles; ++i) {
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }     // a wait that ran out in one lane ends the walk for the whole warp
       const int t0 = (tile0 + i) * TILE;
       if (!mbar_wait(s_full(i & 1), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
       tc_fence_after();
@@ -269,15 +285,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t s_addr = lane_addr + (uint32_t)((i & 1) * C::S_COLS);
         if (NP == 1) {
           tmem_ld64(s_addr, r);
-        } else {
+        } else {                                           // the two column halves of the score buffer in one round trip, added
+          uint32_t y[64];
+          tmem_ld64x2(s_addr, s_addr + (uint32_t)TILE, r, y);
 #pragma unroll
-          for (int c0 = 0; c0 < 64; c0 += 32) {            // the two column halves of the score buffer, added
-            uint32_t x[32], y[32];
-            tmem_ld32(s_addr + (uint32_t)c0, x);
-            tmem_ld32(s_addr + (uint32_t)(TILE + c0), y);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) r[c0 + j] = __float_as_uint(__uint_as_float(x[j]) + __uint_as_float(y[j]));
-          }
+          for (int j = 0; j < 64; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(y[j]));
         }
       }
       tc_fence_before();
@@ -285,18 +297,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (lane == 0) mbar_arrive(s_empty(i & 1));
       float alpha = 1.f;
       if (warp_rows) {
-        const bool need_mask = t0 + TILE > p0;             // the tile reaches into the new rows (or past the end)
+        // visibility word of this row for the tile's 64 keys (bit j: key t0 + j), built once per tile
+        uint64_t vis = row_live ? ~0ull : 0ull;
+        if (t0 + TILE > p0 && row_live) {                  // the tile reaches into the new rows (or past the end)
+          const int shift = t0 - p0;                       // new-slot index of the tile's first key; negative: it is a committed row
+          if (causal) {                                    // new slots 0..row: keys j <= row - shift
+            const int n = row - shift + 1;
+            vis = n >= 64 ? ~0ull : (n <= 0 ? 0ull : ((1ull << n) - 1ull));
+          } else if (shift >= 0) {
+            vis = shift < 64 ? mask >> shift : 0ull;
+          } else {
+            vis = (mask << (-shift)) | ((1ull << (-shift)) - 1ull);
+          }
+          const int nv = total - t0;                       // keys of the tile that exist
+          if (nv < 64) vis &= (1ull << nv) - 1ull;
+        }
         float mx = -INFINITY;
 #pragma unroll
         for (int j = 0; j < 64; ++j) {
-          float v = __uint_as_float(r[j]) * sc;
-          if (need_mask) {
-            const int key = t0 + j, rel = key - p0;
-            const bool vis = row_live && key < total && (rel < 0 || (causal ? rel <= row : (bool)((mask >> rel) & 1ull)));
-            v = vis ? v : -INFINITY;
-          } else if (!row_live) {
-            v = -INFINITY;
-          }
+          const float v = ((vis >> j) & 1ull) ? __uint_as_float(r[j]) * sc : -INFINITY;
           r[j] = __float_as_uint(v);
           mx = fmaxf(mx, v);
         }
@@ -336,7 +355,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           }
         }
         const uint32_t prow = p_s + (i & 1) * C::P_BYTES + (uint32_t)row * 128u;
-        if (row < QROWS) {
+        if (row_valid) {
 #pragma unroll
           for (int ch = 0; ch < 8; ++ch) {
             const uint32_t dst = prow + (uint32_t)((ch ^ (row & 7)) * 16);
@@ -377,75 +396,103 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       __syncwarp();
       if (lane == 0) mbar_arrive(p_full(i & 1));
     }
+    ok = __all_sync(0xffffffffu, ok);
     if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
     // ---- this chunk's partial rows -> shared memory (the ring is idle once the last P V has completed)
     if (ok && ntiles > 0 && !mbar_wait(pv_done((ntiles - 1) & 1), (uint32_t)(((ntiles - 1) >> 1) & 1), limit)) {
       ok = false; atomicOr(a.status, ST_TIMEOUT); s_abort = 1;
     }
+    ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
-    if (row < QROWS) {
+    {
       const uint32_t xo = ring_s + (uint32_t)row * (HD * 4), xml = ring_s + QROWS * HD * 4 + (uint32_t)row * 8;
       const bool have = ok && ntiles > 0 && row_live && m_ref != -INFINITY;
       if (ok && ntiles > 0 && warp_rows) {
 #pragma unroll 1
-        for (int c0 = 0; c0 < HD; c0 += 32) {
-          uint32_t o[32];
-          tmem_ld32(lane_addr + (uint32_t)(C::O_COL0 + c0), o);
+        for (int c0 = 0; c0 < HD; c0 += 64) {              // 64 output columns (both planes' halves) per tensor-memory round trip
+          uint32_t o[64];
           if (NP == 2) {
-            uint32_t o2[32];
-            tmem_ld32(lane_addr + (uint32_t)(C::O_COL0 + HD + c0), o2);
+            uint32_t o2[64];
+            tmem_ld64x2(lane_addr + (uint32_t)(C::O_COL0 + c0), lane_addr + (uint32_t)(C::O_COL0 + HD + c0), o, o2);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) + __uint_as_float(o2[j]));
+            for (int j = 0; j < 64; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) + __uint_as_float(o2[j]));
+          } else {
+            tmem_ld64(lane_addr + (uint32_t)(C::O_COL0 + c0), o);
           }
+          if (row_valid) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {                    // float4 piece k4 of row i sits at position k4 ^ (i & (HD/4 - 1))
-            const int k4 = c0 / 4 + j;
-            const uint32_t dst = xo + (uint32_t)((k4 ^ (row & (HD / 4 - 1))) * 16);
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(o[4 * j]), "r"(o[4 * j + 1]), "r"(o[4 * j + 2]), "r"(o[4 * j + 3]) : "memory");
+            for (int j = 0; j < 16; ++j) {                 // float4 piece k4 of row i sits at position k4 ^ (i & (HD/4 - 1))
+              const int k4 = c0 / 4 + j;
+              const uint32_t dst = xo + (uint32_t)((k4 ^ (row & (HD / 4 - 1))) * 16);
+              asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(o[4 * j]), "r"(o[4 * j + 1]), "r"(o[4 * j + 2]), "r"(o[4 * j + 3]) : "memory");
+            }
           }
         }
       }
-      const float2 ml = have ? make_float2(m_ref, l) : make_float2(-INFINITY, 0.f);
-      asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(xml), "f"(ml.x), "f"(ml.y) : "memory");
+      if (row_valid) {
+        const float2 ml = have ? make_float2(m_ref, l) : make_float2(-INFINITY, 0.f);
+        asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(xml), "f"(ml.x), "f"(ml.y) : "memory");
+      }
     }
   }
+  __syncwarp();                                           // the one-lane roles rejoin their warps before the block-wide barrier
   tc_fence_before();
   __syncthreads();
   // ---- merge the chunks of this (head, sequence): out[r][h][:] = sum_c o_c 2^(m_c - M) / sum_c l_c 2^(m_c - M),
   // chunks in order; this CTA takes rows c, c + nchunks, ...
   cluster_sync_all();                                     // every chunk's rows are in its shared memory
+  if (a.early) pdl_wait();                                // (the producer lane has waited already) before the first global store
   {
     constexpr int V4 = HD / 4;
     const uint32_t xo_s = ring_s, xml_s = ring_s + QROWS * HD * 4;
     const int d = H * HD;
     const int rows_cap = min(rs.tc, QROWS);
     const int my_rows = rows_cap > c ? (rows_cap - c + nchunks - 1) / nchunks : 0;
-    for (int e = tid; e < my_rows * V4; e += 192) {
-      const int i = c + (e / V4) * nchunks, k4 = e % V4;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (i < nr) {
-        float mc[MAX_CHUNKS], lc[MAX_CHUNKS];
-        float M = -INFINITY;
+    // chunk weights of my rows, normalised: w_c = 2^(m_c - M) / sum_c l_c 2^(m_c - M)  (one thread per row, all (m, l) loads in flight together)
+    for (int t = tid; t < my_rows; t += 192) {
+      const int i = c + t * nchunks;
+      float mc[MAX_CHUNKS], lc[MAX_CHUNKS];
+      float M = -INFINITY, L = 0.f;
 #pragma unroll
-        for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
-          mc[cc] = -INFINITY; lc[cc] = 0.f;
-          if (cc < nchunks) { const float2 ml = ld_peer2(peer_smem(xml_s + (uint32_t)i * 8u, (uint32_t)cc)); mc[cc] = ml.x; lc[cc] = ml.y; }
-          M = fmaxf(M, mc[cc]);
-        }
-        float L = 0.f;
-#pragma unroll
-        for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
-          if (cc < nchunks && mc[cc] != -INFINITY) {
-            const float w = exp2f(mc[cc] - M);
-            const float4 v = ld_peer4(peer_smem(xo_s + (uint32_t)(i * HD * 4 + ((k4 ^ (i & (V4 - 1))) * 16)), (uint32_t)cc));
-            L += lc[cc] * w;
-            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
-          }
-        }
-        const float inv = L > 0.f ? 1.f / L : 0.f;
-        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+      for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
+        mc[cc] = -INFINITY; lc[cc] = 0.f;
+        if (cc < nchunks && i < nr) { const float2 ml = ld_peer2(peer_smem(xml_s + (uint32_t)i * 8u, (uint32_t)cc)); mc[cc] = ml.x; lc[cc] = ml.y; }
       }
-      if (!s_abort) {
+#pragma unroll
+      for (int cc = 0; cc < MAX_CHUNKS; ++cc) M = fmaxf(M, mc[cc]);
+#pragma unroll
+      for (int cc = 0; cc < MAX_CHUNKS; ++cc) { mc[cc] = mc[cc] == -INFINITY ? 0.f : exp2f(mc[cc] - M); L += lc[cc] * mc[cc]; }
+      const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+      for (int cc = 0; cc < MAX_CHUNKS; ++cc) s_w[t * MAX_CHUNKS + cc] = mc[cc] * inv;
+    }
+    __syncthreads();
+    // two output pieces per thread and round, all their peer loads in flight together (a load that waits for the
+    // previous one's use costs a shared-memory round trip across the cluster each)
+    for (int e0 = tid; e0 < my_rows * V4; e0 += 2 * 192) {
+      float4 v[2][MAX_CHUNKS];
+      float w[2][MAX_CHUNKS];
+#pragma unroll
+      for (int ib = 0; ib < 2; ++ib) {
+        const int e = e0 + ib * 192, t = e / V4, i = c + t * nchunks, k4 = e % V4;
+        const bool live = e < my_rows * V4;
+#pragma unroll
+        for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
+          w[ib][cc] = live && cc < nchunks ? s_w[t * MAX_CHUNKS + cc] : 0.f;
+          v[ib][cc] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (w[ib][cc] != 0.f)                              // a chunk of weight zero may hold nothing at all
+            v[ib][cc] = ld_peer4(peer_smem(xo_s + (uint32_t)(i * HD * 4 + ((k4 ^ (i & (V4 - 1))) * 16)), (uint32_t)cc));
+        }
+      }
+#pragma unroll
+      for (int ib = 0; ib < 2; ++ib) {
+        const int e = e0 + ib * 192, t = e / V4, i = c + t * nchunks, k4 = e % V4;
+        if (e >= my_rows * V4 || s_abort) continue;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
+          acc.x += v[ib][cc].x * w[ib][cc]; acc.y += v[ib][cc].y * w[ib][cc]; acc.z += v[ib][cc].z * w[ib][cc]; acc.w += v[ib][cc].w * w[ib][cc];
+        }
         bf16* dst = a.out + ((size_t)b * rs.tc + i) * d + h * HD + k4 * 4;      // rows past nr get zeros
         const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x, acc.y), h1 = __floats2bfloat162_rn(acc.z, acc.w);
         *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
@@ -483,7 +530,7 @@ int pick_chunks(int pairs, int len_upper, int sms) {
 
 template <int HD, int QROWS, int NP>
 hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out, size_t out_ps,
-                 int H, int max_seq, int len_upper, int* status, cudaStream_t st) {
+                 int H, int max_seq, int len_upper, int* status, bool stable_lengths, cudaStream_t st) {
   using C = AttCfg<HD, QROWS, NP>;
   CUtensorMap tq, tk, tv;
   const uint64_t cache_rows = (uint64_t)cache_batch * H * max_seq;
@@ -500,7 +547,7 @@ hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc
   }
   AttArgs a{};
   a.rs = rs; a.out = out; a.out_ps = out_ps; a.H = H; a.max_seq = max_seq; a.status = status; a.wait_limit = WAIT_LIMIT;
-  a.q_plane_rows = q_rows; a.kv_plane_rows = (int)cache_rows;
+  a.q_plane_rows = q_rows; a.kv_plane_rows = (int)cache_rows; a.early = stable_lengths ? 1 : 0;
   a.nchunks = pick_chunks(H * rs.batch, len_upper, sm_count());
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(H, rs.batch, a.nchunks); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = C::SMEM_BYTES; cfg.stream = st;
@@ -517,25 +564,26 @@ hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc
 
 template <int NP>
 hydra_status dispatch(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out, size_t out_ps,
-                      int H, int hd, int max_seq, int len_upper, int* status, cudaStream_t st) {
+                      int H, int hd, int max_seq, int len_upper, int* status, bool stable_lengths, cudaStream_t st) {
   const bool wide = rs.tc > 64;
   if (hd == 128 && wide && NP == 2) return HYDRA_ERR_UNSUPPORTED;       // Q, P and a two-stage ring of two planes exceed the shared memory of an SM
-  if (hd == 128) return wide ? run<128, 128, 1>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st)
-                             : run<128, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st);
-  if (hd == 64) return wide ? run<64, 128, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st)
-                            : run<64, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, st);
+  if (hd == 128) return wide ? run<128, 128, 1>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, st)
+                             : run<128, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, st);
+  if (hd == 64) return wide ? run<64, 128, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, st)
+                            : run<64, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, st);
   return HYDRA_ERR_UNSUPPORTED;
 }
 
 }  // namespace
 
 hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, int planes, RowSet rs,
-                               bf16* out, size_t out_ps, int H, int hd, int max_seq, int len_upper, int* status, cudaStream_t st) {
+                               bf16* out, size_t out_ps, int H, int hd, int max_seq, int len_upper, int* status, bool stable_lengths,
+                               cudaStream_t st) {
   if (rs.tc > 128 || (rs.mask && rs.tc > 64) || (planes != 1 && planes != 2)) return HYDRA_ERR_UNSUPPORTED;
   if (!tensor_map_encoder_available()) { set_last_error("cuTensorMapEncodeTiled entry point", cudaErrorUnknown); return HYDRA_ERR_CUDA; }
   if (((uintptr_t)q | (uintptr_t)kc | (uintptr_t)vc) & 15) return HYDRA_ERR_INVALID;
-  return planes == 2 ? dispatch<2>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, hd, max_seq, len_upper, status, st)
-                     : dispatch<1>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, hd, max_seq, len_upper, status, st);
+  return planes == 2 ? dispatch<2>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, hd, max_seq, len_upper, status, stable_lengths, st)
+                     : dispatch<1>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, hd, max_seq, len_upper, status, stable_lengths, st);
 }
 
 }  // namespace hydra

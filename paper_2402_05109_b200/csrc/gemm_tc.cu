@@ -312,6 +312,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       ++seg;
     }
   }
+  __syncwarp();                                          // the one-lane roles rejoin their warps before the block-wide barrier
   tc_fence_before();
   __syncthreads();
   if (s_abort) {                                         // let copies in flight land before the CTA retires

@@ -252,7 +252,8 @@ hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void*
 size_t ps(const hydra_ctx* c, int rows_alloc, size_t cols) { return c->planes == 2 ? (size_t)rows_alloc * cols : 0; }
 
 // RoPE + KV append + tree attention of one layer from the QKV partial sums (*sd) in c->part; result in c->attn_out.
-hydra_status attention_block(hydra_ctx* c, char* kc, char* vc, const RowSet& rs, int len_upper, const SplitDesc& sd, cudaStream_t st) {
+hydra_status attention_block(hydra_ctx* c, char* kc, char* vc, const RowSet& rs, int len_upper, const SplitDesc& sd, bool stable_lengths,
+                             cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int d = m.d_model, dt = m.dtype;
   const size_t q_ps = c->kv_planes == 2 ? (size_t)c->R * d : 0, kv_ps = c->kv_planes == 2 ? kv_layer_elems(m) : 0;
@@ -262,7 +263,7 @@ hydra_status attention_block(hydra_ctx* c, char* kc, char* vc, const RowSet& rs,
     return tree_attention_f32((const float*)c->q, (const float*)kc, (const float*)vc, rs, (float*)c->attn_out, c->att_scratch, m.n_heads,
                               m.head_dim, m.max_seq, len_upper, st);
   return tree_attention_tc((const __half*)c->q, c->R, (const __half*)kc, (const __half*)vc, m.max_batch, c->kv_planes, rs, (bf16*)c->attn_out,
-                           ps(c, c->R, d), m.n_heads, m.head_dim, m.max_seq, len_upper, c->d_status, st);
+                           ps(c, c->R, d), m.n_heads, m.head_dim, m.max_seq, len_upper, c->d_status, stable_lengths, st);
 }
 
 double gemm_bytes(const hydra_ctx* c, int m, int n, int k) {        // weights + activation slab read once, output written once
@@ -290,7 +291,7 @@ hydra_status mlp_block(hydra_ctx* c, const LayerW& w, int rows, const void* next
 // Base model over the rows of `rs` whose tokens are tok[rows]: leaves post-final-norm hidden rows in c->h_tree
 // (float) and c->xn (operand type); with tail_w also the partial sums of xn @ tail_w^T (the LM head) in c->part (*tail_sd).
 hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_upper, const void* tail_w, int tail_n, SplitDesc* tail_sd,
-                      cudaStream_t st) {
+                      bool stable_lengths, cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
   const int rows = rs.batch * rs.tc, d = m.d_model;
   const size_t kvl = kv_layer_elems(m) * c->kv_esize * c->kv_planes;      // bytes of one layer's K (or V) cache, all planes
@@ -301,7 +302,7 @@ hydra_status run_base(hydra_ctx* c, const int* tok, const RowSet& rs, int len_up
   HYDRA_TRY(run_gemm(c, c->xn, c->R, c->layers[0].wqkv, rows, 3 * d, d, &sd, st));
   for (int l = 0; l < m.n_layers; ++l) {
     const bool last = l + 1 == m.n_layers;
-    HYDRA_TRY(attention_block(c, c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs, len_upper, sd, st));
+    HYDRA_TRY(attention_block(c, c->kv_base + (size_t)(2 * l) * kvl, c->kv_base + (size_t)(2 * l + 1) * kvl, rs, len_upper, sd, stable_lengths, st));
     HYDRA_TRY(mlp_block(c, c->layers[l], rows, last ? c->final_norm : c->layers[l + 1].attn_norm, last ? c->h_tree : nullptr,
                         last ? tail_w : c->layers[l + 1].wqkv, last ? tail_n : 3 * d, last ? tail_sd : &sd, st));
   }
@@ -317,7 +318,7 @@ hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int le
   HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, m.dtype, st));
   SplitDesc sd;
   HYDRA_TRY(run_gemm(c, c->xn, c->R, c->pfx.wqkv, rows, 3 * d, d, &sd, st));
-  HYDRA_TRY(attention_block(c, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, sd, st));
+  HYDRA_TRY(attention_block(c, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, sd, false, st));
   return mlp_block(c, c->pfx, rows, nullptr, nullptr, nullptr, 0, nullptr, st);
 }
 
@@ -367,7 +368,9 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
   const int rows = c->batch * c->T;
   RowSet rs{c->batch, c->T, nullptr, c->d_len, c->d_depth, c->d_anc};
   SplitDesc sd;
-  HYDRA_TRY(run_base(c, tree_tok, rs, len_bucket(c, max_len_ub(c) + c->T), c->lm_head, m.vocab, &sd, st));
+  // the lengths a verification reads date from the previous step's acceptance kernel (or the prompt pass), and the
+  // committed cache rows are older still: its attention kernels may fetch committed tiles ahead of their predecessor
+  HYDRA_TRY(run_base(c, tree_tok, rs, len_bucket(c, max_len_ub(c) + c->T), c->lm_head, m.vocab, &sd, true, st));
   return argmax_rows(c->part, sd, logits, amax, c->topk_scratch, c->topk_rows_cap, rows, m.vocab, st);
 }
 
@@ -517,7 +520,7 @@ hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const
   for (int ch = 0; ch < nchunks; ++ch) {
     HYDRA_TRY(set_chunk(c->d_prompt_len, ch, CHUNK, c->d_pos0, c->d_nrows, batch, st));
     HYDRA_TRY(gather_chunk_tokens(tokens, c->d_offsets, ch, CHUNK, c->d_tok, batch, st));
-    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * CHUNK, nullptr, 0, nullptr, st));
+    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * CHUNK, nullptr, 0, nullptr, false, st));
     HYDRA_TRY(capture_last(c->h_tree, c->d_prompt_len, ch, CHUNK, c->h_new, c->h.n_heads + 1, c->d_n_new, c->d_len, batch, m.d_model, st));
     if (c->h.prefix_attn) HYDRA_TRY(run_prefix(c, c->h_tree, rs, (ch + 1) * CHUNK, st));
   }
@@ -771,7 +774,8 @@ hydra_status hydra_tree_attention(const void* q, const void* kc, const void* vc,
   if (!status || (out_planes != 1 && out_planes != 2) || (planes != 1 && planes != 2)) return HYDRA_ERR_INVALID;
   const size_t d = (size_t)n_heads * head_dim;
   return tree_attention_tc((const __half*)q, batch * tc, (const __half*)kc, (const __half*)vc, batch, planes, rs, (bf16*)out,
-                           out_planes == 2 ? (size_t)batch * tc * d : 0, n_heads, head_dim, max_seq, max_seq, status, (cudaStream_t)stream);
+                           out_planes == 2 ? (size_t)batch * tc * d : 0, n_heads, head_dim, max_seq, max_seq, status, false,
+                           (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -44,9 +44,12 @@ hydra_status tree_attention_f32(const float* q, const float* kcache, const float
 // [planes][cache_batch][H][max_seq][hd] are float16 in 1 or 2 planes (hi = f16(v), lo = f16(v - hi)); out is bfloat16
 // [rows][H*hd] in two planes out_ps elements apart (0: hi only).  rs.mask == null selects a causal chunk (row i sees
 // the committed slots and new slots 0..i) of up to 128 rows (one plane, or head_dim 64); with a mask, up to 64 rows.
+// stable_lengths: rs.pos0 / rs.n_rows and every cache row below pos0 were written by kernels that had COMPLETED before the
+// kernel preceding this one in the stream started (true for the layers of a verification: the lengths date from the
+// previous step); the kernel then requests committed cache tiles before it waits for its predecessor.
 hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, int planes, RowSet rs,
                                bf16* out, size_t out_ps, int n_heads, int head_dim, int max_seq, int len_upper, int* status,
-                               cudaStream_t st);
+                               bool stable_lengths, cudaStream_t st);
 hydra_status silu_mul(const float* part, SplitDesc sd, void* act, size_t act_ps, int rows, int f, int dtype,
                       cudaStream_t st);
 // amax[r] = argmax_v of the summed partial logits (lowest id among equal maxima); the sums go to logits_out if given
