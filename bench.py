@@ -225,6 +225,117 @@ def oracle_timed(cfg, weights, parent, warmup, steps, threads):
                  "to %d layers; %.2f s per step" % (min(3, cfg.model.n_layers), cfg.model.n_layers, sec))
 
 
+DRAFT_VARIANTS = {          # comparison workloads: which draft model populates the tree (the base model is the workload's)
+    "hydrapp": dict(n_mlp_layers=4, prefix_attn=True, medusa=False),     # Hydra++: 4-layer heads + the extra decoder layer
+    "hydra": dict(n_mlp_layers=1, prefix_attn=False, medusa=False),      # Hydra: single-hidden-layer heads over [h ; embeddings]
+    "medusa": dict(n_mlp_layers=1, prefix_attn=False, medusa=True),      # Medusa: sequentially independent heads over h
+}
+
+
+def variant_head(cfg, name):
+    from synth.configs import HeadCfg
+    v = DRAFT_VARIANTS[name]
+    return HeadCfg(cfg.head.n_heads, v["n_mlp_layers"], v["prefix_attn"], cfg.head.has_bias, v["medusa"])
+
+
+def variant_weights(cfg, head, base):
+    """The workload's base-model tensors (shared) plus this variant's head / prefix-layer tensors."""
+    from synth.weights import weight_names
+    names = [n for n in weight_names(cfg.model, head) if n not in base]
+    w = dict(base)
+    w.update(make_weights(cfg.model, head, cfg.seed, device="cuda", names=names))
+    return {n: w[n] for n in weight_names(cfg.model, head)}
+
+
+def quick_times(Hydra, model, head, parent, weights, prompts, warmup, steps):
+    """Step and phase times (ms, medians over `steps` steps after `warmup`) of one engine configuration, no planting:
+    whole steps through hydra_step (graph replay), then the phases through the split calls."""
+    B, K, T = len(prompts), head.n_heads, len(parent)
+    max_seq = max(p.numel() for p in prompts) + (2 * (warmup + steps) + 2) * (K + 1) + T + 8
+    g = Hydra(model, head, parent, weights, B, max_seq)
+    stream = torch.cuda.current_stream()
+    g.prefill(prompts)
+    nacc = torch.empty(B, dtype=torch.int32, device="cuda")
+    out = torch.empty(B, K + 1, dtype=torch.int32, device="cuda")
+    for _ in range(warmup):
+        g.step(nacc, out)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        g.step(nacc, out)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    step_ms = e0.elapsed_time(e1) / steps
+    ph = {"draft": [], "verify": [], "accept": []}
+    for _ in range(steps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        ev[0].record(stream)
+        tok = g.draft()
+        ev[1].record(stream)
+        amax = g.verify(tok)
+        ev[2].record(stream)
+        g.accept_compact(tok, amax)
+        ev[3].record(stream)
+        torch.cuda.synchronize()
+        for k, name in enumerate(("draft", "verify", "accept")):
+            ph[name].append(ev[k].elapsed_time(ev[k + 1]))
+    g.poll_status()
+    g.close()
+    med = lambda v: sorted(v)[len(v) // 2]
+    return {"step_ms": step_ms, "draft_ms": med(ph["draft"]), "verify_ms": med(ph["verify"]), "accept_ms": med(ph["accept"])}
+
+
+def overhead_table(args, cfg, parent):
+    """The shape of the paper's draft-overhead table (Appendix "Analysis of Hydra Head overheads") on this GPU: per-step
+    time of plain autoregressive decoding (root-only tree), and the drafting overhead of Medusa, Hydra and Hydra++ heads
+    on the same base model and tree.  Timing only: the heads are random, so acceptance is not measured here."""
+    from paper_2402_05109_b200 import Hydra
+    torch.cuda.set_device(0)
+    torch.cuda.set_stream(torch.cuda.Stream())
+    base_head = variant_head(cfg, "medusa")
+    base = {k: v for k, v in make_weights(cfg.model, base_head, cfg.seed, device="cuda").items() if not k.startswith(("H", "P."))}
+    prompts = make_prompts(cfg.seed, cfg.prompt_lens, cfg.model.vocab)
+    rows = []
+    ar = quick_times(Hydra, cfg.model, base_head, [-1], variant_weights(cfg, base_head, base), prompts, args.warmup, args.steps)
+    rows.append(dict(draft="none (autoregressive, root-only tree)", tree_rows=1, **ar))
+    for name in ("medusa", "hydra", "hydrapp"):
+        head = variant_head(cfg, name)
+        r = quick_times(Hydra, cfg.model, head, parent, variant_weights(cfg, head, base), prompts, args.warmup, args.steps)
+        r["draft_share_of_step"] = r["draft_ms"] / r["step_ms"]
+        r["step_vs_autoregressive_step"] = r["step_ms"] / ar["step_ms"]
+        rows.append(dict(draft=name, tree_rows=len(parent), **r))
+    print(json.dumps({"table": "draft overhead per decoding step", "workload": workload_name(cfg, parent), "steps": args.steps,
+                      "warmup": args.warmup, "rows": rows}))
+
+
+def tree_sweep(args, cfg):
+    """Tree discovery against measured latency (Section "Discovering performant decoding trees"): grow T_1 .. T_63 greedily
+    under the synthetic acceptance model, time whole steps of the engine for a set of sizes and batch sizes, and report
+    for every batch size the size with the best emitted-tokens/s = B (1 + E[accepted]) / t_step."""
+    from paper_2402_05109_b200 import Hydra
+    from paper_2402_05109_b200.tree_search import grow_trees, to_parent_list, expected_accept_length, pick_tree_size
+    from synth import ALPHA, BETA
+    torch.cuda.set_device(0)
+    torch.cuda.set_stream(torch.cuda.Stream())
+    rank_prob = lambda depth, r: ALPHA[depth - 1] * (1.0 - BETA) * BETA ** r
+    trees = grow_trees(63, cfg.head.n_heads, rank_prob)
+    sizes = [0, 3, 7, 15, 31, 47, 63]
+    parents = {n: ([-1] if n == 0 else to_parent_list(trees[n - 1])) for n in sizes}
+    elen = {n: (0.0 if n == 0 else expected_accept_length(parents[n], rank_prob)) for n in sizes}
+    weights = make_weights(cfg.model, cfg.head, cfg.seed, device="cuda")
+    out = []
+    for B in (1, 2, 4, 8):
+        lens = get_config("c3b%d" % B).prompt_lens
+        prompts = make_prompts(cfg.seed, lens, cfg.model.vocab)
+        t = {n: quick_times(Hydra, cfg.model, cfg.head, parents[n], weights, prompts, args.warmup, args.steps)["step_ms"] for n in sizes}
+        best, tps = pick_tree_size(sizes, lambda n: elen[n], lambda n: t[n] * 1e-3, B)
+        out.append({"batch": B, "prompt_lens": lens, "best_candidates": best,
+                    "sizes": [{"candidates": n, "expected_accepted": elen[n], "step_ms": t[n], "emitted_tokens_per_s": tps[n]} for n in sizes]})
+    print(json.dumps({"table": "tree size against measured step latency", "acceptance_model": "synthetic: alpha %s, beta %s" % (list(ALPHA), BETA),
+                      "model": "%d-layer d=%d" % (cfg.model.n_layers, cfg.model.d_model), "steps": args.steps, "warmup": args.warmup,
+                      "rows": out}))
+
+
 def max_over_ranks(value, dist, device):
     """Slowest rank's time: what a replica job's wall clock is.  `dist` is torch.distributed (initialised) or None."""
     if dist is None:
@@ -278,6 +389,8 @@ def main():
     ap.add_argument("--gemm-mode", type=int, default=0, help="0 tcgen05 (default), 1 SIMT")
     ap.add_argument("--blocks", type=int, default=5, help="timed blocks of --steps steps each; the median block is reported")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel of a step separately (profilers' launch lists)")
+    ap.add_argument("--overhead-table", action="store_true", help="autoregressive / Medusa / Hydra / Hydra++ step and draft times on the workload's model")
+    ap.add_argument("--tree-sweep", action="store_true", help="tree size x batch size sweep against measured step latency")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -285,6 +398,10 @@ def main():
     parent = load_tree(cfg.tree)
     if args.impl == "reference":
         return run_reference(args, cfg, parent)
+    if args.overhead_table:
+        return overhead_table(args, cfg, parent)
+    if args.tree_sweep:
+        return tree_sweep(args, cfg)
 
     from paper_2402_05109_b200 import Hydra           # raises if libhydra.so is missing: no fallback
     rank = int(os.environ.get("RANK", "0"))
@@ -400,7 +517,8 @@ def main():
     t_draft, t_verify, t_accept = med(ph["draft"]), med(ph["verify"]), med(ph["accept"])
     mean_lens = [sum(l[b] for l in lens_mid) / len(lens_mid) for b in range(B)]
     vbytes = verify_bytes(m, B, T, mean_lens)                 # the method's bytes: one cache element = one weight element
-    vbytes_read = verify_bytes(m, B, T, mean_lens, skv=4)     # what this library's two-plane (or float) cache really moves
+    skv_lib = 4 if m.dtype == "fp32" else 2 * g.kv_planes      # float, or float16 in kv_planes planes
+    vbytes_read = verify_bytes(m, B, T, mean_lens, skv=skv_lib)     # what this library's cache format really moves
     dbytes = draft_bytes(m, h, mean_lens)
     hbm_peak, peak_kind = peaks()
     verify_gbs = vbytes / (t_verify * 1e-3) / 1e9

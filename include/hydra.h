@@ -72,6 +72,9 @@ typedef struct {
   int n_mlp_layers;  /* m >= 1 */
   int prefix_attn;   /* 0 | 1 */
   int has_bias;      /* 0 | 1 */
+  int medusa;        /* 0: Hydra heads (sequentially dependent).  1: sequentially independent heads, the Medusa baseline
+                        (Background, "Lightweight heads as a draft model" / "Medusa decoding"): head i sees the hidden state
+                        only, head_w1[i-1] is [d][d], and every parent of a tree level gets the same children */
 } hydra_head_cfg;
 
 /* Static candidate tree (Background, "Tree decoding").  parent is a HOST array of n_rows entries:
@@ -148,6 +151,20 @@ hydra_status hydra_step(hydra_ctx*, int32_t* n_acc_dev, int32_t* out_tok_dev, vo
 /* on = 0: hydra_step launches kernel by kernel (for profilers that list kernels); on = 1 (default): graph replay. */
 hydra_status hydra_set_step_graph(hydra_ctx*, int on);
 
+/* Acceptance criterion.  mode 0 (default): greedy, as described at hydra_accept_compact.  mode 1: typical acceptance
+ * (Section "Typical acceptance sampling", paragraph "Typical acceptance criterion"): with p = softmax(logits / tau) of the
+ * base model at a candidate's parent row and H the entropy of p, the candidate passes when
+ * p[token] > min(eps, alpha * exp(-H)) (eps: posterior threshold, alpha: posterior alpha; the paper uses tau = 0.7,
+ * eps in 0.05..0.25, alpha = sqrt(eps)); it is accepted when it passes and its parent is accepted; the deepest accepted
+ * row wins, lowest row among equals, and the cache is compacted as in the greedy case.  The token after the accepted
+ * path is drawn from p at the best row by inverse CDF in token-id order with the uniform number u_dev[b] in [0, 1)
+ * (u_dev: DEVICE float [max_batch], read by every acceptance until replaced; the caller draws the numbers), or is that
+ * row's most likely token when u_dev is NULL.  In mode 1 hydra_verify also writes every row's logits (to logits_dev,
+ * or to a library buffer when that is NULL) and their softmax statistics, which hydra_accept_compact then reads; amax_dev
+ * is still needed (the most likely token).  Errors: INVALID (mode, tau <= 0, negative eps / alpha); STATE (changing the
+ * mode between a verification and its acceptance). */
+hydra_status hydra_set_acceptance(hydra_ctx*, int mode, float tau, float eps, float alpha, const float* u_dev);
+
 /* Accept-exercise mode: plant_dev [batch][n_rows], -1 keeps the drafted token; applied between draft
  * and verify inside hydra_step.  NULL disables.  The buffer is read at every step. */
 hydra_status hydra_set_plant(hydra_ctx*, const int32_t* plant_dev);
@@ -167,8 +184,10 @@ enum {
   HYDRA_BUF_HEAD_LOGITS = 9,/* float [rows][vocab] logits of the last drafted level, row = b*parents+j */
   HYDRA_BUF_N_NEW = 10,     /* int32 [max_batch] rows in H_NEW */
   HYDRA_BUF_H_PRIME = 11,   /* float [max_batch][d] hidden state the heads consumed */
-  HYDRA_BUF_STATUS = 12     /* int32 [64]: [0] the device status word (bit 1 bounds, bit 2 timeout) that hydra_poll_status
+  HYDRA_BUF_STATUS = 12,    /* int32 [64]: [0] the device status word (bit 1 bounds, bit 2 timeout) that hydra_poll_status
                                reads and clears, [8..15] where a bounded wait gave up (site, cta, unit, units, grid, m, n, k-blocks) */
+  HYDRA_BUF_PASS_BITS = 13  /* uint64 [max_batch]: bit i = candidate row i passed the acceptance criterion at its parent in the
+                               last hydra_accept_compact (greedy: equals the parent's argmax; typical: the inequality) */
 };
 hydra_status hydra_get_buffer(hydra_ctx*, int which, void** dev_ptr, size_t* bytes);
 

@@ -12,6 +12,8 @@ What it follows (Hydra: Sequentially-Dependent Draft Heads for Medusa Decoding):
   * Section "Hydra Heads", second displayed equation: head i is a function of the last hidden
     state, x_t and the i-1 tokens speculated before it, concatenated on the feature dimension.
   * Section "Hydra++": MLP depth 4 and one extra decoder layer queried once per step.
+  * Background, "Lightweight heads as a draft model" / "Medusa decoding": the baseline whose head i is a
+    function of the hidden state alone (head.medusa).
   * Background, verification criteria: greedy acceptance (a candidate is kept when it equals the
     base model's most likely token).
   * Section "Typical acceptance sampling", paragraph "Typical acceptance criterion": a candidate is
@@ -243,10 +245,11 @@ class HydraOracle:
 
     def head_logits(self, i: int, hprime: torch.Tensor, path_tok: Sequence[int]) -> torch.Tensor:
         """Hydra head i (1-based) at one parent: MLP over [h' ; E[x_t] ; E[x^_{t+1}] ...] then the
-        shared LM head.  path_tok = tokens on the path root..parent (i of them)."""
+        shared LM head.  path_tok = tokens on the path root..parent (i of them).  A sequentially
+        independent (Medusa) head sees h' alone, so all parents of a level get the same distribution."""
         assert len(path_tok) == i
         E = self.W("embed")
-        z = torch.cat([hprime] + [E[t] for t in path_tok])
+        z = hprime if getattr(self.h, "medusa", False) else torch.cat([hprime] + [E[t] for t in path_tok])
         y = hprime + silu(self.W(f"H{i}.w1") @ z + self.W(f"H{i}.b1"))
         for l in range(self.h.n_mlp_layers - 1):
             y = y + silu(self.W(f"H{i}.wr")[l] @ y + self.W(f"H{i}.br")[l])

@@ -22,7 +22,7 @@ class ModelCfgC(C.Structure):
 
 
 class HeadCfgC(C.Structure):
-    _fields_ = [(n, C.c_int) for n in ("n_heads", "n_mlp_layers", "prefix_attn", "has_bias")]
+    _fields_ = [(n, C.c_int) for n in ("n_heads", "n_mlp_layers", "prefix_attn", "has_bias", "medusa")]
 
 
 class TreeCfgC(C.Structure):
@@ -52,6 +52,7 @@ lib.hydra_verify.argtypes = [_vp, _vp, _vp, _vp, _vp]
 lib.hydra_accept_compact.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.hydra_step.argtypes = [_vp, _vp, _vp, _vp]
 lib.hydra_set_plant.argtypes = [_vp, _vp]
+lib.hydra_set_acceptance.argtypes = [_vp, _i, C.c_float, C.c_float, C.c_float, _vp]
 lib.hydra_get_buffer.argtypes = [_vp, _i, C.POINTER(_vp), C.POINTER(_sz)]
 lib.hydra_poll_status.argtypes = [_vp, _vp]
 lib.hydra_launch_count.restype = C.c_longlong
@@ -73,10 +74,10 @@ lib.hydra_attention_scratch_bytes.argtypes = [_i] * 5
 lib.hydra_tree_attention.argtypes = [_vp] * 8 + [_i] * 8 + [_vp, _vp]
 
 BUF = dict(LEN=0, ROOT_TOK=1, H_TREE=2, H_NEW=3, KV_BASE=4, KV_PREFIX=5, TREE_MASK=6, TREE_TOK=7, AMAX=8,
-           HEAD_LOGITS=9, N_NEW=10, H_PRIME=11, STATUS=12)
+           HEAD_LOGITS=9, N_NEW=10, H_PRIME=11, STATUS=12, PASS_BITS=13)
 _BUF_DTYPE = dict(LEN=torch.int32, ROOT_TOK=torch.int32, H_TREE=torch.float32, H_NEW=torch.float32,
                   TREE_MASK=torch.int64, TREE_TOK=torch.int32, AMAX=torch.int32, HEAD_LOGITS=torch.float32,
-                  N_NEW=torch.int32, H_PRIME=torch.float32, STATUS=torch.int32)
+                  N_NEW=torch.int32, H_PRIME=torch.float32, STATUS=torch.int32, PASS_BITS=torch.int64)
 
 
 def _check(code: int, what: str):
@@ -118,7 +119,8 @@ class Hydra:
                              model.rms_eps, model.rope_theta, 0 if model.dtype == "fp32" else 1, max_batch, max_seq,
                              int(getattr(model, "kv_planes", 2)))
         self.kv_planes = 1 if model.dtype == "fp32" else (1 if self._mc.kv_planes == 1 else 2)
-        self._hc = HeadCfgC(head.n_heads, head.n_mlp_layers, int(head.prefix_attn), int(head.has_bias))
+        self._hc = HeadCfgC(head.n_heads, head.n_mlp_layers, int(head.prefix_attn), int(head.has_bias),
+                            int(getattr(head, "medusa", False)))
         self._parent_arr = (C.c_int32 * self.T)(*self.parent)
         self._tc = TreeCfgC(self.T, self._parent_arr)
         nbytes = lib.hydra_workspace_bytes(C.byref(self._mc), C.byref(self._hc), C.byref(self._tc))
@@ -193,6 +195,16 @@ class Hydra:
     def set_plant(self, plant: Optional[torch.Tensor]):
         self._plant = plant
         _check(lib.hydra_set_plant(self._ctx, _ptr(plant)), "hydra_set_plant")
+
+    def set_acceptance(self, mode: int, tau: float = 1.0, eps: float = 0.0, alpha: float = 0.0,
+                       u: Optional[torch.Tensor] = None):
+        """hydra_set_acceptance: 0 greedy, 1 typical (tau, eps, alpha); u: float32 CUDA tensor [max_batch] of uniform
+        numbers for the token after the accepted path, or None (its most likely token)."""
+        if u is not None:
+            _dense_cuda(u, torch.float32, "u")
+            _need(u.numel() >= self.max_batch, "u [max_batch]")
+        self._u = u
+        _check(lib.hydra_set_acceptance(self._ctx, mode, tau, eps, alpha, _ptr(u)), "hydra_set_acceptance")
 
     def set_gemm_mode(self, mode: int):
         _check(lib.hydra_set_gemm_mode(self._ctx, mode), "hydra_set_gemm_mode")

@@ -65,6 +65,9 @@ struct hydra_ctx {
   std::vector<int*> d_level_parents;
   int *d_len, *d_n_new, *d_root_tok, *d_status, *d_pos0, *d_nrows, *d_prompt_len, *d_offsets, *d_tok, *d_tree_tok, *d_amax;
   unsigned int* d_done;
+  unsigned long long* d_pass_bits; int* d_bonus; float4* d_row_stats;
+  const float* last_logits;                      // logits of the last verification (the caller's buffer or c->logits)
+  int acc_mode; float acc_tau, acc_eps, acc_alpha; const float* acc_u;
   char *kv_base, *kv_pfx;
   float *x, *part, *h_tree, *logits, *h_new, *hprime, *y, *head_logits;
   float2* rope;
@@ -193,6 +196,8 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   auto* plen = b.take<int>(m.max_batch); auto* offs = b.take<int>(m.max_batch + 1);
   auto* tok = b.take<int>(R); auto* tree_tok = b.take<int>((size_t)m.max_batch * T); auto* amax = b.take<int>(R);
   auto* done = b.take<unsigned int>(m.max_batch);
+  auto* pass_bits = b.take<unsigned long long>(m.max_batch); auto* bonus = b.take<int>(m.max_batch);
+  auto* row_stats = b.take<float4>(R);
   auto* kvb = b.take<char>((size_t)m.n_layers * 2 * kvp * kv_layer_elems(m) * ces);
   auto* kvpfx = b.take<char>(h.prefix_attn ? (size_t)2 * kvp * kv_layer_elems(m) * ces : 0);
   auto* x = b.take<float>((size_t)R * d); auto* q = b.take<char>((size_t)kvp * R * d * ces);
@@ -215,6 +220,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
     c->d_chain_depth = chain_depth; c->d_anc = anc; c->d_chain_mask = chain_mask; c->d_level_parents = lvl;
     c->d_len = len; c->d_n_new = n_new; c->d_root_tok = root; c->d_status = status; c->d_pos0 = pos0; c->d_nrows = nrows;
     c->d_prompt_len = plen; c->d_offsets = offs; c->d_tok = tok; c->d_tree_tok = tree_tok; c->d_amax = amax; c->d_done = done;
+    c->d_pass_bits = pass_bits; c->d_bonus = bonus; c->d_row_stats = row_stats;
     c->kv_base = kvb; c->kv_pfx = kvpfx; c->x = x; c->q = q; c->part = part; c->h_tree = h_tree; c->logits = logits;
     c->h_new = h_new; c->hprime = hprime; c->y = y; c->head_logits = head_logits; c->rope = rope; c->xn = xn;
     c->attn_out = attn_out; c->act = act; c->z = z; c->yb = yb; c->att_scratch = att; c->topk_scratch = topk_s; c->topk_rows_cap = topk_cap;
@@ -339,26 +345,32 @@ hydra_status do_draft(hydra_ctx* c, int* tree_tok, cudaStream_t st) {
     HYDRA_TRY(pick_last_row(c->h_new, c->d_n_new, K + 1, c->hprime, B, d, st));
   }
   if (c->Ktree == 0) return copy_i32(tree_tok, c->d_root_tok, B, st);      // root-only tree (T == 1)
+  const bool medusa = c->h.medusa != 0;
   for (int lvl = 1; lvl <= c->Ktree; ++lvl) {
     const int P = (int)c->level_parents[lvl - 1].size();
-    const int rows = B * P;
+    // Hydra heads: one row per (sequence, parent), input [h' ; E of the path tokens].  Sequentially independent heads: one row
+    // per sequence, input h' alone (level 1's parent list, the root, stands in as a one-parent level for the gather)
+    const int rows = medusa ? B : B * P;
+    const int rows_per_b = medusa ? 1 : P;
+    const int in_blocks = medusa ? 1 : lvl + 1;
     LevelDesc lv{lvl, P, c->d_level_parents[lvl - 1]};
-    HYDRA_TRY(head_gather(c->hprime, c->embed, c->d_root_tok, tree_tok, c->d_path_tab, lv, c->z, ps(c, c->RH, (size_t)(lvl + 1) * d), B, c->T, K + 1, d, m.vocab, dt,
-                          c->d_status, st));
+    LevelDesc lv_in = medusa ? LevelDesc{0, 1, c->d_level_parents[0]} : lv;
+    HYDRA_TRY(head_gather(c->hprime, c->embed, c->d_root_tok, tree_tok, c->d_path_tab, lv_in, lvl == 1, c->z, ps(c, c->RH, (size_t)in_blocks * d), B, c->T,
+                          K + 1, d, m.vocab, dt, c->d_status, st));
     SplitDesc sd;
-    HYDRA_TRY(run_gemm(c, c->z, c->RH, c->head_w1[lvl - 1], rows, d, (lvl + 1) * d, &sd, st));
-    HYDRA_TRY(head_act(c->hprime, 1, P, c->part, sd, c->h.has_bias ? c->head_b1[lvl - 1] : nullptr, c->y, c->yb, ps(c, c->RH, d), rows, d, dt, st));
+    HYDRA_TRY(run_gemm(c, c->z, c->RH, c->head_w1[lvl - 1], rows, d, in_blocks * d, &sd, st));
+    HYDRA_TRY(head_act(c->hprime, 1, rows_per_b, c->part, sd, c->h.has_bias ? c->head_b1[lvl - 1] : nullptr, c->y, c->yb, ps(c, c->RH, d), rows, d, dt, st));
     for (int l = 0; l + 1 < c->h.n_mlp_layers; ++l) {
       const char* wr = (const char*)c->head_wr[lvl - 1] + (size_t)l * d * d * c->esize;
       const char* br = c->h.has_bias ? (const char*)c->head_br[lvl - 1] + (size_t)l * d * c->esize : nullptr;
       HYDRA_TRY(run_gemm(c, c->yb, c->RH, wr, rows, d, d, &sd, st));
-      HYDRA_TRY(head_act(c->y, 0, P, c->part, sd, br, c->y, c->yb, ps(c, c->RH, d), rows, d, dt, st));
+      HYDRA_TRY(head_act(c->y, 0, rows_per_b, c->part, sd, br, c->y, c->yb, ps(c, c->RH, d), rows, d, dt, st));
     }
     HYDRA_TRY(run_gemm(c, c->yb, c->RH, c->lm_head, rows, m.vocab, d, &sd, st));
     int max_children = 1;
     for (int p : c->level_parents[lvl - 1]) max_children = std::max(max_children, c->n_child[p]);
     HYDRA_TRY(topk_children(c->part, sd, c->head_logits, lv, max_children, c->d_first_child, c->d_n_child, tree_tok, c->topk_scratch,
-                            c->topk_rows_cap, B, c->T, m.vocab, st));
+                            c->topk_rows_cap, B, c->T, m.vocab, medusa ? 1 : 0, st));
   }
   return HYDRA_OK;
 }
@@ -371,7 +383,11 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
   // the lengths a verification reads date from the previous step's acceptance kernel (or the prompt pass), and the
   // committed cache rows are older still: its attention kernels may fetch committed tiles ahead of their predecessor
   HYDRA_TRY(run_base(c, tree_tok, rs, len_bucket(c, max_len_ub(c) + c->T), c->lm_head, m.vocab, &sd, true, st));
-  return argmax_rows(c->part, sd, logits, amax, c->topk_scratch, c->topk_rows_cap, rows, m.vocab, st);
+  if (c->acc_mode == 1 && !logits) logits = c->logits;              // the typical criterion reads whole rows of logits
+  c->last_logits = logits;
+  HYDRA_TRY(argmax_rows(c->part, sd, logits, amax, c->topk_scratch, c->topk_rows_cap, rows, m.vocab, st));
+  if (c->acc_mode == 1) HYDRA_TRY(softmax_row_stats(logits, c->d_row_stats, rows, m.vocab, c->acc_tau, st));
+  return HYDRA_OK;
 }
 
 hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* n_acc, int* path, int* out_tok, cudaStream_t st) {
@@ -383,6 +399,10 @@ hydra_status do_accept(hydra_ctx* c, const int* tree_tok, const int* amax, int* 
   a.kv_base = c->kv_base; a.h_tree = c->h_tree; a.h_tree_stride = c->T;
   a.h_new = c->h_new; a.n_new = c->d_n_new; a.len = c->d_len; a.root_tok = c->d_root_tok;
   a.n_acc = n_acc; a.path = path; a.out_tok = out_tok; a.done_counter = c->d_done; a.status = c->d_status;
+  a.mode = c->acc_mode; a.tau = c->acc_tau; a.eps = c->acc_eps; a.alpha = c->acc_alpha; a.logits = c->last_logits;
+  a.row_stats = c->d_row_stats; a.vocab = m.vocab; a.u = c->acc_mode == 1 ? c->acc_u : nullptr; a.pass_bits = c->d_pass_bits;
+  a.bonus_tmp = c->d_bonus;
+  if (a.mode == 1 && !a.logits) return HYDRA_ERR_STATE;
   {
     TimeScope ts(c, HYDRA_TIME_ACCEPT, 0.0, st);
     HYDRA_TRY(accept_compact(a, st));
@@ -464,6 +484,7 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
   carve(c, *m, *h, th, (char*)ws);
   c->batch = 0; c->state = ST_CREATED; c->gemm_mode = 0; c->plant = nullptr; c->launches = 0; c->timing = 0; c->steps_done = 0;
   c->use_graph = 1;
+  c->acc_mode = 0; c->acc_tau = 1.f; c->acc_eps = 0.f; c->acc_alpha = 0.f; c->acc_u = nullptr; c->last_logits = nullptr;
   c->len_ub.assign(m->max_batch, 0);
   // clear the workspace, upload the static tables
   auto fail = [&](cudaError_t e, const char* what) { set_last_error(what, e); delete c; return HYDRA_ERR_CUDA; };
@@ -611,6 +632,15 @@ hydra_status hydra_set_plant(hydra_ctx* c, const int32_t* plant) {
   return HYDRA_OK;
 }
 
+hydra_status hydra_set_acceptance(hydra_ctx* c, int mode, float tau, float eps, float alpha, const float* u_dev) {
+  if (!c || (mode != 0 && mode != 1)) return HYDRA_ERR_INVALID;
+  if (mode == 1 && !(tau > 0.f && eps >= 0.f && alpha >= 0.f)) return HYDRA_ERR_INVALID;
+  if (c->state == ST_VERIFIED && mode != c->acc_mode) return HYDRA_ERR_STATE;      // the last verification prepared for the other criterion
+  c->acc_mode = mode; c->acc_tau = tau; c->acc_eps = eps; c->acc_alpha = alpha; c->acc_u = mode == 1 ? u_dev : nullptr;
+  drop_graphs(c);
+  return HYDRA_OK;
+}
+
 hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes) {
   if (!c || !ptr) return HYDRA_ERR_INVALID;
   const hydra_model_cfg& m = c->m;
@@ -631,6 +661,7 @@ hydra_status hydra_get_buffer(hydra_ctx* c, int which, void** ptr, size_t* bytes
     case HYDRA_BUF_N_NEW: p = c->d_n_new; n = m.max_batch * sizeof(int); break;
     case HYDRA_BUF_H_PRIME: p = c->hprime; n = (size_t)m.max_batch * m.d_model * sizeof(float); break;
     case HYDRA_BUF_STATUS: p = c->d_status; n = 64 * sizeof(int); break;
+    case HYDRA_BUF_PASS_BITS: p = c->d_pass_bits; n = m.max_batch * sizeof(unsigned long long); break;
     default: return HYDRA_ERR_INVALID;
   }
   *ptr = p;

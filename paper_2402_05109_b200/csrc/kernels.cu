@@ -563,12 +563,13 @@ __global__ void __launch_bounds__(256) topk_stage1_kernel(const float* __restric
 // out_of(row) and count_of(row): where the winners go.  lv.parents == null: argmax (one winner per row to amax[row]).
 __global__ void __launch_bounds__(256) topk_stage2_kernel(const float* __restrict__ cand_v, const int* __restrict__ cand_i,
                                                           int nblk, int c, LevelDesc lv, const int* __restrict__ first_child,
-                                                          const int* __restrict__ n_child, int* __restrict__ out, int T) {
+                                                          const int* __restrict__ n_child, int* __restrict__ out, int T, int cand_div) {
   pdl_trigger();
   pdl_wait();
   __shared__ float shv[32];
   __shared__ int shi[32];
   const int row = blockIdx.x;
+  const int crow = row / cand_div;                         // row of the candidate lists (one per sequence when the parents share them)
   int* dst = out + row;
   int count = 1;
   if (lv.parents) {
@@ -580,7 +581,7 @@ __global__ void __launch_bounds__(256) topk_stage2_kernel(const float* __restric
   for (int t = 0; t < count; ++t) {
     float bv = -INFINITY; int bi = 0x7fffffff;
     for (int e = threadIdx.x; e < nblk * c; e += blockDim.x) {
-      const size_t at = ((size_t)row * nblk + e / c) * TOPK_MAX + e % c;
+      const size_t at = ((size_t)crow * nblk + e / c) * TOPK_MAX + e % c;
       const float v = cand_v[at]; const int i = cand_i[at];
       const bool after = v < pv || (v == pv && i > pi);          // strictly after the previous pick in the order
       if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
@@ -596,28 +597,31 @@ size_t topk_scratch_bytes(int rows, int vocab) {
   return (size_t)rows * nblk * TOPK_MAX * (sizeof(float) + sizeof(int));
 }
 
-static hydra_status topk_rows(const float* part, SplitDesc sd, float* logits_out, void* scratch, int rows_cap, int rows, int vocab,
+// rows: logits rows (stage 1); out_rows: winner lists (stage 2), out_rows / rows of them per logits row
+static hydra_status topk_rows(const float* part, SplitDesc sd, float* logits_out, void* scratch, int rows_cap, int rows, int out_rows, int vocab,
                               int c, LevelDesc lv, const int* first_child, const int* n_child, int* out, int T, cudaStream_t st) {
-  if (c < 1 || c > TOPK_MAX || rows > rows_cap) return HYDRA_ERR_UNSUPPORTED;
+  if (c < 1 || c > TOPK_MAX || rows > rows_cap || rows < 1 || out_rows % rows) return HYDRA_ERR_UNSUPPORTED;
   const int nblk = (vocab + TOPK_SPAN - 1) / TOPK_SPAN;
   float* cand_v = (float*)scratch;
   int* cand_i = (int*)(cand_v + (size_t)rows_cap * nblk * TOPK_MAX);
   launch_pdl(topk_stage1_kernel, dim3(rows, nblk), dim3(256), 0, st, part, sd, logits_out, cand_v, cand_i, vocab, c);
   HYDRA_LAUNCH_CHECK();
-  launch_pdl(topk_stage2_kernel, dim3(rows), dim3(256), 0, st, (const float*)cand_v, (const int*)cand_i, nblk, c, lv, first_child, n_child, out, T);
+  launch_pdl(topk_stage2_kernel, dim3(out_rows), dim3(256), 0, st, (const float*)cand_v, (const int*)cand_i, nblk, c, lv, first_child, n_child, out, T,
+             out_rows / rows);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
 
 hydra_status argmax_rows(const float* part, SplitDesc sd, float* logits_out, int* amax, void* scratch, int rows_cap, int rows,
                          int vocab, cudaStream_t st) {
-  return topk_rows(part, sd, logits_out, scratch, rows_cap, rows, vocab, 1, LevelDesc{0, 0, nullptr}, nullptr, nullptr, amax, 0, st);
+  return topk_rows(part, sd, logits_out, scratch, rows_cap, rows, rows, vocab, 1, LevelDesc{0, 0, nullptr}, nullptr, nullptr, amax, 0, st);
 }
 
 hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, int max_children, const int* first_child,
-                           const int* n_child, int* tree_tok, void* scratch, int rows_cap, int batch, int T, int vocab,
+                           const int* n_child, int* tree_tok, void* scratch, int rows_cap, int batch, int T, int vocab, int shared_rows,
                            cudaStream_t st) {
-  return topk_rows(part, sd, logits, scratch, rows_cap, batch * lv.n_parents, vocab, max_children, lv, first_child, n_child, tree_tok, T, st);
+  return topk_rows(part, sd, logits, scratch, rows_cap, shared_rows ? batch : batch * lv.n_parents, batch * lv.n_parents, vocab, max_children, lv,
+                   first_child, n_child, tree_tok, T, st);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -626,8 +630,8 @@ hydra_status topk_children(const float* part, SplitDesc sd, float* logits, Level
 template <typename T>
 __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restrict__ hprime, const T* __restrict__ embed,
                                                           const int* __restrict__ root_tok, int* tree_tok,
-                                                          const int* __restrict__ path_tab, LevelDesc lv, T* __restrict__ z, size_t z_ps,
-                                                          int T_rows, int kp1, int d_model, int vocab, int* status) {
+                                                          const int* __restrict__ path_tab, LevelDesc lv, int write_root, T* __restrict__ z,
+                                                          size_t z_ps, int T_rows, int kp1, int d_model, int vocab, int* status) {
   pdl_trigger();
   pdl_wait();
   const int row = blockIdx.x, b = row / lv.n_parents, j = row % lv.n_parents;
@@ -636,7 +640,7 @@ __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restric
   T* dst = z + ((size_t)row * (lv.d + 1) + blk) * d_model;
   if (blk == 0) {
     for (int i = threadIdx.x; i < d_model; i += blockDim.x) put<T>(dst + i, z_ps, hprime[(size_t)b * d_model + i]);
-    if (lv.d == 1 && j == 0 && threadIdx.x == 0) tree_tok[b * T_rows] = root_tok[b];
+    if (write_root && j == 0 && threadIdx.x == 0) tree_tok[b * T_rows] = root_tok[b];
     return;
   }
   int node = path_tab[p * kp1 + (blk - 1)];
@@ -646,15 +650,15 @@ __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restric
   for (int i = threadIdx.x; i < d_model; i += blockDim.x) put<T>(dst + i, z_ps, to_f<T>(e[i]));      // embeddings are exact: lo = 0
 }
 hydra_status head_gather(const float* hprime, const void* embed, const int* root_tok, int* tree_tok, const int* path_tab,
-                         LevelDesc lv, void* z, size_t z_ps, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
-                         cudaStream_t st) {
+                         LevelDesc lv, int write_root, void* z, size_t z_ps, int batch, int T, int kp1, int d_model, int vocab, int dtype,
+                         int* status, cudaStream_t st) {
   dim3 grid(batch * lv.n_parents, lv.d + 1);
   if (dtype == 0)
-    launch_pdl(head_gather_kernel<float>, dim3(grid), dim3(256), 0, st, hprime, (const float*)embed, root_tok, tree_tok, path_tab, lv, (float*)z, z_ps,
-                                                    T, kp1, d_model, vocab, status);
+    launch_pdl(head_gather_kernel<float>, dim3(grid), dim3(256), 0, st, hprime, (const float*)embed, root_tok, tree_tok, path_tab, lv, write_root,
+               (float*)z, z_ps, T, kp1, d_model, vocab, status);
   else
-    launch_pdl(head_gather_kernel<bf16>, dim3(grid), dim3(256), 0, st, hprime, (const bf16*)embed, root_tok, tree_tok, path_tab, lv, (bf16*)z, z_ps,
-                                                   T, kp1, d_model, vocab, status);
+    launch_pdl(head_gather_kernel<bf16>, dim3(grid), dim3(256), 0, st, hprime, (const bf16*)embed, root_tok, tree_tok, path_tab, lv, write_root,
+               (bf16*)z, z_ps, T, kp1, d_model, vocab, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
@@ -697,11 +701,26 @@ hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const
 // same thread has already read, so the in-place move is hazard-free.  The last CTA of a sequence to
 // finish publishes the new length / root token; all CTAs read the old length before they signal.
 // ------------------------------------------------------------------------------------------------
+// Typical criterion for candidate row i of sequence b (Section "Typical acceptance sampling"): with p = softmax(l / tau) at
+// the parent row and H its entropy, accept when p[token] > min(eps, alpha exp(-H)).  From the row statistics (max m,
+// Z = sum exp((l - m)/tau), S = sum exp((l - m)/tau) (l - m)/tau): p[x] = exp((l_x - m)/tau) / Z, H = log Z - S / Z.
+__device__ __forceinline__ bool typical_pass(const AcceptArgs& a, int b, int i) {
+  const int prow = b * a.T + a.parent[i];
+  const int tok = a.tree_tok[b * a.T + i];
+  if (tok < 0 || tok >= a.vocab) return false;
+  const float4 st = a.row_stats[prow];
+  const float z = (a.logits[(size_t)prow * a.vocab + tok] - st.x) / a.tau;
+  const float p = __expf(z) / st.y;
+  const float H = __logf(st.y) - st.z / st.y;
+  return p > fminf(a.eps, a.alpha * __expf(-H));
+}
+
 __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
   pdl_trigger();
   pdl_wait();
   __shared__ int s_path[72];
-  __shared__ int s_n, s_best;
+  __shared__ int s_n, s_best, s_bonus;
+  __shared__ float s_scan[256];
   const int b = blockIdx.y;
   const int T = a.T;
   if (threadIdx.x < 32) {
@@ -711,9 +730,10 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
     for (int half = 0; half < 2; ++half) {
       int i = lane + 32 * half;
       bool mt = false;
-      if (i >= 1 && i < T) mt = a.tree_tok[b * T + i] == a.amax[b * T + a.parent[i]];
+      if (i >= 1 && i < T) mt = a.mode == 1 ? typical_pass(a, b, i) : a.tree_tok[b * T + i] == a.amax[b * T + a.parent[i]];
       bits |= (uint64_t)__ballot_sync(0xffffffffu, mt) << (32 * half);
     }
+    if (lane == 0 && blockIdx.x == 0 && a.pass_bits) a.pass_bits[b] = bits;
     int key = -1;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
@@ -734,6 +754,40 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
   }
   __syncthreads();
   const int n = s_n, best = s_best;
+  // the token after the accepted path: the best row's argmax, or (typical mode with uniform numbers) a draw from its
+  // temperature distribution by inverse CDF in token-id order; only CTA 0 of the sequence works it out
+  const bool sampled = a.mode == 1 && a.u != nullptr;
+  if (blockIdx.x == 0) {
+    if (!sampled) {
+      if (threadIdx.x == 0) s_bonus = a.amax[b * T + best];
+    } else {
+      const float* lg = a.logits + (size_t)(b * T + best) * a.vocab;
+      const float mx = a.row_stats[b * T + best].x, inv_tau = 1.f / a.tau;
+      const int per = (a.vocab + 255) / 256, v0 = threadIdx.x * per, v1 = min(v0 + per, a.vocab);
+      float part = 0.f;
+      for (int v = v0; v < v1; ++v) part += __expf((lg[v] - mx) * inv_tau);
+      s_scan[threadIdx.x] = part;
+      __syncthreads();
+      if (threadIdx.x == 0) {                                          // sequential scan of 256 partial sums: fixed order
+        float run = 0.f;
+        for (int t = 0; t < 256; ++t) { const float p = s_scan[t]; s_scan[t] = run; run += p; }
+        const float target = a.u[b] * run;
+        int owner = 255;
+        for (int t = 0; t < 256; ++t) if (s_scan[t] <= target) owner = t;      // last thread whose range starts at or below the target
+        float acc = s_scan[owner];
+        int pick = -1;
+        const int w0 = owner * per, w1 = min(w0 + per, a.vocab);
+        for (int v = w0; v < w1 && pick < 0; ++v) { acc += __expf((lg[v] - mx) * inv_tau); if (acc > target) pick = v; }
+        if (pick < 0) {                                                   // rounding at a range boundary: the next token of non-zero weight
+          for (int v = w1; v < a.vocab && pick < 0; ++v) if (__expf((lg[v] - mx) * inv_tau) > 0.f) pick = v;
+          if (pick < 0) pick = a.vocab - 1;
+        }
+        s_bonus = pick;
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && a.bonus_tmp) a.bonus_tmp[b] = s_bonus;       // published with the fence before this CTA signs off below
+  }
   const int L = a.len[b];
   const bool in_range = L >= 0 && L + T <= a.max_seq;
   if (!in_range) {
@@ -769,7 +823,7 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
     if (a.out_tok) {
       int v = -1;
       if (k < n) v = a.tree_tok[b * T + s_path[k + 1]];
-      else if (k == n) v = a.amax[b * T + best];
+      else if (k == n) v = s_bonus;
       a.out_tok[b * (a.K + 1) + k] = v;
     }
     if (k == 0 && a.n_acc) a.n_acc[b] = n;
@@ -782,12 +836,42 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
       a.done_counter[b] = 0;
       if (in_range) {
         a.len[b] = L + n + 1;
-        a.root_tok[b] = a.amax[b * T + best];
+        __threadfence();
+        a.root_tok[b] = a.bonus_tmp ? *((volatile int*)a.bonus_tmp + b) : a.amax[b * T + best];
         a.n_new[b] = n + 1;
       }
     }
   }
 }
+// (max, sum exp((l - max)/tau), sum exp((l - max)/tau) (l - max)/tau) of every logits row; one CTA per row, fixed reduction order
+__global__ void __launch_bounds__(1024) softmax_row_stats_kernel(const float* __restrict__ logits, float4* __restrict__ stats, int vocab, float tau) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ float sh[32];
+  const float* lg = logits + (size_t)blockIdx.x * vocab;
+  float mx = -INFINITY;
+  for (int v = threadIdx.x; v < vocab; v += 1024) mx = fmaxf(mx, lg[v]);
+  mx = warp_max(mx);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  mx = sh[0];
+  for (int w = 1; w < 32; ++w) mx = fmaxf(mx, sh[w]);
+  __syncthreads();
+  float z_sum = 0.f, s_sum = 0.f;
+  const float inv_tau = 1.f / tau;
+  for (int v = threadIdx.x; v < vocab; v += 1024) {
+    const float z = (lg[v] - mx) * inv_tau, e = __expf(z);
+    z_sum += e; s_sum += e * z;
+  }
+  const float Z = block_sum(z_sum, sh), S = block_sum(s_sum, sh);
+  if (threadIdx.x == 0) stats[blockIdx.x] = make_float4(mx, Z, S, 0.f);
+}
+hydra_status softmax_row_stats(const float* logits, float4* row_stats, int rows, int vocab, float tau, cudaStream_t st) {
+  launch_pdl(softmax_row_stats_kernel, dim3(rows), dim3(1024), 0, st, logits, row_stats, vocab, tau);
+  HYDRA_LAUNCH_CHECK();
+  return HYDRA_OK;
+}
+
 hydra_status accept_compact(const AcceptArgs& a, cudaStream_t st) {
   long long units = (long long)a.n_layers * 2 * a.kv_planes * a.n_heads * (a.head_dim * a.esize / 16);
   int G = (int)((units + 255) / 256);

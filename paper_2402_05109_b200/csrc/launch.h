@@ -63,17 +63,19 @@ struct LevelDesc {           // one tree level d (1-based): the parents that hav
   int d, n_parents;
   const int* parents;        // device [n_parents] row ids
 };
-// z[b*P+j] = [hprime[b] ; E[tok[b][path(parent j)]]] in act dtype; also tree_tok[b][0] = root_tok[b] when d == 1.
+// z[b*P+j] = [hprime[b] ; E[tok[b][path(parent j)]]] in act dtype (lv.d path tokens; lv.d = 0: the hidden state alone);
+// with write_root also tree_tok[b][0] = root_tok[b].
 hydra_status head_gather(const float* hprime, const void* embed, const int* root_tok, int* tree_tok, const int* path_tab,
-                         LevelDesc lv, void* z, size_t z_ps, int batch, int T, int kp1, int d_model, int vocab, int dtype, int* status,
-                         cudaStream_t st);
+                         LevelDesc lv, int write_root, void* z, size_t z_ps, int batch, int T, int kp1, int d_model, int vocab, int dtype,
+                         int* status, cudaStream_t st);
 // y_out = res + silu(sum_s part[s] + bias); res row = hprime[b] when res_is_hprime else y row.  yb = act-dtype copy.
 hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const float* part, SplitDesc sd,
                       const void* bias, float* y_out, void* yb, size_t yb_ps, int rows, int d, int dtype, cudaStream_t st);
 // children of parent j of sequence b = top n_child tokens of logits row b*P+j, descending (ties: lower id first);
-// the logits are the summed partials, also written to `logits` [rows][vocab]
+// the logits are the summed partials, also written to `logits` [rows][vocab].  shared_rows: the logits have ONE row per
+// sequence (sequentially independent heads) and every parent of the level takes its children from that row.
 hydra_status topk_children(const float* part, SplitDesc sd, float* logits, LevelDesc lv, int max_children, const int* first_child,
-                           const int* n_child, int* tree_tok, void* scratch, int rows_cap, int batch, int T, int vocab,
+                           const int* n_child, int* tree_tok, void* scratch, int rows_cap, int batch, int T, int vocab, int shared_rows,
                            cudaStream_t st);
 
 // ---- acceptance + compaction (one kernel)
@@ -84,7 +86,18 @@ struct AcceptArgs {
   void* kv_base; const float* h_tree; int h_tree_stride;   // h_tree row = b*h_tree_stride + i
   float* h_new; int* n_new; int* len; int* root_tok;
   int* n_acc; int* path; int* out_tok; unsigned int* done_counter; int* status;
+  // acceptance criterion: 0 greedy (token == argmax at the parent); 1 typical (probability of the token under the
+  // temperature-tau distribution at the parent > min(eps, alpha * exp(-entropy)))
+  int mode; float tau, eps, alpha;
+  const float* logits;       // [batch*T][vocab] of the last verification (typical mode)
+  const float4* row_stats;   // [batch*T] (max logit, sum exp((l - max)/tau), sum exp(.) (l - max)/tau, 0) (typical mode)
+  int vocab;
+  const float* u;            // [batch] uniform numbers for the token after the accepted path, or null (= its argmax)
+  unsigned long long* pass_bits;   // [batch] out: bit i = candidate row i passed the criterion at its parent
+  int* bonus_tmp;            // [batch] scratch: the sampled token, handed from CTA 0 of a sequence to the CTA that publishes the state
 };
+// row_stats[r] for every logits row (typical acceptance)
+hydra_status softmax_row_stats(const float* logits, float4* row_stats, int rows, int vocab, float tau, cudaStream_t st);
 hydra_status accept_compact(const AcceptArgs& a, cudaStream_t st);
 
 // ---- small state kernels

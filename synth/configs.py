@@ -23,6 +23,7 @@ class HeadCfg:
     n_mlp_layers: int              # m: MLP layers per head
     prefix_attn: bool              # Hydra++ extra decoder layer
     has_bias: bool = True
+    medusa: bool = False           # sequentially independent heads: head i sees the hidden state only (the Medusa baseline)
 
 
 @dataclass

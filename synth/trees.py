@@ -13,7 +13,31 @@ from typing import List, Sequence
 _DIR = os.path.join(os.path.dirname(os.path.abspath(__file__)), "trees")
 
 
-def grow_tree(n_candidates: int, caps: Sequence[int], alpha=(0.70, 0.55, 0.45, 0.38), beta=0.45) -> List[int]:
+ALPHA = (0.70, 0.55, 0.45, 0.38)     # synthetic acceptance model: chance that head j's list holds the right token at all
+BETA = 0.45                          # ... and how fast it falls with the rank inside the list
+
+
+def node_score(path: Sequence[int], alpha=ALPHA, beta=BETA, normalised=False) -> float:
+    """Acceptance score of the candidate with rank path (r_1..r_k): prod_j alpha[j] * beta**r_j; `normalised` makes every
+    factor a probability over the ranks (times 1 - beta), so that the scores of a tree add up to an expected length."""
+    s = 1.0
+    for j, r in enumerate(path):
+        s *= alpha[j] * beta ** r * ((1.0 - beta) if normalised else 1.0)
+    return s
+
+
+def rank_paths(parent: Sequence[int]) -> List[tuple]:
+    """Rank path of every row (the root's is empty): index among the siblings, level by level."""
+    kids = {}
+    paths = [()] * len(parent)
+    for i in range(1, len(parent)):
+        r = kids.get(parent[i], 0)
+        kids[parent[i]] = r + 1
+        paths[i] = paths[parent[i]] + (r,)
+    return paths
+
+
+def grow_tree(n_candidates: int, caps: Sequence[int], alpha=ALPHA, beta=BETA, normalised=False) -> List[int]:
     """Greedy tree growth: repeatedly add the eligible node with the largest acceptance score.
 
     A candidate with rank path (r_1..r_k) scores prod_j alpha[j] * beta**r_j.  A node is eligible when
@@ -21,10 +45,7 @@ def grow_tree(n_candidates: int, caps: Sequence[int], alpha=(0.70, 0.55, 0.45, 0
     Ties go to the shallower node, then to the lexicographically smaller rank path.
     """
     def score(path):
-        s = 1.0
-        for j, r in enumerate(path):
-            s *= alpha[j] * beta ** r
-        return s
+        return node_score(path, alpha, beta, normalised)
 
     chosen = {()}
     while len(chosen) - 1 < n_candidates:

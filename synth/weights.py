@@ -29,7 +29,8 @@ def weight_shapes(m: ModelCfg, h: HeadCfg) -> Dict[str, tuple]:
     if h.prefix_attn:
         s.update(_layer_shapes("P.", m))
     for i in range(1, h.n_heads + 1):
-        s[f"H{i}.w1"] = (d, (i + 1) * d)        # input = [hidden ; E(x_t) ; E of the i-1 speculated tokens]
+        # input = [hidden ; E(x_t) ; E of the i-1 speculated tokens], or the hidden state alone for sequentially independent heads
+        s[f"H{i}.w1"] = (d, d if h.medusa else (i + 1) * d)
         s[f"H{i}.b1"] = (d,)
         if h.n_mlp_layers > 1:
             s[f"H{i}.wr"] = (h.n_mlp_layers - 1, d, d)

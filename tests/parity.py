@@ -147,10 +147,11 @@ def lockstep(o: HydraOracle, g, prompts, steps: int, seed: int, plant: bool = Tr
                 d = o.tree.K
                 P = o.tree.level_parents[d - 1]
                 hl = g.get_buffer("HEAD_LOGITS").view(-1, m.vocab)
+                shared = getattr(o.h, "medusa", False)             # sequentially independent heads: one logits row per sequence
                 for b in range(B):
                     for j, p in enumerate(P):
                         ref = o.head_logits(d, hp_o[b], [int(tg[b, i]) for i in o.tree.path[p]])
-                        e = float((hl[b * len(P) + j].cpu().double() - ref.double()).abs().max())
+                        e = float((hl[b if shared else b * len(P) + j].cpu().double() - ref.double()).abs().max())
                         st.max_head_logit_err = max(st.max_head_logit_err, e)
                         assert e <= LOGIT_TOL, f"head logits max-abs {e}"
         tok = tok_o.clone()

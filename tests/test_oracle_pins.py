@@ -304,6 +304,31 @@ def test_zeroed_embedding_columns_give_sequentially_independent_heads():
             assert kids == first[:len(kids)]
 
 
+def test_medusa_heads_equal_hydra_heads_with_zeroed_embedding_columns():
+    """Sequentially independent heads (Background, "Medusa decoding") are the special case of Hydra heads whose
+    first layer ignores the token embeddings: same children, same logits."""
+    m, h, w = tiny(mlp=2)
+    hm = HeadCfg(h.n_heads, h.n_mlp_layers, h.prefix_attn, h.has_bias, medusa=True)
+    wm = make_weights(m, hm, 0)
+    w = {k: v.clone() for k, v in w.items()}
+    d = m.d_model
+    for i in range(1, h.n_heads + 1):
+        assert tuple(wm[f"H{i}.w1"].shape) == (d, d)
+        w[f"H{i}.w1"].zero_()
+        w[f"H{i}.w1"][:, :d] = wm[f"H{i}.w1"]
+        for k in ("b1", "wr", "br"):
+            w[f"H{i}.{k}"] = wm[f"H{i}.{k}"]
+    parent = load_tree("tree15_d3")
+    prompt = [make_prompts(2, [6], m.vocab)[0]]
+    oh, om = HydraOracle(m, h, parent, w, 64), HydraOracle(m, hm, parent, wm, 64)
+    oh.prefill(prompt); om.prefill(prompt)
+    th, lh = oh.draft(return_logits=True)
+    tm, lm = om.draft(return_logits=True)
+    assert torch.equal(th, tm)
+    for p in lh[0]:
+        assert float((lh[0][p] - lm[0][p]).abs().max()) < 1e-12
+
+
 def test_children_sorted_by_descending_head_probability():
     cfg, w = c1()
     o = HydraOracle(cfg.model, cfg.head, load_tree(cfg.tree), w, cfg.max_seq)
