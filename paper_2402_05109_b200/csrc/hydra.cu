@@ -258,6 +258,9 @@ hydra_status run_gemm(hydra_ctx* c, const void* x, int x_rows_alloc, const void*
 size_t ps(const hydra_ctx* c, int rows_alloc, size_t cols) { return c->planes == 2 ? (size_t)rows_alloc * cols : 0; }
 
 // RoPE + KV append + tree attention of one layer from the QKV partial sums (*sd) in c->part; result in c->attn_out.
+// stable_lengths: every forward call of the library starts with rope_table, which lets nothing of the call start before all
+// earlier kernels have completed; the row set's lengths and the committed cache rows are written before that kernel, so
+// the attention kernels of the call may fetch committed tiles ahead of their predecessor.
 hydra_status attention_block(hydra_ctx* c, char* kc, char* vc, const RowSet& rs, int len_upper, const SplitDesc& sd, bool stable_lengths,
                              cudaStream_t st) {
   const hydra_model_cfg& m = c->m;
@@ -324,7 +327,7 @@ hydra_status run_prefix(hydra_ctx* c, const float* src, const RowSet& rs, int le
   HYDRA_TRY(residual_rmsnorm(src, nullptr, single_slot(0), c->x, c->pfx.attn_norm, c->xn, ps(c, c->R, d), nullptr, rows, d, m.rms_eps, m.dtype, st));
   SplitDesc sd;
   HYDRA_TRY(run_gemm(c, c->xn, c->R, c->pfx.wqkv, rows, 3 * d, d, &sd, st));
-  HYDRA_TRY(attention_block(c, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, sd, false, st));
+  HYDRA_TRY(attention_block(c, c->kv_pfx, c->kv_pfx + kvl, rs, len_upper, sd, true, st));
   return mlp_block(c, c->pfx, rows, nullptr, nullptr, nullptr, 0, nullptr, st);
 }
 
@@ -380,8 +383,6 @@ hydra_status do_verify(hydra_ctx* c, const int* tree_tok, int* amax, float* logi
   const int rows = c->batch * c->T;
   RowSet rs{c->batch, c->T, nullptr, c->d_len, c->d_depth, c->d_anc};
   SplitDesc sd;
-  // the lengths a verification reads date from the previous step's acceptance kernel (or the prompt pass), and the
-  // committed cache rows are older still: its attention kernels may fetch committed tiles ahead of their predecessor
   HYDRA_TRY(run_base(c, tree_tok, rs, len_bucket(c, max_len_ub(c) + c->T), c->lm_head, m.vocab, &sd, true, st));
   if (c->acc_mode == 1 && !logits) logits = c->logits;              // the typical criterion reads whole rows of logits
   c->last_logits = logits;
@@ -541,7 +542,7 @@ hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const
   for (int ch = 0; ch < nchunks; ++ch) {
     HYDRA_TRY(set_chunk(c->d_prompt_len, ch, CHUNK, c->d_pos0, c->d_nrows, batch, st));
     HYDRA_TRY(gather_chunk_tokens(tokens, c->d_offsets, ch, CHUNK, c->d_tok, batch, st));
-    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * CHUNK, nullptr, 0, nullptr, false, st));
+    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * CHUNK, nullptr, 0, nullptr, true, st));
     HYDRA_TRY(capture_last(c->h_tree, c->d_prompt_len, ch, CHUNK, c->h_new, c->h.n_heads + 1, c->d_n_new, c->d_len, batch, m.d_model, st));
     if (c->h.prefix_attn) HYDRA_TRY(run_prefix(c, c->h_tree, rs, (ch + 1) * CHUNK, st));
   }

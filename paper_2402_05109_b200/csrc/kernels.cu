@@ -209,9 +209,13 @@ hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd,
 // ------------------------------------------------------------------------------------------------
 // Rotary table + QKV post-processing (sum partials, rotate q and k, append K,V to the cache)
 // ------------------------------------------------------------------------------------------------
+// The first kernel of every forward call.  It lets its successors start only AFTER it has waited for everything before
+// it (trigger after wait): no kernel of this call can be resident, however early the following launches are, while a
+// kernel of an earlier call (the acceptance kernel that wrote the lengths, the kernels that filled the committed cache
+// rows) is still running.  The early cache fetches of the attention kernel rely on that.
 __global__ void rope_table_kernel(RowSet rs, float2* __restrict__ table, int half, float theta) {
-  pdl_trigger();
   pdl_wait();
+  pdl_trigger();
   int r = blockIdx.x, b = r / rs.tc, i = r % rs.tc;
   int pos = rs.pos0[b] + rs.depth[i];
   for (int j = threadIdx.x; j < half; j += blockDim.x) {

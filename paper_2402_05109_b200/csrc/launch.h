@@ -45,8 +45,9 @@ hydra_status tree_attention_f32(const float* q, const float* kcache, const float
 // [rows][H*hd] in two planes out_ps elements apart (0: hi only).  rs.mask == null selects a causal chunk (row i sees
 // the committed slots and new slots 0..i) of up to 128 rows (one plane, or head_dim 64); with a mask, up to 64 rows.
 // stable_lengths: rs.pos0 / rs.n_rows and every cache row below pos0 were written by kernels that had COMPLETED before the
-// kernel preceding this one in the stream started (true for the layers of a verification: the lengths date from the
-// previous step); the kernel then requests committed cache tiles before it waits for its predecessor.
+// kernel preceding this one in the stream started (true inside a forward call of the library, whose first kernel holds
+// its successors back until everything earlier has completed); the kernel then requests committed cache tiles before it
+// waits for its predecessor.
 hydra_status tree_attention_tc(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, int planes, RowSet rs,
                                bf16* out, size_t out_ps, int n_heads, int head_dim, int max_seq, int len_upper, int* status,
                                bool stable_lengths, cudaStream_t st);
