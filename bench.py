@@ -23,11 +23,12 @@ from synth import get_config, make_weights, make_prompts, load_tree, plant_row, 
 
 METRIC = "drafted+verified tokens/s (tree rows through draft+verify+accept per second)"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) per algorithmic byte of the tensor-core GEMM kernel, from an ncu capture of three launches
-# on the 4-layer cut of this workload (392.4 MB moved for 386.1 MB algorithmic; traffic is proportional to the weight
-# bytes, so the ratio carries to the full-size step).  Only valid for the bf16 tensor-core path (gemm mode 0); set to
-# None whenever that kernel changes until the counters are taken again.
-GEMM_TRAFFIC_RATIO = 1.016
+# DRAM bytes (read + write) per algorithmic byte of the tensor-core GEMM kernel, from an ncu capture of the two large
+# launches of a step on the 4-layer cut of this workload (the draft's vocabulary projection and a verification QKV
+# projection: 375.99 MB moved for 369.3 MB algorithmic; traffic is proportional to the weight bytes, so the ratio
+# carries to the full-size step).  Only valid for the bf16 tensor-core path (gemm mode 0); set to None whenever that
+# kernel changes until the counters are taken again.
+GEMM_TRAFFIC_RATIO = 1.018
 
 
 def peaks():

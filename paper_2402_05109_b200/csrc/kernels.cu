@@ -700,9 +700,10 @@ hydra_status head_act(const float* res, int res_is_hprime, int rows_per_b, const
 // ------------------------------------------------------------------------------------------------
 // Greedy acceptance + in-place KV compaction + state update, one kernel.
 // grid (G, batch).  Every CTA recomputes the accepted path of its sequence (cheap), then moves its
-// share of 16-byte KV pieces.  A thread moves its piece for k = 1..n in order: the destination slot k
-// can only be the source of a shallower path position (a row at depth j has index >= j), which that
-// same thread has already read, so the in-place move is hazard-free.  The last CTA of a sequence to
+// share of 16-byte KV pieces.  A thread moves its piece for k = 1..n in batches of 8 positions, reading a
+// batch before writing it: the destination slot k can only be the source of a path position j <= k (a row
+// at depth j has index >= j), which the same thread reads in the same or an earlier batch, before the
+// write, so the in-place move is hazard-free.  The last CTA of a sequence to
 // finish publishes the new length / root token; all CTAs read the old length before they signal.
 // ------------------------------------------------------------------------------------------------
 // Typical criterion for candidate row i of sequence b (Section "Typical acceptance sampling"): with p = softmax(l / tau) at
@@ -749,12 +750,16 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
-    if (lane == 0) {
-      int best = 63 - (key & 63), n = key >> 6;
-      s_n = n; s_best = best;
-      int node = best;
-      for (int k = n; k >= 0; --k) { s_path[k] = node; node = a.parent[node]; }
+    // walk from the best row to the root through the parents held in registers (lane i: rows i and i + 32)
+    const int p_lo = lane < T ? a.parent[lane] : 0, p_hi = lane + 32 < T ? a.parent[lane + 32] : 0;
+    const int best = 63 - (key & 63), n = key >> 6;
+    int node = best;
+    for (int k = n; k >= 0; --k) {
+      if (lane == 0) s_path[k] = node;
+      const int up_lo = __shfl_sync(0xffffffffu, p_lo, node & 31), up_hi = __shfl_sync(0xffffffffu, p_hi, node & 31);
+      node = node < 32 ? up_lo : up_hi;
     }
+    if (lane == 0) { s_n = n; s_best = best; }
   }
   __syncthreads();
   const int n = s_n, best = s_best;
@@ -806,11 +811,14 @@ __global__ void __launch_bounds__(256) accept_compact_kernel(AcceptArgs a) {
       int head = (int)(t % a.n_heads);
       long long lk = t / a.n_heads;                                    // (layer*2 + kv)*planes + plane
       char* base = (char*)a.kv_base + ((((size_t)lk * a.max_batch + b) * a.n_heads + head) * a.max_seq) * row_bytes;
-      for (int k = 1; k <= n; ++k) {
-        int src = s_path[k];
-        if (src != k)
-          *reinterpret_cast<uint4*>(base + (size_t)(L + k) * row_bytes + piece * 16) =
-              *reinterpret_cast<const uint4*>(base + (size_t)(L + src) * row_bytes + piece * 16);
+      for (int k0 = 1; k0 <= n; k0 += 8) {                             // all reads of a batch in flight before its writes
+        uint4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (k0 + j <= n) v[j] = *reinterpret_cast<const uint4*>(base + (size_t)(L + s_path[k0 + j]) * row_bytes + piece * 16);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (k0 + j <= n && s_path[k0 + j] != k0 + j) *reinterpret_cast<uint4*>(base + (size_t)(L + k0 + j) * row_bytes + piece * 16) = v[j];
       }
     }
     // hidden rows of the accepted path feed the next draft

@@ -63,6 +63,8 @@ def get_config(name: str) -> RunCfg:
         b = int(name[3:].rstrip("s")) if len(name) > 2 else 8          # "c3b1", "c3b2", "c3b4", "c3b8"
         return RunCfg(name, ModelCfg(**dict(_7B, n_layers=4 if small else 32)), HeadCfg(**_PP), "tree63_d4", b, _ragged(2, b, 128, 1024),
                       16 if small else 64, 2, 1024 + 64 * 5 + 64)
+    if name == "c4s":          # c4 cut to 4 layers: the small case for profiler captures of the long-cache attention
+        return RunCfg("c4s", ModelCfg(**dict(_13B, n_layers=4)), HeadCfg(**_PP), "tree63_d4", 1, [2048], 16, 3, 2048 + 16 * 5 + 64)
     if name == "c4":
         return RunCfg("c4", ModelCfg(**_13B), HeadCfg(**_PP), "tree63_d4", 1, [2048], 64, 3, 2048 + 64 * 5 + 64)
     if name == "c5":
