@@ -96,22 +96,26 @@ template <int HD, int QROWS, int NP> struct AttCfg {
   static constexpr int KH_BYTES = NP * TILE * 128;            // one half of a K tile: [plane][key][128 bytes] (the planes stacked along N)
   static constexpr int K_BYTES = NHALF * KH_BYTES;
   static constexpr int V_BYTES = NP * NHALF * TILE * 128;     // a V tile: [plane][half][key][128 bytes] (N blocks of 64 output columns)
-  static constexpr int STAGE_BYTES = K_BYTES + V_BYTES;
-  static constexpr int NST = NP == 1 ? 3 : (HD == 64 ? 3 : 2);        // ring stages
+  // K and V tiles travel through rings of their own: a K stage is free again as soon as the scores of its tile are done,
+  // long before the tile's P V product frees the V stage, so K runs further ahead inside the same shared memory.
+  static constexpr int NSK = K_BYTES >= 32768 ? 3 : 4;            // K ring stages
+  static constexpr int NSV = V_BYTES >= 32768 ? 2 : 4;            // V ring stages
   // MMA M is 128 whatever QROWS is: with 64 query rows the upper 64 accumulator lanes are unused (M = 64 instructions
   // measured slower per instruction), and the operand reads of a 64-row Q or P tile run 8 KB past the tile, into the next
   // piece of Q, of P or of the ring (never read back), so the order Q, P0, P1, ring keeps them inside the allocation.
   static constexpr int MROWS = 128;
   static constexpr int RPW = MROWS / 4;                       // accumulator rows (tensor-memory lanes) per softmax warp
-  static constexpr int RING_BYTES = NST * STAGE_BYTES;
+  static constexpr int KRING_BYTES = NSK * K_BYTES;
+  static constexpr int RING_BYTES = KRING_BYTES + NSV * V_BYTES;
   static constexpr int MERGE_BYTES = QROWS * HD * 4 + QROWS * 8;     // a chunk's partial rows + (max, sum); aliases the ring
-  static constexpr int NBAR = 1 + 3 * NST + 8;
+  static constexpr int NBAR = 1 + 2 * NSK + 2 * NSV + 8;
   static constexpr int SMEM_BYTES = 1024 + Q_BYTES + 2 * P_BYTES + (RING_BYTES > MERGE_BYTES ? RING_BYTES : MERGE_BYTES) + NBAR * 8 + 16;
   static constexpr int S_COLS = NP * TILE;                    // one score buffer: [Q_hi K_hi + Q_lo K_hi | Q_hi K_lo]
   static constexpr int O_COLS = NP * HD;                      // the output accumulator: [P_hi V_hi + P_lo V_hi | P_hi V_lo]
   static constexpr int O_COL0 = 2 * S_COLS;
   static constexpr int TMEM_COLS = O_COL0 + O_COLS <= 256 ? 256 : 512;
-  static_assert(RING_BYTES >= MERGE_BYTES, "merge area must fit in the ring");
+  static_assert(RING_BYTES >= MERGE_BYTES + 128 * MAX_CHUNKS * 4, "merge area and chunk weights must fit in the ring");
+  static_assert(MERGE_BYTES % 16 == 0, "alignment of the chunk weights");
   static_assert(O_COL0 + O_COLS <= 512, "tensor memory");
   static_assert(SMEM_BYTES <= 232448, "shared memory of one SM");
 };
@@ -121,22 +125,25 @@ __global__ void __launch_bounds__(192, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const AttArgs a) {
   using C = AttCfg<HD, QROWS, NP>;
-  constexpr int NST = C::NST;
+  constexpr int NSK = C::NSK, NSV = C::NSV;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t q_s = base, p_s = q_s + C::Q_BYTES, ring_s = p_s + 2 * C::P_BYTES;
+  const uint32_t q_s = base, p_s = q_s + C::Q_BYTES, ring_s = p_s + 2 * C::P_BYTES, vring_s = ring_s + C::KRING_BYTES;
   const uint32_t bars = ring_s + (C::RING_BYTES > C::MERGE_BYTES ? C::RING_BYTES : C::MERGE_BYTES);
   const uint32_t q_full = bars;
   auto k_full = [&](int s) { return bars + 8u * (1 + s); };
-  auto v_full = [&](int s) { return bars + 8u * (1 + NST + s); };
-  auto kv_empty = [&](int s) { return bars + 8u * (1 + 2 * NST + s); };
-  auto s_full = [&](int i) { return bars + 8u * (1 + 3 * NST + i); };
-  auto s_empty = [&](int i) { return bars + 8u * (1 + 3 * NST + 2 + i); };
-  auto p_full = [&](int i) { return bars + 8u * (1 + 3 * NST + 4 + i); };
-  auto pv_done = [&](int i) { return bars + 8u * (1 + 3 * NST + 6 + i); };
+  auto k_empty = [&](int s) { return bars + 8u * (1 + NSK + s); };
+  auto v_full = [&](int s) { return bars + 8u * (1 + 2 * NSK + s); };
+  auto v_empty = [&](int s) { return bars + 8u * (1 + 2 * NSK + NSV + s); };
+  constexpr int B0 = 1 + 2 * NSK + 2 * NSV;
+  auto s_full = [&](int i) { return bars + 8u * (B0 + i); };
+  auto s_empty = [&](int i) { return bars + 8u * (B0 + 2 + i); };
+  auto p_full = [&](int i) { return bars + 8u * (B0 + 4 + i); };
+  auto pv_done = [&](int i) { return bars + 8u * (B0 + 6 + i); };
   const uint32_t tmem_slot = bars + 8u * C::NBAR;
   __shared__ int s_abort;
-  __shared__ float s_w[128 * MAX_CHUNKS];               // normalised chunk weights of the rows this CTA merges
+  // normalised chunk weights of the rows this CTA merges: in the idle ring, behind the merge area its peers read
+  float* const s_w = reinterpret_cast<float*>(smem_raw + (ring_s - smem_u32(smem_raw)) + C::MERGE_BYTES);
 
   const RowSet& rs = a.rs;
   const int h = blockIdx.x, b = blockIdx.y, c = blockIdx.z;
@@ -146,7 +153,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (tid == 0) {
     s_abort = 0;
     mbar_init(q_full, 1);
-    for (int s = 0; s < NST; ++s) { mbar_init(k_full(s), 1); mbar_init(v_full(s), 1); mbar_init(kv_empty(s), 1); }
+    for (int s = 0; s < NSK; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
+    for (int s = 0; s < NSV; ++s) { mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(s_empty(i), 4); mbar_init(p_full(i), 4); mbar_init(pv_done(i), 1); }
     mbar_init_fence();
     prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
@@ -175,9 +183,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (lane == 0 && has_work) {
       const uint64_t pol = policy_evict_first(), pol_q = policy_evict_last();
       const int row0 = (b * H + h) * a.max_seq;
-      auto request_tile = [&](int i) {
-        const int s = i % NST;
-        const uint32_t k_dst = ring_s + s * C::STAGE_BYTES, v_dst = k_dst + C::K_BYTES;
+      auto request_k = [&](int i) {
+        const int s = i % NSK;
+        const uint32_t k_dst = ring_s + s * C::K_BYTES;
         const int r = row0 + (tile0 + i) * TILE;
         mbar_arrive_expect_tx(k_full(s), C::K_BYTES);
 #pragma unroll
@@ -185,6 +193,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
           for (int hf = 0; hf < C::NHALF; ++hf)
             tma_load_2d(k_dst + hf * C::KH_BYTES + pl * TILE * 128, &tmK, hf * 64, pl * a.kv_plane_rows + r, k_full(s), pol);
+      };
+      auto request_v = [&](int i) {
+        const int s = i % NSV;
+        const uint32_t v_dst = vring_s + s * C::V_BYTES;
+        const int r = row0 + (tile0 + i) * TILE;
         mbar_arrive_expect_tx(v_full(s), C::V_BYTES);
 #pragma unroll
         for (int pl = 0; pl < NP; ++pl)
@@ -192,9 +205,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int hf = 0; hf < C::NHALF; ++hf)
             tma_load_2d(v_dst + (pl * C::NHALF + hf) * TILE * 128, &tmV, hf * 64, pl * a.kv_plane_rows + r, v_full(s), pol);
       };
-      int i = 0;
-      if (a.early) {
-        for (; i < ntiles && i < NST && (tile0 + i + 1) * TILE <= p0; ++i) request_tile(i);     // committed rows only
+      int nk = 0, nv = 0;                                  // next K and V tile to request
+      if (a.early) {                                       // committed rows only
+        for (; nk < ntiles && nk < NSK && (tile0 + nk + 1) * TILE <= p0; ++nk) {
+          request_k(nk);
+          if (nv == nk && nv < NSV) request_v(nv++);
+        }
         pdl_wait();
       }
       mbar_arrive_expect_tx(q_full, C::Q_BYTES);
@@ -203,10 +219,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
         for (int hf = 0; hf < C::NHALF; ++hf)
           tma_load_2d(q_s + pl * C::QP_BYTES + hf * QROWS * 128, &tmQ, h * HD + hf * 64, pl * a.q_plane_rows + b * rs.tc, q_full, pol_q);
-      for (; i < ntiles; ++i) {
-        // stage i % NST was last read by the P V product of tile i - NST, the (i / NST - 1)-th completion of its empty barrier
-        if (i >= NST && !mbar_wait(kv_empty(i % NST), (uint32_t)((i / NST - 1) & 1), limit)) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
-        request_tile(i);
+      // K stage i % NSK was last read by the scores of tile i - NSK (completion i / NSK - 1 of its empty barrier), V stage
+      // i % NSV by the P V product of tile i - NSV; whichever ring has room is served first, K ahead of V
+      uint32_t idle = 0;
+      while (nk < ntiles || nv < ntiles) {
+        bool did = false;
+        if (nk < ntiles && (nk < NSK || mbar_test(k_empty(nk % NSK), (uint32_t)((nk / NSK - 1) & 1)))) { request_k(nk++); did = true; }
+        if (nv < nk && (nv < NSV || mbar_test(v_empty(nv % NSV), (uint32_t)((nv / NSV - 1) & 1)))) { request_v(nv++); did = true; }
+        if (did) idle = 0;
+        else if (++idle > limit) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
       }
     }
   } else if (warp == 1) {
@@ -217,14 +238,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       constexpr uint32_t idesc_pv2 = instr_desc_f16(0, C::MROWS, HD, 1);           // P_lo x V_hi
       // operand descriptors: built once; a byte offset inside shared memory adds offset / 16 to the start-address field
       const uint64_t q_desc = smem_desc_sw128(q_s), p_desc = smem_desc_sw128(p_s), k_desc = smem_desc_sw128(ring_s),
-                     v_desc = smem_desc_sw128_mn(ring_s + C::K_BYTES, TILE * 128);
+                     v_desc = smem_desc_sw128_mn(vring_s, TILE * 128);
       bool ok = mbar_wait(q_full, 0, limit);
       auto issue_s = [&](int i) {                        // S_i = Q K_i^T into score buffer i & 1
-        const int s = i % NST;
-        if (!mbar_wait(k_full(s), (uint32_t)((i / NST) & 1), limit)) return false;
+        const int s = i % NSK;
+        if (!mbar_wait(k_full(s), (uint32_t)((i / NSK) & 1), limit)) return false;
         if (i >= 2 && !mbar_wait(s_empty(i & 1), (uint32_t)(((i >> 1) - 1) & 1), limit)) return false;
         tc_fence_after();
-        const uint64_t kd = k_desc + (uint64_t)((s * C::STAGE_BYTES) >> 4);
+        const uint64_t kd = k_desc + (uint64_t)((s * C::K_BYTES) >> 4);
         const uint32_t d_s = tmem_base + (uint32_t)((i & 1) * C::S_COLS);
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk)
@@ -236,6 +257,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             umma_f16(d_s, q_desc + (uint64_t)((C::QP_BYTES + (kk >> 2) * QROWS * 128 + (kk & 3) * 32) >> 4),
                      kd + (uint64_t)(((kk >> 2) * C::KH_BYTES + (kk & 3) * 32) >> 4), idesc_s2, 1u);
         }
+        umma_commit(k_empty(s));                        // frees the K stage once these MMAs have read it
         umma_commit(s_full(i & 1));
         return true;
       };
@@ -243,11 +265,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       for (int i = 0; i < ntiles && ok; ++i) {
         if (i + 1 < ntiles) ok = issue_s(i + 1);
         if (!ok) break;
-        const int s = i % NST;
+        const int s = i % NSV;
         if (!mbar_wait(p_full(i & 1), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
-        if (!mbar_wait(v_full(s), (uint32_t)((i / NST) & 1), limit)) { ok = false; break; }
+        if (!mbar_wait(v_full(s), (uint32_t)((i / NSV) & 1), limit)) { ok = false; break; }
         tc_fence_after();
-        const uint64_t vd = v_desc + (uint64_t)((s * C::STAGE_BYTES) >> 4), pd = p_desc + (uint64_t)(((i & 1) * C::P_BYTES) >> 4);
+        const uint64_t vd = v_desc + (uint64_t)((s * C::V_BYTES) >> 4), pd = p_desc + (uint64_t)(((i & 1) * C::P_BYTES) >> 4);
         const uint32_t d_o = tmem_base + (uint32_t)C::O_COL0;
 #pragma unroll
         for (int kk = 0; kk < TILE / 16; ++kk)
@@ -257,7 +279,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           for (int kk = 0; kk < TILE / 16; ++kk)
             umma_f16(d_o, pd + (uint64_t)((C::PP_BYTES + kk * 32) >> 4), vd + (uint64_t)((kk * 2048) >> 4), idesc_pv2, 1u);
         }
-        umma_commit(kv_empty(s));
+        umma_commit(v_empty(s));
         umma_commit(pv_done(i & 1));
       }
       if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
@@ -380,9 +402,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (t0 + TILE > total) {
         // rows of the V tile past the end of the sequence hold whatever the cache holds: zero them, so that a
         // zero weight times a non-finite stale value cannot reach the accumulator
-        const int s = i % NST;
-        if (!mbar_wait(v_full(s), (uint32_t)((i / NST) & 1), limit)) { ok = false; break; }
-        const uint32_t v_src = ring_s + s * C::STAGE_BYTES + C::K_BYTES;
+        const int s = i % NSV;
+        if (!mbar_wait(v_full(s), (uint32_t)((i / NSV) & 1), limit)) { ok = false; break; }
+        const uint32_t v_src = vring_s + s * C::V_BYTES;
         const int first = total - t0;                       // first row to clear (>= 1)
         constexpr int BLK = NP * C::NHALF;                  // 64-column blocks of a V tile
         for (int e = st; e < (TILE - first) * BLK * 8; e += 128) {
