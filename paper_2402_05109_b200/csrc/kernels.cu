@@ -161,7 +161,11 @@ template <> __device__ __forceinline__ void put4<bf16>(bf16* p, size_t ps, float
 }
 
 constexpr int NORM_THREADS = 1024;
-template <typename T>
+// x_out = res + sum of the partial-sum slots; with `gain`, also xn = rmsnorm(x_out) * gain (operand planes) and hn (float).
+// A row is shared by the CS CTAs of a thread-block cluster (CTA `part` owns d / CS consecutive columns), so that few rows
+// still pull their partial sums through many SMs; the CTAs push their sums of squares into each other's shared memory and
+// add them in rank order after one cluster barrier.
+template <typename T, int CS>
 __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const float* res, const float* __restrict__ part,
                                                                         SplitDesc sd, float* x_out,
                                                                         const T* __restrict__ gain, T* __restrict__ xn, size_t xn_ps,
@@ -169,39 +173,75 @@ __global__ void __launch_bounds__(NORM_THREADS) residual_rmsnorm_kernel(const fl
   pdl_trigger();
   pdl_wait();
   __shared__ float sh[32];
-  const size_t base = (size_t)blockIdx.x * d;
+  __shared__ float s_ss[CS];
+  const int row = blockIdx.x / CS, rank = blockIdx.x % CS;
+  const int dc = d / CS, c0 = rank * dc;
+  const size_t base = (size_t)row * d;
   float ss = 0.f;
-  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {       // one 16-byte piece per thread and round, all its slot loads in flight together
+  float4 v0 = make_float4(0.f, 0.f, 0.f, 0.f);                          // this thread's first piece stays in registers
+  for (int i = c0 + threadIdx.x * 4, it = 0; i < c0 + dc; i += blockDim.x * 4, ++it) {   // one 16-byte piece per thread and round, all its slot loads in flight together
     size_t off[1] = {base + i};
-    int ns[1] = {part ? split_count(sd, (int)blockIdx.x, i) : 0};
+    int ns[1] = {part ? split_count(sd, row, i) : 0};
     float4 acc[1];
     float4 v = res ? *reinterpret_cast<const float4*>(res + base + i) : make_float4(0.f, 0.f, 0.f, 0.f);
     sum_slots_multi<1, 12>(part, sd.stride, off, ns, acc);             // narrow outputs are cut into up to ~11 slots per tile
     v.x += acc[0].x; v.y += acc[0].y; v.z += acc[0].z; v.w += acc[0].w;
     *reinterpret_cast<float4*>(x_out + base + i) = v;
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    if (it == 0) v0 = v;
   }
   if (!gain) return;
   float tot = block_sum(ss, sh);
-  float inv = rsqrtf(tot / (float)d + eps);
-  for (int i = threadIdx.x * 4; i < d; i += NORM_THREADS * 4) {
-    float4 v = *reinterpret_cast<const float4*>(x_out + base + i);
+  if constexpr (CS > 1) {
+    if (threadIdx.x < CS) {                                              // thread r leaves this CTA's sum in CTA r's slot `rank`
+      uint32_t local = (uint32_t)__cvta_generic_to_shared(&s_ss[rank]), remote;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"((uint32_t)threadIdx.x));
+      asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(tot) : "memory");
+    }
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    tot = 0.f;
+#pragma unroll
+    for (int r = 0; r < CS; ++r) tot += s_ss[r];
+  }
+  const float inv = rsqrtf(tot / (float)d + eps);
+  for (int i = c0 + threadIdx.x * 4, it = 0; i < c0 + dc; i += blockDim.x * 4, ++it) {
+    float4 v = it == 0 ? v0 : *reinterpret_cast<const float4*>(x_out + base + i);
     float4 gn = load4<T>(gain + i);
     v.x *= inv * gn.x; v.y *= inv * gn.y; v.z *= inv * gn.z; v.w *= inv * gn.w;
     if (xn) put4<T>(xn + base + i, xn_ps, v);
     if (hn) *reinterpret_cast<float4*>(hn + base + i) = v;
   }
 }
+template <typename T, int CS>
+static cudaError_t launch_norm(int rows, int d, cudaStream_t st, const float* res, const float* part, SplitDesc sd, float* x_out,
+                               const void* gain, void* xn, size_t xn_ps, float* hn, float eps) {
+  int threads = (d / CS / 4 + 31) / 32 * 32;
+  if (threads > NORM_THREADS) threads = NORM_THREADS;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(rows * CS); cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = CS; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = CS > 1 ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, residual_rmsnorm_kernel<T, CS>, res, part, sd, x_out, (const T*)gain, (T*)xn, xn_ps, hn, d, eps);
+}
 hydra_status residual_rmsnorm(const float* res, const float* part, SplitDesc sd, float* x_out,
                               const void* gain, void* xn, size_t xn_ps, float* hn, int rows, int d, float eps, int dtype,
                               cudaStream_t st) {
   if (d & 3) return HYDRA_ERR_UNSUPPORTED;
-  if (dtype == 0)
-    launch_pdl(residual_rmsnorm_kernel<float>, dim3(rows), dim3(NORM_THREADS), 0, st, res, part, sd, x_out, (const float*)gain,
-                                                                  (float*)xn, xn_ps, hn, d, eps);
-  else
-    launch_pdl(residual_rmsnorm_kernel<bf16>, dim3(rows), dim3(NORM_THREADS), 0, st, res, part, sd, x_out, (const bf16*)gain,
-                                                                 (bf16*)xn, xn_ps, hn, d, eps);
+  // few rows: 4 or 2 CTAs per row (the columns must split into whole 16-byte pieces)
+  const int cs = (rows <= 40 && d % 16 == 0) ? 4 : (rows <= 96 && d % 8 == 0) ? 2 : 1;
+  if (dtype == 0) {
+    if (cs == 4) launch_norm<float, 4>(rows, d, st, res, part, sd, x_out, gain, xn, xn_ps, hn, eps);
+    else if (cs == 2) launch_norm<float, 2>(rows, d, st, res, part, sd, x_out, gain, xn, xn_ps, hn, eps);
+    else launch_norm<float, 1>(rows, d, st, res, part, sd, x_out, gain, xn, xn_ps, hn, eps);
+  } else {
+    if (cs == 4) launch_norm<bf16, 4>(rows, d, st, res, part, sd, x_out, gain, xn, xn_ps, hn, eps);
+    else if (cs == 2) launch_norm<bf16, 2>(rows, d, st, res, part, sd, x_out, gain, xn, xn_ps, hn, eps);
+    else launch_norm<bf16, 1>(rows, d, st, res, part, sd, x_out, gain, xn, xn_ps, hn, eps);
+  }
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }
