@@ -12,13 +12,18 @@
 //
 // One CTA per (head, sequence, KV chunk).  A sequence's KV rows are cut into 64-row tiles and the tiles are dealt
 // to the launch's chunks in equal contiguous runs, computed on the device from the real length (a captured graph
-// keeps balanced chunks as the sequence grows).  192 threads:
-//   warp 0 (one lane)  TMA producer: Q once, then K and V tiles through a ring of stages (K and V of a stage have
-//                      their own "full" barriers, so the scores of a tile start before its V has landed);
-//   warp 1 (one lane)  MMA issue: S_i = Q K_i^T (M = 128 query lanes, N = 64 keys) into one of two score buffers in
+// keeps balanced chunks as the sequence grows).  256 threads:
+//   warp 2 (one lane)  TMA producer: Q once, then K tiles and V tiles through rings of their own (a K stage is free
+//                      as soon as the scores of its tile are done, a V stage after the tile's P V product), each stage
+//                      with its own "full" barrier, so the scores of a tile start before its V has landed;
+//   warp 3 (one lane)  MMA issue: S_i = Q K_i^T (M = 128 query lanes, N = 64 keys) into one of two score buffers in
 //                      tensor memory, issued one tile ahead; O += P_i V_i (N = head_dim, V read as an MN-major operand
 //                      straight from its [key][dim] tile) into one accumulator that lives across the chunk;
-//   warps 2..5         softmax: thread = query row.  Reads its score row from tensor memory, applies the scale and
+//   four softmax warps thread = query row (a tensor-memory lane).  With 64 query rows two warps share a quadrant of
+//                      tensor memory (warps 0 and 4: rows 0..31, warps 1 and 5: rows 32..63) and each takes half of a
+//                      tile's keys; the two swap their row maxima through shared memory, keep the same reference
+//                      maximum and each its own part of the row sum.  With 128 rows warps 4..7 take a quadrant each
+//                      and all keys.  A thread reads its scores from tensor memory, applies the scale and
 //                      the mask (committed slots are visible to every row; tree slot j to row i iff bit j of the
 //                      row's ancestor bitmask, or j <= i for a causal chunk), keeps the row's running reference
 //                      maximum and sum in the exp2 domain, writes P_i as float16 into a swizzled shared-memory
@@ -59,11 +64,6 @@ __device__ __forceinline__ uint32_t peer_smem(uint32_t saddr, uint32_t rank) {  
 __device__ __forceinline__ float4 ld_peer4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ float2 ld_peer2(uint32_t addr) {
-  float2 v;
-  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ float ex2(float x) {
@@ -107,9 +107,15 @@ template <int HD, int QROWS, int NP> struct AttCfg {
   static constexpr int RPW = MROWS / 4;                       // accumulator rows (tensor-memory lanes) per softmax warp
   static constexpr int KRING_BYTES = NSK * K_BYTES;
   static constexpr int RING_BYTES = KRING_BYTES + NSV * V_BYTES;
-  static constexpr int MERGE_BYTES = QROWS * HD * 4 + QROWS * 8;     // a chunk's partial rows + (max, sum); aliases the ring
-  static constexpr int NBAR = 1 + 2 * NSK + 2 * NSV + 8;
-  static constexpr int SMEM_BYTES = 1024 + Q_BYTES + 2 * P_BYTES + (RING_BYTES > MERGE_BYTES ? RING_BYTES : MERGE_BYTES) + NBAR * 8 + 16;
+  static constexpr int MERGE_BYTES = QROWS * HD * 4 + QROWS * 16;    // a chunk's partial rows + (max, sum, max, sum of the other key half); aliases the ring
+  // 64 query rows: two softmax warps per tensor-memory quadrant, each with half of a tile's keys (SPLIT); they exchange
+  // their row maxima through XM_BYTES of shared memory.  128 rows: one warp per quadrant, thread = row, all keys.
+  static constexpr bool SPLIT = QROWS == 64;
+  static constexpr int KPT = SPLIT ? TILE / 2 : TILE;                // keys per softmax thread and tile
+  static constexpr int XM_BYTES = 2 * 2 * 64 * 4;                    // [tile parity][key half][row]
+  static constexpr int NBAR = 1 + 2 * NSK + 2 * NSV + 8 + 4;
+  static constexpr int SMEM_BYTES = 1024 + Q_BYTES + 2 * P_BYTES + (RING_BYTES > MERGE_BYTES ? RING_BYTES : MERGE_BYTES) + XM_BYTES + NBAR * 8 + 16;
+  static constexpr int NTHREADS = 256;
   static constexpr int S_COLS = NP * TILE;                    // one score buffer: [Q_hi K_hi + Q_lo K_hi | Q_hi K_lo]
   static constexpr int O_COLS = NP * HD;                      // the output accumulator: [P_hi V_hi + P_lo V_hi | P_hi V_lo]
   static constexpr int O_COL0 = 2 * S_COLS;
@@ -121,7 +127,7 @@ template <int HD, int QROWS, int NP> struct AttCfg {
 };
 
 template <int HD, int QROWS, int NP>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(256, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const AttArgs a) {
   using C = AttCfg<HD, QROWS, NP>;
@@ -129,7 +135,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_s = base, p_s = q_s + C::Q_BYTES, ring_s = p_s + 2 * C::P_BYTES, vring_s = ring_s + C::KRING_BYTES;
-  const uint32_t bars = ring_s + (C::RING_BYTES > C::MERGE_BYTES ? C::RING_BYTES : C::MERGE_BYTES);
+  const uint32_t xm_s = ring_s + (C::RING_BYTES > C::MERGE_BYTES ? C::RING_BYTES : C::MERGE_BYTES);
+  const uint32_t bars = xm_s + C::XM_BYTES;
   const uint32_t q_full = bars;
   auto k_full = [&](int s) { return bars + 8u * (1 + s); };
   auto k_empty = [&](int s) { return bars + 8u * (1 + NSK + s); };
@@ -140,6 +147,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   auto s_empty = [&](int i) { return bars + 8u * (B0 + 2 + i); };
   auto p_full = [&](int i) { return bars + 8u * (B0 + 4 + i); };
   auto pv_done = [&](int i) { return bars + 8u * (B0 + 6 + i); };
+  auto xm_bar = [&](int par, int quad) { return bars + 8u * (B0 + 8 + 2 * par + quad); };   // both key halves of a quadrant have left their maxima
   const uint32_t tmem_slot = bars + 8u * C::NBAR;
   __shared__ int s_abort;
   // normalised chunk weights of the rows this CTA merges: in the idle ring, behind the merge area its peers read
@@ -156,10 +164,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     for (int s = 0; s < NSK; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
     for (int s = 0; s < NSV; ++s) { mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(s_empty(i), 4); mbar_init(p_full(i), 4); mbar_init(pv_done(i), 1); }
+    for (int i = 0; i < 4; ++i) mbar_init(xm_bar(i >> 1, i & 1), 2);
     mbar_init_fence();
     prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
   }
-  if (warp == 1) tmem_alloc(tmem_slot, C::TMEM_COLS);
+  if (warp == 3) tmem_alloc(tmem_slot, C::TMEM_COLS);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -179,7 +188,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const int ntiles = has_work ? tile1 - tile0 : 0;
   const uint32_t limit = a.wait_limit;
 
-  if (warp == 0) {
+  // warp 2: TMA producer (one lane); warp 3: MMA issue (one lane); softmax: warps 0, 1, 4, 5 (quadrants 0, 1, 0, 1; key halves
+  // 0, 0, 1, 1) for 64 query rows, warps 4..7 (quadrants 0..3) for 128
+  const bool softmax_warp = C::SPLIT ? (warp & 2) == 0 : warp >= 4;
+  if (warp == 2) {
     if (lane == 0 && has_work) {
       const uint64_t pol = policy_evict_first(), pol_q = policy_evict_last();
       const int row0 = (b * H + h) * a.max_seq;
@@ -230,7 +242,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         else if (++idle > limit) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; break; }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 3) {
     if (lane == 0 && has_work) {
       constexpr uint32_t idesc_s = instr_desc_f16(0, C::MROWS, NP * TILE, 0);      // Q_hi x [K_hi ; K_lo]
       constexpr uint32_t idesc_s2 = instr_desc_f16(0, C::MROWS, TILE, 0);          // Q_lo x K_hi
@@ -284,9 +296,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
       if (!ok) { atomicOr(a.status, ST_TIMEOUT); s_abort = 1; }
     }
-  } else {
-    // ---- softmax warps: thread = accumulator row = a tensor-memory lane of the warp's quadrant
-    const int quad = warp & 3, row = quad * C::RPW + lane;
+  } else if (softmax_warp) {
+    // ---- softmax warps: thread = accumulator row = a tensor-memory lane of the warp's quadrant; KPT of the tile's keys
+    constexpr int KPT = C::KPT;
+    const int quad = warp & 3, half = C::SPLIT ? warp >> 2 : 0, row = quad * C::RPW + lane;
+    const int kb0 = half * KPT;                           // first key of the tile this thread looks at
     const bool row_valid = row < QROWS;
     const bool warp_rows = quad * C::RPW < nr;            // any row of this warp in use
     const bool row_live = row_valid && row < nr;
@@ -294,24 +308,24 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint64_t mask = (row_live && rs.mask) ? rs.mask[row] : 0ull;
     const bool causal = rs.mask == nullptr;
     const float sc = rsqrtf((float)HD) * 1.4426950408889634f;   // 1/sqrt(hd) * log2(e)
-    float m_ref = -INFINITY, l = 0.f;
+    float m_ref = -INFINITY, l = 0.f;                     // l: the sum over this thread's keys only
     bool ok = true;
-    const int st = tid - 64;                              // 0..127 among the softmax threads
+    const int st = (C::SPLIT ? half * 2 + quad : warp - 4) * 32 + lane;      // 0..127 among the softmax threads
     for (int i = 0; i < ntiles; ++i) {
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }     // a wait that ran out in one lane ends the walk for the whole warp
       const int t0 = (tile0 + i) * TILE;
       if (!mbar_wait(s_full(i & 1), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
       tc_fence_after();
-      uint32_t r[64];
+      uint32_t r[KPT];
       if (warp_rows) {
-        const uint32_t s_addr = lane_addr + (uint32_t)((i & 1) * C::S_COLS);
-        if (NP == 1) {
-          tmem_ld64(s_addr, r);
+        const uint32_t s_addr = lane_addr + (uint32_t)((i & 1) * C::S_COLS + kb0);
+        if constexpr (NP == 1) {
+          if constexpr (KPT == 64) tmem_ld64(s_addr, r); else tmem_ld32(s_addr, r);
         } else {                                           // the two column halves of the score buffer in one round trip, added
-          uint32_t y[64];
-          tmem_ld64x2(s_addr, s_addr + (uint32_t)TILE, r, y);
+          uint32_t y[KPT];
+          if constexpr (KPT == 64) tmem_ld64x2(s_addr, s_addr + (uint32_t)TILE, r, y); else tmem_ld32x2(s_addr, s_addr + (uint32_t)TILE, r, y);
 #pragma unroll
-          for (int j = 0; j < 64; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(y[j]));
+          for (int j = 0; j < KPT; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(y[j]));
         }
       }
       tc_fence_before();
@@ -334,12 +348,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           const int nv = total - t0;                       // keys of the tile that exist
           if (nv < 64) vis &= (1ull << nv) - 1ull;
         }
+        if constexpr (C::SPLIT) vis >>= kb0;
         float mx = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 64; ++j) {
+        for (int j = 0; j < KPT; ++j) {
           const float v = ((vis >> j) & 1ull) ? __uint_as_float(r[j]) * sc : -INFINITY;
           r[j] = __float_as_uint(v);
           mx = fmaxf(mx, v);
+        }
+        if constexpr (C::SPLIT) {
+          // the row's maximum over all 64 keys: the two warps of the quadrant swap theirs (buffer and barrier of the tile's
+          // parity; a buffer is rewritten two tiles later, after the P V product that followed this read has been issued)
+          const uint32_t xm = xm_s + (uint32_t)(((i & 1) * 2) * 64 * 4);
+          asm volatile("st.shared.f32 [%0], %1;" ::"r"(xm + (uint32_t)((half * 64 + row) * 4)), "f"(mx) : "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(xm_bar(i & 1, quad));
+          if (!mbar_wait(xm_bar(i & 1, quad), (uint32_t)((i >> 1) & 1), limit)) { ok = false; break; }
+          float other;
+          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(other) : "r"(xm + (uint32_t)(((half ^ 1) * 64 + row) * 4)) : "memory");
+          mx = fmaxf(mx, other);
         }
         float m_new = m_ref;
         if (mx > m_ref + RESCALE_STEP) m_new = mx;          // also the first finite maximum (m_ref = -inf)
@@ -348,9 +375,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         m_ref = m_new;
         const float bse = m_new == -INFINITY ? 0.f : m_new;
         float sum = 0.f;
-        uint32_t pk[32];
+        uint32_t pk[KPT / 2];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
+        for (int j = 0; j < KPT / 2; ++j) {
           const float p0v = ex2(__uint_as_float(r[2 * j]) - bse), p1v = ex2(__uint_as_float(r[2 * j + 1]) - bse);
           pk[j] = pack_half2(p0v, p1v);
           if (NP == 1) {
@@ -364,11 +391,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         l = l * alpha + sum;
         // P buffer i & 1 was last read by P V of tile i - 2; the row's accumulator by P V of tile i - 1
         if (i >= 2 && !mbar_wait(pv_done(i & 1), (uint32_t)(((i >> 1) - 1) & 1), limit)) { ok = false; break; }
-        if (__any_sync(0xffffffffu, rescale)) {
+        if (__any_sync(0xffffffffu, rescale)) {            // both warps of a quadrant decide alike; each scales its half of the columns
           if (i >= 1 && !mbar_wait(pv_done((i - 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), limit)) { ok = false; break; }
           tc_fence_after();
+          constexpr int OC = C::SPLIT ? C::O_COLS / 2 : C::O_COLS;
 #pragma unroll 1
-          for (int c0 = 0; c0 < C::O_COLS; c0 += 32) {
+          for (int c0 = half * OC; c0 < (half + 1) * OC; c0 += 32) {
             uint32_t o[32];
             tmem_ld32(lane_addr + (uint32_t)(C::O_COL0 + c0), o);
 #pragma unroll
@@ -379,19 +407,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t prow = p_s + (i & 1) * C::P_BYTES + (uint32_t)row * 128u;
         if (row_valid) {
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch) {
-            const uint32_t dst = prow + (uint32_t)((ch ^ (row & 7)) * 16);
+          for (int ch = 0; ch < KPT / 8; ++ch) {
+            const uint32_t dst = prow + (uint32_t)(((kb0 / 8 + ch) ^ (row & 7)) * 16);
             asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]), "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3]) : "memory");
           }
           if (NP == 2) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {                 // lo = f16(p - f16(p))
+            for (int j = 0; j < KPT / 2; ++j) {            // lo = f16(p - f16(p))
               const __half2 hv = *reinterpret_cast<const __half2*>(&pk[j]);
               pk[j] = pack_half2(__uint_as_float(r[2 * j]) - __low2float(hv), __uint_as_float(r[2 * j + 1]) - __high2float(hv));
             }
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-              const uint32_t dst = prow + (uint32_t)(C::PP_BYTES + (ch ^ (row & 7)) * 16);
+            for (int ch = 0; ch < KPT / 8; ++ch) {
+              const uint32_t dst = prow + (uint32_t)(C::PP_BYTES + ((kb0 / 8 + ch) ^ (row & 7)) * 16);
               asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]), "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3]) : "memory");
             }
           }
@@ -427,11 +455,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
     {
-      const uint32_t xo = ring_s + (uint32_t)row * (HD * 4), xml = ring_s + QROWS * HD * 4 + (uint32_t)row * 8;
+      const uint32_t xo = ring_s + (uint32_t)row * (HD * 4), xml = ring_s + QROWS * HD * 4 + (uint32_t)row * 16 + (uint32_t)half * 8;
       const bool have = ok && ntiles > 0 && row_live && m_ref != -INFINITY;
       if (ok && ntiles > 0 && warp_rows) {
+        // 64 output columns (both planes' halves) per tensor-memory round trip; with two warps per quadrant each takes
+        // every other block of 64
 #pragma unroll 1
-        for (int c0 = 0; c0 < HD; c0 += 64) {              // 64 output columns (both planes' halves) per tensor-memory round trip
+        for (int c0 = half * 64; c0 < HD; c0 += C::SPLIT ? 128 : 64) {
           uint32_t o[64];
           if (NP == 2) {
             uint32_t o2[64];
@@ -451,9 +481,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           }
         }
       }
-      if (row_valid) {
+      if (row_valid) {                                     // (max, this thread's part of the sum); without a second key half its slot reads (max, 0)
         const float2 ml = have ? make_float2(m_ref, l) : make_float2(-INFINITY, 0.f);
         asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(xml), "f"(ml.x), "f"(ml.y) : "memory");
+        if constexpr (!C::SPLIT) asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(xml + 8u), "f"(ml.x), "f"(0.f) : "memory");
       }
     }
   }
@@ -471,14 +502,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int rows_cap = min(rs.tc, QROWS);
     const int my_rows = rows_cap > c ? (rows_cap - c + nchunks - 1) / nchunks : 0;
     // chunk weights of my rows, normalised: w_c = 2^(m_c - M) / sum_c l_c 2^(m_c - M)  (one thread per row, all (m, l) loads in flight together)
-    for (int t = tid; t < my_rows; t += 192) {
+    for (int t = tid; t < my_rows; t += C::NTHREADS) {
       const int i = c + t * nchunks;
       float mc[MAX_CHUNKS], lc[MAX_CHUNKS];
       float M = -INFINITY, L = 0.f;
 #pragma unroll
       for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
         mc[cc] = -INFINITY; lc[cc] = 0.f;
-        if (cc < nchunks && i < nr) { const float2 ml = ld_peer2(peer_smem(xml_s + (uint32_t)i * 8u, (uint32_t)cc)); mc[cc] = ml.x; lc[cc] = ml.y; }
+        if (cc < nchunks && i < nr) { const float4 ml = ld_peer4(peer_smem(xml_s + (uint32_t)i * 16u, (uint32_t)cc)); mc[cc] = ml.x; lc[cc] = ml.y + ml.w; }
       }
 #pragma unroll
       for (int cc = 0; cc < MAX_CHUNKS; ++cc) M = fmaxf(M, mc[cc]);
@@ -491,12 +522,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     // two output pieces per thread and round, all their peer loads in flight together (a load that waits for the
     // previous one's use costs a shared-memory round trip across the cluster each)
-    for (int e0 = tid; e0 < my_rows * V4; e0 += 2 * 192) {
+    for (int e0 = tid; e0 < my_rows * V4; e0 += 2 * C::NTHREADS) {
       float4 v[2][MAX_CHUNKS];
       float w[2][MAX_CHUNKS];
 #pragma unroll
       for (int ib = 0; ib < 2; ++ib) {
-        const int e = e0 + ib * 192, t = e / V4, i = c + t * nchunks, k4 = e % V4;
+        const int e = e0 + ib * C::NTHREADS, t = e / V4, i = c + t * nchunks, k4 = e % V4;
         const bool live = e < my_rows * V4;
 #pragma unroll
         for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
@@ -508,7 +539,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
 #pragma unroll
       for (int ib = 0; ib < 2; ++ib) {
-        const int e = e0 + ib * 192, t = e / V4, i = c + t * nchunks, k4 = e % V4;
+        const int e = e0 + ib * C::NTHREADS, t = e / V4, i = c + t * nchunks, k4 = e % V4;
         if (e >= my_rows * V4 || s_abort) continue;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -530,7 +561,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (s_abort) {                                          // let copies in flight land before the CTA retires
     for (int i = 0; i < 2000; ++i) __nanosleep(100);
   }
-  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, C::TMEM_COLS); }
+  if (warp == 3) { tc_fence_after(); tmem_dealloc(tmem_base, C::TMEM_COLS); }
 }
 
 // Number of KV chunks per (head, sequence) for lengths up to len_upper: the count (at most 8) that minimises the
@@ -572,7 +603,7 @@ hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc
   a.q_plane_rows = q_rows; a.kv_plane_rows = (int)cache_rows; a.early = stable_lengths ? 1 : 0;
   a.nchunks = pick_chunks(H * rs.batch, len_upper, sm_count());
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(H, rs.batch, a.nchunks); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = C::SMEM_BYTES; cfg.stream = st;
+  cfg.gridDim = dim3(H, rs.batch, a.nchunks); cfg.blockDim = dim3(C::NTHREADS); cfg.dynamicSmemBytes = C::SMEM_BYTES; cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = (unsigned)a.nchunks;

@@ -289,7 +289,7 @@ __global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __rest
   const int slot = rs.pos0[b] + i;
   if (slot < 0 || slot >= max_seq) { if (threadIdx.x == 0 && blockIdx.y == 0) atomicOr(status, ST_BOUNDS); return; }
   const int tph = half >> 2;                                       // threads per head
-  const int h = blockIdx.y * (256 / tph) + threadIdx.x / tph;
+  const int h = blockIdx.y * (blockDim.x / tph) + threadIdx.x / tph;
   if (h >= H) return;
   const int j = (threadIdx.x % tph) * 4;
   const int c0 = h * hd + j, c1 = c0 + half;
@@ -325,13 +325,15 @@ __global__ void __launch_bounds__(256) qkv_rope_store_kernel(const float* __rest
 hydra_status qkv_rope_store(const float* part, SplitDesc sd, const float2* table, void* q, size_t q_ps, void* kcache, void* vcache,
                             size_t kv_ps, RowSet rs, int H, int hd, int max_seq, int dtype, int* status, cudaStream_t st) {
   if (hd % 8) return HYDRA_ERR_UNSUPPORTED;
-  const int heads_per_block = 256 / (hd / 8);
+  // 128 threads per CTA: with 64 rows twice as many SMs pull the partial sums as with 256
+  const int threads = 128 % (hd / 8) == 0 ? 128 : 256;
+  const int heads_per_block = threads / (hd / 8);
   dim3 grid(rs.batch * rs.tc, (H + heads_per_block - 1) / heads_per_block);
   if (dtype == 0)
-    launch_pdl(qkv_rope_store_kernel<float>, grid, dim3(256), 0, st, part, sd, table, (float*)q, q_ps, (float*)kcache, (float*)vcache,
+    launch_pdl(qkv_rope_store_kernel<float>, grid, dim3(threads), 0, st, part, sd, table, (float*)q, q_ps, (float*)kcache, (float*)vcache,
                kv_ps, rs, H, hd, max_seq, status);
   else
-    launch_pdl(qkv_rope_store_kernel<__half>, grid, dim3(256), 0, st, part, sd, table, (__half*)q, q_ps, (__half*)kcache, (__half*)vcache,
+    launch_pdl(qkv_rope_store_kernel<__half>, grid, dim3(threads), 0, st, part, sd, table, (__half*)q, q_ps, (__half*)kcache, (__half*)vcache,
                kv_ps, rs, H, hd, max_seq, status);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
