@@ -566,7 +566,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
 // Number of KV chunks per (head, sequence) for lengths up to len_upper: the count (at most 8) that minimises the
 // largest number of tiles any SM walks, with about three tiles' worth of set-up and merging per CTA; ties go to
-// fewer chunks.  Two CTAs share an SM (shared memory and tensor memory allow it).
+// fewer chunks.  One CTA per SM (the rings take nearly all of its shared memory).
 int pick_chunks(int pairs, int len_upper, int sms) {
   const int nt = (len_upper + TILE - 1) / TILE;
   int hi = nt < MAX_CHUNKS ? nt : MAX_CHUNKS;
