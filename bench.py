@@ -428,9 +428,16 @@ def main():
     g.set_step_graph(not args.no_graph)
     stream = torch.cuda.current_stream()
 
+    prefill_ms = []
+
     def fresh():
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
         g.prefill(prompts)
+        p1.record(stream)
         g.poll_status()
+        torch.cuda.synchronize()
+        prefill_ms.append(p0.elapsed_time(p1))
 
     # ---- device-resident timed runs: `blocks` identical blocks (prompt pass, W warm-up steps, then K whole steps back
     # to back between two events); the median block is the reported one
@@ -599,6 +606,7 @@ def main():
         "emitted_tokens_per_s": world * (acc + 1) * B / (ms_step * 1e-3), "mean_accepted": acc,
         "planned_mean_accepted": sum(sum(r) for r in planned[args.warmup:]) / (args.steps * B),
         "final_lens": lens_end,
+        "prefill_ms": sorted(prefill_ms)[len(prefill_ms) // 2], "prefill_tokens": int(sum(cfg.prompt_lens)),
         "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel (weight-streaming bf16 GEMM, all shapes of a step)",
                      "achieved": gemm_gbs, "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": gemm_gbs / hbm_peak, "frac_of_8TBs": gemm_gbs / NOMINAL_HBM_GBS, "traffic": traffic,

@@ -111,7 +111,8 @@ hydra_status hydra_destroy(hydra_ctx*);
  * attention) filling the KV caches, and, with prefix_attn, the extra layer's cache (Section "Hydra++",
  * "Prefix Attention"); leaves, per sequence, the committed length, the root token (argmax after the last
  * prompt token) and the last hidden state.  tokens_dev holds the prompts back to back; seq_offsets_host
- * has batch+1 entries (read before the call returns).  Synchronises the stream once (see Conventions).
+ * has batch+1 entries (read before the call returns).  The prompts are processed in passes of 128 rows per sequence
+ * (dtype 1) or 64 (dtype 0), every pass streaming the weights once.  Synchronises the stream once (see Conventions).
  * Errors: INVALID (null pointer, batch outside 1..max_batch, empty prompt), CAPACITY (prompt + tree rows
  * exceed max_seq). */
 hydra_status hydra_prefill(hydra_ctx*, int batch, const int32_t* tokens_dev, const int32_t* seq_offsets_host,
@@ -228,8 +229,8 @@ const char* hydra_last_error(void); /* text of the last CUDA error seen by this 
  *   dtype 0: q, caches and out [rows][n_heads*head_dim] are float, tc <= 64, scratch_dev needs
  *   hydra_attention_scratch_bytes(...) bytes, planes = out_planes = 1, status_dev unused.  dtype 1: q and the caches are
  *   float16 in `planes` planes (2: hi = f16(v), lo = f16(v - hi)), out is bfloat16 [out_planes][rows][n_heads*head_dim]
- *   (2: hi = bf16(v) and lo = bf16(v - hi)); tc <= 64 with a mask, <= 128 causal (one plane or head_dim 64 only, else
- *   UNSUPPORTED); scratch_dev unused (may be NULL); status_dev is an int32 status word (bit 2: a bounded wait ran out). */
+ *   (2: hi = bf16(v) and lo = bf16(v - hi)); tc <= 64 with a mask, <= 128 causal (two planes at head_dim 128: computed as launches of 64 rows each, the rows of
+ *   an earlier launch being cache rows to a later one, so the K and V rows of the whole chunk must be in the caches); scratch_dev unused (may be NULL); status_dev is an int32 status word (bit 2: a bounded wait ran out). */
 size_t hydra_gemm_partial_floats(int m, int n, int k, int dtype, int mode);
 hydra_status hydra_gemm(const void* x_dev, const void* w_dev, float* out_dev, float* partial_dev, int m, int n, int k,
                         int dtype, int mode, int x_planes, int32_t* status_dev, void* stream);

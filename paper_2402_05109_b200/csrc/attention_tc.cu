@@ -83,6 +83,8 @@ struct AttArgs {
   int H, max_seq, nchunks;
   int* status;
   uint32_t wait_limit;
+  int row_off;                         // first row (of each sequence's rs.tc row slots) this launch computes: a wide causal chunk
+                                       // runs as several launches of QROWS rows, each seeing the earlier ones as cache rows
   int early;                           // the lengths (rs.pos0, rs.n_rows) and the committed cache rows were written by kernels that
                                        // completed before the preceding kernel started (see tree_attention_tc)
 };
@@ -179,8 +181,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   uint32_t tmem_base;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 
-  const int nr = min(rs.n_rows ? rs.n_rows[b] : rs.tc, QROWS);
-  const int p0 = rs.pos0[b];
+  const int nr = min(max((rs.n_rows ? rs.n_rows[b] : rs.tc) - a.row_off, 0), QROWS);
+  const int p_call = rs.pos0[b];                         // first cache slot written by this forward call
+  const int p0 = p_call + a.row_off;                     // first slot of this launch's rows
   const int total = p0 + nr;
   const int nt = (total + TILE - 1) / TILE;
   const int tile0 = chunk_first_tile(c, nt, nchunks), tile1 = chunk_first_tile(c + 1, nt, nchunks);
@@ -219,7 +222,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       };
       int nk = 0, nv = 0;                                  // next K and V tile to request
       if (a.early) {                                       // committed rows only
-        for (; nk < ntiles && nk < NSK && (tile0 + nk + 1) * TILE <= p0; ++nk) {
+        for (; nk < ntiles && nk < NSK && (tile0 + nk + 1) * TILE <= p_call; ++nk) {
           request_k(nk);
           if (nv == nk && nv < NSV) request_v(nv++);
         }
@@ -230,7 +233,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       for (int pl = 0; pl < NP; ++pl)
 #pragma unroll
         for (int hf = 0; hf < C::NHALF; ++hf)
-          tma_load_2d(q_s + pl * C::QP_BYTES + hf * QROWS * 128, &tmQ, h * HD + hf * 64, pl * a.q_plane_rows + b * rs.tc, q_full, pol_q);
+          tma_load_2d(q_s + pl * C::QP_BYTES + hf * QROWS * 128, &tmQ, h * HD + hf * 64, pl * a.q_plane_rows + b * rs.tc + a.row_off, q_full, pol_q);
       // K stage i % NSK was last read by the scores of tile i - NSK (completion i / NSK - 1 of its empty barrier), V stage
       // i % NSV by the P V product of tile i - NSV; whichever ring has room is served first, K ahead of V
       uint32_t idle = 0;
@@ -499,7 +502,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     constexpr int V4 = HD / 4;
     const uint32_t xo_s = ring_s, xml_s = ring_s + QROWS * HD * 4;
     const int d = H * HD;
-    const int rows_cap = min(rs.tc, QROWS);
+    const int rows_cap = min(rs.tc - a.row_off, QROWS);
     const int my_rows = rows_cap > c ? (rows_cap - c + nchunks - 1) / nchunks : 0;
     // chunk weights of my rows, normalised: w_c = 2^(m_c - M) / sum_c l_c 2^(m_c - M)  (one thread per row, all (m, l) loads in flight together)
     for (int t = tid; t < my_rows; t += C::NTHREADS) {
@@ -546,7 +549,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int cc = 0; cc < MAX_CHUNKS; ++cc) {
           acc.x += v[ib][cc].x * w[ib][cc]; acc.y += v[ib][cc].y * w[ib][cc]; acc.z += v[ib][cc].z * w[ib][cc]; acc.w += v[ib][cc].w * w[ib][cc];
         }
-        bf16* dst = a.out + ((size_t)b * rs.tc + i) * d + h * HD + k4 * 4;      // rows past nr get zeros
+        bf16* dst = a.out + ((size_t)b * rs.tc + a.row_off + i) * d + h * HD + k4 * 4;      // rows past nr get zeros
         const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x, acc.y), h1 = __floats2bfloat162_rn(acc.z, acc.w);
         *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
         if (a.out_ps) {
@@ -583,7 +586,7 @@ int pick_chunks(int pairs, int len_upper, int sms) {
 
 template <int HD, int QROWS, int NP>
 hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out, size_t out_ps,
-                 int H, int max_seq, int len_upper, int* status, bool stable_lengths, cudaStream_t st) {
+                 int H, int max_seq, int len_upper, int* status, bool stable_lengths, int row_off, cudaStream_t st) {
   using C = AttCfg<HD, QROWS, NP>;
   CUtensorMap tq, tk, tv;
   const uint64_t cache_rows = (uint64_t)cache_batch * H * max_seq;
@@ -600,7 +603,7 @@ hydra_status run(const __half* q, int q_rows, const __half* kc, const __half* vc
   }
   AttArgs a{};
   a.rs = rs; a.out = out; a.out_ps = out_ps; a.H = H; a.max_seq = max_seq; a.status = status; a.wait_limit = WAIT_LIMIT;
-  a.q_plane_rows = q_rows; a.kv_plane_rows = (int)cache_rows; a.early = stable_lengths ? 1 : 0;
+  a.q_plane_rows = q_rows; a.kv_plane_rows = (int)cache_rows; a.early = stable_lengths ? 1 : 0; a.row_off = row_off;
   a.nchunks = pick_chunks(H * rs.batch, len_upper, sm_count());
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(H, rs.batch, a.nchunks); cfg.blockDim = dim3(C::NTHREADS); cfg.dynamicSmemBytes = C::SMEM_BYTES; cfg.stream = st;
@@ -619,11 +622,19 @@ template <int NP>
 hydra_status dispatch(const __half* q, int q_rows, const __half* kc, const __half* vc, int cache_batch, RowSet rs, bf16* out, size_t out_ps,
                       int H, int hd, int max_seq, int len_upper, int* status, bool stable_lengths, cudaStream_t st) {
   const bool wide = rs.tc > 64;
-  if (hd == 128 && wide && NP == 2) return HYDRA_ERR_UNSUPPORTED;       // Q, P and a two-stage ring of two planes exceed the shared memory of an SM
-  if (hd == 128) return wide ? run<128, 128, 1>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, st)
-                             : run<128, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, st);
-  if (hd == 64) return wide ? run<64, 128, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, st)
-                            : run<64, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, st);
+  if (hd == 128 && wide && NP == 2) {
+    // Q, P and the rings of two planes for 128 query rows exceed the shared memory of an SM: 64 rows per launch; the rows of
+    // an earlier launch are cache rows to a later one (the preceding kernel has appended the K and V rows of the whole chunk)
+    for (int off = 0; off < rs.tc; off += 64) {
+      hydra_status r = run<128, 64, 2>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, off, st);
+      if (r != HYDRA_OK) return r;
+    }
+    return HYDRA_OK;
+  }
+  if (hd == 128) return wide ? run<128, 128, 1>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, 0, st)
+                             : run<128, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, 0, st);
+  if (hd == 64) return wide ? run<64, 128, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, 0, st)
+                            : run<64, 64, NP>(q, q_rows, kc, vc, cache_batch, rs, out, out_ps, H, max_seq, len_upper, status, stable_lengths, 0, st);
   return HYDRA_ERR_UNSUPPORTED;
 }
 

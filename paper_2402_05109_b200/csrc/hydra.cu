@@ -20,7 +20,10 @@ void set_last_error(const char* what, cudaError_t e) {
 
 namespace {
 
-constexpr int CHUNK = 64;          // rows per sequence of one prefill pass (and the row capacity of a forward call)
+constexpr int CHUNK = 64;          // rows per sequence that a masked forward call can hold (64-bit ancestor masks)
+// Rows per sequence of one prefill pass: 128 causal rows on the bfloat16 path (half as many passes over the weights; the
+// attention kernel takes them as a causal chunk), 64 chain-masked rows on the float path.
+inline int prefill_chunk(const hydra_model_cfg& m) { return m.dtype == 1 ? 2 * CHUNK : CHUNK; }
 
 struct LayerW { const void *attn_norm, *wqkv, *wo, *ffn_norm, *w_gate_up, *w_down; };
 
@@ -164,7 +167,8 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
   const int ces = m.dtype == 0 ? 4 : 2;         // q and the KV caches: float, or float16 in kvp planes
   const int kvp = m.dtype == 0 ? 1 : (m.kv_planes == 1 ? 1 : 2);
   const int d = m.d_model, f = m.d_ffn, V = m.vocab, K = h.n_heads, T = t.T;
-  const int R = pad_rows(m.max_batch * CHUNK);
+  const int PC = prefill_chunk(m);
+  const int R = pad_rows(m.max_batch * PC);
   const int RH = pad_rows(m.max_batch * t.maxP);
   // largest partial-sum buffer over every GEMM shape and row count the library issues
   size_t part_floats = 0;
@@ -175,7 +179,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
       part_floats = std::max(part_floats, (size_t)slots * mm * n);
     };
     const int shapes[][2] = {{3 * d, d}, {d, d}, {2 * f, d}, {d, f}, {V, d}};
-    const int per_seq[] = {CHUNK, T, K + 1, 1};
+    const int per_seq[] = {PC, T, K + 1, 1};
     for (auto& sh : shapes)
       for (int rows : per_seq)
         for (int bb = 1; bb <= m.max_batch; ++bb) need(rows * bb, sh[0], sh[1]);
@@ -186,7 +190,7 @@ size_t carve(hydra_ctx* c, const hydra_model_cfg& m, const hydra_head_cfg& h, co
     }
   }
   auto* parent = b.take<int>(T); auto* depth = b.take<int>(T); auto* fc = b.take<int>(T); auto* nc = b.take<int>(T);
-  auto* path_tab = b.take<int>((size_t)T * (K + 1)); auto* chain_depth = b.take<int>(CHUNK);
+  auto* path_tab = b.take<int>((size_t)T * (K + 1)); auto* chain_depth = b.take<int>(PC);
   auto* anc = b.take<uint64_t>(T); auto* chain_mask = b.take<uint64_t>(CHUNK);
   std::vector<int*> lvl;
   for (auto& lv : t.level_parents) lvl.push_back(b.take<int>(lv.size()));
@@ -494,13 +498,15 @@ hydra_status hydra_create(hydra_ctx** out, const hydra_model_cfg* m, const hydra
   if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "cudaDeviceSynchronize");
   if ((e = cudaMemset(ws, 0, need)) != cudaSuccess) return fail(e, "cudaMemset(workspace)");
   const int T = th.T, K = h->n_heads;
-  std::vector<int> chain_depth(CHUNK); std::vector<uint64_t> chain_mask(CHUNK);
-  for (int i = 0; i < CHUNK; ++i) { chain_depth[i] = i; chain_mask[i] = i == 63 ? ~0ull : ((1ull << (i + 1)) - 1); }
+  const int PC = prefill_chunk(c->m);
+  std::vector<int> chain_depth(PC); std::vector<uint64_t> chain_mask(CHUNK);
+  for (int i = 0; i < PC; ++i) chain_depth[i] = i;
+  for (int i = 0; i < CHUNK; ++i) chain_mask[i] = i == 63 ? ~0ull : ((1ull << (i + 1)) - 1);
 #define UP(dst, src, bytes) if ((bytes) && (e = cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice)) != cudaSuccess) return fail(e, "cudaMemcpy(tables)")
   UP(c->d_parent, th.parent.data(), T * sizeof(int)); UP(c->d_depth, th.depth.data(), T * sizeof(int));
   UP(c->d_first_child, th.first_child.data(), T * sizeof(int)); UP(c->d_n_child, th.n_child.data(), T * sizeof(int));
   UP(c->d_path_tab, th.path_tab.data(), (size_t)T * (K + 1) * sizeof(int));
-  UP(c->d_chain_depth, chain_depth.data(), CHUNK * sizeof(int)); UP(c->d_chain_mask, chain_mask.data(), CHUNK * sizeof(uint64_t));
+  UP(c->d_chain_depth, chain_depth.data(), PC * sizeof(int)); UP(c->d_chain_mask, chain_mask.data(), CHUNK * sizeof(uint64_t));
   UP(c->d_anc, th.anc.data(), T * sizeof(uint64_t));
   for (size_t i = 0; i < th.level_parents.size(); ++i) UP(c->d_level_parents[i], th.level_parents[i].data(), th.level_parents[i].size() * sizeof(int));
 #undef UP
@@ -537,14 +543,16 @@ hydra_status hydra_prefill(hydra_ctx* c, int batch, const int32_t* tokens, const
   HYDRA_CUDA(cudaMemcpyAsync(c->d_prompt_len, plen.data(), batch * sizeof(int), cudaMemcpyHostToDevice, st));
   HYDRA_CUDA(cudaMemcpyAsync(c->d_offsets, offs, (batch + 1) * sizeof(int), cudaMemcpyHostToDevice, st));
   HYDRA_CUDA(cudaStreamSynchronize(st));           // the host vectors above go out of scope
-  const int nchunks = (maxlen + CHUNK - 1) / CHUNK;
-  RowSet rs{batch, CHUNK, c->d_nrows, c->d_pos0, c->d_chain_depth, c->d_chain_mask};
+  const int PC = prefill_chunk(m);
+  const int nchunks = (maxlen + PC - 1) / PC;
+  // a chunk is a chain: row i sees the rows before it (an explicit mask for 64 rows, the causal rule of the attention kernel for 128)
+  RowSet rs{batch, PC, c->d_nrows, c->d_pos0, c->d_chain_depth, PC > CHUNK ? nullptr : c->d_chain_mask};
   for (int ch = 0; ch < nchunks; ++ch) {
-    HYDRA_TRY(set_chunk(c->d_prompt_len, ch, CHUNK, c->d_pos0, c->d_nrows, batch, st));
-    HYDRA_TRY(gather_chunk_tokens(tokens, c->d_offsets, ch, CHUNK, c->d_tok, batch, st));
-    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * CHUNK, nullptr, 0, nullptr, true, st));
-    HYDRA_TRY(capture_last(c->h_tree, c->d_prompt_len, ch, CHUNK, c->h_new, c->h.n_heads + 1, c->d_n_new, c->d_len, batch, m.d_model, st));
-    if (c->h.prefix_attn) HYDRA_TRY(run_prefix(c, c->h_tree, rs, (ch + 1) * CHUNK, st));
+    HYDRA_TRY(set_chunk(c->d_prompt_len, ch, PC, c->d_pos0, c->d_nrows, batch, st));
+    HYDRA_TRY(gather_chunk_tokens(tokens, c->d_offsets, ch, PC, c->d_tok, batch, st));
+    HYDRA_TRY(run_base(c, c->d_tok, rs, (ch + 1) * PC, nullptr, 0, nullptr, true, st));
+    HYDRA_TRY(capture_last(c->h_tree, c->d_prompt_len, ch, PC, c->h_new, c->h.n_heads + 1, c->d_n_new, c->d_len, batch, m.d_model, st));
+    if (c->h.prefix_attn) HYDRA_TRY(run_prefix(c, c->h_tree, rs, (ch + 1) * PC, st));
   }
   // root token = argmax of the logits of the last prompt row
   HYDRA_TRY(pick_last_row(c->h_new, c->d_n_new, c->h.n_heads + 1, c->hprime, batch, m.d_model, st));

@@ -966,7 +966,7 @@ __global__ void gather_chunk_tokens_kernel(const int* tokens, const int* offsets
 }
 hydra_status gather_chunk_tokens(const int* tokens, const int* offsets, int chunk, int tc, int* tok_out, int batch,
                                  cudaStream_t st) {
-  launch_pdl(gather_chunk_tokens_kernel, dim3(batch), dim3(64), 0, st, tokens, offsets, chunk, tc, tok_out);
+  launch_pdl(gather_chunk_tokens_kernel, dim3(batch), dim3((tc + 31) / 32 * 32), 0, st, tokens, offsets, chunk, tc, tok_out);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
 }

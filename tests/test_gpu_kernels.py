@@ -140,7 +140,7 @@ def test_tree_attention_rescales_when_the_maximum_climbs(hd, planes):
     assert float((out[0].double() - ref).abs().max()) <= (1.5e-3 if planes == 1 else 1e-4)
 
 
-@pytest.mark.parametrize("hd,tc,planes", [(128, 128, 1), (64, 100, 1), (64, 128, 2), (128, 64, 2), (128, 40, 1)])
+@pytest.mark.parametrize("hd,tc,planes", [(128, 128, 1), (64, 100, 1), (64, 128, 2), (128, 64, 2), (128, 40, 1), (128, 128, 2), (128, 90, 2)])
 def test_causal_chunk_attention(hd, tc, planes):
     """mask = NULL: a causal chunk of up to 128 rows on top of the committed slots (the prompt pass)."""
     from paper_2402_05109_b200 import tree_attention
