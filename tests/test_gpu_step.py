@@ -45,6 +45,17 @@ def test_small_bf16_hydrapp_ragged_batch():
     assert seen >= {0, 1, 2, 3, 4}, seen
 
 
+@pytest.mark.parametrize("head_dim,kv_planes", [(128, 2), (128, 1), (64, 2)])
+def test_prompt_lengths_around_the_prefill_chunk(head_dim, kv_planes):
+    """Prompts that end just before, on and just after the 64- and 128-row boundaries of the prompt pass (the bfloat16 path
+    walks 128-row causal chunks: two 64-row attention launches at head_dim 128 with two planes, one 128-row launch otherwise):
+    the lock-step protocol compares the caches of both layers, the last hidden state and the first steps with the oracle."""
+    m = ModelCfg(2, 256, 256 // head_dim, head_dim, 512, 1024, dtype="bf16", kv_planes=kv_planes)
+    h = HeadCfg(3, 2, True)
+    st, _ = run(m, h, load_tree("tree15_d3"), [127, 128, 129, 64, 65, 191, 256, 1], 2, 31, 320, kv_layers=(0, 1))
+    assert st.steps == 2
+
+
 @pytest.mark.parametrize("dtype,mlp,prefix", [("bf16", 1, False), ("bf16", 3, True), ("fp32", 2, False)])
 def test_medusa_mode_heads(dtype, mlp, prefix):
     """Sequentially independent heads (the Medusa baseline): head i sees the hidden state alone, one logits row per
