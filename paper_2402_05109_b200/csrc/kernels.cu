@@ -533,31 +533,14 @@ hydra_status silu_mul(const float* part, SplitDesc sd, void* act, size_t act_ps,
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
 
-__device__ __forceinline__ void block_best(float& v, int& i, float* shv, int* shi) {
+// The best (value, index) of a warp, in every lane.
+__device__ __forceinline__ void warp_best(float& v, int& i) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     float ov = __shfl_xor_sync(0xffffffffu, v, o);
     int oi = __shfl_xor_sync(0xffffffffu, i, o);
     if (better(ov, oi, v, i)) { v = ov; i = oi; }
   }
-  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  __syncthreads();
-  if (lane == 0) { shv[warp] = v; shi[warp] = i; }
-  __syncthreads();
-  if (warp == 0) {
-    int nw = blockDim.x >> 5;
-    v = lane < nw ? shv[lane] : -INFINITY;
-    i = lane < nw ? shi[lane] : 0x7fffffff;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, v, o);
-      int oi = __shfl_xor_sync(0xffffffffu, i, o);
-      if (better(ov, oi, v, i)) { v = ov; i = oi; }
-    }
-    if (lane == 0) { shv[0] = v; shi[0] = i; }
-  }
-  __syncthreads();
-  v = shv[0]; i = shi[0];
 }
 
 __device__ __forceinline__ float summed(const float* part, const SplitDesc& sd, int row, int col, int n) {
@@ -565,20 +548,23 @@ __device__ __forceinline__ float summed(const float* part, const SplitDesc& sd, 
 }
 
 // Top-c of every logits row in two stages.  Stage 1: grid (rows, blocks of TOPK_SPAN columns); each block sums the
-// partial slots of its columns (optionally storing the sums as the row's logits), then picks its c best in c
-// rounds of a block-wide reduction over register-resident values.  Stage 2: one block per row merges the
-// candidates of all column blocks the same way and writes the winners (children of a tree node, or the argmax).
+// partial slots of its columns (optionally storing the sums as the row's logits); every warp then picks the c best of
+// its register-resident values in c rounds of a warp-wide reduction (no block barrier inside the rounds), and one warp
+// merges the eight sorted lists.  Stage 2: one warp per winner list merges the sorted candidate lists of all column
+// blocks out of shared memory and writes the winners (children of a tree node, or the argmax).
 constexpr int TOPK_SPAN = 2048;           // columns per stage-1 block (8 per thread)
 constexpr int TOPK_MAX = 64;              // a tree node has at most 63 children
+constexpr int TOPK_LISTS_PER_LANE = 4;    // stage 2: at most 128 column blocks (262144 tokens)
 
 __global__ void __launch_bounds__(256) topk_stage1_kernel(const float* __restrict__ part, SplitDesc sd,
                                                           float* __restrict__ logits_out, float* __restrict__ cand_v,
                                                           int* __restrict__ cand_i, int vocab, int c) {
   pdl_trigger();
   pdl_wait();
-  __shared__ float shv[32];
-  __shared__ int shi[32];
+  __shared__ float wv[8][TOPK_MAX];
+  __shared__ int wi[8][TOPK_MAX];
   const int row = blockIdx.x, blk = blockIdx.y, nblk = gridDim.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   float v[8]; int idx[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
@@ -592,29 +578,43 @@ __global__ void __launch_bounds__(256) topk_stage1_kernel(const float* __restric
       idx[j] = 0x7fffffff;
     }
   }
-  for (int t = 0; t < c; ++t) {
+  for (int t = 0; t < c; ++t) {                            // this warp's c best, in order
     float bv = -INFINITY; int bi = 0x7fffffff;
 #pragma unroll
     for (int j = 0; j < 8; ++j) if (better(v[j], idx[j], bv, bi)) { bv = v[j]; bi = idx[j]; }
-    block_best(bv, bi, shv, shi);
-    if (threadIdx.x == 0) {
-      cand_v[((size_t)row * nblk + blk) * TOPK_MAX + t] = bv;
-      cand_i[((size_t)row * nblk + blk) * TOPK_MAX + t] = bi;
-    }
+    warp_best(bv, bi);
+    if (lane == 0) { wv[warp][t] = bv; wi[warp][t] = bi; }
 #pragma unroll
     for (int j = 0; j < 8; ++j) if (idx[j] == bi) { v[j] = -INFINITY; idx[j] = 0x7fffffff; }    // taken
+  }
+  __syncthreads();
+  if (warp == 0) {                                         // merge: lane w < 8 walks warp w's list
+    int ptr = 0;
+    for (int t = 0; t < c; ++t) {
+      float hv = -INFINITY; int hi = 0x7fffffff;
+      if (lane < 8 && ptr < c) { hv = wv[lane][ptr]; hi = wi[lane][ptr]; }
+      float bv = hv; int bi = hi;
+      warp_best(bv, bi);
+      if (lane == 0) {
+        cand_v[((size_t)row * nblk + blk) * TOPK_MAX + t] = bv;
+        cand_i[((size_t)row * nblk + blk) * TOPK_MAX + t] = bi;
+      }
+      if (hi == bi && bi != 0x7fffffff) ++ptr;
+    }
   }
 }
 
 // out_of(row) and count_of(row): where the winners go.  lv.parents == null: argmax (one winner per row to amax[row]).
-__global__ void __launch_bounds__(256) topk_stage2_kernel(const float* __restrict__ cand_v, const int* __restrict__ cand_i,
-                                                          int nblk, int c, LevelDesc lv, const int* __restrict__ first_child,
-                                                          const int* __restrict__ n_child, int* __restrict__ out, int T, int cand_div) {
+// One warp per winner list; dynamic shared memory: nblk * c (value, index) pairs.
+__global__ void __launch_bounds__(32) topk_stage2_kernel(const float* __restrict__ cand_v, const int* __restrict__ cand_i,
+                                                         int nblk, int c, LevelDesc lv, const int* __restrict__ first_child,
+                                                         const int* __restrict__ n_child, int* __restrict__ out, int T, int cand_div) {
   pdl_trigger();
   pdl_wait();
-  __shared__ float shv[32];
-  __shared__ int shi[32];
-  const int row = blockIdx.x;
+  extern __shared__ float s_cand[];
+  float* sv = s_cand;
+  int* si = reinterpret_cast<int*>(s_cand + nblk * c);
+  const int row = blockIdx.x, lane = threadIdx.x;
   const int crow = row / cand_div;                         // row of the candidate lists (one per sequence when the parents share them)
   int* dst = out + row;
   int count = 1;
@@ -623,18 +623,28 @@ __global__ void __launch_bounds__(256) topk_stage2_kernel(const float* __restric
     dst = out + b * T + first_child[p];
     count = n_child[p];
   }
-  float pv = INFINITY; int pi = -1;
+  for (int e = lane; e < nblk * c; e += 32) {
+    const size_t at = ((size_t)crow * nblk + e / c) * TOPK_MAX + e % c;
+    sv[e] = cand_v[at]; si[e] = cand_i[at];
+  }
+  __syncwarp();
+  int ptr[TOPK_LISTS_PER_LANE];                            // lane l walks the sorted lists l, l + 32, ...
+#pragma unroll
+  for (int q = 0; q < TOPK_LISTS_PER_LANE; ++q) ptr[q] = 0;
   for (int t = 0; t < count; ++t) {
     float bv = -INFINITY; int bi = 0x7fffffff;
-    for (int e = threadIdx.x; e < nblk * c; e += blockDim.x) {
-      const size_t at = ((size_t)crow * nblk + e / c) * TOPK_MAX + e % c;
-      const float v = cand_v[at]; const int i = cand_i[at];
-      const bool after = v < pv || (v == pv && i > pi);          // strictly after the previous pick in the order
-      if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
+#pragma unroll
+    for (int q = 0; q < TOPK_LISTS_PER_LANE; ++q) {
+      const int l = lane + 32 * q;
+      if (l < nblk && ptr[q] < c && better(sv[l * c + ptr[q]], si[l * c + ptr[q]], bv, bi)) { bv = sv[l * c + ptr[q]]; bi = si[l * c + ptr[q]]; }
     }
-    block_best(bv, bi, shv, shi);
-    if (threadIdx.x == 0) dst[t] = bi;
-    pv = bv; pi = bi;
+    warp_best(bv, bi);
+    if (lane == 0) dst[t] = bi;
+#pragma unroll
+    for (int q = 0; q < TOPK_LISTS_PER_LANE; ++q) {
+      const int l = lane + 32 * q;
+      if (l < nblk && ptr[q] < c && si[l * c + ptr[q]] == bi && bi != 0x7fffffff) ++ptr[q];
+    }
   }
 }
 
@@ -648,11 +658,13 @@ static hydra_status topk_rows(const float* part, SplitDesc sd, float* logits_out
                               int c, LevelDesc lv, const int* first_child, const int* n_child, int* out, int T, cudaStream_t st) {
   if (c < 1 || c > TOPK_MAX || rows > rows_cap || rows < 1 || out_rows % rows) return HYDRA_ERR_UNSUPPORTED;
   const int nblk = (vocab + TOPK_SPAN - 1) / TOPK_SPAN;
+  const size_t merge_bytes = (size_t)nblk * c * 8;         // stage 2 keeps every candidate of a row in shared memory
+  if (nblk > 32 * TOPK_LISTS_PER_LANE || merge_bytes > 48 * 1024) return HYDRA_ERR_UNSUPPORTED;
   float* cand_v = (float*)scratch;
   int* cand_i = (int*)(cand_v + (size_t)rows_cap * nblk * TOPK_MAX);
   launch_pdl(topk_stage1_kernel, dim3(rows, nblk), dim3(256), 0, st, part, sd, logits_out, cand_v, cand_i, vocab, c);
   HYDRA_LAUNCH_CHECK();
-  launch_pdl(topk_stage2_kernel, dim3(out_rows), dim3(256), 0, st, (const float*)cand_v, (const int*)cand_i, nblk, c, lv, first_child, n_child, out, T,
+  launch_pdl(topk_stage2_kernel, dim3(out_rows), dim3(32), merge_bytes, st, (const float*)cand_v, (const int*)cand_i, nblk, c, lv, first_child, n_child, out, T,
              out_rows / rows);
   HYDRA_LAUNCH_CHECK();
   return HYDRA_OK;
@@ -684,8 +696,9 @@ __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restric
   const int blk = blockIdx.y;                               // 0: hidden, 1..d: path tokens root..parent
   const int p = lv.parents[j];
   T* dst = z + ((size_t)row * (lv.d + 1) + blk) * d_model;
-  if (blk == 0) {
-    for (int i = threadIdx.x; i < d_model; i += blockDim.x) put<T>(dst + i, z_ps, hprime[(size_t)b * d_model + i]);
+  if (blk == 0) {                                          // 16-byte pieces (d_model is a multiple of 4)
+    for (int i = threadIdx.x * 4; i < d_model; i += blockDim.x * 4)
+      put4<T>(dst + i, z_ps, *reinterpret_cast<const float4*>(hprime + (size_t)b * d_model + i));
     if (write_root && j == 0 && threadIdx.x == 0) tree_tok[b * T_rows] = root_tok[b];
     return;
   }
@@ -693,7 +706,7 @@ __global__ void __launch_bounds__(256) head_gather_kernel(const float* __restric
   int t = node == 0 ? root_tok[b] : tree_tok[b * T_rows + node];
   if (t < 0 || t >= vocab) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); t = 0; }
   const T* e = embed + (size_t)t * d_model;
-  for (int i = threadIdx.x; i < d_model; i += blockDim.x) put<T>(dst + i, z_ps, to_f<T>(e[i]));      // embeddings are exact: lo = 0
+  for (int i = threadIdx.x * 4; i < d_model; i += blockDim.x * 4) put4<T>(dst + i, z_ps, load4<T>(e + i));      // embeddings are exact: lo = 0
 }
 hydra_status head_gather(const float* hprime, const void* embed, const int* root_tok, int* tree_tok, const int* path_tab,
                          LevelDesc lv, int write_root, void* z, size_t z_ps, int batch, int T, int kp1, int d_model, int vocab, int dtype,
