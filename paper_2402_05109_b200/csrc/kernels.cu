@@ -80,6 +80,12 @@ hydra_status reduce_splits(const float* part, SplitDesc sd, float* out, int m, i
 // ------------------------------------------------------------------------------------------------
 // Embedding gather
 // ------------------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float4 load4(const T* p);
+template <> __device__ __forceinline__ float4 load4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
+template <> __device__ __forceinline__ float4 load4<bf16>(const bf16* p) {
+  float v[4]; Vec4<bf16>::load(p, v); return make_float4(v[0], v[1], v[2], v[3]);
+}
+
 template <typename T>
 __global__ void embed_rows_kernel(const T* __restrict__ embed, const int* __restrict__ tok, float* __restrict__ x, int d,
                                   int vocab, int* status) {
@@ -89,7 +95,7 @@ __global__ void embed_rows_kernel(const T* __restrict__ embed, const int* __rest
   int t = tok[r];
   if (t < 0 || t >= vocab) { if (threadIdx.x == 0) atomicOr(status, ST_BOUNDS); t = 0; }
   const T* e = embed + (size_t)t * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)r * d + i] = to_f<T>(e[i]);
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) *reinterpret_cast<float4*>(x + (size_t)r * d + i) = load4<T>(e + i);   // d % 4 == 0
 }
 hydra_status embed_rows(const void* embed, const int* tok, float* x, int rows, int d, int vocab, int dtype, int* status,
                         cudaStream_t st) {
@@ -135,11 +141,6 @@ template <> __device__ __forceinline__ void put4h<__half>(__half* p, size_t ps, 
                                __half2float(__float2half_rn(v.z)), __half2float(__float2half_rn(v.w)));
   store4<__half>(p, h);
   if (ps) store4<__half>(p + ps, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
-}
-template <typename T> __device__ __forceinline__ float4 load4(const T* p);
-template <> __device__ __forceinline__ float4 load4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
-template <> __device__ __forceinline__ float4 load4<bf16>(const bf16* p) {
-  float v[4]; Vec4<bf16>::load(p, v); return make_float4(v[0], v[1], v[2], v[3]);
 }
 
 // Operand storage.  float buffers hold one plane.  bfloat16 operand buffers hold two planes `ps` elements apart:
@@ -1022,7 +1023,8 @@ __global__ void pick_last_row_kernel(const float* x, const int* n_rows, int tc, 
   int b = blockIdx.x;
   int i = n_rows[b] - 1;
   if (i < 0) i = 0;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) hprime[(size_t)b * d + c] = x[((size_t)b * tc + i) * d + c];
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4)                                  // d % 4 == 0
+    *reinterpret_cast<float4*>(hprime + (size_t)b * d + c) = *reinterpret_cast<const float4*>(x + ((size_t)b * tc + i) * d + c);
 }
 hydra_status pick_last_row(const float* x, const int* n_rows, int tc, float* hprime, int batch, int d, cudaStream_t st) {
   launch_pdl(pick_last_row_kernel, dim3(batch), dim3(256), 0, st, x, n_rows, tc, hprime, d);
